@@ -1,0 +1,421 @@
+"""Plain fp64 statement of one minibatch-SGD training step in matrix form.
+
+TEST INFRASTRUCTURE: imported only by tests, the smoke check and the
+CPU-baseline leg of the benchmark.  Shares no code with the CUDA path.
+
+Notation follows the paper (Section 1): activations are matrices with one
+COLUMN per sample, X_i in R^{d_{i-1} x B}, Y_i in R^{d_i x B}, and
+W_i in R^{d_i x d_{i-1}}.  Convolution layers carry NCHW tensors
+[B, C, H, W] instead (Section 2.1/2.2).  Everything is numpy float64; the
+only library primitive used as a step is the dense matrix product `@`
+(and `einsum` for the channel contraction inside the convolution).
+
+    forward    Y_i = W_i X_i (+ b_i 1^T),  X_{i+1} = f(Y_i)      Section 1
+    backward   dX_i = W_i^T dY_i,  dW_i = dY_i X_i^T             Section 1, Appendix A.2
+    update     w <- w - eta (1/B) sum_{i in Batch} grad f_i      Eq. 1
+
+Readings taken where the paper is silent: f = ReLU with derivative 0 at 0,
+none after the last layer; gradients are SUMS over the batch and the 1/B of
+Eq. 1 is applied once, in the update; softmax cross-entropy with natural log
+(sum over samples) or half sum of squares as the loss; dX_1 is not formed
+(Section 2.2: nothing is back-propagated beyond the first layer);
+convolution is cross-correlation with zero padding.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------
+# layers
+# --------------------------------------------------------------------------
+@dataclass
+class FC:
+    """Fully connected layer: W is d_i x d_{i-1}, b is d_i or None."""
+    W: np.ndarray
+    b: Optional[np.ndarray] = None
+    relu: bool = True
+
+
+@dataclass
+class Conv3x3:
+    """3x3, stride 1, zero-pad 1 convolution: K is [C_out, C_in, 3, 3]."""
+    K: np.ndarray
+    relu: bool = True
+
+
+def balanced_ranges(n: int, P: int):
+    """Index ranges [floor(p n / P), floor((p+1) n / P)) for p = 0..P-1."""
+    return [((p * n) // P, ((p + 1) * n) // P) for p in range(P)]
+
+
+# --------------------------------------------------------------------------
+# single operations (un-blocked definitions)
+# --------------------------------------------------------------------------
+def affine(W, X, b=None):
+    """Y = W X (+ b 1^T)   -- Section 1."""
+    Y = np.asarray(W, F64) @ np.asarray(X, F64)
+    if b is not None:
+        Y = Y + np.asarray(b, F64)[:, None]
+    return Y
+
+
+def relu(Y):
+    return np.maximum(Y, 0.0)
+
+
+def fc_dX(W, dY):
+    """dX = W^T dY   -- Section 1, Appendix A.2."""
+    return np.asarray(W, F64).T @ np.asarray(dY, F64)
+
+
+def fc_dW(dY, X):
+    """dW = dY X^T = sum_b dY[:, b] X[:, b]^T   -- Appendix A.2."""
+    return np.asarray(dY, F64) @ np.asarray(X, F64).T
+
+
+def conv3x3(K, X):
+    """Y[b,o,h,w] = sum_{c,u,v} K[o,c,u,v] X[b,c,h+u-1,w+v-1], zero outside."""
+    K = np.asarray(K, F64)
+    X = np.asarray(X, F64)
+    B, C, H, W = X.shape
+    Xp = np.zeros((B, C, H + 2, W + 2), F64)
+    Xp[:, :, 1:H + 1, 1:W + 1] = X
+    Y = np.zeros((B, K.shape[0], H, W), F64)
+    for u in range(3):
+        for v in range(3):
+            Y += np.einsum("oc,bchw->bohw", K[:, :, u, v], Xp[:, :, u:u + H, v:v + W])
+    return Y
+
+
+def conv3x3_dX(K, dY):
+    """dX[b,c,h,w] = sum_{o,u,v} K[o,c,u,v] dY[b,o,h-u+1,w-v+1], zero outside."""
+    K = np.asarray(K, F64)
+    dY = np.asarray(dY, F64)
+    B, O, H, W = dY.shape
+    dYp = np.zeros((B, O, H + 2, W + 2), F64)
+    dYp[:, :, 1:H + 1, 1:W + 1] = dY
+    dX = np.zeros((B, K.shape[1], H, W), F64)
+    for u in range(3):
+        for v in range(3):
+            # index h-u+1 in dY  ==  (h-u+2) in the padded array
+            dX += np.einsum("oc,bohw->bchw", K[:, :, u, v],
+                            dYp[:, :, 2 - u:2 - u + H, 2 - v:2 - v + W])
+    return dX
+
+
+def conv3x3_dK(dY, X):
+    """dK[o,c,u,v] = sum_{b,h,w} dY[b,o,h,w] X[b,c,h+u-1,w+v-1]."""
+    dY = np.asarray(dY, F64)
+    X = np.asarray(X, F64)
+    B, C, H, W = X.shape
+    Xp = np.zeros((B, C, H + 2, W + 2), F64)
+    Xp[:, :, 1:H + 1, 1:W + 1] = X
+    dK = np.zeros((dY.shape[1], C, 3, 3), F64)
+    for u in range(3):
+        for v in range(3):
+            dK[:, :, u, v] = np.einsum("bohw,bchw->oc", dY, Xp[:, :, u:u + H, v:v + W])
+    return dK
+
+
+def softmax_ce(Y_L, labels):
+    """J = sum_b [logsumexp_k Y[k,b] - Y[y_b,b]];  dY[:,b] = softmax(Y[:,b]) - e_{y_b}.
+
+    Y_L is d_L x B (one column per sample).  Returns (J, per-sample loss, dY).
+    """
+    Y = np.asarray(Y_L, F64)
+    labels = np.asarray(labels).astype(np.int64)
+    d, B = Y.shape
+    m = Y.max(axis=0)
+    E = np.exp(Y - m[None, :])
+    Z = E.sum(axis=0)
+    lse = m + np.log(Z)
+    cols = np.arange(B)
+    per = lse - Y[labels, cols]
+    dY = E / Z[None, :]
+    dY[labels, cols] -= 1.0
+    return float(per.sum()), per, dY
+
+
+def half_ssq(Y_L):
+    """J = 1/2 sum Y^2,  dY = Y."""
+    Y = np.asarray(Y_L, F64)
+    return float(0.5 * np.sum(Y * Y)), Y.copy()
+
+
+def sgd(w, dw, eta, B):
+    """Eq. 1 with dw = sum over the batch of per-sample gradients."""
+    return np.asarray(w, F64) - (eta / B) * np.asarray(dw, F64)
+
+
+# --------------------------------------------------------------------------
+# one training step, un-blocked
+# --------------------------------------------------------------------------
+def _batch_of(X):
+    return X.shape[1] if X.ndim == 2 else X.shape[0]
+
+
+def forward(layers: Sequence, X1):
+    """Returns (Xs, Ys): Xs[i] is the input of layer i (0-based), Ys[i] its
+    affine output before the nonlinearity."""
+    Xs: List[np.ndarray] = [np.asarray(X1, F64)]
+    Ys: List[np.ndarray] = []
+    for i, lay in enumerate(layers):
+        if isinstance(lay, FC):
+            Y = affine(lay.W, Xs[i], lay.b)
+        else:
+            Y = conv3x3(lay.K, Xs[i])
+        Ys.append(Y)
+        if i + 1 < len(layers):
+            Xs.append(relu(Y) if lay.relu else Y)
+    return Xs, Ys
+
+
+def loss_and_top_grad(Y_L, loss: str, labels=None):
+    if loss == "softmax_ce":
+        J, per, dY = softmax_ce(Y_L, labels)
+        return J, per, dY
+    if loss == "half_ssq":
+        J, dY = half_ssq(Y_L)
+        return J, None, dY
+    raise ValueError(loss)
+
+
+def train_step(layers: Sequence, X1, labels, loss: str, eta: float):
+    """One full step.  Returns a dict with
+       Xs, Ys, J, per_sample, dYs (dJ/dY_i), dXs (dJ/dX_i, None for i=0),
+       dWs, dbs, new_W, new_b   (lists indexed by layer, 0-based)."""
+    L = len(layers)
+    Xs, Ys = forward(layers, X1)
+    B = _batch_of(Xs[0])
+    J, per, dY_top = loss_and_top_grad(Ys[-1], loss, labels)
+    dYs = [None] * L
+    dXs = [None] * L
+    dWs = [None] * L
+    dbs = [None] * L
+    dYs[L - 1] = dY_top
+    for i in range(L - 1, -1, -1):
+        lay = layers[i]
+        if isinstance(lay, FC):
+            dWs[i] = fc_dW(dYs[i], Xs[i])
+            dbs[i] = dYs[i].sum(axis=1) if lay.b is not None else None
+        else:
+            dWs[i] = conv3x3_dK(dYs[i], Xs[i])
+        if i > 0:
+            dXs[i] = fc_dX(lay.W, dYs[i]) if isinstance(lay, FC) else conv3x3_dX(lay.K, dYs[i])
+            prev = layers[i - 1]
+            dYs[i - 1] = dXs[i] * (Ys[i - 1] > 0.0) if prev.relu else dXs[i]
+    new_W, new_b = [], []
+    for i, lay in enumerate(layers):
+        w = lay.W if isinstance(lay, FC) else lay.K
+        new_W.append(sgd(w, dWs[i], eta, B))
+        if isinstance(lay, FC) and lay.b is not None:
+            new_b.append(sgd(lay.b, dbs[i], eta, B))
+        else:
+            new_b.append(None)
+    return dict(Xs=Xs, Ys=Ys, J=J, per_sample=per, dYs=dYs, dXs=dXs, dWs=dWs,
+                dbs=dbs, new_W=new_W, new_b=new_b)
+
+
+# --------------------------------------------------------------------------
+# the same step over a logical P_r x P_c grid (Section 2.3; Appendix A.1/A.2)
+# --------------------------------------------------------------------------
+def fc_forward_blocked(W, X, b, P_r, P_c):
+    """Block (r,c) forms Y(r,c) = W(r,:) X(:,c); the all-gather over P_r only
+    concatenates the row blocks (Appendix A.1)."""
+    W = np.asarray(W, F64)
+    X = np.asarray(X, F64)
+    d, B = W.shape[0], X.shape[1]
+    Y = np.empty((d, B), F64)
+    for (r0, r1) in balanced_ranges(d, P_r):
+        for (c0, c1) in balanced_ranges(B, P_c):
+            blk = W[r0:r1, :] @ X[:, c0:c1]
+            if b is not None:
+                blk = blk + np.asarray(b, F64)[r0:r1, None]
+            Y[r0:r1, c0:c1] = blk
+    return Y
+
+
+def fc_dX_blocked(W, dY, P_r, P_c):
+    """Process row r holds W(r,:) and forms the partial W(r,:)^T dY(r,c); the
+    all-reduce over the P_r group adds the partials (Appendix A.2).  Added in
+    ascending r.  Returns (dX, partials[r])."""
+    W = np.asarray(W, F64)
+    dY = np.asarray(dY, F64)
+    d_out, d_in = W.shape
+    B = dY.shape[1]
+    parts = []
+    for (r0, r1) in balanced_ranges(d_out, P_r):
+        part = np.zeros((d_in, B), F64)
+        for (c0, c1) in balanced_ranges(B, P_c):
+            part[:, c0:c1] = W[r0:r1, :].T @ dY[r0:r1, c0:c1]
+        parts.append(part)
+    dX = np.zeros((d_in, B), F64)
+    for part in parts:
+        dX = dX + part
+    return dX, parts
+
+
+def fc_dW_blocked(dY, X, P_r, P_c):
+    """Process column c holds B/P_c samples and forms the partial
+    sum_{b in c} dY_b X_b^T; the all-reduce over the P_c group adds them
+    (Appendix A.2).  Added in ascending c.  Returns (dW, partials[c])."""
+    dY = np.asarray(dY, F64)
+    X = np.asarray(X, F64)
+    d_out, B = dY.shape
+    d_in = X.shape[0]
+    parts = []
+    for (c0, c1) in balanced_ranges(B, P_c):
+        part = np.zeros((d_out, d_in), F64)
+        for (r0, r1) in balanced_ranges(d_out, P_r):
+            part[r0:r1, :] = dY[r0:r1, c0:c1] @ X[:, c0:c1].T
+        parts.append(part)
+    dW = np.zeros((d_out, d_in), F64)
+    for part in parts:
+        dW = dW + part
+    return dW, parts
+
+
+def strip_with_halo(T, h0, h1):
+    """Rows [h0-1, h1+1) of an NCHW tensor as a strip owner sees them after
+    the halo exchange (Section 2.2): its own rows plus one boundary row copied
+    from each neighbour; zero rows where there is no neighbour."""
+    B, C, H, W = T.shape
+    S = np.zeros((B, C, h1 - h0 + 2, W), F64)
+    S[:, :, 1:1 + (h1 - h0), :] = T[:, :, h0:h1, :]
+    if h0 > 0:
+        S[:, :, 0, :] = T[:, :, h0 - 1, :]       # copy of the upper neighbour's last row
+    if h1 < H:
+        S[:, :, -1, :] = T[:, :, h1, :]          # copy of the lower neighbour's first row
+    return S
+
+
+def _conv_rows_valid(K, S):
+    """Correlate a haloed strip S [B,C,hs+2,W]: zero padding in W only, the
+    halo rows supply the H neighbours.  Output [B,O,hs,W]."""
+    B, C, Hh, W = S.shape
+    hs = Hh - 2
+    Sp = np.zeros((B, C, Hh, W + 2), F64)
+    Sp[:, :, :, 1:W + 1] = S
+    Y = np.zeros((B, K.shape[0], hs, W), F64)
+    for u in range(3):
+        for v in range(3):
+            Y += np.einsum("oc,bchw->bohw", K[:, :, u, v], Sp[:, :, u:u + hs, v:v + W])
+    return Y
+
+
+def conv3x3_strips(K, X, P_r):
+    """Domain-parallel forward: each of P_r strips correlates its own rows
+    after receiving one halo row per neighbour (Section 2.2, Eq. 7)."""
+    K = np.asarray(K, F64)
+    X = np.asarray(X, F64)
+    B, C, H, W = X.shape
+    Y = np.empty((B, K.shape[0], H, W), F64)
+    for (h0, h1) in balanced_ranges(H, P_r):
+        Y[:, :, h0:h1, :] = _conv_rows_valid(K, strip_with_halo(X, h0, h1))
+    return Y
+
+
+def conv3x3_dX_strips(K, dY, P_r):
+    """Domain-parallel backward-data: needs the dY halo rows (second term of
+    Eq. 7); the transposed correlation flips the taps and swaps channels."""
+    K = np.asarray(K, F64)
+    dY = np.asarray(dY, F64)
+    Kt = np.ascontiguousarray(K[:, :, ::-1, ::-1].transpose(1, 0, 2, 3))
+    B, O, H, W = dY.shape
+    dX = np.empty((B, K.shape[1], H, W), F64)
+    for (h0, h1) in balanced_ranges(H, P_r):
+        dX[:, :, h0:h1, :] = _conv_rows_valid(Kt, strip_with_halo(dY, h0, h1))
+    return dX
+
+
+def conv3x3_dK_strips(dY, X, P_r):
+    """Each strip forms a partial dK from its own output rows and its haloed
+    input; the all-reduce over the strips adds them in ascending order
+    (third term of Eq. 7).  Returns (dK, partials)."""
+    dY = np.asarray(dY, F64)
+    X = np.asarray(X, F64)
+    B, C, H, W = X.shape
+    parts = []
+    for (h0, h1) in balanced_ranges(H, P_r):
+        S = strip_with_halo(X, h0, h1)
+        hs = h1 - h0
+        Sp = np.zeros((B, C, hs + 2, W + 2), F64)
+        Sp[:, :, :, 1:W + 1] = S
+        part = np.zeros((dY.shape[1], C, 3, 3), F64)
+        for u in range(3):
+            for v in range(3):
+                part[:, :, u, v] = np.einsum("bohw,bchw->oc", dY[:, :, h0:h1, :],
+                                             Sp[:, :, u:u + hs, v:v + W])
+        parts.append(part)
+    dK = np.zeros_like(parts[0])
+    for part in parts:
+        dK = dK + part
+    return dK, parts
+
+
+def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
+                       P_r: int, P_c: int):
+    """The step of `train_step`, every contraction formed block by block over
+    the P_r x P_c grid and every cross-block sum taken as P separate partials
+    added in ascending block index.  FC layers split the model over P_r and the
+    batch over P_c; convolution layers split the image into P_r row strips
+    (P_c must be 1 for them)."""
+    L = len(layers)
+    Xs = [np.asarray(X1, F64)]
+    Ys = []
+    for i, lay in enumerate(layers):
+        if isinstance(lay, FC):
+            Y = fc_forward_blocked(lay.W, Xs[i], lay.b, P_r, P_c)
+        else:
+            assert P_c == 1
+            Y = conv3x3_strips(lay.K, Xs[i], P_r)
+        Ys.append(Y)
+        if i + 1 < L:
+            Xs.append(relu(Y) if lay.relu else Y)
+    B = _batch_of(Xs[0])
+    J, per, dY_top = loss_and_top_grad(Ys[-1], loss, labels)
+    dYs = [None] * L
+    dXs = [None] * L
+    dWs = [None] * L
+    dbs = [None] * L
+    dYs[L - 1] = dY_top
+    for i in range(L - 1, -1, -1):
+        lay = layers[i]
+        if isinstance(lay, FC):
+            dWs[i], _ = fc_dW_blocked(dYs[i], Xs[i], P_r, P_c)
+            if lay.b is not None:
+                db = np.zeros(lay.W.shape[0], F64)
+                for (c0, c1) in balanced_ranges(B, P_c):
+                    db = db + dYs[i][:, c0:c1].sum(axis=1)
+                dbs[i] = db
+        else:
+            dWs[i], _ = conv3x3_dK_strips(dYs[i], Xs[i], P_r)
+        if i > 0:
+            if isinstance(lay, FC):
+                dXs[i], _ = fc_dX_blocked(lay.W, dYs[i], P_r, P_c)
+            else:
+                dXs[i] = conv3x3_dX_strips(lay.K, dYs[i], P_r)
+            prev = layers[i - 1]
+            dYs[i - 1] = dXs[i] * (Ys[i - 1] > 0.0) if prev.relu else dXs[i]
+    new_W, new_b = [], []
+    for i, lay in enumerate(layers):
+        w = lay.W if isinstance(lay, FC) else lay.K
+        new_W.append(sgd(w, dWs[i], eta, B))
+        if isinstance(lay, FC) and lay.b is not None:
+            new_b.append(sgd(lay.b, dbs[i], eta, B))
+        else:
+            new_b.append(None)
+    return dict(Xs=Xs, Ys=Ys, J=J, per_sample=per, dYs=dYs, dXs=dXs, dWs=dWs,
+                dbs=dbs, new_W=new_W, new_b=new_b)
+
+
+def total_loss(layers: Sequence, X1, labels, loss: str) -> float:
+    """J alone (used by the finite-difference pins)."""
+    _, Ys = forward(layers, X1)
+    return loss_and_top_grad(Ys[-1], loss, labels)[0]

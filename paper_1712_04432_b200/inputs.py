@@ -1,0 +1,135 @@
+"""Seeded synthetic inputs shared by the tests, the benchmark and the smoke check.
+
+This module holds NO arithmetic of the method: it only draws random numbers
+(numpy Philox, counter based), rounds them to the storage type and describes
+the five workloads.  Both the CUDA path and the CPU oracle are fed from the
+arrays made here, so neither depends on the other.
+
+The workloads stand in for the paper's AlexNet / ImageNet setting (Section 3):
+fully connected stacks with classifier-head shapes, post-ReLU-like inputs and
+uniform class labels, and a two-layer 3x3 convolution on 224x224 images.
+
+Drawing order for one workload: X, then W_1..W_L, then the labels.
+Layout: X is [B, d_0] row-major (row = sample, i.e. the paper's column of
+X_1), W_i is [d_i, d_{i-1}] row-major, convolution input is NCHW and its
+kernel [C_out, C_in, 3, 3].
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional, Tuple
+
+import numpy as np
+
+
+def round_to_bf16(a: np.ndarray) -> np.ndarray:
+    """Round float32 values to the nearest bfloat16 (ties to even); the result
+    is float32 holding exactly representable bf16 values."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    u = a.view(np.uint32)
+    r = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32)
+
+
+def bf16_bits(a: np.ndarray) -> np.ndarray:
+    """uint16 bit patterns of float32 values that are already bf16-exact."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return (a.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+
+
+def bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    """float32 values of bf16 bit patterns."""
+    return (np.ascontiguousarray(bits).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+@dataclass
+class Workload:
+    name: str
+    kind: str                      # "fc" or "conv"
+    dims: Tuple[int, ...]          # fc: d_0..d_L ; conv: (C, H, W) with C_in == C_out
+    B: int
+    dtype: str                     # "f32" or "bf16"
+    x_dist: str                    # "normal" or "relu_normal"
+    loss: str                      # "softmax_ce" or "half_ssq"
+    eta: float = 0.01
+    n_layers: int = 0
+    grids: List[Tuple[int, int]] = field(default_factory=list)
+
+    @property
+    def L(self) -> int:
+        return self.n_layers if self.kind == "conv" else len(self.dims) - 1
+
+
+WORKLOADS = {
+    "cfg1": Workload("cfg1", "fc", (784, 512, 512, 10), 64, "f32", "normal", "softmax_ce",
+                     grids=[(1, 1), (2, 2), (4, 1), (1, 4)]),
+    "cfg2": Workload("cfg2", "fc", (9216, 4096, 4096, 1000), 256, "bf16", "relu_normal",
+                     "softmax_ce", grids=[(1, 1), (8, 1), (1, 8), (2, 4), (4, 2)]),
+    "cfg3": Workload("cfg3", "fc", (25088, 4096, 4096, 1000), 512, "bf16", "relu_normal",
+                     "softmax_ce", grids=[(1, 1), (4, 4), (16, 1), (1, 16)]),
+    "cfg4": Workload("cfg4", "conv", (64, 224, 224), 32, "bf16", "normal", "half_ssq",
+                     n_layers=2, grids=[(1, 1), (2, 1), (4, 1), (8, 1)]),
+    "cfg5": Workload("cfg5", "fc", (8192,) * 9, 8192, "bf16", "normal", "softmax_ce",
+                     grids=[(1, 1), (16, 16), (64, 4), (4, 64)]),
+}
+
+
+def fc_workload(dims, B, dtype="bf16", x_dist="normal", name="custom") -> Workload:
+    return Workload(name, "fc", tuple(int(d) for d in dims), int(B), dtype, x_dist, "softmax_ce")
+
+
+def conv_workload(C, H, W, B, n_layers=2, dtype="bf16", name="custom_conv") -> Workload:
+    return Workload(name, "conv", (int(C), int(H), int(W)), int(B), dtype, "normal",
+                    "half_ssq", n_layers=n_layers)
+
+
+@dataclass
+class Inputs:
+    X: np.ndarray                    # fc: [B, d_0] ; conv: [B, C, H, W]   (float32 values)
+    Ws: List[np.ndarray]             # fc: [d_i, d_{i-1}] ; conv: [C_out, C_in, 3, 3]
+    bs: List[Optional[np.ndarray]]   # zeros (fc) or None (conv)
+    labels: Optional[np.ndarray]     # int32 [B] or None
+
+
+def make_inputs(w: Workload, seed: int = 0) -> Inputs:
+    """Draw one workload's tensors.  Values are float32; for dtype "bf16" they
+    are already rounded to bf16 so that both paths start from identical data."""
+    rng = np.random.Generator(np.random.Philox(key=seed))
+    rnd = round_to_bf16 if w.dtype == "bf16" else (lambda a: np.ascontiguousarray(a, np.float32))
+    if w.kind == "fc":
+        d = w.dims
+        X = rng.standard_normal((w.B, d[0]), dtype=np.float32)
+        if w.x_dist == "relu_normal":
+            np.maximum(X, 0.0, out=X)
+        X = rnd(X)
+        Ws, bs = [], []
+        for i in range(1, len(d)):
+            Wi = rng.standard_normal((d[i], d[i - 1]), dtype=np.float32)
+            Wi *= np.float32(1.0 / np.sqrt(d[i - 1]))            # N(0, 1/fan_in)
+            Ws.append(rnd(Wi))
+            bs.append(np.zeros(d[i], np.float32))
+        labels = rng.integers(0, d[-1], size=w.B, dtype=np.int64).astype(np.int32)
+        return Inputs(X, Ws, bs, labels)
+    C, H, Wd = w.dims
+    X = rnd(rng.standard_normal((w.B, C, H, Wd), dtype=np.float32))
+    Ws = []
+    for _ in range(w.n_layers):
+        K = rng.standard_normal((C, C, 3, 3), dtype=np.float32)
+        K *= np.float32(np.sqrt(2.0 / (9 * C)))                  # N(0, 2/(9 C))
+        Ws.append(rnd(K))
+    return Inputs(X, Ws, [None] * w.n_layers, None)
+
+
+def step_flops(w: Workload) -> int:
+    """2 x MACs of the dense contractions one step needs: forward and
+    backward-weight for every layer, backward-data for layers 2..L."""
+    if w.kind == "fc":
+        d = w.dims
+        macs = 0
+        for i in range(1, len(d)):
+            per = w.B * d[i] * d[i - 1]
+            macs += (3 if i >= 2 else 2) * per
+        return 2 * macs
+    C, H, Wd = w.dims
+    per = w.B * H * Wd * C * C * 9
+    return 2 * per * (3 * w.n_layers - 1)
