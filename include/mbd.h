@@ -1,0 +1,172 @@
+/* mbd.h -- C ABI of libmbd: one minibatch-SGD training step in matrix form,
+ * computed on one B200 over a logical P_r x P_c block grid.
+ *
+ * Per layer i = 1..L (Section 1 and Appendix A.1/A.2 of the paper):
+ *     forward          Y_i  = W_i X_i (+ b_i),  X_{i+1} = ReLU(Y_i)
+ *     backward-data    dX_i = W_i^T dY_i            (i >= 2)
+ *     backward-weight  dW_i = dY_i X_i^T = sum_b dY_i[:,b] X_i[:,b]^T
+ *     update (Eq. 1)   W_i <- W_i - (eta/B) dW_i
+ * The grid (Section 2.3): P_r splits the model dimension d_i (or, for a
+ * domain-split convolution layer, the image height into row strips with halo
+ * rows, Section 2.2/2.4); P_c splits the batch.  The sum over the P_r row
+ * blocks that forms dX and the sum over the P_c batch blocks that forms dW
+ * (the paper's all-reduces) are taken on the device: consecutive logical
+ * blocks are either chained in the tensor-memory accumulator or written as
+ * fp32 partials and added, in ascending block order, by a reduction kernel.
+ *
+ * Conventions
+ *   - Every pointer named *_dev is DEVICE memory, every *_host is HOST memory.
+ *   - Activations are [B, d] row-major (row = sample = one column of the
+ *     paper's X_i); weights are [d_i, d_{i-1}] row-major; convolution input is
+ *     NCHW, its kernel [C_out, C_in, 3, 3].
+ *   - dtype MBD_BF16: X, W, activations and dY are bfloat16 bit patterns,
+ *     accumulation, logits, loss, partials, dW, biases are float.
+ *     dtype MBD_F32: everything float (no tensor cores; the <=1e-5 check mode).
+ *   - Calls only enqueue work on the stream given at creation; nothing
+ *     synchronises except mbd_poll_status, mbd_train_step_host and creation /
+ *     destruction.  The library owns weights, activations, gradients and
+ *     workspace; the caller owns every buffer it passes in.
+ *   - Errors are return codes; nothing aborts, throws or traps.
+ */
+#ifndef MBD_H
+#define MBD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define MBD_API __attribute__((visibility("default")))
+#else
+#define MBD_API
+#endif
+
+typedef struct mbd_net mbd_net; /* opaque */
+
+typedef enum {
+  MBD_OK = 0,
+  MBD_E_INVALID = 1,     /* null pointer, bad enum, bad size                        */
+  MBD_E_GRID = 2,        /* grid not realisable for these layers / batch            */
+  MBD_E_ALLOC = 3,       /* device or host allocation failed                        */
+  MBD_E_CUDA = 4,        /* a CUDA runtime / driver call failed                     */
+  MBD_E_STATE = 5,       /* call order violated (forward -> backward -> sgd_step)   */
+  MBD_E_TIMEOUT = 6,     /* a bounded device-side wait gave up (see mbd_poll_status)*/
+  MBD_E_UNSUPPORTED = 7  /* shape / layer kind outside what the kernels cover       */
+} mbd_status;
+
+enum { MBD_FC = 0, MBD_CONV3X3 = 1 };                 /* mbd_layer.kind                      */
+enum { MBD_SPLIT_MODEL = 0, MBD_SPLIT_DOMAIN = 1 };   /* mbd_layer.split: L_M or L_D, Eq. 9  */
+enum { MBD_F32 = 0, MBD_BF16 = 1 };                   /* dtype                               */
+enum { MBD_LOSS_SOFTMAX_CE = 0, MBD_LOSS_HALF_SSQ = 1 };
+
+/* One layer.  FC: d_in, d_out.  Convolution (3x3, stride 1, zero pad 1, NCHW):
+ * C_in, C_out, H, W, kh = kw = 3; d_in = C_in*H*W, d_out = C_out*H*W (Eq. 2).
+ * relu: apply f = ReLU after this layer (ignored for the last layer).
+ * bias: FC only. */
+typedef struct {
+  int32_t kind, split, relu, bias;
+  int64_t d_in, d_out;
+  int32_t C_in, C_out, H, W, kh, kw;
+} mbd_layer;
+
+/* Words (matrix elements) one process moves for one layer under the chosen
+ * grid: the bandwidth terms of Eq. 8 (model-split layers) and Eq. 9
+ * (domain-split layers). */
+typedef struct {
+  int64_t allgather_y;   /* Eq. 8 term 1:  B/P_c (P_r-1)/P_r d_i                    */
+  int64_t allreduce_dx;  /* Eq. 8 term 2:  2 B/P_c (P_r-1)/P_r d_{i-1}, 0 for i = 1 */
+  int64_t allreduce_dw;  /* Eq. 8 term 3:  2 (P_c-1)/P_c |W_i|/P_r ; Eq. 9 term 6:  */
+                         /*                2 (P-1)/P |W_i| for a domain-split layer */
+  int64_t halo_fwd;      /* Eq. 9 term 4:  B/P_c X_W X_C floor(k_h/2), 0 if P_r = 1 */
+  int64_t halo_bwd;      /* Eq. 9 term 5:  B/P_c Y_W Y_C floor(k_h/2), 0 if P_r = 1 */
+} mbd_words;
+
+/* Tensors readable through mbd_get_tensor. */
+enum {
+  MBD_T_ACT = 0,      /* stored forward output of `layer`: ReLU(Y_i) in the activation dtype,
+                         or the raw fp32 logits Y_L for the last FC layer; [B, d_i]          */
+  MBD_T_DY = 1,       /* dJ/dY_i, activation dtype, [B, d_i]                                 */
+  MBD_T_DW = 2,       /* dW_i, float, weight shape (valid after mbd_backward(net, 0))        */
+  MBD_T_DB = 3,       /* db_i, float [d_i]                                                   */
+  MBD_T_LOSS = 4,     /* per-sample loss, float [B] (softmax-CE); layer ignored              */
+  MBD_T_PARTIALS = 5  /* fp32 partial-sum workspace as left by the LAST reduction executed   */
+};
+
+/* Section 2.3 / 2.4.  Builds the plan for an L-layer network on batch B over a
+ * logical P_r x P_c grid and allocates all device state (weights start at zero).
+ *   max_partials  how many fp32 partial sums a reduction over P blocks may
+ *                 materialise: S = min(P, max_partials) partials, each chaining
+ *                 P/S consecutive logical blocks in the accumulator; 0 selects
+ *                 the default (4); 1 never materialises; >= P materialises every
+ *                 block's partial exactly as the paper's processes would hold it.
+ *   cuda_stream   a cudaStream_t (may be NULL for the default stream).
+ * MBD_E_GRID if P_r < 1, P_c < 1, P_c > B, P_r > min d_i over model-split layers,
+ * a strip would be shorter than its halo, or P_c != 1 with a domain-split layer.
+ * MBD_E_UNSUPPORTED for convolutions other than 3x3/s1/p1 with C_in = C_out = 64,
+ * or bf16 FC dims that are not multiples of 8. */
+MBD_API mbd_status mbd_net_create(const mbd_layer* layers_host, int L, int64_t B, int P_r, int P_c,
+                          int dtype, int loss, int max_partials, void* cuda_stream, mbd_net** out);
+MBD_API mbd_status mbd_net_destroy(mbd_net* net);
+
+/* Copy weights (network dtype) and bias (float, may be NULL) device -> library / back. */
+MBD_API mbd_status mbd_set_weights(mbd_net* net, int layer, const void* W_dev, const float* bias_dev);
+MBD_API mbd_status mbd_get_weights(mbd_net* net, int layer, void* W_dev, float* bias_dev);
+
+/* Forward pass (Section 1, Appendix A.1) and loss.  X_dev [B, d_0] (or NCHW) in the
+ * network dtype must stay valid and unchanged until the following mbd_backward has
+ * finished on the stream.  labels_dev: int32 [B] in [0, d_L) (softmax-CE; NULL for
+ * half-SSQ).  loss_sum_dev (may be NULL) receives J = sum over the batch. */
+MBD_API mbd_status mbd_forward(mbd_net* net, const void* X_dev, const int32_t* labels_dev,
+                       float* loss_sum_dev);
+
+/* Backward pass (Section 1, Appendix A.2) over the grid.  fused_eta == 0: dW_i and
+ * db_i are materialised in float and weights are left alone.  fused_eta > 0: the update
+ * of Eq. 1 with eta = fused_eta is applied inside the backward-weight epilogue (or the
+ * tail of its reduction) and dW is not kept. */
+MBD_API mbd_status mbd_backward(mbd_net* net, float fused_eta);
+
+/* Eq. 1 from the materialised gradients.  MBD_E_STATE if there was no backward since
+ * the last forward, or if that backward already applied the update. */
+MBD_API mbd_status mbd_sgd_step(mbd_net* net, float eta);
+
+/* One whole step from HOST buffers: copies X_host / labels_host to the device, runs
+ * forward, backward with the fused update, copies J back to *loss_host and waits. */
+MBD_API mbd_status mbd_train_step_host(mbd_net* net, const void* X_host, const int32_t* labels_host,
+                               float eta, float* loss_host);
+
+/* Eq. 8 / Eq. 9 bandwidth terms, one row per layer, exact integers (a term that is not
+ * integral is rounded up).  Host only: needs no GPU and no network object. */
+MBD_API mbd_status mbd_comm_words(const mbd_layer* layers_host, int L, int64_t B, int P_r, int P_c,
+                          mbd_words* out_host);
+
+/* Copy an internal tensor to dst_dev; `bytes` must equal the tensor's size. */
+MBD_API mbd_status mbd_get_tensor(mbd_net* net, int which, int layer, void* dst_dev, size_t bytes);
+
+/* Waits for the stream and reads the device status word: MBD_OK, or MBD_E_TIMEOUT if
+ * a kernel's bounded barrier wait ran out, or MBD_E_CUDA. */
+MBD_API mbd_status mbd_poll_status(mbd_net* net);
+
+/* Kernels launched by this network since creation (host counter). */
+MBD_API int64_t mbd_launch_count(const mbd_net* net);
+
+/* Stand-alone dense contraction on the tensor cores, used by the unit tests:
+ *   variant 0 (forward)          D[M,N] = A[M,K]   * B[N,K]^T   A, B row-major, K contiguous
+ *   variant 1 (backward-data)    D[M,N] = A[M,K]   * B[K,N]     B row-major, N contiguous
+ *   variant 2 (backward-weight)  D[M,N] = A[K,M]^T * B[K,N]     A, B row-major
+ * bf16 inputs, fp32 accumulation.  The K range is cut into k_splits balanced pieces;
+ * k_splits == 1 writes D_dev [M,N] float directly, otherwise partials_dev
+ * [k_splits][M][N] float receives the pieces and D_dev their sum (ascending order).
+ * Leading dimensions are in elements and, like M/N/K offsets, multiples of 8. */
+MBD_API mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, const void* A_dev,
+                         int64_t lda, const void* B_dev, int64_t ldb, float* D_dev, int64_t ldd,
+                         int k_splits, float* partials_dev, void* cuda_stream);
+
+MBD_API const char* mbd_strerror(mbd_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MBD_H */

@@ -1,0 +1,21 @@
+// Domain-parallel 3x3 convolution stack (Section 2.2 / 2.4): interface used by net.cu.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/mbd.h"
+
+namespace mbd {
+struct ConvNet;
+mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int max_partials, int num_sms, int* status,
+                       cudaStream_t stream, ConvNet** out);
+void conv_destroy(ConvNet* c);
+mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev);
+mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev);
+mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev, int64_t* launches);
+mbd_status conv_backward(ConvNet* c, float fused_eta, int64_t* launches);
+mbd_status conv_sgd_step(ConvNet* c, float eta, int64_t* launches);
+mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t bytes);
+size_t conv_input_bytes(const ConvNet* c);
+}  // namespace mbd

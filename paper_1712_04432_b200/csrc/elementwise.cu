@@ -1,0 +1,265 @@
+// Memory-bound kernels of the training step:
+//   reduce_partials  sum of the per-block fp32 partial sums in ascending block order,
+//                    standing in for the all-reduce over the P_r group (dX) or the P_c
+//                    group (dW) of Section 2.3 / Appendix A.2, with the tail operation
+//                    (ReLU mask, SGD update, plain store) fused
+//   softmax_xent     loss and top gradient dY_L = softmax(Y_L) - onehot
+//   colsum           db = dY 1 (bias gradient), deterministic two-stage
+//   sgd_update       Eq. 1 applied to materialised gradients
+//   sum_f32          fixed-order sum (total loss)
+// All of them are bound by HBM bandwidth: 16-byte accesses, grids sized in multiples of
+// the SM count, no atomics on floats (results are bitwise reproducible).
+#include "epi.cuh"
+
+namespace mbd {
+namespace {
+
+// ------------------------------------------------------------------ reduce_partials
+// Vector path: M*N and N multiples of 8; each thread owns 8 consecutive columns of a row.
+__global__ void __launch_bounds__(256)
+reduce_partials_vec8(const float* __restrict__ parts, int S, int64_t M, int64_t N, const Epi epi) {
+  const int64_t n8 = N >> 3;
+  const int64_t total = M * n8;
+  const int64_t plane = M * N;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t m = i / n8;
+    const int64_t n0 = (i - m * n8) << 3;
+    const float* src = parts + m * N + n0;
+    float4 a = __ldcs(reinterpret_cast<const float4*>(src));
+    float4 b = __ldcs(reinterpret_cast<const float4*>(src + 4));
+    for (int s = 1; s < S; ++s) {
+      const float4 c = __ldcs(reinterpret_cast<const float4*>(src + s * plane));
+      const float4 d = __ldcs(reinterpret_cast<const float4*>(src + s * plane + 4));
+      a.x += c.x; a.y += c.y; a.z += c.z; a.w += c.w;
+      b.x += d.x; b.y += d.y; b.z += d.z; b.w += d.w;
+    }
+    float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    epi_apply8(epi, m, n0, v);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+reduce_partials_scalar(const float* __restrict__ parts, int S, int64_t M, int64_t N, const Epi epi) {
+  const int64_t total = M * N;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    float a = parts[i];
+    for (int s = 1; s < S; ++s) a += parts[i + s * total];
+    const int64_t m = i / N;
+    epi_apply1(epi, m, i - m * N, a);
+  }
+}
+
+// ------------------------------------------------------------------ softmax cross-entropy
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// One CTA of NW warps per sample (row).  Three passes over the row (max, sum of exp,
+// write); the row (<= 32 KB) stays in L1/L2 between them.
+template <int NW>
+__global__ void __launch_bounds__(NW * 32)
+softmax_xent_kernel(const float* __restrict__ logits, int64_t d, const int32_t* __restrict__ labels,
+                    void* __restrict__ dY, int dy_bf16, float* __restrict__ per_sample) {
+  __shared__ float red[NW];
+  const int64_t b = blockIdx.x;
+  const float* row = logits + b * d;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float mx = -INFINITY;
+  for (int64_t k = tid; k < d; k += NW * 32) mx = fmaxf(mx, row[k]);
+  mx = warp_max(mx);
+  if (NW > 1) {
+    if (lane == 0) red[warp] = mx;
+    __syncthreads();
+    mx = red[0];
+#pragma unroll
+    for (int i = 1; i < NW; ++i) mx = fmaxf(mx, red[i]);
+    __syncthreads();
+  }
+  float sum = 0.f;
+  for (int64_t k = tid; k < d; k += NW * 32) sum += expf(row[k] - mx);
+  sum = warp_sum(sum);
+  if (NW > 1) {
+    if (lane == 0) red[warp] = sum;
+    __syncthreads();
+    sum = red[0];
+#pragma unroll
+    for (int i = 1; i < NW; ++i) sum += red[i];
+  }
+  const float inv = 1.f / sum;
+  const int label = labels[b];
+  for (int64_t k = tid; k < d; k += NW * 32) {
+    float g = expf(row[k] - mx) * inv;
+    if (k == label) g -= 1.f;
+    if (dy_bf16) reinterpret_cast<__nv_bfloat16*>(dY)[b * d + k] = __float2bfloat16_rn(g);
+    else reinterpret_cast<float*>(dY)[b * d + k] = g;
+  }
+  if (tid == 0) per_sample[b] = mx + logf(sum) - row[label];
+}
+
+// ------------------------------------------------------------------ fixed-order sum
+__global__ void __launch_bounds__(1024)
+sum_f32_kernel(const float* __restrict__ x, int64_t n, float scale, float* __restrict__ out) {
+  __shared__ float red[1024];
+  float a = 0.f;
+  for (int64_t i = threadIdx.x; i < n; i += 1024) a += x[i];
+  red[threadIdx.x] = a;
+  __syncthreads();
+  for (int s = 512; s > 0; s >>= 1) {
+    if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = red[0] * scale;
+}
+
+// ------------------------------------------------------------------ column sums (bias gradient)
+// Stage 1: grid (ceil(N/64), row_splits); 256 threads = 8 warps; a warp covers 64 columns
+// (2 per lane), warps stride over the rows of this split; the 8 warps are added in order.
+__global__ void __launch_bounds__(256)
+colsum_stage1(const void* __restrict__ dY, int dy_bf16, int64_t M, int64_t N, int row_splits,
+              float* __restrict__ scratch) {
+  __shared__ float red[8][64];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t n = static_cast<int64_t>(blockIdx.x) * 64 + lane * 2;
+  const int64_t r0 = (static_cast<int64_t>(blockIdx.y) * M) / row_splits;
+  const int64_t r1 = (static_cast<int64_t>(blockIdx.y + 1) * M) / row_splits;
+  float a0 = 0.f, a1 = 0.f;
+  if (n < N) {
+    const bool two = n + 1 < N;
+    for (int64_t m = r0 + warp; m < r1; m += 8) {
+      if (dy_bf16) {
+        const __nv_bfloat16* p = reinterpret_cast<const __nv_bfloat16*>(dY) + m * N + n;
+        a0 += __bfloat162float(p[0]);
+        if (two) a1 += __bfloat162float(p[1]);
+      } else {
+        const float* p = reinterpret_cast<const float*>(dY) + m * N + n;
+        a0 += p[0];
+        if (two) a1 += p[1];
+      }
+    }
+  }
+  red[warp][lane * 2] = a0;
+  red[warp][lane * 2 + 1] = a1;
+  __syncthreads();
+  if (threadIdx.x < 64) {
+    float s = red[0][threadIdx.x];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) s += red[w][threadIdx.x];
+    const int64_t nn = static_cast<int64_t>(blockIdx.x) * 64 + threadIdx.x;
+    if (nn < N) scratch[static_cast<int64_t>(blockIdx.y) * N + nn] = s;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+colsum_stage2(const float* __restrict__ scratch, int row_splits, int64_t N, float* __restrict__ db,
+              float* __restrict__ bias, float scale) {
+  const int64_t n = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+  if (n >= N) return;
+  float s = scratch[n];
+  for (int r = 1; r < row_splits; ++r) s += scratch[static_cast<int64_t>(r) * N + n];
+  if (db) db[n] = s;
+  if (bias) bias[n] = fmaf(scale, s, bias[n]);
+}
+
+// ------------------------------------------------------------------ SGD update (Eq. 1)
+__global__ void __launch_bounds__(256)
+sgd_update_bf16_vec8(__nv_bfloat16* __restrict__ w, const float* __restrict__ g, int64_t n8, float scale) {
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n8;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const float4 a = __ldcs(reinterpret_cast<const float4*>(g + i * 8));
+    const float4 b = __ldcs(reinterpret_cast<const float4*>(g + i * 8 + 4));
+    uint4* p = reinterpret_cast<uint4*>(w + i * 8);
+    const uint4 q = *p;
+    uint4 o;
+    o.x = pack_bf16x2(fmaf(scale, a.x, bf16_bits_to_f32(q.x & 0xFFFFu)), fmaf(scale, a.y, bf16_bits_to_f32(q.x >> 16)));
+    o.y = pack_bf16x2(fmaf(scale, a.z, bf16_bits_to_f32(q.y & 0xFFFFu)), fmaf(scale, a.w, bf16_bits_to_f32(q.y >> 16)));
+    o.z = pack_bf16x2(fmaf(scale, b.x, bf16_bits_to_f32(q.z & 0xFFFFu)), fmaf(scale, b.y, bf16_bits_to_f32(q.z >> 16)));
+    o.w = pack_bf16x2(fmaf(scale, b.z, bf16_bits_to_f32(q.w & 0xFFFFu)), fmaf(scale, b.w, bf16_bits_to_f32(q.w >> 16)));
+    *p = o;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+sgd_update_scalar(void* __restrict__ w, int w_bf16, const float* __restrict__ g, int64_t n, float scale) {
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    if (w_bf16) {
+      __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(w) + i;
+      *p = __float2bfloat16_rn(fmaf(scale, g[i], __bfloat162float(*p)));
+    } else {
+      float* p = reinterpret_cast<float*>(w) + i;
+      *p = fmaf(scale, g[i], *p);
+    }
+  }
+}
+
+int grid_for(int64_t work_items, int num_sms, int per_sm) {
+  int64_t blocks = (work_items + 255) / 256;
+  const int64_t cap = static_cast<int64_t>(num_sms) * per_sm;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return static_cast<int>(blocks);
+}
+
+}  // namespace
+
+cudaError_t reduce_partials_launch(const float* parts, int S, int64_t M, int64_t N, const Epi& epi, int num_sms,
+                                   cudaStream_t stream) {
+  const bool vec = (N % 8 == 0) && (epi.ldo % 8 == 0) && (epi.mask == nullptr || epi.ldmask % 8 == 0);
+  if (vec) {
+    reduce_partials_vec8<<<grid_for(M * (N / 8), num_sms, 8), 256, 0, stream>>>(parts, S, M, N, epi);
+  } else {
+    reduce_partials_scalar<<<grid_for(M * N, num_sms, 8), 256, 0, stream>>>(parts, S, M, N, epi);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t softmax_xent_launch(const float* logits, int64_t B, int64_t d, const int32_t* labels, void* dY,
+                                int dy_bf16, float* per_sample, cudaStream_t stream) {
+  if (d <= 64) softmax_xent_kernel<1><<<static_cast<unsigned>(B), 32, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  else if (d <= 2048) softmax_xent_kernel<4><<<static_cast<unsigned>(B), 128, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  else softmax_xent_kernel<8><<<static_cast<unsigned>(B), 256, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  return cudaGetLastError();
+}
+
+cudaError_t sum_f32_launch(const float* x, int64_t n, float scale, float* out, cudaStream_t stream) {
+  sum_f32_kernel<<<1, 1024, 0, stream>>>(x, n, scale, out);
+  return cudaGetLastError();
+}
+
+int colsum_row_splits(int64_t M) {
+  int64_t r = M / 64;
+  if (r < 1) r = 1;
+  if (r > 32) r = 32;
+  return static_cast<int>(r);
+}
+
+cudaError_t colsum_launch(const void* dY, int dy_bf16, int64_t M, int64_t N, float* scratch, int row_splits,
+                          float* db, float* bias, float scale, cudaStream_t stream) {
+  dim3 g1(static_cast<unsigned>((N + 63) / 64), row_splits);
+  colsum_stage1<<<g1, 256, 0, stream>>>(dY, dy_bf16, M, N, row_splits, scratch);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  colsum_stage2<<<static_cast<unsigned>((N + 255) / 256), 256, 0, stream>>>(scratch, row_splits, N, db, bias, scale);
+  return cudaGetLastError();
+}
+
+cudaError_t sgd_update_launch(void* w, int w_bf16, const float* g, int64_t n, float scale, int num_sms,
+                              cudaStream_t stream) {
+  if (w_bf16 && n % 8 == 0) {
+    sgd_update_bf16_vec8<<<grid_for(n / 8, num_sms, 8), 256, 0, stream>>>(reinterpret_cast<__nv_bfloat16*>(w), g, n / 8, scale);
+  } else {
+    sgd_update_scalar<<<grid_for(n, num_sms, 8), 256, 0, stream>>>(w, w_bf16, g, n, scale);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace mbd

@@ -1,0 +1,432 @@
+// Dense bf16 contraction on the 5th-generation tensor cores (tcgen05) for the three
+// products of a layer: forward Y = W X, backward-data dX = W^T dY, backward-weight
+// dW = dY X^T (Section 1 of the paper), with the K range optionally cut into the
+// partial sums a P_r x P_c grid would form (Appendix A.2).
+//
+// One persistent CTA per SM, 192 threads, warp-specialised:
+//   warp 0      TMA producer: operand tiles -> 128B-swizzled shared-memory ring
+//   warp 1      allocates tensor memory; one lane issues tcgen05.mma (128 x BN x 16 per
+//               instruction, fp32 accumulator in TMEM) and commits to mbarriers
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (lane = row), apply the epilogue
+//               operation and store; two accumulators alternate so the epilogue of one
+//               tile runs under the MMAs of the next
+// Transposed operands are not copied: an operand whose contiguous dimension is M or N is
+// loaded as 64-wide column chunks and described to the MMA as "MN-major".
+// Every mbarrier wait is bounded; on time-out the kernel records a code and leaves.
+#include "epi.cuh"
+
+namespace mbd {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;
+constexpr int NUM_THREADS = 192;
+constexpr int SMEM_RING_BYTES = 192 * 1024;
+constexpr int GROUP_M = 16;            // m-tiles per raster group (L2 reuse of the B operand)
+constexpr unsigned long long WAIT_LIMIT_NS = 4000000000ull;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false after WAIT_LIMIT_NS or when another role has given up.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            int* status, int code) {
+  const unsigned long long t0 = globaltimer_ns();
+  for (;;) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+      *abort_flag = 1;
+      atomicCAS(status, 0, code);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status, int code) {
+  for (int i = 0; i < 64; ++i)
+    if (mbar_try(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status, code);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.
+//   K-major tile (rows of 128 B): 8-row groups are 1024 B apart (stride offset); the leading
+//     offset is unused.  Stepping 16 elements along K adds 32 B to the start address.
+//   MN-major tile (64-wide column chunks, each row of 128 B is one k): 8-k groups are 1024 B
+//     apart (stride offset), chunks are `chunk_bytes` apart (leading offset).  Stepping 16
+//     along K adds 16 rows = 2048 B.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;   // descriptor version for this architecture
+  d |= 2ull << 61;   // 128-byte swizzle
+  return d;
+}
+
+struct Params {
+  int M, N, K;
+  int tiles_m, tiles_n, kb_total, S;
+  float* partials;
+  Epi epi;
+  int* status;
+};
+
+struct Work {
+  int tm, tn, s, kb0, kb1;
+};
+
+__device__ __forceinline__ Work decode_work(const Params& p, int w) {
+  const int num_tiles = p.tiles_m * p.tiles_n;
+  Work o;
+  o.s = w / num_tiles;
+  const int t = w - o.s * num_tiles;
+  const int per_group = GROUP_M * p.tiles_n;
+  const int g = t / per_group;
+  const int first_m = g * GROUP_M;
+  const int gsize = min(p.tiles_m - first_m, GROUP_M);
+  const int r = t - g * per_group;
+  o.tm = first_m + r % gsize;
+  o.tn = r / gsize;
+  o.kb0 = static_cast<int>((static_cast<long long>(o.s) * p.kb_total) / p.S);
+  o.kb1 = static_cast<int>((static_cast<long long>(o.s + 1) * p.kb_total) / p.S);
+  return o;
+}
+
+template <int A_MN, int B_MN, int BN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
+  constexpr int A_BYTES = BM * BK * 2;
+  constexpr int B_BYTES = BN * BK * 2;
+  constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int STAGES = SMEM_RING_BYTES / STAGE_BYTES;
+  constexpr int TMEM_COLS = 2 * BN;
+  constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(A_MN) << 15) | (uint32_t(B_MN) << 16) |
+                             (uint32_t(BN >> 3) << 17) | (uint32_t(BM >> 4) << 24);
+
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[STAGES];
+  __shared__ __align__(8) uint64_t tmem_full_bar[2];
+  __shared__ __align__(8) uint64_t tmem_empty_bar[2];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  // 1024-byte alignment of the ring (needed by the 128B swizzle pattern)
+  const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(smem_u32(&full_bar[i]), 1);
+      mbar_init(smem_u32(&empty_bar[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&tmem_full_bar[i]), 1);
+      mbar_init(smem_u32(&tmem_empty_bar[i]), 4);
+    }
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  const int total_work = p.tiles_m * p.tiles_n * p.S;
+  volatile int* abortp = &abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+        const Work wk = decode_work(p, w);
+        for (int kb = wk.kb0; kb < wk.kb1; ++kb) {
+          ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
+          if (!ok) break;
+          const uint32_t fb = smem_u32(&full_bar[stage]);
+          const uint32_t sa = ring + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+          mbar_expect_tx(fb, STAGE_BYTES);
+          if (A_MN == 0) {
+            tma_load_2d(sa, &tmA, kb * BK, wk.tm * BM, fb);
+          } else {
+#pragma unroll
+            for (int c = 0; c < BM / 64; ++c) tma_load_2d(sa + c * (64 * BK * 2), &tmA, wk.tm * BM + c * 64, kb * BK, fb);
+          }
+          if (B_MN == 0) {
+            tma_load_2d(sb, &tmB, kb * BK, wk.tn * BN, fb);
+          } else {
+#pragma unroll
+            for (int c = 0; c < BN / 64; ++c) tma_load_2d(sb + c * (64 * BK * 2), &tmB, wk.tn * BN + c * 64, kb * BK, fb);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++it) {
+        const Work wk = decode_work(p, w);
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1u;
+        ok = mbar_wait(smem_u32(&tmem_empty_bar[acc]), acc_phase ^ 1u, abortp, p.status, DEV_TIMEOUT_MMA_TMEM);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = wk.kb0; kb < wk.kb1; ++kb) {
+          ok = mbar_wait(smem_u32(&full_bar[stage]), phase, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = ring + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+          const uint64_t adesc = A_MN ? make_desc(sa, 64 * BK * 2, 1024) : make_desc(sa, 16, 1024);
+          const uint64_t bdesc = B_MN ? make_desc(sb, 64 * BK * 2, 1024) : make_desc(sb, 16, 1024);
+          constexpr uint64_t A_STEP = (A_MN ? (UMMA_K * 128) : (UMMA_K * 2)) >> 4;
+          constexpr uint64_t B_STEP = (B_MN ? (UMMA_K * 128) : (UMMA_K * 2)) >> 4;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            tc_mma_bf16(d_tmem, adesc + k * A_STEP, bdesc + k * B_STEP, IDESC, (kb > wk.kb0 || k > 0) ? 1u : 0u);
+          tc_commit(smem_u32(&empty_bar[stage]));   // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(smem_u32(&tmem_full_bar[acc]));   // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int q = warp & 3;                       // TMEM lane quarter this warp may read
+    int it = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++it) {
+      const Work wk = decode_work(p, w);
+      const int acc = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1u;
+      ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int64_t m = static_cast<int64_t>(wk.tm) * BM + q * 32 + lane;
+      const bool row_ok = m < p.M;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
+      float* part = p.S > 1 ? p.partials + static_cast<int64_t>(wk.s) * p.M * p.N : nullptr;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tc_ld32(taddr + c * 32, r);
+        tc_wait_ld();
+        const int64_t n0 = static_cast<int64_t>(wk.tn) * BN + c * 32;
+        if (row_ok) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int64_t n = n0 + j * 8;
+            if (n < p.N) {
+              float v[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j * 8 + i]);
+              if (part) {
+                float* dst = part + m * p.N + n;
+                *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+                *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
+              } else {
+                epi_apply8(p.epi, m, n, v);
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ----------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+bool g_init_done = false;
+
+// 2-D bf16 tensor map: `inner` contiguous elements per row, `rows` rows `ld` elements apart.
+cudaError_t make_map(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t rows, uint64_t ld,
+                     uint32_t box_inner, uint32_t box_rows) {
+  const cuuint64_t dims[2] = {inner, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {box_inner, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+template <int A_MN, int B_MN, int BN>
+cudaError_t set_attr() {
+  return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              SMEM_RING_BYTES + 1024);
+}
+
+template <int A_MN, int B_MN, int BN>
+cudaError_t launch_t(const TcGemm& g, const Params& p, cudaStream_t stream) {
+  gemm_tc_kernel<A_MN, B_MN, BN><<<g.grid, NUM_THREADS, SMEM_RING_BYTES + 1024, stream>>>(g.tmA, g.tmB, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t tc_gemm_init() {
+  if (g_init_done) return cudaSuccess;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return e;
+  if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if ((e = set_attr<0, 0, 256>()) != cudaSuccess) return e;
+  if ((e = set_attr<0, 0, 128>()) != cudaSuccess) return e;
+  if ((e = set_attr<0, 1, 256>()) != cudaSuccess) return e;
+  if ((e = set_attr<0, 1, 128>()) != cudaSuccess) return e;
+  if ((e = set_attr<1, 1, 256>()) != cudaSuccess) return e;
+  if ((e = set_attr<1, 1, 128>()) != cudaSuccess) return e;
+  g_init_done = true;
+  return cudaSuccess;
+}
+
+cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B, int64_t ldb, int num_sms) {
+  cudaError_t e = tc_gemm_init();
+  if (e != cudaSuccess) return e;
+  const int tiles_m = (g.M + BM - 1) / BM;
+  // Narrower tiles when 256-wide ones would leave SMs without work.
+  const int t256 = tiles_m * ((g.N + 255) / 256) * g.k_splits;
+  g.BN = t256 >= num_sms ? 256 : 128;
+  const int tiles_n = (g.N + g.BN - 1) / g.BN;
+  const int kb_total = (g.K + BK - 1) / BK;
+  if (g.k_splits > kb_total) g.k_splits = kb_total;
+  const long long total = 1ll * tiles_m * tiles_n * g.k_splits;
+  g.grid = static_cast<int>(total < num_sms ? total : num_sms);
+  const bool a_mn = g.variant == 2, b_mn = g.variant >= 1;
+  if (!a_mn) e = make_map(&g.tmA, A, g.K, g.M, lda, BK, BM);      // A[M,K]: inner = K
+  else e = make_map(&g.tmA, A, g.M, g.K, lda, 64, BK);             // A[K,M]: inner = M, one 64-wide chunk per box
+  if (e != cudaSuccess) return e;
+  if (!b_mn) e = make_map(&g.tmB, B, g.K, g.N, ldb, BK, g.BN);    // B[N,K]
+  else e = make_map(&g.tmB, B, g.N, g.K, ldb, 64, BK);             // B[K,N]
+  return e;
+}
+
+cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
+  Params p;
+  p.M = g.M; p.N = g.N; p.K = g.K;
+  p.tiles_m = (g.M + BM - 1) / BM;
+  p.tiles_n = (g.N + g.BN - 1) / g.BN;
+  p.kb_total = (g.K + BK - 1) / BK;
+  p.S = g.k_splits;
+  p.partials = g.partials;
+  p.epi = g.epi;
+  p.status = g.status;
+  if (g.variant == 0) return g.BN == 256 ? launch_t<0, 0, 256>(g, p, stream) : launch_t<0, 0, 128>(g, p, stream);
+  if (g.variant == 1) return g.BN == 256 ? launch_t<0, 1, 256>(g, p, stream) : launch_t<0, 1, 128>(g, p, stream);
+  return g.BN == 256 ? launch_t<1, 1, 256>(g, p, stream) : launch_t<1, 1, 128>(g, p, stream);
+}
+
+}  // namespace mbd

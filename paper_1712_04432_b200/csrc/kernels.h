@@ -1,0 +1,95 @@
+// Internal interface between the host plan (net.cu) and the kernel files.
+// Nothing here is exported; the C ABI lives in include/mbd.h.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mbd {
+
+// Device status word values (0 = fine).  A kernel that gives up a bounded wait
+// stores one of these with atomicCAS(status, 0, code) and returns.
+enum : int {
+  DEV_OK = 0,
+  DEV_TIMEOUT_PRODUCER = 101,   // TMA producer waited too long for a free stage
+  DEV_TIMEOUT_MMA_FULL = 102,   // MMA issuer waited too long for operands
+  DEV_TIMEOUT_MMA_TMEM = 103,   // MMA issuer waited too long for a drained accumulator
+  DEV_TIMEOUT_EPILOGUE = 104,   // epilogue waited too long for a finished accumulator
+  DEV_BAD_SCRATCH = 105
+};
+
+// What happens to a finished fp32 accumulator element acc at (m, n).
+enum EpiOp : int {
+  EPI_ACT = 0,    // v = acc (+ bias[n]); relu ? max(v,0) : v; store (bf16 or f32)
+  EPI_MASK = 1,   // v = (mask == null || mask[m,n] > 0) ? acc : 0; store (bf16 or f32)
+  EPI_SGD = 2     // out[m,n] = out[m,n] + scale * acc   (Eq. 1 with scale = -eta/B)
+};
+
+struct Epi {
+  int op;
+  int out_bf16;        // 1: out (and mask) are bf16, 0: float
+  int relu;
+  void* out;           // [M, ldo]
+  int64_t ldo;
+  const float* bias;   // [N] or null
+  const void* mask;    // [M, ldmask] in out's dtype, or null
+  int64_t ldmask;
+  float scale;
+};
+
+// ---- tcgen05 GEMM -----------------------------------------------------------
+// variant 0: D[M,N] = A[M,K] B[N,K]^T      (A, B K-contiguous)          forward
+// variant 1: D[M,N] = A[M,K] B[K,N]        (B N-contiguous)             backward-data
+// variant 2: D[M,N] = A[K,M]^T B[K,N]      (A M-contiguous, B N-cont.)  backward-weight
+struct TcGemm {
+  CUtensorMap tmA, tmB;
+  int variant;
+  int BN;               // CTA tile width: 256 or 128
+  int M, N, K;
+  int k_splits;         // S >= 1; S > 1 writes partials[S][M][N] (fp32) and skips the epilogue op
+  float* partials;
+  Epi epi;
+  int* status;
+  int grid;
+};
+
+// Fills tmA/tmB/BN/grid.  Returns cudaSuccess or an error.
+cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B, int64_t ldb,
+                            int num_sms);
+cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream);
+cudaError_t tc_gemm_init();   // driver entry point lookup + kernel attributes; idempotent
+
+// ---- fp32 SIMT GEMM (check mode) ----------------------------------------------
+struct SimtGemm {
+  int M, N, K;
+  const float* A; int64_t a_sm, a_sk;   // A(m,k) = A[m*a_sm + k*a_sk]
+  const float* B; int64_t b_sn, b_sk;   // B(n,k) = B[n*b_sn + k*b_sk]
+  int k_splits;                         // balanced ranges [floor(s K/S), floor((s+1) K/S))
+  float* partials;                      // [S][M][N] when S > 1
+  Epi epi;
+};
+cudaError_t simt_gemm_launch(const SimtGemm& g, cudaStream_t stream);
+
+// ---- memory-bound kernels ---------------------------------------------------------
+// out = sum_{s<S} parts[s] (ascending s), then the epilogue op.  parts is [S][M][N] dense.
+cudaError_t reduce_partials_launch(const float* parts, int S, int64_t M, int64_t N, const Epi& epi,
+                                   int num_sms, cudaStream_t stream);
+// As above with the partials addressed through a device pointer variable.
+cudaError_t softmax_xent_launch(const float* logits, int64_t B, int64_t d, const int32_t* labels,
+                                void* dY, int dy_bf16, float* per_sample, cudaStream_t stream);
+// sum of n floats in a fixed order into *out (single CTA, deterministic); scale applied.
+cudaError_t sum_f32_launch(const float* x, int64_t n, float scale, float* out, cudaStream_t stream);
+// db[n] = sum_m dY[m,n]; two deterministic stages through `scratch` [rows_split][N].
+// If bias != null: bias[n] += scale * db[n].  If db != null: db[n] stored.
+cudaError_t colsum_launch(const void* dY, int dy_bf16, int64_t M, int64_t N, float* scratch,
+                          int row_splits, float* db, float* bias, float scale, cudaStream_t stream);
+int colsum_row_splits(int64_t M);
+// w[i] += scale * g[i]   (w bf16 or f32, g f32)
+cudaError_t sgd_update_launch(void* w, int w_bf16, const float* g, int64_t n, float scale,
+                              int num_sms, cudaStream_t stream);
+
+// ---- domain-parallel 3x3 convolution (conv.cu) ------------------------------------------
+struct ConvNet;   // defined in conv.cu
+}  // namespace mbd

@@ -1,0 +1,508 @@
+// Host plan and C ABI: owns the device state of one network, fixes the launch order of
+// a training step (Section 1; Appendix A.1/A.2) and maps the logical P_r x P_c grid of
+// Section 2.3 onto K-range partial sums.
+//
+//   forward   i = 1..L : Y_i = W_i X_i (+b), X_{i+1} = ReLU(Y_i); loss and dY_L
+//   backward  i = L..1 : db_i; dX_i (i >= 2) as a sum over P_r row blocks of W_i, then the
+//                        ReLU mask; dW_i as a sum over P_c batch blocks, then Eq. 1
+// A sum over P blocks is taken as S = min(P, max_partials) fp32 partials (each chaining
+// P/S consecutive blocks inside the accumulator) followed by reduce_partials.  The update
+// of W_i is ordered after the dX_i product of the same layer, which still reads the old W_i.
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "../../include/mbd.h"
+#include "conv.h"
+#include "kernels.h"
+
+using namespace mbd;
+
+namespace {
+
+enum { ST_IDLE = 0, ST_FWD = 1, ST_BWD_UNFUSED = 2, ST_BWD_FUSED = 3 };
+
+struct Layer {
+  mbd_layer spec;
+  int64_t d_in = 0, d_out = 0, nW = 0;
+  void* W = nullptr;
+  float* bias = nullptr;
+  float* dW = nullptr;
+  float* db = nullptr;
+  void* act = nullptr;   // stored forward output [B, d_out]; float logits for the last FC layer
+  void* dY = nullptr;    // [B, d_out] activation dtype
+  TcGemm fwd, bwd_data, bwd_weight;
+};
+
+}  // namespace
+
+struct mbd_net {
+  int L = 0;
+  int64_t B = 0;
+  int P_r = 1, P_c = 1, dtype = MBD_BF16, loss = 0, max_partials = 4;
+  cudaStream_t stream = nullptr;
+  int num_sms = 148;
+  int device = 0;
+  bool is_conv = false;
+  std::vector<Layer> layers;
+  float* partials = nullptr;
+  size_t partial_elems = 0;
+  float* colsum_scratch = nullptr;
+  float* per_sample = nullptr;
+  float* loss_dev = nullptr;
+  int* status = nullptr;
+  const void* X = nullptr;
+  const void* X_mapped = nullptr;   // input pointer the layer-1 tensor maps were built for
+  const int32_t* labels = nullptr;
+  int state = ST_IDLE;
+  int64_t launches = 0;
+  void* X_stage = nullptr;
+  int32_t* labels_stage = nullptr;
+  ConvNet* conv = nullptr;
+  size_t elt() const { return dtype == MBD_BF16 ? 2 : 4; }
+};
+
+namespace {
+
+#define CK(expr)                          \
+  do {                                    \
+    cudaError_t e_ = (expr);              \
+    if (e_ != cudaSuccess) {              \
+      (void)cudaGetLastError();           \
+      return MBD_E_CUDA;                  \
+    }                                     \
+  } while (0)
+
+mbd_status dev_alloc(void** p, size_t bytes) {
+  if (bytes == 0) bytes = 16;
+  cudaError_t e = cudaMalloc(p, bytes);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    *p = nullptr;
+    return MBD_E_ALLOC;
+  }
+  return MBD_OK;
+}
+
+int splits_for(int P, int max_partials) { return P < max_partials ? P : max_partials; }
+
+Epi epi_act(void* out, int64_t ldo, int out_bf16, const float* bias, int relu) {
+  Epi e{};
+  e.op = EPI_ACT; e.out_bf16 = out_bf16; e.relu = relu; e.out = out; e.ldo = ldo; e.bias = bias;
+  return e;
+}
+Epi epi_mask(void* out, int64_t ldo, int out_bf16, const void* mask, int64_t ldmask) {
+  Epi e{};
+  e.op = EPI_MASK; e.out_bf16 = out_bf16; e.out = out; e.ldo = ldo; e.mask = mask; e.ldmask = ldmask;
+  return e;
+}
+Epi epi_sgd(void* w, int64_t ldo, int out_bf16, float scale) {
+  Epi e{};
+  e.op = EPI_SGD; e.out_bf16 = out_bf16; e.out = w; e.ldo = ldo; e.scale = scale;
+  return e;
+}
+
+// One contraction on the path that matches the network dtype, followed by the reduction
+// of its partials when the K range was split.
+mbd_status run_gemm(mbd_net* n, TcGemm& tc, int variant, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                    const void* Bm, int64_t ldb, int S, const Epi& epi) {
+  if (n->dtype == MBD_BF16) {
+    tc.epi = epi;
+    tc.partials = n->partials;
+    CK(tc_gemm_launch(tc, n->stream));
+    n->launches++;
+    S = tc.k_splits;
+  } else {
+    SimtGemm g{};
+    g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
+    g.A = static_cast<const float*>(A);
+    g.B = static_cast<const float*>(Bm);
+    if (variant == 0) { g.a_sm = lda; g.a_sk = 1; g.b_sn = ldb; g.b_sk = 1; }
+    else if (variant == 1) { g.a_sm = lda; g.a_sk = 1; g.b_sn = 1; g.b_sk = ldb; }
+    else { g.a_sm = 1; g.a_sk = lda; g.b_sn = 1; g.b_sk = ldb; }
+    if (S > K) S = static_cast<int>(K);
+    g.k_splits = S;
+    g.partials = n->partials;
+    g.epi = epi;
+    CK(simt_gemm_launch(g, n->stream));
+    n->launches++;
+  }
+  if (S > 1) {
+    CK(reduce_partials_launch(n->partials, S, M, N, epi, n->num_sms, n->stream));
+    n->launches++;
+  }
+  return MBD_OK;
+}
+
+mbd_status prepare_tc(mbd_net* n, TcGemm& g, int variant, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                      const void* Bm, int64_t ldb, int S) {
+  g = TcGemm{};
+  g.variant = variant;
+  g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
+  g.k_splits = S;
+  g.status = n->status;
+  CK(tc_gemm_prepare(g, A, lda, Bm, ldb, n->num_sms));
+  return MBD_OK;
+}
+
+const void* layer_input(const mbd_net* n, int i) { return i == 0 ? n->X : n->layers[i - 1].act; }
+
+// (Re)build the tensor maps that reference the caller's input buffer.
+mbd_status map_input(mbd_net* n) {
+  if (n->dtype != MBD_BF16 || n->is_conv || n->X_mapped == n->X) return MBD_OK;
+  Layer& l = n->layers[0];
+  const int S_c = splits_for(n->P_c, n->max_partials);
+  mbd_status s = prepare_tc(n, l.fwd, 0, n->B, l.d_out, l.d_in, n->X, l.d_in, l.W, l.d_in, 1);
+  if (s != MBD_OK) return s;
+  s = prepare_tc(n, l.bwd_weight, 2, l.d_out, l.d_in, n->B, l.dY, l.d_out, n->X, l.d_in, S_c);
+  if (s != MBD_OK) return s;
+  n->X_mapped = n->X;
+  return MBD_OK;
+}
+
+void free_net(mbd_net* n) {
+  if (!n) return;
+  for (Layer& l : n->layers) {
+    cudaFree(l.W); cudaFree(l.bias); cudaFree(l.dW); cudaFree(l.db); cudaFree(l.act); cudaFree(l.dY);
+  }
+  cudaFree(n->partials); cudaFree(n->colsum_scratch); cudaFree(n->per_sample); cudaFree(n->loss_dev);
+  cudaFree(n->status); cudaFree(n->X_stage); cudaFree(n->labels_stage);
+  if (n->conv) conv_destroy(n->conv);
+  (void)cudaGetLastError();
+  delete n;
+}
+
+}  // namespace
+
+extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, int dtype, int loss,
+                                     int max_partials, void* cuda_stream, mbd_net** out) {
+  if (!layers || !out || L < 1 || B < 1) return MBD_E_INVALID;
+  if (dtype != MBD_F32 && dtype != MBD_BF16) return MBD_E_INVALID;
+  if (loss != MBD_LOSS_SOFTMAX_CE && loss != MBD_LOSS_HALF_SSQ) return MBD_E_INVALID;
+  if (max_partials < 0) return MBD_E_INVALID;
+  *out = nullptr;
+  if (P_r < 1 || P_c < 1 || P_c > B) return MBD_E_GRID;
+  const bool is_conv = layers[0].kind == MBD_CONV3X3;
+  for (int i = 0; i < L; ++i) {
+    const mbd_layer& l = layers[i];
+    if ((l.kind == MBD_CONV3X3) != is_conv) return MBD_E_UNSUPPORTED;   // no mixed stacks yet
+    if (l.kind == MBD_FC) {
+      if (l.d_in < 1 || l.d_out < 1) return MBD_E_INVALID;
+      if (l.split != MBD_SPLIT_MODEL) return MBD_E_INVALID;
+      if (i > 0 && l.d_in != layers[i - 1].d_out) return MBD_E_INVALID;
+      if (P_r > l.d_out) return MBD_E_GRID;
+      if (dtype == MBD_BF16 && (l.d_in % 8 || l.d_out % 8)) return MBD_E_UNSUPPORTED;
+      if (l.d_in > INT32_MAX || l.d_out > INT32_MAX || B > INT32_MAX) return MBD_E_UNSUPPORTED;
+    } else if (l.kind == MBD_CONV3X3) {
+      if (l.kh != 3 || l.kw != 3 || l.C_in != 64 || l.C_out != 64 || dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
+      if (l.split != MBD_SPLIT_DOMAIN) return MBD_E_UNSUPPORTED;
+      if (P_c != 1) return MBD_E_GRID;
+      if (l.H < 1 || l.W < 1 || P_r > l.H) return MBD_E_GRID;   // a strip needs >= 1 row (halo = 1)
+      if (i > 0 && (l.H != layers[0].H || l.W != layers[0].W)) return MBD_E_INVALID;
+    } else {
+      return MBD_E_INVALID;
+    }
+  }
+  if (is_conv && loss != MBD_LOSS_HALF_SSQ) return MBD_E_UNSUPPORTED;
+  if (!is_conv && loss != MBD_LOSS_SOFTMAX_CE) return MBD_E_UNSUPPORTED;
+
+  mbd_net* n = new (std::nothrow) mbd_net();
+  if (!n) return MBD_E_ALLOC;
+  n->L = L; n->B = B; n->P_r = P_r; n->P_c = P_c; n->dtype = dtype; n->loss = loss;
+  n->max_partials = max_partials == 0 ? 4 : max_partials;
+  n->stream = static_cast<cudaStream_t>(cuda_stream);
+  n->is_conv = is_conv;
+  mbd_status st = MBD_OK;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&n->device) != cudaSuccess || cudaGetDeviceProperties(&prop, n->device) != cudaSuccess) {
+    (void)cudaGetLastError();
+    delete n;
+    return MBD_E_CUDA;
+  }
+  n->num_sms = prop.multiProcessorCount;
+  if (dtype == MBD_BF16 && prop.major != 10) {   // tcgen05 kernels need compute capability 10.x
+    delete n;
+    return MBD_E_UNSUPPORTED;
+  }
+
+#define ALLOC(ptr, bytes)                                                   \
+  do {                                                                      \
+    st = dev_alloc(reinterpret_cast<void**>(&(ptr)), (bytes));              \
+    if (st != MBD_OK) { free_net(n); return st; }                           \
+  } while (0)
+
+  ALLOC(n->status, sizeof(int));
+  ALLOC(n->loss_dev, sizeof(float));
+  if (cudaMemsetAsync(n->status, 0, sizeof(int), n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
+
+  if (is_conv) {
+    st = conv_create(layers, L, B, P_r, n->max_partials, n->num_sms, n->status, n->stream, &n->conv);
+    if (st != MBD_OK) { free_net(n); return st; }
+    *out = n;
+    return MBD_OK;
+  }
+
+  const size_t es = n->elt();
+  const int S_r = splits_for(P_r, n->max_partials), S_c = splits_for(P_c, n->max_partials);
+  n->layers.resize(L);
+  size_t part_elems = 0, max_d = 0;
+  for (int i = 0; i < L; ++i) {
+    Layer& l = n->layers[i];
+    l.spec = layers[i];
+    l.d_in = layers[i].d_in; l.d_out = layers[i].d_out; l.nW = l.d_in * l.d_out;
+    ALLOC(l.W, l.nW * es);
+    ALLOC(l.dW, l.nW * sizeof(float));
+    if (l.spec.bias) {
+      ALLOC(l.bias, l.d_out * sizeof(float));
+      ALLOC(l.db, l.d_out * sizeof(float));
+      if (cudaMemsetAsync(l.bias, 0, l.d_out * sizeof(float), n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
+    }
+    const bool last = i == L - 1;
+    ALLOC(l.act, static_cast<size_t>(B) * l.d_out * (last ? sizeof(float) : es));
+    ALLOC(l.dY, static_cast<size_t>(B) * l.d_out * es);
+    if (cudaMemsetAsync(l.W, 0, l.nW * es, n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
+    if (S_c > 1) part_elems = std::max(part_elems, static_cast<size_t>(S_c) * l.nW);
+    if (i > 0 && S_r > 1) part_elems = std::max(part_elems, static_cast<size_t>(S_r) * B * l.d_in);
+    max_d = std::max(max_d, static_cast<size_t>(l.d_out));
+  }
+  n->partial_elems = part_elems;
+  if (part_elems) ALLOC(n->partials, part_elems * sizeof(float));
+  ALLOC(n->colsum_scratch, static_cast<size_t>(colsum_row_splits(B)) * max_d * sizeof(float));
+  ALLOC(n->per_sample, B * sizeof(float));
+#undef ALLOC
+
+  if (dtype == MBD_BF16) {
+    for (int i = 0; i < L; ++i) {
+      Layer& l = n->layers[i];
+      if (i > 0) {
+        st = prepare_tc(n, l.fwd, 0, B, l.d_out, l.d_in, n->layers[i - 1].act, l.d_in, l.W, l.d_in, 1);
+        if (st == MBD_OK) st = prepare_tc(n, l.bwd_data, 1, B, l.d_in, l.d_out, l.dY, l.d_out, l.W, l.d_in, S_r);
+        if (st == MBD_OK) st = prepare_tc(n, l.bwd_weight, 2, l.d_out, l.d_in, B, l.dY, l.d_out, n->layers[i - 1].act, l.d_in, S_c);
+        if (st != MBD_OK) { free_net(n); return st; }
+      }
+    }
+  }
+  if (cudaStreamSynchronize(n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
+  *out = n;
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_net_destroy(mbd_net* n) {
+  if (!n) return MBD_E_INVALID;
+  cudaStreamSynchronize(n->stream);
+  free_net(n);
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_set_weights(mbd_net* n, int layer, const void* W_dev, const float* bias_dev) {
+  if (!n || !W_dev || layer < 0 || layer >= n->L) return MBD_E_INVALID;
+  if (n->is_conv) return conv_set_weights(n->conv, layer, W_dev);
+  Layer& l = n->layers[layer];
+  CK(cudaMemcpyAsync(l.W, W_dev, l.nW * n->elt(), cudaMemcpyDeviceToDevice, n->stream));
+  if (bias_dev) {
+    if (!l.bias) return MBD_E_INVALID;
+    CK(cudaMemcpyAsync(l.bias, bias_dev, l.d_out * sizeof(float), cudaMemcpyDeviceToDevice, n->stream));
+  }
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_get_weights(mbd_net* n, int layer, void* W_dev, float* bias_dev) {
+  if (!n || !W_dev || layer < 0 || layer >= n->L) return MBD_E_INVALID;
+  if (n->is_conv) return conv_get_weights(n->conv, layer, W_dev);
+  Layer& l = n->layers[layer];
+  CK(cudaMemcpyAsync(W_dev, l.W, l.nW * n->elt(), cudaMemcpyDeviceToDevice, n->stream));
+  if (bias_dev) {
+    if (!l.bias) return MBD_E_INVALID;
+    CK(cudaMemcpyAsync(bias_dev, l.bias, l.d_out * sizeof(float), cudaMemcpyDeviceToDevice, n->stream));
+  }
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_forward(mbd_net* n, const void* X_dev, const int32_t* labels_dev, float* loss_sum_dev) {
+  if (!n || !X_dev) return MBD_E_INVALID;
+  if (n->is_conv) {
+    mbd_status s = conv_forward(n->conv, X_dev, loss_sum_dev, &n->launches);
+    if (s == MBD_OK) n->state = ST_FWD;
+    return s;
+  }
+  if (!labels_dev) return MBD_E_INVALID;
+  n->X = X_dev;
+  n->labels = labels_dev;
+  mbd_status s = map_input(n);
+  if (s != MBD_OK) return s;
+  const int bf = n->dtype == MBD_BF16;
+  for (int i = 0; i < n->L; ++i) {
+    Layer& l = n->layers[i];
+    const bool last = i == n->L - 1;
+    const Epi e = epi_act(l.act, l.d_out, last ? 0 : bf, l.bias, (!last && l.spec.relu) ? 1 : 0);
+    s = run_gemm(n, l.fwd, 0, n->B, l.d_out, l.d_in, layer_input(n, i), l.d_in, l.W, l.d_in, 1, e);
+    if (s != MBD_OK) return s;
+  }
+  Layer& top = n->layers[n->L - 1];
+  CK(softmax_xent_launch(static_cast<const float*>(top.act), n->B, top.d_out, labels_dev, top.dY, bf, n->per_sample, n->stream));
+  n->launches++;
+  if (loss_sum_dev) {
+    CK(sum_f32_launch(n->per_sample, n->B, 1.f, loss_sum_dev, n->stream));
+    n->launches++;
+  }
+  n->state = ST_FWD;
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
+  if (!n || fused_eta < 0.f) return MBD_E_INVALID;
+  if (n->state != ST_FWD) return MBD_E_STATE;
+  if (n->is_conv) {
+    mbd_status s = conv_backward(n->conv, fused_eta, &n->launches);
+    if (s == MBD_OK) n->state = fused_eta > 0.f ? ST_BWD_FUSED : ST_BWD_UNFUSED;
+    return s;
+  }
+  const int bf = n->dtype == MBD_BF16;
+  const bool fused = fused_eta > 0.f;
+  const float scale = -fused_eta / static_cast<float>(n->B);
+  const int S_r = splits_for(n->P_r, n->max_partials), S_c = splits_for(n->P_c, n->max_partials);
+  for (int i = n->L - 1; i >= 0; --i) {
+    Layer& l = n->layers[i];
+    if (l.bias) {
+      CK(colsum_launch(l.dY, bf, n->B, l.d_out, n->colsum_scratch, colsum_row_splits(n->B), fused ? nullptr : l.db,
+                       fused ? l.bias : nullptr, scale, n->stream));
+      n->launches += 2;
+    }
+    if (i > 0) {   // nothing is propagated below the first layer
+      Layer& prev = n->layers[i - 1];
+      const Epi e = epi_mask(prev.dY, l.d_in, bf, prev.spec.relu ? prev.act : nullptr, l.d_in);
+      mbd_status s = run_gemm(n, l.bwd_data, 1, n->B, l.d_in, l.d_out, l.dY, l.d_out, l.W, l.d_in, S_r, e);
+      if (s != MBD_OK) return s;
+    }
+    const Epi e = fused ? epi_sgd(l.W, l.d_in, bf, scale) : epi_act(l.dW, l.d_in, 0, nullptr, 0);
+    mbd_status s = run_gemm(n, l.bwd_weight, 2, l.d_out, l.d_in, n->B, l.dY, l.d_out, layer_input(n, i), l.d_in, S_c, e);
+    if (s != MBD_OK) return s;
+  }
+  n->state = fused ? ST_BWD_FUSED : ST_BWD_UNFUSED;
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_sgd_step(mbd_net* n, float eta) {
+  if (!n || eta < 0.f) return MBD_E_INVALID;
+  if (n->state != ST_BWD_UNFUSED) return MBD_E_STATE;
+  if (n->is_conv) {
+    mbd_status s = conv_sgd_step(n->conv, eta, &n->launches);
+    if (s == MBD_OK) n->state = ST_IDLE;
+    return s;
+  }
+  const float scale = -eta / static_cast<float>(n->B);
+  for (int i = 0; i < n->L; ++i) {
+    Layer& l = n->layers[i];
+    CK(sgd_update_launch(l.W, n->dtype == MBD_BF16, l.dW, l.nW, scale, n->num_sms, n->stream));
+    n->launches++;
+    if (l.bias) {
+      CK(sgd_update_launch(l.bias, 0, l.db, l.d_out, scale, n->num_sms, n->stream));
+      n->launches++;
+    }
+  }
+  n->state = ST_IDLE;
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_train_step_host(mbd_net* n, const void* X_host, const int32_t* labels_host, float eta,
+                                          float* loss_host) {
+  if (!n || !X_host || !loss_host || eta <= 0.f) return MBD_E_INVALID;
+  size_t x_bytes;
+  if (n->is_conv) x_bytes = conv_input_bytes(n->conv);
+  else x_bytes = static_cast<size_t>(n->B) * n->layers[0].d_in * n->elt();
+  if (!n->X_stage) {
+    mbd_status s = dev_alloc(&n->X_stage, x_bytes);
+    if (s != MBD_OK) return s;
+    s = dev_alloc(reinterpret_cast<void**>(&n->labels_stage), n->B * sizeof(int32_t));
+    if (s != MBD_OK) return s;
+  }
+  CK(cudaMemcpyAsync(n->X_stage, X_host, x_bytes, cudaMemcpyHostToDevice, n->stream));
+  if (!n->is_conv) {
+    if (!labels_host) return MBD_E_INVALID;
+    CK(cudaMemcpyAsync(n->labels_stage, labels_host, n->B * sizeof(int32_t), cudaMemcpyHostToDevice, n->stream));
+  }
+  mbd_status s = mbd_forward(n, n->X_stage, n->labels_stage, n->loss_dev);
+  if (s != MBD_OK) return s;
+  s = mbd_backward(n, eta);
+  if (s != MBD_OK) return s;
+  CK(cudaMemcpyAsync(loss_host, n->loss_dev, sizeof(float), cudaMemcpyDeviceToHost, n->stream));
+  CK(cudaStreamSynchronize(n->stream));
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_get_tensor(mbd_net* n, int which, int layer, void* dst, size_t bytes) {
+  if (!n || !dst) return MBD_E_INVALID;
+  if (n->is_conv) return conv_get_tensor(n->conv, which, layer, dst, bytes);
+  const void* src = nullptr;
+  size_t size = 0;
+  if (which == MBD_T_LOSS) {
+    src = n->per_sample; size = n->B * sizeof(float);
+  } else if (which == MBD_T_PARTIALS) {
+    src = n->partials; size = bytes;
+    if (bytes > n->partial_elems * sizeof(float)) return MBD_E_INVALID;
+  } else {
+    if (layer < 0 || layer >= n->L) return MBD_E_INVALID;
+    Layer& l = n->layers[layer];
+    const bool last = layer == n->L - 1;
+    switch (which) {
+      case MBD_T_ACT: src = l.act; size = static_cast<size_t>(n->B) * l.d_out * (last ? sizeof(float) : n->elt()); break;
+      case MBD_T_DY: src = l.dY; size = static_cast<size_t>(n->B) * l.d_out * n->elt(); break;
+      case MBD_T_DW: src = l.dW; size = l.nW * sizeof(float); break;
+      case MBD_T_DB: src = l.db; size = l.d_out * sizeof(float); break;
+      default: return MBD_E_INVALID;
+    }
+  }
+  if (!src || bytes != size) return MBD_E_INVALID;
+  CK(cudaMemcpyAsync(dst, src, size, cudaMemcpyDeviceToDevice, n->stream));
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_poll_status(mbd_net* n) {
+  if (!n) return MBD_E_INVALID;
+  CK(cudaStreamSynchronize(n->stream));
+  int h = 0;
+  CK(cudaMemcpy(&h, n->status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (h != 0) {
+    CK(cudaMemset(n->status, 0, sizeof(int)));
+    return MBD_E_TIMEOUT;
+  }
+  return MBD_OK;
+}
+
+extern "C" int64_t mbd_launch_count(const mbd_net* n) { return n ? n->launches : -1; }
+
+extern "C" mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                    const void* Bm, int64_t ldb, float* D, int64_t ldd, int k_splits, float* partials,
+                                    void* cuda_stream) {
+  if (!A || !Bm || !D || variant < 0 || variant > 2 || M < 1 || N < 1 || K < 1 || k_splits < 1) return MBD_E_INVALID;
+  if (lda % 8 || ldb % 8 || ldd % 8 || N % 8) return MBD_E_UNSUPPORTED;
+  if (k_splits > 1 && !partials) return MBD_E_INVALID;
+  if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return MBD_E_UNSUPPORTED;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int dev = 0, sms = 0;
+  CK(cudaGetDevice(&dev));
+  CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  int* status = nullptr;
+  if (dev_alloc(reinterpret_cast<void**>(&status), sizeof(int)) != MBD_OK) return MBD_E_ALLOC;
+  cudaMemsetAsync(status, 0, sizeof(int), stream);
+  TcGemm g{};
+  g.variant = variant;
+  g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
+  g.k_splits = k_splits;
+  g.status = status;
+  mbd_status ret = MBD_OK;
+  do {
+    if (tc_gemm_prepare(g, A, lda, Bm, ldb, sms) != cudaSuccess) { ret = MBD_E_CUDA; break; }
+    g.epi = epi_act(D, ldd, 0, nullptr, 0);
+    g.partials = partials;
+    if (tc_gemm_launch(g, stream) != cudaSuccess) { ret = MBD_E_CUDA; break; }
+    if (g.k_splits > 1 && reduce_partials_launch(partials, g.k_splits, M, N, g.epi, sms, stream) != cudaSuccess) { ret = MBD_E_CUDA; break; }
+    if (cudaStreamSynchronize(stream) != cudaSuccess) { ret = MBD_E_CUDA; break; }
+    int h = 0;
+    if (cudaMemcpy(&h, status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { ret = MBD_E_CUDA; break; }
+    if (h != 0) ret = MBD_E_TIMEOUT;
+  } while (0);
+  (void)cudaGetLastError();
+  cudaFree(status);
+  return ret;
+}

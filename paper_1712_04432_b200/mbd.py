@@ -1,0 +1,236 @@
+"""Thin ctypes binding of libmbd.so: argument marshalling only.
+
+Every step of the training path runs inside the CUDA library; torch is used
+here for device memory and streams.  Loading fails loudly when the library has
+not been built (`python -m paper_1712_04432_b200.build`); there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmbd.so")
+
+OK, E_INVALID, E_GRID, E_ALLOC, E_CUDA, E_STATE, E_TIMEOUT, E_UNSUPPORTED = range(8)
+FC, CONV3X3 = 0, 1
+SPLIT_MODEL, SPLIT_DOMAIN = 0, 1
+F32, BF16 = 0, 1
+LOSS_SOFTMAX_CE, LOSS_HALF_SSQ = 0, 1
+T_ACT, T_DY, T_DW, T_DB, T_LOSS, T_PARTIALS = range(6)
+
+EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weights", "mbd_forward",
+           "mbd_backward", "mbd_sgd_step", "mbd_train_step_host", "mbd_comm_words", "mbd_get_tensor",
+           "mbd_poll_status", "mbd_launch_count", "mbd_gemm_bf16", "mbd_strerror"]
+
+
+class MbdError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({strerror(status)})")
+
+
+class Layer(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("split", C.c_int32), ("relu", C.c_int32), ("bias", C.c_int32),
+                ("d_in", C.c_int64), ("d_out", C.c_int64),
+                ("C_in", C.c_int32), ("C_out", C.c_int32), ("H", C.c_int32), ("W", C.c_int32),
+                ("kh", C.c_int32), ("kw", C.c_int32)]
+
+
+class Words(C.Structure):
+    _fields_ = [("allgather_y", C.c_int64), ("allreduce_dx", C.c_int64), ("allreduce_dw", C.c_int64),
+                ("halo_fwd", C.c_int64), ("halo_bwd", C.c_int64)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library; raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_1712_04432_b200.build` "
+                              "(there is no CPU or PyTorch fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, f32 = C.c_void_p, C.c_int, C.c_int64, C.c_float
+        L.mbd_net_create.argtypes = [C.POINTER(Layer), i32, i64, i32, i32, i32, i32, i32, vp, C.POINTER(vp)]
+        L.mbd_net_destroy.argtypes = [vp]
+        L.mbd_set_weights.argtypes = [vp, i32, vp, vp]
+        L.mbd_get_weights.argtypes = [vp, i32, vp, vp]
+        L.mbd_forward.argtypes = [vp, vp, vp, vp]
+        L.mbd_backward.argtypes = [vp, f32]
+        L.mbd_sgd_step.argtypes = [vp, f32]
+        L.mbd_train_step_host.argtypes = [vp, vp, vp, f32, C.POINTER(f32)]
+        L.mbd_comm_words.argtypes = [C.POINTER(Layer), i32, i64, i32, i32, C.POINTER(Words)]
+        L.mbd_get_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
+        L.mbd_poll_status.argtypes = [vp]
+        L.mbd_launch_count.argtypes = [vp]
+        L.mbd_launch_count.restype = i64
+        L.mbd_gemm_bf16.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp, vp]
+        L.mbd_strerror.argtypes = [i32]
+        L.mbd_strerror.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def strerror(status: int) -> str:
+    return lib().mbd_strerror(int(status)).decode()
+
+
+def _check(status: int, what: str):
+    if status != OK:
+        raise MbdError(status, what)
+
+
+def fc_layers(dims: Sequence[int], bias: bool = True, relu: bool = True) -> List[Layer]:
+    """Layer table of a fully connected stack d_0 -> ... -> d_L (model-split)."""
+    return [Layer(kind=FC, split=SPLIT_MODEL, relu=int(relu), bias=int(bias), d_in=int(dims[i - 1]),
+                  d_out=int(dims[i])) for i in range(1, len(dims))]
+
+
+def conv_layers(n: int, C_: int, H: int, W: int, relu: bool = True) -> List[Layer]:
+    """n domain-split 3x3 convolution layers C -> C on H x W images."""
+    return [Layer(kind=CONV3X3, split=SPLIT_DOMAIN, relu=int(relu), bias=0, d_in=C_ * H * W, d_out=C_ * H * W,
+                  C_in=C_, C_out=C_, H=H, W=W, kh=3, kw=3) for _ in range(n)]
+
+
+def _layer_array(layers: Sequence[Layer]):
+    arr = (Layer * len(layers))()
+    for i, l in enumerate(layers):
+        arr[i] = l
+    return arr
+
+
+def comm_words(layers: Sequence[Layer], B: int, P_r: int, P_c: int) -> List[Dict[str, int]]:
+    """mbd_comm_words: per-layer word counts of Eq. 8 / Eq. 9 (host only, no GPU)."""
+    out = (Words * len(layers))()
+    _check(lib().mbd_comm_words(_layer_array(layers), len(layers), int(B), int(P_r), int(P_c), out), "mbd_comm_words")
+    return [{k: int(getattr(w, k)) for k, _ in Words._fields_} for w in out]
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+class Net:
+    """One network on the current CUDA device (see include/mbd.h for semantics)."""
+
+    def __init__(self, layers: Sequence[Layer], B: int, P_r: int = 1, P_c: int = 1, dtype: int = BF16,
+                 loss: int = LOSS_SOFTMAX_CE, max_partials: int = 0, stream=None):
+        import torch
+        self._torch = torch
+        self.layers = list(layers)
+        self.L, self.B, self.P_r, self.P_c, self.dtype, self.loss = len(layers), int(B), P_r, P_c, dtype, loss
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        self._h = C.c_void_p()
+        self._keep = []
+        _check(lib().mbd_net_create(_layer_array(layers), self.L, self.B, P_r, P_c, dtype, loss, max_partials,
+                                    C.c_void_p(self.stream.cuda_stream), C.byref(self._h)), "mbd_net_create")
+
+    # -- helpers
+    @property
+    def act_dtype(self):
+        return self._torch.bfloat16 if self.dtype == BF16 else self._torch.float32
+
+    def _wshape(self, i):
+        l = self.layers[i]
+        return (l.C_out, l.C_in, 3, 3) if l.kind == CONV3X3 else (l.d_out, l.d_in)
+
+    def close(self):
+        if self._h:
+            lib().mbd_net_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- C ABI calls
+    def set_weights(self, i: int, W, bias=None):
+        assert W.is_cuda and W.is_contiguous() and W.dtype == self.act_dtype and tuple(W.shape) == self._wshape(i)
+        if bias is not None:
+            assert bias.is_cuda and bias.dtype == self._torch.float32 and bias.is_contiguous()
+        _check(lib().mbd_set_weights(self._h, i, _ptr(W), _ptr(bias)), "mbd_set_weights")
+
+    def get_weights(self, i: int, with_bias: bool = False):
+        t = self._torch
+        W = t.empty(self._wshape(i), dtype=self.act_dtype, device="cuda")
+        b = t.empty(self.layers[i].d_out, dtype=t.float32, device="cuda") if with_bias else None
+        _check(lib().mbd_get_weights(self._h, i, _ptr(W), _ptr(b)), "mbd_get_weights")
+        return (W, b) if with_bias else W
+
+    def forward(self, X, labels=None, loss_out=None):
+        assert X.is_cuda and X.is_contiguous() and X.dtype == self.act_dtype
+        if labels is not None:
+            assert labels.is_cuda and labels.dtype == self._torch.int32 and labels.is_contiguous()
+        self._keep = [X, labels, loss_out]      # the library reads X again during backward
+        _check(lib().mbd_forward(self._h, _ptr(X), _ptr(labels), _ptr(loss_out)), "mbd_forward")
+
+    def backward(self, fused_eta: float = 0.0):
+        _check(lib().mbd_backward(self._h, float(fused_eta)), "mbd_backward")
+
+    def sgd_step(self, eta: float):
+        _check(lib().mbd_sgd_step(self._h, float(eta)), "mbd_sgd_step")
+
+    def train_step_host(self, X_host, labels_host, eta: float) -> float:
+        """One step from host (ideally pinned) tensors; returns J."""
+        assert not X_host.is_cuda and X_host.is_contiguous()
+        out = C.c_float(0.0)
+        _check(lib().mbd_train_step_host(self._h, _ptr(X_host), _ptr(labels_host), float(eta), C.byref(out)),
+               "mbd_train_step_host")
+        return out.value
+
+    def get_tensor(self, which: int, layer: int = 0, numel: Optional[int] = None):
+        t = self._torch
+        l = self.layers[min(layer, self.L - 1)]
+        last = layer == self.L - 1
+        conv = l.kind == CONV3X3
+        if which == T_ACT:
+            shape, dt = ((self.B, l.C_out, l.H, l.W) if conv else (self.B, l.d_out)), \
+                (t.float32 if (last and not conv) else self.act_dtype)
+        elif which == T_DY:
+            shape, dt = ((self.B, l.C_out, l.H, l.W) if conv else (self.B, l.d_out)), self.act_dtype
+        elif which == T_DW:
+            shape, dt = self._wshape(layer), t.float32
+        elif which == T_DB:
+            shape, dt = (l.d_out,), t.float32
+        elif which == T_LOSS:
+            shape, dt = (self.B,), t.float32
+        elif which == T_PARTIALS:
+            shape, dt = (int(numel),), t.float32
+        else:
+            raise ValueError(which)
+        out = t.empty(shape, dtype=dt, device="cuda")
+        _check(lib().mbd_get_tensor(self._h, which, layer, _ptr(out), out.numel() * out.element_size()), "mbd_get_tensor")
+        return out
+
+    def poll(self):
+        _check(lib().mbd_poll_status(self._h), "mbd_poll_status")
+
+    @property
+    def launch_count(self) -> int:
+        return int(lib().mbd_launch_count(self._h))
+
+
+def gemm_bf16(variant: int, A, B, k_splits: int = 1, return_partials: bool = False):
+    """mbd_gemm_bf16 on torch bf16 CUDA tensors.
+    variant 0: A[M,K], B[N,K];  1: A[M,K], B[K,N];  2: A[K,M], B[K,N].  Returns float D[M,N]."""
+    import torch
+    assert A.is_cuda and B.is_cuda and A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16
+    assert A.stride(1) == 1 and B.stride(1) == 1
+    if variant == 0:
+        M, K = A.shape; N = B.shape[0]; assert B.shape[1] == K
+    elif variant == 1:
+        M, K = A.shape; N = B.shape[1]; assert B.shape[0] == K
+    else:
+        K, M = A.shape; N = B.shape[1]; assert B.shape[0] == K
+    D = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    parts = torch.empty((k_splits, M, N), dtype=torch.float32, device="cuda") if k_splits > 1 else None
+    st = lib().mbd_gemm_bf16(variant, M, N, K, _ptr(A), A.stride(0), _ptr(B), B.stride(0), _ptr(D), D.stride(0),
+                             k_splits, _ptr(parts), C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    _check(st, "mbd_gemm_bf16")
+    return (D, parts) if return_partials else D
