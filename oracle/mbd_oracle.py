@@ -160,9 +160,19 @@ def _batch_of(X):
     return X.shape[1] if X.ndim == 2 else X.shape[0]
 
 
-def forward(layers: Sequence, X1):
+def _stored(A, store):
+    return A if store is None else np.asarray(store(A), F64)
+
+
+def forward(layers: Sequence, X1, store=None):
     """Returns (Xs, Ys): Xs[i] is the input of layer i (0-based), Ys[i] its
-    affine output before the nonlinearity."""
+    affine output before the nonlinearity.
+
+    `store`, if given, is applied to every activation X_{i+1} = f(Y_i) that is
+    kept for the next layer.  It models the storage type of the activations
+    (e.g. rounding to bfloat16): the ReLU decision [Y_i > 0] of the layers
+    above is a discrete decision, so it has to be taken on the same stored
+    values on both sides of a comparison.  The arithmetic stays fp64."""
     Xs: List[np.ndarray] = [np.asarray(X1, F64)]
     Ys: List[np.ndarray] = []
     for i, lay in enumerate(layers):
@@ -172,7 +182,7 @@ def forward(layers: Sequence, X1):
             Y = conv3x3(lay.K, Xs[i])
         Ys.append(Y)
         if i + 1 < len(layers):
-            Xs.append(relu(Y) if lay.relu else Y)
+            Xs.append(_stored(relu(Y) if lay.relu else Y, store))
     return Xs, Ys
 
 
@@ -186,12 +196,12 @@ def loss_and_top_grad(Y_L, loss: str, labels=None):
     raise ValueError(loss)
 
 
-def train_step(layers: Sequence, X1, labels, loss: str, eta: float):
-    """One full step.  Returns a dict with
+def train_step(layers: Sequence, X1, labels, loss: str, eta: float, store=None):
+    """One full step (`store`: see `forward`).  Returns a dict with
        Xs, Ys, J, per_sample, dYs (dJ/dY_i), dXs (dJ/dX_i, None for i=0),
        dWs, dbs, new_W, new_b   (lists indexed by layer, 0-based)."""
     L = len(layers)
-    Xs, Ys = forward(layers, X1)
+    Xs, Ys = forward(layers, X1, store)
     B = _batch_of(Xs[0])
     J, per, dY_top = loss_and_top_grad(Ys[-1], loss, labels)
     dYs = [None] * L
@@ -360,7 +370,7 @@ def conv3x3_dK_strips(dY, X, P_r):
 
 
 def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
-                       P_r: int, P_c: int):
+                       P_r: int, P_c: int, store=None):
     """The step of `train_step`, every contraction formed block by block over
     the P_r x P_c grid and every cross-block sum taken as P separate partials
     added in ascending block index.  FC layers split the model over P_r and the
@@ -377,7 +387,7 @@ def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
             Y = conv3x3_strips(lay.K, Xs[i], P_r)
         Ys.append(Y)
         if i + 1 < L:
-            Xs.append(relu(Y) if lay.relu else Y)
+            Xs.append(_stored(relu(Y) if lay.relu else Y, store))
     B = _batch_of(Xs[0])
     J, per, dY_top = loss_and_top_grad(Ys[-1], loss, labels)
     dYs = [None] * L

@@ -29,3 +29,92 @@ def to_np(t):
     if t.dtype == torch.bfloat16:
         return t.float().cpu().numpy().astype(np.float64)
     return t.cpu().numpy().astype(np.float64)
+
+
+# ---------------------------------------------------------------------------
+# one training step on both sides
+# ---------------------------------------------------------------------------
+def bf16_store(A):
+    """Storage rounding handed to the oracle for bf16 workloads: the kept activations
+    are bfloat16 on the device, and the ReLU decisions above them must see the same
+    stored values on both sides."""
+    return I.round_to_bf16(np.asarray(A, np.float32)).astype(np.float64)
+
+
+def oracle_fc_step(w, inp, blocked_grid=None, exact=False):
+    """fp64 oracle step for a fully connected workload (paper orientation: d x B).
+    bf16 workloads round the STORED activations to bf16 unless `exact`."""
+    from oracle import mbd_oracle as O
+    store = bf16_store if (w.dtype == "bf16" and not exact) else None
+    L = len(inp.Ws)
+    layers = [O.FC(inp.Ws[i].astype(np.float64), None if inp.bs[i] is None else inp.bs[i].astype(np.float64),
+                   relu=True) for i in range(L)]
+    X1 = inp.X.astype(np.float64).T
+    if blocked_grid is None:
+        return O.train_step(layers, X1, inp.labels, "softmax_ce", w.eta, store=store)
+    return O.train_step_blocked(layers, X1, inp.labels, "softmax_ce", w.eta, *blocked_grid, store=store)
+
+
+def gpu_fc_step(w, inp, grid=(1, 1), max_partials=0, fused=False):
+    """The same step through the C ABI.  Returns numpy fp64 arrays in the GPU's
+    [B, d] / [d_out, d_in] layouts."""
+    import torch
+    from paper_1712_04432_b200 import mbd
+    bf = w.dtype == "bf16"
+    L = len(inp.Ws)
+    net = mbd.Net(mbd.fc_layers(w.dims, bias=True), w.B, grid[0], grid[1], mbd.BF16 if bf else mbd.F32,
+                  mbd.LOSS_SOFTMAX_CE, max_partials)
+    for i in range(L):
+        net.set_weights(i, to_dev(inp.Ws[i], bf), torch.from_numpy(inp.bs[i]).cuda())
+    X = to_dev(inp.X, bf)
+    labels = torch.from_numpy(inp.labels).cuda()
+    J = torch.zeros(1, dtype=torch.float32, device="cuda")
+    out = {}
+    net.forward(X, labels, J)
+    if fused:
+        net.backward(w.eta)
+    else:
+        net.backward(0.0)
+        out["dW"] = [to_np(net.get_tensor(mbd.T_DW, i)) for i in range(L)]
+        out["db"] = [to_np(net.get_tensor(mbd.T_DB, i)) for i in range(L)]
+        net.sgd_step(w.eta)
+    net.poll()
+    out["J"] = float(J.item())
+    out["loss"] = to_np(net.get_tensor(mbd.T_LOSS))
+    out["act"] = [to_np(net.get_tensor(mbd.T_ACT, i)) for i in range(L)]
+    out["dY"] = [to_np(net.get_tensor(mbd.T_DY, i)) for i in range(L)]
+    nw = [net.get_weights(i, with_bias=True) for i in range(L)]
+    out["new_W"] = [to_np(a) for a, _ in nw]
+    out["new_b"] = [to_np(b) for _, b in nw]
+    out["launches"] = net.launch_count
+    net.close()
+    return out
+
+
+def compare_fc_step(g, o, tol, fused=False):
+    """Element-by-element comparison, tensor by tensor; returns the worst relative
+    Frobenius error and raises on the first tensor beyond `tol`."""
+    L = len(o["Ys"])
+    worst = 0.0
+    report = []
+
+    def chk(name, got, ref):
+        nonlocal worst
+        e = rel_fro(got, ref)
+        worst = max(worst, e)
+        report.append(f"{name}: {e:.3e}")
+
+    assert abs(g["J"] - o["J"]) <= max(tol, 1e-4) * abs(o["J"]), (g["J"], o["J"])
+    chk("per-sample loss", g["loss"], o["per_sample"])
+    for i in range(L):
+        ref_act = o["Ys"][i] if i == L - 1 else o["Xs"][i + 1]
+        chk(f"Y[{i}]", g["act"][i], ref_act.T)
+        chk(f"dY[{i}]", g["dY"][i], o["dYs"][i].T)        # for i < L-1 this is dX_{i+1} after the mask
+        if not fused:
+            chk(f"dW[{i}]", g["dW"][i], o["dWs"][i])
+            chk(f"db[{i}]", g["db"][i], o["dbs"][i])
+        chk(f"W_new[{i}]", g["new_W"][i], o["new_W"][i])
+        ref_b = o["new_b"][i]
+        assert np.abs(g["new_b"][i] - ref_b).max() <= tol * max(1.0, np.abs(ref_b).max()), f"b_new[{i}]"
+    assert worst <= tol, "rel. Frobenius errors beyond %.1e: %s" % (tol, "; ".join(report))
+    return worst

@@ -360,3 +360,19 @@ def test_half_ssq():
     Y = np.array([[1.0, -2.0], [3.0, 0.5]])
     J, dY = O.half_ssq(Y)
     assert J == 0.5 * (1 + 4 + 9 + 0.25) and np.array_equal(dY, Y)
+
+
+def test_storage_rounding_only_touches_kept_activations():
+    # `store` models the activation storage type: identity leaves the step unchanged, and a
+    # coarse rounding changes exactly what the next layer reads (X_{i+1}), not Y_i itself
+    layers, X, labels = tiny_mlp(seed=60)
+    a = O.train_step(layers, X, labels, "softmax_ce", 0.01)
+    b = O.train_step(layers, X, labels, "softmax_ce", 0.01, store=lambda A: A)
+    assert all(np.array_equal(x, y) for x, y in zip(a["dWs"], b["dWs"]))
+    q = lambda A: np.round(A * 8) / 8
+    c = O.train_step(layers, X, labels, "softmax_ce", 0.01, store=q)
+    assert np.array_equal(c["Ys"][0], a["Ys"][0])
+    assert np.array_equal(c["Xs"][1], q(np.maximum(a["Ys"][0], 0)))
+    assert np.array_equal(c["Ys"][1], O.affine(layers[1].W, c["Xs"][1], layers[1].b))
+    d = O.train_step_blocked(layers, X, labels, "softmax_ce", 0.01, 2, 2, store=q)
+    assert all(relerr(x, y) < 1e-12 for x, y in zip(c["dWs"], d["dWs"]))

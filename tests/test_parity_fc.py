@@ -1,0 +1,115 @@
+"""Parity of the fully connected training step with the fp64 oracle, element by
+element, through the C ABI: every tensor of every layer, for the grids of the
+workloads, materialised and chained partial sums, fused and un-fused update."""
+import numpy as np
+import pytest
+
+from paper_1712_04432_b200 import inputs as I
+from tests.helpers import compare_fc_step, gpu_fc_step, oracle_fc_step, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-5     # fp32 check mode
+TOL_BF16 = 1e-2    # bf16 storage, fp32 accumulation
+
+
+@pytest.fixture(scope="module")
+def cfg1():
+    w = I.WORKLOADS["cfg1"]
+    inp = I.make_inputs(w, seed=0)
+    return w, inp, oracle_fc_step(w, inp)
+
+
+@pytest.mark.parametrize("grid", [(1, 1), (2, 2), (4, 1), (1, 4)])
+@pytest.mark.parametrize("fused", [False, True])
+def test_cfg1_fp32_all_grids(cfg1, grid, fused):
+    w, inp, o = cfg1
+    g = gpu_fc_step(w, inp, grid, max_partials=64, fused=fused)   # every block's partial materialised
+    compare_fc_step(g, o, TOL_F32, fused)
+    if not fused:
+        # the update itself, not just the updated weights
+        for i in range(3):
+            delta = (g["new_W"][i] - inp.Ws[i].astype(np.float64)) / (-w.eta / w.B)
+            assert rel_fro(delta, o["dWs"][i]) < 2e-3
+
+
+def test_cfg1_same_result_for_every_grid_and_chaining(cfg1):
+    w, inp, o = cfg1
+    ref = gpu_fc_step(w, inp, (1, 1))
+    for grid, mp in [((2, 2), 1), ((4, 1), 2), ((1, 4), 4), ((4, 4), 64)]:
+        g = gpu_fc_step(w, inp, grid, max_partials=mp)
+        for i in range(3):
+            assert rel_fro(g["dW"][i], ref["dW"][i]) < 1e-6
+            assert rel_fro(g["new_W"][i], ref["new_W"][i]) < 1e-6
+
+
+@pytest.fixture(scope="module")
+def small_bf16():
+    # several 128x256 tiles with ragged edges in every dimension, K tails that are not
+    # multiples of 64, a 1000-wide classifier like the large workloads
+    w = I.fc_workload((1160, 520, 392, 1000), 328, "bf16", "relu_normal", name="small_bf16")
+    inp = I.make_inputs(w, seed=3)
+    return w, inp, oracle_fc_step(w, inp)
+
+
+@pytest.mark.parametrize("grid,mp", [((1, 1), 0), ((8, 1), 8), ((1, 8), 8), ((2, 4), 4), ((4, 2), 1), ((16, 16), 2),
+                                     ((3, 5), 8)])
+@pytest.mark.parametrize("fused", [False, True])
+def test_small_bf16_grids(small_bf16, grid, mp, fused):
+    w, inp, o = small_bf16
+    g = gpu_fc_step(w, inp, grid, max_partials=mp, fused=fused)
+    compare_fc_step(g, o, TOL_BF16, fused)
+
+
+def test_small_bf16_against_unrounded_oracle(small_bf16):
+    # Against the oracle WITHOUT storage rounding the forward pass (continuous in its inputs)
+    # still meets the tolerance.  The gradients below a ReLU do not have to: a bf16 rounding
+    # of X_i moves a few Y_i across zero, each flip changes one element of the mask by its
+    # full size, and a fraction f of flipped elements costs about sqrt(f) in Frobenius norm.
+    w, inp, _ = small_bf16
+    o = oracle_fc_step(w, inp, exact=True)
+    g = gpu_fc_step(w, inp, (1, 1))
+    for i in range(3):
+        ref = o["Ys"][i] if i == 2 else o["Xs"][i + 1]
+        assert rel_fro(g["act"][i], ref.T) < TOL_BF16
+    assert rel_fro(g["dY"][2], o["dYs"][2].T) < TOL_BF16       # top gradient: no mask above it
+    assert rel_fro(g["dW"][2], o["dWs"][2]) < TOL_BF16
+    for i in range(2):
+        assert rel_fro(g["dW"][i], o["dWs"][i]) < 0.1
+
+
+def test_small_bf16_against_blocked_oracle(small_bf16):
+    # the oracle formed block by block over the same grid (Appendix A.2) agrees as well
+    w, inp, _ = small_bf16
+    ob = oracle_fc_step(w, inp, blocked_grid=(4, 2))
+    g = gpu_fc_step(w, inp, (4, 2), max_partials=8)
+    compare_fc_step(g, ob, TOL_BF16)
+
+
+def test_fp32_mode_on_ragged_shapes():
+    w = I.fc_workload((200, 136, 72, 24), 40, "f32", "normal", name="small_f32")
+    inp = I.make_inputs(w, seed=5)
+    o = oracle_fc_step(w, inp)
+    for grid in [(1, 1), (3, 2), (8, 5)]:
+        compare_fc_step(gpu_fc_step(w, inp, grid, max_partials=64), o, TOL_F32)
+
+
+def test_run_to_run_bitwise_reproducible(small_bf16):
+    w, inp, _ = small_bf16
+    a = gpu_fc_step(w, inp, (4, 4), max_partials=4, fused=True)
+    b = gpu_fc_step(w, inp, (4, 4), max_partials=4, fused=True)
+    for i in range(3):
+        assert np.array_equal(a["new_W"][i], b["new_W"][i])
+        assert np.array_equal(a["dY"][i], b["dY"][i])
+
+
+@pytest.mark.parametrize("name,grid,mp", [("cfg2", (1, 1), 0), ("cfg2", (2, 4), 4), ("cfg2", (8, 1), 8), ("cfg2", (1, 8), 8),
+                                          ("cfg3", (4, 4), 4)])
+def test_full_size_fc_workloads(name, grid, mp):
+    w = I.WORKLOADS[name]
+    inp = I.make_inputs(w, seed=0)
+    o = oracle_fc_step(w, inp)
+    g = gpu_fc_step(w, inp, grid, max_partials=mp)
+    compare_fc_step(g, o, TOL_BF16)
+    gf = gpu_fc_step(w, inp, grid, max_partials=mp, fused=True)
+    compare_fc_step(gf, o, TOL_BF16, fused=True)
