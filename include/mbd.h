@@ -145,6 +145,11 @@ MBD_API mbd_status mbd_comm_words(const mbd_layer* layers_host, int L, int64_t B
 /* Copy an internal tensor to dst_dev; `bytes` must equal the tensor's size. */
 MBD_API mbd_status mbd_get_tensor(mbd_net* net, int which, int layer, void* dst_dev, size_t bytes);
 
+/* Overwrite an internal tensor (MBD_T_ACT or MBD_T_DY) from src_dev, same shapes and types
+ * as mbd_get_tensor.  A test hook: writing the stored activations between mbd_forward and
+ * mbd_backward fixes the ReLU decisions [X_{i+1} > 0] the backward pass will take. */
+MBD_API mbd_status mbd_set_tensor(mbd_net* net, int which, int layer, const void* src_dev, size_t bytes);
+
 /* Waits for the stream and reads the device status word: MBD_OK, or MBD_E_TIMEOUT if
  * a kernel's bounded barrier wait ran out, or MBD_E_CUDA. */
 MBD_API mbd_status mbd_poll_status(mbd_net* net);

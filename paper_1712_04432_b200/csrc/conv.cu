@@ -9,5 +9,6 @@ mbd_status conv_forward(ConvNet*, const void*, float*, int64_t*) { return MBD_E_
 mbd_status conv_backward(ConvNet*, float, int64_t*) { return MBD_E_UNSUPPORTED; }
 mbd_status conv_sgd_step(ConvNet*, float, int64_t*) { return MBD_E_UNSUPPORTED; }
 mbd_status conv_get_tensor(ConvNet*, int, int, void*, size_t) { return MBD_E_UNSUPPORTED; }
+mbd_status conv_set_tensor(ConvNet*, int, int, const void*, size_t) { return MBD_E_UNSUPPORTED; }
 size_t conv_input_bytes(const ConvNet*) { return 0; }
 }  // namespace mbd

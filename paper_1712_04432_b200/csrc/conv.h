@@ -17,5 +17,6 @@ mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev, int
 mbd_status conv_backward(ConvNet* c, float fused_eta, int64_t* launches);
 mbd_status conv_sgd_step(ConvNet* c, float eta, int64_t* launches);
 mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t bytes);
+mbd_status conv_set_tensor(ConvNet* c, int which, int layer, const void* src, size_t bytes);
 size_t conv_input_bytes(const ConvNet* c);
 }  // namespace mbd

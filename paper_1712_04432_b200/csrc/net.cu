@@ -457,6 +457,22 @@ extern "C" mbd_status mbd_get_tensor(mbd_net* n, int which, int layer, void* dst
   return MBD_OK;
 }
 
+extern "C" mbd_status mbd_set_tensor(mbd_net* n, int which, int layer, const void* src, size_t bytes) {
+  if (!n || !src) return MBD_E_INVALID;
+  if (n->is_conv) return conv_set_tensor(n->conv, which, layer, src, bytes);
+  if (layer < 0 || layer >= n->L) return MBD_E_INVALID;
+  Layer& l = n->layers[layer];
+  const bool last = layer == n->L - 1;
+  void* dst = nullptr;
+  size_t size = 0;
+  if (which == MBD_T_ACT) { dst = l.act; size = static_cast<size_t>(n->B) * l.d_out * (last ? sizeof(float) : n->elt()); }
+  else if (which == MBD_T_DY) { dst = l.dY; size = static_cast<size_t>(n->B) * l.d_out * n->elt(); }
+  else return MBD_E_INVALID;
+  if (bytes != size) return MBD_E_INVALID;
+  CK(cudaMemcpyAsync(dst, src, size, cudaMemcpyDeviceToDevice, n->stream));
+  return MBD_OK;
+}
+
 extern "C" mbd_status mbd_poll_status(mbd_net* n) {
   if (!n) return MBD_E_INVALID;
   CK(cudaStreamSynchronize(n->stream));

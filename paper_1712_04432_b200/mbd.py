@@ -22,7 +22,7 @@ T_ACT, T_DY, T_DW, T_DB, T_LOSS, T_PARTIALS = range(6)
 
 EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weights", "mbd_forward",
            "mbd_backward", "mbd_sgd_step", "mbd_train_step_host", "mbd_comm_words", "mbd_get_tensor",
-           "mbd_poll_status", "mbd_launch_count", "mbd_gemm_bf16", "mbd_strerror"]
+           "mbd_set_tensor", "mbd_poll_status", "mbd_launch_count", "mbd_gemm_bf16", "mbd_strerror"]
 
 
 class MbdError(RuntimeError):
@@ -65,6 +65,7 @@ def lib():
         L.mbd_train_step_host.argtypes = [vp, vp, vp, f32, C.POINTER(f32)]
         L.mbd_comm_words.argtypes = [C.POINTER(Layer), i32, i64, i32, i32, C.POINTER(Words)]
         L.mbd_get_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
+        L.mbd_set_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
         L.mbd_poll_status.argtypes = [vp]
         L.mbd_launch_count.argtypes = [vp]
         L.mbd_launch_count.restype = i64
@@ -207,6 +208,10 @@ class Net:
         out = t.empty(shape, dtype=dt, device="cuda")
         _check(lib().mbd_get_tensor(self._h, which, layer, _ptr(out), out.numel() * out.element_size()), "mbd_get_tensor")
         return out
+
+    def set_tensor(self, which: int, layer: int, src):
+        assert src.is_cuda and src.is_contiguous()
+        _check(lib().mbd_set_tensor(self._h, which, layer, _ptr(src), src.numel() * src.element_size()), "mbd_set_tensor")
 
     def poll(self):
         _check(lib().mbd_poll_status(self._h), "mbd_poll_status")

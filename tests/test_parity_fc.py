@@ -5,12 +5,18 @@ import numpy as np
 import pytest
 
 from paper_1712_04432_b200 import inputs as I
-from tests.helpers import compare_fc_step, gpu_fc_step, oracle_fc_step, rel_fro
+from tests.helpers import compare_fc_step, gpu_fc_step, oracle_fc_step, oracle_hidden_acts, rel_fro
 
 pytestmark = pytest.mark.gpu
 
 TOL_F32 = 1e-5     # fp32 check mode
 TOL_BF16 = 1e-2    # bf16 storage, fp32 accumulation
+# Free-running bf16 step, gradients below a ReLU: fp32 (device) and fp64 (oracle) sums round a
+# few stored activations to neighbouring bf16 values, which moves a few pre-activations of the
+# next layer across zero; a flipped mask element is wrong by its full size, so a fraction f of
+# flips costs about sqrt(f) (f ~ 1e-4 at K = 25088 gives ~1.3e-2).  With the ReLU decisions
+# forced to the oracle's stored activations the plain 1e-2 holds.
+TOL_BF16_FREE = 5e-2
 
 
 @pytest.fixture(scope="module")
@@ -58,6 +64,8 @@ def small_bf16():
 def test_small_bf16_grids(small_bf16, grid, mp, fused):
     w, inp, o = small_bf16
     g = gpu_fc_step(w, inp, grid, max_partials=mp, fused=fused)
+    compare_fc_step(g, o, TOL_BF16, fused, tol_below_relu=TOL_BF16_FREE)
+    g = gpu_fc_step(w, inp, grid, max_partials=mp, fused=fused, force_acts=oracle_hidden_acts(o))
     compare_fc_step(g, o, TOL_BF16, fused)
 
 
@@ -110,6 +118,8 @@ def test_full_size_fc_workloads(name, grid, mp):
     inp = I.make_inputs(w, seed=0)
     o = oracle_fc_step(w, inp)
     g = gpu_fc_step(w, inp, grid, max_partials=mp)
+    compare_fc_step(g, o, TOL_BF16, tol_below_relu=TOL_BF16_FREE)
+    g = gpu_fc_step(w, inp, grid, max_partials=mp, force_acts=oracle_hidden_acts(o))
     compare_fc_step(g, o, TOL_BF16)
     gf = gpu_fc_step(w, inp, grid, max_partials=mp, fused=True)
-    compare_fc_step(gf, o, TOL_BF16, fused=True)
+    compare_fc_step(gf, o, TOL_BF16, fused=True, tol_below_relu=TOL_BF16_FREE)
