@@ -1,0 +1,368 @@
+#!/usr/bin/env python
+"""Training-step throughput of the matrix-form minibatch-SGD step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5] [--grid 16x16]
+                    [--max-partials 2] [--impl ours|reference]
+
+One step = forward + loss + backward over the logical P_r x P_c grid + fused SGD update
+on one batch of synthetic input.  `value` is timed with inputs resident in HBM; `e2e` goes
+through mbd_train_step_host with pinned host buffers (H2D of the batch and D2H of the loss
+inside the timed region).  With N > 1 (torchrun) every rank runs an independent replica
+(weak scaling, no data-path collective); time is the max over ranks.  `--impl reference`
+times the fp64 CPU oracle on a bounded sample of the same workload.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1712_04432_b200 import inputs as I  # noqa: E402
+
+METRIC = "training-step TFLOP/s (fwd+bwd+update)"
+SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg5", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--grid", default=None, help="P_r x P_c, e.g. 16x16 (default: the workload's second grid)")
+    ap.add_argument("--max-partials", type=int, default=2)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons of one GPU, sampled every 200 ms while running."""
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={SMI_QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def pick_grid(w, arg):
+    if arg:
+        a, b = arg.lower().split("x")
+        return int(a), int(b)
+    return w.grids[1] if len(w.grids) > 1 else w.grids[0]
+
+
+def workload_config(w, grid, max_partials):
+    if w.kind == "fc":
+        desc = f"{w.name}: FC stack {'-'.join(str(d) for d in w.dims)}, B={w.B}, ReLU, softmax-CE, {w.dtype}"
+    else:
+        desc = f"{w.name}: {w.n_layers}x conv3x3 {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, B={w.B}, half-SSQ, {w.dtype}"
+    return dict(workload=desc, grid=f"{grid[0]}x{grid[1]}", max_partials=max_partials, batch=w.B,
+                l2="weights + activations per step exceed the 126 MB L2 (no flush needed)"
+                if I.step_flops(w) > 1e12 else "L2 flushed by a 256 MB write between steps")
+
+
+# ------------------------------------------------------------------------------ oracle timing
+def oracle_sample(w, inp, max_seconds_hint=20.0):
+    """Time the fp64 oracle, as it stands, on a bounded sample of the workload: the whole
+    network on the first `Bs` samples of the batch.  Returns (flops, seconds, description)."""
+    from oracle import mbd_oracle as O
+    if w.kind == "fc":
+        flops_per_sample = I.step_flops(w) / w.B
+        # aim at roughly 1.5 TFLOP of fp64 work at most
+        Bs = int(max(1, min(w.B, 1.5e12 // flops_per_sample)))
+        layers = [O.FC(inp.Ws[i].astype(np.float64), inp.bs[i].astype(np.float64)) for i in range(len(inp.Ws))]
+        X = inp.X[:Bs].astype(np.float64).T
+        labels = inp.labels[:Bs]
+        t0 = time.perf_counter()
+        O.train_step(layers, X, labels, "softmax_ce", w.eta)
+        dt = time.perf_counter() - t0
+        return flops_per_sample * Bs, dt, f"whole {len(layers)}-layer network, first {Bs} of {w.B} samples, fp64 numpy"
+    C, H, Wd = w.dims
+    Bs, Hs = 1, min(H, 56)
+    layers = [O.Conv3x3(k.astype(np.float64)) for k in inp.Ws]
+    X = inp.X[:Bs, :, :Hs, :].astype(np.float64)
+    t0 = time.perf_counter()
+    O.train_step(layers, X, None, "half_ssq", w.eta)
+    dt = time.perf_counter() - t0
+    flops = 2.0 * Bs * Hs * Wd * C * C * 9 * (3 * w.n_layers - 1)
+    return flops, dt, f"{w.n_layers} conv layers on {Bs} image(s), first {Hs} rows, fp64 numpy"
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info()]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def small_inputs_for_oracle(w):
+    """Inputs for the oracle sample without drawing the whole batch when it is huge."""
+    if w.kind == "fc" and w.B > 1024:
+        ws = I.Workload(w.name, w.kind, w.dims, 1024, w.dtype, w.x_dist, w.loss, w.eta)
+        inp = I.make_inputs(ws, seed=0)
+        return inp
+    return I.make_inputs(w, seed=0)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = I.WORKLOADS[args.workload]
+    grid = pick_grid(w, args.grid)
+    inp = small_inputs_for_oracle(w)
+    times, flops, desc = [], 0.0, ""
+    for i in range(args.warmup + args.steps):
+        flops, dt, desc = oracle_sample(w, inp)
+        if i >= args.warmup:
+            times.append(dt)
+        if sum(times) > 150.0:      # keep the whole run within a few minutes
+            break
+    dt = sum(times) / len(times)
+    val = flops / dt / 1e12
+    cores = host_threads()
+    line = dict(impl="reference", metric=METRIC, value=val, unit="TFLOP/s", n_gpus=args.gpus, steps=len(times),
+                warmup=args.warmup, ms_per_step=dt * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", config=workload_config(w, grid, args.max_partials),
+                cpu_baseline=dict(value=val, unit="TFLOP/s", cores=cores, kind="oracle", sample=desc),
+                e2e=dict(value=val, unit="TFLOP/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------ our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1712_04432_b200 import mbd
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    w = I.WORKLOADS[args.workload]
+    grid = pick_grid(w, args.grid)
+    bf = w.dtype == "bf16"
+    inp = I.make_inputs(w, seed=rank)          # every replica draws its own batch and weights
+    flops = float(I.step_flops(w))
+
+    def dev(a):
+        a = np.ascontiguousarray(a, np.float32)
+        if bf:
+            return torch.from_numpy(I.bf16_bits(a).view(np.int16)).cuda().view(torch.bfloat16)
+        return torch.from_numpy(a).cuda()
+
+    if w.kind == "fc":
+        net = mbd.Net(mbd.fc_layers(w.dims, bias=True), w.B, grid[0], grid[1], mbd.BF16 if bf else mbd.F32,
+                      mbd.LOSS_SOFTMAX_CE, args.max_partials)
+        for i, Wi in enumerate(inp.Ws):
+            net.set_weights(i, dev(Wi), torch.from_numpy(inp.bs[i]).cuda())
+        labels = torch.from_numpy(inp.labels).cuda()
+        labels_host = torch.from_numpy(inp.labels).pin_memory()
+    else:
+        C_, H, Wd = w.dims
+        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd), w.B, grid[0], 1, mbd.BF16, mbd.LOSS_HALF_SSQ,
+                      args.max_partials)
+        for i, Ki in enumerate(inp.Ws):
+            net.set_weights(i, dev(Ki))
+        labels = labels_host = None
+    X = dev(inp.X)
+    X_host = X.cpu().pin_memory()
+    J = torch.zeros(1, dtype=torch.float32, device="cuda")
+    flush = None
+    if flops < 1e12:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def step():
+        if flush is not None:
+            flush.fill_(1)
+        net.forward(X, labels, J)
+        net.backward(w.eta)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    net.poll()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    net.profile_enable(True)
+    launches0 = net.launch_count
+    barrier()
+    per_step = []
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    t_all0 = torch.cuda.Event(enable_timing=True)
+    t_all1 = torch.cuda.Event(enable_timing=True)
+    t_all0.record()
+    for k in range(args.steps):
+        if flush is not None:
+            flush.fill_(1)
+        evs[k][0].record()
+        net.forward(X, labels, J)
+        net.backward(w.eta)
+        evs[k][1].record()
+    t_all1.record()
+    torch.cuda.synchronize()
+    barrier()
+    launches = net.launch_count - launches0
+    per_step = [a.elapsed_time(b) for a, b in evs]
+    ms = sum(per_step) / len(per_step)               # flush time excluded
+    ms = max_over_ranks(ms)
+    prof = net.profile_read()
+    net.profile_enable(False)
+    net.poll()
+    loss_last = float(J.item())
+
+    # ---- end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        for _ in range(2):
+            net.train_step_host(X_host, labels_host, w.eta)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            net.train_step_host(X_host, labels_host, w.eta)      # returns after the loss is on the host
+        torch.cuda.synchronize()
+        dt = (time.perf_counter() - t0) / args.steps
+        dt = max_over_ranks(dt)
+        h2d = X_host.numel() * X_host.element_size() + (labels_host.numel() * 4 if labels_host is not None else 0)
+        e2e = dict(value=flops * world / dt / 1e12, unit="TFLOP/s", h2d_bytes_per_step=int(h2d), d2h_bytes_per_step=4,
+                   ms_per_step=dt * 1e3)
+    clocks = sampler.stop() if rank == 0 else None
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    # dominant kernel class by device time
+    dom = max(prof.items(), key=lambda kv: kv[1]["ms"])[0] if prof else None
+    gemm = {k: v for k, v in prof.items() if k.startswith("gemm") or k.startswith("conv")}
+    roofline = None
+    if gemm:
+        g_ms = sum(v["ms"] for v in gemm.values())
+        g_fl = sum(v["work"] for v in gemm.values())
+        g_n = sum(v["launches"] for v in gemm.values())
+        ach = g_fl / (g_ms * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"] if bf else None
+        roofline = dict(bound="tensor" if bf else "alu", kernel="gemm_tc_kernel (all three operand layouts)",
+                        achieved=ach, peak=peak, unit="TFLOP/s", frac=(ach / peak) if peak else None,
+                        peak_kind=f"{peaks['source']} sustained bf16 (kernel timed inside a long step); "
+                                  f"burst {peaks['bf16_tflops']}", frac_of_burst=ach / peaks["bf16_tflops"] if bf else None,
+                        launches=g_n, avg_launch_ms=g_ms / g_n, flops_per_launch=g_fl / g_n,
+                        share_of_step=g_ms / (ms * args.steps), traffic=TRAFFIC.get(w.name))
+    kernels = {k: dict(ms_per_step=v["ms"] / args.steps, launches_per_step=v["launches"] / args.steps,
+                       rate=(v["work"] / (v["ms"] * 1e-3) / (1e12 if (k.startswith("gemm") or k.startswith("conv_")) else 1e9))
+                       if v["ms"] > 0 else None,
+                       rate_unit="TFLOP/s" if (k.startswith("gemm") or k.startswith("conv_")) else "GB/s")
+               for k, v in prof.items()}
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        inp_o = small_inputs_for_oracle(w)
+        fl, dt, desc = oracle_sample(w, inp_o)
+        cpu = dict(value=fl / dt / 1e12, unit="TFLOP/s", cores=host_threads(), kind="oracle", sample=desc,
+                   seconds=dt)
+
+    line = dict(metric=METRIC, value=flops * world / (ms * 1e-3) / 1e12, unit="TFLOP/s", n_gpus=world,
+                steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=ms, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype=w.dtype, data="synthetic",
+                config=workload_config(w, grid, args.max_partials), clocks=clocks, e2e=e2e,
+                gpu_launches=int(launches) * world, roofline=roofline, cpu_baseline=cpu,
+                frac_of_burst_peak=flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"] if bf else None,
+                kernels=kernels, dominant_kernel_class=dom, loss_last=loss_last)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# DRAM bytes per launch of the dominant kernel from an ncu capture (see profiles/); null until captured.
+TRAFFIC = {}
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

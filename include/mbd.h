@@ -154,6 +154,20 @@ MBD_API mbd_status mbd_set_tensor(mbd_net* net, int which, int layer, const void
  * a kernel's bounded barrier wait ran out, or MBD_E_CUDA. */
 MBD_API mbd_status mbd_poll_status(mbd_net* net);
 
+/* Per-kernel-class device timing with CUDA events on the network's stream.  While enabled,
+ * every launch is bracketed by two events; mbd_profile_read waits for the stream and returns,
+ * for one class, the summed duration (ms), the number of launches and the summed ALGORITHMIC
+ * work of those launches: flops (2 M N K) for the contraction classes, bytes for the others.
+ * mbd_profile_enable(net, 1) also clears the counters. */
+enum {
+  MBD_K_GEMM_FWD = 0, MBD_K_GEMM_BWD_DATA = 1, MBD_K_GEMM_BWD_WEIGHT = 2, MBD_K_REDUCE = 3,
+  MBD_K_SOFTMAX = 4, MBD_K_COLSUM = 5, MBD_K_SGD = 6, MBD_K_HALO = 7, MBD_K_CONV_FWD = 8,
+  MBD_K_CONV_BWD_DATA = 9, MBD_K_CONV_BWD_WEIGHT = 10, MBD_K_OTHER = 11, MBD_K_COUNT = 12
+};
+MBD_API mbd_status mbd_profile_enable(mbd_net* net, int on);
+MBD_API mbd_status mbd_profile_read(mbd_net* net, int kclass, double* ms_total, int64_t* launches,
+                            double* work_total);
+
 /* Kernels launched by this network since creation (host counter). */
 MBD_API int64_t mbd_launch_count(const mbd_net* net);
 

@@ -5,17 +5,18 @@
 #include <stdint.h>
 
 #include "../../include/mbd.h"
+#include "kernels.h"
 
 namespace mbd {
 struct ConvNet;
 mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int max_partials, int num_sms, int* status,
-                       cudaStream_t stream, ConvNet** out);
+                       cudaStream_t stream, Profiler* prof, ConvNet** out);
 void conv_destroy(ConvNet* c);
 mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev);
 mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev);
-mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev, int64_t* launches);
-mbd_status conv_backward(ConvNet* c, float fused_eta, int64_t* launches);
-mbd_status conv_sgd_step(ConvNet* c, float eta, int64_t* launches);
+mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev);
+mbd_status conv_backward(ConvNet* c, float fused_eta);
+mbd_status conv_sgd_step(ConvNet* c, float eta);
 mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t bytes);
 mbd_status conv_set_tensor(ConvNet* c, int which, int layer, const void* src, size_t bytes);
 size_t conv_input_bytes(const ConvNet* c);

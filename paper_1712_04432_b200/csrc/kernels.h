@@ -90,6 +90,28 @@ int colsum_row_splits(int64_t M);
 cudaError_t sgd_update_launch(void* w, int w_bf16, const float* g, int64_t n, float scale,
                               int num_sms, cudaStream_t stream);
 
+// ---- per-class event timing (host) ---------------------------------------------------------
+struct Profiler {
+  static constexpr int NCLS = 12;
+  bool on = false;
+  cudaStream_t stream = nullptr;
+  struct Pending { cudaEvent_t a, b; int cls; };
+  Pending* pending = nullptr;
+  int n_pending = 0, cap = 0;
+  cudaEvent_t* pool = nullptr;
+  int n_pool = 0, pool_cap = 0;
+  double ms[NCLS] = {0}, work[NCLS] = {0};
+  long long launches[NCLS] = {0};
+  int64_t total_launches = 0;
+
+  cudaEvent_t get_event();
+  void begin(int cls, double w);
+  void end();
+  void collect();          // synchronises the stream
+  void reset();
+  void destroy();
+};
+
 // ---- domain-parallel 3x3 convolution (conv.cu) ------------------------------------------
 struct ConvNet;   // defined in conv.cu
 }  // namespace mbd

@@ -55,7 +55,7 @@ struct mbd_net {
   const void* X_mapped = nullptr;   // input pointer the layer-1 tensor maps were built for
   const int32_t* labels = nullptr;
   int state = ST_IDLE;
-  int64_t launches = 0;
+  Profiler prof;
   void* X_stage = nullptr;
   int32_t* labels_stage = nullptr;
   ConvNet* conv = nullptr;
@@ -106,11 +106,13 @@ Epi epi_sgd(void* w, int64_t ldo, int out_bf16, float scale) {
 // of its partials when the K range was split.
 mbd_status run_gemm(mbd_net* n, TcGemm& tc, int variant, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                     const void* Bm, int64_t ldb, int S, const Epi& epi) {
+  const double flops = 2.0 * static_cast<double>(M) * static_cast<double>(N) * static_cast<double>(K);
   if (n->dtype == MBD_BF16) {
     tc.epi = epi;
     tc.partials = n->partials;
+    n->prof.begin(MBD_K_GEMM_FWD + variant, flops);
     CK(tc_gemm_launch(tc, n->stream));
-    n->launches++;
+    n->prof.end();
     S = tc.k_splits;
   } else {
     SimtGemm g{};
@@ -124,12 +126,18 @@ mbd_status run_gemm(mbd_net* n, TcGemm& tc, int variant, int64_t M, int64_t N, i
     g.k_splits = S;
     g.partials = n->partials;
     g.epi = epi;
+    n->prof.begin(MBD_K_GEMM_FWD + variant, flops);
     CK(simt_gemm_launch(g, n->stream));
-    n->launches++;
+    n->prof.end();
   }
   if (S > 1) {
+    // (S + 1) planes of M N floats cross HBM, plus what the tail operation touches
+    const double esz = epi.out_bf16 ? 2.0 : 4.0;
+    double bytes = static_cast<double>(M) * N * (4.0 * S + esz);
+    if (epi.op == EPI_SGD || (epi.op == EPI_MASK && epi.mask)) bytes += static_cast<double>(M) * N * esz;
+    n->prof.begin(MBD_K_REDUCE, bytes);
     CK(reduce_partials_launch(n->partials, S, M, N, epi, n->num_sms, n->stream));
-    n->launches++;
+    n->prof.end();
   }
   return MBD_OK;
 }
@@ -168,6 +176,7 @@ void free_net(mbd_net* n) {
   cudaFree(n->partials); cudaFree(n->colsum_scratch); cudaFree(n->per_sample); cudaFree(n->loss_dev);
   cudaFree(n->status); cudaFree(n->X_stage); cudaFree(n->labels_stage);
   if (n->conv) conv_destroy(n->conv);
+  n->prof.destroy();
   (void)cudaGetLastError();
   delete n;
 }
@@ -211,6 +220,7 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   n->L = L; n->B = B; n->P_r = P_r; n->P_c = P_c; n->dtype = dtype; n->loss = loss;
   n->max_partials = max_partials == 0 ? 4 : max_partials;
   n->stream = static_cast<cudaStream_t>(cuda_stream);
+  n->prof.stream = n->stream;
   n->is_conv = is_conv;
   mbd_status st = MBD_OK;
   cudaDeviceProp prop;
@@ -236,7 +246,7 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   if (cudaMemsetAsync(n->status, 0, sizeof(int), n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
 
   if (is_conv) {
-    st = conv_create(layers, L, B, P_r, n->max_partials, n->num_sms, n->status, n->stream, &n->conv);
+    st = conv_create(layers, L, B, P_r, n->max_partials, n->num_sms, n->status, n->stream, &n->prof, &n->conv);
     if (st != MBD_OK) { free_net(n); return st; }
     *out = n;
     return MBD_OK;
@@ -321,7 +331,7 @@ extern "C" mbd_status mbd_get_weights(mbd_net* n, int layer, void* W_dev, float*
 extern "C" mbd_status mbd_forward(mbd_net* n, const void* X_dev, const int32_t* labels_dev, float* loss_sum_dev) {
   if (!n || !X_dev) return MBD_E_INVALID;
   if (n->is_conv) {
-    mbd_status s = conv_forward(n->conv, X_dev, loss_sum_dev, &n->launches);
+    mbd_status s = conv_forward(n->conv, X_dev, loss_sum_dev);
     if (s == MBD_OK) n->state = ST_FWD;
     return s;
   }
@@ -339,11 +349,13 @@ extern "C" mbd_status mbd_forward(mbd_net* n, const void* X_dev, const int32_t* 
     if (s != MBD_OK) return s;
   }
   Layer& top = n->layers[n->L - 1];
+  n->prof.begin(MBD_K_SOFTMAX, static_cast<double>(n->B) * top.d_out * (4.0 + (bf ? 2.0 : 4.0)));
   CK(softmax_xent_launch(static_cast<const float*>(top.act), n->B, top.d_out, labels_dev, top.dY, bf, n->per_sample, n->stream));
-  n->launches++;
+  n->prof.end();
   if (loss_sum_dev) {
+    n->prof.begin(MBD_K_OTHER, static_cast<double>(n->B) * 4.0);
     CK(sum_f32_launch(n->per_sample, n->B, 1.f, loss_sum_dev, n->stream));
-    n->launches++;
+    n->prof.end();
   }
   n->state = ST_FWD;
   return MBD_OK;
@@ -353,7 +365,7 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
   if (!n || fused_eta < 0.f) return MBD_E_INVALID;
   if (n->state != ST_FWD) return MBD_E_STATE;
   if (n->is_conv) {
-    mbd_status s = conv_backward(n->conv, fused_eta, &n->launches);
+    mbd_status s = conv_backward(n->conv, fused_eta);
     if (s == MBD_OK) n->state = fused_eta > 0.f ? ST_BWD_FUSED : ST_BWD_UNFUSED;
     return s;
   }
@@ -364,9 +376,11 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
   for (int i = n->L - 1; i >= 0; --i) {
     Layer& l = n->layers[i];
     if (l.bias) {
+      n->prof.begin(MBD_K_COLSUM, static_cast<double>(n->B) * l.d_out * (bf ? 2.0 : 4.0));
       CK(colsum_launch(l.dY, bf, n->B, l.d_out, n->colsum_scratch, colsum_row_splits(n->B), fused ? nullptr : l.db,
                        fused ? l.bias : nullptr, scale, n->stream));
-      n->launches += 2;
+      n->prof.end();
+      n->prof.total_launches++;   // two kernels
     }
     if (i > 0) {   // nothing is propagated below the first layer
       Layer& prev = n->layers[i - 1];
@@ -386,18 +400,20 @@ extern "C" mbd_status mbd_sgd_step(mbd_net* n, float eta) {
   if (!n || eta < 0.f) return MBD_E_INVALID;
   if (n->state != ST_BWD_UNFUSED) return MBD_E_STATE;
   if (n->is_conv) {
-    mbd_status s = conv_sgd_step(n->conv, eta, &n->launches);
+    mbd_status s = conv_sgd_step(n->conv, eta);
     if (s == MBD_OK) n->state = ST_IDLE;
     return s;
   }
   const float scale = -eta / static_cast<float>(n->B);
   for (int i = 0; i < n->L; ++i) {
     Layer& l = n->layers[i];
+    n->prof.begin(MBD_K_SGD, static_cast<double>(l.nW) * (4.0 + 2.0 * n->elt()));
     CK(sgd_update_launch(l.W, n->dtype == MBD_BF16, l.dW, l.nW, scale, n->num_sms, n->stream));
-    n->launches++;
+    n->prof.end();
     if (l.bias) {
+      n->prof.begin(MBD_K_SGD, static_cast<double>(l.d_out) * 12.0);
       CK(sgd_update_launch(l.bias, 0, l.db, l.d_out, scale, n->num_sms, n->stream));
-      n->launches++;
+      n->prof.end();
     }
   }
   n->state = ST_IDLE;
@@ -485,7 +501,23 @@ extern "C" mbd_status mbd_poll_status(mbd_net* n) {
   return MBD_OK;
 }
 
-extern "C" int64_t mbd_launch_count(const mbd_net* n) { return n ? n->launches : -1; }
+extern "C" int64_t mbd_launch_count(const mbd_net* n) { return n ? n->prof.total_launches : -1; }
+
+extern "C" mbd_status mbd_profile_enable(mbd_net* n, int on) {
+  if (!n) return MBD_E_INVALID;
+  n->prof.reset();
+  n->prof.on = on != 0;
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_profile_read(mbd_net* n, int kclass, double* ms_total, int64_t* launches, double* work_total) {
+  if (!n || kclass < 0 || kclass >= MBD_K_COUNT) return MBD_E_INVALID;
+  n->prof.collect();
+  if (ms_total) *ms_total = n->prof.ms[kclass];
+  if (launches) *launches = n->prof.launches[kclass];
+  if (work_total) *work_total = n->prof.work[kclass];
+  return MBD_OK;
+}
 
 extern "C" mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                                     const void* Bm, int64_t ldb, float* D, int64_t ldd, int k_splits, float* partials,

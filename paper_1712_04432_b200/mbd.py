@@ -20,9 +20,12 @@ F32, BF16 = 0, 1
 LOSS_SOFTMAX_CE, LOSS_HALF_SSQ = 0, 1
 T_ACT, T_DY, T_DW, T_DB, T_LOSS, T_PARTIALS = range(6)
 
+KERNEL_CLASSES = ["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce_partials", "softmax_xent", "colsum",
+                  "sgd_update", "halo_stage", "conv_fwd", "conv_bwd_data", "conv_bwd_weight", "other"]
+
 EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weights", "mbd_forward",
            "mbd_backward", "mbd_sgd_step", "mbd_train_step_host", "mbd_comm_words", "mbd_get_tensor",
-           "mbd_set_tensor", "mbd_poll_status", "mbd_launch_count", "mbd_gemm_bf16", "mbd_strerror"]
+           "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_strerror"]
 
 
 class MbdError(RuntimeError):
@@ -67,6 +70,8 @@ def lib():
         L.mbd_get_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
         L.mbd_set_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
         L.mbd_poll_status.argtypes = [vp]
+        L.mbd_profile_enable.argtypes = [vp, i32]
+        L.mbd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double)]
         L.mbd_launch_count.argtypes = [vp]
         L.mbd_launch_count.restype = i64
         L.mbd_gemm_bf16.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp, vp]
@@ -215,6 +220,19 @@ class Net:
 
     def poll(self):
         _check(lib().mbd_poll_status(self._h), "mbd_poll_status")
+
+    def profile_enable(self, on: bool = True):
+        _check(lib().mbd_profile_enable(self._h, int(on)), "mbd_profile_enable")
+
+    def profile_read(self) -> Dict[str, Dict[str, float]]:
+        """Per kernel class: summed ms, launches, summed algorithmic work (flops or bytes)."""
+        out = {}
+        for k, name in enumerate(KERNEL_CLASSES):
+            ms, n, w = C.c_double(0), C.c_int64(0), C.c_double(0)
+            _check(lib().mbd_profile_read(self._h, k, C.byref(ms), C.byref(n), C.byref(w)), "mbd_profile_read")
+            if n.value:
+                out[name] = dict(ms=ms.value, launches=int(n.value), work=w.value)
+        return out
 
     @property
     def launch_count(self) -> int:
