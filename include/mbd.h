@@ -54,7 +54,8 @@ typedef enum {
   MBD_E_CUDA = 4,        /* a CUDA runtime / driver call failed                     */
   MBD_E_STATE = 5,       /* call order violated (forward -> backward -> sgd_step)   */
   MBD_E_TIMEOUT = 6,     /* a bounded device-side wait gave up (see mbd_poll_status)*/
-  MBD_E_UNSUPPORTED = 7  /* shape / layer kind outside what the kernels cover       */
+  MBD_E_UNSUPPORTED = 7, /* shape / layer kind outside what the kernels cover       */
+  MBD_E_TOO_LARGE = 8    /* beyond the fixed scratch of an allocation-free entry    */
 } mbd_status;
 
 enum { MBD_FC = 0, MBD_CONV3X3 = 1 };                 /* mbd_layer.kind                      */
@@ -182,6 +183,24 @@ MBD_API int64_t mbd_launch_count(const mbd_net* net);
 MBD_API mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, const void* A_dev,
                          int64_t lda, const void* B_dev, int64_t ldb, float* D_dev, int64_t ldd,
                          int k_splits, float* partials_dev, void* cuda_stream);
+
+/* No counterpart in the paper: a convenience for callers that cannot allocate device memory
+ * themselves and cannot let a library do it -- a service whose own pool owns all of the GPU's
+ * memory, a plug-in that runs where cudaMalloc would stall or fail (memory exhausted, or an
+ * environment that forbids implicit synchronisation), or code that wants a fixed footprint.
+ * Same contraction, operand layouts, splitting and result as mbd_gemm_bf16, but the fp32
+ * partial sums (k_splits > 1) and the status word live in a fixed 16 MiB array inside the
+ * library's device image (present on every GPU that loads the library, until exit) and the
+ * call makes no cudaMalloc / cudaFree nor any other allocating call.
+ *   - MBD_E_TOO_LARGE if min(k_splits, ceil(K/64)) * M * N exceeds 4 Mi floats (k_splits > 1).
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current, as for every call); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the
+ *     entry clears what has to start at zero.  Calls whose GPU work overlaps -- different
+ *     streams or threads -- race on it: serialise them.  The call returns after its work is done. */
+MBD_API mbd_status mbd_gemm_bf16_noalloc(int variant, int64_t M, int64_t N, int64_t K, const void* A_dev,
+                                 int64_t lda, const void* B_dev, int64_t ldb, float* D_dev, int64_t ldd,
+                                 int k_splits, void* cuda_stream);
 
 MBD_API const char* mbd_strerror(mbd_status s);
 

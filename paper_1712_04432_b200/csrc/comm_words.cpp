@@ -73,6 +73,7 @@ extern "C" const char* mbd_strerror(mbd_status s) {
     case MBD_E_STATE: return "call order violated (forward -> backward -> sgd_step)";
     case MBD_E_TIMEOUT: return "a bounded device-side wait timed out";
     case MBD_E_UNSUPPORTED: return "unsupported shape or layer kind";
+    case MBD_E_TOO_LARGE: return "problem exceeds the fixed scratch capacity of the allocation-free entry point";
   }
   return "unknown status";
 }

@@ -13,7 +13,7 @@ from typing import Dict, List, Optional, Sequence
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmbd.so")
 
-OK, E_INVALID, E_GRID, E_ALLOC, E_CUDA, E_STATE, E_TIMEOUT, E_UNSUPPORTED = range(8)
+OK, E_INVALID, E_GRID, E_ALLOC, E_CUDA, E_STATE, E_TIMEOUT, E_UNSUPPORTED, E_TOO_LARGE = range(9)
 FC, CONV3X3 = 0, 1
 SPLIT_MODEL, SPLIT_DOMAIN = 0, 1
 F32, BF16 = 0, 1
@@ -25,7 +25,7 @@ KERNEL_CLASSES = ["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce_partia
 
 EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weights", "mbd_forward",
            "mbd_backward", "mbd_sgd_step", "mbd_train_step_host", "mbd_comm_words", "mbd_get_tensor",
-           "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_strerror"]
+           "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_gemm_bf16_noalloc", "mbd_strerror"]
 
 
 class MbdError(RuntimeError):
@@ -75,6 +75,7 @@ def lib():
         L.mbd_launch_count.argtypes = [vp]
         L.mbd_launch_count.restype = i64
         L.mbd_gemm_bf16.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp, vp]
+        L.mbd_gemm_bf16_noalloc.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
         L.mbd_strerror.argtypes = [i32]
         L.mbd_strerror.restype = C.c_char_p
         _lib = L
@@ -257,3 +258,25 @@ def gemm_bf16(variant: int, A, B, k_splits: int = 1, return_partials: bool = Fal
                              k_splits, _ptr(parts), C.c_void_p(torch.cuda.current_stream().cuda_stream))
     _check(st, "mbd_gemm_bf16")
     return (D, parts) if return_partials else D
+
+
+def gemm_bf16_noalloc(variant: int, A, B, k_splits: int = 1, out=None):
+    """mbd_gemm_bf16_noalloc: as gemm_bf16, for callers that may not allocate device memory.
+    The partial sums live in a fixed array inside the library (at most 4 Mi floats for
+    k_splits * M * N); the library allocates nothing.  Pass `out` (float32 [M, N], CUDA) to
+    keep this wrapper from allocating the result as well."""
+    import torch
+    assert A.is_cuda and B.is_cuda and A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16
+    assert A.stride(1) == 1 and B.stride(1) == 1
+    if variant == 0:
+        M, K = A.shape; N = B.shape[0]
+    elif variant == 1:
+        M, K = A.shape; N = B.shape[1]
+    else:
+        K, M = A.shape; N = B.shape[1]
+    D = out if out is not None else torch.empty((M, N), dtype=torch.float32, device="cuda")
+    assert D.dtype == torch.float32 and tuple(D.shape) == (M, N) and D.stride(1) == 1
+    st = lib().mbd_gemm_bf16_noalloc(variant, M, N, K, _ptr(A), A.stride(0), _ptr(B), B.stride(0), _ptr(D),
+                                     D.stride(0), k_splits, C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    _check(st, "mbd_gemm_bf16_noalloc")
+    return D
