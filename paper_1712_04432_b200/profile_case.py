@@ -1,0 +1,45 @@
+"""Runs a few launches of ONE kernel of the training step on synthetic data, for use under
+a profiler (small, self-terminating):
+
+    python -m paper_1712_04432_b200.profile_case gemm_fwd --size 8192 --launches 3
+    python -m paper_1712_04432_b200.profile_case gemm_bwd_weight --size 4096
+    python -m paper_1712_04432_b200.profile_case reduce --size 8192 --splits 2
+
+gemm_*: one tensor-core contraction of size^3 in the operand layout of that product.
+reduce: a split contraction followed by the partial-sum reduction (the reduction reads
+`splits` fp32 planes of size^2 and writes one).
+"""
+import argparse
+
+import torch
+
+from . import mbd
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("case", choices=["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce"])
+    ap.add_argument("--size", type=int, default=8192)
+    ap.add_argument("--launches", type=int, default=3)
+    ap.add_argument("--splits", type=int, default=2)
+    a = ap.parse_args()
+    g = torch.Generator(device="cuda").manual_seed(0)
+    n = a.size
+    A = torch.randn((n, n), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    B = torch.randn((n, n), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    variant = {"gemm_fwd": 0, "gemm_bwd_data": 1, "gemm_bwd_weight": 2, "reduce": 2}[a.case]
+    splits = a.splits if a.case == "reduce" else 1
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(a.launches):
+        D = mbd.gemm_bf16(variant, A, B, k_splits=splits)
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / a.launches
+    print(f"{a.case} size={n} splits={splits}: {ms:.3f} ms per call, {2 * n ** 3 / ms / 1e9:.1f} TFLOP/s, "
+          f"checksum {float(D.double().sum()):.6e}")
+
+
+if __name__ == "__main__":
+    main()
