@@ -89,7 +89,7 @@ def conv3x3(K, X):
     Y = np.zeros((B, K.shape[0], H, W), F64)
     for u in range(3):
         for v in range(3):
-            Y += np.einsum("oc,bchw->bohw", K[:, :, u, v], Xp[:, :, u:u + H, v:v + W])
+            Y += np.einsum("oc,bchw->bohw", K[:, :, u, v], Xp[:, :, u:u + H, v:v + W], optimize=True)
     return Y
 
 
@@ -105,7 +105,7 @@ def conv3x3_dX(K, dY):
         for v in range(3):
             # index h-u+1 in dY  ==  (h-u+2) in the padded array
             dX += np.einsum("oc,bohw->bchw", K[:, :, u, v],
-                            dYp[:, :, 2 - u:2 - u + H, 2 - v:2 - v + W])
+                            dYp[:, :, 2 - u:2 - u + H, 2 - v:2 - v + W], optimize=True)
     return dX
 
 
@@ -119,7 +119,7 @@ def conv3x3_dK(dY, X):
     dK = np.zeros((dY.shape[1], C, 3, 3), F64)
     for u in range(3):
         for v in range(3):
-            dK[:, :, u, v] = np.einsum("bohw,bchw->oc", dY, Xp[:, :, u:u + H, v:v + W])
+            dK[:, :, u, v] = np.einsum("bohw,bchw->oc", dY, Xp[:, :, u:u + H, v:v + W], optimize=True)
     return dK
 
 
@@ -315,7 +315,7 @@ def _conv_rows_valid(K, S):
     Y = np.zeros((B, K.shape[0], hs, W), F64)
     for u in range(3):
         for v in range(3):
-            Y += np.einsum("oc,bchw->bohw", K[:, :, u, v], Sp[:, :, u:u + hs, v:v + W])
+            Y += np.einsum("oc,bchw->bohw", K[:, :, u, v], Sp[:, :, u:u + hs, v:v + W], optimize=True)
     return Y
 
 
@@ -361,7 +361,7 @@ def conv3x3_dK_strips(dY, X, P_r):
         for u in range(3):
             for v in range(3):
                 part[:, :, u, v] = np.einsum("bohw,bchw->oc", dY[:, :, h0:h1, :],
-                                             Sp[:, :, u:u + hs, v:v + W])
+                                             Sp[:, :, u:u + hs, v:v + W], optimize=True)
         parts.append(part)
     dK = np.zeros_like(parts[0])
     for part in parts:

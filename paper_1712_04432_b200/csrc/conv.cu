@@ -1,14 +1,787 @@
+// Domain-parallel 3x3 convolution stack (Section 2.2 and 2.4 of the paper): every image is
+// cut into P_r row strips; a strip owner holds its rows plus one halo row per neighbour,
+// exchanged before each convolution that needs them (forward: X halos, backward-data: dY
+// halos); the weight gradient is formed as per-owner partial sums that are then added (the
+// all-reduce over the strips, third term of Eq. 7).
+//
+// Layout in HBM: every activation / gradient tensor lives as "strips": [Z = B*P_r][R = Hs+2]
+// [W][C = 64] bf16 (channels innermost), row 0 and row Hs+1 of a strip being the halo rows
+// (zero at the image border).  One pixel = 128 contiguous bytes = one 128B-swizzle row, so a
+// TMA box {64 c, n pixels} is directly a K-major (forward, backward-data) or MN-major
+// (backward-weight: pixels are the reduction index) tensor-core operand.
+//
+// conv_fwd_kernel  (forward and, with flipped / transposed weights, backward-data)
+//     one output row segment of 126 pixels per accumulator: for u = 0..2 the input row h+u-1
+//     (128 pixels starting one to the left) is multiplied by the stacked taps [K(u,0); K(u,1);
+//     K(u,2)] (N = 192), giving D_v[p] = sum_{u,c} K[.,c,u,v] X[h+u-1, p, c]; the horizontal
+//     shift is applied on the accumulator side in the epilogue: Y[p] = D_0[p-1] + D_1[p] +
+//     D_2[p+1] (warp shuffles across TMEM lanes).  Input rows sit in a shared-memory ring and
+//     are loaded once per row block; the weights (72 KB) stay resident.
+// conv_wgrad_kernel
+//     dK[o,c,u,v] = sum_pixels dY[p,o] X[p + (u-1,v-1), c]: the three horizontal shifts of an X
+//     row are three TMA boxes (the W coordinate of a box start is free); two shifted copies
+//     form one M = 128 operand; all nine taps accumulate in TMEM for the whole kernel and each
+//     CTA writes one fp32 partial, summed in CTA order (= strip order) by wgrad_finish.
+#include <new>
+#include <vector>
+
 #include "conv.h"
+#include "epi.cuh"
+#include "tc_common.cuh"
+
 namespace mbd {
-struct ConvNet { int dummy; };
-mbd_status conv_create(const mbd_layer*, int, int64_t, int, int, int, int*, cudaStream_t, Profiler*, ConvNet**) { return MBD_E_UNSUPPORTED; }
-void conv_destroy(ConvNet*) {}
-mbd_status conv_set_weights(ConvNet*, int, const void*) { return MBD_E_UNSUPPORTED; }
-mbd_status conv_get_weights(ConvNet*, int, void*) { return MBD_E_UNSUPPORTED; }
-mbd_status conv_forward(ConvNet*, const void*, float*) { return MBD_E_UNSUPPORTED; }
-mbd_status conv_backward(ConvNet*, float) { return MBD_E_UNSUPPORTED; }
-mbd_status conv_sgd_step(ConvNet*, float) { return MBD_E_UNSUPPORTED; }
-mbd_status conv_get_tensor(ConvNet*, int, int, void*, size_t) { return MBD_E_UNSUPPORTED; }
-mbd_status conv_set_tensor(ConvNet*, int, int, const void*, size_t) { return MBD_E_UNSUPPORTED; }
-size_t conv_input_bytes(const ConvNet*) { return 0; }
+
+using namespace tc;
+typedef __nv_bfloat16 bf16;
+
+namespace {
+
+constexpr int C = 64;                 // channels in and out
+constexpr int FWD_PIX = 126;          // output pixels per forward tile (lanes 1..126 of 128)
+constexpr int FWD_STAGES = 8;         // ring of input rows, 16 KB each
+constexpr int FWD_ROW_BYTES = 128 * 128;
+constexpr int FWD_W_BYTES = 3 * 192 * 128;   // stacked taps, 72 KB
+constexpr int FWD_SMEM = FWD_W_BYTES + FWD_STAGES * FWD_ROW_BYTES + 1024;
+constexpr int WG_PIX = 64;            // pixels (reduction length) per backward-weight block
+constexpr int WG_XSTAGES = 6;         // X rows: 3 shifted copies of 8 KB each
+constexpr int WG_YSTAGES = 4;         // dY rows: 8 KB each
+constexpr int WG_CHUNK = WG_PIX * 128;
+constexpr int WG_SMEM = WG_XSTAGES * 3 * WG_CHUNK + WG_YSTAGES * WG_CHUNK + WG_CHUNK /*junk pad*/ + 1024;
+constexpr int NUM_THREADS = 192;
+
+enum { MODE_RELU_STORE = 0, MODE_STORE_SSQ = 1, MODE_MASK = 2 };
+
+// ------------------------------------------------------------------------------ layout kernels
+// NCHW -> strips.  Block = (32-pixel segment, image row h, image b); 256 threads.  A row that
+// borders another strip is also written into that neighbour's halo row: this is the forward
+// halo exchange for the network input, fused into the staging pass.
+__global__ void __launch_bounds__(256)
+nchw_to_strips_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int H, int W, int P_r, int Hs) {
+  __shared__ bf16 tile[C][32 + 2];
+  const int w0 = blockIdx.x * 32, h = blockIdx.y, b = blockIdx.z;
+  const int t = threadIdx.x;
+  {
+    const int c = t >> 2, wq = (t & 3) * 8;
+    const bf16* p = src + ((static_cast<int64_t>(b) * C + c) * H + h) * W + w0 + wq;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) tile[c][wq + i] = (w0 + wq + i < W) ? p[i] : __float2bfloat16(0.f);
+  }
+  __syncthreads();
+  const int px = t >> 3, cq = (t & 7) * 8;
+  if (w0 + px >= W) return;
+  uint4 v;
+  uint32_t* vw = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint16_t lo = __bfloat16_as_ushort(tile[cq + 2 * i][px]);
+    const uint16_t hi = __bfloat16_as_ushort(tile[cq + 2 * i + 1][px]);
+    vw[i] = static_cast<uint32_t>(lo) | (static_cast<uint32_t>(hi) << 16);
+  }
+  const int R = Hs + 2;
+  const int s = h / Hs, r = h - s * Hs + 1;
+  auto put = [&](int ss, int rr) {
+    bf16* q = dst + (((static_cast<int64_t>(b) * P_r + ss) * R + rr) * W + (w0 + px)) * C + cq;
+    *reinterpret_cast<uint4*>(q) = v;
+  };
+  put(s, r);
+  if (r == 1 && s > 0) put(s - 1, Hs + 1);          // first row of a strip: lower halo of the strip above
+  if (r == Hs && s < P_r - 1) put(s + 1, 0);        // last row of a strip: upper halo of the strip below
+}
+
+// strips -> NCHW (read-back only).
+__global__ void __launch_bounds__(256)
+strips_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int H, int W, int P_r, int Hs) {
+  __shared__ bf16 tile[32][C + 2];
+  const int w0 = blockIdx.x * 32, h = blockIdx.y, b = blockIdx.z;
+  const int t = threadIdx.x;
+  const int R = Hs + 2;
+  const int s = h / Hs, r = h - s * Hs + 1;
+  {
+    const int px = t >> 3, cq = (t & 7) * 8;
+    if (w0 + px < W) {
+      const bf16* q = src + (((static_cast<int64_t>(b) * P_r + s) * R + r) * W + (w0 + px)) * C + cq;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) tile[px][cq + i] = q[i];
+    }
+  }
+  __syncthreads();
+  const int c = t >> 2, wq = (t & 3) * 8;
+  bf16* p = dst + ((static_cast<int64_t>(b) * C + c) * H + h) * W + w0 + wq;
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+    if (w0 + wq + i < W) p[i] = tile[wq + i][c];
+}
+
+// Halo exchange between neighbouring strips of one tensor: the last own row of strip s becomes
+// the upper halo of strip s+1 and the first own row of strip s+1 the lower halo of strip s.
+// grid = (B * (P_r - 1), 2 directions); one boundary row = W*C bf16, copied with 16-byte accesses.
+__global__ void __launch_bounds__(256)
+halo_stage_kernel(bf16* __restrict__ buf, int W, int P_r, int Hs) {
+  const int R = Hs + 2;
+  const int b = blockIdx.x / (P_r - 1), s = blockIdx.x % (P_r - 1);
+  const int64_t row = static_cast<int64_t>(W) * C;           // elements per row
+  const int64_t z0 = (static_cast<int64_t>(b) * P_r + s) * R, z1 = z0 + R;
+  const bf16* src;
+  bf16* dst;
+  if (blockIdx.y == 0) { src = buf + (z0 + Hs) * row; dst = buf + (z1 + 0) * row; }
+  else { src = buf + (z1 + 1) * row; dst = buf + (z0 + Hs + 1) * row; }
+  const uint4* s4 = reinterpret_cast<const uint4*>(src);
+  uint4* d4 = reinterpret_cast<uint4*>(dst);
+  for (int64_t i = threadIdx.x; i < row / 8; i += 256) d4[i] = s4[i];
+}
+
+// Canonical K[o][c][u][v] -> forward operand Wf[u][(v,o)][c] and backward-data operand
+// Wb[u'][(v',c)][o] = K[o][c][2-u'][2-v'] (taps flipped, channels swapped).
+__global__ void pack_weights_kernel(const bf16* __restrict__ K, bf16* __restrict__ Wf, bf16* __restrict__ Wb) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= C * C * 9) return;
+  const int o = i / (C * 9), c = (i / 9) % C, u = (i % 9) / 3, v = i % 3;
+  const bf16 k = K[i];
+  Wf[((u * 3 + v) * C + o) * C + c] = k;
+  Wb[(((2 - u) * 3 + (2 - v)) * C + c) * C + o] = k;
+}
+
+// Sum of the per-CTA partials [G][9][c][o] in CTA order, into canonical [o][c][u][v]:
+// either stored (dK) or applied as K += scale * dK (Eq. 1).
+__global__ void wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ dK, bf16* __restrict__ K,
+                                    float scale) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= 9 * C * C) return;
+  const int t = i / (C * C), c = (i / C) % C, o = i % C;
+  float s = part[i];
+  for (int g = 1; g < G; ++g) s += part[static_cast<int64_t>(g) * 9 * C * C + i];
+  const int e = (o * C + c) * 9 + t;
+  if (dK) dK[e] = s;
+  if (K) K[e] = __float2bfloat16_rn(fmaf(scale, s, __bfloat162float(K[e])));
+}
+
+// ------------------------------------------------------------------------------ forward kernel
+struct FwdParams {
+  int W, Hs, R, RB, nrb, nseg, n_items;
+  int mode;
+  bf16* out;              // strips
+  const bf16* mask_src;   // strips (MODE_MASK)
+  float* loss_part;       // [gridDim.x * 4] (MODE_STORE_SSQ)
+  int* status;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const FwdParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[FWD_STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[FWD_STAGES];
+  __shared__ __align__(8) uint64_t tmem_full_bar[2];
+  __shared__ __align__(8) uint64_t tmem_empty_bar[2];
+  __shared__ __align__(8) uint64_t w_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+  __shared__ float xch[4][2][C];     // lane-31 D_0 and lane-0 D_2 of each epilogue warp
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t w_smem = base;                         // 3 x (192 rows x 128 B)
+  const uint32_t ring = base + FWD_W_BYTES;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < FWD_STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tmem_full_bar[i]), 1); mbar_init(smem_u32(&tmem_empty_bar[i]), 4); }
+    mbar_init(smem_u32(&w_bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc<512>(smem_u32(&tmem_base_slot));
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  volatile int* abortp = &abort_flag;
+
+  const int i0 = static_cast<int>((static_cast<long long>(blockIdx.x) * p.n_items) / gridDim.x);
+  const int i1 = static_cast<int>((static_cast<long long>(blockIdx.x + 1) * p.n_items) / gridDim.x);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(smem_u32(&w_bar), FWD_W_BYTES);
+      for (int u = 0; u < 3; ++u) tma_load_2d(w_smem + u * (192 * 128), &tmW, 0, u * 192, smem_u32(&w_bar));
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int it = i0; it < i1 && ok; ++it) {
+        const int seg = it % p.nseg, rb = (it / p.nseg) % p.nrb, z = it / (p.nseg * p.nrb);
+        for (int r = 0; r < p.RB + 2; ++r) {
+          ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
+          if (!ok) break;
+          const uint32_t fb = smem_u32(&full_bar[stage]);
+          mbar_expect_tx(fb, FWD_ROW_BYTES);
+          tma_load_4d(ring + stage * FWD_ROW_BYTES, &tmX, 0, seg * FWD_PIX - 1, rb * p.RB + r, z, fb);
+          if (++stage == FWD_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t IDESC = make_idesc(128, 192, 0, 0);
+      bool ok = mbar_wait(smem_u32(&w_bar), 0, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
+      int wstage = 0;          // next ring slot to wait for
+      uint32_t wphase = 0;
+      int slot0 = 0;           // ring slot of the current item's row 0
+      int n_out = 0;           // output rows issued so far (accumulator alternation)
+      for (int it = i0; it < i1 && ok; ++it) {
+        int have = 0;
+        for (int i = 0; i < p.RB && ok; ++i) {
+          while (have < i + 3 && ok) {
+            ok = mbar_wait(smem_u32(&full_bar[wstage]), wphase, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
+            if (++wstage == FWD_STAGES) { wstage = 0; wphase ^= 1u; }
+            ++have;
+          }
+          if (!ok) break;
+          const int acc = n_out & 1;
+          const uint32_t acc_phase = (n_out >> 1) & 1u;
+          ok = mbar_wait(smem_u32(&tmem_empty_bar[acc]), acc_phase ^ 1u, abortp, p.status, DEV_TIMEOUT_MMA_TMEM);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + acc * 256;
+#pragma unroll
+          for (int u = 0; u < 3; ++u) {
+            const int slot = (slot0 + i + u) % FWD_STAGES;
+            const uint64_t adesc = make_desc(ring + slot * FWD_ROW_BYTES, 16, 1024);
+            const uint64_t bdesc = make_desc(w_smem + u * (192 * 128), 16, 1024);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) tc_mma_bf16(d_tmem, adesc + k * 2, bdesc + k * 2, IDESC, (u > 0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit(smem_u32(&tmem_full_bar[acc]));
+          tc_commit(smem_u32(&empty_bar[(slot0 + i) % FWD_STAGES]));       // row i has no later reader
+          ++n_out;
+        }
+        if (!ok) break;
+        tc_commit(smem_u32(&empty_bar[(slot0 + p.RB) % FWD_STAGES]));
+        tc_commit(smem_u32(&empty_bar[(slot0 + p.RB + 1) % FWD_STAGES]));
+        slot0 = (slot0 + p.RB + 2) % FWD_STAGES;
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    const int pl = q * 32 + lane;         // TMEM lane = pixel index inside the 128-pixel window
+    int n_out = 0;
+    float ssq = 0.f;
+    bool ok = true;
+    for (int it = i0; it < i1 && ok; ++it) {
+      const int seg = it % p.nseg, rb = (it / p.nseg) % p.nrb, z = it / (p.nseg * p.nrb);
+      const int x = seg * FWD_PIX - 1 + pl;
+      const bool valid = pl >= 1 && pl <= FWD_PIX && x < p.W;
+      for (int i = 0; i < p.RB; ++i, ++n_out) {
+        const int acc = n_out & 1;
+        const uint32_t acc_phase = (n_out >> 1) & 1u;
+        ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+        // all four epilogue warps must agree before they meet at the exchange barrier
+        int bad;
+        asm volatile(
+            "{\n\t.reg .pred pi, po;\n\t"
+            "setp.ne.b32 pi, %1, 0;\n\t"
+            "barrier.cta.red.or.pred po, 1, 128, pi;\n\t"
+            "selp.u32 %0, 1, 0, po;\n\t}"
+            : "=r"(bad) : "r"(ok ? 0 : 1) : "memory");
+        if (bad) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * 256;
+        const int64_t opix = ((static_cast<int64_t>(z) * p.R + rb * p.RB + i + 1) * p.W + x) * C;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          uint32_t d0[32], d1[32], d2[32];
+          tc_ld32(taddr + half * 32, d0);
+          tc_ld32(taddr + 64 + half * 32, d1);
+          tc_ld32(taddr + 128 + half * 32, d2);
+          tc_wait_ld();
+          if (lane == 31) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) xch[q][0][half * 32 + c] = __uint_as_float(d0[c]);
+          }
+          if (lane == 0) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) xch[q][1][half * 32 + c] = __uint_as_float(d2[c]);
+          }
+          asm volatile("barrier.cta.sync 2, 128;" ::: "memory");
+          float y[32];
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            float left = __shfl_up_sync(0xffffffffu, __uint_as_float(d0[c]), 1);
+            float right = __shfl_down_sync(0xffffffffu, __uint_as_float(d2[c]), 1);
+            if (lane == 0) left = q > 0 ? xch[q - 1][0][half * 32 + c] : 0.f;
+            if (lane == 31) right = q < 3 ? xch[q + 1][1][half * 32 + c] : 0.f;
+            y[c] = left + __uint_as_float(d1[c]) + right;
+          }
+          asm volatile("barrier.cta.sync 2, 128;" ::: "memory");      // xch may be rewritten after this
+          if (valid) {
+            if (p.mode == MODE_RELU_STORE) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) y[c] = fmaxf(y[c], 0.f);
+            } else if (p.mode == MODE_STORE_SSQ) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) ssq = fmaf(y[c], y[c], ssq);
+            } else if (p.mask_src) {
+              const uint4* m4 = reinterpret_cast<const uint4*>(p.mask_src + opix + half * 32);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const uint4 mq = m4[j];
+                const uint32_t mw[4] = {mq.x, mq.y, mq.z, mq.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  if (!(bf16_bits_to_f32(mw[e] & 0xFFFFu) > 0.f)) y[j * 8 + 2 * e] = 0.f;
+                  if (!(bf16_bits_to_f32(mw[e] >> 16) > 0.f)) y[j * 8 + 2 * e + 1] = 0.f;
+                }
+              }
+            }
+            uint4* o4 = reinterpret_cast<uint4*>(p.out + opix + half * 32);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint4 o;
+              o.x = pack_bf16x2(y[j * 8 + 0], y[j * 8 + 1]); o.y = pack_bf16x2(y[j * 8 + 2], y[j * 8 + 3]);
+              o.z = pack_bf16x2(y[j * 8 + 4], y[j * 8 + 5]); o.w = pack_bf16x2(y[j * 8 + 6], y[j * 8 + 7]);
+              o4[j] = o;
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+      }
+    }
+    if (p.mode == MODE_STORE_SSQ) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, o);
+      if (lane == 0) p.loss_part[blockIdx.x * 4 + q] = ssq;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc<512>(tmem_base);
+  }
+}
+
+// ------------------------------------------------------------------------------ backward-weight kernel
+struct WgParams {
+  int W, Hs, R, RB, nrb, nseg, n_items;
+  float* part;            // [gridDim.x][9][C][C]
+  int* status;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const WgParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t xfull[WG_XSTAGES], xempty[WG_XSTAGES], yfull[WG_YSTAGES], yempty[WG_YSTAGES];
+  __shared__ __align__(8) uint64_t done_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t xring = base;                                    // slot = 3 chunks (v = 0,1,2)
+  const uint32_t yring = base + WG_XSTAGES * 3 * WG_CHUNK;        // followed by one pad chunk
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < WG_XSTAGES; ++i) { mbar_init(smem_u32(&xfull[i]), 1); mbar_init(smem_u32(&xempty[i]), 1); }
+    for (int i = 0; i < WG_YSTAGES; ++i) { mbar_init(smem_u32(&yfull[i]), 1); mbar_init(smem_u32(&yempty[i]), 1); }
+    mbar_init(smem_u32(&done_bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc<512>(smem_u32(&tmem_base_slot));
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  volatile int* abortp = &abort_flag;
+
+  const int i0 = static_cast<int>((static_cast<long long>(blockIdx.x) * p.n_items) / gridDim.x);
+  const int i1 = static_cast<int>((static_cast<long long>(blockIdx.x + 1) * p.n_items) / gridDim.x);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int xs = 0, ys = 0;
+      uint32_t xph = 0, yph = 0;
+      bool ok = true;
+      for (int it = i0; it < i1 && ok; ++it) {
+        const int seg = it % p.nseg, rb = (it / p.nseg) % p.nrb, z = it / (p.nseg * p.nrb);
+        const int x0 = seg * WG_PIX;
+        // X rows r = 0..RB+1 and dY rows i = 0..RB-1, interleaved in the order the MMAs need them
+        for (int r = 0; r < p.RB + 2 && ok; ++r) {
+          ok = mbar_wait(smem_u32(&xempty[xs]), xph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
+          if (!ok) break;
+          const uint32_t fb = smem_u32(&xfull[xs]);
+          mbar_expect_tx(fb, 3 * WG_CHUNK);
+          for (int v = 0; v < 3; ++v)
+            tma_load_4d(xring + (xs * 3 + v) * WG_CHUNK, &tmX, 0, x0 + v - 1, rb * p.RB + r, z, fb);
+          if (++xs == WG_XSTAGES) { xs = 0; xph ^= 1u; }
+          if (r >= 2) {
+            const int i = r - 2;
+            ok = mbar_wait(smem_u32(&yempty[ys]), yph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
+            if (!ok) break;
+            const uint32_t fy = smem_u32(&yfull[ys]);
+            mbar_expect_tx(fy, WG_CHUNK);
+            tma_load_4d(yring + ys * WG_CHUNK, &tmY, 0, x0, rb * p.RB + i + 1, z, fy);
+            if (++ys == WG_YSTAGES) { ys = 0; yph ^= 1u; }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t IDESC = make_idesc(128, 64, 1, 1);
+      int xw = 0, yw = 0;
+      uint32_t xwph = 0, ywph = 0;
+      int slot0 = 0;
+      bool first = true, ok = true;
+      for (int it = i0; it < i1 && ok; ++it) {
+        const int seg = it % p.nseg;
+        const int npx = min(WG_PIX, p.W - seg * WG_PIX);
+        const int ksteps = (npx + UMMA_K - 1) / UMMA_K;
+        int have = 0;
+        for (int i = 0; i < p.RB && ok; ++i) {
+          while (have < i + 3 && ok) {
+            ok = mbar_wait(smem_u32(&xfull[xw]), xwph, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
+            if (++xw == WG_XSTAGES) { xw = 0; xwph ^= 1u; }
+            ++have;
+          }
+          if (!ok) break;
+          ok = mbar_wait(smem_u32(&yfull[yw]), ywph, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t bdesc = make_desc(yring + yw * WG_CHUNK, WG_CHUNK, 1024);
+#pragma unroll
+          for (int u = 0; u < 3; ++u) {
+            const int slot = (slot0 + i + u) % WG_XSTAGES;
+            const uint32_t xa = xring + slot * 3 * WG_CHUNK;
+            const uint64_t a01 = make_desc(xa, WG_CHUNK, 1024);                 // rows: (v=0 | v=1) x c
+            const uint64_t a2x = make_desc(xa + 2 * WG_CHUNK, WG_CHUNK, 1024);  // rows: (v=2 | whatever follows) x c
+            for (int k = 0; k < ksteps; ++k) {
+              const uint32_t accf = (first && k == 0) ? 0u : 1u;
+              tc_mma_bf16(tmem_base + (u * 2 + 0) * 64, a01 + k * 128, bdesc + k * 128, IDESC, accf);
+              tc_mma_bf16(tmem_base + (u * 2 + 1) * 64, a2x + k * 128, bdesc + k * 128, IDESC, accf);
+            }
+          }
+          first = false;
+          tc_commit(smem_u32(&yempty[yw]));
+          if (++yw == WG_YSTAGES) { yw = 0; ywph ^= 1u; }
+          tc_commit(smem_u32(&xempty[(slot0 + i) % WG_XSTAGES]));
+        }
+        if (!ok) break;
+        tc_commit(smem_u32(&xempty[(slot0 + p.RB) % WG_XSTAGES]));
+        tc_commit(smem_u32(&xempty[(slot0 + p.RB + 1) % WG_XSTAGES]));
+        slot0 = (slot0 + p.RB + 2) % WG_XSTAGES;
+      }
+      if (ok) tc_commit(smem_u32(&done_bar));
+    }
+  } else {
+    const int q = warp & 3;
+    bool ok = true;
+    if (i1 > i0) ok = mbar_wait(smem_u32(&done_bar), 0, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      const int row = q * 32 + lane;                 // TMEM lane: (v-in-pair, c)
+      float* dst_base = p.part + static_cast<int64_t>(blockIdx.x) * 9 * C * C;
+      for (int a = 0; a < 6; ++a) {
+        const int u = a >> 1, pair = a & 1;
+        const int v = pair == 0 ? (row >> 6) : 2;
+        const bool keep = pair == 0 || row < 64;
+        const int c = row & 63;
+        float* dst = dst_base + ((u * 3 + v) * C + c) * C;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r[32];
+          if (i1 > i0) {
+            tc_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * 64 + half * 32, r);
+            tc_wait_ld();
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] = 0u;
+          }
+          if (keep) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              *reinterpret_cast<float4*>(dst + half * 32 + j * 4) =
+                  make_float4(__uint_as_float(r[j * 4]), __uint_as_float(r[j * 4 + 1]), __uint_as_float(r[j * 4 + 2]),
+                              __uint_as_float(r[j * 4 + 3]));
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc<512>(tmem_base);
+  }
+}
+
+// ------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+cudaError_t conv_init() {
+  if (g_encode) return cudaSuccess;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return e;
+  if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+  if ((e = cudaFuncSetAttribute(conv_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM)) != cudaSuccess) return e;
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return cudaSuccess;
+}
+
+// strips tensor [Z][R][W][64] as a 4-D map (c, w, r, z) with a box of `box_w` pixels of one row.
+bool make_strip_map(CUtensorMap* tm, const void* base, int W, int R, int64_t Z, int box_w) {
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(R),
+                              static_cast<cuuint64_t>(Z)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C) * 2, static_cast<cuuint64_t>(W) * C * 2,
+                                 static_cast<cuuint64_t>(R) * W * C * 2};
+  const cuuint32_t box[4] = {static_cast<cuuint32_t>(C), static_cast<cuuint32_t>(box_w), 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool make_weight_map(CUtensorMap* tm, const void* base) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(C), 9 * C};
+  const cuuint64_t strides[1] = {C * 2};
+  const cuuint32_t box[2] = {C, 192};
+  const cuuint32_t estr[2] = {1, 1};
+  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int largest_divisor_at_most(int n, int cap) {
+  for (int d = cap; d >= 1; --d)
+    if (n % d == 0) return d;
+  return 1;
+}
+
+}  // namespace
+
+struct ConvNet {
+  int L = 0, H = 0, W = 0, P_r = 1, Hs = 0, R = 0, num_sms = 148, grid = 148;
+  int64_t B = 0, Z = 0;
+  size_t strip_elems = 0;
+  int* status = nullptr;
+  cudaStream_t stream = nullptr;
+  Profiler* prof = nullptr;
+  std::vector<bf16*> act;            // act[0] = staged input, act[i+1] = stored output of layer i
+  std::vector<bf16*> dY;             // dY[i]: gradient w.r.t. the output of layer i; dY[L-1] == act[L]
+  std::vector<bf16*> K, Wf, Wb;
+  std::vector<float*> dK;
+  std::vector<int> relu;
+  std::vector<CUtensorMap> act_fwd, act_wg, dY_fwd, dY_wg, wf_map, wb_map;
+  float* wpart = nullptr;
+  float* loss_part = nullptr;
+  bf16* scratch_nchw = nullptr;
+  int fwd_RB = 1, wg_RB = 1;
+  int state = 0;                     // 0 idle, 1 forward done, 2 backward (gradients kept), 3 backward (fused)
+};
+
+namespace {
+
+void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w, bf16* out, int mode, const bf16* mask) {
+  FwdParams p;
+  p.W = c->W; p.Hs = c->Hs; p.R = c->R; p.RB = c->fwd_RB; p.nrb = c->Hs / c->fwd_RB;
+  p.nseg = (c->W + FWD_PIX - 1) / FWD_PIX;
+  p.n_items = static_cast<int>(c->Z) * p.nrb * p.nseg;
+  p.mode = mode; p.out = out; p.mask_src = mask; p.loss_part = c->loss_part; p.status = c->status;
+  const int grid = p.n_items < c->grid ? p.n_items : c->grid;
+  if (mode == MODE_STORE_SSQ) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 4, c->stream);
+  const double flops = 2.0 * c->B * c->H * c->W * 9.0 * C * C;
+  c->prof->begin(cls, flops);
+  conv_fwd_kernel<<<grid, NUM_THREADS, FWD_SMEM, c->stream>>>(in, w, p);
+  c->prof->end();
+}
+
+void launch_halo(ConvNet* c, bf16* buf) {
+  if (c->P_r < 2) return;
+  dim3 g(static_cast<unsigned>(c->B * (c->P_r - 1)), 2);
+  c->prof->begin(MBD_K_HALO, 2.0 * 2.0 * c->B * (c->P_r - 1) * c->W * C * 2.0);
+  halo_stage_kernel<<<g, 256, 0, c->stream>>>(buf, c->W, c->P_r, c->Hs);
+  c->prof->end();
+}
+
+void launch_stage_in(ConvNet* c, const bf16* nchw, bf16* strips) {
+  dim3 g((c->W + 31) / 32, c->H, static_cast<unsigned>(c->B));
+  c->prof->begin(MBD_K_HALO, 2.0 * c->B * C * c->H * c->W * 2.0);
+  nchw_to_strips_kernel<<<g, 256, 0, c->stream>>>(nchw, strips, c->H, c->W, c->P_r, c->Hs);
+  c->prof->end();
+}
+
+}  // namespace
+
+mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int max_partials, int num_sms, int* status,
+                       cudaStream_t stream, Profiler* prof, ConvNet** out) {
+  (void)max_partials;
+  if (conv_init() != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
+  const int H = layers[0].H, W = layers[0].W;
+  if (H % P_r != 0) return MBD_E_UNSUPPORTED;      // strips of equal height only
+  ConvNet* c = new (std::nothrow) ConvNet();
+  if (!c) return MBD_E_ALLOC;
+  c->L = L; c->B = B; c->H = H; c->W = W; c->P_r = P_r; c->Hs = H / P_r; c->R = c->Hs + 2; c->Z = B * P_r;
+  c->num_sms = num_sms; c->grid = num_sms; c->status = status; c->stream = stream; c->prof = prof;
+  c->strip_elems = static_cast<size_t>(c->Z) * c->R * W * C;
+  c->fwd_RB = largest_divisor_at_most(c->Hs, 14);
+  c->wg_RB = largest_divisor_at_most(c->Hs, 14);
+  auto alloc = [&](void** p, size_t bytes) -> bool {
+    if (cudaMalloc(p, bytes) != cudaSuccess) { (void)cudaGetLastError(); *p = nullptr; return false; }
+    return cudaMemsetAsync(*p, 0, bytes, stream) == cudaSuccess;
+  };
+  bool ok = true;
+  c->act.assign(L + 1, nullptr); c->dY.assign(L, nullptr);
+  c->K.assign(L, nullptr); c->Wf.assign(L, nullptr); c->Wb.assign(L, nullptr); c->dK.assign(L, nullptr);
+  c->relu.resize(L);
+  for (int i = 0; i <= L && ok; ++i) ok = alloc(reinterpret_cast<void**>(&c->act[i]), c->strip_elems * 2);
+  for (int i = 0; i < L && ok; ++i) {
+    c->relu[i] = layers[i].relu;
+    if (i < L - 1) ok = alloc(reinterpret_cast<void**>(&c->dY[i]), c->strip_elems * 2);
+    else c->dY[i] = c->act[L];                       // half-SSQ loss: dY_L = Y_L
+    ok = ok && alloc(reinterpret_cast<void**>(&c->K[i]), 9 * C * C * 2) && alloc(reinterpret_cast<void**>(&c->Wf[i]), 9 * C * C * 2) &&
+         alloc(reinterpret_cast<void**>(&c->Wb[i]), 9 * C * C * 2) && alloc(reinterpret_cast<void**>(&c->dK[i]), 9 * C * C * 4);
+  }
+  ok = ok && alloc(reinterpret_cast<void**>(&c->wpart), static_cast<size_t>(c->grid) * 9 * C * C * 4);
+  ok = ok && alloc(reinterpret_cast<void**>(&c->loss_part), sizeof(float) * c->grid * 4);
+  ok = ok && alloc(reinterpret_cast<void**>(&c->scratch_nchw), static_cast<size_t>(B) * C * H * W * 2);
+  if (!ok) { conv_destroy(c); return MBD_E_ALLOC; }
+  c->act_fwd.resize(L + 1); c->act_wg.resize(L + 1); c->dY_fwd.resize(L); c->dY_wg.resize(L);
+  c->wf_map.resize(L); c->wb_map.resize(L);
+  for (int i = 0; i <= L && ok; ++i)
+    ok = make_strip_map(&c->act_fwd[i], c->act[i], W, c->R, c->Z, 128) && make_strip_map(&c->act_wg[i], c->act[i], W, c->R, c->Z, WG_PIX);
+  for (int i = 0; i < L && ok; ++i)
+    ok = make_strip_map(&c->dY_fwd[i], c->dY[i], W, c->R, c->Z, 128) && make_strip_map(&c->dY_wg[i], c->dY[i], W, c->R, c->Z, WG_PIX) &&
+         make_weight_map(&c->wf_map[i], c->Wf[i]) && make_weight_map(&c->wb_map[i], c->Wb[i]);
+  if (!ok) { conv_destroy(c); return MBD_E_CUDA; }
+  if (cudaStreamSynchronize(stream) != cudaSuccess) { conv_destroy(c); return MBD_E_CUDA; }
+  *out = c;
+  return MBD_OK;
+}
+
+void conv_destroy(ConvNet* c) {
+  if (!c) return;
+  for (size_t i = 0; i < c->act.size(); ++i) cudaFree(c->act[i]);
+  for (int i = 0; i + 1 < c->L; ++i) cudaFree(c->dY[i]);
+  for (int i = 0; i < c->L; ++i) { cudaFree(c->K[i]); cudaFree(c->Wf[i]); cudaFree(c->Wb[i]); cudaFree(c->dK[i]); }
+  cudaFree(c->wpart); cudaFree(c->loss_part); cudaFree(c->scratch_nchw);
+  (void)cudaGetLastError();
+  delete c;
+}
+
+mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev) {
+  if (cudaMemcpyAsync(c->K[layer], K_dev, 9 * C * C * 2, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) return MBD_E_CUDA;
+  return MBD_OK;
+}
+
+mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev) {
+  if (cudaMemcpyAsync(K_dev, c->K[layer], 9 * C * C * 2, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) return MBD_E_CUDA;
+  return MBD_OK;
+}
+
+size_t conv_input_bytes(const ConvNet* c) { return static_cast<size_t>(c->B) * C * c->H * c->W * 2; }
+
+mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
+  // stage the input into strips (with its halo rows) and pack the current weights
+  launch_stage_in(c, static_cast<const bf16*>(X_nchw), c->act[0]);
+  for (int i = 0; i < c->L; ++i) {
+    c->prof->begin(MBD_K_OTHER, 9.0 * C * C * 6.0);
+    pack_weights_kernel<<<(9 * C * C + 255) / 256, 256, 0, c->stream>>>(c->K[i], c->Wf[i], c->Wb[i]);
+    c->prof->end();
+  }
+  for (int i = 0; i < c->L; ++i) {
+    const bool last = i == c->L - 1;
+    if (i > 0) launch_halo(c, c->act[i]);            // forward halo exchange (first halo term of Eq. 7)
+    launch_fwd(c, MBD_K_CONV_FWD, c->act_fwd[i], c->wf_map[i], c->act[i + 1],
+               last ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK), nullptr);
+  }
+  if (loss_sum_dev) {
+    c->prof->begin(MBD_K_OTHER, c->grid * 16.0);
+    if (sum_f32_launch(c->loss_part, c->grid * 4, 0.5f, loss_sum_dev, c->stream) != cudaSuccess) return MBD_E_CUDA;
+    c->prof->end();
+  }
+  if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
+  c->state = 1;
+  return MBD_OK;
+}
+
+mbd_status conv_backward(ConvNet* c, float fused_eta) {
+  const bool fused = fused_eta > 0.f;
+  const float scale = -fused_eta / static_cast<float>(c->B);
+  for (int i = c->L - 1; i >= 0; --i) {
+    if (i > 0) {
+      // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0]
+      launch_halo(c, c->dY[i]);
+      launch_fwd(c, MBD_K_CONV_BWD_DATA, c->dY_fwd[i], c->wb_map[i], c->dY[i - 1], MODE_MASK,
+                 c->relu[i - 1] ? c->act[i] : nullptr);
+    }
+    WgParams p;
+    p.W = c->W; p.Hs = c->Hs; p.R = c->R; p.RB = c->wg_RB; p.nrb = c->Hs / c->wg_RB;
+    p.nseg = (c->W + WG_PIX - 1) / WG_PIX;
+    p.n_items = static_cast<int>(c->Z) * p.nrb * p.nseg;
+    p.part = c->wpart; p.status = c->status;
+    const int grid = p.n_items < c->grid ? p.n_items : c->grid;
+    c->prof->begin(MBD_K_CONV_BWD_WEIGHT, 2.0 * c->B * c->H * c->W * 9.0 * C * C);
+    conv_wgrad_kernel<<<grid, NUM_THREADS, WG_SMEM, c->stream>>>(c->act_wg[i], c->dY_wg[i], p);
+    c->prof->end();
+    c->prof->begin(MBD_K_REDUCE, (grid + 1.0) * 9 * C * C * 4.0);
+    wgrad_finish_kernel<<<(9 * C * C + 255) / 256, 256, 0, c->stream>>>(c->wpart, grid, fused ? nullptr : c->dK[i],
+                                                                      fused ? c->K[i] : nullptr, scale);
+    c->prof->end();
+  }
+  if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
+  c->state = fused ? 3 : 2;
+  return MBD_OK;
+}
+
+mbd_status conv_sgd_step(ConvNet* c, float eta) {
+  const float scale = -eta / static_cast<float>(c->B);
+  for (int i = 0; i < c->L; ++i) {
+    c->prof->begin(MBD_K_SGD, 9.0 * C * C * 8.0);
+    if (sgd_update_launch(c->K[i], 1, c->dK[i], 9 * C * C, scale, c->num_sms, c->stream) != cudaSuccess) return MBD_E_CUDA;
+    c->prof->end();
+  }
+  return MBD_OK;
+}
+
+mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t bytes) {
+  const size_t nchw_bytes = conv_input_bytes(c);
+  if (which == MBD_T_DW) {
+    if (layer < 0 || layer >= c->L || bytes != 9 * C * C * 4) return MBD_E_INVALID;
+    if (cudaMemcpyAsync(dst, c->dK[layer], bytes, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) return MBD_E_CUDA;
+    return MBD_OK;
+  }
+  if (which == MBD_T_PARTIALS) {
+    if (bytes > static_cast<size_t>(c->grid) * 9 * C * C * 4) return MBD_E_INVALID;
+    if (cudaMemcpyAsync(dst, c->wpart, bytes, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) return MBD_E_CUDA;
+    return MBD_OK;
+  }
+  if (layer < 0 || layer >= c->L || bytes != nchw_bytes) return MBD_E_INVALID;
+  const bf16* src = which == MBD_T_ACT ? c->act[layer + 1] : which == MBD_T_DY ? c->dY[layer] : nullptr;
+  if (!src) return MBD_E_INVALID;
+  dim3 g((c->W + 31) / 32, c->H, static_cast<unsigned>(c->B));
+  strips_to_nchw_kernel<<<g, 256, 0, c->stream>>>(src, static_cast<bf16*>(dst), c->H, c->W, c->P_r, c->Hs);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+mbd_status conv_set_tensor(ConvNet* c, int which, int layer, const void* src, size_t bytes) {
+  if (layer < 0 || layer >= c->L || bytes != conv_input_bytes(c)) return MBD_E_INVALID;
+  bf16* dst = which == MBD_T_ACT ? c->act[layer + 1] : which == MBD_T_DY ? c->dY[layer] : nullptr;
+  if (!dst) return MBD_E_INVALID;
+  dim3 g((c->W + 31) / 32, c->H, static_cast<unsigned>(c->B));
+  nchw_to_strips_kernel<<<g, 256, 0, c->stream>>>(static_cast<const bf16*>(src), dst, c->H, c->W, c->P_r, c->Hs);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
 }  // namespace mbd

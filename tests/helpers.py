@@ -135,3 +135,72 @@ def compare_fc_step(g, o, tol, fused=False, tol_below_relu=None):
         assert np.abs(g["new_b"][i] - ref_b).max() <= tol * max(1.0, np.abs(ref_b).max()), f"b_new[{i}]"
     assert not bad, "rel. Frobenius error too large for %s: %s" % (bad, "; ".join(report))
     return worst
+
+
+# ---------------------------------------------------------------------------
+# convolution workloads
+# ---------------------------------------------------------------------------
+def oracle_conv_step(w, inp, strips=None):
+    """fp64 oracle step for a domain-parallel conv workload (NCHW); stored activations are
+    rounded to bf16 like the device's.  `strips` = P_r runs the strip / halo formulation."""
+    from oracle import mbd_oracle as O
+    layers = [O.Conv3x3(k.astype(np.float64), relu=True) for k in inp.Ws]
+    X = inp.X.astype(np.float64)
+    if strips is None:
+        return O.train_step(layers, X, None, "half_ssq", w.eta, store=bf16_store)
+    return O.train_step_blocked(layers, X, None, "half_ssq", w.eta, strips, 1, store=bf16_store)
+
+
+def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None):
+    import torch
+    from paper_1712_04432_b200 import mbd
+    C_, H, Wd = w.dims
+    L = w.n_layers
+    net = mbd.Net(mbd.conv_layers(L, C_, H, Wd), w.B, P_r, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+    for i in range(L):
+        net.set_weights(i, to_dev(inp.Ws[i], True))
+    X = to_dev(inp.X, True)
+    J = torch.zeros(1, dtype=torch.float32, device="cuda")
+    out = {}
+    net.forward(X, None, J)
+    out["act"] = [to_np(net.get_tensor(mbd.T_ACT, i)) for i in range(L)]
+    if force_acts is not None:
+        for i in range(L - 1):
+            net.set_tensor(mbd.T_ACT, i, to_dev(force_acts[i], True))
+    if fused:
+        net.backward(w.eta)
+    else:
+        net.backward(0.0)
+        out["dW"] = [to_np(net.get_tensor(mbd.T_DW, i)) for i in range(L)]
+        net.sgd_step(w.eta)
+    net.poll()
+    out["J"] = float(J.item())
+    out["dY"] = [to_np(net.get_tensor(mbd.T_DY, i)) for i in range(L)]
+    out["new_W"] = [to_np(net.get_weights(i)) for i in range(L)]
+    out["launches"] = net.launch_count
+    net.close()
+    return out
+
+
+def compare_conv_step(g, o, tol, fused=False, tol_below_relu=None):
+    L = len(o["Ys"])
+    report, bad = [], []
+    if tol_below_relu is None:
+        tol_below_relu = tol
+
+    def chk(name, got, ref, t):
+        e = rel_fro(got, ref)
+        report.append(f"{name}: {e:.3e}")
+        if e > t:
+            bad.append(name)
+
+    assert abs(g["J"] - o["J"]) <= tol * abs(o["J"]), (g["J"], o["J"])
+    for i in range(L):
+        chk(f"Y[{i}]", g["act"][i], o["Ys"][i] if i == L - 1 else o["Xs"][i + 1], tol)
+        tg = tol if i == L - 1 else tol_below_relu
+        chk(f"dY[{i}]", g["dY"][i], o["dYs"][i], tg)
+        if not fused:
+            chk(f"dK[{i}]", g["dW"][i], o["dWs"][i], tg)
+        chk(f"K_new[{i}]", g["new_W"][i], o["new_W"][i], tol)
+    assert not bad, "rel. Frobenius error too large for %s: %s" % (bad, "; ".join(report))
+    return report

@@ -1,0 +1,77 @@
+"""Parity of the domain-parallel 3x3 convolution step (strips + halo rows) with the fp64
+oracle, through the C ABI: forward outputs, the back-propagated gradient, the kernel gradients
+and the updated kernels, for every strip count."""
+import numpy as np
+import pytest
+
+from paper_1712_04432_b200 import inputs as I
+from tests.helpers import compare_conv_step, gpu_conv_step, oracle_conv_step, rel_fro
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+TOL_FREE = 5e-2      # free-running gradients below a ReLU (see test_parity_fc.py)
+
+
+def stored_hidden(o):
+    return [np.ascontiguousarray(x, np.float32) for x in o["Xs"][1:]]
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    w = I.conv_workload(64, 8, 40, 2, name="conv_tiny")
+    inp = I.make_inputs(w, seed=21)
+    return w, inp, oracle_conv_step(w, inp)
+
+
+@pytest.mark.parametrize("P_r", [1, 2, 4, 8])
+def test_tiny_all_strip_counts(tiny, P_r):
+    w, inp, o = tiny
+    g = gpu_conv_step(w, inp, P_r, force_acts=stored_hidden(o))
+    compare_conv_step(g, o, TOL)
+    g = gpu_conv_step(w, inp, P_r)
+    compare_conv_step(g, o, TOL, tol_below_relu=TOL_FREE)
+
+
+@pytest.fixture(scope="module")
+def ragged():
+    # two forward segments (126 + 4 pixels), three backward-weight segments (64 + 64 + 2),
+    # 28 rows (row blocks of 14 or 7 or 4), three images
+    w = I.conv_workload(64, 28, 130, 3, name="conv_ragged")
+    inp = I.make_inputs(w, seed=22)
+    return w, inp, oracle_conv_step(w, inp)
+
+
+@pytest.mark.parametrize("P_r", [1, 2, 7])
+@pytest.mark.parametrize("fused", [False, True])
+def test_ragged_shapes(ragged, P_r, fused):
+    w, inp, o = ragged
+    g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o))
+    compare_conv_step(g, o, TOL, fused)
+
+
+def test_strip_oracle_agrees(ragged):
+    w, inp, _ = ragged
+    ob = oracle_conv_step(w, inp, strips=4)
+    g = gpu_conv_step(w, inp, 4, force_acts=stored_hidden(ob))
+    compare_conv_step(g, ob, TOL)
+
+
+def test_three_layers_and_reproducibility():
+    w = I.conv_workload(64, 12, 64, 2, n_layers=3, name="conv3")
+    inp = I.make_inputs(w, seed=23)
+    o = oracle_conv_step(w, inp)
+    a = gpu_conv_step(w, inp, 3, fused=True, force_acts=stored_hidden(o))
+    compare_conv_step(a, o, TOL, fused=True)
+    b = gpu_conv_step(w, inp, 3, fused=True, force_acts=stored_hidden(o))
+    for i in range(3):
+        assert np.array_equal(a["new_W"][i], b["new_W"][i]) and np.array_equal(a["dY"][i], b["dY"][i])
+
+
+@pytest.mark.parametrize("P_r", [1, 8])
+def test_full_resolution_two_images(P_r):
+    # the 224 x 224 geometry of the large workload (strips of 224 / 28 rows), two images
+    w = I.conv_workload(64, 224, 224, 2, name="conv_224")
+    inp = I.make_inputs(w, seed=24)
+    o = oracle_conv_step(w, inp)
+    g = gpu_conv_step(w, inp, P_r, force_acts=stored_hidden(o))
+    compare_conv_step(g, o, TOL)
