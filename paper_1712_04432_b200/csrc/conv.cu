@@ -38,15 +38,17 @@ namespace {
 
 constexpr int C = 64;                 // channels in and out
 constexpr int FWD_PIX = 126;          // output pixels per forward tile (lanes 1..126 of 128)
-constexpr int FWD_STAGES = 8;         // ring of input rows, 16 KB each
+constexpr int FWD_STAGES = 5;         // ring of input rows, 16 KB each (3 live + 2 in flight)
 constexpr int FWD_ROW_BYTES = 128 * 128;
 constexpr int FWD_W_BYTES = 3 * 192 * 128;   // stacked taps, 72 KB
-constexpr int FWD_SMEM = FWD_W_BYTES + FWD_STAGES * FWD_ROW_BYTES + 1024;
+constexpr int FWD_XCH_BYTES = 2 * 2 * 128 * 32 * 4;   // per channel half: D_0 and D_2 planes, 128 pixels x 32 floats
+constexpr int FWD_SMEM = FWD_W_BYTES + FWD_STAGES * FWD_ROW_BYTES + FWD_XCH_BYTES + 1024;
+constexpr int FWD_THREADS = 320;      // producer warp, MMA warp, 8 epilogue warps
 constexpr int WG_PIX = 64;            // pixels (reduction length) per backward-weight block
-constexpr int WG_XSTAGES = 6;         // X rows: 3 shifted copies of 8 KB each
-constexpr int WG_YSTAGES = 4;         // dY rows: 8 KB each
+constexpr int WG_XSTAGES = 4;         // X rows: 3 shifted copies of 8 KB each, each row used once
+constexpr int WG_YSTAGES = 6;         // dY rows: 8 KB each, plus 2 mirror slots
 constexpr int WG_CHUNK = WG_PIX * 128;
-constexpr int WG_SMEM = WG_XSTAGES * 3 * WG_CHUNK + WG_YSTAGES * WG_CHUNK + WG_CHUNK /*junk pad*/ + 1024;
+constexpr int WG_SMEM = WG_XSTAGES * 3 * WG_CHUNK + (WG_YSTAGES + 2) * WG_CHUNK + 1024;
 constexpr int NUM_THREADS = 192;
 
 enum { MODE_RELU_STORE = 0, MODE_STORE_SSQ = 1, MODE_MASK = 2 };
@@ -161,11 +163,11 @@ struct FwdParams {
   int mode;
   bf16* out;              // strips
   const bf16* mask_src;   // strips (MODE_MASK)
-  float* loss_part;       // [gridDim.x * 4] (MODE_STORE_SSQ)
+  float* loss_part;       // [gridDim.x * 8] (MODE_STORE_SSQ)
   int* status;
 };
 
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(FWD_THREADS, 1)
 conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const FwdParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[FWD_STAGES];
@@ -175,16 +177,17 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   __shared__ __align__(8) uint64_t w_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
-  __shared__ float xch[4][2][C];     // lane-31 D_0 and lane-0 D_2 of each epilogue warp
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t w_smem = base;                         // 3 x (192 rows x 128 B)
   const uint32_t ring = base + FWD_W_BYTES;
+  float* xch_base = reinterpret_cast<float*>(smem_raw + (base - smem_u32(smem_raw)) + FWD_W_BYTES +
+                                             FWD_STAGES * FWD_ROW_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < FWD_STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tmem_full_bar[i]), 1); mbar_init(smem_u32(&tmem_empty_bar[i]), 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tmem_full_bar[i]), 1); mbar_init(smem_u32(&tmem_empty_bar[i]), 8); }
     mbar_init(smem_u32(&w_bar), 1);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -260,8 +263,14 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       }
     }
   } else {
+    // Eight epilogue warps: warp & 3 selects the TMEM lane quarter (32 pixels), (warp - 2) >> 2 the
+    // channel half.  The horizontal shift goes through shared memory: D_0 of pixel p is written
+    // to row p + 1, D_2 of pixel p to row p - 1, and every thread reads back its own row.
     const int q = warp & 3;
+    const int half = (warp - 2) >> 2;
     const int pl = q * 32 + lane;         // TMEM lane = pixel index inside the 128-pixel window
+    float* s0 = xch_base + half * (2 * 128 * 32);
+    float* s2 = s0 + 128 * 32;
     int n_out = 0;
     float ssq = 0.f;
     bool ok = true;
@@ -273,83 +282,92 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const int acc = n_out & 1;
         const uint32_t acc_phase = (n_out >> 1) & 1u;
         ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
-        // all four epilogue warps must agree before they meet at the exchange barrier
+        // all epilogue warps must agree before they meet at the exchange barriers
         int bad;
         asm volatile(
             "{\n\t.reg .pred pi, po;\n\t"
             "setp.ne.b32 pi, %1, 0;\n\t"
-            "barrier.cta.red.or.pred po, 1, 128, pi;\n\t"
+            "barrier.cta.red.or.pred po, 1, 256, pi;\n\t"
             "selp.u32 %0, 1, 0, po;\n\t}"
             : "=r"(bad) : "r"(ok ? 0 : 1) : "memory");
         if (bad) { ok = false; break; }
         tc_fence_after();
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * 256;
-        const int64_t opix = ((static_cast<int64_t>(z) * p.R + rb * p.RB + i + 1) * p.W + x) * C;
-#pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-          uint32_t d0[32], d1[32], d2[32];
-          tc_ld32(taddr + half * 32, d0);
-          tc_ld32(taddr + 64 + half * 32, d1);
-          tc_ld32(taddr + 128 + half * 32, d2);
-          tc_wait_ld();
-          if (lane == 31) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) xch[q][0][half * 32 + c] = __uint_as_float(d0[c]);
-          }
-          if (lane == 0) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) xch[q][1][half * 32 + c] = __uint_as_float(d2[c]);
-          }
-          asm volatile("barrier.cta.sync 2, 128;" ::: "memory");
-          float y[32];
-#pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            float left = __shfl_up_sync(0xffffffffu, __uint_as_float(d0[c]), 1);
-            float right = __shfl_down_sync(0xffffffffu, __uint_as_float(d2[c]), 1);
-            if (lane == 0) left = q > 0 ? xch[q - 1][0][half * 32 + c] : 0.f;
-            if (lane == 31) right = q < 3 ? xch[q + 1][1][half * 32 + c] : 0.f;
-            y[c] = left + __uint_as_float(d1[c]) + right;
-          }
-          asm volatile("barrier.cta.sync 2, 128;" ::: "memory");      // xch may be rewritten after this
-          if (valid) {
-            if (p.mode == MODE_RELU_STORE) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c) y[c] = fmaxf(y[c], 0.f);
-            } else if (p.mode == MODE_STORE_SSQ) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c) ssq = fmaf(y[c], y[c], ssq);
-            } else if (p.mask_src) {
-              const uint4* m4 = reinterpret_cast<const uint4*>(p.mask_src + opix + half * 32);
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const uint4 mq = m4[j];
-                const uint32_t mw[4] = {mq.x, mq.y, mq.z, mq.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  if (!(bf16_bits_to_f32(mw[e] & 0xFFFFu) > 0.f)) y[j * 8 + 2 * e] = 0.f;
-                  if (!(bf16_bits_to_f32(mw[e] >> 16) > 0.f)) y[j * 8 + 2 * e + 1] = 0.f;
-                }
-              }
-            }
-            uint4* o4 = reinterpret_cast<uint4*>(p.out + opix + half * 32);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              uint4 o;
-              o.x = pack_bf16x2(y[j * 8 + 0], y[j * 8 + 1]); o.y = pack_bf16x2(y[j * 8 + 2], y[j * 8 + 3]);
-              o.z = pack_bf16x2(y[j * 8 + 4], y[j * 8 + 5]); o.w = pack_bf16x2(y[j * 8 + 6], y[j * 8 + 7]);
-              o4[j] = o;
-            }
-          }
-        }
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * 256 + half * 32;
+        const int64_t opix = ((static_cast<int64_t>(z) * p.R + rb * p.RB + i + 1) * p.W + x) * C + half * 32;
+        uint32_t d0[32], d1[32], d2[32];
+        tc_ld32(taddr, d0);
+        tc_ld32(taddr + 64, d1);
+        tc_ld32(taddr + 128, d2);
+        tc_wait_ld();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+        if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));    // accumulator is in registers now
+        if (pl < 127) {
+          float4* row = reinterpret_cast<float4*>(s0 + (pl + 1) * 32);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            row[j ^ ((pl + 1) & 7)] = make_float4(__uint_as_float(d0[4 * j]), __uint_as_float(d0[4 * j + 1]),
+                                                  __uint_as_float(d0[4 * j + 2]), __uint_as_float(d0[4 * j + 3]));
+        }
+        if (pl > 0) {
+          float4* row = reinterpret_cast<float4*>(s2 + (pl - 1) * 32);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            row[j ^ ((pl - 1) & 7)] = make_float4(__uint_as_float(d2[4 * j]), __uint_as_float(d2[4 * j + 1]),
+                                                  __uint_as_float(d2[4 * j + 2]), __uint_as_float(d2[4 * j + 3]));
+        }
+        if (half == 0) asm volatile("barrier.cta.sync 2, 128;" ::: "memory");
+        else asm volatile("barrier.cta.sync 3, 128;" ::: "memory");
+        float y[32];
+        {
+          const float4* r0 = reinterpret_cast<const float4*>(s0 + pl * 32);
+          const float4* r2 = reinterpret_cast<const float4*>(s2 + pl * 32);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float4 a = r0[j ^ (pl & 7)], b = r2[j ^ (pl & 7)];
+            y[4 * j + 0] = a.x + __uint_as_float(d1[4 * j + 0]) + b.x;
+            y[4 * j + 1] = a.y + __uint_as_float(d1[4 * j + 1]) + b.y;
+            y[4 * j + 2] = a.z + __uint_as_float(d1[4 * j + 2]) + b.z;
+            y[4 * j + 3] = a.w + __uint_as_float(d1[4 * j + 3]) + b.w;
+          }
+        }
+        if (half == 0) asm volatile("barrier.cta.sync 2, 128;" ::: "memory");   // planes may be rewritten after this
+        else asm volatile("barrier.cta.sync 3, 128;" ::: "memory");
+        if (valid) {
+          if (p.mode == MODE_RELU_STORE) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) y[c] = fmaxf(y[c], 0.f);
+          } else if (p.mode == MODE_STORE_SSQ) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) ssq = fmaf(y[c], y[c], ssq);
+          } else if (p.mask_src) {
+            const uint4* m4 = reinterpret_cast<const uint4*>(p.mask_src + opix);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint4 mq = m4[j];
+              const uint32_t mw[4] = {mq.x, mq.y, mq.z, mq.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                if (!(bf16_bits_to_f32(mw[e] & 0xFFFFu) > 0.f)) y[j * 8 + 2 * e] = 0.f;
+                if (!(bf16_bits_to_f32(mw[e] >> 16) > 0.f)) y[j * 8 + 2 * e + 1] = 0.f;
+              }
+            }
+          }
+          uint4* o4 = reinterpret_cast<uint4*>(p.out + opix);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint4 o;
+            o.x = pack_bf16x2(y[j * 8 + 0], y[j * 8 + 1]); o.y = pack_bf16x2(y[j * 8 + 2], y[j * 8 + 3]);
+            o.z = pack_bf16x2(y[j * 8 + 4], y[j * 8 + 5]); o.w = pack_bf16x2(y[j * 8 + 6], y[j * 8 + 7]);
+            o4[j] = o;
+          }
+        }
       }
     }
     if (p.mode == MODE_STORE_SSQ) {
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, o);
-      if (lane == 0) p.loss_part[blockIdx.x * 4 + q] = ssq;
+      if (lane == 0) p.loss_part[blockIdx.x * 8 + (warp - 2)] = ssq;
     }
   }
 
@@ -369,23 +387,29 @@ struct WgParams {
   int* status;
 };
 
+// One X row (three shifted copies) meets the up to three dY rows it contributes to in ONE
+// instruction group: B = [dY_{r-2} | dY_{r-1} | dY_r] (N = 64 per row, rows adjacent in the dY
+// ring), A = (shift 0 | shift 1) and (shift 2 | don't care), so tap (u, v) accumulates in
+// TMEM lanes (v, c) and columns (2 - u, o).  The dY ring mirrors its first two slots behind
+// its last one so that a window of three rows is always contiguous in shared memory.
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const WgParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t xfull[WG_XSTAGES], xempty[WG_XSTAGES], yfull[WG_YSTAGES], yempty[WG_YSTAGES];
-  __shared__ __align__(8) uint64_t done_bar;
+  __shared__ __align__(8) uint64_t done_bar, init_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t xring = base;                                    // slot = 3 chunks (v = 0,1,2)
-  const uint32_t yring = base + WG_XSTAGES * 3 * WG_CHUNK;        // followed by one pad chunk
+  const uint32_t xring = base;                                    // slot = 3 chunks (shift 0,1,2)
+  const uint32_t yring = base + WG_XSTAGES * 3 * WG_CHUNK;        // WG_YSTAGES slots + 2 mirror slots
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < WG_XSTAGES; ++i) { mbar_init(smem_u32(&xfull[i]), 1); mbar_init(smem_u32(&xempty[i]), 1); }
     for (int i = 0; i < WG_YSTAGES; ++i) { mbar_init(smem_u32(&yfull[i]), 1); mbar_init(smem_u32(&yempty[i]), 1); }
     mbar_init(smem_u32(&done_bar), 1);
+    mbar_init(smem_u32(&init_bar), 4);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -407,8 +431,17 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       for (int it = i0; it < i1 && ok; ++it) {
         const int seg = it % p.nseg, rb = (it / p.nseg) % p.nrb, z = it / (p.nseg * p.nrb);
         const int x0 = seg * WG_PIX;
-        // X rows r = 0..RB+1 and dY rows i = 0..RB-1, interleaved in the order the MMAs need them
         for (int r = 0; r < p.RB + 2 && ok; ++r) {
+          if (r < p.RB) {
+            ok = mbar_wait(smem_u32(&yempty[ys]), yph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
+            if (!ok) break;
+            const uint32_t fy = smem_u32(&yfull[ys]);
+            const bool mirrored = ys < 2;
+            mbar_expect_tx(fy, mirrored ? 2 * WG_CHUNK : WG_CHUNK);
+            tma_load_4d(yring + ys * WG_CHUNK, &tmY, 0, x0, rb * p.RB + r + 1, z, fy);
+            if (mirrored) tma_load_4d(yring + (WG_YSTAGES + ys) * WG_CHUNK, &tmY, 0, x0, rb * p.RB + r + 1, z, fy);
+            if (++ys == WG_YSTAGES) { ys = 0; yph ^= 1u; }
+          }
           ok = mbar_wait(smem_u32(&xempty[xs]), xph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
           if (!ok) break;
           const uint32_t fb = smem_u32(&xfull[xs]);
@@ -416,90 +449,87 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           for (int v = 0; v < 3; ++v)
             tma_load_4d(xring + (xs * 3 + v) * WG_CHUNK, &tmX, 0, x0 + v - 1, rb * p.RB + r, z, fb);
           if (++xs == WG_XSTAGES) { xs = 0; xph ^= 1u; }
-          if (r >= 2) {
-            const int i = r - 2;
-            ok = mbar_wait(smem_u32(&yempty[ys]), yph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
-            if (!ok) break;
-            const uint32_t fy = smem_u32(&yfull[ys]);
-            mbar_expect_tx(fy, WG_CHUNK);
-            tma_load_4d(yring + ys * WG_CHUNK, &tmY, 0, x0, rb * p.RB + i + 1, z, fy);
-            if (++ys == WG_YSTAGES) { ys = 0; yph ^= 1u; }
-          }
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t IDESC = make_idesc(128, 64, 1, 1);
-      int xw = 0, yw = 0;
+      int xw = 0, yw = 0;            // next slots to wait for
       uint32_t xwph = 0, ywph = 0;
-      int slot0 = 0;
-      bool first = true, ok = true;
+      int y_slot0 = 0;               // ring slot of the current item's dY row 0
+      bool ok = mbar_wait(smem_u32(&init_bar), 0, abortp, p.status, DEV_TIMEOUT_MMA_TMEM);   // accumulators zeroed
+      tc_fence_after();
       for (int it = i0; it < i1 && ok; ++it) {
         const int seg = it % p.nseg;
         const int npx = min(WG_PIX, p.W - seg * WG_PIX);
         const int ksteps = (npx + UMMA_K - 1) / UMMA_K;
-        int have = 0;
-        for (int i = 0; i < p.RB && ok; ++i) {
-          while (have < i + 3 && ok) {
-            ok = mbar_wait(smem_u32(&xfull[xw]), xwph, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
-            if (++xw == WG_XSTAGES) { xw = 0; xwph ^= 1u; }
-            ++have;
+        int yhave = 0;
+        for (int r = 0; r < p.RB + 2 && ok; ++r) {
+          const int i_hi = min(r, p.RB - 1), i_lo = max(0, r - 2);
+          while (yhave <= i_hi && ok) {
+            ok = mbar_wait(smem_u32(&yfull[yw]), ywph, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
+            if (++yw == WG_YSTAGES) { yw = 0; ywph ^= 1u; }
+            ++yhave;
           }
           if (!ok) break;
-          ok = mbar_wait(smem_u32(&yfull[yw]), ywph, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
+          ok = mbar_wait(smem_u32(&xfull[xw]), xwph, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
           if (!ok) break;
           tc_fence_after();
-          const uint64_t bdesc = make_desc(yring + yw * WG_CHUNK, WG_CHUNK, 1024);
-#pragma unroll
-          for (int u = 0; u < 3; ++u) {
-            const int slot = (slot0 + i + u) % WG_XSTAGES;
-            const uint32_t xa = xring + slot * 3 * WG_CHUNK;
-            const uint64_t a01 = make_desc(xa, WG_CHUNK, 1024);                 // rows: (v=0 | v=1) x c
-            const uint64_t a2x = make_desc(xa + 2 * WG_CHUNK, WG_CHUNK, 1024);  // rows: (v=2 | whatever follows) x c
-            for (int k = 0; k < ksteps; ++k) {
-              const uint32_t accf = (first && k == 0) ? 0u : 1u;
-              tc_mma_bf16(tmem_base + (u * 2 + 0) * 64, a01 + k * 128, bdesc + k * 128, IDESC, accf);
-              tc_mma_bf16(tmem_base + (u * 2 + 1) * 64, a2x + k * 128, bdesc + k * 128, IDESC, accf);
-            }
+          const int n = i_hi - i_lo + 1;                       // dY rows in the window
+          const int b0 = 2 - (r - i_lo);                       // column block of the first of them
+          const uint32_t idesc = make_idesc(128, 64 * n, 1, 1);
+          const int ys0 = (y_slot0 + i_lo) % WG_YSTAGES;       // window may run into the mirror slots
+          const uint64_t bdesc = make_desc(yring + ys0 * WG_CHUNK, WG_CHUNK, 1024);
+          const uint32_t xa = xring + xw * 3 * WG_CHUNK;
+          const uint64_t a01 = make_desc(xa, WG_CHUNK, 1024);                 // lanes: (shift 0 | shift 1) x c
+          const uint64_t a2x = make_desc(xa + 2 * WG_CHUNK, WG_CHUNK, 1024);  // lanes: (shift 2 | don't care) x c
+          for (int k = 0; k < ksteps; ++k) {
+            tc_mma_bf16(tmem_base + b0 * 64, a01 + k * 128, bdesc + k * 128, idesc, 1u);
+            tc_mma_bf16(tmem_base + 256 + b0 * 64, a2x + k * 128, bdesc + k * 128, idesc, 1u);
           }
-          first = false;
-          tc_commit(smem_u32(&yempty[yw]));
-          if (++yw == WG_YSTAGES) { yw = 0; ywph ^= 1u; }
-          tc_commit(smem_u32(&xempty[(slot0 + i) % WG_XSTAGES]));
+          tc_commit(smem_u32(&xempty[xw]));
+          if (++xw == WG_XSTAGES) { xw = 0; xwph ^= 1u; }
+          if (r >= 2) tc_commit(smem_u32(&yempty[(y_slot0 + r - 2) % WG_YSTAGES]));   // dY row r-2 has no later reader
         }
-        if (!ok) break;
-        tc_commit(smem_u32(&xempty[(slot0 + p.RB) % WG_XSTAGES]));
-        tc_commit(smem_u32(&xempty[(slot0 + p.RB + 1) % WG_XSTAGES]));
-        slot0 = (slot0 + p.RB + 2) % WG_XSTAGES;
+        y_slot0 = (y_slot0 + p.RB) % WG_YSTAGES;
       }
       if (ok) tc_commit(smem_u32(&done_bar));
     }
   } else {
     const int q = warp & 3;
-    bool ok = true;
-    if (i1 > i0) ok = mbar_wait(smem_u32(&done_bar), 0, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+    {   // zero both accumulators (columns 0..191 and 256..447) before the first MMA
+      for (int cb = 0; cb < 12; ++cb) {
+        const uint32_t col = (cb < 6 ? 0 : 256) + (cb % 6) * 32;
+        asm volatile(
+            "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+            "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
+            "%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+            ::"r"(lane_base + col), "r"(0u) : "memory");
+      }
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&init_bar));
+    }
+    bool ok = mbar_wait(smem_u32(&done_bar), 0, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       tc_fence_after();
-      const int row = q * 32 + lane;                 // TMEM lane: (v-in-pair, c)
+      const int row = q * 32 + lane;                 // TMEM lane: (shift-in-pair, c)
+      const int c = row & 63;
       float* dst_base = p.part + static_cast<int64_t>(blockIdx.x) * 9 * C * C;
       for (int a = 0; a < 6; ++a) {
-        const int u = a >> 1, pair = a & 1;
+        const int pair = a / 3, blk = a % 3;
+        const int u = 2 - blk;
         const int v = pair == 0 ? (row >> 6) : 2;
         const bool keep = pair == 0 || row < 64;
-        const int c = row & 63;
         float* dst = dst_base + ((u * 3 + v) * C + c) * C;
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
           uint32_t r[32];
-          if (i1 > i0) {
-            tc_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * 64 + half * 32, r);
-            tc_wait_ld();
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) r[j] = 0u;
-          }
+          tc_ld32(lane_base + pair * 256 + blk * 64 + half * 32, r);
+          tc_wait_ld();
           if (keep) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -600,10 +630,10 @@ void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w
   p.n_items = static_cast<int>(c->Z) * p.nrb * p.nseg;
   p.mode = mode; p.out = out; p.mask_src = mask; p.loss_part = c->loss_part; p.status = c->status;
   const int grid = p.n_items < c->grid ? p.n_items : c->grid;
-  if (mode == MODE_STORE_SSQ) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 4, c->stream);
+  if (mode == MODE_STORE_SSQ) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 8, c->stream);
   const double flops = 2.0 * c->B * c->H * c->W * 9.0 * C * C;
   c->prof->begin(cls, flops);
-  conv_fwd_kernel<<<grid, NUM_THREADS, FWD_SMEM, c->stream>>>(in, w, p);
+  conv_fwd_kernel<<<grid, FWD_THREADS, FWD_SMEM, c->stream>>>(in, w, p);
   c->prof->end();
 }
 
@@ -654,7 +684,7 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
          alloc(reinterpret_cast<void**>(&c->Wb[i]), 9 * C * C * 2) && alloc(reinterpret_cast<void**>(&c->dK[i]), 9 * C * C * 4);
   }
   ok = ok && alloc(reinterpret_cast<void**>(&c->wpart), static_cast<size_t>(c->grid) * 9 * C * C * 4);
-  ok = ok && alloc(reinterpret_cast<void**>(&c->loss_part), sizeof(float) * c->grid * 4);
+  ok = ok && alloc(reinterpret_cast<void**>(&c->loss_part), sizeof(float) * c->grid * 8);
   ok = ok && alloc(reinterpret_cast<void**>(&c->scratch_nchw), static_cast<size_t>(B) * C * H * W * 2);
   if (!ok) { conv_destroy(c); return MBD_E_ALLOC; }
   c->act_fwd.resize(L + 1); c->act_wg.resize(L + 1); c->dY_fwd.resize(L); c->dY_wg.resize(L);
@@ -707,8 +737,8 @@ mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
                last ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK), nullptr);
   }
   if (loss_sum_dev) {
-    c->prof->begin(MBD_K_OTHER, c->grid * 16.0);
-    if (sum_f32_launch(c->loss_part, c->grid * 4, 0.5f, loss_sum_dev, c->stream) != cudaSuccess) return MBD_E_CUDA;
+    c->prof->begin(MBD_K_OTHER, c->grid * 32.0);
+    if (sum_f32_launch(c->loss_part, c->grid * 8, 0.5f, loss_sum_dev, c->stream) != cudaSuccess) return MBD_E_CUDA;
     c->prof->end();
   }
   if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;

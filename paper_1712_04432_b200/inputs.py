@@ -67,7 +67,8 @@ WORKLOADS = {
                      "softmax_ce", grids=[(1, 1), (8, 1), (1, 8), (2, 4), (4, 2)]),
     "cfg3": Workload("cfg3", "fc", (25088, 4096, 4096, 1000), 512, "bf16", "relu_normal",
                      "softmax_ce", grids=[(1, 1), (4, 4), (16, 1), (1, 16)]),
-    "cfg4": Workload("cfg4", "conv", (64, 224, 224), 32, "bf16", "normal", "half_ssq",
+    # eta: the half-sum-of-squares loss runs over 1e8 outputs; 1e-7 keeps repeated steps finite
+    "cfg4": Workload("cfg4", "conv", (64, 224, 224), 32, "bf16", "normal", "half_ssq", eta=1e-7,
                      n_layers=2, grids=[(1, 1), (2, 1), (4, 1), (8, 1)]),
     "cfg5": Workload("cfg5", "fc", (8192,) * 9, 8192, "bf16", "normal", "softmax_ce",
                      grids=[(1, 1), (16, 16), (64, 4), (4, 64)]),

@@ -4,10 +4,13 @@ a profiler (small, self-terminating):
     python -m paper_1712_04432_b200.profile_case gemm_fwd --size 8192 --launches 3
     python -m paper_1712_04432_b200.profile_case gemm_bwd_weight --size 4096
     python -m paper_1712_04432_b200.profile_case reduce --size 8192 --splits 2
+    python -m paper_1712_04432_b200.profile_case conv --batch 4 --strips 4
 
 gemm_*: one tensor-core contraction of size^3 in the operand layout of that product.
 reduce: a split contraction followed by the partial-sum reduction (the reduction reads
 `splits` fp32 planes of size^2 and writes one).
+conv:   `launches` training steps of the two-layer 3x3 convolution stack on `batch` images of
+64 x 224 x 224, cut into `strips` row strips.
 """
 import argparse
 
@@ -18,11 +21,15 @@ from . import mbd
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce"])
+    ap.add_argument("case", choices=["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce", "conv"])
+    ap.add_argument("--batch", type=int, default=4)
+    ap.add_argument("--strips", type=int, default=4)
     ap.add_argument("--size", type=int, default=8192)
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--splits", type=int, default=2)
     a = ap.parse_args()
+    if a.case == "conv":
+        return conv_case(a)
     g = torch.Generator(device="cuda").manual_seed(0)
     n = a.size
     A = torch.randn((n, n), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
@@ -39,6 +46,26 @@ def main():
     ms = ev0.elapsed_time(ev1) / a.launches
     print(f"{a.case} size={n} splits={splits}: {ms:.3f} ms per call, {2 * n ** 3 / ms / 1e9:.1f} TFLOP/s, "
           f"checksum {float(D.double().sum()):.6e}")
+
+
+def conv_case(a):
+    g = torch.Generator(device="cuda").manual_seed(0)
+    net = mbd.Net(mbd.conv_layers(2, 64, 224, 224), a.batch, a.strips, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+    for i in range(2):
+        K = (torch.randn((64, 64, 3, 3), generator=g, device="cuda") * (2.0 / 576) ** 0.5).to(torch.bfloat16)
+        net.set_weights(i, K)
+    X = torch.randn((a.batch, 64, 224, 224), generator=g, device="cuda").to(torch.bfloat16)
+    J = torch.zeros(1, device="cuda")
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(a.launches):
+        net.forward(X, None, J)
+        net.backward(1e-6)
+    ev1.record()
+    torch.cuda.synchronize()
+    net.poll()
+    print(f"conv batch={a.batch} strips={a.strips}: {ev0.elapsed_time(ev1) / a.launches:.3f} ms per step, J = {J.item():.4e}")
 
 
 if __name__ == "__main__":
