@@ -3,16 +3,19 @@
 // dW = dY X^T (Section 1 of the paper), with the K range optionally cut into the
 // partial sums a P_r x P_c grid would form (Appendix A.2).
 //
-// One persistent CTA per SM, 192 threads, warp-specialised:
+// One persistent CTA per SM, 320 threads, warp-specialised:
 //   warp 0      TMA producer: operand tiles -> 128B-swizzled shared-memory ring
 //   warp 1      allocates tensor memory; one lane issues tcgen05.mma (128 x BN x 16 per
 //               instruction, fp32 accumulator in TMEM) and commits to mbarriers
-//   warps 2..5  epilogue: tcgen05.ld the accumulator (lane = row), apply the epilogue
-//               operation and store; two accumulators alternate so the epilogue of one
-//               tile runs under the MMAs of the next
+//   warps 2..9  epilogue: tcgen05.ld the accumulator (lane = row; each warp owns 32 rows and
+//               half of the columns), apply the epilogue operation and store; operands the
+//               operation reads are prefetched under the MMAs; two accumulators alternate so
+//               the epilogue of one tile runs under the MMAs of the next
 // Transposed operands are not copied: an operand whose contiguous dimension is M or N is
 // loaded as 64-wide column chunks and described to the MMA as "MN-major".
 // Every mbarrier wait is bounded; on time-out the kernel records a code and leaves.
+#include <stdlib.h>
+
 #include "epi.cuh"
 #include "tc_common.cuh"
 
@@ -24,7 +27,7 @@ using namespace tc;
 
 constexpr int BM = 128;
 constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;      // TMA warp, MMA warp, 8 epilogue warps
 constexpr int SMEM_RING_BYTES = 192 * 1024;
 constexpr int GROUP_M = 16;            // m-tiles per raster group (L2 reuse of the B operand)
 
@@ -88,7 +91,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&tmem_full_bar[i]), 1);
-      mbar_init(smem_u32(&tmem_empty_bar[i]), 4);
+      mbar_init(smem_u32(&tmem_empty_bar[i]), 8);
     }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -175,31 +178,56 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else {
     // ------------------------------------------------------------------ epilogue
-    const int q = warp & 3;                       // TMEM lane quarter this warp may read
+    // Eight warps: warp & 3 = TMEM lane quarter (32 rows), (warp - 2) >> 2 = column half.
+    // What the tail operation has to READ (old weights for the SGD update, stored activations
+    // for the ReLU mask) is requested before the accumulator is waited for, so that its HBM
+    // latency hides under the MMAs of this tile.
+    constexpr int HC = BN / 2;                    // columns per warp
+    constexpr int NV = HC / 8;                    // 16-byte vectors per thread and tile
+    const int q = warp & 3;
+    const int half = (warp - 2) >> 2;
+    const bool prefetch = p.S == 1 && p.epi.out_bf16 &&
+                          (p.epi.op == EPI_SGD || (p.epi.op == EPI_MASK && p.epi.mask != nullptr));
+    const __nv_bfloat16* pre_src = p.epi.op == EPI_SGD ? reinterpret_cast<const __nv_bfloat16*>(p.epi.out)
+                                                       : reinterpret_cast<const __nv_bfloat16*>(p.epi.mask);
+    const int64_t pre_ld = p.epi.op == EPI_SGD ? p.epi.ldo : p.epi.ldmask;
     int it = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++it) {
       const Work wk = decode_work(p, w);
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1u;
+      const int64_t m = static_cast<int64_t>(wk.tm) * BM + q * 32 + lane;
+      const bool row_ok = m < p.M;
+      const int64_t nbase = static_cast<int64_t>(wk.tn) * BN + half * HC;
+      uint4 pre[NV];
+      if (prefetch) {
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+          const int64_t n = nbase + j * 8;
+          pre[j] = (row_ok && n < p.N) ? *reinterpret_cast<const uint4*>(pre_src + m * pre_ld + n) : make_uint4(0, 0, 0, 0);
+        }
+      }
       ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int64_t m = static_cast<int64_t>(wk.tm) * BM + q * 32 + lane;
-      const bool row_ok = m < p.M;
-      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + half * HC;
       float* part = p.S > 1 ? p.partials + static_cast<int64_t>(wk.s) * p.M * p.N : nullptr;
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+#pragma unroll
+      for (int c = 0; c < HC / 32; ++c) {
         uint32_t r[32];
         tc_ld32(taddr + c * 32, r);
         tc_wait_ld();
-        const int64_t n0 = static_cast<int64_t>(wk.tn) * BN + c * 32;
+        if (c == HC / 32 - 1) {                    // accumulator fully in registers: hand it back
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+        }
         if (row_ok) {
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const int64_t n = n0 + j * 8;
+            const int64_t n = nbase + c * 32 + j * 8;
             if (n < p.N) {
               float v[8];
 #pragma unroll
@@ -208,6 +236,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 float* dst = part + m * p.N + n;
                 *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
                 *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
+              } else if (prefetch) {
+                const uint4 qv = pre[c * 4 + j];
+                const uint32_t wv[4] = {qv.x, qv.y, qv.z, qv.w};
+                if (p.epi.op == EPI_SGD) {
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    v[2 * i] = fmaf(p.epi.scale, v[2 * i], bf16_bits_to_f32(wv[i] & 0xFFFFu));
+                    v[2 * i + 1] = fmaf(p.epi.scale, v[2 * i + 1], bf16_bits_to_f32(wv[i] >> 16));
+                  }
+                } else {
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    if (!(bf16_bits_to_f32(wv[i] & 0xFFFFu) > 0.f)) v[2 * i] = 0.f;
+                    if (!(bf16_bits_to_f32(wv[i] >> 16) > 0.f)) v[2 * i + 1] = 0.f;
+                  }
+                }
+                uint4 o;
+                o.x = pack_bf16x2(v[0], v[1]); o.y = pack_bf16x2(v[2], v[3]);
+                o.z = pack_bf16x2(v[4], v[5]); o.w = pack_bf16x2(v[6], v[7]);
+                *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.epi.out) + m * p.epi.ldo + n) = o;
               } else {
                 epi_apply8(p.epi, m, n, v);
               }
@@ -215,9 +263,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
     }
   }
 
@@ -286,12 +331,17 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
   cudaError_t e = tc_gemm_init();
   if (e != cudaSuccess) return e;
   const int tiles_m = (g.M + BM - 1) / BM;
-  // Narrower tiles when 256-wide ones would leave SMs without work.
-  const int t256 = tiles_m * ((g.N + 255) / 256) * g.k_splits;
-  g.BN = t256 >= num_sms ? 256 : 128;
-  const int tiles_n = (g.N + g.BN - 1) / g.BN;
   const int kb_total = (g.K + BK - 1) / BK;
   if (g.k_splits > kb_total) g.k_splits = kb_total;
+  // 256-wide tiles unless they would leave SMs without work; then 128.  (64-wide tiles and an
+  // extra cut of K for occupancy were measured on the small-batch workloads and lost: the
+  // narrow MMAs are issue-bound and the extra partial sums cost more HBM time than they save.)
+  g.BN = 1ll * tiles_m * ((g.N + 255) / 256) * g.k_splits >= num_sms ? 256 : 128;
+  if (const char* ev = getenv("MBD_TC_BN")) {          // tuning knob
+    const int bn = atoi(ev);
+    if (bn == 128 || bn == 256) g.BN = bn;
+  }
+  const int tiles_n = (g.N + g.BN - 1) / g.BN;
   const long long total = 1ll * tiles_m * tiles_n * g.k_splits;
   g.grid = static_cast<int>(total < num_sms ? total : num_sms);
   const bool a_mn = g.variant == 2, b_mn = g.variant >= 1;

@@ -271,27 +271,32 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
     ALLOC(l.act, static_cast<size_t>(B) * l.d_out * (last ? sizeof(float) : es));
     ALLOC(l.dY, static_cast<size_t>(B) * l.d_out * es);
     if (cudaMemsetAsync(l.W, 0, l.nW * es, n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
-    if (S_c > 1) part_elems = std::max(part_elems, static_cast<size_t>(S_c) * l.nW);
-    if (i > 0 && S_r > 1) part_elems = std::max(part_elems, static_cast<size_t>(S_r) * B * l.d_in);
+    if (dtype != MBD_BF16) {
+      if (S_c > 1) part_elems = std::max(part_elems, static_cast<size_t>(S_c) * l.nW);
+      if (i > 0 && S_r > 1) part_elems = std::max(part_elems, static_cast<size_t>(S_r) * B * l.d_in);
+    }
     max_d = std::max(max_d, static_cast<size_t>(l.d_out));
+  }
+  if (dtype == MBD_BF16) {
+    // Plan every contraction now (tile width, number of K pieces); the partial-sum workspace is
+    // sized from the plans.  The first layer's maps are rebuilt once the caller's X is known.
+    for (int i = 0; i < L; ++i) {
+      Layer& l = n->layers[i];
+      const void* x_in = i > 0 ? n->layers[i - 1].act : l.W;       // placeholder address for layer 1
+      st = prepare_tc(n, l.fwd, 0, B, l.d_out, l.d_in, x_in, l.d_in, l.W, l.d_in, 1);
+      if (st == MBD_OK && i > 0) st = prepare_tc(n, l.bwd_data, 1, B, l.d_in, l.d_out, l.dY, l.d_out, l.W, l.d_in, S_r);
+      if (st == MBD_OK) st = prepare_tc(n, l.bwd_weight, 2, l.d_out, l.d_in, B, l.dY, l.d_out, x_in, l.d_in, S_c);
+      if (st != MBD_OK) { free_net(n); return st; }
+      if (l.fwd.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.fwd.k_splits) * B * l.d_out);
+      if (i > 0 && l.bwd_data.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.bwd_data.k_splits) * B * l.d_in);
+      if (l.bwd_weight.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.bwd_weight.k_splits) * l.nW);
+    }
   }
   n->partial_elems = part_elems;
   if (part_elems) ALLOC(n->partials, part_elems * sizeof(float));
   ALLOC(n->colsum_scratch, static_cast<size_t>(colsum_row_splits(B)) * max_d * sizeof(float));
   ALLOC(n->per_sample, B * sizeof(float));
 #undef ALLOC
-
-  if (dtype == MBD_BF16) {
-    for (int i = 0; i < L; ++i) {
-      Layer& l = n->layers[i];
-      if (i > 0) {
-        st = prepare_tc(n, l.fwd, 0, B, l.d_out, l.d_in, n->layers[i - 1].act, l.d_in, l.W, l.d_in, 1);
-        if (st == MBD_OK) st = prepare_tc(n, l.bwd_data, 1, B, l.d_in, l.d_out, l.dY, l.d_out, l.W, l.d_in, S_r);
-        if (st == MBD_OK) st = prepare_tc(n, l.bwd_weight, 2, l.d_out, l.d_in, B, l.dY, l.d_out, n->layers[i - 1].act, l.d_in, S_c);
-        if (st != MBD_OK) { free_net(n); return st; }
-      }
-    }
-  }
   if (cudaStreamSynchronize(n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
   *out = n;
   return MBD_OK;
