@@ -196,6 +196,22 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------ our arm
+def max_over_ranks(x: float, world: int, device="cuda") -> float:
+    """The slowest rank decides a multi-GPU time."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tflops(flops_per_replica: float, world: int, ms: float) -> float:
+    """Whole-job throughput: every rank runs one replica of the step (weak scaling)."""
+    return flops_per_replica * world / (ms * 1e-3) / 1e12
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -213,13 +229,6 @@ def run_ours(args):
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
-
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
 
     w = I.WORKLOADS[args.workload]
     grid = pick_grid(w, args.grid)
@@ -287,7 +296,7 @@ def run_ours(args):
     launches = net.launch_count - launches0
     per_step = [a.elapsed_time(b) for a, b in evs]
     ms = sum(per_step) / len(per_step)               # flush time excluded
-    ms = max_over_ranks(ms)
+    ms = max_over_ranks(ms, world)
     prof = net.profile_read()
     net.profile_enable(False)
     net.poll()
@@ -304,9 +313,9 @@ def run_ours(args):
             net.train_step_host(X_host, labels_host, w.eta)      # returns after the loss is on the host
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / args.steps
-        dt = max_over_ranks(dt)
+        dt = max_over_ranks(dt, world)
         h2d = X_host.numel() * X_host.element_size() + (labels_host.numel() * 4 if labels_host is not None else 0)
-        e2e = dict(value=flops * world / dt / 1e12, unit="TFLOP/s", h2d_bytes_per_step=int(h2d), d2h_bytes_per_step=4,
+        e2e = dict(value=aggregate_tflops(flops, world, dt * 1e3), unit="TFLOP/s", h2d_bytes_per_step=int(h2d), d2h_bytes_per_step=4,
                    ms_per_step=dt * 1e3)
     clocks = sampler.stop() if rank == 0 else None
     if rank != 0:
@@ -344,7 +353,7 @@ def run_ours(args):
         cpu = dict(value=fl / dt / 1e12, unit="TFLOP/s", cores=host_threads(), kind="oracle", sample=desc,
                    seconds=dt)
 
-    line = dict(metric=METRIC, value=flops * world / (ms * 1e-3) / 1e12, unit="TFLOP/s", n_gpus=world,
+    line = dict(metric=METRIC, value=aggregate_tflops(flops, world, ms), unit="TFLOP/s", n_gpus=world,
                 steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=ms, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype=w.dtype, data="synthetic",
                 config=workload_config(w, grid, args.max_partials), clocks=clocks, e2e=e2e,

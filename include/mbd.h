@@ -184,6 +184,14 @@ MBD_API mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, c
                          int64_t lda, const void* B_dev, int64_t ldb, float* D_dev, int64_t ldd,
                          int k_splits, float* partials_dev, void* cuda_stream);
 
+/* Failure-detection self test: launches one small kernel whose only job is to wait, with a
+ * limit of `limit_ms` milliseconds, on a barrier that nothing will ever signal.  The kernel
+ * gives up when the limit runs out, records a status code and returns normally; the call then
+ * reports MBD_E_TIMEOUT (MBD_OK would mean the bounded wait did not fire).  The device context
+ * stays usable.  This is the same bounded-wait path every pipeline barrier of the tensor-core
+ * kernels uses (their limit is 4 s). */
+MBD_API mbd_status mbd_selftest_timeout(int limit_ms, void* cuda_stream);
+
 /* No counterpart in the paper: a convenience for callers that cannot allocate device memory
  * themselves and cannot let a library do it -- a service whose own pool owns all of the GPU's
  * memory, a plug-in that runs where cudaMalloc would stall or fail (memory exhausted, or an

@@ -275,6 +275,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 }
 
+// A wait that cannot succeed: nothing ever arrives at `bar`.  Exercises the give-up path.
+__global__ void selftest_timeout_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait_slow(smem_u32(&bar), 0, &abort_flag, status, DEV_TIMEOUT_EPILOGUE, limit_ns);
+  __syncthreads();
+}
+
 // ----------------------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -325,6 +339,11 @@ cudaError_t tc_gemm_init() {
   if ((e = set_attr<1, 1, 128>()) != cudaSuccess) return e;
   g_init_done = true;
   return cudaSuccess;
+}
+
+cudaError_t selftest_timeout_launch(int* status, int limit_ms, cudaStream_t stream) {
+  selftest_timeout_kernel<<<1, 32, 0, stream>>>(status, static_cast<unsigned long long>(limit_ms) * 1000000ull);
+  return cudaGetLastError();
 }
 
 cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B, int64_t ldb, int num_sms) {

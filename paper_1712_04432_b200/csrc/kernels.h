@@ -59,6 +59,7 @@ struct TcGemm {
 cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B, int64_t ldb,
                             int num_sms);
 cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream);
+cudaError_t selftest_timeout_launch(int* status, int limit_ms, cudaStream_t stream);
 cudaError_t tc_gemm_init();   // driver entry point lookup + kernel attributes; idempotent
 
 // ---- fp32 SIMT GEMM (check mode) ----------------------------------------------

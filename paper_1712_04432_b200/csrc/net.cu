@@ -559,3 +559,21 @@ extern "C" mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K
   cudaFree(status);
   return ret;
 }
+
+extern "C" mbd_status mbd_selftest_timeout(int limit_ms, void* cuda_stream) {
+  if (limit_ms < 1 || limit_ms > 2000) return MBD_E_INVALID;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int* status = nullptr;
+  if (dev_alloc(reinterpret_cast<void**>(&status), sizeof(int)) != MBD_OK) return MBD_E_ALLOC;
+  mbd_status ret = MBD_OK;
+  int h = 0;
+  if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess || selftest_timeout_launch(status, limit_ms, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess || cudaMemcpy(&h, status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    ret = MBD_E_CUDA;
+  } else if (h != 0) {
+    ret = MBD_E_TIMEOUT;
+  }
+  (void)cudaGetLastError();
+  cudaFree(status);
+  return ret;
+}

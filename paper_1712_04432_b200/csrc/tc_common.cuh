@@ -43,15 +43,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait.  Returns false after WAIT_LIMIT_NS or when another role has given up.
+// Bounded wait.  Returns false after `limit_ns` or when another role has given up.
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                            int* status, int code) {
+                                            int* status, int code, unsigned long long limit_ns = WAIT_LIMIT_NS) {
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
     for (int i = 0; i < 256; ++i)
       if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+    if (globaltimer_ns() - t0 > limit_ns) {
       *abort_flag = 1;
       atomicCAS(status, 0, code);
       return false;

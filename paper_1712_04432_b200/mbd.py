@@ -25,7 +25,7 @@ KERNEL_CLASSES = ["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce_partia
 
 EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weights", "mbd_forward",
            "mbd_backward", "mbd_sgd_step", "mbd_train_step_host", "mbd_comm_words", "mbd_get_tensor",
-           "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_gemm_bf16_noalloc", "mbd_strerror"]
+           "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_gemm_bf16_noalloc", "mbd_selftest_timeout", "mbd_strerror"]
 
 
 class MbdError(RuntimeError):
@@ -76,6 +76,7 @@ def lib():
         L.mbd_launch_count.restype = i64
         L.mbd_gemm_bf16.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp, vp]
         L.mbd_gemm_bf16_noalloc.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
+        L.mbd_selftest_timeout.argtypes = [i32, vp]
         L.mbd_strerror.argtypes = [i32]
         L.mbd_strerror.restype = C.c_char_p
         _lib = L
@@ -258,6 +259,12 @@ def gemm_bf16(variant: int, A, B, k_splits: int = 1, return_partials: bool = Fal
                              k_splits, _ptr(parts), C.c_void_p(torch.cuda.current_stream().cuda_stream))
     _check(st, "mbd_gemm_bf16")
     return (D, parts) if return_partials else D
+
+
+def selftest_timeout(limit_ms: int = 50) -> int:
+    """mbd_selftest_timeout: returns the status (E_TIMEOUT when the bounded wait fired)."""
+    import torch
+    return int(lib().mbd_selftest_timeout(int(limit_ms), C.c_void_p(torch.cuda.current_stream().cuda_stream)))
 
 
 def gemm_bf16_noalloc(variant: int, A, B, k_splits: int = 1, out=None):

@@ -1,0 +1,60 @@
+"""Host-side logic of the C ABI that needs no GPU: argument validation of mbd_net_create
+(checked before any CUDA call), and the loud failure when no device is present."""
+import ctypes as C
+
+import pytest
+
+from paper_1712_04432_b200 import mbd
+
+
+def create(layers, B, P_r=1, P_c=1, dtype=mbd.BF16, loss=mbd.LOSS_SOFTMAX_CE, max_partials=0):
+    h = C.c_void_p()
+    st = mbd.lib().mbd_net_create(mbd._layer_array(layers), len(layers), B, P_r, P_c, dtype, loss, max_partials,
+                                  None, C.byref(h))
+    if st == mbd.OK:
+        mbd.lib().mbd_net_destroy(h)
+    return st
+
+
+def test_grid_errors():
+    fc = mbd.fc_layers((64, 32, 16))
+    assert create(fc, 8, 0, 1) == mbd.E_GRID
+    assert create(fc, 8, 1, 0) == mbd.E_GRID
+    assert create(fc, 8, 1, 9) == mbd.E_GRID          # more batch blocks than samples
+    assert create(fc, 8, 17, 1) == mbd.E_GRID         # more row blocks than neurons of the last layer
+    conv = mbd.conv_layers(2, 64, 8, 16)
+    assert create(conv, 4, 9, 1, loss=mbd.LOSS_HALF_SSQ) == mbd.E_GRID    # strips shorter than one row
+    assert create(conv, 4, 2, 2, loss=mbd.LOSS_HALF_SSQ) == mbd.E_GRID    # batch split with a domain layer
+
+
+def test_invalid_and_unsupported():
+    fc = mbd.fc_layers((64, 32, 16))
+    assert create(fc, 0) == mbd.E_INVALID
+    assert create(fc, 8, dtype=5) == mbd.E_INVALID
+    assert create(fc, 8, loss=9) == mbd.E_INVALID
+    assert create(fc, 8, max_partials=-1) == mbd.E_INVALID
+    assert create(mbd.fc_layers((64, 32)) + mbd.fc_layers((48, 16)), 8) == mbd.E_INVALID   # dims do not chain
+    assert create(mbd.fc_layers((60, 30)), 8) == mbd.E_UNSUPPORTED                         # bf16 needs multiples of 8
+    conv5 = mbd.conv_layers(1, 64, 8, 16)
+    conv5[0].kh = conv5[0].kw = 5
+    assert create(conv5, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
+    assert create(mbd.conv_layers(1, 64, 8, 16), 4, loss=mbd.LOSS_SOFTMAX_CE) == mbd.E_UNSUPPORTED
+
+
+def test_null_handles_are_rejected():
+    L = mbd.lib()
+    assert L.mbd_forward(None, None, None, None) == mbd.E_INVALID
+    assert L.mbd_backward(None, 0.0) == mbd.E_INVALID
+    assert L.mbd_sgd_step(None, 0.1) == mbd.E_INVALID
+    assert L.mbd_poll_status(None) == mbd.E_INVALID
+    assert L.mbd_launch_count(None) == -1
+    assert L.mbd_net_destroy(None) == mbd.E_INVALID
+
+
+def test_no_silent_fallback_without_a_gpu():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    # valid arguments, but no device: the library reports a CUDA error instead of computing elsewhere
+    assert create(mbd.fc_layers((64, 32, 16)), 8) == mbd.E_CUDA
+    assert create(mbd.fc_layers((64, 32, 16)), 8, dtype=mbd.F32) == mbd.E_CUDA
