@@ -65,8 +65,18 @@ nchw_to_strips_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int 
   {
     const int c = t >> 2, wq = (t & 3) * 8;
     const bf16* p = src + ((static_cast<int64_t>(b) * C + c) * H + h) * W + w0 + wq;
+    if ((W & 7) == 0 && w0 + wq + 8 <= W) {
+      const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p));
+      const uint32_t qw[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-    for (int i = 0; i < 8; ++i) tile[c][wq + i] = (w0 + wq + i < W) ? p[i] : __float2bfloat16(0.f);
+      for (int i = 0; i < 4; ++i) {
+        tile[c][wq + 2 * i] = __ushort_as_bfloat16(static_cast<unsigned short>(qw[i] & 0xFFFFu));
+        tile[c][wq + 2 * i + 1] = __ushort_as_bfloat16(static_cast<unsigned short>(qw[i] >> 16));
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) tile[c][wq + i] = (w0 + wq + i < W) ? p[i] : __float2bfloat16(0.f);
+    }
   }
   __syncthreads();
   const int px = t >> 3, cq = (t & 7) * 8;
@@ -281,6 +291,14 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       for (int i = 0; i < p.RB; ++i, ++n_out) {
         const int acc = n_out & 1;
         const uint32_t acc_phase = (n_out >> 1) & 1u;
+        const int64_t opix = ((static_cast<int64_t>(z) * p.R + rb * p.RB + i + 1) * p.W + x) * C + half * 32;
+        uint4 mpre[4];
+        const bool use_mask = p.mode == MODE_MASK && p.mask_src != nullptr;
+        if (use_mask && valid) {                           // requested before the accumulator is ready
+          const uint4* m4 = reinterpret_cast<const uint4*>(p.mask_src + opix);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mpre[j] = m4[j];
+        }
         ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
         // all epilogue warps must agree before they meet at the exchange barriers
         int bad;
@@ -293,7 +311,6 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         if (bad) { ok = false; break; }
         tc_fence_after();
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * 256 + half * 32;
-        const int64_t opix = ((static_cast<int64_t>(z) * p.R + rb * p.RB + i + 1) * p.W + x) * C + half * 32;
         uint32_t d0[32], d1[32], d2[32];
         tc_ld32(taddr, d0);
         tc_ld32(taddr + 64, d1);
@@ -340,11 +357,10 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           } else if (p.mode == MODE_STORE_SSQ) {
 #pragma unroll
             for (int c = 0; c < 32; ++c) ssq = fmaf(y[c], y[c], ssq);
-          } else if (p.mask_src) {
-            const uint4* m4 = reinterpret_cast<const uint4*>(p.mask_src + opix);
+          } else if (use_mask) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              const uint4 mq = m4[j];
+              const uint4 mq = mpre[j];
               const uint32_t mw[4] = {mq.x, mq.y, mq.z, mq.w};
 #pragma unroll
               for (int e = 0; e < 4; ++e) {

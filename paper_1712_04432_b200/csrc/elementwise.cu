@@ -121,40 +121,59 @@ sum_f32_kernel(const float* __restrict__ x, int64_t n, float scale, float* __res
 }
 
 // ------------------------------------------------------------------ column sums (bias gradient)
-// Stage 1: grid (ceil(N/64), row_splits); 256 threads = 8 warps; a warp covers 64 columns
-// (2 per lane), warps stride over the rows of this split; the 8 warps are added in order.
+// Stage 1: grid (ceil(N/256), row_splits); 256 threads = 8 warps; a lane owns 8 consecutive
+// columns (one 16-byte load per row for bf16), a warp 256 columns, the 8 warps stride over the
+// rows of this split and are added in warp order.  With a single split the result is final and
+// the bias update is applied here; otherwise stage 2 adds the splits in order.
+template <bool BF16>
 __global__ void __launch_bounds__(256)
-colsum_stage1(const void* __restrict__ dY, int dy_bf16, int64_t M, int64_t N, int row_splits,
-              float* __restrict__ scratch) {
-  __shared__ float red[8][64];
+colsum_stage1(const void* __restrict__ dY, int64_t M, int64_t N, int row_splits, float* __restrict__ scratch,
+              float* __restrict__ db, float* __restrict__ bias, float scale) {
+  __shared__ float red[8][256 + 8];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t n = static_cast<int64_t>(blockIdx.x) * 64 + lane * 2;
+  const int64_t n0 = static_cast<int64_t>(blockIdx.x) * 256 + lane * 8;
   const int64_t r0 = (static_cast<int64_t>(blockIdx.y) * M) / row_splits;
   const int64_t r1 = (static_cast<int64_t>(blockIdx.y + 1) * M) / row_splits;
-  float a0 = 0.f, a1 = 0.f;
-  if (n < N) {
-    const bool two = n + 1 < N;
-    for (int64_t m = r0 + warp; m < r1; m += 8) {
-      if (dy_bf16) {
-        const __nv_bfloat16* p = reinterpret_cast<const __nv_bfloat16*>(dY) + m * N + n;
-        a0 += __bfloat162float(p[0]);
-        if (two) a1 += __bfloat162float(p[1]);
+  float a[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) a[i] = 0.f;
+  const bool vec = (N % 8 == 0) && n0 + 8 <= N;
+  for (int64_t m = r0 + warp; m < r1; m += 8) {
+    if (vec) {
+      if (BF16) {
+        const uint4 q = __ldcs(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(dY) + m * N + n0));
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { a[2 * i] += bf16_bits_to_f32(w[i] & 0xFFFFu); a[2 * i + 1] += bf16_bits_to_f32(w[i] >> 16); }
       } else {
-        const float* p = reinterpret_cast<const float*>(dY) + m * N + n;
-        a0 += p[0];
-        if (two) a1 += p[1];
+        const float* p = reinterpret_cast<const float*>(dY) + m * N + n0;
+        const float4 u = *reinterpret_cast<const float4*>(p), v = *reinterpret_cast<const float4*>(p + 4);
+        a[0] += u.x; a[1] += u.y; a[2] += u.z; a[3] += u.w; a[4] += v.x; a[5] += v.y; a[6] += v.z; a[7] += v.w;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (n0 + i < N) {
+          a[i] += BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(dY)[m * N + n0 + i])
+                       : reinterpret_cast<const float*>(dY)[m * N + n0 + i];
+        }
       }
     }
   }
-  red[warp][lane * 2] = a0;
-  red[warp][lane * 2 + 1] = a1;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) red[warp][lane * 8 + i] = a[i];
   __syncthreads();
-  if (threadIdx.x < 64) {
+  const int64_t n = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  if (n < N) {
     float s = red[0][threadIdx.x];
 #pragma unroll
     for (int w = 1; w < 8; ++w) s += red[w][threadIdx.x];
-    const int64_t nn = static_cast<int64_t>(blockIdx.x) * 64 + threadIdx.x;
-    if (nn < N) scratch[static_cast<int64_t>(blockIdx.y) * N + nn] = s;
+    if (row_splits == 1) {
+      if (db) db[n] = s;
+      if (bias) bias[n] = fmaf(scale, s, bias[n]);
+    } else {
+      scratch[static_cast<int64_t>(blockIdx.y) * N + n] = s;
+    }
   }
 }
 
@@ -235,19 +254,25 @@ cudaError_t sum_f32_launch(const float* x, int64_t n, float scale, float* out, c
   return cudaGetLastError();
 }
 
-int colsum_row_splits(int64_t M) {
-  int64_t r = M / 64;
-  if (r < 1) r = 1;
+// Row splits (<= 32) so that the first stage has about two CTAs per SM, each with >= 8 rows.
+int colsum_row_splits(int64_t M, int64_t N, int num_sms) {
+  const int64_t gx = (N + 255) / 256;
+  int64_t r = (2 * static_cast<int64_t>(num_sms) + gx - 1) / gx;
+  if (r > M / 8) r = M / 8;
   if (r > 32) r = 32;
+  if (r < 1) r = 1;
   return static_cast<int>(r);
 }
 
+int colsum_launches(int64_t M, int64_t N, int num_sms) { return colsum_row_splits(M, N, num_sms) == 1 ? 1 : 2; }
+
 cudaError_t colsum_launch(const void* dY, int dy_bf16, int64_t M, int64_t N, float* scratch, int row_splits,
                           float* db, float* bias, float scale, cudaStream_t stream) {
-  dim3 g1(static_cast<unsigned>((N + 63) / 64), row_splits);
-  colsum_stage1<<<g1, 256, 0, stream>>>(dY, dy_bf16, M, N, row_splits, scratch);
+  dim3 g1(static_cast<unsigned>((N + 255) / 256), row_splits);
+  if (dy_bf16) colsum_stage1<true><<<g1, 256, 0, stream>>>(dY, M, N, row_splits, scratch, db, bias, scale);
+  else colsum_stage1<false><<<g1, 256, 0, stream>>>(dY, M, N, row_splits, scratch, db, bias, scale);
   cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  if (e != cudaSuccess || row_splits == 1) return e;
   colsum_stage2<<<static_cast<unsigned>((N + 255) / 256), 256, 0, stream>>>(scratch, row_splits, N, db, bias, scale);
   return cudaGetLastError();
 }

@@ -29,11 +29,10 @@ constexpr int BM = 128;
 constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
 constexpr int NUM_THREADS = 320;      // TMA warp, MMA warp, 8 epilogue warps
 constexpr int SMEM_RING_BYTES = 192 * 1024;
-constexpr int GROUP_M = 16;            // m-tiles per raster group (L2 reuse of the B operand)
 
 struct Params {
   int M, N, K;
-  int tiles_m, tiles_n, kb_total, S;
+  int tiles_m, tiles_n, kb_total, S, group_m;
   float* partials;
   Epi epi;
   int* status;
@@ -48,10 +47,10 @@ __device__ __forceinline__ Work decode_work(const Params& p, int w) {
   Work o;
   o.s = w / num_tiles;
   const int t = w - o.s * num_tiles;
-  const int per_group = GROUP_M * p.tiles_n;
+  const int per_group = p.group_m * p.tiles_n;
   const int g = t / per_group;
-  const int first_m = g * GROUP_M;
-  const int gsize = min(p.tiles_m - first_m, GROUP_M);
+  const int first_m = g * p.group_m;
+  const int gsize = min(p.tiles_m - first_m, p.group_m);
   const int r = t - g * per_group;
   o.tm = first_m + r % gsize;
   o.tn = r / gsize;
@@ -379,6 +378,8 @@ cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
   p.tiles_n = (g.N + g.BN - 1) / g.BN;
   p.kb_total = (g.K + BK - 1) / BK;
   p.S = g.k_splits;
+  p.group_m = 16;                       // m-tiles per raster group (L2 reuse of the B operand)
+  if (const char* ev = getenv("MBD_TC_GROUP_M")) { const int gm = atoi(ev); if (gm >= 1) p.group_m = gm; }
   p.partials = g.partials;
   p.epi = g.epi;
   p.status = g.status;

@@ -86,7 +86,8 @@ cudaError_t sum_f32_launch(const float* x, int64_t n, float scale, float* out, c
 // If bias != null: bias[n] += scale * db[n].  If db != null: db[n] stored.
 cudaError_t colsum_launch(const void* dY, int dy_bf16, int64_t M, int64_t N, float* scratch,
                           int row_splits, float* db, float* bias, float scale, cudaStream_t stream);
-int colsum_row_splits(int64_t M);
+int colsum_row_splits(int64_t M, int64_t N, int num_sms);   // at most 32
+int colsum_launches(int64_t M, int64_t N, int num_sms);    // kernels one colsum_launch issues (1 or 2)
 // w[i] += scale * g[i]   (w bf16 or f32, g f32)
 cudaError_t sgd_update_launch(void* w, int w_bf16, const float* g, int64_t n, float scale,
                               int num_sms, cudaStream_t stream);

@@ -294,7 +294,7 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   }
   n->partial_elems = part_elems;
   if (part_elems) ALLOC(n->partials, part_elems * sizeof(float));
-  ALLOC(n->colsum_scratch, static_cast<size_t>(colsum_row_splits(B)) * max_d * sizeof(float));
+  ALLOC(n->colsum_scratch, static_cast<size_t>(32) * max_d * sizeof(float));
   ALLOC(n->per_sample, B * sizeof(float));
 #undef ALLOC
   if (cudaStreamSynchronize(n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
@@ -382,10 +382,10 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
     Layer& l = n->layers[i];
     if (l.bias) {
       n->prof.begin(MBD_K_COLSUM, static_cast<double>(n->B) * l.d_out * (bf ? 2.0 : 4.0));
-      CK(colsum_launch(l.dY, bf, n->B, l.d_out, n->colsum_scratch, colsum_row_splits(n->B), fused ? nullptr : l.db,
+      CK(colsum_launch(l.dY, bf, n->B, l.d_out, n->colsum_scratch, colsum_row_splits(n->B, l.d_out, n->num_sms), fused ? nullptr : l.db,
                        fused ? l.bias : nullptr, scale, n->stream));
       n->prof.end();
-      n->prof.total_launches++;   // two kernels
+      n->prof.total_launches += colsum_launches(n->B, l.d_out, n->num_sms) - 1;
     }
     if (i > 0) {   // nothing is propagated below the first layer
       Layer& prev = n->layers[i - 1];

@@ -80,7 +80,7 @@ def test_launch_accounting_and_profile():
     n0 = net.launch_count
     net.forward(X, lab, J)
     net.backward(0.01)
-    # forward: 2 GEMMs + softmax + loss sum; backward: 2 x (colsum stage 1+2) + dX GEMM + its reduction
+    # forward: 2 GEMMs + softmax + loss sum; backward: 2 x colsum (two stages) + dX GEMM + its reduction
     # + 2 x (dW GEMM + reduction with the fused update)
     assert net.launch_count - n0 == 4 + 4 + 2 + 4
     prof = net.profile_read()
