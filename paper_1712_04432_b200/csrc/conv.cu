@@ -11,12 +11,12 @@
 // (backward-weight: pixels are the reduction index) tensor-core operand.
 //
 // conv_fwd_kernel  (forward and, with flipped / transposed weights, backward-data)
-//     one output row segment of 126 pixels per accumulator: for u = 0..2 the input row h+u-1
-//     (128 pixels starting one to the left) is multiplied by the stacked taps [K(u,0); K(u,1);
-//     K(u,2)] (N = 192), giving D_v[p] = sum_{u,c} K[.,c,u,v] X[h+u-1, p, c]; the horizontal
-//     shift is applied on the accumulator side in the epilogue: Y[p] = D_0[p-1] + D_1[p] +
-//     D_2[p+1] (warp shuffles across TMEM lanes).  Input rows sit in a shared-memory ring and
-//     are loaded once per row block; the weights (72 KB) stay resident.
+//     input-row stationary: every input row segment is loaded once per row block as three
+//     horizontally shifted copies (three TMA boxes) and, for each shift v, multiplied by the
+//     stacked taps [K(0,v); K(1,v); K(2,v)] (N = 192); the three 64-column results belong to the
+//     output rows r, r-1, r-2, whose accumulators sit next to each other in a ring of eight
+//     TMEM blocks.  An output row is complete after three input rows; the epilogue drains it,
+//     zeroes the block and stores.  The weights (72 KB) stay resident in shared memory.
 // conv_wgrad_kernel
 //     dK[o,c,u,v] = sum_pixels dY[p,o] X[p + (u-1,v-1), c]: the three horizontal shifts of an X
 //     row are three TMA boxes (the W coordinate of a box start is free); two shifted copies
@@ -37,12 +37,11 @@ typedef __nv_bfloat16 bf16;
 namespace {
 
 constexpr int C = 64;                 // channels in and out
-constexpr int FWD_PIX = 126;          // output pixels per forward tile (lanes 1..126 of 128)
-constexpr int FWD_STAGES = 5;         // ring of input rows, 16 KB each (3 live + 2 in flight)
+constexpr int FWD_PIX = 128;          // output pixels per forward tile (one per TMEM lane)
+constexpr int FWD_STAGES = 3;         // ring of input rows: 3 shifted copies of 16 KB each; a row is used once
 constexpr int FWD_ROW_BYTES = 128 * 128;
 constexpr int FWD_W_BYTES = 3 * 192 * 128;   // stacked taps, 72 KB
-constexpr int FWD_XCH_BYTES = 2 * 2 * 128 * 32 * 4;   // per channel half: D_0 and D_2 planes, 128 pixels x 32 floats
-constexpr int FWD_SMEM = FWD_W_BYTES + FWD_STAGES * FWD_ROW_BYTES + FWD_XCH_BYTES + 1024;
+constexpr int FWD_SMEM = FWD_W_BYTES + FWD_STAGES * 3 * FWD_ROW_BYTES + 1024;
 constexpr int FWD_THREADS = 320;      // producer warp, MMA warp, 8 epilogue warps
 constexpr int WG_PIX = 64;            // pixels (reduction length) per backward-weight block
 constexpr int WG_XSTAGES = 4;         // X rows: 3 shifted copies of 8 KB each, each row used once
@@ -142,15 +141,15 @@ halo_stage_kernel(bf16* __restrict__ buf, int W, int P_r, int Hs) {
   for (int64_t i = threadIdx.x; i < row / 8; i += 256) d4[i] = s4[i];
 }
 
-// Canonical K[o][c][u][v] -> forward operand Wf[u][(v,o)][c] and backward-data operand
-// Wb[u'][(v',c)][o] = K[o][c][2-u'][2-v'] (taps flipped, channels swapped).
+// Canonical K[o][c][u][v] -> forward operand Wf[v][(u,o)][c] and backward-data operand
+// Wb[v'][(u',c)][o] = K[o][c][2-u'][2-v'] (taps flipped, channels swapped).
 __global__ void pack_weights_kernel(const bf16* __restrict__ K, bf16* __restrict__ Wf, bf16* __restrict__ Wb) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= C * C * 9) return;
   const int o = i / (C * 9), c = (i / 9) % C, u = (i % 9) / 3, v = i % 3;
   const bf16 k = K[i];
-  Wf[((u * 3 + v) * C + o) * C + c] = k;
-  Wb[(((2 - u) * 3 + (2 - v)) * C + c) * C + o] = k;
+  Wf[((v * 3 + u) * C + o) * C + c] = k;
+  Wb[(((2 - v) * 3 + (2 - u)) * C + c) * C + o] = k;
 }
 
 // Sum of the per-CTA partials [G][9][c][o] in CTA order, into canonical [o][c][u][v]:
@@ -177,27 +176,32 @@ struct FwdParams {
   int* status;
 };
 
+// TMEM holds a ring of eight 64-column accumulators, one per output row in flight; output
+// row g uses block 7 - (g mod 8), so that the rows r, r-1, r-2 fed by input row r sit in
+// ascending, adjacent blocks and one N = 192 instruction updates all three (two instructions
+// when the window wraps around the ring).  The epilogue zeroes a block after draining it, so
+// every MMA accumulates.
+__device__ __forceinline__ int acc_block(int g) { return 7 - (g & 7); }
+
 __global__ void __launch_bounds__(FWD_THREADS, 1)
 conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const FwdParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[FWD_STAGES];
   __shared__ __align__(8) uint64_t empty_bar[FWD_STAGES];
-  __shared__ __align__(8) uint64_t tmem_full_bar[2];
-  __shared__ __align__(8) uint64_t tmem_empty_bar[2];
+  __shared__ __align__(8) uint64_t acc_full_bar[8];
+  __shared__ __align__(8) uint64_t acc_empty_bar[8];
   __shared__ __align__(8) uint64_t w_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t w_smem = base;                         // 3 x (192 rows x 128 B)
-  const uint32_t ring = base + FWD_W_BYTES;
-  float* xch_base = reinterpret_cast<float*>(smem_raw + (base - smem_u32(smem_raw)) + FWD_W_BYTES +
-                                             FWD_STAGES * FWD_ROW_BYTES);
+  const uint32_t w_smem = base;                         // 3 (v) x [192 rows (u, o) x 128 B]
+  const uint32_t ring = base + FWD_W_BYTES;             // slot = 3 shifted copies of one input row
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < FWD_STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tmem_full_bar[i]), 1); mbar_init(smem_u32(&tmem_empty_bar[i]), 8); }
+    for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&acc_full_bar[i]), 1); mbar_init(smem_u32(&acc_empty_bar[i]), 8); }
     mbar_init(smem_u32(&w_bar), 1);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -215,7 +219,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   if (warp == 0) {
     if (lane == 0) {
       mbar_expect_tx(smem_u32(&w_bar), FWD_W_BYTES);
-      for (int u = 0; u < 3; ++u) tma_load_2d(w_smem + u * (192 * 128), &tmW, 0, u * 192, smem_u32(&w_bar));
+      for (int v = 0; v < 3; ++v) tma_load_2d(w_smem + v * (192 * 128), &tmW, 0, v * 192, smem_u32(&w_bar));
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -225,72 +229,82 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
           if (!ok) break;
           const uint32_t fb = smem_u32(&full_bar[stage]);
-          mbar_expect_tx(fb, FWD_ROW_BYTES);
-          tma_load_4d(ring + stage * FWD_ROW_BYTES, &tmX, 0, seg * FWD_PIX - 1, rb * p.RB + r, z, fb);
+          mbar_expect_tx(fb, 3 * FWD_ROW_BYTES);
+          for (int v = 0; v < 3; ++v)
+            tma_load_4d(ring + (stage * 3 + v) * FWD_ROW_BYTES, &tmX, 0, seg * FWD_PIX + v - 1, rb * p.RB + r, z, fb);
           if (++stage == FWD_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t IDESC = make_idesc(128, 192, 0, 0);
       bool ok = mbar_wait(smem_u32(&w_bar), 0, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
-      int wstage = 0;          // next ring slot to wait for
-      uint32_t wphase = 0;
-      int slot0 = 0;           // ring slot of the current item's row 0
-      int n_out = 0;           // output rows issued so far (accumulator alternation)
+      int stage = 0;
+      uint32_t phase = 0;
+      int g0 = 0;              // output rows of earlier items of this CTA
       for (int it = i0; it < i1 && ok; ++it) {
-        int have = 0;
-        for (int i = 0; i < p.RB && ok; ++i) {
-          while (have < i + 3 && ok) {
-            ok = mbar_wait(smem_u32(&full_bar[wstage]), wphase, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
-            if (++wstage == FWD_STAGES) { wstage = 0; wphase ^= 1u; }
-            ++have;
+        for (int r = 0; r < p.RB + 2 && ok; ++r) {
+          if (r < p.RB) {      // this input row opens output row r: its block must be drained and zeroed
+            const int g = g0 + r;
+            ok = mbar_wait(smem_u32(&acc_empty_bar[acc_block(g)]), (g >> 3) & 1u, abortp, p.status, DEV_TIMEOUT_MMA_TMEM);
+            if (!ok) break;
           }
-          if (!ok) break;
-          const int acc = n_out & 1;
-          const uint32_t acc_phase = (n_out >> 1) & 1u;
-          ok = mbar_wait(smem_u32(&tmem_empty_bar[acc]), acc_phase ^ 1u, abortp, p.status, DEV_TIMEOUT_MMA_TMEM);
+          ok = mbar_wait(smem_u32(&full_bar[stage]), phase, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t d_tmem = tmem_base + acc * 256;
+          const int u_lo = max(0, r - (p.RB - 1)), u_hi = min(2, r);      // taps whose output row r - u exists
+          const uint32_t xa = ring + stage * 3 * FWD_ROW_BYTES;
+          int u_s = u_lo;
+          while (u_s <= u_hi) {
+            const int bs = acc_block(g0 + r - u_s);
+            int u_e = u_s;
+            while (u_e < u_hi && bs + (u_e + 1 - u_s) <= 7) ++u_e;          // stay inside the ring
+            const uint32_t idesc = make_idesc(128, 64 * (u_e - u_s + 1), 0, 0);
+            const uint32_t d_tmem = tmem_base + bs * 64;
 #pragma unroll
-          for (int u = 0; u < 3; ++u) {
-            const int slot = (slot0 + i + u) % FWD_STAGES;
-            const uint64_t adesc = make_desc(ring + slot * FWD_ROW_BYTES, 16, 1024);
-            const uint64_t bdesc = make_desc(w_smem + u * (192 * 128), 16, 1024);
+            for (int v = 0; v < 3; ++v) {
+              const uint64_t adesc = make_desc(xa + v * FWD_ROW_BYTES, 16, 1024);
+              const uint64_t bdesc = make_desc(w_smem + v * (192 * 128) + u_s * (64 * 128), 16, 1024);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) tc_mma_bf16(d_tmem, adesc + k * 2, bdesc + k * 2, IDESC, (u > 0 || k > 0) ? 1u : 0u);
+              for (int k = 0; k < 4; ++k) tc_mma_bf16(d_tmem, adesc + k * 2, bdesc + k * 2, idesc, 1u);
+            }
+            u_s = u_e + 1;
           }
-          tc_commit(smem_u32(&tmem_full_bar[acc]));
-          tc_commit(smem_u32(&empty_bar[(slot0 + i) % FWD_STAGES]));       // row i has no later reader
-          ++n_out;
+          tc_commit(smem_u32(&empty_bar[stage]));                           // the row is used only here
+          if (++stage == FWD_STAGES) { stage = 0; phase ^= 1u; }
+          if (r >= 2) tc_commit(smem_u32(&acc_full_bar[acc_block(g0 + r - 2)]));   // output row r-2 is complete
         }
-        if (!ok) break;
-        tc_commit(smem_u32(&empty_bar[(slot0 + p.RB) % FWD_STAGES]));
-        tc_commit(smem_u32(&empty_bar[(slot0 + p.RB + 1) % FWD_STAGES]));
-        slot0 = (slot0 + p.RB + 2) % FWD_STAGES;
+        g0 += p.RB;
       }
     }
   } else {
     // Eight epilogue warps: warp & 3 selects the TMEM lane quarter (32 pixels), (warp - 2) >> 2 the
-    // channel half.  The horizontal shift goes through shared memory: D_0 of pixel p is written
-    // to row p + 1, D_2 of pixel p to row p - 1, and every thread reads back its own row.
+    // channel half.  Drain a finished block, zero it for its next use, apply the tail operation.
     const int q = warp & 3;
     const int half = (warp - 2) >> 2;
-    const int pl = q * 32 + lane;         // TMEM lane = pixel index inside the 128-pixel window
-    float* s0 = xch_base + half * (2 * 128 * 32);
-    float* s2 = s0 + 128 * 32;
-    int n_out = 0;
+    const int pl = q * 32 + lane;                       // pixel inside the 128-pixel segment
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * 32;
+    for (int b = 0; b < 8; ++b) {                        // all blocks start out zero and free
+      asm volatile(
+          "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+          "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
+          "%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+          ::"r"(lane_base + b * 64), "r"(0u) : "memory");
+    }
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0)
+      for (int b = 0; b < 8; ++b) mbar_arrive(smem_u32(&acc_empty_bar[b]));
+    int g = 0;
     float ssq = 0.f;
     bool ok = true;
     for (int it = i0; it < i1 && ok; ++it) {
       const int seg = it % p.nseg, rb = (it / p.nseg) % p.nrb, z = it / (p.nseg * p.nrb);
-      const int x = seg * FWD_PIX - 1 + pl;
-      const bool valid = pl >= 1 && pl <= FWD_PIX && x < p.W;
-      for (int i = 0; i < p.RB; ++i, ++n_out) {
-        const int acc = n_out & 1;
-        const uint32_t acc_phase = (n_out >> 1) & 1u;
+      const int x = seg * FWD_PIX + pl;
+      const bool valid = x < p.W;
+      for (int i = 0; i < p.RB; ++i, ++g) {
+        const int blk = acc_block(g);
         const int64_t opix = ((static_cast<int64_t>(z) * p.R + rb * p.RB + i + 1) * p.W + x) * C + half * 32;
         uint4 mpre[4];
         const bool use_mask = p.mode == MODE_MASK && p.mask_src != nullptr;
@@ -299,58 +313,26 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 #pragma unroll
           for (int j = 0; j < 4; ++j) mpre[j] = m4[j];
         }
-        ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
-        // all epilogue warps must agree before they meet at the exchange barriers
-        int bad;
-        asm volatile(
-            "{\n\t.reg .pred pi, po;\n\t"
-            "setp.ne.b32 pi, %1, 0;\n\t"
-            "barrier.cta.red.or.pred po, 1, 256, pi;\n\t"
-            "selp.u32 %0, 1, 0, po;\n\t}"
-            : "=r"(bad) : "r"(ok ? 0 : 1) : "memory");
-        if (bad) { ok = false; break; }
+        ok = mbar_wait(smem_u32(&acc_full_bar[blk]), (g >> 3) & 1u, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
         tc_fence_after();
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * 256 + half * 32;
-        uint32_t d0[32], d1[32], d2[32];
-        tc_ld32(taddr, d0);
-        tc_ld32(taddr + 64, d1);
-        tc_ld32(taddr + 128, d2);
+        uint32_t d[32];
+        tc_ld32(lane_base + blk * 64, d);
         tc_wait_ld();
+        asm volatile(
+            "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+            "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
+            "%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+            ::"r"(lane_base + blk * 64), "r"(0u) : "memory");
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));    // accumulator is in registers now
-        if (pl < 127) {
-          float4* row = reinterpret_cast<float4*>(s0 + (pl + 1) * 32);
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            row[j ^ ((pl + 1) & 7)] = make_float4(__uint_as_float(d0[4 * j]), __uint_as_float(d0[4 * j + 1]),
-                                                  __uint_as_float(d0[4 * j + 2]), __uint_as_float(d0[4 * j + 3]));
-        }
-        if (pl > 0) {
-          float4* row = reinterpret_cast<float4*>(s2 + (pl - 1) * 32);
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            row[j ^ ((pl - 1) & 7)] = make_float4(__uint_as_float(d2[4 * j]), __uint_as_float(d2[4 * j + 1]),
-                                                  __uint_as_float(d2[4 * j + 2]), __uint_as_float(d2[4 * j + 3]));
-        }
-        if (half == 0) asm volatile("barrier.cta.sync 2, 128;" ::: "memory");
-        else asm volatile("barrier.cta.sync 3, 128;" ::: "memory");
-        float y[32];
-        {
-          const float4* r0 = reinterpret_cast<const float4*>(s0 + pl * 32);
-          const float4* r2 = reinterpret_cast<const float4*>(s2 + pl * 32);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float4 a = r0[j ^ (pl & 7)], b = r2[j ^ (pl & 7)];
-            y[4 * j + 0] = a.x + __uint_as_float(d1[4 * j + 0]) + b.x;
-            y[4 * j + 1] = a.y + __uint_as_float(d1[4 * j + 1]) + b.y;
-            y[4 * j + 2] = a.z + __uint_as_float(d1[4 * j + 2]) + b.z;
-            y[4 * j + 3] = a.w + __uint_as_float(d1[4 * j + 3]) + b.w;
-          }
-        }
-        if (half == 0) asm volatile("barrier.cta.sync 2, 128;" ::: "memory");   // planes may be rewritten after this
-        else asm volatile("barrier.cta.sync 3, 128;" ::: "memory");
+        if (lane == 0) mbar_arrive(smem_u32(&acc_empty_bar[blk]));
         if (valid) {
+          float y[32];
+#pragma unroll
+          for (int c = 0; c < 32; ++c) y[c] = __uint_as_float(d[c]);
           if (p.mode == MODE_RELU_STORE) {
 #pragma unroll
             for (int c = 0; c < 32; ++c) y[c] = fmaxf(y[c], 0.f);
