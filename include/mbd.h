@@ -133,6 +133,15 @@ MBD_API mbd_status mbd_backward(mbd_net* net, float fused_eta);
  * the last forward, or if that backward already applied the update. */
 MBD_API mbd_status mbd_sgd_step(mbd_net* net, float eta);
 
+/* One whole step on DEVICE buffers: mbd_forward + mbd_backward(eta) with the fused update, J
+ * written to loss_sum_dev (may be NULL).  The launch sequence is captured into a CUDA graph at the
+ * first call with a given (X_dev, labels_dev, eta, loss_sum_dev) and replayed afterwards, which
+ * removes the per-kernel launch cost that dominates small networks; any change of these arguments
+ * re-captures.  While profiling is enabled, or if the network was created on the default stream
+ * (which cannot be captured), the kernels are launched directly.  Enqueue only. */
+MBD_API mbd_status mbd_train_step(mbd_net* net, const void* X_dev, const int32_t* labels_dev, float eta,
+                          float* loss_sum_dev);
+
 /* One whole step from HOST buffers: copies X_host / labels_host to the device, runs
  * forward, backward with the fused update, copies J back to *loss_host and waits. */
 MBD_API mbd_status mbd_train_step_host(mbd_net* net, const void* X_host, const int32_t* labels_host,

@@ -7,10 +7,14 @@
 namespace mbd {
 namespace {
 
-constexpr int TM = 64, TN = 64, TK = 16;
+constexpr int TK = 16;
 
+// 256 threads as 16 x 16; each thread owns an R x R micro-tile of a (16R) x (16R) CTA tile.
+// R = 4 for large outputs, R = 2 when 64 x 64 tiles would leave most SMs idle.
+template <int R>
 __global__ void __launch_bounds__(256)
 simt_gemm_kernel(const SimtGemm g) {
+  constexpr int TM = 16 * R, TN = 16 * R;
   __shared__ float As[TK][TM + 4];
   __shared__ float Bs[TK][TN + 4];
   const int tid = threadIdx.x;
@@ -22,22 +26,22 @@ simt_gemm_kernel(const SimtGemm g) {
   const int k_hi = static_cast<int>((static_cast<int64_t>(s + 1) * g.K) / g.k_splits);
   const bool a_kcontig = g.a_sk == 1, b_kcontig = g.b_sk == 1;
 
-  float acc[4][4];
+  float acc[R][R];
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < R; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int j = 0; j < R; ++j) acc[i][j] = 0.f;
 
   for (int k0 = k_lo; k0 < k_hi; k0 += TK) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < (TM * TK) / 256; ++i) {
       const int e = tid + i * 256;
       int row, kk;
-      if (a_kcontig) { row = e >> 4; kk = e & 15; } else { row = e & 63; kk = e >> 6; }
+      if (a_kcontig) { row = e >> 4; kk = e & 15; } else { row = e % TM; kk = e / TM; }
       const int64_t m = m0 + row;
       const int k = k0 + kk;
       As[kk][row] = (m < g.M && k < k_hi) ? g.A[m * g.a_sm + k * g.a_sk] : 0.f;
-      if (b_kcontig) { row = e >> 4; kk = e & 15; } else { row = e & 63; kk = e >> 6; }
+      if (b_kcontig) { row = e >> 4; kk = e & 15; } else { row = e % TN; kk = e / TN; }
       const int64_t n = n0 + row;
       const int kb = k0 + kk;
       Bs[kk][row] = (n < g.N && kb < k_hi) ? g.B[n * g.b_sn + kb * g.b_sk] : 0.f;
@@ -45,27 +49,27 @@ simt_gemm_kernel(const SimtGemm g) {
     __syncthreads();
 #pragma unroll
     for (int kk = 0; kk < TK; ++kk) {
-      float a[4], b[4];
+      float a[R], b[R];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+      for (int i = 0; i < R; ++i) a[i] = As[kk][ty * R + i];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+      for (int j = 0; j < R; ++j) b[j] = Bs[kk][tx * R + j];
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < R; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        for (int j = 0; j < R; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
     }
     __syncthreads();
   }
 
   float* part = g.k_splits > 1 ? g.partials + static_cast<int64_t>(s) * g.M * g.N : nullptr;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int64_t m = m0 + ty * 4 + i;
+  for (int i = 0; i < R; ++i) {
+    const int64_t m = m0 + ty * R + i;
     if (m >= g.M) continue;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int64_t n = n0 + tx * 4 + j;
+    for (int j = 0; j < R; ++j) {
+      const int64_t n = n0 + tx * R + j;
       if (n >= g.N) continue;
       if (part) part[m * g.N + n] = acc[i][j];
       else epi_apply1(g.epi, m, n, acc[i][j]);
@@ -76,8 +80,14 @@ simt_gemm_kernel(const SimtGemm g) {
 }  // namespace
 
 cudaError_t simt_gemm_launch(const SimtGemm& g, cudaStream_t stream) {
-  dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM, g.k_splits);
-  simt_gemm_kernel<<<grid, 256, 0, stream>>>(g);
+  const long long big = 1ll * ((g.N + 63) / 64) * ((g.M + 63) / 64) * g.k_splits;
+  if (big >= 148) {
+    dim3 grid((g.N + 63) / 64, (g.M + 63) / 64, g.k_splits);
+    simt_gemm_kernel<4><<<grid, 256, 0, stream>>>(g);
+  } else {
+    dim3 grid((g.N + 31) / 32, (g.M + 31) / 32, g.k_splits);
+    simt_gemm_kernel<2><<<grid, 256, 0, stream>>>(g);
+  }
   return cudaGetLastError();
 }
 

@@ -59,6 +59,13 @@ struct mbd_net {
   void* X_stage = nullptr;
   int32_t* labels_stage = nullptr;
   ConvNet* conv = nullptr;
+  // cached CUDA graph of one fused step and the arguments it was captured for
+  cudaGraphExec_t graph_exec = nullptr;
+  const void* g_X = nullptr;
+  const int32_t* g_labels = nullptr;
+  float* g_loss = nullptr;
+  float g_eta = 0.f;
+  int64_t graph_launches = 0;
   size_t elt() const { return dtype == MBD_BF16 ? 2 : 4; }
 };
 
@@ -176,6 +183,7 @@ void free_net(mbd_net* n) {
   cudaFree(n->partials); cudaFree(n->colsum_scratch); cudaFree(n->per_sample); cudaFree(n->loss_dev);
   cudaFree(n->status); cudaFree(n->X_stage); cudaFree(n->labels_stage);
   if (n->conv) conv_destroy(n->conv);
+  if (n->graph_exec) cudaGraphExecDestroy(n->graph_exec);
   n->prof.destroy();
   (void)cudaGetLastError();
   delete n;
@@ -425,6 +433,44 @@ extern "C" mbd_status mbd_sgd_step(mbd_net* n, float eta) {
   return MBD_OK;
 }
 
+extern "C" mbd_status mbd_train_step(mbd_net* n, const void* X_dev, const int32_t* labels_dev, float eta, float* loss_sum_dev) {
+  if (!n || !X_dev || eta <= 0.f) return MBD_E_INVALID;
+  // per-kernel events cannot be recorded inside a graph, and the default stream cannot be captured
+  if (n->prof.on || n->stream == nullptr || n->stream == cudaStreamLegacy || n->stream == cudaStreamPerThread) {
+    mbd_status s = mbd_forward(n, X_dev, labels_dev, loss_sum_dev);
+    return s != MBD_OK ? s : mbd_backward(n, eta);
+  }
+  const bool same = n->graph_exec && n->g_X == X_dev && n->g_labels == labels_dev && n->g_loss == loss_sum_dev && n->g_eta == eta;
+  if (!same) {
+    if (n->graph_exec) { cudaGraphExecDestroy(n->graph_exec); n->graph_exec = nullptr; }
+    // first use of these buffers: build the tensor maps that refer to X outside the capture
+    n->X = X_dev;
+    mbd_status s = map_input(n);
+    if (s != MBD_OK) return s;
+    const int64_t launches_before = n->prof.total_launches;
+    CK(cudaStreamBeginCapture(n->stream, cudaStreamCaptureModeThreadLocal));
+    s = mbd_forward(n, X_dev, labels_dev, loss_sum_dev);
+    if (s == MBD_OK) s = mbd_backward(n, eta);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t ce = cudaStreamEndCapture(n->stream, &graph);
+    n->graph_launches = n->prof.total_launches - launches_before;   // kernels of one step
+    n->prof.total_launches = launches_before;                        // nothing has run yet
+    if (s != MBD_OK || ce != cudaSuccess || !graph) {
+      if (graph) cudaGraphDestroy(graph);
+      (void)cudaGetLastError();
+      return s != MBD_OK ? s : MBD_E_CUDA;
+    }
+    const cudaError_t ie = cudaGraphInstantiate(&n->graph_exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ie != cudaSuccess) { n->graph_exec = nullptr; (void)cudaGetLastError(); return MBD_E_CUDA; }
+    n->g_X = X_dev; n->g_labels = labels_dev; n->g_loss = loss_sum_dev; n->g_eta = eta;
+  }
+  CK(cudaGraphLaunch(n->graph_exec, n->stream));
+  n->prof.total_launches += n->graph_launches;
+  n->state = ST_BWD_FUSED;
+  return MBD_OK;
+}
+
 extern "C" mbd_status mbd_train_step_host(mbd_net* n, const void* X_host, const int32_t* labels_host, float eta,
                                           float* loss_host) {
   if (!n || !X_host || !loss_host || eta <= 0.f) return MBD_E_INVALID;
@@ -442,9 +488,7 @@ extern "C" mbd_status mbd_train_step_host(mbd_net* n, const void* X_host, const 
     if (!labels_host) return MBD_E_INVALID;
     CK(cudaMemcpyAsync(n->labels_stage, labels_host, n->B * sizeof(int32_t), cudaMemcpyHostToDevice, n->stream));
   }
-  mbd_status s = mbd_forward(n, n->X_stage, n->labels_stage, n->loss_dev);
-  if (s != MBD_OK) return s;
-  s = mbd_backward(n, eta);
+  mbd_status s = mbd_train_step(n, n->X_stage, n->is_conv ? nullptr : n->labels_stage, eta, n->loss_dev);
   if (s != MBD_OK) return s;
   CK(cudaMemcpyAsync(loss_host, n->loss_dev, sizeof(float), cudaMemcpyDeviceToHost, n->stream));
   CK(cudaStreamSynchronize(n->stream));

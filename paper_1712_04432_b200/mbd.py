@@ -24,7 +24,7 @@ KERNEL_CLASSES = ["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce_partia
                   "sgd_update", "halo_stage", "conv_fwd", "conv_bwd_data", "conv_bwd_weight", "other"]
 
 EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weights", "mbd_forward",
-           "mbd_backward", "mbd_sgd_step", "mbd_train_step_host", "mbd_comm_words", "mbd_get_tensor",
+           "mbd_backward", "mbd_sgd_step", "mbd_train_step", "mbd_train_step_host", "mbd_comm_words", "mbd_get_tensor",
            "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_gemm_bf16_noalloc", "mbd_selftest_timeout", "mbd_strerror"]
 
 
@@ -65,6 +65,7 @@ def lib():
         L.mbd_forward.argtypes = [vp, vp, vp, vp]
         L.mbd_backward.argtypes = [vp, f32]
         L.mbd_sgd_step.argtypes = [vp, f32]
+        L.mbd_train_step.argtypes = [vp, vp, vp, f32, vp]
         L.mbd_train_step_host.argtypes = [vp, vp, vp, f32, C.POINTER(f32)]
         L.mbd_comm_words.argtypes = [C.POINTER(Layer), i32, i64, i32, i32, C.POINTER(Words)]
         L.mbd_get_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
@@ -183,6 +184,12 @@ class Net:
 
     def sgd_step(self, eta: float):
         _check(lib().mbd_sgd_step(self._h, float(eta)), "mbd_sgd_step")
+
+    def train_step(self, X, labels, eta: float, loss_out=None):
+        """One fused step on device tensors, replayed from a CUDA graph after the first call."""
+        assert X.is_cuda and X.is_contiguous() and X.dtype == self.act_dtype
+        self._keep = [X, labels, loss_out]
+        _check(lib().mbd_train_step(self._h, _ptr(X), _ptr(labels), float(eta), _ptr(loss_out)), "mbd_train_step")
 
     def train_step_host(self, X_host, labels_host, eta: float) -> float:
         """One step from host (ideally pinned) tensors; returns J."""

@@ -107,3 +107,35 @@ def test_train_step_from_host_buffers():
         got = net.get_weights(i).float().cpu().numpy()
         assert np.linalg.norm(got - o["new_W"][i]) / np.linalg.norm(o["new_W"][i]) < 1e-2
     net.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_graph_replayed_step_equals_direct_launches(dtype):
+    import torch
+    from paper_1712_04432_b200 import mbd
+    w = I.fc_workload((136, 136, 72), 128, dtype)
+    inp = I.make_inputs(w, seed=7)
+    bf = dtype == "bf16"
+
+    def make():
+        net = mbd.Net(mbd.fc_layers(w.dims), w.B, 2, 2, mbd.BF16 if bf else mbd.F32, mbd.LOSS_SOFTMAX_CE, 2)
+        for i in range(2):
+            net.set_weights(i, to_dev(inp.Ws[i], bf), torch.from_numpy(inp.bs[i]).cuda())
+        return net
+
+    X, lab = to_dev(inp.X, bf), torch.from_numpy(inp.labels).cuda()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()                           # the default stream cannot be captured
+    with torch.cuda.stream(side):
+        a, b = make(), make()
+        Ja, Jb = torch.zeros(1, device="cuda"), torch.zeros(1, device="cuda")
+        for _ in range(3):                               # three steps: capture once, replay twice
+            a.train_step(X, lab, w.eta, Ja)
+            b.forward(X, lab, Jb)
+            b.backward(w.eta)
+        a.poll(); b.poll()
+    assert a.launch_count == b.launch_count
+    assert torch.equal(Ja, Jb)
+    for i in range(2):
+        assert torch.equal(a.get_weights(i), b.get_weights(i))
+    a.close(); b.close()
