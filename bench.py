@@ -392,7 +392,7 @@ def run_ours(args):
 # DRAM bytes per launch of the dominant kernel from an ncu capture (see profiles/); null until captured.
 # cfg5: gemm_tc_kernel at 8192^3, dram__bytes_read.sum + dram__bytes_write.sum of one launch
 # (profiles/gemm_tc_kernel_8192cubed.md; the captured launch wrote an fp32 result).
-TRAFFIC = {"cfg5": 1.29e9}
+TRAFFIC = {"cfg5": 1.06e9}
 
 
 if __name__ == "__main__":
