@@ -105,6 +105,58 @@ softmax_xent_kernel(const float* __restrict__ logits, int64_t d, const int32_t* 
   if (tid == 0) per_sample[b] = mx + logf(sum) - row[label];
 }
 
+// Same, with the whole row held in registers (VPT values per thread): one pass over HBM.
+template <int NW, int VPT>
+__global__ void __launch_bounds__(NW * 32)
+softmax_xent_reg_kernel(const float* __restrict__ logits, int64_t d, const int32_t* __restrict__ labels,
+                        void* __restrict__ dY, int dy_bf16, float* __restrict__ per_sample) {
+  __shared__ float red[NW];
+  const int64_t b = blockIdx.x;
+  const float* row = logits + b * d;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float v[VPT];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int64_t k = tid + static_cast<int64_t>(i) * NW * 32;
+    v[i] = k < d ? __ldcs(row + k) : -INFINITY;
+    mx = fmaxf(mx, v[i]);
+  }
+  mx = warp_max(mx);
+  if (NW > 1) {
+    if (lane == 0) red[warp] = mx;
+    __syncthreads();
+    mx = red[0];
+#pragma unroll
+    for (int i = 1; i < NW; ++i) mx = fmaxf(mx, red[i]);
+    __syncthreads();
+  }
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) { v[i] = expf(v[i] - mx); sum += v[i]; }     // exp(-inf) = 0 past the end
+  sum = warp_sum(sum);
+  if (NW > 1) {
+    if (lane == 0) red[warp] = sum;
+    __syncthreads();
+    sum = red[0];
+#pragma unroll
+    for (int i = 1; i < NW; ++i) sum += red[i];
+  }
+  const float inv = 1.f / sum;
+  const int label = labels[b];
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int64_t k = tid + static_cast<int64_t>(i) * NW * 32;
+    if (k < d) {
+      float g = v[i] * inv;
+      if (k == label) g -= 1.f;
+      if (dy_bf16) reinterpret_cast<__nv_bfloat16*>(dY)[b * d + k] = __float2bfloat16_rn(g);
+      else reinterpret_cast<float*>(dY)[b * d + k] = g;
+    }
+  }
+  if (tid == 0) per_sample[b] = mx + logf(sum) - row[label];
+}
+
 // ------------------------------------------------------------------ fixed-order sum
 __global__ void __launch_bounds__(1024)
 sum_f32_kernel(const float* __restrict__ x, int64_t n, float scale, float* __restrict__ out) {
@@ -243,9 +295,11 @@ cudaError_t reduce_partials_launch(const float* parts, int S, int64_t M, int64_t
 
 cudaError_t softmax_xent_launch(const float* logits, int64_t B, int64_t d, const int32_t* labels, void* dY,
                                 int dy_bf16, float* per_sample, cudaStream_t stream) {
-  if (d <= 64) softmax_xent_kernel<1><<<static_cast<unsigned>(B), 32, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
-  else if (d <= 2048) softmax_xent_kernel<4><<<static_cast<unsigned>(B), 128, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
-  else softmax_xent_kernel<8><<<static_cast<unsigned>(B), 256, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  const unsigned nb = static_cast<unsigned>(B);
+  if (d <= 64) softmax_xent_reg_kernel<1, 2><<<nb, 32, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  else if (d <= 1024) softmax_xent_reg_kernel<4, 8><<<nb, 128, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  else if (d <= 8192) softmax_xent_reg_kernel<8, 32><<<nb, 256, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  else softmax_xent_kernel<8><<<nb, 256, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
   return cudaGetLastError();
 }
 

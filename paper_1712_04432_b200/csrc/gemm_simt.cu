@@ -7,14 +7,14 @@
 namespace mbd {
 namespace {
 
-constexpr int TK = 16;
-
 // 256 threads as 16 x 16; each thread owns an R x R micro-tile of a (16R) x (16R) CTA tile.
-// R = 4 for large outputs, R = 2 when 64 x 64 tiles would leave most SMs idle.
+// R = 4 for large outputs, R = 2 (with a deeper K step, fewer load-sync round trips) when
+// 64 x 64 tiles would leave most SMs idle.
 template <int R>
 __global__ void __launch_bounds__(256)
 simt_gemm_kernel(const SimtGemm g) {
   constexpr int TM = 16 * R, TN = 16 * R;
+  constexpr int TK = R == 2 ? 64 : 16;
   __shared__ float As[TK][TM + 4];
   __shared__ float Bs[TK][TN + 4];
   const int tid = threadIdx.x;
@@ -37,11 +37,11 @@ simt_gemm_kernel(const SimtGemm g) {
     for (int i = 0; i < (TM * TK) / 256; ++i) {
       const int e = tid + i * 256;
       int row, kk;
-      if (a_kcontig) { row = e >> 4; kk = e & 15; } else { row = e % TM; kk = e / TM; }
+      if (a_kcontig) { row = e / TK; kk = e % TK; } else { row = e % TM; kk = e / TM; }
       const int64_t m = m0 + row;
       const int k = k0 + kk;
       As[kk][row] = (m < g.M && k < k_hi) ? g.A[m * g.a_sm + k * g.a_sk] : 0.f;
-      if (b_kcontig) { row = e >> 4; kk = e & 15; } else { row = e % TN; kk = e / TN; }
+      if (b_kcontig) { row = e / TK; kk = e % TK; } else { row = e % TN; kk = e / TN; }
       const int64_t n = n0 + row;
       const int kb = k0 + kk;
       Bs[kk][row] = (n < g.N && kb < k_hi) ? g.B[n * g.b_sn + kb * g.b_sk] : 0.f;

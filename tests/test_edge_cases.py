@@ -139,3 +139,10 @@ def test_graph_replayed_step_equals_direct_launches(dtype):
     for i in range(2):
         assert torch.equal(a.get_weights(i), b.get_weights(i))
     a.close(); b.close()
+
+
+def test_wide_classifier_uses_the_streaming_softmax():
+    # more than 8192 classes: the row no longer fits the register-resident kernel
+    w = I.fc_workload((72, 8264), 24, "bf16")
+    inp = I.make_inputs(w, seed=8)
+    compare_fc_step(gpu_fc_step(w, inp), oracle_fc_step(w, inp), 1e-2)
