@@ -28,7 +28,8 @@ using namespace tc;
 constexpr int BM = 128;
 constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
 constexpr int NUM_THREADS = 320;      // TMA warp, MMA warp, 8 epilogue warps
-constexpr int SMEM_RING_BYTES = 192 * 1024;
+constexpr int SMEM_DYN_BYTES = 226 * 1024;       // dynamic shared memory of every instantiation
+constexpr int RING_MAX_BYTES = SMEM_DYN_BYTES - 1024;   // after 1024-byte alignment
 
 struct Params {
   int M, N, K;
@@ -36,6 +37,7 @@ struct Params {
   float* partials;
   Epi epi;
   int* status;
+  int te;                 // epilogue moves its global data with TMA through shared memory
 };
 
 struct Work {
@@ -65,12 +67,18 @@ __device__ __forceinline__ Work decode_work(const Params& p, int w) {
 // TMEM, so the epilogue of a tile no longer overlaps the next tile's MMAs.
 template <int A_MN, int B_MN, int BN, int MH>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmAux, const Params p) {
   constexpr int BMT = BM * MH;
   constexpr int A_BYTES = BMT * BK * 2;
   constexpr int B_BYTES = BN * BK * 2;
   constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  constexpr int STAGES = SMEM_RING_BYTES / STAGE_BYTES;
+  constexpr int STAGES = RING_MAX_BYTES / STAGE_BYTES;
+  // TMA epilogue (128-row tiles only): every epilogue warp owns BN/128 staging boxes of
+  // [32 rows][64 columns] bf16 (4 KB, 128B-swizzled) behind a shorter ring.
+  constexpr int TE_BOXES = BN / 128;
+  constexpr int TE_BYTES = 8 * TE_BOXES * 4096;
+  constexpr int STAGES_TE = (RING_MAX_BYTES - TE_BYTES) / STAGE_BYTES;
   constexpr int ACC_COLS = MH * BN;                           // TMEM columns of one tile
   constexpr int ACC_BUFS = ACC_COLS * 2 <= 512 ? 2 : 1;
   constexpr int TMEM_COLS = ACC_COLS * ACC_BUFS;
@@ -82,11 +90,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __shared__ __align__(8) uint64_t empty_bar[STAGES];
   __shared__ __align__(8) uint64_t tmem_full_bar[2];
   __shared__ __align__(8) uint64_t tmem_empty_bar[2];
+  __shared__ __align__(8) uint64_t te_bar[8];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
   // 1024-byte alignment of the ring (needed by the 128B swizzle pattern)
   const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const bool te = MH == 1 && p.te != 0;
+  const int stages = te ? STAGES_TE : STAGES;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
@@ -99,6 +110,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(smem_u32(&tmem_full_bar[i]), 1);
       mbar_init(smem_u32(&tmem_empty_bar[i]), 8);
     }
+    for (int i = 0; i < 8; ++i) mbar_init(smem_u32(&te_bar[i]), 1);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -143,7 +155,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
             for (int c = 0; c < BN / 64; ++c) tma_load_2d(sb + c * (64 * BK * 2), &tmB, wk.tn * BN + c * 64, kb * BK, fb);
           }
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
     }
@@ -181,7 +193,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                           (kb > wk.kb0 || k > 0) ? 1u : 0u);
           }
           tc_commit(smem_u32(&empty_bar[stage]));   // frees the stage once these MMAs have read it
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         tc_commit(smem_u32(&tmem_full_bar[acc]));   // accumulator complete
@@ -197,6 +209,110 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     constexpr int NV = HC / 8;                    // 16-byte vectors per thread and tile
     const int q = warp & 3;
     const int half = (warp - 2) >> 2;
+    if (te) {
+      // ---- TMA epilogue: the tile's old weights / mask source arrive in this warp's staging boxes by
+      // TMA (requested before the accumulator is waited for), are combined in place with the
+      // accumulator, and leave by TMA store; the LSU never touches global memory.
+      const int e = warp - 2;
+      const uint32_t stg = ring + STAGES_TE * STAGE_BYTES + e * (TE_BOXES * 4096);
+      uint8_t* stg_gen = smem_raw + (stg - smem_u32(smem_raw));
+      const uint32_t lbar = smem_u32(&te_bar[e]);
+      uint32_t lphase = 0;
+      const bool need_load = p.epi.op == EPI_SGD || (p.epi.op == EPI_MASK && p.epi.mask != nullptr);
+      const CUtensorMap* src_map = p.epi.op == EPI_SGD ? &tmOut : &tmAux;
+      int it = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++it) {
+        const Work wk = decode_work(p, w);
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1u;
+        const int row0 = wk.tm * BM + q * 32;
+        const int col0 = wk.tn * BN + half * HC;
+        if (lane == 0) {
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");     // earlier stores have read the boxes
+          if (need_load) {
+            mbar_expect_tx(lbar, TE_BOXES * 4096);
+#pragma unroll
+            for (int b = 0; b < TE_BOXES; ++b) tma_load_2d(stg + b * 4096, src_map, col0 + b * 64, row0, lbar);
+          }
+        }
+        __syncwarp();
+        ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+        if (ok && need_load) {
+          ok = mbar_wait(lbar, lphase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+          lphase ^= 1u;
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_COLS + half * HC;
+#pragma unroll
+        for (int c = 0; c < HC / 32; ++c) {
+          uint32_t r[32];
+          tc_ld32(taddr + c * 32, r);
+          tc_wait_ld();
+          if (c == HC / 32 - 1) {                  // accumulator fully in registers: hand it back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+          }
+          uint8_t* box = stg_gen + (c >> 1) * 4096 + lane * 128;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint4* cell = reinterpret_cast<uint4*>(box + ((((c & 1) * 4 + j) ^ (lane & 7)) << 4));
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j * 8 + i]);
+            if (need_load) {
+              const uint4 qv = *cell;
+              const uint32_t wv[4] = {qv.x, qv.y, qv.z, qv.w};
+              if (p.epi.op == EPI_SGD) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  v[2 * i] = fmaf(p.epi.scale, v[2 * i], bf16_bits_to_f32(wv[i] & 0xFFFFu));
+                  v[2 * i + 1] = fmaf(p.epi.scale, v[2 * i + 1], bf16_bits_to_f32(wv[i] >> 16));
+                }
+              } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  if (!(bf16_bits_to_f32(wv[i] & 0xFFFFu) > 0.f)) v[2 * i] = 0.f;
+                  if (!(bf16_bits_to_f32(wv[i] >> 16) > 0.f)) v[2 * i + 1] = 0.f;
+                }
+              }
+            } else if (p.epi.op == EPI_ACT) {
+              const int n = col0 + c * 32 + j * 8;
+              if (p.epi.bias && n < p.N) {
+                const float4 b0 = *reinterpret_cast<const float4*>(p.epi.bias + n);
+                const float4 b1 = *reinterpret_cast<const float4*>(p.epi.bias + n + 4);
+                v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
+                v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+              }
+              if (p.epi.relu) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] = fmaxf(v[i], 0.f);
+              }
+            }
+            uint4 o;
+            o.x = pack_bf16x2(v[0], v[1]); o.y = pack_bf16x2(v[2], v[3]);
+            o.z = pack_bf16x2(v[4], v[5]); o.w = pack_bf16x2(v[6], v[7]);
+            *cell = o;
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // generic writes -> visible to TMA
+        __syncwarp();
+        if (lane == 0) {
+#pragma unroll
+          for (int b = 0; b < TE_BOXES; ++b) {
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                         ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(col0 + b * 64), "r"(row0), "r"(stg + b * 4096)
+                         : "memory");
+          }
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+      }
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // stores done before the CTA exits
+      __syncwarp();
+    } else {
     const bool prefetch = p.S == 1 && p.epi.out_bf16 &&
                           (p.epi.op == EPI_SGD || (p.epi.op == EPI_MASK && p.epi.mask != nullptr));
     const __nv_bfloat16* pre_src = p.epi.op == EPI_SGD ? reinterpret_cast<const __nv_bfloat16*>(p.epi.out)
@@ -280,6 +396,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
       }   // h
     }
+    }   // register epilogue
   }
 
   tc_fence_before();
@@ -328,19 +445,19 @@ cudaError_t make_map(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t
 template <int A_MN, int B_MN>
 cudaError_t set_attr() {
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_RING_BYTES + 1024)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_RING_BYTES + 1024)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_RING_BYTES + 1024)) != cudaSuccess) return e;
-  return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_RING_BYTES + 1024);
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES);
 }
 
 template <int A_MN, int B_MN>
 cudaError_t launch_t(const TcGemm& g, const Params& p, cudaStream_t stream) {
-  const size_t smem = SMEM_RING_BYTES + 1024;
-  if (g.BN == 256 && g.MH == 1) gemm_tc_kernel<A_MN, B_MN, 256, 1><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, p);
-  else if (g.BN == 128 && g.MH == 1) gemm_tc_kernel<A_MN, B_MN, 128, 1><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, p);
-  else if (g.BN == 256) gemm_tc_kernel<A_MN, B_MN, 256, 2><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, p);
-  else gemm_tc_kernel<A_MN, B_MN, 128, 2><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, p);
+  const size_t smem = SMEM_DYN_BYTES;
+  if (g.BN == 256 && g.MH == 1) gemm_tc_kernel<A_MN, B_MN, 256, 1><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  else if (g.BN == 128 && g.MH == 1) gemm_tc_kernel<A_MN, B_MN, 128, 1><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  else if (g.BN == 256) gemm_tc_kernel<A_MN, B_MN, 256, 2><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  else gemm_tc_kernel<A_MN, B_MN, 128, 2><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
   return cudaGetLastError();
 }
 
@@ -366,7 +483,8 @@ cudaError_t selftest_timeout_launch(int* status, int limit_ms, cudaStream_t stre
   return cudaGetLastError();
 }
 
-cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B, int64_t ldb, int num_sms) {
+cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B, int64_t ldb, int num_sms,
+                            const Epi* te_epi) {
   cudaError_t e = tc_gemm_init();
   if (e != cudaSuccess) return e;
   const int kb_total = (g.K + BK - 1) / BK;
@@ -399,6 +517,21 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
   if (e != cudaSuccess) return e;
   if (!b_mn) e = make_map(&g.tmB, B, g.K, g.N, ldb, BK, g.BN);    // B[N,K]
   else e = make_map(&g.tmB, B, g.N, g.K, ldb, 64, BK);             // B[K,N]
+  if (e != cudaSuccess) return e;
+  // TMA epilogue: bf16 output of an unsplit contraction on 128-row tiles
+  g.te = 0;
+  g.tmOut = g.tmA;
+  g.tmAux = g.tmA;
+  if (te_epi && te_epi->out_bf16 && te_epi->out && g.MH == 1 && g.k_splits == 1 && !getenv("MBD_TC_NO_TE")) {
+    e = make_map(&g.tmOut, te_epi->out, g.N, g.M, te_epi->ldo, 64, 32);
+    if (e != cudaSuccess) return e;
+    if (te_epi->op == EPI_MASK && te_epi->mask) {
+      e = make_map(&g.tmAux, te_epi->mask, g.N, g.M, te_epi->ldmask, 64, 32);
+      if (e != cudaSuccess) return e;
+    }
+    g.te = 1;
+    g.te_epi = *te_epi;
+  }
   return e;
 }
 
@@ -414,6 +547,8 @@ cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
   p.partials = g.partials;
   p.epi = g.epi;
   p.status = g.status;
+  p.te = g.te && g.epi.op == g.te_epi.op && g.epi.out == g.te_epi.out && g.epi.out_bf16 && g.epi.mask == g.te_epi.mask &&
+         g.epi.ldo == g.te_epi.ldo && g.k_splits == 1;
   if (g.variant == 0) return launch_t<0, 0>(g, p, stream);
   if (g.variant == 1) return launch_t<0, 1>(g, p, stream);
   return launch_t<1, 1>(g, p, stream);

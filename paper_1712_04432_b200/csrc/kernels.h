@@ -45,6 +45,9 @@ struct Epi {
 // variant 2: D[M,N] = A[K,M]^T B[K,N]      (A M-contiguous, B N-cont.)  backward-weight
 struct TcGemm {
   CUtensorMap tmA, tmB;
+  CUtensorMap tmOut, tmAux;   // output / mask-source maps of the TMA epilogue (valid when te)
+  int te;                     // plan allows the TMA epilogue for te_epi
+  Epi te_epi;
   int variant;
   int BN;               // CTA tile width: 256 or 128
   int MH;               // CTA tile height in units of 128 rows: 1 or 2
@@ -57,8 +60,10 @@ struct TcGemm {
 };
 
 // Fills tmA/tmB/BN/grid.  Returns cudaSuccess or an error.
+// `te_epi` (may be null): the epilogue this contraction will run with, if its output is bf16;
+// lets the plan move the epilogue's global traffic with TMA.
 cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B, int64_t ldb,
-                            int num_sms);
+                            int num_sms, const Epi* te_epi);
 cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream);
 cudaError_t selftest_timeout_launch(int* status, int limit_ms, cudaStream_t stream);
 cudaError_t tc_gemm_init();   // driver entry point lookup + kernel attributes; idempotent

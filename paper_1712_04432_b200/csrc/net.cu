@@ -150,26 +150,39 @@ mbd_status run_gemm(mbd_net* n, TcGemm& tc, int variant, int64_t M, int64_t N, i
 }
 
 mbd_status prepare_tc(mbd_net* n, TcGemm& g, int variant, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
-                      const void* Bm, int64_t ldb, int S) {
+                      const void* Bm, int64_t ldb, int S, const Epi* te_epi) {
   g = TcGemm{};
   g.variant = variant;
   g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
   g.k_splits = S;
   g.status = n->status;
-  CK(tc_gemm_prepare(g, A, lda, Bm, ldb, n->num_sms));
+  CK(tc_gemm_prepare(g, A, lda, Bm, ldb, n->num_sms, te_epi));
   return MBD_OK;
 }
 
 const void* layer_input(const mbd_net* n, int i) { return i == 0 ? n->X : n->layers[i - 1].act; }
+
+// The epilogues of the three products of layer i (the scale of the update is set at launch).
+Epi fwd_epi(mbd_net* n, int i) {
+  Layer& l = n->layers[i];
+  const bool last = i == n->L - 1;
+  return epi_act(l.act, l.d_out, last ? 0 : (n->dtype == MBD_BF16), l.bias, (!last && l.spec.relu) ? 1 : 0);
+}
+Epi bwd_data_epi(mbd_net* n, int i) {
+  Layer& l = n->layers[i];
+  Layer& prev = n->layers[i - 1];
+  return epi_mask(prev.dY, l.d_in, n->dtype == MBD_BF16, prev.spec.relu ? prev.act : nullptr, l.d_in);
+}
 
 // (Re)build the tensor maps that reference the caller's input buffer.
 mbd_status map_input(mbd_net* n) {
   if (n->dtype != MBD_BF16 || n->is_conv || n->X_mapped == n->X) return MBD_OK;
   Layer& l = n->layers[0];
   const int S_c = splits_for(n->P_c, n->max_partials);
-  mbd_status s = prepare_tc(n, l.fwd, 0, n->B, l.d_out, l.d_in, n->X, l.d_in, l.W, l.d_in, 1);
+  const Epi ef = fwd_epi(n, 0), ew = epi_sgd(l.W, l.d_in, 1, 0.f);
+  mbd_status s = prepare_tc(n, l.fwd, 0, n->B, l.d_out, l.d_in, n->X, l.d_in, l.W, l.d_in, 1, &ef);
   if (s != MBD_OK) return s;
-  s = prepare_tc(n, l.bwd_weight, 2, l.d_out, l.d_in, n->B, l.dY, l.d_out, n->X, l.d_in, S_c);
+  s = prepare_tc(n, l.bwd_weight, 2, l.d_out, l.d_in, n->B, l.dY, l.d_out, n->X, l.d_in, S_c, &ew);
   if (s != MBD_OK) return s;
   n->X_mapped = n->X;
   return MBD_OK;
@@ -291,9 +304,13 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
     for (int i = 0; i < L; ++i) {
       Layer& l = n->layers[i];
       const void* x_in = i > 0 ? n->layers[i - 1].act : l.W;       // placeholder address for layer 1
-      st = prepare_tc(n, l.fwd, 0, B, l.d_out, l.d_in, x_in, l.d_in, l.W, l.d_in, 1);
-      if (st == MBD_OK && i > 0) st = prepare_tc(n, l.bwd_data, 1, B, l.d_in, l.d_out, l.dY, l.d_out, l.W, l.d_in, S_r);
-      if (st == MBD_OK) st = prepare_tc(n, l.bwd_weight, 2, l.d_out, l.d_in, B, l.dY, l.d_out, x_in, l.d_in, S_c);
+      const Epi ef = fwd_epi(n, i), ew = epi_sgd(l.W, l.d_in, 1, 0.f);
+      st = prepare_tc(n, l.fwd, 0, B, l.d_out, l.d_in, x_in, l.d_in, l.W, l.d_in, 1, &ef);
+      if (st == MBD_OK && i > 0) {
+        const Epi ed = bwd_data_epi(n, i);
+        st = prepare_tc(n, l.bwd_data, 1, B, l.d_in, l.d_out, l.dY, l.d_out, l.W, l.d_in, S_r, &ed);
+      }
+      if (st == MBD_OK) st = prepare_tc(n, l.bwd_weight, 2, l.d_out, l.d_in, B, l.dY, l.d_out, x_in, l.d_in, S_c, &ew);
       if (st != MBD_OK) { free_net(n); return st; }
       if (l.fwd.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.fwd.k_splits) * B * l.d_out);
       if (i > 0 && l.bwd_data.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.bwd_data.k_splits) * B * l.d_in);
@@ -357,7 +374,7 @@ extern "C" mbd_status mbd_forward(mbd_net* n, const void* X_dev, const int32_t* 
   for (int i = 0; i < n->L; ++i) {
     Layer& l = n->layers[i];
     const bool last = i == n->L - 1;
-    const Epi e = epi_act(l.act, l.d_out, last ? 0 : bf, l.bias, (!last && l.spec.relu) ? 1 : 0);
+    const Epi e = fwd_epi(n, i);
     s = run_gemm(n, l.fwd, 0, n->B, l.d_out, l.d_in, layer_input(n, i), l.d_in, l.W, l.d_in, 1, e);
     if (s != MBD_OK) return s;
   }
@@ -396,8 +413,7 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
       n->prof.total_launches += colsum_launches(n->B, l.d_out, n->num_sms) - 1;
     }
     if (i > 0) {   // nothing is propagated below the first layer
-      Layer& prev = n->layers[i - 1];
-      const Epi e = epi_mask(prev.dY, l.d_in, bf, prev.spec.relu ? prev.act : nullptr, l.d_in);
+      const Epi e = bwd_data_epi(n, i);
       mbd_status s = run_gemm(n, l.bwd_data, 1, n->B, l.d_in, l.d_out, l.dY, l.d_out, l.W, l.d_in, S_r, e);
       if (s != MBD_OK) return s;
     }
@@ -589,7 +605,7 @@ extern "C" mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K
   g.status = status;
   mbd_status ret = MBD_OK;
   do {
-    if (tc_gemm_prepare(g, A, lda, Bm, ldb, sms) != cudaSuccess) { ret = MBD_E_CUDA; break; }
+    if (tc_gemm_prepare(g, A, lda, Bm, ldb, sms, nullptr) != cudaSuccess) { ret = MBD_E_CUDA; break; }
     g.epi = epi_act(D, ldd, 0, nullptr, 0);
     g.partials = partials;
     if (tc_gemm_launch(g, stream) != cudaSuccess) { ret = MBD_E_CUDA; break; }

@@ -61,7 +61,7 @@ extern "C" mbd_status mbd_gemm_bf16_noalloc(int variant, int64_t M, int64_t N, i
   g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
   g.k_splits = static_cast<int>(S);
   g.status = status;
-  if (tc_gemm_prepare(g, A, lda, Bm, ldb, sms) != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
+  if (tc_gemm_prepare(g, A, lda, Bm, ldb, sms, nullptr) != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
   g.epi = Epi{};
   g.epi.op = EPI_ACT; g.epi.out = D; g.epi.ldo = ldd;
   g.partials = scratch;
