@@ -106,7 +106,8 @@ softmax_xent_kernel(const float* __restrict__ logits, int64_t d, const int32_t* 
 }
 
 // Same, with the whole row held in registers (VPT values per thread): one pass over HBM.
-template <int NW, int VPT>
+// VEC: d is a multiple of 4 and every thread owns groups of 4 consecutive classes (16-byte loads).
+template <int NW, int VPT, bool VEC>
 __global__ void __launch_bounds__(NW * 32)
 softmax_xent_reg_kernel(const float* __restrict__ logits, int64_t d, const int32_t* __restrict__ labels,
                         void* __restrict__ dY, int dy_bf16, float* __restrict__ per_sample) {
@@ -114,14 +115,27 @@ softmax_xent_reg_kernel(const float* __restrict__ logits, int64_t d, const int32
   const int64_t b = blockIdx.x;
   const float* row = logits + b * d;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int G = VEC ? 4 : 1;                 // consecutive classes per group
+  auto index = [&](int i) -> int64_t { return (static_cast<int64_t>(i / G) * NW * 32 + tid) * G + (i % G); };
   float v[VPT];
   float mx = -INFINITY;
+  if (VEC) {
 #pragma unroll
-  for (int i = 0; i < VPT; ++i) {
-    const int64_t k = tid + static_cast<int64_t>(i) * NW * 32;
-    v[i] = k < d ? __ldcs(row + k) : -INFINITY;
-    mx = fmaxf(mx, v[i]);
+    for (int i = 0; i < VPT; i += 4) {
+      const int64_t k = index(i);
+      float4 q = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+      if (k < d) q = __ldcs(reinterpret_cast<const float4*>(row + k));
+      v[i] = q.x; v[i + 1] = q.y; v[i + 2] = q.z; v[i + 3] = q.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int64_t k = index(i);
+      v[i] = k < d ? __ldcs(row + k) : -INFINITY;
+    }
   }
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) mx = fmaxf(mx, v[i]);
   mx = warp_max(mx);
   if (NW > 1) {
     if (lane == 0) red[warp] = mx;
@@ -146,12 +160,31 @@ softmax_xent_reg_kernel(const float* __restrict__ logits, int64_t d, const int32
   const int label = labels[b];
 #pragma unroll
   for (int i = 0; i < VPT; ++i) {
-    const int64_t k = tid + static_cast<int64_t>(i) * NW * 32;
-    if (k < d) {
-      float g = v[i] * inv;
-      if (k == label) g -= 1.f;
-      if (dy_bf16) reinterpret_cast<__nv_bfloat16*>(dY)[b * d + k] = __float2bfloat16_rn(g);
-      else reinterpret_cast<float*>(dY)[b * d + k] = g;
+    v[i] *= inv;
+    if (index(i) == label) v[i] -= 1.f;
+  }
+  if (VEC) {
+#pragma unroll
+    for (int i = 0; i < VPT; i += 4) {
+      const int64_t k = index(i);
+      if (k < d) {
+        if (dy_bf16) {
+          uint2 o;
+          o.x = pack_bf16x2(v[i], v[i + 1]); o.y = pack_bf16x2(v[i + 2], v[i + 3]);
+          *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(dY) + b * d + k) = o;
+        } else {
+          *reinterpret_cast<float4*>(reinterpret_cast<float*>(dY) + b * d + k) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+        }
+      }
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int64_t k = index(i);
+      if (k < d) {
+        if (dy_bf16) reinterpret_cast<__nv_bfloat16*>(dY)[b * d + k] = __float2bfloat16_rn(v[i]);
+        else reinterpret_cast<float*>(dY)[b * d + k] = v[i];
+      }
     }
   }
   if (tid == 0) per_sample[b] = mx + logf(sum) - row[label];
@@ -296,9 +329,12 @@ cudaError_t reduce_partials_launch(const float* parts, int S, int64_t M, int64_t
 cudaError_t softmax_xent_launch(const float* logits, int64_t B, int64_t d, const int32_t* labels, void* dY,
                                 int dy_bf16, float* per_sample, cudaStream_t stream) {
   const unsigned nb = static_cast<unsigned>(B);
-  if (d <= 64) softmax_xent_reg_kernel<1, 2><<<nb, 32, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
-  else if (d <= 1024) softmax_xent_reg_kernel<4, 8><<<nb, 128, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
-  else if (d <= 8192) softmax_xent_reg_kernel<8, 32><<<nb, 256, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  const bool vec = d % 4 == 0;
+  if (d <= 64) softmax_xent_reg_kernel<1, 2, false><<<nb, 32, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  else if (d <= 1024 && vec) softmax_xent_reg_kernel<4, 8, true><<<nb, 128, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  else if (d <= 1024) softmax_xent_reg_kernel<4, 8, false><<<nb, 128, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  else if (d <= 8192 && vec) softmax_xent_reg_kernel<8, 32, true><<<nb, 256, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
+  else if (d <= 8192) softmax_xent_reg_kernel<8, 32, false><<<nb, 256, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
   else softmax_xent_kernel<8><<<nb, 256, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
   return cudaGetLastError();
 }

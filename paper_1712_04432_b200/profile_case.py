@@ -5,10 +5,13 @@ a profiler (small, self-terminating):
     python -m paper_1712_04432_b200.profile_case gemm_bwd_weight --size 4096
     python -m paper_1712_04432_b200.profile_case reduce --size 8192 --splits 2
     python -m paper_1712_04432_b200.profile_case conv --batch 4 --strips 4
+    python -m paper_1712_04432_b200.profile_case fc --batch 8192 --dims 1024,8192
 
 gemm_*: one tensor-core contraction of size^3 in the operand layout of that product.
 reduce: a split contraction followed by the partial-sum reduction (the reduction reads
 `splits` fp32 planes of size^2 and writes one).
+fc:     `launches` training steps of a small fully connected net (softmax, bias-gradient and
+        update kernels at a size where their DRAM figures mean something).
 conv:   `launches` training steps of the two-layer 3x3 convolution stack on `batch` images of
 64 x 224 x 224, cut into `strips` row strips.
 """
@@ -21,7 +24,8 @@ from . import mbd
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce", "conv"])
+    ap.add_argument("case", choices=["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce", "conv", "fc"])
+    ap.add_argument("--dims", default="1024,8192")
     ap.add_argument("--batch", type=int, default=4)
     ap.add_argument("--strips", type=int, default=4)
     ap.add_argument("--size", type=int, default=8192)
@@ -30,6 +34,8 @@ def main():
     a = ap.parse_args()
     if a.case == "conv":
         return conv_case(a)
+    if a.case == "fc":
+        return fc_case(a)
     g = torch.Generator(device="cuda").manual_seed(0)
     n = a.size
     A = torch.randn((n, n), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
@@ -46,6 +52,24 @@ def main():
     ms = ev0.elapsed_time(ev1) / a.launches
     print(f"{a.case} size={n} splits={splits}: {ms:.3f} ms per call, {2 * n ** 3 / ms / 1e9:.1f} TFLOP/s, "
           f"checksum {float(D.double().sum()):.6e}")
+
+
+def fc_case(a):
+    g = torch.Generator(device="cuda").manual_seed(0)
+    dims = [int(d) for d in a.dims.split(",")]
+    net = mbd.Net(mbd.fc_layers(dims), a.batch, 1, 1, mbd.BF16, mbd.LOSS_SOFTMAX_CE, 0)
+    for i in range(len(dims) - 1):
+        W = (torch.randn((dims[i + 1], dims[i]), generator=g, device="cuda") / dims[i] ** 0.5).to(torch.bfloat16)
+        net.set_weights(i, W)
+    X = torch.randn((a.batch, dims[0]), generator=g, device="cuda").to(torch.bfloat16)
+    labels = torch.randint(0, dims[-1], (a.batch,), generator=g, device="cuda", dtype=torch.int32)
+    J = torch.zeros(1, device="cuda")
+    for _ in range(a.launches):
+        net.forward(X, labels, J)
+        net.backward(0.01)
+    torch.cuda.synchronize()
+    net.poll()
+    print(f"fc dims={dims} batch={a.batch}: J = {J.item():.4e}")
 
 
 def conv_case(a):
