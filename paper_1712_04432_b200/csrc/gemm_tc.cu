@@ -489,25 +489,53 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
   if (e != cudaSuccess) return e;
   const int kb_total = (g.K + BK - 1) / BK;
   if (g.k_splits > kb_total) g.k_splits = kb_total;
-  // 256 x 256 tiles when there are enough of them for every SM and K is long enough (>= 32
-  // k-blocks per piece) to amortise the epilogue that such a tile cannot overlap; measured on
-  // 8192^3: 1236 -> 1445 TFLOP/s for the backward-weight layout.  Otherwise 128-row tiles.
-  g.MH = 1;
-  if (1ll * ((g.M + 255) / 256) * ((g.N + 255) / 256) * g.k_splits >= num_sms && kb_total / g.k_splits >= 32) g.MH = 2;
-  if (const char* ev = getenv("MBD_TC_MH")) {          // tuning knob
+  // Tile shape and (for the network's own contractions) an extra cut of K, chosen by a small cost
+  // model in SM clocks.  Per 64-wide k-block a CTA either waits for the tensor pipe (128 x BN x 16
+  // MMAs at 75 % / 85 % of peak for BN = 128 / 256) or for its operand fill (about 70 B/clk into
+  // shared memory, measured); 256 x 256 tiles cannot overlap their epilogue; every extra piece of K
+  // costs fp32 partial traffic and the reduction launch.  Checked against measurements: 8192^3 picks
+  // 256 x 256 (1236 -> 1445 TFLOP/s), the batch-512 forward product 512 x 4096 x 25088 picks
+  // 256 x 256 with K cut in 4.
+  {
+    double best = 1e30;
+    int best_bn = 128, best_mh = 1, best_x = 1;
+    const int x_max = g.allow_extra_split ? 8 : 1;
+    for (int mh = 1; mh <= 2; ++mh) {
+      for (int bn = 128; bn <= 256; bn += 128) {
+        for (int x = 1; x <= x_max; x *= 2) {
+          const long long S = 1ll * g.k_splits * x;
+          if (S > kb_total || (x > 1 && kb_total / S < 8)) continue;
+          const double kb = static_cast<double>(kb_total) / S;
+          const long long units = 1ll * ((g.M + 128 * mh - 1) / (128 * mh)) * ((g.N + bn - 1) / bn) * S;
+          const double waves = static_cast<double>((units + num_sms - 1) / num_sms);
+          const double mma = 4.0 * mh * (bn / 2) / (bn == 256 ? 0.85 : 0.75);
+          const double fill = (128.0 * mh + bn) * 128.0 / 70.0;
+          const double mainloop = kb * (mma > fill ? mma : fill);
+          const double epi = 2500.0 * mh * bn / 256.0 * (S > 1 ? 2.0 : 1.0);
+          const bool overlapped = mh * bn <= 256;
+          double unit = overlapped ? (mainloop > epi ? mainloop : epi) : mainloop + epi;
+          double t = waves * unit + 4000.0;
+          if (S > 1 && x > 1) {          // the reduction exists anyway when the grid itself splits K
+            const double bytes = (static_cast<double>(S) + 1.0) * g.M * g.N * 4.0;
+            t += (5e-6 + bytes / 5.5e12) * 1.9e9;
+          }
+          if (t < best) { best = t; best_bn = bn; best_mh = mh; best_x = x; }
+        }
+      }
+    }
+    g.BN = best_bn; g.MH = best_mh;
+    g.k_splits *= best_x;
+  }
+  if (const char* ev = getenv("MBD_TC_MH")) {          // tuning knobs
     const int mh = atoi(ev);
     if (mh == 1 || mh == 2) g.MH = mh;
   }
-  const int bmt = BM * g.MH;
-  const int tiles_m = (g.M + bmt - 1) / bmt;
-  // 256-wide tiles unless they would leave SMs without work; then 128.  (64-wide tiles and an
-  // extra cut of K for occupancy were measured on the small-batch workloads and lost: the
-  // narrow MMAs are issue-bound and the extra partial sums cost more HBM time than they save.)
-  g.BN = 1ll * tiles_m * ((g.N + 255) / 256) * g.k_splits >= num_sms ? 256 : 128;
-  if (const char* ev = getenv("MBD_TC_BN")) {          // tuning knob
+  if (const char* ev = getenv("MBD_TC_BN")) {
     const int bn = atoi(ev);
     if (bn == 128 || bn == 256) g.BN = bn;
   }
+  const int bmt = BM * g.MH;
+  const int tiles_m = (g.M + bmt - 1) / bmt;
   const int tiles_n = (g.N + g.BN - 1) / g.BN;
   const long long total = 1ll * tiles_m * tiles_n * g.k_splits;
   g.grid = static_cast<int>(total < num_sms ? total : num_sms);

@@ -155,6 +155,7 @@ mbd_status prepare_tc(mbd_net* n, TcGemm& g, int variant, int64_t M, int64_t N, 
   g.variant = variant;
   g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
   g.k_splits = S;
+  g.allow_extra_split = variant != 2;     // forward and backward-data: small outputs, cheap partials
   g.status = n->status;
   CK(tc_gemm_prepare(g, A, lda, Bm, ldb, n->num_sms, te_epi));
   return MBD_OK;
