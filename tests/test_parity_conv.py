@@ -75,3 +75,12 @@ def test_full_resolution_two_images(P_r):
     o = oracle_conv_step(w, inp)
     g = gpu_conv_step(w, inp, P_r, force_acts=stored_hidden(o))
     compare_conv_step(g, o, TOL)
+
+
+def test_full_workload_32_images_two_strips():
+    # the benchmark's launch configuration: 32 images of 64 x 224 x 224, two strips per image
+    w = I.WORKLOADS["cfg4"]
+    inp = I.make_inputs(w, seed=0)
+    o = oracle_conv_step(w, inp)
+    g = gpu_conv_step(w, inp, 2, force_acts=stored_hidden(o))
+    compare_conv_step(g, o, TOL)

@@ -111,8 +111,9 @@ def test_run_to_run_bitwise_reproducible(small_bf16):
         assert np.array_equal(a["dY"][i], b["dY"][i])
 
 
-@pytest.mark.parametrize("name,grid,mp", [("cfg2", (1, 1), 0), ("cfg2", (2, 4), 4), ("cfg2", (8, 1), 8), ("cfg2", (1, 8), 8),
-                                          ("cfg3", (4, 4), 4)])
+@pytest.mark.parametrize("name,grid,mp", [("cfg2", (1, 1), 0), ("cfg2", (2, 4), 4), ("cfg2", (4, 2), 2), ("cfg2", (8, 1), 8),
+                                          ("cfg2", (1, 8), 8), ("cfg3", (1, 1), 0), ("cfg3", (4, 4), 4), ("cfg3", (16, 1), 2),
+                                          ("cfg3", (1, 16), 16)])
 def test_full_size_fc_workloads(name, grid, mp):
     w = I.WORKLOADS[name]
     inp = I.make_inputs(w, seed=0)
