@@ -31,6 +31,47 @@ constexpr int NUM_THREADS = 320;      // TMA warp, MMA warp, 8 epilogue warps
 constexpr int SMEM_DYN_BYTES = 226 * 1024;       // dynamic shared memory of every instantiation
 constexpr int RING_MAX_BYTES = SMEM_DYN_BYTES - 1024;   // after 1024-byte alignment
 
+// ---- CTA-pair (cta_group::2) helpers
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {   // same variable in CTA `rank` of the cluster
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load issued by either CTA of a pair; the transaction bytes are counted on `bar`, which may
+// live in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far are done
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
+}
+
 struct Params {
   int M, N, K;
   int tiles_m, tiles_n, kb_total, S, group_m;
@@ -65,13 +106,22 @@ __device__ __forceinline__ Work decode_work(const Params& p, int w) {
 // issues two MMAs per k-step against the same B tile, which cuts the shared-memory fill per
 // flop by a third (64 instead of 96 bytes per clock at BN = 256); with BN = 256 it fills all of
 // TMEM, so the epilogue of a tile no longer overlaps the next tile's MMAs.
-template <int A_MN, int B_MN, int BN, int MH>
+//
+// PAIR = 1: two CTAs of a cluster work on one 256 x BN tile with cta_group::2 MMAs issued by the
+// even CTA.  Each CTA loads its own 128 rows of A and its own half of the B tile (the tensor core
+// reads both halves), keeps its 128 rows of the accumulator in its own TMEM and runs its own
+// epilogue: 64 B/clk of operand fill like the 256 x 256 tile, but with two accumulators (the
+// epilogue overlaps the next tile), 32 KB stages and the TMA epilogue.
+template <int A_MN, int B_MN, int BN, int MH, int PAIR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmAux, const Params p) {
-  constexpr int BMT = BM * MH;
+  static_assert(!PAIR || MH == 1, "a CTA of a pair owns 128 rows");
+  constexpr int BMT = BM * MH;                                // rows owned by this CTA
+  constexpr int TILE_M = BMT * (PAIR ? 2 : 1);                // rows of the (pair's) tile
+  constexpr int BNL = PAIR ? BN / 2 : BN;                     // B rows (tile columns) loaded by this CTA
   constexpr int A_BYTES = BMT * BK * 2;
-  constexpr int B_BYTES = BN * BK * 2;
+  constexpr int B_BYTES = BNL * BK * 2;
   constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   constexpr int STAGES = RING_MAX_BYTES / STAGE_BYTES;
   // TMA epilogue (128-row tiles only): every epilogue warp owns BN/128 staging boxes of
@@ -83,7 +133,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   constexpr int ACC_BUFS = ACC_COLS * 2 <= 512 ? 2 : 1;
   constexpr int TMEM_COLS = ACC_COLS * ACC_BUFS;
   constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(A_MN) << 15) | (uint32_t(B_MN) << 16) |
-                             (uint32_t(BN >> 3) << 17) | (uint32_t(BM >> 4) << 24);
+                             (uint32_t(BN >> 3) << 17) | (uint32_t((PAIR ? 2 * BM : BM) >> 4) << 24);
 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[STAGES];
@@ -100,6 +150,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int stages = te ? STAGES_TE : STAGES;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;        // 0 = the CTA that issues the MMAs
+  const int w_first = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int w_step = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) {
@@ -108,20 +161,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&tmem_full_bar[i]), 1);
-      mbar_init(smem_u32(&tmem_empty_bar[i]), 8);
+      mbar_init(smem_u32(&tmem_empty_bar[i]), PAIR ? 16 : 8);
     }
     for (int i = 0; i < 8; ++i) mbar_init(smem_u32(&te_bar[i]), 1);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                 "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (PAIR) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                   "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                   "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();            // both CTAs' barriers exist before anything remote touches them
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
@@ -134,26 +193,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+      for (int w = w_first; w < total_work && ok; w += w_step) {
         const Work wk = decode_work(p, w);
+        const int row0 = wk.tm * TILE_M + static_cast<int>(rank) * BMT;       // this CTA's rows of A
+        const int col0 = wk.tn * BN + static_cast<int>(rank) * BNL;           // this CTA's part of the B tile
         for (int kb = wk.kb0; kb < wk.kb1; ++kb) {
           ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
           if (!ok) break;
-          const uint32_t fb = smem_u32(&full_bar[stage]);
           const uint32_t sa = ring + stage * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
-          mbar_expect_tx(fb, STAGE_BYTES);
+          // pair: the bytes of both CTAs are counted on the full barrier of CTA 0, which expects them
+          const uint32_t fb = PAIR ? map_to_cta(smem_u32(&full_bar[stage]), 0) : smem_u32(&full_bar[stage]);
+          if (!PAIR) mbar_expect_tx(fb, STAGE_BYTES);
+          else if (rank == 0) mbar_expect_tx(smem_u32(&full_bar[stage]), 2 * STAGE_BYTES);
+          auto load = [&](uint32_t dst, const CUtensorMap* tm, int x, int y) {
+            if (PAIR) tma_load_2d_pair(dst, tm, x, y, fb);
+            else tma_load_2d(dst, tm, x, y, fb);
+          };
           if (A_MN == 0) {
-            tma_load_2d(sa, &tmA, kb * BK, wk.tm * BMT, fb);
+            load(sa, &tmA, kb * BK, row0);
           } else {
 #pragma unroll
-            for (int c = 0; c < BMT / 64; ++c) tma_load_2d(sa + c * (64 * BK * 2), &tmA, wk.tm * BMT + c * 64, kb * BK, fb);
+            for (int c = 0; c < BMT / 64; ++c) load(sa + c * (64 * BK * 2), &tmA, row0 + c * 64, kb * BK);
           }
           if (B_MN == 0) {
-            tma_load_2d(sb, &tmB, kb * BK, wk.tn * BN, fb);
+            load(sb, &tmB, kb * BK, col0);
           } else {
 #pragma unroll
-            for (int c = 0; c < BN / 64; ++c) tma_load_2d(sb + c * (64 * BK * 2), &tmB, wk.tn * BN + c * 64, kb * BK, fb);
+            for (int c = 0; c < BNL / 64; ++c) load(sb + c * (64 * BK * 2), &tmB, col0 + c * 64, kb * BK);
           }
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
@@ -161,12 +228,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++it) {
+      for (int w = w_first; w < total_work && ok; w += w_step, ++it) {
         const Work wk = decode_work(p, w);
         const int acc = it % ACC_BUFS;
         const uint32_t acc_phase = (it / ACC_BUFS) & 1u;
@@ -188,15 +255,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
 #pragma unroll
-            for (int h = 0; h < MH; ++h)
-              tc_mma_bf16(d_tmem + h * BN, adesc + h * A_HALF + k * A_STEP, bdesc + k * B_STEP, IDESC,
-                          (kb > wk.kb0 || k > 0) ? 1u : 0u);
+            for (int h = 0; h < MH; ++h) {
+              if (PAIR) tc_mma_bf16_pair(d_tmem, adesc + k * A_STEP, bdesc + k * B_STEP, IDESC, (kb > wk.kb0 || k > 0) ? 1u : 0u);
+              else tc_mma_bf16(d_tmem + h * BN, adesc + h * A_HALF + k * A_STEP, bdesc + k * B_STEP, IDESC,
+                               (kb > wk.kb0 || k > 0) ? 1u : 0u);
+            }
           }
-          tc_commit(smem_u32(&empty_bar[stage]));   // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if (PAIR) tc_commit_pair(smem_u32(&empty_bar[stage]));
+          else tc_commit(smem_u32(&empty_bar[stage]));
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        tc_commit(smem_u32(&tmem_full_bar[acc]));   // accumulator complete
+        if (PAIR) tc_commit_pair(smem_u32(&tmem_full_bar[acc]));   // accumulator complete (both CTAs' halves)
+        else tc_commit(smem_u32(&tmem_full_bar[acc]));
       }
     }
   } else {
@@ -222,11 +294,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const CUtensorMap* src_map = p.epi.op == EPI_SGD ? &tmOut : &tmAux;
       int it = 0;
       bool ok = true;
-      for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++it) {
+      for (int w = w_first; w < total_work && ok; w += w_step, ++it) {
         const Work wk = decode_work(p, w);
         const int acc = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1u;
-        const int row0 = wk.tm * BM + q * 32;
+        const int row0 = wk.tm * TILE_M + static_cast<int>(rank) * BMT + q * 32;
         const int col0 = wk.tn * BN + half * HC;
         if (lane == 0) {
           asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");     // earlier stores have read the boxes
@@ -254,7 +326,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (c == HC / 32 - 1) {                  // accumulator fully in registers: hand it back
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+            if (lane == 0) {
+              if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty_bar[acc]), 0));
+              else mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+            }
           }
           uint8_t* box = stg_gen + (c >> 1) * 4096 + lane * 128;
 #pragma unroll
@@ -320,7 +395,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int64_t pre_ld = p.epi.op == EPI_SGD ? p.epi.ldo : p.epi.ldmask;
     int it = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++it) {
+    for (int w = w_first; w < total_work && ok; w += w_step, ++it) {
       const Work wk = decode_work(p, w);
       const int acc = it % ACC_BUFS;
       const uint32_t acc_phase = (it / ACC_BUFS) & 1u;
@@ -328,7 +403,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       float* part = p.S > 1 ? p.partials + static_cast<int64_t>(wk.s) * p.M * p.N : nullptr;
 #pragma unroll 1
       for (int h = 0; h < MH; ++h) {
-      const int64_t m = static_cast<int64_t>(wk.tm) * BMT + h * 128 + q * 32 + lane;
+      const int64_t m = static_cast<int64_t>(wk.tm) * TILE_M + rank * BMT + h * 128 + q * 32 + lane;
       const bool row_ok = m < p.M;
       uint4 pre[NV];
       if (prefetch) {
@@ -353,7 +428,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (h == MH - 1 && c == HC / 32 - 1) {     // accumulator fully in registers: hand it back
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+          if (lane == 0) {
+            if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty_bar[acc]), 0));
+            else mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+          }
         }
         if (row_ok) {
 #pragma unroll
@@ -401,10 +479,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();            // the peer may still signal barriers in this CTA's shared memory
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
@@ -445,19 +525,33 @@ cudaError_t make_map(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t
 template <int A_MN, int B_MN>
 cudaError_t set_attr() {
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
-  return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES);
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES);
 }
 
 template <int A_MN, int B_MN>
 cudaError_t launch_t(const TcGemm& g, const Params& p, cudaStream_t stream) {
   const size_t smem = SMEM_DYN_BYTES;
-  if (g.BN == 256 && g.MH == 1) gemm_tc_kernel<A_MN, B_MN, 256, 1><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  else if (g.BN == 128 && g.MH == 1) gemm_tc_kernel<A_MN, B_MN, 128, 1><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  else if (g.BN == 256) gemm_tc_kernel<A_MN, B_MN, 256, 2><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  else gemm_tc_kernel<A_MN, B_MN, 128, 2><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  if (g.pair) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(g.grid);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<A_MN, B_MN, 256, 1, 1>, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  }
+  if (g.BN == 256 && g.MH == 1) gemm_tc_kernel<A_MN, B_MN, 256, 1, 0><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  else if (g.BN == 128 && g.MH == 1) gemm_tc_kernel<A_MN, B_MN, 128, 1, 0><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  else if (g.BN == 256) gemm_tc_kernel<A_MN, B_MN, 256, 2, 0><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  else gemm_tc_kernel<A_MN, B_MN, 128, 2, 0><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
   return cudaGetLastError();
 }
 
@@ -534,16 +628,24 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
     const int bn = atoi(ev);
     if (bn == 128 || bn == 256) g.BN = bn;
   }
-  const int bmt = BM * g.MH;
+  g.pair = 0;
+  if (const char* ev = getenv("MBD_TC_PAIR")) {        // tuning knob: CTA pairs (256 x 256 per pair)
+    if (atoi(ev) == 1) { g.pair = 1; g.MH = 1; g.BN = 256; }
+  }
+  const int bmt = BM * g.MH * (g.pair ? 2 : 1);        // rows of one work unit's tile
   const int tiles_m = (g.M + bmt - 1) / bmt;
   const int tiles_n = (g.N + g.BN - 1) / g.BN;
   const long long total = 1ll * tiles_m * tiles_n * g.k_splits;
   g.grid = static_cast<int>(total < num_sms ? total : num_sms);
+  if (g.pair) {
+    const long long pairs = total < num_sms / 2 ? total : num_sms / 2;
+    g.grid = static_cast<int>(2 * pairs);
+  }
   const bool a_mn = g.variant == 2, b_mn = g.variant >= 1;
-  if (!a_mn) e = make_map(&g.tmA, A, g.K, g.M, lda, BK, bmt);     // A[M,K]: inner = K
+  if (!a_mn) e = make_map(&g.tmA, A, g.K, g.M, lda, BK, BM * g.MH);   // A[M,K]: inner = K; box = the rows one CTA loads
   else e = make_map(&g.tmA, A, g.M, g.K, lda, 64, BK);             // A[K,M]: inner = M, one 64-wide chunk per box
   if (e != cudaSuccess) return e;
-  if (!b_mn) e = make_map(&g.tmB, B, g.K, g.N, ldb, BK, g.BN);    // B[N,K]
+  if (!b_mn) e = make_map(&g.tmB, B, g.K, g.N, ldb, BK, g.pair ? g.BN / 2 : g.BN);    // B[N,K]
   else e = make_map(&g.tmB, B, g.N, g.K, ldb, 64, BK);             // B[K,N]
   if (e != cudaSuccess) return e;
   // TMA epilogue: bf16 output of an unsplit contraction on 128-row tiles
@@ -566,7 +668,7 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
 cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
   Params p;
   p.M = g.M; p.N = g.N; p.K = g.K;
-  p.tiles_m = (g.M + BM * g.MH - 1) / (BM * g.MH);
+  p.tiles_m = (g.M + BM * g.MH * (g.pair ? 2 : 1) - 1) / (BM * g.MH * (g.pair ? 2 : 1));
   p.tiles_n = (g.N + g.BN - 1) / g.BN;
   p.kb_total = (g.K + BK - 1) / BK;
   p.S = g.k_splits;

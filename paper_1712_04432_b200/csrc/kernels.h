@@ -51,6 +51,7 @@ struct TcGemm {
   int variant;
   int BN;               // CTA tile width: 256 or 128
   int MH;               // CTA tile height in units of 128 rows: 1 or 2
+  int pair;             // two CTAs of a cluster share one 256 x 256 tile (cta_group::2)
   int allow_extra_split; // the planner may cut K further than asked (its pieces go through the same reduction)
   int M, N, K;
   int k_splits;         // S >= 1; S > 1 writes partials[S][M][N] (fp32) and skips the epilogue op
