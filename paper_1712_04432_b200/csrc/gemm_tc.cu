@@ -589,49 +589,55 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
   // shared memory, measured); 256 x 256 tiles cannot overlap their epilogue; every extra piece of K
   // costs fp32 partial traffic and the reduction launch.  Checked against measurements: 8192^3 picks
   // 256 x 256 (1236 -> 1445 TFLOP/s), the batch-512 forward product 512 x 4096 x 25088 picks
-  // 256 x 256 with K cut in 4.
+  // 256 x 256 with K cut in 4; short-K and split products pick CTA pairs (cta_group::2).
   {
     double best = 1e30;
-    int best_bn = 128, best_mh = 1, best_x = 1;
+    int best_bn = 128, best_mh = 1, best_x = 1, best_pair = 0;
     const int x_max = g.allow_extra_split ? 8 : 1;
-    for (int mh = 1; mh <= 2; ++mh) {
-      for (int bn = 128; bn <= 256; bn += 128) {
+    for (int cand = 0; cand < 3; ++cand) {           // 0: 128-row tiles, 1: 256-row tiles, 2: CTA pairs
+      const int mh = cand == 1 ? 2 : 1;
+      const bool pair = cand == 2;
+      for (int bn = pair ? 256 : 128; bn <= 256; bn += 128) {
         for (int x = 1; x <= x_max; x *= 2) {
           const long long S = 1ll * g.k_splits * x;
           if (S > kb_total || (x > 1 && kb_total / S < 8)) continue;
           const double kb = static_cast<double>(kb_total) / S;
-          const long long units = 1ll * ((g.M + 128 * mh - 1) / (128 * mh)) * ((g.N + bn - 1) / bn) * S;
-          const double waves = static_cast<double>((units + num_sms - 1) / num_sms);
-          const double mma = 4.0 * mh * (bn / 2) / (bn == 256 ? 0.85 : 0.75);
-          const double fill = (128.0 * mh + bn) * 128.0 / 70.0;
+          const int tile_m = pair ? 256 : 128 * mh;
+          const long long units = 1ll * ((g.M + tile_m - 1) / tile_m) * ((g.N + bn - 1) / bn) * S;
+          const int slots = pair ? num_sms / 2 : num_sms;
+          const double waves = static_cast<double>((units + slots - 1) / slots);
+          // per SM and k-block: tensor-pipe clocks and operand-fill clocks
+          const double mma = pair ? 4.0 * 128.0 / 0.80 : 4.0 * mh * (bn / 2) / (bn == 256 ? 0.85 : 0.75);
+          const double fill = (pair ? 256.0 : 128.0 * mh + bn) * 128.0 / 70.0;
           const double mainloop = kb * (mma > fill ? mma : fill);
           const double epi = 2500.0 * mh * bn / 256.0 * (S > 1 ? 2.0 : 1.0);
-          const bool overlapped = mh * bn <= 256;
+          const bool overlapped = pair || mh * bn <= 256;
           double unit = overlapped ? (mainloop > epi ? mainloop : epi) : mainloop + epi;
           double t = waves * unit + 4000.0;
           if (S > 1 && x > 1) {          // the reduction exists anyway when the grid itself splits K
             const double bytes = (static_cast<double>(S) + 1.0) * g.M * g.N * 4.0;
             t += (5e-6 + bytes / 5.5e12) * 1.9e9;
           }
-          if (t < best) { best = t; best_bn = bn; best_mh = mh; best_x = x; }
+          if (t < best) { best = t; best_bn = bn; best_mh = mh; best_x = x; best_pair = pair ? 1 : 0; }
         }
       }
     }
-    g.BN = best_bn; g.MH = best_mh;
+    g.BN = best_bn; g.MH = best_mh; g.pair = best_pair;
     g.k_splits *= best_x;
   }
   if (const char* ev = getenv("MBD_TC_MH")) {          // tuning knobs
     const int mh = atoi(ev);
-    if (mh == 1 || mh == 2) g.MH = mh;
+    if (mh == 1 || mh == 2) { g.MH = mh; g.pair = 0; }
   }
   if (const char* ev = getenv("MBD_TC_BN")) {
     const int bn = atoi(ev);
     if (bn == 128 || bn == 256) g.BN = bn;
   }
-  g.pair = 0;
   if (const char* ev = getenv("MBD_TC_PAIR")) {        // tuning knob: CTA pairs (256 x 256 per pair)
     if (atoi(ev) == 1) { g.pair = 1; g.MH = 1; g.BN = 256; }
+    else if (atoi(ev) == 0) g.pair = 0;
   }
+  if (g.pair) { g.MH = 1; g.BN = 256; }
   const int bmt = BM * g.MH * (g.pair ? 2 : 1);        // rows of one work unit's tile
   const int tiles_m = (g.M + bmt - 1) / bmt;
   const int tiles_n = (g.N + g.BN - 1) / g.BN;
