@@ -678,7 +678,7 @@ cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
   p.tiles_n = (g.N + g.BN - 1) / g.BN;
   p.kb_total = (g.K + BK - 1) / BK;
   p.S = g.k_splits;
-  p.group_m = 16;                       // m-tiles per raster group (L2 reuse of the B operand)
+  p.group_m = 8;                        // m-tiles per raster group (L2 reuse of the B operand)
   if (const char* ev = getenv("MBD_TC_GROUP_M")) { const int gm = atoi(ev); if (gm >= 1) p.group_m = gm; }
   p.partials = g.partials;
   p.epi = g.epi;
