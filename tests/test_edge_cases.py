@@ -146,3 +146,34 @@ def test_wide_classifier_uses_the_streaming_softmax():
     w = I.fc_workload((72, 8264), 24, "bf16")
     inp = I.make_inputs(w, seed=8)
     compare_fc_step(gpu_fc_step(w, inp), oracle_fc_step(w, inp), 1e-2)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_layers_without_bias_and_without_relu(dtype):
+    # a linear hidden layer (no ReLU, no bias): the mask and bias paths are switched off per layer
+    import torch
+    from oracle import mbd_oracle as O
+    from paper_1712_04432_b200 import mbd
+    from tests.helpers import bf16_store, rel_fro, to_np
+    bf = dtype == "bf16"
+    w = I.fc_workload((136, 72, 40, 24), 32, dtype)
+    inp = I.make_inputs(w, seed=9)
+    flags = [(1, 0), (0, 1), (1, 1)]                    # (relu, bias) per layer
+    layers = [mbd.Layer(kind=mbd.FC, split=mbd.SPLIT_MODEL, relu=r, bias=b, d_in=w.dims[i], d_out=w.dims[i + 1])
+              for i, (r, b) in enumerate(flags)]
+    net = mbd.Net(layers, w.B, 2, 2, mbd.BF16 if bf else mbd.F32, mbd.LOSS_SOFTMAX_CE, 4)
+    for i in range(3):
+        net.set_weights(i, to_dev(inp.Ws[i], bf), torch.from_numpy(inp.bs[i]).cuda() if flags[i][1] else None)
+    X, lab = to_dev(inp.X, bf), torch.from_numpy(inp.labels).cuda()
+    net.forward(X, lab)
+    net.backward(0.0)
+    net.poll()
+    ol = [O.FC(inp.Ws[i].astype(np.float64), inp.bs[i].astype(np.float64) if flags[i][1] else None, relu=bool(flags[i][0]))
+          for i in range(3)]
+    o = O.train_step(ol, inp.X.astype(np.float64).T, inp.labels, "softmax_ce", w.eta, store=bf16_store if bf else None)
+    tol = 5e-2 if bf else 1e-5                            # free-running bf16 step (no forced ReLU decisions)
+    for i in range(3):
+        assert rel_fro(to_np(net.get_tensor(mbd.T_DW, i)), o["dWs"][i]) < tol
+        assert rel_fro(to_np(net.get_tensor(mbd.T_DY, i)), o["dYs"][i].T) < tol
+    assert rel_fro(to_np(net.get_tensor(mbd.T_DB, 1)), o["dbs"][1]) < tol
+    net.close()

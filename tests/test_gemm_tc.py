@@ -82,3 +82,25 @@ def test_asymmetric_values_catch_transposition():
     B = np.repeat(np.arange(N, dtype=np.float32)[:, None] % 8, K, axis=1)
     D = to_np(mbd.gemm_bf16(0, to_dev(A, True), to_dev(B, True)))
     assert np.array_equal(D, K * np.outer(np.arange(M) % 16, np.arange(N) % 8))
+
+
+MODES = {
+    "tile128x128": {"MBD_TC_MH": "1", "MBD_TC_BN": "128", "MBD_TC_PAIR": "0"},
+    "tile128x256": {"MBD_TC_MH": "1", "MBD_TC_BN": "256", "MBD_TC_PAIR": "0"},
+    "tile256x256": {"MBD_TC_MH": "2", "MBD_TC_BN": "256", "MBD_TC_PAIR": "0"},
+    "cta_pair": {"MBD_TC_PAIR": "1"},
+}
+
+
+@pytest.mark.parametrize("mode", sorted(MODES))
+@pytest.mark.parametrize("variant", [0, 1, 2])
+def test_every_tile_shape_and_the_cta_pair(monkeypatch, mode, variant):
+    # the planner normally picks the tile shape; force each one (tuning knobs) on ragged sizes
+    from paper_1712_04432_b200 import mbd
+    for k, v in MODES[mode].items():
+        monkeypatch.setenv(k, v)
+    for (M, N, K, S) in [(648, 776, 328, 1), (392, 1000, 520, 3)]:
+        A, B = operands(variant, M, N, K, seed=31 * variant + S)
+        D = mbd.gemm_bf16(variant, to_dev(A, True), to_dev(B, True), k_splits=S)
+        err = rel_fro(to_np(D), reference(variant, A, B))
+        assert err < TOL, (mode, variant, M, N, K, S, err)
