@@ -124,7 +124,7 @@ def workload_config(w, grid, max_partials):
 
 
 # ------------------------------------------------------------------------------ oracle timing
-def oracle_sample(w, inp, max_seconds_hint=20.0):
+def oracle_sample(w, inp):
     """Time the fp64 oracle, as it stands, on a bounded sample of the workload: the whole
     network on the first `Bs` samples of the batch.  Returns (flops, seconds, description)."""
     from oracle import mbd_oracle as O

@@ -13,6 +13,11 @@
 //               the epilogue of one tile runs under the MMAs of the next
 // Transposed operands are not copied: an operand whose contiguous dimension is M or N is
 // loaded as 64-wide column chunks and described to the MMA as "MN-major".
+// Tile shapes: 128 x 128, 128 x 256, 256 x 256 per CTA, or 256 x 256 per CTA pair
+// (cta_group::2); tc_gemm_prepare picks one per contraction with a small cost model.  With a
+// bf16 result on 128-row tiles the epilogue moves all its global data by TMA through per-warp
+// staging boxes.  Tuning knobs (environment): MBD_TC_MH, MBD_TC_BN, MBD_TC_PAIR, MBD_TC_GROUP_M,
+// MBD_TC_NO_TE.
 // Every mbarrier wait is bounded; on time-out the kernel records a code and leaves.
 #include <stdlib.h>
 

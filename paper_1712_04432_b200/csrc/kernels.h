@@ -16,8 +16,7 @@ enum : int {
   DEV_TIMEOUT_PRODUCER = 101,   // TMA producer waited too long for a free stage
   DEV_TIMEOUT_MMA_FULL = 102,   // MMA issuer waited too long for operands
   DEV_TIMEOUT_MMA_TMEM = 103,   // MMA issuer waited too long for a drained accumulator
-  DEV_TIMEOUT_EPILOGUE = 104,   // epilogue waited too long for a finished accumulator
-  DEV_BAD_SCRATCH = 105
+  DEV_TIMEOUT_EPILOGUE = 104    // epilogue waited too long for a finished accumulator
 };
 
 // What happens to a finished fp32 accumulator element acc at (m, n).
@@ -85,7 +84,6 @@ cudaError_t simt_gemm_launch(const SimtGemm& g, cudaStream_t stream);
 // out = sum_{s<S} parts[s] (ascending s), then the epilogue op.  parts is [S][M][N] dense.
 cudaError_t reduce_partials_launch(const float* parts, int S, int64_t M, int64_t N, const Epi& epi,
                                    int num_sms, cudaStream_t stream);
-// As above with the partials addressed through a device pointer variable.
 cudaError_t softmax_xent_launch(const float* logits, int64_t B, int64_t d, const int32_t* labels,
                                 void* dY, int dy_bf16, float* per_sample, cudaStream_t stream);
 // sum of n floats in a fixed order into *out (single CTA, deterministic); scale applied.
