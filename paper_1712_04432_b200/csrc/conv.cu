@@ -43,9 +43,9 @@ constexpr int FWD_ROW_BYTES = 128 * 128;
 constexpr int FWD_W_BYTES = 3 * 192 * 128;   // stacked taps, 72 KB
 constexpr int FWD_SMEM = FWD_W_BYTES + FWD_STAGES * 3 * FWD_ROW_BYTES + 1024;
 constexpr int FWD_THREADS = 320;      // producer warp, MMA warp, 8 epilogue warps
-constexpr int WG_PIX = 64;            // pixels (reduction length) per backward-weight block
-constexpr int WG_XSTAGES = 4;         // X rows: 3 shifted copies of 8 KB each, each row used once
-constexpr int WG_YSTAGES = 6;         // dY rows: 8 KB each, plus 2 mirror slots
+constexpr int WG_PIX = 128;           // pixels (reduction length) per backward-weight block
+constexpr int WG_XSTAGES = 2;          // X rows: 3 shifted copies of 16 KB each, each row used once
+constexpr int WG_YSTAGES = 4;          // dY rows: 16 KB each, plus 2 mirror slots
 constexpr int WG_CHUNK = WG_PIX * 128;
 constexpr int WG_SMEM = WG_XSTAGES * 3 * WG_CHUNK + (WG_YSTAGES + 2) * WG_CHUNK + 1024;
 constexpr int NUM_THREADS = 192;
