@@ -53,46 +53,52 @@ constexpr int NUM_THREADS = 192;
 enum { MODE_RELU_STORE = 0, MODE_STORE_SSQ = 1, MODE_MASK = 2 };
 
 // ------------------------------------------------------------------------------ layout kernels
-// NCHW -> strips.  Block = (32-pixel segment, image row h, image b); 256 threads.  A row that
+// NCHW -> strips.  Block = (32-pixel segment, image row h, image b); 128 threads.  A row that
 // borders another strip is also written into that neighbour's halo row: this is the forward
 // halo exchange for the network input, fused into the staging pass.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 nchw_to_strips_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int H, int W, int P_r, int Hs) {
-  __shared__ bf16 tile[C][32 + 2];
+  // 32 pixels x 64 channels per block; shared memory holds channel PAIRS as 32-bit words,
+  // [pixel][pair] with an odd pitch, so both phases are free of bank conflicts.
+  __shared__ uint32_t tile[32][33];
   const int w0 = blockIdx.x * 32, h = blockIdx.y, b = blockIdx.z;
   const int t = threadIdx.x;
   {
-    const int c = t >> 2, wq = (t & 3) * 8;
-    const bf16* p = src + ((static_cast<int64_t>(b) * C + c) * H + h) * W + w0 + wq;
+    const int cp = t >> 2, wq = (t & 3) * 8;          // channels 2cp, 2cp+1; pixels wq..wq+7
+    const bf16* p0 = src + ((static_cast<int64_t>(b) * C + 2 * cp) * H + h) * W + w0 + wq;
+    const bf16* p1 = p0 + static_cast<int64_t>(H) * W;
+    uint16_t lo[8], hi[8];
     if ((W & 7) == 0 && w0 + wq + 8 <= W) {
-      const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p));
-      const uint32_t qw[4] = {q.x, q.y, q.z, q.w};
+      const uint4 a = __ldcs(reinterpret_cast<const uint4*>(p0)), c = __ldcs(reinterpret_cast<const uint4*>(p1));
+      const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        tile[c][wq + 2 * i] = __ushort_as_bfloat16(static_cast<unsigned short>(qw[i] & 0xFFFFu));
-        tile[c][wq + 2 * i + 1] = __ushort_as_bfloat16(static_cast<unsigned short>(qw[i] >> 16));
+        lo[2 * i] = aw[i] & 0xFFFFu; lo[2 * i + 1] = aw[i] >> 16;
+        hi[2 * i] = cw[i] & 0xFFFFu; hi[2 * i + 1] = cw[i] >> 16;
       }
     } else {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) tile[c][wq + i] = (w0 + wq + i < W) ? p[i] : __float2bfloat16(0.f);
+      for (int i = 0; i < 8; ++i) {
+        const bool in = w0 + wq + i < W;
+        lo[i] = in ? __bfloat16_as_ushort(p0[i]) : 0;
+        hi[i] = in ? __bfloat16_as_ushort(p1[i]) : 0;
+      }
     }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) tile[wq + i][cp] = static_cast<uint32_t>(lo[i]) | (static_cast<uint32_t>(hi[i]) << 16);
   }
   __syncthreads();
-  const int px = t >> 3, cq = (t & 7) * 8;
+  const int px = t >> 2, cq = (t & 3) * 8;            // 8 words = channels 2cq .. 2cq+15 of pixel px
   if (w0 + px >= W) return;
-  uint4 v;
-  uint32_t* vw = reinterpret_cast<uint32_t*>(&v);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const uint16_t lo = __bfloat16_as_ushort(tile[cq + 2 * i][px]);
-    const uint16_t hi = __bfloat16_as_ushort(tile[cq + 2 * i + 1][px]);
-    vw[i] = static_cast<uint32_t>(lo) | (static_cast<uint32_t>(hi) << 16);
-  }
+  uint4 v0, v1;
+  v0.x = tile[px][cq + 0]; v0.y = tile[px][cq + 1]; v0.z = tile[px][cq + 2]; v0.w = tile[px][cq + 3];
+  v1.x = tile[px][cq + 4]; v1.y = tile[px][cq + 5]; v1.z = tile[px][cq + 6]; v1.w = tile[px][cq + 7];
   const int R = Hs + 2;
   const int s = h / Hs, r = h - s * Hs + 1;
   auto put = [&](int ss, int rr) {
-    bf16* q = dst + (((static_cast<int64_t>(b) * P_r + ss) * R + rr) * W + (w0 + px)) * C + cq;
-    *reinterpret_cast<uint4*>(q) = v;
+    bf16* q = dst + (((static_cast<int64_t>(b) * P_r + ss) * R + rr) * W + (w0 + px)) * C + 2 * cq;
+    *reinterpret_cast<uint4*>(q) = v0;
+    *reinterpret_cast<uint4*>(q + 8) = v1;
   };
   put(s, r);
   if (r == 1 && s > 0) put(s - 1, Hs + 1);          // first row of a strip: lower halo of the strip above
@@ -154,13 +160,29 @@ __global__ void pack_weights_kernel(const bf16* __restrict__ K, bf16* __restrict
 
 // Sum of the per-CTA partials [G][9][c][o] in CTA order, into canonical [o][c][u][v]:
 // either stored (dK) or applied as K += scale * dK (Eq. 1).
-__global__ void wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ dK, bf16* __restrict__ K,
-                                    float scale) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= 9 * C * C) return;
+__global__ void __launch_bounds__(256)
+wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ dK, bf16* __restrict__ K, float scale) {
+  // 64 outputs per block; four thread groups each add a contiguous quarter of the CTA partials in
+  // ascending order, and the four sub-sums are added in ascending order too (a fixed order).
+  __shared__ float sub[4][64];
+  const int j = threadIdx.x & 63, q = threadIdx.x >> 6;
+  const int i = blockIdx.x * 64 + j;
+  const int g0 = (q * G) / 4, g1 = ((q + 1) * G) / 4;
+  float s = 0.f;
+  int g = g0;
+  for (; g + 8 <= g1; g += 8) {
+    float v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = __ldcs(part + static_cast<int64_t>(g + e) * 9 * C * C + i);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) s += v[e];
+  }
+  for (; g < g1; ++g) s += part[static_cast<int64_t>(g) * 9 * C * C + i];
+  sub[q][j] = s;
+  __syncthreads();
+  if (q != 0) return;
+  s = ((sub[0][j] + sub[1][j]) + sub[2][j]) + sub[3][j];
   const int t = i / (C * C), c = (i / C) % C, o = i % C;
-  float s = part[i];
-  for (int g = 1; g < G; ++g) s += part[static_cast<int64_t>(g) * 9 * C * C + i];
   const int e = (o * C + c) * 9 + t;
   if (dK) dK[e] = s;
   if (K) K[e] = __float2bfloat16_rn(fmaf(scale, s, __bfloat162float(K[e])));
@@ -646,7 +668,7 @@ void launch_halo(ConvNet* c, bf16* buf) {
 void launch_stage_in(ConvNet* c, const bf16* nchw, bf16* strips) {
   dim3 g((c->W + 31) / 32, c->H, static_cast<unsigned>(c->B));
   c->prof->begin(MBD_K_HALO, 2.0 * c->B * C * c->H * c->W * 2.0);
-  nchw_to_strips_kernel<<<g, 256, 0, c->stream>>>(nchw, strips, c->H, c->W, c->P_r, c->Hs);
+  nchw_to_strips_kernel<<<g, 128, 0, c->stream>>>(nchw, strips, c->H, c->W, c->P_r, c->Hs);
   c->prof->end();
 }
 
@@ -764,7 +786,7 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
     conv_wgrad_kernel<<<grid, NUM_THREADS, WG_SMEM, c->stream>>>(c->act_wg[i], c->dY_wg[i], p);
     c->prof->end();
     c->prof->begin(MBD_K_REDUCE, (grid + 1.0) * 9 * C * C * 4.0);
-    wgrad_finish_kernel<<<(9 * C * C + 255) / 256, 256, 0, c->stream>>>(c->wpart, grid, fused ? nullptr : c->dK[i],
+    wgrad_finish_kernel<<<9 * C * C / 64, 256, 0, c->stream>>>(c->wpart, grid, fused ? nullptr : c->dK[i],
                                                                       fused ? c->K[i] : nullptr, scale);
     c->prof->end();
   }
@@ -808,7 +830,7 @@ mbd_status conv_set_tensor(ConvNet* c, int which, int layer, const void* src, si
   bf16* dst = which == MBD_T_ACT ? c->act[layer + 1] : which == MBD_T_DY ? c->dY[layer] : nullptr;
   if (!dst) return MBD_E_INVALID;
   dim3 g((c->W + 31) / 32, c->H, static_cast<unsigned>(c->B));
-  nchw_to_strips_kernel<<<g, 256, 0, c->stream>>>(static_cast<const bf16*>(src), dst, c->H, c->W, c->P_r, c->Hs);
+  nchw_to_strips_kernel<<<g, 128, 0, c->stream>>>(static_cast<const bf16*>(src), dst, c->H, c->W, c->P_r, c->Hs);
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
