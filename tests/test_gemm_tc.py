@@ -104,3 +104,18 @@ def test_every_tile_shape_and_the_cta_pair(monkeypatch, mode, variant):
         D = mbd.gemm_bf16(variant, to_dev(A, True), to_dev(B, True), k_splits=S)
         err = rel_fro(to_np(D), reference(variant, A, B))
         assert err < TOL, (mode, variant, M, N, K, S, err)
+
+
+def test_random_shapes_sweep():
+    # 24 seeded random problems: sizes are multiples of 8 (the 16-byte rule of TMA), any layout,
+    # K cut into 1..5 pieces; whatever tile shape the planner picks must agree with fp64
+    from paper_1712_04432_b200 import mbd
+    r = np.random.default_rng(2024)
+    for case in range(24):
+        variant = int(r.integers(0, 3))
+        M, N, K = (8 * int(r.integers(1, 150)) for _ in range(3))
+        S = int(r.integers(1, 6))
+        A, B = operands(variant, M, N, K, seed=1000 + case)
+        D = mbd.gemm_bf16(variant, to_dev(A, True), to_dev(B, True), k_splits=S)
+        err = rel_fro(to_np(D), reference(variant, A, B))
+        assert err < TOL, (case, variant, M, N, K, S, err)
