@@ -354,11 +354,20 @@ def run_ours(args):
         g_fl = sum(v["work"] for v in gemm.values())
         g_n = sum(v["launches"] for v in gemm.values())
         ach = g_fl / (g_ms * 1e-3) / 1e12
-        peak = peaks["bf16_tflops_sustained"] if bf else None
-        roofline = dict(bound="tensor" if bf else "alu", kernel="gemm_tc_kernel (all three operand layouts)",
+        # fp32 check mode runs on the FMA pipes: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
+        peak = peaks["bf16_tflops_sustained"] if bf else 148 * 128 * 2 * 1.965e9 / 1e12
+        if w.kind == "conv":
+            kname = "conv_fwd_kernel (forward, backward-data) + conv_wgrad_kernel"
+        elif bf:
+            kname = "gemm_tc_kernel (all three operand layouts)"
+        else:
+            kname = "simt_gemm_kernel (fp32 check mode)"
+        roofline = dict(bound="tensor" if bf else "alu", kernel=kname,
                         achieved=ach, peak=peak, unit="TFLOP/s", frac=(ach / peak) if peak else None,
-                        peak_kind=f"{peaks['source']} sustained bf16 (kernel timed inside a long step); "
-                                  f"burst {peaks['bf16_tflops']}", frac_of_burst=ach / peaks["bf16_tflops"] if bf else None,
+                        peak_kind=(f"{peaks['source']} sustained bf16 (kernel timed inside a long step); "
+                                   f"burst {peaks['bf16_tflops']}") if bf else
+                                  "derived fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x 1965 MHz",
+                        frac_of_burst=ach / peaks["bf16_tflops"] if bf else None,
                         launches=g_n, avg_launch_ms=g_ms / g_n, flops_per_launch=g_fl / g_n,
                         share_of_step=g_ms / (prof_ms * args.steps), traffic=TRAFFIC.get(w.name),
                         timed_in="second pass, direct launches" if use_graph else "the timed region")
