@@ -16,9 +16,10 @@
 // Tile shapes: 128 x 128, 128 x 256, 256 x 256 per CTA, or 256 x 256 per CTA pair
 // (cta_group::2); tc_gemm_prepare picks one per contraction with a small cost model.  With a
 // bf16 result on 128-row tiles the epilogue moves all its global data by TMA through per-warp
-// staging boxes.  Tuning knobs (environment): MBD_TC_MH, MBD_TC_BN, MBD_TC_PAIR, MBD_TC_GROUP_M,
+// staging boxes.  Tuning knobs (environment): MBD_TC_MH, MBD_TC_BN, MBD_TC_PAIR, MBD_TC_GROUP_M, MBD_TC_DEBUG,
 // MBD_TC_NO_TE.
 // Every mbarrier wait is bounded; on time-out the kernel records a code and leaves.
+#include <stdio.h>
 #include <stdlib.h>
 
 #include "epi.cuh"
@@ -121,7 +122,6 @@ template <int A_MN, int B_MN, int BN, int MH, int PAIR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmAux, const Params p) {
-  static_assert(!PAIR || MH == 1, "a CTA of a pair owns 128 rows");
   constexpr int BMT = BM * MH;                                // rows owned by this CTA
   constexpr int TILE_M = BMT * (PAIR ? 2 : 1);                // rows of the (pair's) tile
   constexpr int BNL = PAIR ? BN / 2 : BN;                     // B rows (tile columns) loaded by this CTA
@@ -261,7 +261,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int k = 0; k < BK / UMMA_K; ++k) {
 #pragma unroll
             for (int h = 0; h < MH; ++h) {
-              if (PAIR) tc_mma_bf16_pair(d_tmem, adesc + k * A_STEP, bdesc + k * B_STEP, IDESC, (kb > wk.kb0 || k > 0) ? 1u : 0u);
+              if (PAIR) tc_mma_bf16_pair(d_tmem + h * BN, adesc + h * A_HALF + k * A_STEP, bdesc + k * B_STEP, IDESC,
+                                         (kb > wk.kb0 || k > 0) ? 1u : 0u);
               else tc_mma_bf16(d_tmem + h * BN, adesc + h * A_HALF + k * A_STEP, bdesc + k * B_STEP, IDESC,
                                (kb > wk.kb0 || k > 0) ? 1u : 0u);
             }
@@ -534,6 +535,7 @@ cudaError_t set_attr() {
   if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
   return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES);
 }
 
@@ -551,6 +553,7 @@ cudaError_t launch_t(const TcGemm& g, const Params& p, cudaStream_t stream) {
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (g.MH == 2) return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<A_MN, B_MN, 256, 2, 1>, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
     return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<A_MN, B_MN, 256, 1, 1>, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
   }
   if (g.BN == 256 && g.MH == 1) gemm_tc_kernel<A_MN, B_MN, 256, 1, 0><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
@@ -599,24 +602,26 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
     double best = 1e30;
     int best_bn = 128, best_mh = 1, best_x = 1, best_pair = 0;
     const int x_max = g.allow_extra_split ? 8 : 1;
-    for (int cand = 0; cand < 3; ++cand) {           // 0: 128-row tiles, 1: 256-row tiles, 2: CTA pairs
-      const int mh = cand == 1 ? 2 : 1;
-      const bool pair = cand == 2;
+    for (int cand = 0; cand < 4; ++cand) {           // 0: 128-row tiles, 1: 256-row tiles, 2: CTA pairs, 3: pairs of 256-row CTAs
+      const int mh = (cand == 1 || cand == 3) ? 2 : 1;
+      const bool pair = cand >= 2;
       for (int bn = pair ? 256 : 128; bn <= 256; bn += 128) {
         for (int x = 1; x <= x_max; x *= 2) {
           const long long S = 1ll * g.k_splits * x;
           if (S > kb_total || (x > 1 && kb_total / S < 8)) continue;
           const double kb = static_cast<double>(kb_total) / S;
-          const int tile_m = pair ? 256 : 128 * mh;
+          const int tile_m = 128 * mh * (pair ? 2 : 1);
           const long long units = 1ll * ((g.M + tile_m - 1) / tile_m) * ((g.N + bn - 1) / bn) * S;
           const int slots = pair ? num_sms / 2 : num_sms;
           const double waves = static_cast<double>((units + slots - 1) / slots);
-          // per SM and k-block: tensor-pipe clocks and operand-fill clocks
-          const double mma = pair ? 4.0 * 128.0 / 0.80 : 4.0 * mh * (bn / 2) / (bn == 256 ? 0.85 : 0.75);
-          const double fill = (pair ? 256.0 : 128.0 * mh + bn) * 128.0 / 70.0;
+          // per SM and k-block: tensor-pipe clocks and operand-fill clocks; the efficiencies follow
+          // the measured order 256 x 256 single < 256 x 256 pair < 512 x 256 pair on 8192^3
+          const double eff = pair ? (mh == 2 ? 0.87 : 0.84) : (mh == 2 ? 0.80 : (bn == 256 ? 0.85 : 0.75));
+          const double mma = 4.0 * mh * ((pair ? 256 : bn) / 2) / eff;
+          const double fill = (pair ? 128.0 * mh + 128.0 : 128.0 * mh + bn) * 128.0 / 70.0;
           const double mainloop = kb * (mma > fill ? mma : fill);
           const double epi = 2500.0 * mh * bn / 256.0 * (S > 1 ? 2.0 : 1.0);
-          const bool overlapped = pair || mh * bn <= 256;
+          const bool overlapped = mh * bn <= 256;        // two accumulators fit in TMEM
           double unit = overlapped ? (mainloop > epi ? mainloop : epi) : mainloop + epi;
           double t = waves * unit + 4000.0;
           if (S > 1 && x > 1) {          // the reduction exists anyway when the grid itself splits K
@@ -640,9 +645,13 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
   }
   if (const char* ev = getenv("MBD_TC_PAIR")) {        // tuning knob: CTA pairs (256 x 256 per pair)
     if (atoi(ev) == 1) { g.pair = 1; g.MH = 1; g.BN = 256; }
+    else if (atoi(ev) == 2) { g.pair = 1; g.MH = 2; g.BN = 256; }      // 512 x 256 per pair
     else if (atoi(ev) == 0) g.pair = 0;
   }
-  if (g.pair) { g.MH = 1; g.BN = 256; }
+  if (g.pair) g.BN = 256;
+  if (getenv("MBD_TC_DEBUG"))
+    fprintf(stderr, "tc_gemm_prepare: variant %d  M %d N %d K %d  pieces of K %d  ->  %d x %d tile%s\n", g.variant, g.M, g.N,
+            g.K, g.k_splits, 128 * g.MH * (g.pair ? 2 : 1), g.BN, g.pair ? " (CTA pair)" : "");
   const int bmt = BM * g.MH * (g.pair ? 2 : 1);        // rows of one work unit's tile
   const int tiles_m = (g.M + bmt - 1) / bmt;
   const int tiles_n = (g.N + g.BN - 1) / g.BN;

@@ -48,6 +48,12 @@ struct mbd_net {
   float* partials = nullptr;
   size_t partial_elems = 0;
   float* colsum_scratch = nullptr;
+  // The bias gradients (column sums of dY_i) are small and independent of the contractions of
+  // their layer: they run on a side stream, forked after dY_i exists and joined at the end of
+  // the backward pass, next to the persistent GEMM CTAs.
+  cudaStream_t aux = nullptr;
+  std::vector<cudaEvent_t> ev_fork;
+  cudaEvent_t ev_join = nullptr;
   float* per_sample = nullptr;
   float* loss_dev = nullptr;
   int* status = nullptr;
@@ -198,6 +204,9 @@ void free_net(mbd_net* n) {
   cudaFree(n->status); cudaFree(n->X_stage); cudaFree(n->labels_stage);
   if (n->conv) conv_destroy(n->conv);
   if (n->graph_exec) cudaGraphExecDestroy(n->graph_exec);
+  for (cudaEvent_t e : n->ev_fork) if (e) cudaEventDestroy(e);
+  if (n->ev_join) cudaEventDestroy(n->ev_join);
+  if (n->aux) cudaStreamDestroy(n->aux);
   n->prof.destroy();
   (void)cudaGetLastError();
   delete n;
@@ -323,6 +332,13 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   ALLOC(n->colsum_scratch, static_cast<size_t>(32) * max_d * sizeof(float));
   ALLOC(n->per_sample, B * sizeof(float));
 #undef ALLOC
+  {
+    bool ok = cudaStreamCreateWithFlags(&n->aux, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&n->ev_join, cudaEventDisableTiming) == cudaSuccess;
+    n->ev_fork.assign(L, nullptr);
+    for (int i = 0; i < L && ok; ++i) ok = cudaEventCreateWithFlags(&n->ev_fork[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { free_net(n); return MBD_E_CUDA; }
+  }
   if (cudaStreamSynchronize(n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
   *out = n;
   return MBD_OK;
@@ -404,12 +420,22 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
   const bool fused = fused_eta > 0.f;
   const float scale = -fused_eta / static_cast<float>(n->B);
   const int S_r = splits_for(n->P_r, n->max_partials), S_c = splits_for(n->P_c, n->max_partials);
+  // per-kernel events bracket launches on the main stream only, so a profiled pass stays on it
+  const bool side = n->aux != nullptr && !n->prof.on;
+  bool forked = false;
   for (int i = n->L - 1; i >= 0; --i) {
     Layer& l = n->layers[i];
     if (l.bias) {
+      cudaStream_t cs = n->stream;
+      if (side) {
+        CK(cudaEventRecord(n->ev_fork[i], n->stream));
+        CK(cudaStreamWaitEvent(n->aux, n->ev_fork[i], 0));
+        cs = n->aux;
+        forked = true;
+      }
       n->prof.begin(MBD_K_COLSUM, static_cast<double>(n->B) * l.d_out * (bf ? 2.0 : 4.0));
       CK(colsum_launch(l.dY, bf, n->B, l.d_out, n->colsum_scratch, colsum_row_splits(n->B, l.d_out, n->num_sms), fused ? nullptr : l.db,
-                       fused ? l.bias : nullptr, scale, n->stream));
+                       fused ? l.bias : nullptr, scale, cs));
       n->prof.end();
       n->prof.total_launches += colsum_launches(n->B, l.d_out, n->num_sms) - 1;
     }
@@ -421,6 +447,10 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
     const Epi e = fused ? epi_sgd(l.W, l.d_in, bf, scale) : epi_act(l.dW, l.d_in, 0, nullptr, 0);
     mbd_status s = run_gemm(n, l.bwd_weight, 2, l.d_out, l.d_in, n->B, l.dY, l.d_out, layer_input(n, i), l.d_in, S_c, e);
     if (s != MBD_OK) return s;
+  }
+  if (forked) {
+    CK(cudaEventRecord(n->ev_join, n->aux));
+    CK(cudaStreamWaitEvent(n->stream, n->ev_join, 0));
   }
   n->state = fused ? ST_BWD_FUSED : ST_BWD_UNFUSED;
   return MBD_OK;

@@ -89,6 +89,7 @@ MODES = {
     "tile128x256": {"MBD_TC_MH": "1", "MBD_TC_BN": "256", "MBD_TC_PAIR": "0"},
     "tile256x256": {"MBD_TC_MH": "2", "MBD_TC_BN": "256", "MBD_TC_PAIR": "0"},
     "cta_pair": {"MBD_TC_PAIR": "1"},
+    "cta_pair512x256": {"MBD_TC_PAIR": "2"},
 }
 
 
