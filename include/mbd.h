@@ -152,6 +152,64 @@ MBD_API mbd_status mbd_train_step_host(mbd_net* net, const void* X_host, const i
 MBD_API mbd_status mbd_comm_words(const mbd_layer* layers_host, int L, int64_t B, int P_r, int P_c,
                           mbd_words* out_host);
 
+/* ---- Communication time model and choice of the grid (Eq. 3-9 with their latency terms;
+ * Section 3).  Host only, no GPU.  A collective costs alpha * messages + beta * words:
+ * all-gather of Y_i over P_r: ceil(log2 P_r) messages; all-reduce of dX_i (layers >= 2) over
+ * P_r: 2 ceil(log2 P_r); all-reduce of dW_i over P_c: 2 ceil(log2 P_c); a domain-split layer:
+ * one message per halo exchange (none for a single strip) and 2 ceil(log2 P) for its
+ * all-reduce over all P processes.  The words are those of mbd_comm_words before rounding. */
+typedef struct {
+  double alpha;   /* latency per message, seconds                           */
+  double beta;    /* inverse bandwidth, seconds per word (one matrix element) */
+} mbd_machine;
+
+typedef struct { double allgather_y, allreduce_dx, allreduce_dw, halo_fwd, halo_bwd; } mbd_times;  /* seconds */
+
+typedef enum {
+  MBD_GRID_UNIFORM = 0,     /* every layer on the same P_r x P_c grid, split as its `split` field says     */
+  MBD_GRID_CONV_BATCH = 1   /* convolutions batch-parallel on 1 x P, fully connected layers on P_r x P_c   */
+} mbd_grid_policy;
+
+typedef struct {
+  int P_r, P_c;
+  double comm_fwd;   /* all-gathers, forward halos, redistribution (Eq. 6) */
+  double comm_bwd;   /* all-reduces, backward halos                        */
+  double comm;       /* comm_fwd + comm_bwd                                */
+  double total;      /* with the compute time, see mbd_total_time          */
+} mbd_grid_row;
+
+/* Per-layer terms of Eq. 9 (Eq. 8 if no layer is domain-split) in seconds; out_host has L rows.
+ * MBD_E_GRID as for mbd_comm_words. */
+MBD_API mbd_status mbd_comm_time(const mbd_layer* layers_host, int L, int64_t B, int P_r, int P_c,
+                                 const mbd_machine* machine, mbd_times* out_host);
+
+/* Eq. 6 for a grid: all-gather of a (B / P_c) x d block over the P_r processes of a group,
+ * paid when a batch-parallel layer feeds a layer on a P_r x P_c grid (P_c = 1: Eq. 6 itself). */
+MBD_API mbd_status mbd_redistribute_time(int64_t B, int P_r, int P_c, int64_t d, const mbd_machine* machine,
+                                         double* out_host);
+
+/* compute + comm_fwd + comm_bwd; with overlap != 0 the backward communication hides behind
+ * the backward compute, taken as two thirds of `compute` (two of the three products per
+ * layer): compute + comm_fwd + max(0, comm_bwd - 2/3 compute).  The paper shows this variant
+ * only as a figure; the formula is this library's reading of it. */
+MBD_API mbd_status mbd_total_time(double compute, double comm_fwd, double comm_bwd, int overlap, double* out_host);
+
+/* One row per feasible factorisation P = P_r * P_c, ascending P_r.  Feasible: P_c <= B; P_r
+ * at most the outputs of every model-split layer and at most the rows H of every domain-split
+ * layer; MBD_GRID_CONV_BATCH also needs P <= B and charges Eq. 6 at the first fully connected
+ * layer that follows a convolution when P_r > 1 and charge_redistribution != 0.
+ * rows_host may be NULL (cap 0) to ask for the count; *n_rows is always the full count;
+ * MBD_E_INVALID if cap is smaller than that and rows_host is not NULL. */
+MBD_API mbd_status mbd_grid_table(const mbd_layer* layers_host, int L, int64_t B, int P, const mbd_machine* machine,
+                                  int policy, double compute, int overlap, int charge_redistribution,
+                                  mbd_grid_row* rows_host, int cap, int* n_rows);
+
+/* The row of mbd_grid_table with the least `total`; ties go to the smaller P_r.  MBD_E_GRID if
+ * no factorisation is feasible. */
+MBD_API mbd_status mbd_choose_grid(const mbd_layer* layers_host, int L, int64_t B, int P, const mbd_machine* machine,
+                                   int policy, double compute, int overlap, int charge_redistribution,
+                                   mbd_grid_row* best_host);
+
 /* Copy an internal tensor to dst_dev; `bytes` must equal the tensor's size. */
 MBD_API mbd_status mbd_get_tensor(mbd_net* net, int which, int layer, void* dst_dev, size_t bytes);
 

@@ -25,7 +25,8 @@ KERNEL_CLASSES = ["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce_partia
 
 EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weights", "mbd_forward",
            "mbd_backward", "mbd_sgd_step", "mbd_train_step", "mbd_train_step_host", "mbd_comm_words", "mbd_get_tensor",
-           "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_gemm_bf16_noalloc", "mbd_selftest_timeout", "mbd_strerror"]
+           "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_gemm_bf16_noalloc", "mbd_selftest_timeout", "mbd_strerror",
+           "mbd_comm_time", "mbd_redistribute_time", "mbd_total_time", "mbd_grid_table", "mbd_choose_grid"]
 
 
 class MbdError(RuntimeError):
@@ -45,6 +46,28 @@ class Words(C.Structure):
     _fields_ = [("allgather_y", C.c_int64), ("allreduce_dx", C.c_int64), ("allreduce_dw", C.c_int64),
                 ("halo_fwd", C.c_int64), ("halo_bwd", C.c_int64)]
 
+
+class Machine(C.Structure):
+    """alpha: seconds per message; beta: seconds per word (one matrix element)."""
+    _fields_ = [("alpha", C.c_double), ("beta", C.c_double)]
+
+
+class Times(C.Structure):
+    _fields_ = [("allgather_y", C.c_double), ("allreduce_dx", C.c_double), ("allreduce_dw", C.c_double),
+                ("halo_fwd", C.c_double), ("halo_bwd", C.c_double)]
+
+
+class GridRow(C.Structure):
+    _fields_ = [("P_r", C.c_int32), ("P_c", C.c_int32), ("comm_fwd", C.c_double), ("comm_bwd", C.c_double),
+                ("comm", C.c_double), ("total", C.c_double)]
+
+
+GRID_UNIFORM, GRID_CONV_BATCH = 0, 1
+# Table 1 of the paper: 2 microseconds, 6 GB/s, 4-byte words
+MACHINE_CORI_KNL = (2e-6, 4.0 / 6e9)
+# One B200 on NVLink 5: measured peer copy 770 GB/s per direction, 2-byte words; the latency is a
+# nominal few microseconds per collective step, not a measurement
+MACHINE_B200_NVLINK5 = (5e-6, 2.0 / 770e9)
 
 _lib = None
 
@@ -68,6 +91,14 @@ def lib():
         L.mbd_train_step.argtypes = [vp, vp, vp, f32, vp]
         L.mbd_train_step_host.argtypes = [vp, vp, vp, f32, C.POINTER(f32)]
         L.mbd_comm_words.argtypes = [C.POINTER(Layer), i32, i64, i32, i32, C.POINTER(Words)]
+        f64 = C.c_double
+        L.mbd_comm_time.argtypes = [C.POINTER(Layer), i32, i64, i32, i32, C.POINTER(Machine), C.POINTER(Times)]
+        L.mbd_redistribute_time.argtypes = [i64, i32, i32, i64, C.POINTER(Machine), C.POINTER(f64)]
+        L.mbd_total_time.argtypes = [f64, f64, f64, i32, C.POINTER(f64)]
+        L.mbd_grid_table.argtypes = [C.POINTER(Layer), i32, i64, i32, C.POINTER(Machine), i32, f64, i32, i32,
+                                     C.POINTER(GridRow), i32, C.POINTER(i32)]
+        L.mbd_choose_grid.argtypes = [C.POINTER(Layer), i32, i64, i32, C.POINTER(Machine), i32, f64, i32, i32,
+                                      C.POINTER(GridRow)]
         L.mbd_get_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
         L.mbd_set_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
         L.mbd_poll_status.argtypes = [vp]
@@ -117,6 +148,59 @@ def comm_words(layers: Sequence[Layer], B: int, P_r: int, P_c: int) -> List[Dict
     out = (Words * len(layers))()
     _check(lib().mbd_comm_words(_layer_array(layers), len(layers), int(B), int(P_r), int(P_c), out), "mbd_comm_words")
     return [{k: int(getattr(w, k)) for k, _ in Words._fields_} for w in out]
+
+
+def _machine(machine) -> Machine:
+    return machine if isinstance(machine, Machine) else Machine(float(machine[0]), float(machine[1]))
+
+
+def _row(r: GridRow) -> Dict[str, float]:
+    return {k: (int(getattr(r, k)) if k in ("P_r", "P_c") else float(getattr(r, k))) for k, _ in GridRow._fields_}
+
+
+def comm_time(layers: Sequence[Layer], B: int, P_r: int, P_c: int, machine) -> List[Dict[str, float]]:
+    """mbd_comm_time: per-layer terms of Eq. 8 / Eq. 9 in seconds, latency terms included (host only)."""
+    out = (Times * len(layers))()
+    m = _machine(machine)
+    _check(lib().mbd_comm_time(_layer_array(layers), len(layers), int(B), int(P_r), int(P_c), C.byref(m), out), "mbd_comm_time")
+    return [{k: float(getattr(t, k)) for k, _ in Times._fields_} for t in out]
+
+
+def redistribute_time(B: int, P_r: int, P_c: int, d: int, machine) -> float:
+    """mbd_redistribute_time: Eq. 6 for a grid."""
+    out = C.c_double()
+    m = _machine(machine)
+    _check(lib().mbd_redistribute_time(int(B), int(P_r), int(P_c), int(d), C.byref(m), C.byref(out)), "mbd_redistribute_time")
+    return out.value
+
+
+def total_time(compute: float, comm_fwd: float, comm_bwd: float, overlap: bool = False) -> float:
+    out = C.c_double()
+    _check(lib().mbd_total_time(float(compute), float(comm_fwd), float(comm_bwd), int(overlap), C.byref(out)), "mbd_total_time")
+    return out.value
+
+
+def grid_table(layers: Sequence[Layer], B: int, P: int, machine, policy: int = GRID_UNIFORM, compute: float = 0.0,
+               overlap: bool = False, charge_redistribution: bool = True) -> List[Dict[str, float]]:
+    """mbd_grid_table: one row per feasible factorisation P = P_r * P_c (Section 3)."""
+    m = _machine(machine)
+    arr = _layer_array(layers)
+    n = C.c_int()
+    args = (arr, len(layers), int(B), int(P), C.byref(m), int(policy), float(compute), int(overlap), int(charge_redistribution))
+    _check(lib().mbd_grid_table(*args, None, 0, C.byref(n)), "mbd_grid_table")
+    rows = (GridRow * max(n.value, 1))()
+    _check(lib().mbd_grid_table(*args, rows, n.value, C.byref(n)), "mbd_grid_table")
+    return [_row(rows[i]) for i in range(n.value)]
+
+
+def choose_grid(layers: Sequence[Layer], B: int, P: int, machine, policy: int = GRID_UNIFORM, compute: float = 0.0,
+                overlap: bool = False, charge_redistribution: bool = True) -> Dict[str, float]:
+    """mbd_choose_grid: the factorisation with the least total time."""
+    m = _machine(machine)
+    best = GridRow()
+    _check(lib().mbd_choose_grid(_layer_array(layers), len(layers), int(B), int(P), C.byref(m), int(policy), float(compute),
+                                 int(overlap), int(charge_redistribution), C.byref(best)), "mbd_choose_grid")
+    return _row(best)
 
 
 def _ptr(t) -> Optional[int]:
