@@ -208,13 +208,12 @@ sum_f32_kernel(const float* __restrict__ x, int64_t n, float scale, float* __res
 // ------------------------------------------------------------------ column sums (bias gradient)
 // Stage 1: grid (ceil(N/256), row_splits); 256 threads = 8 warps; a lane owns 8 consecutive
 // columns (one 16-byte load per row for bf16), a warp 256 columns, the 8 warps stride over the
-// rows of this split and are added in warp order.  With a single split the result is final and
-// the bias update is applied here; otherwise stage 2 adds the splits in order.
+// rows of this split.  Every warp stores its own partial row, scratch[(split * 8 + warp)][N];
+// stage 2 adds the 8 * row_splits rows in order.  No shared memory: the CTAs fit on an SM next
+// to a resident tensor-core GEMM CTA, so the kernel can run on the side stream under a product.
 template <bool BF16>
 __global__ void __launch_bounds__(256)
-colsum_stage1(const void* __restrict__ dY, int64_t M, int64_t N, int row_splits, float* __restrict__ scratch,
-              float* __restrict__ db, float* __restrict__ bias, float scale) {
-  __shared__ float red[8][256 + 8];
+colsum_stage1(const void* __restrict__ dY, int64_t M, int64_t N, int row_splits, float* __restrict__ scratch) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t n0 = static_cast<int64_t>(blockIdx.x) * 256 + lane * 8;
   const int64_t r0 = (static_cast<int64_t>(blockIdx.y) * M) / row_splits;
@@ -245,21 +244,10 @@ colsum_stage1(const void* __restrict__ dY, int64_t M, int64_t N, int row_splits,
       }
     }
   }
+  float* dst = scratch + (static_cast<int64_t>(blockIdx.y) * 8 + warp) * N + n0;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) red[warp][lane * 8 + i] = a[i];
-  __syncthreads();
-  const int64_t n = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
-  if (n < N) {
-    float s = red[0][threadIdx.x];
-#pragma unroll
-    for (int w = 1; w < 8; ++w) s += red[w][threadIdx.x];
-    if (row_splits == 1) {
-      if (db) db[n] = s;
-      if (bias) bias[n] = fmaf(scale, s, bias[n]);
-    } else {
-      scratch[static_cast<int64_t>(blockIdx.y) * N + n] = s;
-    }
-  }
+  for (int i = 0; i < 8; ++i)
+    if (n0 + i < N) dst[i] = a[i];
 }
 
 __global__ void __launch_bounds__(256)
@@ -267,8 +255,16 @@ colsum_stage2(const float* __restrict__ scratch, int row_splits, int64_t N, floa
               float* __restrict__ bias, float scale) {
   const int64_t n = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
   if (n >= N) return;
-  float s = scratch[n];
-  for (int r = 1; r < row_splits; ++r) s += scratch[static_cast<int64_t>(r) * N + n];
+  float s = 0.f;
+  int r = 0;
+  for (; r + 8 <= row_splits; r += 8) {        // eight loads in flight, added in row order
+    float v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = scratch[static_cast<int64_t>(r + j) * N + n];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s += v[j];
+  }
+  for (; r < row_splits; ++r) s += scratch[static_cast<int64_t>(r) * N + n];
   if (db) db[n] = s;
   if (bias) bias[n] = fmaf(scale, s, bias[n]);
 }
@@ -354,16 +350,16 @@ int colsum_row_splits(int64_t M, int64_t N, int num_sms) {
   return static_cast<int>(r);
 }
 
-int colsum_launches(int64_t M, int64_t N, int num_sms) { return colsum_row_splits(M, N, num_sms) == 1 ? 1 : 2; }
+int colsum_launches(int64_t, int64_t, int) { return 2; }
 
 cudaError_t colsum_launch(const void* dY, int dy_bf16, int64_t M, int64_t N, float* scratch, int row_splits,
                           float* db, float* bias, float scale, cudaStream_t stream) {
   dim3 g1(static_cast<unsigned>((N + 255) / 256), row_splits);
-  if (dy_bf16) colsum_stage1<true><<<g1, 256, 0, stream>>>(dY, M, N, row_splits, scratch, db, bias, scale);
-  else colsum_stage1<false><<<g1, 256, 0, stream>>>(dY, M, N, row_splits, scratch, db, bias, scale);
+  if (dy_bf16) colsum_stage1<true><<<g1, 256, 0, stream>>>(dY, M, N, row_splits, scratch);
+  else colsum_stage1<false><<<g1, 256, 0, stream>>>(dY, M, N, row_splits, scratch);
   cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess || row_splits == 1) return e;
-  colsum_stage2<<<static_cast<unsigned>((N + 255) / 256), 256, 0, stream>>>(scratch, row_splits, N, db, bias, scale);
+  if (e != cudaSuccess) return e;
+  colsum_stage2<<<static_cast<unsigned>((N + 255) / 256), 256, 0, stream>>>(scratch, row_splits * 8, N, db, bias, scale);
   return cudaGetLastError();
 }
 

@@ -34,8 +34,14 @@ using namespace tc;
 constexpr int BM = 128;
 constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
 constexpr int NUM_THREADS = 320;      // TMA warp, MMA warp, 8 epilogue warps
-constexpr int SMEM_DYN_BYTES = 226 * 1024;       // dynamic shared memory of every instantiation
-constexpr int RING_MAX_BYTES = SMEM_DYN_BYTES - 1024;   // after 1024-byte alignment
+// Dynamic shared memory of every instantiation: seven 32 KB stages (or any of the other rings),
+// nothing more.  With the kernel's static variables (padded to 1 KB by the alignment of the ring)
+// and the 1 KB the system keeps per CTA, that leaves 2 KB of an SM's 228 KB: CTAs of kernels that
+// use no shared memory (a reduction, a column sum on the side stream) can be resident next to a
+// GEMM CTA.  The ring must start on a 1024-byte boundary (128B swizzle); the declaration asks for
+// that, and the kernel checks it and gives up cleanly otherwise.
+constexpr int SMEM_DYN_BYTES = 224 * 1024;
+constexpr int RING_MAX_BYTES = SMEM_DYN_BYTES;
 
 // ---- CTA-pair (cta_group::2) helpers
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -119,7 +125,11 @@ __device__ __forceinline__ Work decode_work(const Params& p, int w) {
 // epilogue: 64 B/clk of operand fill like the 256 x 256 tile, but with two accumulators (the
 // epilogue overlaps the next tile), 32 KB stages and the TMA epilogue.
 template <int A_MN, int B_MN, int BN, int MH, int PAIR>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+// 136 registers per thread at most (a few bytes of spill in three instantiations): the register file
+// is split over the SM's four sub-partitions, the busiest of which holds three of this CTA's ten
+// warps; at 136 registers it keeps room for two warps of a side-stream kernel (a reduction, a
+// column sum), whose CTAs could not be placed on the SM otherwise.
+__global__ void __maxnreg__(136)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmAux, const Params p) {
   constexpr int BMT = BM * MH;                                // rows owned by this CTA
@@ -150,7 +160,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __shared__ int abort_flag;
 
   // 1024-byte alignment of the ring (needed by the 128B swizzle pattern)
-  const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t ring = smem_u32(smem_raw);
+  if (ring & 1023u) {                      // same answer in every CTA: all of them leave before any barrier exists
+    if (threadIdx.x == 0) atomicCAS(p.status, 0, DEV_SMEM_MISALIGNED);
+    return;
+  }
   const bool te = MH == 1 && p.te != 0;
   const int stages = te ? STAGES_TE : STAGES;
   const int warp = threadIdx.x >> 5;

@@ -16,7 +16,8 @@ enum : int {
   DEV_TIMEOUT_PRODUCER = 101,   // TMA producer waited too long for a free stage
   DEV_TIMEOUT_MMA_FULL = 102,   // MMA issuer waited too long for operands
   DEV_TIMEOUT_MMA_TMEM = 103,   // MMA issuer waited too long for a drained accumulator
-  DEV_TIMEOUT_EPILOGUE = 104    // epilogue waited too long for a finished accumulator
+  DEV_TIMEOUT_EPILOGUE = 104,   // epilogue waited too long for a finished accumulator
+  DEV_SMEM_MISALIGNED = 105     // dynamic shared memory did not start on a 1024-byte boundary; nothing ran
 };
 
 // What happens to a finished fp32 accumulator element acc at (m, n).
@@ -88,12 +89,13 @@ cudaError_t softmax_xent_launch(const float* logits, int64_t B, int64_t d, const
                                 void* dY, int dy_bf16, float* per_sample, cudaStream_t stream);
 // sum of n floats in a fixed order into *out (single CTA, deterministic); scale applied.
 cudaError_t sum_f32_launch(const float* x, int64_t n, float scale, float* out, cudaStream_t stream);
-// db[n] = sum_m dY[m,n]; two deterministic stages through `scratch` [rows_split][N].
+// db[n] = sum_m dY[m,n]; two deterministic stages through `scratch` [8 * row_splits][N]; the kernels
+// use no shared memory, so their CTAs fit on an SM next to a resident tensor-core GEMM CTA.
 // If bias != null: bias[n] += scale * db[n].  If db != null: db[n] stored.
 cudaError_t colsum_launch(const void* dY, int dy_bf16, int64_t M, int64_t N, float* scratch,
                           int row_splits, float* db, float* bias, float scale, cudaStream_t stream);
 int colsum_row_splits(int64_t M, int64_t N, int num_sms);   // at most 32
-int colsum_launches(int64_t M, int64_t N, int num_sms);    // kernels one colsum_launch issues (1 or 2)
+int colsum_launches(int64_t M, int64_t N, int num_sms);    // kernels one colsum_launch issues
 // w[i] += scale * g[i]   (w bf16 or f32, g f32)
 cudaError_t sgd_update_launch(void* w, int w_bf16, const float* g, int64_t n, float scale,
                               int num_sms, cudaStream_t stream);
@@ -113,7 +115,8 @@ struct Profiler {
   int64_t total_launches = 0;
 
   cudaEvent_t get_event();
-  void begin(int cls, double w);
+  cudaStream_t cur = nullptr;             // stream of the launch being bracketed
+  void begin(int cls, double w, cudaStream_t launch_stream = nullptr);   // null: the main stream
   void end();
   void collect();          // synchronises the stream
   void reset();

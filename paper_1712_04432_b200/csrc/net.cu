@@ -50,7 +50,10 @@ struct mbd_net {
   float* colsum_scratch = nullptr;
   // The bias gradients (column sums of dY_i) are small and independent of the contractions of
   // their layer: they run on a side stream, forked after dY_i exists and joined at the end of
-  // the backward pass, next to the persistent GEMM CTAs.
+  // the backward pass, next to the persistent GEMM CTAs (the column-sum kernels use no shared
+  // memory and few registers, and the GEMM leaves room for them in every SM sub-partition).
+  // The partial-sum reductions stay on the main stream: beside a product they reach about
+  // 1 TB/s and slow that product by a third, which costs more than it hides (measured).
   cudaStream_t aux = nullptr;
   std::vector<cudaEvent_t> ev_fork;
   cudaEvent_t ev_join = nullptr;
@@ -329,7 +332,7 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   }
   n->partial_elems = part_elems;
   if (part_elems) ALLOC(n->partials, part_elems * sizeof(float));
-  ALLOC(n->colsum_scratch, static_cast<size_t>(32) * max_d * sizeof(float));
+  ALLOC(n->colsum_scratch, static_cast<size_t>(8 * 32) * max_d * sizeof(float));
   ALLOC(n->per_sample, B * sizeof(float));
 #undef ALLOC
   {
@@ -420,8 +423,7 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
   const bool fused = fused_eta > 0.f;
   const float scale = -fused_eta / static_cast<float>(n->B);
   const int S_r = splits_for(n->P_r, n->max_partials), S_c = splits_for(n->P_c, n->max_partials);
-  // per-kernel events bracket launches on the main stream only, so a profiled pass stays on it
-  const bool side = n->aux != nullptr && !n->prof.on;
+  const bool side = n->aux != nullptr;
   bool forked = false;
   for (int i = n->L - 1; i >= 0; --i) {
     Layer& l = n->layers[i];
@@ -433,7 +435,7 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
         cs = n->aux;
         forked = true;
       }
-      n->prof.begin(MBD_K_COLSUM, static_cast<double>(n->B) * l.d_out * (bf ? 2.0 : 4.0));
+      n->prof.begin(MBD_K_COLSUM, static_cast<double>(n->B) * l.d_out * (bf ? 2.0 : 4.0), cs);
       CK(colsum_launch(l.dY, bf, n->B, l.d_out, n->colsum_scratch, colsum_row_splits(n->B, l.d_out, n->num_sms), fused ? nullptr : l.db,
                        fused ? l.bias : nullptr, scale, cs));
       n->prof.end();
@@ -592,7 +594,7 @@ extern "C" mbd_status mbd_poll_status(mbd_net* n) {
   CK(cudaMemcpy(&h, n->status, sizeof(int), cudaMemcpyDeviceToHost));
   if (h != 0) {
     CK(cudaMemset(n->status, 0, sizeof(int)));
-    return MBD_E_TIMEOUT;
+    return h == DEV_SMEM_MISALIGNED ? MBD_E_CUDA : MBD_E_TIMEOUT;
   }
   return MBD_OK;
 }
