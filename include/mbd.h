@@ -147,6 +147,16 @@ MBD_API mbd_status mbd_train_step(mbd_net* net, const void* X_dev, const int32_t
 MBD_API mbd_status mbd_train_step_host(mbd_net* net, const void* X_host, const int32_t* labels_host,
                                float eta, float* loss_host);
 
+/* The same step, pipelined over two batches: _begin enqueues the host-to-device copy of this
+ * batch on a copy stream of the library (into one of two device staging slots), then the step
+ * and the device-to-host copy of J on the network's stream, and returns at once; _end waits
+ * for the OLDEST step begun and returns its J.  With two steps in flight the copy of batch
+ * k+1 runs under the compute of batch k.  X_host / labels_host must stay unchanged until the
+ * matching _end has returned; pinned host memory keeps the copies asynchronous.
+ * MBD_E_STATE: _begin with two steps already in flight, _end with none. */
+MBD_API mbd_status mbd_train_step_host_begin(mbd_net* net, const void* X_host, const int32_t* labels_host, float eta);
+MBD_API mbd_status mbd_train_step_host_end(mbd_net* net, float* loss_host);
+
 /* Eq. 8 / Eq. 9 bandwidth terms, one row per layer, exact integers (a term that is not
  * integral is rounded up).  Host only: needs no GPU and no network object. */
 MBD_API mbd_status mbd_comm_words(const mbd_layer* layers_host, int L, int64_t B, int P_r, int P_c,

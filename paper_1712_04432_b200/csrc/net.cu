@@ -67,6 +67,14 @@ struct mbd_net {
   Profiler prof;
   void* X_stage = nullptr;
   int32_t* labels_stage = nullptr;
+  // pipelined host steps: two landing slots for the batch, filled on a copy stream
+  cudaStream_t h2d = nullptr;
+  void* X_in[2] = {nullptr, nullptr};
+  int32_t* labels_in[2] = {nullptr, nullptr};
+  float* loss_pinned = nullptr;             // two floats of pinned host memory
+  cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_slot_free[2] = {nullptr, nullptr}, ev_step_done[2] = {nullptr, nullptr};
+  bool slot_used[2] = {false, false};
+  int pipe_head = 0, pipe_count = 0;
   ConvNet* conv = nullptr;
   // cached CUDA graph of one fused step and the arguments it was captured for
   cudaGraphExec_t graph_exec = nullptr;
@@ -205,6 +213,14 @@ void free_net(mbd_net* n) {
   }
   cudaFree(n->partials); cudaFree(n->colsum_scratch); cudaFree(n->per_sample); cudaFree(n->loss_dev);
   cudaFree(n->status); cudaFree(n->X_stage); cudaFree(n->labels_stage);
+  for (int k = 0; k < 2; ++k) {
+    cudaFree(n->X_in[k]); cudaFree(n->labels_in[k]);
+    if (n->ev_copied[k]) cudaEventDestroy(n->ev_copied[k]);
+    if (n->ev_slot_free[k]) cudaEventDestroy(n->ev_slot_free[k]);
+    if (n->ev_step_done[k]) cudaEventDestroy(n->ev_step_done[k]);
+  }
+  if (n->loss_pinned) cudaFreeHost(n->loss_pinned);
+  if (n->h2d) cudaStreamDestroy(n->h2d);
   if (n->conv) conv_destroy(n->conv);
   if (n->graph_exec) cudaGraphExecDestroy(n->graph_exec);
   for (cudaEvent_t e : n->ev_fork) if (e) cudaEventDestroy(e);
@@ -541,6 +557,69 @@ extern "C" mbd_status mbd_train_step_host(mbd_net* n, const void* X_host, const 
   if (s != MBD_OK) return s;
   CK(cudaMemcpyAsync(loss_host, n->loss_dev, sizeof(float), cudaMemcpyDeviceToHost, n->stream));
   CK(cudaStreamSynchronize(n->stream));
+  return MBD_OK;
+}
+
+namespace {
+size_t input_bytes(const mbd_net* n) {
+  return n->is_conv ? conv_input_bytes(n->conv) : static_cast<size_t>(n->B) * n->layers[0].d_in * n->elt();
+}
+
+mbd_status pipe_setup(mbd_net* n) {
+  if (n->h2d) return MBD_OK;
+  const size_t x_bytes = input_bytes(n);
+  mbd_status s;
+  if (!n->X_stage) {
+    if ((s = dev_alloc(&n->X_stage, x_bytes)) != MBD_OK) return s;
+    if ((s = dev_alloc(reinterpret_cast<void**>(&n->labels_stage), n->B * sizeof(int32_t))) != MBD_OK) return s;
+  }
+  for (int k = 0; k < 2; ++k) {
+    if ((s = dev_alloc(&n->X_in[k], x_bytes)) != MBD_OK) return s;
+    if ((s = dev_alloc(reinterpret_cast<void**>(&n->labels_in[k]), n->B * sizeof(int32_t))) != MBD_OK) return s;
+    CK(cudaEventCreateWithFlags(&n->ev_copied[k], cudaEventDisableTiming));
+    CK(cudaEventCreateWithFlags(&n->ev_slot_free[k], cudaEventDisableTiming));
+    CK(cudaEventCreateWithFlags(&n->ev_step_done[k], cudaEventDisableTiming));
+  }
+  CK(cudaMallocHost(reinterpret_cast<void**>(&n->loss_pinned), 2 * sizeof(float)));
+  CK(cudaStreamCreateWithFlags(&n->h2d, cudaStreamNonBlocking));
+  return MBD_OK;
+}
+}  // namespace
+
+extern "C" mbd_status mbd_train_step_host_begin(mbd_net* n, const void* X_host, const int32_t* labels_host, float eta) {
+  if (!n || !X_host || eta <= 0.f || (!n->is_conv && !labels_host)) return MBD_E_INVALID;
+  if (n->pipe_count == 2) return MBD_E_STATE;
+  mbd_status s = pipe_setup(n);
+  if (s != MBD_OK) return s;
+  const size_t x_bytes = input_bytes(n), l_bytes = n->B * sizeof(int32_t);
+  const int k = (n->pipe_head + n->pipe_count) & 1;
+  // copy stream: the slot must have been drained by the step that used it last
+  if (n->slot_used[k]) CK(cudaStreamWaitEvent(n->h2d, n->ev_slot_free[k], 0));
+  CK(cudaMemcpyAsync(n->X_in[k], X_host, x_bytes, cudaMemcpyHostToDevice, n->h2d));
+  if (!n->is_conv) CK(cudaMemcpyAsync(n->labels_in[k], labels_host, l_bytes, cudaMemcpyHostToDevice, n->h2d));
+  CK(cudaEventRecord(n->ev_copied[k], n->h2d));
+  // compute stream: move the batch to the buffer the (graph-captured) step reads, free the slot, run
+  CK(cudaStreamWaitEvent(n->stream, n->ev_copied[k], 0));
+  CK(cudaMemcpyAsync(n->X_stage, n->X_in[k], x_bytes, cudaMemcpyDeviceToDevice, n->stream));
+  if (!n->is_conv) CK(cudaMemcpyAsync(n->labels_stage, n->labels_in[k], l_bytes, cudaMemcpyDeviceToDevice, n->stream));
+  CK(cudaEventRecord(n->ev_slot_free[k], n->stream));
+  n->slot_used[k] = true;
+  s = mbd_train_step(n, n->X_stage, n->is_conv ? nullptr : n->labels_stage, eta, n->loss_dev);
+  if (s != MBD_OK) return s;
+  CK(cudaMemcpyAsync(n->loss_pinned + k, n->loss_dev, sizeof(float), cudaMemcpyDeviceToHost, n->stream));
+  CK(cudaEventRecord(n->ev_step_done[k], n->stream));
+  n->pipe_count++;
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_train_step_host_end(mbd_net* n, float* loss_host) {
+  if (!n || !loss_host) return MBD_E_INVALID;
+  if (n->pipe_count == 0) return MBD_E_STATE;
+  const int k = n->pipe_head;
+  CK(cudaEventSynchronize(n->ev_step_done[k]));
+  *loss_host = n->loss_pinned[k];
+  n->pipe_head ^= 1;
+  n->pipe_count--;
   return MBD_OK;
 }
 

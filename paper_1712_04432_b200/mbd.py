@@ -26,6 +26,7 @@ KERNEL_CLASSES = ["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce_partia
 EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weights", "mbd_forward",
            "mbd_backward", "mbd_sgd_step", "mbd_train_step", "mbd_train_step_host", "mbd_comm_words", "mbd_get_tensor",
            "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_gemm_bf16_noalloc", "mbd_selftest_timeout", "mbd_strerror",
+           "mbd_train_step_host_begin", "mbd_train_step_host_end",
            "mbd_comm_time", "mbd_redistribute_time", "mbd_total_time", "mbd_grid_table", "mbd_choose_grid"]
 
 
@@ -90,6 +91,8 @@ def lib():
         L.mbd_sgd_step.argtypes = [vp, f32]
         L.mbd_train_step.argtypes = [vp, vp, vp, f32, vp]
         L.mbd_train_step_host.argtypes = [vp, vp, vp, f32, C.POINTER(f32)]
+        L.mbd_train_step_host_begin.argtypes = [vp, vp, vp, f32]
+        L.mbd_train_step_host_end.argtypes = [vp, C.POINTER(f32)]
         L.mbd_comm_words.argtypes = [C.POINTER(Layer), i32, i64, i32, i32, C.POINTER(Words)]
         f64 = C.c_double
         L.mbd_comm_time.argtypes = [C.POINTER(Layer), i32, i64, i32, i32, C.POINTER(Machine), C.POINTER(Times)]
@@ -281,6 +284,18 @@ class Net:
         out = C.c_float(0.0)
         _check(lib().mbd_train_step_host(self._h, _ptr(X_host), _ptr(labels_host), float(eta), C.byref(out)),
                "mbd_train_step_host")
+        return out.value
+
+    def train_step_host_begin(self, X_host, labels_host, eta: float):
+        """Enqueue one step from host tensors (copy on the library's copy stream); at most two in flight.
+        The host tensors must stay unchanged until the matching train_step_host_end()."""
+        assert not X_host.is_cuda and X_host.is_contiguous()
+        _check(lib().mbd_train_step_host_begin(self._h, _ptr(X_host), _ptr(labels_host), float(eta)), "mbd_train_step_host_begin")
+
+    def train_step_host_end(self) -> float:
+        """Wait for the oldest step begun; returns its J."""
+        out = C.c_float(0.0)
+        _check(lib().mbd_train_step_host_end(self._h, C.byref(out)), "mbd_train_step_host_end")
         return out.value
 
     def get_tensor(self, which: int, layer: int = 0, numel: Optional[int] = None):

@@ -109,6 +109,50 @@ def test_train_step_from_host_buffers():
     net.close()
 
 
+def test_pipelined_host_steps_equal_synchronous_ones():
+    # two steps in flight (copy of batch k+1 under the compute of batch k): same losses and
+    # weights, bit for bit, as the synchronous entry point on the same sequence of batches
+    import torch
+    from paper_1712_04432_b200 import mbd
+    w = I.fc_workload((264, 136, 24), 40, "bf16")
+    batches = [I.make_inputs(w, seed=20 + k) for k in range(5)]
+    Xs = [to_dev(b.X, True).cpu().pin_memory() for b in batches]
+    ls = [torch.from_numpy(b.labels).pin_memory() for b in batches]
+
+    def fresh():
+        net = mbd.Net(mbd.fc_layers(w.dims), w.B, 2, 2, stream=torch.cuda.Stream())
+        for i in range(2):
+            net.set_weights(i, to_dev(batches[0].Ws[i], True), torch.from_numpy(batches[0].bs[i]).cuda())
+        return net
+
+    net = fresh()
+    J_sync = [net.train_step_host(Xs[k], ls[k], 0.05) for k in range(5)]
+    W_sync = [net.get_weights(i).clone() for i in range(2)]
+    torch.cuda.synchronize()
+    net.close()
+
+    net = fresh()
+    with pytest.raises(mbd.MbdError) as e:
+        net.train_step_host_end()                        # nothing in flight
+    assert e.value.status == mbd.E_STATE
+    J_pipe = []
+    net.train_step_host_begin(Xs[0], ls[0], 0.05)
+    for k in range(1, 5):
+        net.train_step_host_begin(Xs[k], ls[k], 0.05)
+        if k == 1:
+            with pytest.raises(mbd.MbdError) as e:
+                net.train_step_host_begin(Xs[k], ls[k], 0.05)    # a third step in flight
+            assert e.value.status == mbd.E_STATE
+        J_pipe.append(net.train_step_host_end())
+    J_pipe.append(net.train_step_host_end())
+    torch.cuda.synchronize()
+    assert J_pipe == J_sync
+    for i in range(2):
+        assert torch.equal(net.get_weights(i), W_sync[i])
+    assert len(set(J_sync)) == 5                         # the batches really differed
+    net.close()
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_graph_replayed_step_equals_direct_launches(dtype):
     import torch
