@@ -340,11 +340,12 @@ cudaError_t sum_f32_launch(const float* x, int64_t n, float scale, float* out, c
   return cudaGetLastError();
 }
 
-// Row splits (<= 32) so that the first stage has about eight CTAs per SM, each with >= 8 rows.
+// Row splits (<= 32) so that the first stage has about eight CTAs per SM and every warp of a CTA
+// (each writes a partial row of its own) at least eight rows to add.
 int colsum_row_splits(int64_t M, int64_t N, int num_sms) {
   const int64_t gx = (N + 255) / 256;
   int64_t r = (8 * static_cast<int64_t>(num_sms) + gx - 1) / gx;
-  if (r > M / 8) r = M / 8;
+  if (r > M / 64) r = M / 64;
   if (r > 32) r = 32;
   if (r < 1) r = 1;
   return static_cast<int>(r);
