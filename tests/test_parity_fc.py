@@ -124,3 +124,26 @@ def test_full_size_fc_workloads(name, grid, mp):
     compare_fc_step(g, o, TOL_BF16)
     gf = gpu_fc_step(w, inp, grid, max_partials=mp, fused=True)
     compare_fc_step(gf, o, TOL_BF16, fused=True, tol_below_relu=TOL_BF16_FREE)
+
+
+@pytest.mark.parametrize("case", range(10))
+def test_seeded_random_networks_and_grids(case):
+    # depth, widths (multiples of 8, so the tensor-core path applies), batch, grid, number of
+    # materialised partials and dtype drawn from a seeded generator
+    r = np.random.default_rng(4242 + case)
+    L = int(r.integers(1, 5))
+    dims = tuple(8 * int(r.integers(2, 90)) for _ in range(L + 1))
+    B = 8 * int(r.integers(1, 40))
+    dtype = "bf16" if case % 3 else "f32"
+    P_r = int(r.integers(1, min(dims[1:]) // 8 + 1))
+    P_c = int(r.integers(1, min(B, 12) + 1))
+    mp = int(r.choice([1, 2, 4, 64]))
+    fused = bool(r.integers(0, 2))
+    w = I.fc_workload(dims, B, dtype, "relu_normal" if case % 2 else "normal", name=f"random{case}")
+    inp = I.make_inputs(w, seed=100 + case)
+    o = oracle_fc_step(w, inp)
+    if dtype == "f32":
+        compare_fc_step(gpu_fc_step(w, inp, (P_r, P_c), max_partials=mp, fused=fused), o, TOL_F32, fused)
+    else:
+        g = gpu_fc_step(w, inp, (P_r, P_c), max_partials=mp, fused=fused, force_acts=oracle_hidden_acts(o))
+        compare_fc_step(g, o, TOL_BF16, fused)
