@@ -22,8 +22,11 @@
  *   - dtype MBD_BF16: X, W, activations and dY are bfloat16 bit patterns,
  *     accumulation, logits, loss, partials, dW, biases are float.
  *     dtype MBD_F32: everything float (no tensor cores; the <=1e-5 check mode).
- *   - Calls only enqueue work on the stream given at creation; nothing
- *     synchronises except mbd_poll_status, mbd_train_step_host and creation /
+ *   - Calls only enqueue work on the stream given at creation (the bias-gradient
+ *     column sums use a side stream of the library that is forked from and joined
+ *     back into that stream inside mbd_backward; the pipelined host step copies
+ *     its batches on a copy stream of the library); nothing synchronises except
+ *     mbd_poll_status, mbd_train_step_host, mbd_train_step_host_end and creation /
  *     destruction.  The library owns weights, activations, gradients and
  *     workspace; the caller owns every buffer it passes in.
  *   - Errors are return codes; nothing aborts, throws or traps.
