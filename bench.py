@@ -382,6 +382,8 @@ def run_ours(args):
                        if v["ms"] > 0 else None,
                        rate_unit="TFLOP/s" if (k.startswith("gemm") or k.startswith("conv_")) else "GB/s")
                for k, v in prof.items()}
+    if "colsum" in kernels:
+        kernels["colsum"]["note"] = "side stream, beside the products: the events span the co-running time, off the critical path"
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
