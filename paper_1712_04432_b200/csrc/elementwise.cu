@@ -18,6 +18,7 @@ namespace {
 // Vector path: M*N and N multiples of 8; each thread owns 8 consecutive columns of a row.
 __global__ void __launch_bounds__(256)
 reduce_partials_vec8(const float* __restrict__ parts, int S, int64_t M, int64_t N, const Epi epi) {
+  pdl_wait();                            // everything this kernel reads or overwrites comes from earlier kernels
   const int64_t n8 = N >> 3;
   const int64_t total = M * n8;
   const int64_t plane = M * N;
@@ -41,6 +42,7 @@ reduce_partials_vec8(const float* __restrict__ parts, int S, int64_t M, int64_t 
 
 __global__ void __launch_bounds__(256)
 reduce_partials_scalar(const float* __restrict__ parts, int S, int64_t M, int64_t N, const Epi epi) {
+  pdl_wait();                            // everything this kernel reads or overwrites comes from earlier kernels
   const int64_t total = M * N;
   for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
        i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
@@ -69,6 +71,7 @@ template <int NW>
 __global__ void __launch_bounds__(NW * 32)
 softmax_xent_kernel(const float* __restrict__ logits, int64_t d, const int32_t* __restrict__ labels,
                     void* __restrict__ dY, int dy_bf16, float* __restrict__ per_sample) {
+  pdl_wait();                            // everything this kernel reads or overwrites comes from earlier kernels
   __shared__ float red[NW];
   const int64_t b = blockIdx.x;
   const float* row = logits + b * d;
@@ -111,6 +114,7 @@ template <int NW, int VPT, bool VEC>
 __global__ void __launch_bounds__(NW * 32)
 softmax_xent_reg_kernel(const float* __restrict__ logits, int64_t d, const int32_t* __restrict__ labels,
                         void* __restrict__ dY, int dy_bf16, float* __restrict__ per_sample) {
+  pdl_wait();                            // everything this kernel reads or overwrites comes from earlier kernels
   __shared__ float red[NW];
   const int64_t b = blockIdx.x;
   const float* row = logits + b * d;
@@ -193,6 +197,7 @@ softmax_xent_reg_kernel(const float* __restrict__ logits, int64_t d, const int32
 // ------------------------------------------------------------------ fixed-order sum
 __global__ void __launch_bounds__(1024)
 sum_f32_kernel(const float* __restrict__ x, int64_t n, float scale, float* __restrict__ out) {
+  pdl_wait();                            // everything this kernel reads or overwrites comes from earlier kernels
   __shared__ float red[1024];
   float a = 0.f;
   for (int64_t i = threadIdx.x; i < n; i += 1024) a += x[i];
@@ -214,6 +219,7 @@ sum_f32_kernel(const float* __restrict__ x, int64_t n, float scale, float* __res
 template <bool BF16>
 __global__ void __launch_bounds__(256)
 colsum_stage1(const void* __restrict__ dY, int64_t M, int64_t N, int row_splits, float* __restrict__ scratch) {
+  pdl_wait();                            // everything this kernel reads or overwrites comes from earlier kernels
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t n0 = static_cast<int64_t>(blockIdx.x) * 256 + lane * 8;
   const int64_t r0 = (static_cast<int64_t>(blockIdx.y) * M) / row_splits;
@@ -253,6 +259,7 @@ colsum_stage1(const void* __restrict__ dY, int64_t M, int64_t N, int row_splits,
 __global__ void __launch_bounds__(256)
 colsum_stage2(const float* __restrict__ scratch, int row_splits, int64_t N, float* __restrict__ db,
               float* __restrict__ bias, float scale) {
+  pdl_wait();                            // everything this kernel reads or overwrites comes from earlier kernels
   const int64_t n = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
   if (n >= N) return;
   float s = 0.f;
@@ -272,6 +279,7 @@ colsum_stage2(const float* __restrict__ scratch, int row_splits, int64_t N, floa
 // ------------------------------------------------------------------ SGD update (Eq. 1)
 __global__ void __launch_bounds__(256)
 sgd_update_bf16_vec8(__nv_bfloat16* __restrict__ w, const float* __restrict__ g, int64_t n8, float scale) {
+  pdl_wait();                            // everything this kernel reads or overwrites comes from earlier kernels
   for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n8;
        i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
     const float4 a = __ldcs(reinterpret_cast<const float4*>(g + i * 8));
@@ -289,6 +297,7 @@ sgd_update_bf16_vec8(__nv_bfloat16* __restrict__ w, const float* __restrict__ g,
 
 __global__ void __launch_bounds__(256)
 sgd_update_scalar(void* __restrict__ w, int w_bf16, const float* __restrict__ g, int64_t n, float scale) {
+  pdl_wait();                            // everything this kernel reads or overwrites comes from earlier kernels
   for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n;
        i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
     if (w_bf16) {
@@ -315,29 +324,25 @@ cudaError_t reduce_partials_launch(const float* parts, int S, int64_t M, int64_t
                                    cudaStream_t stream) {
   const bool vec = (N % 8 == 0) && (epi.ldo % 8 == 0) && (epi.mask == nullptr || epi.ldmask % 8 == 0);
   if (vec) {
-    reduce_partials_vec8<<<grid_for(M * (N / 8), num_sms, 8), 256, 0, stream>>>(parts, S, M, N, epi);
-  } else {
-    reduce_partials_scalar<<<grid_for(M * N, num_sms, 8), 256, 0, stream>>>(parts, S, M, N, epi);
+    return launch_pdl(reduce_partials_vec8, dim3(grid_for(M * (N / 8), num_sms, 8)), dim3(256), 0, stream, 1, parts, S, M, N, epi);
   }
-  return cudaGetLastError();
+  return launch_pdl(reduce_partials_scalar, dim3(grid_for(M * N, num_sms, 8)), dim3(256), 0, stream, 1, parts, S, M, N, epi);
 }
 
 cudaError_t softmax_xent_launch(const float* logits, int64_t B, int64_t d, const int32_t* labels, void* dY,
                                 int dy_bf16, float* per_sample, cudaStream_t stream) {
   const unsigned nb = static_cast<unsigned>(B);
   const bool vec = d % 4 == 0;
-  if (d <= 64) softmax_xent_reg_kernel<1, 2, false><<<nb, 32, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
-  else if (d <= 1024 && vec) softmax_xent_reg_kernel<4, 8, true><<<nb, 128, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
-  else if (d <= 1024) softmax_xent_reg_kernel<4, 8, false><<<nb, 128, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
-  else if (d <= 8192 && vec) softmax_xent_reg_kernel<8, 32, true><<<nb, 256, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
-  else if (d <= 8192) softmax_xent_reg_kernel<8, 32, false><<<nb, 256, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
-  else softmax_xent_kernel<8><<<nb, 256, 0, stream>>>(logits, d, labels, dY, dy_bf16, per_sample);
-  return cudaGetLastError();
+  if (d <= 64) return launch_pdl(softmax_xent_reg_kernel<1, 2, false>, dim3(nb), dim3(32), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
+  if (d <= 1024 && vec) return launch_pdl(softmax_xent_reg_kernel<4, 8, true>, dim3(nb), dim3(128), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
+  if (d <= 1024) return launch_pdl(softmax_xent_reg_kernel<4, 8, false>, dim3(nb), dim3(128), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
+  if (d <= 8192 && vec) return launch_pdl(softmax_xent_reg_kernel<8, 32, true>, dim3(nb), dim3(256), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
+  if (d <= 8192) return launch_pdl(softmax_xent_reg_kernel<8, 32, false>, dim3(nb), dim3(256), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
+  return launch_pdl(softmax_xent_kernel<8>, dim3(nb), dim3(256), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
 }
 
 cudaError_t sum_f32_launch(const float* x, int64_t n, float scale, float* out, cudaStream_t stream) {
-  sum_f32_kernel<<<1, 1024, 0, stream>>>(x, n, scale, out);
-  return cudaGetLastError();
+  return launch_pdl(sum_f32_kernel, dim3(1), dim3(1024), 0, stream, 1, x, n, scale, out);
 }
 
 // Row splits (<= 32) so that the first stage has about eight CTAs per SM and every warp of a CTA
@@ -356,22 +361,19 @@ int colsum_launches(int64_t, int64_t, int) { return 2; }
 cudaError_t colsum_launch(const void* dY, int dy_bf16, int64_t M, int64_t N, float* scratch, int row_splits,
                           float* db, float* bias, float scale, cudaStream_t stream) {
   dim3 g1(static_cast<unsigned>((N + 255) / 256), row_splits);
-  if (dy_bf16) colsum_stage1<true><<<g1, 256, 0, stream>>>(dY, M, N, row_splits, scratch);
-  else colsum_stage1<false><<<g1, 256, 0, stream>>>(dY, M, N, row_splits, scratch);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = dy_bf16 ? launch_pdl(colsum_stage1<true>, g1, dim3(256), 0, stream, 1, dY, M, N, row_splits, scratch)
+                          : launch_pdl(colsum_stage1<false>, g1, dim3(256), 0, stream, 1, dY, M, N, row_splits, scratch);
   if (e != cudaSuccess) return e;
-  colsum_stage2<<<static_cast<unsigned>((N + 255) / 256), 256, 0, stream>>>(scratch, row_splits * 8, N, db, bias, scale);
-  return cudaGetLastError();
+  return launch_pdl(colsum_stage2, dim3(static_cast<unsigned>((N + 255) / 256)), dim3(256), 0, stream, 1, static_cast<const float*>(scratch),
+                    row_splits * 8, N, db, bias, scale);
 }
 
 cudaError_t sgd_update_launch(void* w, int w_bf16, const float* g, int64_t n, float scale, int num_sms,
                               cudaStream_t stream) {
   if (w_bf16 && n % 8 == 0) {
-    sgd_update_bf16_vec8<<<grid_for(n / 8, num_sms, 8), 256, 0, stream>>>(reinterpret_cast<__nv_bfloat16*>(w), g, n / 8, scale);
-  } else {
-    sgd_update_scalar<<<grid_for(n, num_sms, 8), 256, 0, stream>>>(w, w_bf16, g, n, scale);
+    return launch_pdl(sgd_update_bf16_vec8, dim3(grid_for(n / 8, num_sms, 8)), dim3(256), 0, stream, 1, reinterpret_cast<__nv_bfloat16*>(w), g, n / 8, scale);
   }
-  return cudaGetLastError();
+  return launch_pdl(sgd_update_scalar, dim3(grid_for(n, num_sms, 8)), dim3(256), 0, stream, 1, w, w_bf16, g, n, scale);
 }
 
 }  // namespace mbd

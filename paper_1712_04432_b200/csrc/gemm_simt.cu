@@ -13,6 +13,7 @@ namespace {
 template <int R>
 __global__ void __launch_bounds__(256)
 simt_gemm_kernel(const SimtGemm g) {
+  pdl_wait();                            // operands come from earlier kernels
   constexpr int TM = 16 * R, TN = 16 * R;
   constexpr int TK = R == 2 ? 64 : 16;
   __shared__ float As[TK][TM + 4];
@@ -83,12 +84,10 @@ cudaError_t simt_gemm_launch(const SimtGemm& g, cudaStream_t stream) {
   const long long big = 1ll * ((g.N + 63) / 64) * ((g.M + 63) / 64) * g.k_splits;
   if (big >= 148) {
     dim3 grid((g.N + 63) / 64, (g.M + 63) / 64, g.k_splits);
-    simt_gemm_kernel<4><<<grid, 256, 0, stream>>>(g);
-  } else {
-    dim3 grid((g.N + 31) / 32, (g.M + 31) / 32, g.k_splits);
-    simt_gemm_kernel<2><<<grid, 256, 0, stream>>>(g);
+    return launch_pdl(simt_gemm_kernel<4>, grid, dim3(256), 0, stream, 1, g);
   }
-  return cudaGetLastError();
+  dim3 grid((g.N + 31) / 32, (g.M + 31) / 32, g.k_splits);
+  return launch_pdl(simt_gemm_kernel<2>, grid, dim3(256), 0, stream, 1, g);
 }
 
 }  // namespace mbd

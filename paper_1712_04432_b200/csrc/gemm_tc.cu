@@ -202,6 +202,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (PAIR) cluster_sync_all();            // both CTAs' barriers exist before anything remote touches them
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
+  // Set-up is done: the kernel after this one may be scheduled; and from here on this one touches
+  // global memory, so whatever ran before it must have finished.
+  pdl_trigger();
+  pdl_wait();
 
   const int total_work = p.tiles_m * p.tiles_n * p.S;
   volatile int* abortp = &abort_flag;
@@ -556,25 +560,13 @@ cudaError_t set_attr() {
 template <int A_MN, int B_MN>
 cudaError_t launch_t(const TcGemm& g, const Params& p, cudaStream_t stream) {
   const size_t smem = SMEM_DYN_BYTES;
-  if (g.pair) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(g.grid);
-    cfg.blockDim = dim3(NUM_THREADS);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (g.MH == 2) return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<A_MN, B_MN, 256, 2, 1>, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<A_MN, B_MN, 256, 1, 1>, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  }
-  if (g.BN == 256 && g.MH == 1) gemm_tc_kernel<A_MN, B_MN, 256, 1, 0><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  else if (g.BN == 128 && g.MH == 1) gemm_tc_kernel<A_MN, B_MN, 128, 1, 0><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  else if (g.BN == 256) gemm_tc_kernel<A_MN, B_MN, 256, 2, 0><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  else gemm_tc_kernel<A_MN, B_MN, 128, 2, 0><<<g.grid, NUM_THREADS, smem, stream>>>(g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  return cudaGetLastError();
+  const dim3 grid(g.grid), block(NUM_THREADS);
+  if (g.pair && g.MH == 2) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  if (g.pair) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  if (g.BN == 256 && g.MH == 1) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 1, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  if (g.BN == 128 && g.MH == 1) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 128, 1, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  if (g.BN == 256) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 2, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 128, 2, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
 }
 
 }  // namespace

@@ -8,6 +8,11 @@
 
 namespace mbd {
 
+bool pdl_enabled() {
+  static const bool on = getenv("MBD_NO_PDL") == nullptr;
+  return on;
+}
+
 cudaEvent_t Profiler::get_event() {
   if (n_pool > 0) return pool[--n_pool];
   cudaEvent_t e = nullptr;
