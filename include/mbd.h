@@ -169,7 +169,7 @@ MBD_API mbd_status mbd_comm_words(const mbd_layer* layers_host, int L, int64_t B
  * Section 3).  Host only, no GPU.  A collective costs alpha * messages + beta * words:
  * all-gather of Y_i over P_r: ceil(log2 P_r) messages; all-reduce of dX_i (layers >= 2) over
  * P_r: 2 ceil(log2 P_r); all-reduce of dW_i over P_c: 2 ceil(log2 P_c); a domain-split layer:
- * one message per halo exchange (none for a single strip) and 2 ceil(log2 P) for its
+ * one message per halo exchange (none for a single strip or a 1 x 1 kernel) and 2 ceil(log2 P) for its
  * all-reduce over all P processes.  The words are those of mbd_comm_words before rounding. */
 typedef struct {
   double alpha;   /* latency per message, seconds                           */

@@ -20,7 +20,8 @@ Readings taken (the paper leaves these open):
     coincide with the integer word counts whenever those are integral;
   * "d_{i-1}" is the size of the layer's own input (they differ when a pooling layer sits
     between two weighted layers);
-  * the halo terms, latency included, vanish for a single strip (P_r = 1);
+  * the halo terms, latency included, vanish for a single strip (P_r = 1) and for a 1 x 1
+    convolution (floor(k_h/2) = 0: "no communication is needed", remark after Eq. 7);
   * sums run over the layers that own a weight matrix;
   * overlap (Section 3, the variant with communication hidden behind back-propagation): the
     two all-reduces (two thirds of the products' communication) run behind the backward
@@ -66,7 +67,7 @@ def layer_messages(layers: Sequence[Dict], P_r: int, P_c: int) -> List[Dict[str,
                 row["allreduce_dx"] = 2 * ceil_log2(P_r)
             row["allreduce_dw"] = 2 * ceil_log2(P_c)
         else:
-            if P_r > 1:
+            if P_r > 1 and l["kh"] // 2 > 0:      # a 1 x 1 convolution exchanges nothing (remark after Eq. 7)
                 row["halo_fwd"] = 1
                 row["halo_bwd"] = 1
             row["allreduce_dw"] = 2 * ceil_log2(P)
@@ -126,7 +127,7 @@ def eq7_domain_time(layers: Sequence[Dict], B: int, P: int, alpha: float, beta: 
     t = 0.0
     lg = ceil_log2(P)
     for l in layers:
-        if P > 1:
+        if P > 1 and l["kh"] // 2 > 0:
             t += alpha + beta * B * l["W"] * l["C_in"] * (l["kh"] // 2)
             t += alpha + beta * B * l["W"] * l["C_out"] * (l["kh"] // 2)
         t += 2.0 * (alpha * lg + beta * float(Fraction((P - 1) * n_weights(l), P)))

@@ -58,7 +58,7 @@ mbd_status layer_row(const mbd_layer& l, int split, bool first, double B, int P_
   }
   if (split == MBD_SPLIT_DOMAIN) {
     if (!d.conv) return MBD_E_INVALID;   // no halo notion for a fully connected layer
-    if (P_r > 1) {
+    if (P_r > 1 && l.kh / 2 > 0) {         // a 1 x 1 convolution exchanges nothing (remark after Eq. 7)
       const double rows = static_cast<double>(l.kh / 2);
       t->halo_fwd = m.alpha + m.beta * (B / pc) * l.W * l.C_in * rows;
       t->halo_bwd = m.alpha + m.beta * (B / pc) * l.W * l.C_out * rows;

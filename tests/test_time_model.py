@@ -20,8 +20,9 @@ def random_net(r: random.Random, kind: str):
     convs = []
     for _ in range(r.randint(1, 4)):
         c = r.choice([3, 16, 64, 384])
+        k = r.choice([1, 3, 3, 5])
         convs.append(dict(kind="conv", C_in=c, C_out=r.choice([16, 64, 256]), H=r.choice([13, 32, 224]), W=r.choice([13, 32, 224]),
-                          kh=3, kw=3, split="domain" if kind == "conv_domain" else "model"))
+                          kh=k, kw=k, split="domain" if kind == "conv_domain" else "model"))
     if kind == "mixed":
         convs += [dict(kind="fc", d_in=convs[-1]["C_out"] * convs[-1]["H"] * convs[-1]["W"], d_out=256), dict(kind="fc", d_in=256, d_out=10)]
     return convs

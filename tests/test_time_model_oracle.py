@@ -88,6 +88,18 @@ def test_domain_layers_contain_pure_domain_parallelism():
         assert T.eq7_domain_time(layers, 32, P, A, Bt) > T.eq4_batch_time(layers, P, A, Bt)
 
 
+def test_one_by_one_convolution_needs_no_halo_exchange():
+    # remark after Eq. 7: for a 1 x 1 convolution no communication is needed beyond the all-reduce of dW
+    l = dict(kind="conv", C_in=64, C_out=64, H=56, W=56, kh=1, kw=1, split="domain")
+    row = T.layer_times([l], 32, 4, 1, A, Bt)[0]
+    assert row["halo_fwd"] == 0.0 and row["halo_bwd"] == 0.0
+    assert math.isclose(row["allreduce_dw"], 2 * (A * 2 + Bt * 3 / 4 * 64 * 64), rel_tol=1e-13)
+    assert math.isclose(T.eq7_domain_time([l], 32, 4, A, Bt), row["allreduce_dw"], rel_tol=1e-13)
+    # a 3 x 3 kernel on the same activations does pay two halo messages
+    l3 = dict(l, kh=3, kw=3)
+    assert T.layer_times([l3], 32, 4, 1, 1.0, 0.0)[0]["halo_fwd"] == 1.0
+
+
 def test_hand_computed_example():
     # two layers 6 -> 4 -> 2, B = 12, grid 2 x 3, alpha = 1, beta = 1/10 (by hand):
     # layer 1: all-gather 1 msg + 12/3 * 1/2 * 4 = 8 words; dW 2*2 msgs + 2 * 2/3 * 24/2 = 16 words
