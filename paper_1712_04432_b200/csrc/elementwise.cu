@@ -324,25 +324,25 @@ cudaError_t reduce_partials_launch(const float* parts, int S, int64_t M, int64_t
                                    cudaStream_t stream) {
   const bool vec = (N % 8 == 0) && (epi.ldo % 8 == 0) && (epi.mask == nullptr || epi.ldmask % 8 == 0);
   if (vec) {
-    return launch_pdl(reduce_partials_vec8, dim3(grid_for(M * (N / 8), num_sms, 8)), dim3(256), 0, stream, 1, parts, S, M, N, epi);
+    return launch_pdl(reduce_partials_vec8, dim3(grid_for(M * (N / 8), num_sms, 8)), dim3(256), 0, stream, 0, parts, S, M, N, epi);
   }
-  return launch_pdl(reduce_partials_scalar, dim3(grid_for(M * N, num_sms, 8)), dim3(256), 0, stream, 1, parts, S, M, N, epi);
+  return launch_pdl(reduce_partials_scalar, dim3(grid_for(M * N, num_sms, 8)), dim3(256), 0, stream, 0, parts, S, M, N, epi);
 }
 
 cudaError_t softmax_xent_launch(const float* logits, int64_t B, int64_t d, const int32_t* labels, void* dY,
                                 int dy_bf16, float* per_sample, cudaStream_t stream) {
   const unsigned nb = static_cast<unsigned>(B);
   const bool vec = d % 4 == 0;
-  if (d <= 64) return launch_pdl(softmax_xent_reg_kernel<1, 2, false>, dim3(nb), dim3(32), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
-  if (d <= 1024 && vec) return launch_pdl(softmax_xent_reg_kernel<4, 8, true>, dim3(nb), dim3(128), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
-  if (d <= 1024) return launch_pdl(softmax_xent_reg_kernel<4, 8, false>, dim3(nb), dim3(128), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
-  if (d <= 8192 && vec) return launch_pdl(softmax_xent_reg_kernel<8, 32, true>, dim3(nb), dim3(256), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
-  if (d <= 8192) return launch_pdl(softmax_xent_reg_kernel<8, 32, false>, dim3(nb), dim3(256), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
-  return launch_pdl(softmax_xent_kernel<8>, dim3(nb), dim3(256), 0, stream, 1, logits, d, labels, dY, dy_bf16, per_sample);
+  if (d <= 64) return launch_pdl(softmax_xent_reg_kernel<1, 2, false>, dim3(nb), dim3(32), 0, stream, 0, logits, d, labels, dY, dy_bf16, per_sample);
+  if (d <= 1024 && vec) return launch_pdl(softmax_xent_reg_kernel<4, 8, true>, dim3(nb), dim3(128), 0, stream, 0, logits, d, labels, dY, dy_bf16, per_sample);
+  if (d <= 1024) return launch_pdl(softmax_xent_reg_kernel<4, 8, false>, dim3(nb), dim3(128), 0, stream, 0, logits, d, labels, dY, dy_bf16, per_sample);
+  if (d <= 8192 && vec) return launch_pdl(softmax_xent_reg_kernel<8, 32, true>, dim3(nb), dim3(256), 0, stream, 0, logits, d, labels, dY, dy_bf16, per_sample);
+  if (d <= 8192) return launch_pdl(softmax_xent_reg_kernel<8, 32, false>, dim3(nb), dim3(256), 0, stream, 0, logits, d, labels, dY, dy_bf16, per_sample);
+  return launch_pdl(softmax_xent_kernel<8>, dim3(nb), dim3(256), 0, stream, 0, logits, d, labels, dY, dy_bf16, per_sample);
 }
 
 cudaError_t sum_f32_launch(const float* x, int64_t n, float scale, float* out, cudaStream_t stream) {
-  return launch_pdl(sum_f32_kernel, dim3(1), dim3(1024), 0, stream, 1, x, n, scale, out);
+  return launch_pdl(sum_f32_kernel, dim3(1), dim3(1024), 0, stream, 0, x, n, scale, out);
 }
 
 // Row splits (<= 32) so that the first stage has about eight CTAs per SM and every warp of a CTA
@@ -361,19 +361,19 @@ int colsum_launches(int64_t, int64_t, int) { return 2; }
 cudaError_t colsum_launch(const void* dY, int dy_bf16, int64_t M, int64_t N, float* scratch, int row_splits,
                           float* db, float* bias, float scale, cudaStream_t stream) {
   dim3 g1(static_cast<unsigned>((N + 255) / 256), row_splits);
-  cudaError_t e = dy_bf16 ? launch_pdl(colsum_stage1<true>, g1, dim3(256), 0, stream, 1, dY, M, N, row_splits, scratch)
-                          : launch_pdl(colsum_stage1<false>, g1, dim3(256), 0, stream, 1, dY, M, N, row_splits, scratch);
+  cudaError_t e = dy_bf16 ? launch_pdl(colsum_stage1<true>, g1, dim3(256), 0, stream, 0, dY, M, N, row_splits, scratch)
+                          : launch_pdl(colsum_stage1<false>, g1, dim3(256), 0, stream, 0, dY, M, N, row_splits, scratch);
   if (e != cudaSuccess) return e;
-  return launch_pdl(colsum_stage2, dim3(static_cast<unsigned>((N + 255) / 256)), dim3(256), 0, stream, 1, static_cast<const float*>(scratch),
+  return launch_pdl(colsum_stage2, dim3(static_cast<unsigned>((N + 255) / 256)), dim3(256), 0, stream, 0, static_cast<const float*>(scratch),
                     row_splits * 8, N, db, bias, scale);
 }
 
 cudaError_t sgd_update_launch(void* w, int w_bf16, const float* g, int64_t n, float scale, int num_sms,
                               cudaStream_t stream) {
   if (w_bf16 && n % 8 == 0) {
-    return launch_pdl(sgd_update_bf16_vec8, dim3(grid_for(n / 8, num_sms, 8)), dim3(256), 0, stream, 1, reinterpret_cast<__nv_bfloat16*>(w), g, n / 8, scale);
+    return launch_pdl(sgd_update_bf16_vec8, dim3(grid_for(n / 8, num_sms, 8)), dim3(256), 0, stream, 0, reinterpret_cast<__nv_bfloat16*>(w), g, n / 8, scale);
   }
-  return launch_pdl(sgd_update_scalar, dim3(grid_for(n, num_sms, 8)), dim3(256), 0, stream, 1, w, w_bf16, g, n, scale);
+  return launch_pdl(sgd_update_scalar, dim3(grid_for(n, num_sms, 8)), dim3(256), 0, stream, 0, w, w_bf16, g, n, scale);
 }
 
 }  // namespace mbd

@@ -17,6 +17,9 @@ namespace mbd {
 // call pdl_wait() before it reads or writes anything the predecessor touches.  What comes before
 // pdl_wait() -- barrier set-up, tensor-memory allocation, the launch itself -- then overlaps the
 // predecessor's tail.  Both calls do nothing in a kernel launched the ordinary way.
+// Only the GEMMs are launched this way (cluster_x >= 1; pass 0 for an ordinary launch): a
+// memory-bound kernel that becomes resident early just waits beside the product it depends on and
+// slowed the split products' steps by 4 % when it was tried.
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -38,7 +41,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     attr[n].val.clusterDim.x = static_cast<unsigned>(cluster_x); attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;
     ++n;
   }
-  if (pdl_enabled()) {
+  if (pdl_enabled() && cluster_x >= 1) {
     attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[n].val.programmaticStreamSerializationAllowed = 1;
     ++n;
