@@ -234,6 +234,8 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
   volatile int* abortp = &abort_flag;
+  pdl_trigger();                           // set-up done: the next kernel may be scheduled
+  pdl_wait();                              // from here on global memory: earlier kernels must have finished
 
   const int i0 = static_cast<int>((static_cast<long long>(blockIdx.x) * p.n_items) / gridDim.x);
   const int i1 = static_cast<int>((static_cast<long long>(blockIdx.x + 1) * p.n_items) / gridDim.x);
@@ -439,6 +441,8 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
   volatile int* abortp = &abort_flag;
+  pdl_trigger();                           // set-up done: the next kernel may be scheduled
+  pdl_wait();                              // from here on global memory: earlier kernels must have finished
 
   const int i0 = static_cast<int>((static_cast<long long>(blockIdx.x) * p.n_items) / gridDim.x);
   const int i1 = static_cast<int>((static_cast<long long>(blockIdx.x + 1) * p.n_items) / gridDim.x);
@@ -653,7 +657,7 @@ void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w
   if (mode == MODE_STORE_SSQ) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 8, c->stream);
   const double flops = 2.0 * c->B * c->H * c->W * 9.0 * C * C;
   c->prof->begin(cls, flops);
-  conv_fwd_kernel<<<grid, FWD_THREADS, FWD_SMEM, c->stream>>>(in, w, p);
+  launch_pdl(conv_fwd_kernel, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, p);
   c->prof->end();
 }
 
@@ -783,7 +787,7 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
     p.part = c->wpart; p.status = c->status;
     const int grid = p.n_items < c->grid ? p.n_items : c->grid;
     c->prof->begin(MBD_K_CONV_BWD_WEIGHT, 2.0 * c->B * c->H * c->W * 9.0 * C * C);
-    conv_wgrad_kernel<<<grid, NUM_THREADS, WG_SMEM, c->stream>>>(c->act_wg[i], c->dY_wg[i], p);
+    launch_pdl(conv_wgrad_kernel, dim3(grid), dim3(NUM_THREADS), WG_SMEM, c->stream, 1, c->act_wg[i], c->dY_wg[i], p);
     c->prof->end();
     c->prof->begin(MBD_K_REDUCE, (grid + 1.0) * 9 * C * C * 4.0);
     wgrad_finish_kernel<<<9 * C * C / 64, 256, 0, c->stream>>>(c->wpart, grid, fused ? nullptr : c->dK[i],
