@@ -10,6 +10,7 @@
 // of W_i is ordered after the dX_i product of the same layer, which still reads the old W_i.
 #include <algorithm>
 #include <new>
+#include <stdlib.h>
 #include <vector>
 
 #include "../../include/mbd.h"
@@ -439,13 +440,17 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
   const bool fused = fused_eta > 0.f;
   const float scale = -fused_eta / static_cast<float>(n->B);
   const int S_r = splits_for(n->P_r, n->max_partials), S_c = splits_for(n->P_c, n->max_partials);
-  const bool side = n->aux != nullptr;
+  static const bool no_side = getenv("MBD_NO_SIDE") != nullptr;      // tuning knob: column sums on the main stream
+  const bool side = n->aux != nullptr && !no_side;
   bool forked = false;
   for (int i = n->L - 1; i >= 0; --i) {
     Layer& l = n->layers[i];
     if (l.bias) {
       cudaStream_t cs = n->stream;
-      if (side) {
+      // Small sums are launch-bound and hide entirely beside the products; a large one (cfg5: 134 MB)
+      // slows the product it runs beside by more than its own 0.04 ms, so it stays in line.
+      const bool small = static_cast<double>(n->B) * l.d_out * (bf ? 2.0 : 4.0) <= 32.0 * 1024 * 1024;
+      if (side && small) {
         CK(cudaEventRecord(n->ev_fork[i], n->stream));
         CK(cudaStreamWaitEvent(n->aux, n->ev_fork[i], 0));
         cs = n->aux;
