@@ -58,6 +58,9 @@ struct mbd_net {
   cudaStream_t aux = nullptr;
   std::vector<cudaEvent_t> ev_fork;
   cudaEvent_t ev_join = nullptr;
+  cudaEvent_t ev_loss = nullptr;            // forward done -> the sum of the per-sample losses may start
+  bool defer_loss = false;                  // set by mbd_train_step: J is only needed when the step is over
+  bool loss_pending = false;                // the loss sum runs on the side stream, not joined yet
   float* per_sample = nullptr;
   float* loss_dev = nullptr;
   int* status = nullptr;
@@ -226,6 +229,7 @@ void free_net(mbd_net* n) {
   if (n->graph_exec) cudaGraphExecDestroy(n->graph_exec);
   for (cudaEvent_t e : n->ev_fork) if (e) cudaEventDestroy(e);
   if (n->ev_join) cudaEventDestroy(n->ev_join);
+  if (n->ev_loss) cudaEventDestroy(n->ev_loss);
   if (n->aux) cudaStreamDestroy(n->aux);
   n->prof.destroy();
   (void)cudaGetLastError();
@@ -354,7 +358,8 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
 #undef ALLOC
   {
     bool ok = cudaStreamCreateWithFlags(&n->aux, cudaStreamNonBlocking) == cudaSuccess &&
-              cudaEventCreateWithFlags(&n->ev_join, cudaEventDisableTiming) == cudaSuccess;
+              cudaEventCreateWithFlags(&n->ev_join, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&n->ev_loss, cudaEventDisableTiming) == cudaSuccess;
     n->ev_fork.assign(L, nullptr);
     for (int i = 0; i < L && ok; ++i) ok = cudaEventCreateWithFlags(&n->ev_fork[i], cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { free_net(n); return MBD_E_CUDA; }
@@ -420,8 +425,16 @@ extern "C" mbd_status mbd_forward(mbd_net* n, const void* X_dev, const int32_t* 
   CK(softmax_xent_launch(static_cast<const float*>(top.act), n->B, top.d_out, labels_dev, top.dY, bf, n->per_sample, n->stream));
   n->prof.end();
   if (loss_sum_dev) {
-    n->prof.begin(MBD_K_OTHER, static_cast<double>(n->B) * 4.0);
-    CK(sum_f32_launch(n->per_sample, n->B, 1.f, loss_sum_dev, n->stream));
+    // inside a whole step nothing waits for J: its (single-CTA) sum goes to the side stream
+    cudaStream_t ls = n->stream;
+    if (n->defer_loss && n->aux) {
+      CK(cudaEventRecord(n->ev_loss, n->stream));
+      CK(cudaStreamWaitEvent(n->aux, n->ev_loss, 0));
+      ls = n->aux;
+      n->loss_pending = true;
+    }
+    n->prof.begin(MBD_K_OTHER, static_cast<double>(n->B) * 4.0, ls);
+    CK(sum_f32_launch(n->per_sample, n->B, 1.f, loss_sum_dev, ls));
     n->prof.end();
   }
   n->state = ST_FWD;
@@ -471,6 +484,7 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
     mbd_status s = run_gemm(n, l.bwd_weight, 2, l.d_out, l.d_in, n->B, l.dY, l.d_out, layer_input(n, i), l.d_in, S_c, e);
     if (s != MBD_OK) return s;
   }
+  if (n->loss_pending) { forked = true; n->loss_pending = false; }
   if (forked) {
     CK(cudaEventRecord(n->ev_join, n->aux));
     CK(cudaStreamWaitEvent(n->stream, n->ev_join, 0));
@@ -507,7 +521,9 @@ extern "C" mbd_status mbd_train_step(mbd_net* n, const void* X_dev, const int32_
   if (!n || !X_dev || eta <= 0.f) return MBD_E_INVALID;
   // per-kernel events cannot be recorded inside a graph, and the default stream cannot be captured
   if (n->prof.on || n->stream == nullptr || n->stream == cudaStreamLegacy || n->stream == cudaStreamPerThread) {
+    n->defer_loss = !n->is_conv;
     mbd_status s = mbd_forward(n, X_dev, labels_dev, loss_sum_dev);
+    n->defer_loss = false;
     return s != MBD_OK ? s : mbd_backward(n, eta);
   }
   const bool same = n->graph_exec && n->g_X == X_dev && n->g_labels == labels_dev && n->g_loss == loss_sum_dev && n->g_eta == eta;
@@ -519,7 +535,9 @@ extern "C" mbd_status mbd_train_step(mbd_net* n, const void* X_dev, const int32_
     if (s != MBD_OK) return s;
     const int64_t launches_before = n->prof.total_launches;
     CK(cudaStreamBeginCapture(n->stream, cudaStreamCaptureModeThreadLocal));
+    n->defer_loss = !n->is_conv;
     s = mbd_forward(n, X_dev, labels_dev, loss_sum_dev);
+    n->defer_loss = false;
     if (s == MBD_OK) s = mbd_backward(n, eta);
     cudaGraph_t graph = nullptr;
     const cudaError_t ce = cudaStreamEndCapture(n->stream, &graph);
