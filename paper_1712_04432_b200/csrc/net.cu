@@ -58,6 +58,17 @@ struct mbd_net {
   cudaStream_t aux = nullptr;
   std::vector<cudaEvent_t> ev_fork;
   cudaEvent_t ev_join = nullptr;
+  // Small networks (every backward-weight product under 0.2 TFLOP): the backward-weight products,
+  // which nothing inside the step waits for, run on a stream of their own beside the chain of
+  // backward-data products; their kernels leave SMs idle that the other stream's CTAs fill.
+  // dW_i starts once the backward-data product of layer i (the last reader of the old W_i) is done.
+  cudaStream_t wstream = nullptr;
+  bool overlap_dw = false;
+  std::vector<cudaEvent_t> ev_dx;           // per layer: dY_i final and W_i no longer read
+  cudaEvent_t ev_wjoin = nullptr;
+  float* partials_dw = nullptr;             // partials of the backward-weight products when they run beside the others
+  size_t last_dw_elems = 0;
+  bool last_red_dw = false;                 // the last reduction executed used partials_dw
   cudaEvent_t ev_loss = nullptr;            // forward done -> the sum of the per-sample losses may start
   bool defer_loss = false;                  // set by mbd_train_step: J is only needed when the step is over
   bool loss_pending = false;                // the loss sum runs on the side stream, not joined yet
@@ -132,14 +143,18 @@ Epi epi_sgd(void* w, int64_t ldo, int out_bf16, float scale) {
 
 // One contraction on the path that matches the network dtype, followed by the reduction
 // of its partials when the K range was split.
+// `stream` / `parts`: null selects the network's stream and the common partial-sum workspace.
 mbd_status run_gemm(mbd_net* n, TcGemm& tc, int variant, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
-                    const void* Bm, int64_t ldb, int S, const Epi& epi) {
+                    const void* Bm, int64_t ldb, int S, const Epi& epi, cudaStream_t stream = nullptr, float* parts = nullptr) {
   const double flops = 2.0 * static_cast<double>(M) * static_cast<double>(N) * static_cast<double>(K);
+  if (!stream) stream = n->stream;
+  const bool own_parts = parts != nullptr;
+  if (!parts) parts = n->partials;
   if (n->dtype == MBD_BF16) {
     tc.epi = epi;
-    tc.partials = n->partials;
-    n->prof.begin(MBD_K_GEMM_FWD + variant, flops);
-    CK(tc_gemm_launch(tc, n->stream));
+    tc.partials = parts;
+    n->prof.begin(MBD_K_GEMM_FWD + variant, flops, stream);
+    CK(tc_gemm_launch(tc, stream));
     n->prof.end();
     S = tc.k_splits;
   } else {
@@ -152,10 +167,10 @@ mbd_status run_gemm(mbd_net* n, TcGemm& tc, int variant, int64_t M, int64_t N, i
     else { g.a_sm = 1; g.a_sk = lda; g.b_sn = 1; g.b_sk = ldb; }
     if (S > K) S = static_cast<int>(K);
     g.k_splits = S;
-    g.partials = n->partials;
+    g.partials = parts;
     g.epi = epi;
-    n->prof.begin(MBD_K_GEMM_FWD + variant, flops);
-    CK(simt_gemm_launch(g, n->stream));
+    n->prof.begin(MBD_K_GEMM_FWD + variant, flops, stream);
+    CK(simt_gemm_launch(g, stream));
     n->prof.end();
   }
   if (S > 1) {
@@ -163,9 +178,10 @@ mbd_status run_gemm(mbd_net* n, TcGemm& tc, int variant, int64_t M, int64_t N, i
     const double esz = epi.out_bf16 ? 2.0 : 4.0;
     double bytes = static_cast<double>(M) * N * (4.0 * S + esz);
     if (epi.op == EPI_SGD || (epi.op == EPI_MASK && epi.mask)) bytes += static_cast<double>(M) * N * esz;
-    n->prof.begin(MBD_K_REDUCE, bytes);
-    CK(reduce_partials_launch(n->partials, S, M, N, epi, n->num_sms, n->stream));
+    n->prof.begin(MBD_K_REDUCE, bytes, stream);
+    CK(reduce_partials_launch(parts, S, M, N, epi, n->num_sms, stream));
     n->prof.end();
+    n->last_red_dw = own_parts;
   }
   return MBD_OK;
 }
@@ -230,6 +246,10 @@ void free_net(mbd_net* n) {
   for (cudaEvent_t e : n->ev_fork) if (e) cudaEventDestroy(e);
   if (n->ev_join) cudaEventDestroy(n->ev_join);
   if (n->ev_loss) cudaEventDestroy(n->ev_loss);
+  for (cudaEvent_t e : n->ev_dx) if (e) cudaEventDestroy(e);
+  if (n->ev_wjoin) cudaEventDestroy(n->ev_wjoin);
+  if (n->wstream) cudaStreamDestroy(n->wstream);
+  cudaFree(n->partials_dw);
   if (n->aux) cudaStreamDestroy(n->aux);
   n->prof.destroy();
   (void)cudaGetLastError();
@@ -353,6 +373,20 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   }
   n->partial_elems = part_elems;
   if (part_elems) ALLOC(n->partials, part_elems * sizeof(float));
+  {
+    // backward-weight products beside the backward-data chain: only where every one of them is small
+    // (a product that fills the GPU for a long time gains nothing from a neighbour), bf16 path only
+    bool small = dtype == MBD_BF16 && L > 1 && !getenv("MBD_NO_DW_OVERLAP");
+    size_t dw_elems = 0;
+    for (int i = 0; i < L && small; ++i) {
+      const Layer& l = n->layers[i];
+      if (2.0 * static_cast<double>(l.nW) * static_cast<double>(B) > 2e11) small = false;
+      if (l.bwd_weight.k_splits > 1) dw_elems = std::max(dw_elems, static_cast<size_t>(l.bwd_weight.k_splits) * l.nW);
+    }
+    n->overlap_dw = small;
+    if (small && dw_elems) ALLOC(n->partials_dw, dw_elems * sizeof(float));
+    n->last_dw_elems = dw_elems;
+  }
   ALLOC(n->colsum_scratch, static_cast<size_t>(8 * 32) * max_d * sizeof(float));
   ALLOC(n->per_sample, B * sizeof(float));
 #undef ALLOC
@@ -362,6 +396,12 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
               cudaEventCreateWithFlags(&n->ev_loss, cudaEventDisableTiming) == cudaSuccess;
     n->ev_fork.assign(L, nullptr);
     for (int i = 0; i < L && ok; ++i) ok = cudaEventCreateWithFlags(&n->ev_fork[i], cudaEventDisableTiming) == cudaSuccess;
+    if (ok && n->overlap_dw) {
+      ok = cudaStreamCreateWithFlags(&n->wstream, cudaStreamNonBlocking) == cudaSuccess &&
+           cudaEventCreateWithFlags(&n->ev_wjoin, cudaEventDisableTiming) == cudaSuccess;
+      n->ev_dx.assign(L, nullptr);
+      for (int i = 0; i < L && ok; ++i) ok = cudaEventCreateWithFlags(&n->ev_dx[i], cudaEventDisableTiming) == cudaSuccess;
+    }
     if (!ok) { free_net(n); return MBD_E_CUDA; }
   }
   if (cudaStreamSynchronize(n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
@@ -455,7 +495,7 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
   const int S_r = splits_for(n->P_r, n->max_partials), S_c = splits_for(n->P_c, n->max_partials);
   static const bool no_side = getenv("MBD_NO_SIDE") != nullptr;      // tuning knob: column sums on the main stream
   const bool side = n->aux != nullptr && !no_side;
-  bool forked = false;
+  bool forked = false, dw_forked = false;
   for (int i = n->L - 1; i >= 0; --i) {
     Layer& l = n->layers[i];
     if (l.bias) {
@@ -481,8 +521,22 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
       if (s != MBD_OK) return s;
     }
     const Epi e = fused ? epi_sgd(l.W, l.d_in, bf, scale) : epi_act(l.dW, l.d_in, 0, nullptr, 0);
-    mbd_status s = run_gemm(n, l.bwd_weight, 2, l.d_out, l.d_in, n->B, l.dY, l.d_out, layer_input(n, i), l.d_in, S_c, e);
+    cudaStream_t ws = nullptr;
+    if (n->overlap_dw) {
+      // dY_i is final and the last reader of the old W_i has been enqueued: dW_i may start beside
+      // the backward-data products of the layers below
+      CK(cudaEventRecord(n->ev_dx[i], n->stream));
+      CK(cudaStreamWaitEvent(n->wstream, n->ev_dx[i], 0));
+      ws = n->wstream;
+      dw_forked = true;
+    }
+    mbd_status s = run_gemm(n, l.bwd_weight, 2, l.d_out, l.d_in, n->B, l.dY, l.d_out, layer_input(n, i), l.d_in, S_c, e, ws,
+                            ws ? n->partials_dw : nullptr);
     if (s != MBD_OK) return s;
+  }
+  if (dw_forked) {
+    CK(cudaEventRecord(n->ev_wjoin, n->wstream));
+    CK(cudaStreamWaitEvent(n->stream, n->ev_wjoin, 0));
   }
   if (n->loss_pending) { forked = true; n->loss_pending = false; }
   if (forked) {
@@ -654,8 +708,8 @@ extern "C" mbd_status mbd_get_tensor(mbd_net* n, int which, int layer, void* dst
   if (which == MBD_T_LOSS) {
     src = n->per_sample; size = n->B * sizeof(float);
   } else if (which == MBD_T_PARTIALS) {
-    src = n->partials; size = bytes;
-    if (bytes > n->partial_elems * sizeof(float)) return MBD_E_INVALID;
+    src = n->last_red_dw ? n->partials_dw : n->partials; size = bytes;
+    if (bytes > (n->last_red_dw ? n->last_dw_elems : n->partial_elems) * sizeof(float)) return MBD_E_INVALID;
   } else {
     if (layer < 0 || layer >= n->L) return MBD_E_INVALID;
     Layer& l = n->layers[layer];
