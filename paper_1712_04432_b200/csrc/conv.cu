@@ -22,6 +22,8 @@
 //     row are three TMA boxes (the W coordinate of a box start is free); two shifted copies
 //     form one M = 128 operand; all nine taps accumulate in TMEM for the whole kernel and each
 //     CTA writes one fp32 partial, summed in CTA order (= strip order) by wgrad_finish.
+#include <stdlib.h>
+
 #include <new>
 #include <vector>
 
@@ -42,6 +44,13 @@ constexpr int FWD_STAGES = 3;         // ring of input rows: 3 shifted copies of
 constexpr int FWD_ROW_BYTES = 128 * 128;
 constexpr int FWD_W_BYTES = 3 * 192 * 128;   // stacked taps, 72 KB
 constexpr int FWD_SMEM = FWD_W_BYTES + FWD_STAGES * 3 * FWD_ROW_BYTES + 1024;
+// One-copy ring: a stage holds ONE box of 130 pixels (x0 - 1 .. x0 + 128); the three horizontally
+// shifted operands are views of it that start 0, 1 and 2 pixel rows (128 bytes each) into the box.
+constexpr int FWD1_BOX_PIX = FWD_PIX + 2;
+constexpr int FWD1_ROW_BYTES = 17 * 1024;     // 130 x 128 B = 16640 B, padded to the swizzle span
+constexpr int FWD1_STAGES = 8;
+constexpr int FWD_MAX_STAGES = 8;
+static_assert(FWD_W_BYTES + FWD1_STAGES * FWD1_ROW_BYTES + 1024 <= FWD_SMEM, "one-copy ring fits the same allocation");
 constexpr int FWD_THREADS = 320;      // producer warp, MMA warp, 8 epilogue warps
 constexpr int WG_PIX = 128;           // pixels (reduction length) per backward-weight block
 constexpr int WG_XSTAGES = 2;          // X rows: 3 shifted copies of 16 KB each, each row used once
@@ -192,6 +201,7 @@ wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ d
 struct FwdParams {
   int W, Hs, R, RB, nrb, nseg, n_items;
   int mode;
+  int one_copy;           // ring layout: 1 = one 130-pixel box per row, 0 = three shifted copies
   bf16* out;              // strips
   const bf16* mask_src;   // strips (MODE_MASK)
   float* loss_part;       // [gridDim.x * 8] (MODE_STORE_SSQ)
@@ -208,8 +218,8 @@ __device__ __forceinline__ int acc_block(int g) { return 7 - (g & 7); }
 __global__ void __launch_bounds__(FWD_THREADS, 1)
 conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const FwdParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[FWD_STAGES];
-  __shared__ __align__(8) uint64_t empty_bar[FWD_STAGES];
+  __shared__ __align__(8) uint64_t full_bar[FWD_MAX_STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[FWD_MAX_STAGES];
   __shared__ __align__(8) uint64_t acc_full_bar[8];
   __shared__ __align__(8) uint64_t acc_empty_bar[8];
   __shared__ __align__(8) uint64_t w_bar;
@@ -218,11 +228,12 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t w_smem = base;                         // 3 (v) x [192 rows (u, o) x 128 B]
-  const uint32_t ring = base + FWD_W_BYTES;             // slot = 3 shifted copies of one input row
+  const uint32_t ring = base + FWD_W_BYTES;             // slot = one input row (one box, or 3 shifted copies)
+  const int n_stages = p.one_copy ? FWD1_STAGES : FWD_STAGES;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < FWD_STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
+    for (int i = 0; i < FWD_MAX_STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
     for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&acc_full_bar[i]), 1); mbar_init(smem_u32(&acc_empty_bar[i]), 8); }
     mbar_init(smem_u32(&w_bar), 1);
     abort_flag = 0;
@@ -253,10 +264,15 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
           if (!ok) break;
           const uint32_t fb = smem_u32(&full_bar[stage]);
-          mbar_expect_tx(fb, 3 * FWD_ROW_BYTES);
-          for (int v = 0; v < 3; ++v)
-            tma_load_4d(ring + (stage * 3 + v) * FWD_ROW_BYTES, &tmX, 0, seg * FWD_PIX + v - 1, rb * p.RB + r, z, fb);
-          if (++stage == FWD_STAGES) { stage = 0; phase ^= 1u; }
+          if (p.one_copy) {
+            mbar_expect_tx(fb, FWD1_BOX_PIX * 128);
+            tma_load_4d(ring + stage * FWD1_ROW_BYTES, &tmX, 0, seg * FWD_PIX - 1, rb * p.RB + r, z, fb);
+          } else {
+            mbar_expect_tx(fb, 3 * FWD_ROW_BYTES);
+            for (int v = 0; v < 3; ++v)
+              tma_load_4d(ring + (stage * 3 + v) * FWD_ROW_BYTES, &tmX, 0, seg * FWD_PIX + v - 1, rb * p.RB + r, z, fb);
+          }
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
         }
       }
     }
@@ -277,7 +293,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           if (!ok) break;
           tc_fence_after();
           const int u_lo = max(0, r - (p.RB - 1)), u_hi = min(2, r);      // taps whose output row r - u exists
-          const uint32_t xa = ring + stage * 3 * FWD_ROW_BYTES;
+          const uint32_t xa = p.one_copy ? ring + stage * FWD1_ROW_BYTES : ring + stage * 3 * FWD_ROW_BYTES;
           int u_s = u_lo;
           while (u_s <= u_hi) {
             const int bs = acc_block(g0 + r - u_s);
@@ -287,7 +303,10 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             const uint32_t d_tmem = tmem_base + bs * 64;
 #pragma unroll
             for (int v = 0; v < 3; ++v) {
-              const uint64_t adesc = make_desc(xa + v * FWD_ROW_BYTES, 16, 1024);
+              // one-copy: the view shifted by v pixels starts v rows (128 bytes each) into the box.  The
+              // 128-byte swizzle is a function of the shared-memory address itself, so the rows of a view
+              // are read back exactly as TMA wrote them (checked: bit-identical to three shifted copies).
+              const uint64_t adesc = p.one_copy ? make_desc(xa + v * 128, 16, 1024) : make_desc(xa + v * FWD_ROW_BYTES, 16, 1024);
               const uint64_t bdesc = make_desc(w_smem + v * (192 * 128) + u_s * (64 * 128), 16, 1024);
 #pragma unroll
               for (int k = 0; k < 4; ++k) tc_mma_bf16(d_tmem, adesc + k * 2, bdesc + k * 2, idesc, 1u);
@@ -295,7 +314,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             u_s = u_e + 1;
           }
           tc_commit(smem_u32(&empty_bar[stage]));                           // the row is used only here
-          if (++stage == FWD_STAGES) { stage = 0; phase ^= 1u; }
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
           if (r >= 2) tc_commit(smem_u32(&acc_full_bar[acc_block(g0 + r - 2)]));   // output row r-2 is complete
         }
         g0 += p.RB;
@@ -642,6 +661,7 @@ struct ConvNet {
   float* loss_part = nullptr;
   bf16* scratch_nchw = nullptr;
   int fwd_RB = 1, wg_RB = 1;
+  int one_copy = 1;                   // ring layout of the forward kernel (tuning knob MBD_CONV_3COPY)
   int state = 0;                     // 0 idle, 1 forward done, 2 backward (gradients kept), 3 backward (fused)
 };
 
@@ -653,6 +673,7 @@ void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w
   p.nseg = (c->W + FWD_PIX - 1) / FWD_PIX;
   p.n_items = static_cast<int>(c->Z) * p.nrb * p.nseg;
   p.mode = mode; p.out = out; p.mask_src = mask; p.loss_part = c->loss_part; p.status = c->status;
+  p.one_copy = c->one_copy;
   const int grid = p.n_items < c->grid ? p.n_items : c->grid;
   if (mode == MODE_STORE_SSQ) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 8, c->stream);
   const double flops = 2.0 * c->B * c->H * c->W * 9.0 * C * C;
@@ -711,12 +732,14 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   ok = ok && alloc(reinterpret_cast<void**>(&c->loss_part), sizeof(float) * c->grid * 8);
   ok = ok && alloc(reinterpret_cast<void**>(&c->scratch_nchw), static_cast<size_t>(B) * C * H * W * 2);
   if (!ok) { conv_destroy(c); return MBD_E_ALLOC; }
+  c->one_copy = getenv("MBD_CONV_3COPY") ? 0 : 1;
+  const int fwd_box = c->one_copy ? FWD1_BOX_PIX : 128;
   c->act_fwd.resize(L + 1); c->act_wg.resize(L + 1); c->dY_fwd.resize(L); c->dY_wg.resize(L);
   c->wf_map.resize(L); c->wb_map.resize(L);
   for (int i = 0; i <= L && ok; ++i)
-    ok = make_strip_map(&c->act_fwd[i], c->act[i], W, c->R, c->Z, 128) && make_strip_map(&c->act_wg[i], c->act[i], W, c->R, c->Z, WG_PIX);
+    ok = make_strip_map(&c->act_fwd[i], c->act[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->act_wg[i], c->act[i], W, c->R, c->Z, WG_PIX);
   for (int i = 0; i < L && ok; ++i)
-    ok = make_strip_map(&c->dY_fwd[i], c->dY[i], W, c->R, c->Z, 128) && make_strip_map(&c->dY_wg[i], c->dY[i], W, c->R, c->Z, WG_PIX) &&
+    ok = make_strip_map(&c->dY_fwd[i], c->dY[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->dY_wg[i], c->dY[i], W, c->R, c->Z, WG_PIX) &&
          make_weight_map(&c->wf_map[i], c->Wf[i]) && make_weight_map(&c->wb_map[i], c->Wb[i]);
   if (!ok) { conv_destroy(c); return MBD_E_CUDA; }
   if (cudaStreamSynchronize(stream) != cudaSuccess) { conv_destroy(c); return MBD_E_CUDA; }
