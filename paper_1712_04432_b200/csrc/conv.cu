@@ -48,9 +48,13 @@ constexpr int FWD_SMEM = FWD_W_BYTES + FWD_STAGES * 3 * FWD_ROW_BYTES + 1024;
 // shifted operands are views of it that start 0, 1 and 2 pixel rows (128 bytes each) into the box.
 constexpr int FWD1_BOX_PIX = FWD_PIX + 2;
 constexpr int FWD1_ROW_BYTES = 17 * 1024;     // 130 x 128 B = 16640 B, padded to the swizzle span
-constexpr int FWD1_STAGES = 8;
-constexpr int FWD_MAX_STAGES = 8;
-static_assert(FWD_W_BYTES + FWD1_STAGES * FWD1_ROW_BYTES + 1024 <= FWD_SMEM, "one-copy ring fits the same allocation");
+constexpr int FWD1_STAGES = 4;
+constexpr int FWD_MAX_STAGES = 4;
+// ... and, behind the ring, two staging tiles of one output row segment each ([128 pixels][64 channels]
+// bf16, 16 KB, 128B-swizzled like the strips' tensor maps) for TMA stores, and two for the rows of the
+// mask source that the backward-data mode reads: the epilogue's global traffic goes through TMA.
+constexpr int FWD_TILE_BYTES = FWD_PIX * 128;
+static_assert(FWD_W_BYTES + FWD1_STAGES * FWD1_ROW_BYTES + 4 * FWD_TILE_BYTES + 1024 <= FWD_SMEM, "one-copy layout fits the same allocation");
 constexpr int FWD_THREADS = 320;      // producer warp, MMA warp, 8 epilogue warps
 constexpr int WG_PIX = 128;           // pixels (reduction length) per backward-weight block
 constexpr int WG_XSTAGES = 2;          // X rows: 3 shifted copies of 16 KB each, each row used once
@@ -216,13 +220,15 @@ struct FwdParams {
 __device__ __forceinline__ int acc_block(int g) { return 7 - (g & 7); }
 
 __global__ void __launch_bounds__(FWD_THREADS, 1)
-conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const FwdParams p) {
+conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
+                const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmMask, const FwdParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[FWD_MAX_STAGES];
   __shared__ __align__(8) uint64_t empty_bar[FWD_MAX_STAGES];
   __shared__ __align__(8) uint64_t acc_full_bar[8];
   __shared__ __align__(8) uint64_t acc_empty_bar[8];
   __shared__ __align__(8) uint64_t w_bar;
+  __shared__ __align__(8) uint64_t mask_full_bar[2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
@@ -236,6 +242,8 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     for (int i = 0; i < FWD_MAX_STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
     for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&acc_full_bar[i]), 1); mbar_init(smem_u32(&acc_empty_bar[i]), 8); }
     mbar_init(smem_u32(&w_bar), 1);
+    mbar_init(smem_u32(&mask_full_bar[0]), 1);
+    mbar_init(smem_u32(&mask_full_bar[1]), 1);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -342,6 +350,119 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     int g = 0;
     float ssq = 0.f;
     bool ok = true;
+    if (p.one_copy) {
+      // ---- TMA epilogue.  The eight warps fill one staging tile per output row segment (a thread owns
+      // 32 channels of one pixel: four 16-byte cells of that pixel's 128-byte row, at the cell positions of
+      // the 128-byte swizzle), one thread stores the tile with TMA; the mask source of the backward-data
+      // mode arrives the same way, two rows ahead.  The LSU never touches global memory (32 sectors per
+      // instruction made it the bottleneck of this kernel).
+      const uint32_t stg_out = ring + FWD1_STAGES * FWD1_ROW_BYTES;
+      const uint32_t stg_mask = stg_out + 2 * FWD_TILE_BYTES;
+      uint8_t* out_gen = smem_raw + (stg_out - smem_u32(smem_raw));
+      const uint8_t* mask_gen = smem_raw + (stg_mask - smem_u32(smem_raw));
+      const bool use_mask = p.mode == MODE_MASK && p.mask_src != nullptr;
+      const bool issuer = warp == 2 && lane == 0;
+      const int n_rows = (i1 - i0) * p.RB;
+      auto row_coords = [&](int k, int& x0, int& row, int& z) {
+        const int it = i0 + k / p.RB, i = k % p.RB;
+        const int seg = it % p.nseg, rb = (it / p.nseg) % p.nrb;
+        z = it / (p.nseg * p.nrb);
+        x0 = seg * FWD_PIX;
+        row = rb * p.RB + i + 1;
+      };
+      auto load_mask = [&](int k) {
+        int x0, row, z;
+        row_coords(k, x0, row, z);
+        const uint32_t mb = smem_u32(&mask_full_bar[k & 1]);
+        mbar_expect_tx(mb, FWD_TILE_BYTES);
+        tma_load_4d(stg_mask + (k & 1) * FWD_TILE_BYTES, &tmMask, 0, x0, row, z, mb);
+      };
+      if (use_mask && issuer) {
+        if (n_rows > 0) load_mask(0);
+        if (n_rows > 1) load_mask(1);
+      }
+      const int cell0 = half * 4;                         // first 16-byte cell of this thread's channels
+      for (; g < n_rows; ++g) {
+        const int buf = g & 1;
+        int x0, row, z;
+        row_coords(g, x0, row, z);
+        const bool valid = x0 + pl < p.W;
+        const int blk = acc_block(g);
+        if (issuer) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store of row g - 2 has read this tile
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        ok = mbar_wait(smem_u32(&acc_full_bar[blk]), (g >> 3) & 1u, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+        if (ok && use_mask) ok = mbar_wait(smem_u32(&mask_full_bar[buf]), (g >> 1) & 1u, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+          tc_fence_after();
+          uint32_t d[32];
+          tc_ld32(lane_base + blk * 64, d);
+          tc_wait_ld();
+          asm volatile(
+              "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+              "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
+              "%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+              ::"r"(lane_base + blk * 64), "r"(0u) : "memory");
+          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&acc_empty_bar[blk]));
+          float y[32];
+#pragma unroll
+          for (int c = 0; c < 32; ++c) y[c] = __uint_as_float(d[c]);
+          if (p.mode == MODE_RELU_STORE) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) y[c] = fmaxf(y[c], 0.f);
+          } else if (p.mode == MODE_STORE_SSQ) {
+            if (valid) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) ssq = fmaf(y[c], y[c], ssq);
+            }
+          } else if (use_mask) {
+            const uint8_t* mrow = mask_gen + buf * FWD_TILE_BYTES + pl * 128;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint4 mq = *reinterpret_cast<const uint4*>(mrow + (((cell0 + j) ^ (pl & 7)) << 4));
+              const uint32_t mw[4] = {mq.x, mq.y, mq.z, mq.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                if (!(bf16_bits_to_f32(mw[e] & 0xFFFFu) > 0.f)) y[j * 8 + 2 * e] = 0.f;
+                if (!(bf16_bits_to_f32(mw[e] >> 16) > 0.f)) y[j * 8 + 2 * e + 1] = 0.f;
+              }
+            }
+          }
+          uint8_t* orow = out_gen + buf * FWD_TILE_BYTES + pl * 128;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint4 o;
+            o.x = pack_bf16x2(y[j * 8 + 0], y[j * 8 + 1]); o.y = pack_bf16x2(y[j * 8 + 2], y[j * 8 + 3]);
+            o.z = pack_bf16x2(y[j * 8 + 4], y[j * 8 + 5]); o.w = pack_bf16x2(y[j * 8 + 6], y[j * 8 + 7]);
+            *reinterpret_cast<uint4*>(orow + (((cell0 + j) ^ (pl & 7)) << 4)) = o;
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // tile written (and mask tile read) before TMA touches them
+        {   // the eight warps meet here: either all of them go on or none does
+          int all_ok;
+          asm volatile(
+              "{\n\t.reg .pred pp, qq;\n\t"
+              "setp.ne.b32 pp, %1, 0;\n\t"
+              "bar.red.and.pred qq, 1, 256, pp;\n\t"
+              "selp.b32 %0, 1, 0, qq;\n\t}"
+              : "=r"(all_ok) : "r"(static_cast<int>(ok)) : "memory");
+          ok = all_ok != 0;
+        }
+        if (!ok) break;
+        if (issuer) {
+          asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+                       ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(row), "r"(z),
+                         "r"(stg_out + buf * FWD_TILE_BYTES)
+                       : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          if (use_mask && g + 2 < n_rows) load_mask(g + 2);
+        }
+      }
+      if (issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // stores done before the CTA exits
+    } else
     for (int it = i0; it < i1 && ok; ++it) {
       const int seg = it % p.nseg, rb = (it / p.nseg) % p.nrb, z = it / (p.nseg * p.nrb);
       const int x = seg * FWD_PIX + pl;
@@ -657,6 +778,7 @@ struct ConvNet {
   std::vector<float*> dK;
   std::vector<int> relu;
   std::vector<CUtensorMap> act_fwd, act_wg, dY_fwd, dY_wg, wf_map, wb_map;
+  std::vector<CUtensorMap> act_tile, dY_tile;     // [128 pixels][64 channels] boxes: TMA stores of outputs, mask rows
   float* wpart = nullptr;
   float* loss_part = nullptr;
   bf16* scratch_nchw = nullptr;
@@ -667,7 +789,8 @@ struct ConvNet {
 
 namespace {
 
-void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w, bf16* out, int mode, const bf16* mask) {
+void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w, bf16* out, const CUtensorMap& out_tile, int mode,
+                const bf16* mask, const CUtensorMap* mask_tile) {
   FwdParams p;
   p.W = c->W; p.Hs = c->Hs; p.R = c->R; p.RB = c->fwd_RB; p.nrb = c->Hs / c->fwd_RB;
   p.nseg = (c->W + FWD_PIX - 1) / FWD_PIX;
@@ -678,7 +801,7 @@ void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w
   if (mode == MODE_STORE_SSQ) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 8, c->stream);
   const double flops = 2.0 * c->B * c->H * c->W * 9.0 * C * C;
   c->prof->begin(cls, flops);
-  launch_pdl(conv_fwd_kernel, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, p);
+  launch_pdl(conv_fwd_kernel, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, out_tile, mask_tile ? *mask_tile : out_tile, p);
   c->prof->end();
 }
 
@@ -735,11 +858,14 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   c->one_copy = getenv("MBD_CONV_3COPY") ? 0 : 1;
   const int fwd_box = c->one_copy ? FWD1_BOX_PIX : 128;
   c->act_fwd.resize(L + 1); c->act_wg.resize(L + 1); c->dY_fwd.resize(L); c->dY_wg.resize(L);
+  c->act_tile.resize(L + 1); c->dY_tile.resize(L);
   c->wf_map.resize(L); c->wb_map.resize(L);
   for (int i = 0; i <= L && ok; ++i)
-    ok = make_strip_map(&c->act_fwd[i], c->act[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->act_wg[i], c->act[i], W, c->R, c->Z, WG_PIX);
+    ok = make_strip_map(&c->act_fwd[i], c->act[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->act_wg[i], c->act[i], W, c->R, c->Z, WG_PIX) &&
+         make_strip_map(&c->act_tile[i], c->act[i], W, c->R, c->Z, FWD_PIX);
   for (int i = 0; i < L && ok; ++i)
     ok = make_strip_map(&c->dY_fwd[i], c->dY[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->dY_wg[i], c->dY[i], W, c->R, c->Z, WG_PIX) &&
+         make_strip_map(&c->dY_tile[i], c->dY[i], W, c->R, c->Z, FWD_PIX) &&
          make_weight_map(&c->wf_map[i], c->Wf[i]) && make_weight_map(&c->wb_map[i], c->Wb[i]);
   if (!ok) { conv_destroy(c); return MBD_E_CUDA; }
   if (cudaStreamSynchronize(stream) != cudaSuccess) { conv_destroy(c); return MBD_E_CUDA; }
@@ -780,8 +906,8 @@ mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
   for (int i = 0; i < c->L; ++i) {
     const bool last = i == c->L - 1;
     if (i > 0) launch_halo(c, c->act[i]);            // forward halo exchange (first halo term of Eq. 7)
-    launch_fwd(c, MBD_K_CONV_FWD, c->act_fwd[i], c->wf_map[i], c->act[i + 1],
-               last ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK), nullptr);
+    launch_fwd(c, MBD_K_CONV_FWD, c->act_fwd[i], c->wf_map[i], c->act[i + 1], c->act_tile[i + 1],
+               last ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK), nullptr, nullptr);
   }
   if (loss_sum_dev) {
     c->prof->begin(MBD_K_OTHER, c->grid * 32.0);
@@ -800,8 +926,8 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
     if (i > 0) {
       // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0]
       launch_halo(c, c->dY[i]);
-      launch_fwd(c, MBD_K_CONV_BWD_DATA, c->dY_fwd[i], c->wb_map[i], c->dY[i - 1], MODE_MASK,
-                 c->relu[i - 1] ? c->act[i] : nullptr);
+      launch_fwd(c, MBD_K_CONV_BWD_DATA, c->dY_fwd[i], c->wb_map[i], c->dY[i - 1], c->dY_tile[i - 1], MODE_MASK,
+                 c->relu[i - 1] ? c->act[i] : nullptr, c->relu[i - 1] ? &c->act_tile[i] : nullptr);
     }
     WgParams p;
     p.W = c->W; p.Hs = c->Hs; p.R = c->R; p.RB = c->wg_RB; p.nrb = c->Hs / c->wg_RB;
