@@ -40,21 +40,18 @@ namespace {
 
 constexpr int C = 64;                 // channels in and out
 constexpr int FWD_PIX = 128;          // output pixels per forward tile (one per TMEM lane)
-constexpr int FWD_STAGES = 3;         // ring of input rows: 3 shifted copies of 16 KB each; a row is used once
-constexpr int FWD_ROW_BYTES = 128 * 128;
 constexpr int FWD_W_BYTES = 3 * 192 * 128;   // stacked taps, 72 KB
-constexpr int FWD_SMEM = FWD_W_BYTES + FWD_STAGES * 3 * FWD_ROW_BYTES + 1024;
-// One-copy ring: a stage holds ONE box of 130 pixels (x0 - 1 .. x0 + 128); the three horizontally
-// shifted operands are views of it that start 0, 1 and 2 pixel rows (128 bytes each) into the box.
+// Ring of input rows: a stage holds ONE box of 130 pixels (x0 - 1 .. x0 + 128) of one row; the three
+// horizontally shifted operands are views of it that start 0, 1 and 2 pixel rows (128 bytes each) into the box.
 constexpr int FWD1_BOX_PIX = FWD_PIX + 2;
 constexpr int FWD1_ROW_BYTES = 17 * 1024;     // 130 x 128 B = 16640 B, padded to the swizzle span
-constexpr int FWD1_STAGES = 4;
-constexpr int FWD_MAX_STAGES = 4;
-// ... and, behind the ring, two staging tiles of one output row segment each ([128 pixels][64 channels]
-// bf16, 16 KB, 128B-swizzled like the strips' tensor maps) for TMA stores, and two for the rows of the
-// mask source that the backward-data mode reads: the epilogue's global traffic goes through TMA.
+constexpr int FWD1_STAGES = 5;
+// Behind the ring: two staging tiles of one output row segment each ([128 pixels][64 channels] bf16, 16 KB,
+// 128B-swizzled like the strips' tensor maps) for TMA stores, and two for the rows of the mask source that
+// the backward-data mode reads: the epilogue's global traffic goes through TMA.
 constexpr int FWD_TILE_BYTES = FWD_PIX * 128;
-static_assert(FWD_W_BYTES + FWD1_STAGES * FWD1_ROW_BYTES + 4 * FWD_TILE_BYTES + 1024 <= FWD_SMEM, "one-copy layout fits the same allocation");
+constexpr int FWD_SMEM = FWD_W_BYTES + FWD1_STAGES * FWD1_ROW_BYTES + 4 * FWD_TILE_BYTES + 1024;
+static_assert(FWD_SMEM <= 227 * 1024, "forward kernel's shared memory");
 constexpr int FWD_THREADS = 320;      // producer warp, MMA warp, 8 epilogue warps
 constexpr int WG_PIX = 128;           // pixels (reduction length) per backward-weight block
 constexpr int WG_XSTAGES = 2;          // X rows: 3 shifted copies of 16 KB each, each row used once
@@ -203,14 +200,30 @@ wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ d
 
 // ------------------------------------------------------------------------------ forward kernel
 struct FwdParams {
-  int W, Hs, R, RB, nrb, nseg, n_items;
+  int W, Hs, R, nseg;
+  long long rows_total;   // output row segments: (strip z, segment, row) flattened with the row fastest
   int mode;
-  int one_copy;           // ring layout: 1 = one 130-pixel box per row, 0 = three shifted copies
   bf16* out;              // strips
   const bf16* mask_src;   // strips (MODE_MASK)
   float* loss_part;       // [gridDim.x * 8] (MODE_STORE_SSQ)
   int* status;
 };
+
+// A CTA owns a contiguous span of the flattened output rows and walks it as runs of rows of one
+// (strip, segment) column; a run of n output rows reads n + 2 input rows.
+struct FwdRun {
+  int z, seg, h0, n;
+};
+__device__ __forceinline__ FwdRun fwd_run(const FwdParams& p, long long pos, long long end) {
+  const long long col = pos / p.Hs;
+  FwdRun r;
+  r.h0 = static_cast<int>(pos - col * p.Hs);
+  const long long left = end - pos;
+  r.n = static_cast<int>(left < p.Hs - r.h0 ? left : p.Hs - r.h0);
+  r.seg = static_cast<int>(col % p.nseg);
+  r.z = static_cast<int>(col / p.nseg);
+  return r;
+}
 
 // TMEM holds a ring of eight 64-column accumulators, one per output row in flight; output
 // row g uses block 7 - (g mod 8), so that the rows r, r-1, r-2 fed by input row r sit in
@@ -223,8 +236,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 1)
 conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
                 const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmMask, const FwdParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[FWD_MAX_STAGES];
-  __shared__ __align__(8) uint64_t empty_bar[FWD_MAX_STAGES];
+  __shared__ __align__(8) uint64_t full_bar[FWD1_STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[FWD1_STAGES];
   __shared__ __align__(8) uint64_t acc_full_bar[8];
   __shared__ __align__(8) uint64_t acc_empty_bar[8];
   __shared__ __align__(8) uint64_t w_bar;
@@ -235,11 +248,10 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t w_smem = base;                         // 3 (v) x [192 rows (u, o) x 128 B]
   const uint32_t ring = base + FWD_W_BYTES;             // slot = one input row (one box, or 3 shifted copies)
-  const int n_stages = p.one_copy ? FWD1_STAGES : FWD_STAGES;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < FWD_MAX_STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
+    for (int i = 0; i < FWD1_STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
     for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&acc_full_bar[i]), 1); mbar_init(smem_u32(&acc_empty_bar[i]), 8); }
     mbar_init(smem_u32(&w_bar), 1);
     mbar_init(smem_u32(&mask_full_bar[0]), 1);
@@ -256,8 +268,8 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   pdl_trigger();                           // set-up done: the next kernel may be scheduled
   pdl_wait();                              // from here on global memory: earlier kernels must have finished
 
-  const int i0 = static_cast<int>((static_cast<long long>(blockIdx.x) * p.n_items) / gridDim.x);
-  const int i1 = static_cast<int>((static_cast<long long>(blockIdx.x + 1) * p.n_items) / gridDim.x);
+  const long long r0 = (static_cast<long long>(blockIdx.x) * p.rows_total) / gridDim.x;
+  const long long r1 = (static_cast<long long>(blockIdx.x + 1) * p.rows_total) / gridDim.x;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -266,22 +278,17 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int it = i0; it < i1 && ok; ++it) {
-        const int seg = it % p.nseg, rb = (it / p.nseg) % p.nrb, z = it / (p.nseg * p.nrb);
-        for (int r = 0; r < p.RB + 2; ++r) {
+      for (long long pos = r0; pos < r1 && ok;) {
+        const FwdRun run = fwd_run(p, pos, r1);
+        for (int r = 0; r < run.n + 2; ++r) {
           ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
           if (!ok) break;
           const uint32_t fb = smem_u32(&full_bar[stage]);
-          if (p.one_copy) {
-            mbar_expect_tx(fb, FWD1_BOX_PIX * 128);
-            tma_load_4d(ring + stage * FWD1_ROW_BYTES, &tmX, 0, seg * FWD_PIX - 1, rb * p.RB + r, z, fb);
-          } else {
-            mbar_expect_tx(fb, 3 * FWD_ROW_BYTES);
-            for (int v = 0; v < 3; ++v)
-              tma_load_4d(ring + (stage * 3 + v) * FWD_ROW_BYTES, &tmX, 0, seg * FWD_PIX + v - 1, rb * p.RB + r, z, fb);
-          }
-          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+          mbar_expect_tx(fb, FWD1_BOX_PIX * 128);
+          tma_load_4d(ring + stage * FWD1_ROW_BYTES, &tmX, 0, run.seg * FWD_PIX - 1, run.h0 + r, run.z, fb);
+          if (++stage == FWD1_STAGES) { stage = 0; phase ^= 1u; }
         }
+        pos += run.n;
       }
     }
   } else if (warp == 1) {
@@ -289,10 +296,11 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       bool ok = mbar_wait(smem_u32(&w_bar), 0, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
       int stage = 0;
       uint32_t phase = 0;
-      int g0 = 0;              // output rows of earlier items of this CTA
-      for (int it = i0; it < i1 && ok; ++it) {
-        for (int r = 0; r < p.RB + 2 && ok; ++r) {
-          if (r < p.RB) {      // this input row opens output row r: its block must be drained and zeroed
+      int g0 = 0;              // output rows of earlier runs of this CTA
+      for (long long pos = r0; pos < r1 && ok;) {
+        const FwdRun run = fwd_run(p, pos, r1);
+        for (int r = 0; r < run.n + 2 && ok; ++r) {
+          if (r < run.n) {     // this input row opens output row r: its block must be drained and zeroed
             const int g = g0 + r;
             ok = mbar_wait(smem_u32(&acc_empty_bar[acc_block(g)]), (g >> 3) & 1u, abortp, p.status, DEV_TIMEOUT_MMA_TMEM);
             if (!ok) break;
@@ -300,8 +308,8 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           ok = mbar_wait(smem_u32(&full_bar[stage]), phase, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
           if (!ok) break;
           tc_fence_after();
-          const int u_lo = max(0, r - (p.RB - 1)), u_hi = min(2, r);      // taps whose output row r - u exists
-          const uint32_t xa = p.one_copy ? ring + stage * FWD1_ROW_BYTES : ring + stage * 3 * FWD_ROW_BYTES;
+          const int u_lo = max(0, r - (run.n - 1)), u_hi = min(2, r);     // taps whose output row r - u exists
+          const uint32_t xa = ring + stage * FWD1_ROW_BYTES;
           int u_s = u_lo;
           while (u_s <= u_hi) {
             const int bs = acc_block(g0 + r - u_s);
@@ -311,10 +319,10 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             const uint32_t d_tmem = tmem_base + bs * 64;
 #pragma unroll
             for (int v = 0; v < 3; ++v) {
-              // one-copy: the view shifted by v pixels starts v rows (128 bytes each) into the box.  The
-              // 128-byte swizzle is a function of the shared-memory address itself, so the rows of a view
-              // are read back exactly as TMA wrote them (checked: bit-identical to three shifted copies).
-              const uint64_t adesc = p.one_copy ? make_desc(xa + v * 128, 16, 1024) : make_desc(xa + v * FWD_ROW_BYTES, 16, 1024);
+              // The view shifted by v pixels starts v rows (128 bytes each) into the box.  The 128-byte
+              // swizzle is a function of the shared-memory address itself, so the rows of a view are read
+              // back exactly as TMA wrote them (checked: bit-identical to three separately loaded copies).
+              const uint64_t adesc = make_desc(xa + v * 128, 16, 1024);
               const uint64_t bdesc = make_desc(w_smem + v * (192 * 128) + u_s * (64 * 128), 16, 1024);
 #pragma unroll
               for (int k = 0; k < 4; ++k) tc_mma_bf16(d_tmem, adesc + k * 2, bdesc + k * 2, idesc, 1u);
@@ -322,10 +330,11 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             u_s = u_e + 1;
           }
           tc_commit(smem_u32(&empty_bar[stage]));                           // the row is used only here
-          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+          if (++stage == FWD1_STAGES) { stage = 0; phase ^= 1u; }
           if (r >= 2) tc_commit(smem_u32(&acc_full_bar[acc_block(g0 + r - 2)]));   // output row r-2 is complete
         }
-        g0 += p.RB;
+        g0 += run.n;
+        pos += run.n;
       }
     }
   } else {
@@ -350,7 +359,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     int g = 0;
     float ssq = 0.f;
     bool ok = true;
-    if (p.one_copy) {
+    {
       // ---- TMA epilogue.  The eight warps fill one staging tile per output row segment (a thread owns
       // 32 channels of one pixel: four 16-byte cells of that pixel's 128-byte row, at the cell positions of
       // the 128-byte swizzle), one thread stores the tile with TMA; the mask source of the backward-data
@@ -362,13 +371,13 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       const uint8_t* mask_gen = smem_raw + (stg_mask - smem_u32(smem_raw));
       const bool use_mask = p.mode == MODE_MASK && p.mask_src != nullptr;
       const bool issuer = warp == 2 && lane == 0;
-      const int n_rows = (i1 - i0) * p.RB;
+      const int n_rows = static_cast<int>(r1 - r0);
       auto row_coords = [&](int k, int& x0, int& row, int& z) {
-        const int it = i0 + k / p.RB, i = k % p.RB;
-        const int seg = it % p.nseg, rb = (it / p.nseg) % p.nrb;
-        z = it / (p.nseg * p.nrb);
-        x0 = seg * FWD_PIX;
-        row = rb * p.RB + i + 1;
+        const long long pos = r0 + k;
+        const long long col = pos / p.Hs;
+        z = static_cast<int>(col / p.nseg);
+        x0 = static_cast<int>(col % p.nseg) * FWD_PIX;
+        row = static_cast<int>(pos - col * p.Hs) + 1;
       };
       auto load_mask = [&](int k) {
         int x0, row, z;
@@ -462,69 +471,6 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         }
       }
       if (issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // stores done before the CTA exits
-    } else
-    for (int it = i0; it < i1 && ok; ++it) {
-      const int seg = it % p.nseg, rb = (it / p.nseg) % p.nrb, z = it / (p.nseg * p.nrb);
-      const int x = seg * FWD_PIX + pl;
-      const bool valid = x < p.W;
-      for (int i = 0; i < p.RB; ++i, ++g) {
-        const int blk = acc_block(g);
-        const int64_t opix = ((static_cast<int64_t>(z) * p.R + rb * p.RB + i + 1) * p.W + x) * C + half * 32;
-        uint4 mpre[4];
-        const bool use_mask = p.mode == MODE_MASK && p.mask_src != nullptr;
-        if (use_mask && valid) {                           // requested before the accumulator is ready
-          const uint4* m4 = reinterpret_cast<const uint4*>(p.mask_src + opix);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) mpre[j] = m4[j];
-        }
-        ok = mbar_wait(smem_u32(&acc_full_bar[blk]), (g >> 3) & 1u, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t d[32];
-        tc_ld32(lane_base + blk * 64, d);
-        tc_wait_ld();
-        asm volatile(
-            "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-            "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
-            "%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
-            ::"r"(lane_base + blk * 64), "r"(0u) : "memory");
-        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&acc_empty_bar[blk]));
-        if (valid) {
-          float y[32];
-#pragma unroll
-          for (int c = 0; c < 32; ++c) y[c] = __uint_as_float(d[c]);
-          if (p.mode == MODE_RELU_STORE) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) y[c] = fmaxf(y[c], 0.f);
-          } else if (p.mode == MODE_STORE_SSQ) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) ssq = fmaf(y[c], y[c], ssq);
-          } else if (use_mask) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const uint4 mq = mpre[j];
-              const uint32_t mw[4] = {mq.x, mq.y, mq.z, mq.w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                if (!(bf16_bits_to_f32(mw[e] & 0xFFFFu) > 0.f)) y[j * 8 + 2 * e] = 0.f;
-                if (!(bf16_bits_to_f32(mw[e] >> 16) > 0.f)) y[j * 8 + 2 * e + 1] = 0.f;
-              }
-            }
-          }
-          uint4* o4 = reinterpret_cast<uint4*>(p.out + opix);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint4 o;
-            o.x = pack_bf16x2(y[j * 8 + 0], y[j * 8 + 1]); o.y = pack_bf16x2(y[j * 8 + 2], y[j * 8 + 3]);
-            o.z = pack_bf16x2(y[j * 8 + 4], y[j * 8 + 5]); o.w = pack_bf16x2(y[j * 8 + 6], y[j * 8 + 7]);
-            o4[j] = o;
-          }
-        }
-      }
     }
     if (p.mode == MODE_STORE_SSQ) {
 #pragma unroll
@@ -782,8 +728,7 @@ struct ConvNet {
   float* wpart = nullptr;
   float* loss_part = nullptr;
   bf16* scratch_nchw = nullptr;
-  int fwd_RB = 1, wg_RB = 1;
-  int one_copy = 1;                   // ring layout of the forward kernel (tuning knob MBD_CONV_3COPY)
+  int wg_RB = 1;
   int state = 0;                     // 0 idle, 1 forward done, 2 backward (gradients kept), 3 backward (fused)
 };
 
@@ -792,12 +737,11 @@ namespace {
 void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w, bf16* out, const CUtensorMap& out_tile, int mode,
                 const bf16* mask, const CUtensorMap* mask_tile) {
   FwdParams p;
-  p.W = c->W; p.Hs = c->Hs; p.R = c->R; p.RB = c->fwd_RB; p.nrb = c->Hs / c->fwd_RB;
+  p.W = c->W; p.Hs = c->Hs; p.R = c->R;
   p.nseg = (c->W + FWD_PIX - 1) / FWD_PIX;
-  p.n_items = static_cast<int>(c->Z) * p.nrb * p.nseg;
+  p.rows_total = static_cast<long long>(c->Z) * p.nseg * c->Hs;
   p.mode = mode; p.out = out; p.mask_src = mask; p.loss_part = c->loss_part; p.status = c->status;
-  p.one_copy = c->one_copy;
-  const int grid = p.n_items < c->grid ? p.n_items : c->grid;
+  const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
   if (mode == MODE_STORE_SSQ) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 8, c->stream);
   const double flops = 2.0 * c->B * c->H * c->W * 9.0 * C * C;
   c->prof->begin(cls, flops);
@@ -833,7 +777,6 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   c->L = L; c->B = B; c->H = H; c->W = W; c->P_r = P_r; c->Hs = H / P_r; c->R = c->Hs + 2; c->Z = B * P_r;
   c->num_sms = num_sms; c->grid = num_sms; c->status = status; c->stream = stream; c->prof = prof;
   c->strip_elems = static_cast<size_t>(c->Z) * c->R * W * C;
-  c->fwd_RB = largest_divisor_at_most(c->Hs, 14);
   c->wg_RB = largest_divisor_at_most(c->Hs, 14);
   auto alloc = [&](void** p, size_t bytes) -> bool {
     if (cudaMalloc(p, bytes) != cudaSuccess) { (void)cudaGetLastError(); *p = nullptr; return false; }
@@ -855,8 +798,7 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   ok = ok && alloc(reinterpret_cast<void**>(&c->loss_part), sizeof(float) * c->grid * 8);
   ok = ok && alloc(reinterpret_cast<void**>(&c->scratch_nchw), static_cast<size_t>(B) * C * H * W * 2);
   if (!ok) { conv_destroy(c); return MBD_E_ALLOC; }
-  c->one_copy = getenv("MBD_CONV_3COPY") ? 0 : 1;
-  const int fwd_box = c->one_copy ? FWD1_BOX_PIX : 128;
+  const int fwd_box = FWD1_BOX_PIX;
   c->act_fwd.resize(L + 1); c->act_wg.resize(L + 1); c->dY_fwd.resize(L); c->dY_wg.resize(L);
   c->act_tile.resize(L + 1); c->dY_tile.resize(L);
   c->wf_map.resize(L); c->wb_map.resize(L);
