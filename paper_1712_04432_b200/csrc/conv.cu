@@ -490,10 +490,27 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 
 // ------------------------------------------------------------------------------ backward-weight kernel
 struct WgParams {
-  int W, Hs, R, RB, nrb, nseg, n_items;
+  int W, Hs, R, nseg;
+  long long rows_total;   // dY row segments: (strip z, segment, row) flattened with the row fastest
   float* part;            // [gridDim.x][9][C][C]
   int* status;
 };
+
+// As in the forward kernel a CTA owns a contiguous span of the flattened rows and walks it as runs
+// of rows of one (strip, segment) column; a run of n dY rows meets n + 2 X rows.
+struct WgRun {
+  int z, seg, h0, n;
+};
+__device__ __forceinline__ WgRun wg_run(const WgParams& p, long long pos, long long end) {
+  const long long col = pos / p.Hs;
+  WgRun r;
+  r.h0 = static_cast<int>(pos - col * p.Hs);
+  const long long left = end - pos;
+  r.n = static_cast<int>(left < p.Hs - r.h0 ? left : p.Hs - r.h0);
+  r.seg = static_cast<int>(col % p.nseg);
+  r.z = static_cast<int>(col / p.nseg);
+  return r;
+}
 
 // One X row (three shifted copies) meets the up to three dY rows it contributes to in ONE
 // instruction group: B = [dY_{r-2} | dY_{r-1} | dY_r] (N = 64 per row, rows adjacent in the dY
@@ -530,26 +547,28 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   pdl_trigger();                           // set-up done: the next kernel may be scheduled
   pdl_wait();                              // from here on global memory: earlier kernels must have finished
 
-  const int i0 = static_cast<int>((static_cast<long long>(blockIdx.x) * p.n_items) / gridDim.x);
-  const int i1 = static_cast<int>((static_cast<long long>(blockIdx.x + 1) * p.n_items) / gridDim.x);
+  const long long r0 = (static_cast<long long>(blockIdx.x) * p.rows_total) / gridDim.x;
+  const long long r1 = (static_cast<long long>(blockIdx.x + 1) * p.rows_total) / gridDim.x;
 
   if (warp == 0) {
     if (lane == 0) {
       int xs = 0, ys = 0;
       uint32_t xph = 0, yph = 0;
       bool ok = true;
-      for (int it = i0; it < i1 && ok; ++it) {
-        const int seg = it % p.nseg, rb = (it / p.nseg) % p.nrb, z = it / (p.nseg * p.nrb);
-        const int x0 = seg * WG_PIX;
-        for (int r = 0; r < p.RB + 2 && ok; ++r) {
-          if (r < p.RB) {
+      for (long long pos = r0; pos < r1 && ok;) {
+        const WgRun run = wg_run(p, pos, r1);
+        pos += run.n;
+        const int z = run.z;
+        const int x0 = run.seg * WG_PIX;
+        for (int r = 0; r < run.n + 2 && ok; ++r) {
+          if (r < run.n) {
             ok = mbar_wait(smem_u32(&yempty[ys]), yph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
             if (!ok) break;
             const uint32_t fy = smem_u32(&yfull[ys]);
             const bool mirrored = ys < 2;
             mbar_expect_tx(fy, mirrored ? 2 * WG_CHUNK : WG_CHUNK);
-            tma_load_4d(yring + ys * WG_CHUNK, &tmY, 0, x0, rb * p.RB + r + 1, z, fy);
-            if (mirrored) tma_load_4d(yring + (WG_YSTAGES + ys) * WG_CHUNK, &tmY, 0, x0, rb * p.RB + r + 1, z, fy);
+            tma_load_4d(yring + ys * WG_CHUNK, &tmY, 0, x0, run.h0 + r + 1, z, fy);
+            if (mirrored) tma_load_4d(yring + (WG_YSTAGES + ys) * WG_CHUNK, &tmY, 0, x0, run.h0 + r + 1, z, fy);
             if (++ys == WG_YSTAGES) { ys = 0; yph ^= 1u; }
           }
           ok = mbar_wait(smem_u32(&xempty[xs]), xph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
@@ -557,7 +576,7 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           const uint32_t fb = smem_u32(&xfull[xs]);
           mbar_expect_tx(fb, 3 * WG_CHUNK);
           for (int v = 0; v < 3; ++v)
-            tma_load_4d(xring + (xs * 3 + v) * WG_CHUNK, &tmX, 0, x0 + v - 1, rb * p.RB + r, z, fb);
+            tma_load_4d(xring + (xs * 3 + v) * WG_CHUNK, &tmX, 0, x0 + v - 1, run.h0 + r, z, fb);
           if (++xs == WG_XSTAGES) { xs = 0; xph ^= 1u; }
         }
       }
@@ -569,13 +588,14 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       int y_slot0 = 0;               // ring slot of the current item's dY row 0
       bool ok = mbar_wait(smem_u32(&init_bar), 0, abortp, p.status, DEV_TIMEOUT_MMA_TMEM);   // accumulators zeroed
       tc_fence_after();
-      for (int it = i0; it < i1 && ok; ++it) {
-        const int seg = it % p.nseg;
-        const int npx = min(WG_PIX, p.W - seg * WG_PIX);
+      for (long long pos = r0; pos < r1 && ok;) {
+        const WgRun run = wg_run(p, pos, r1);
+        pos += run.n;
+        const int npx = min(WG_PIX, p.W - run.seg * WG_PIX);
         const int ksteps = (npx + UMMA_K - 1) / UMMA_K;
         int yhave = 0;
-        for (int r = 0; r < p.RB + 2 && ok; ++r) {
-          const int i_hi = min(r, p.RB - 1), i_lo = max(0, r - 2);
+        for (int r = 0; r < run.n + 2 && ok; ++r) {
+          const int i_hi = min(r, run.n - 1), i_lo = max(0, r - 2);
           while (yhave <= i_hi && ok) {
             ok = mbar_wait(smem_u32(&yfull[yw]), ywph, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
             if (++yw == WG_YSTAGES) { yw = 0; ywph ^= 1u; }
@@ -601,7 +621,7 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           if (++xw == WG_XSTAGES) { xw = 0; xwph ^= 1u; }
           if (r >= 2) tc_commit(smem_u32(&yempty[(y_slot0 + r - 2) % WG_YSTAGES]));   // dY row r-2 has no later reader
         }
-        y_slot0 = (y_slot0 + p.RB) % WG_YSTAGES;
+        y_slot0 = (y_slot0 + run.n) % WG_YSTAGES;
       }
       if (ok) tc_commit(smem_u32(&done_bar));
     }
@@ -703,12 +723,6 @@ bool make_weight_map(CUtensorMap* tm, const void* base) {
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int largest_divisor_at_most(int n, int cap) {
-  for (int d = cap; d >= 1; --d)
-    if (n % d == 0) return d;
-  return 1;
-}
-
 }  // namespace
 
 struct ConvNet {
@@ -728,7 +742,6 @@ struct ConvNet {
   float* wpart = nullptr;
   float* loss_part = nullptr;
   bf16* scratch_nchw = nullptr;
-  int wg_RB = 1;
   int state = 0;                     // 0 idle, 1 forward done, 2 backward (gradients kept), 3 backward (fused)
 };
 
@@ -777,7 +790,6 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   c->L = L; c->B = B; c->H = H; c->W = W; c->P_r = P_r; c->Hs = H / P_r; c->R = c->Hs + 2; c->Z = B * P_r;
   c->num_sms = num_sms; c->grid = num_sms; c->status = status; c->stream = stream; c->prof = prof;
   c->strip_elems = static_cast<size_t>(c->Z) * c->R * W * C;
-  c->wg_RB = largest_divisor_at_most(c->Hs, 14);
   auto alloc = [&](void** p, size_t bytes) -> bool {
     if (cudaMalloc(p, bytes) != cudaSuccess) { (void)cudaGetLastError(); *p = nullptr; return false; }
     return cudaMemsetAsync(*p, 0, bytes, stream) == cudaSuccess;
@@ -872,11 +884,11 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
                  c->relu[i - 1] ? c->act[i] : nullptr, c->relu[i - 1] ? &c->act_tile[i] : nullptr);
     }
     WgParams p;
-    p.W = c->W; p.Hs = c->Hs; p.R = c->R; p.RB = c->wg_RB; p.nrb = c->Hs / c->wg_RB;
+    p.W = c->W; p.Hs = c->Hs; p.R = c->R;
     p.nseg = (c->W + WG_PIX - 1) / WG_PIX;
-    p.n_items = static_cast<int>(c->Z) * p.nrb * p.nseg;
+    p.rows_total = static_cast<long long>(c->Z) * p.nseg * c->Hs;
     p.part = c->wpart; p.status = c->status;
-    const int grid = p.n_items < c->grid ? p.n_items : c->grid;
+    const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
     c->prof->begin(MBD_K_CONV_BWD_WEIGHT, 2.0 * c->B * c->H * c->W * 9.0 * C * C);
     launch_pdl(conv_wgrad_kernel, dim3(grid), dim3(NUM_THREADS), WG_SMEM, c->stream, 1, c->act_wg[i], c->dY_wg[i], p);
     c->prof->end();
