@@ -11,17 +11,21 @@
 // (backward-weight: pixels are the reduction index) tensor-core operand.
 //
 // conv_fwd_kernel  (forward and, with flipped / transposed weights, backward-data)
-//     input-row stationary: every input row segment is loaded once per row block as three
-//     horizontally shifted copies (three TMA boxes) and, for each shift v, multiplied by the
+//     input-row stationary: every input row segment is loaded once, as ONE box of 130 pixels; the
+//     three horizontally shifted operands are views of that box whose descriptors start 0, 1, 2
+//     pixel rows (128 bytes) into it (the 128-byte swizzle depends on the shared-memory address
+//     only, so a shifted view reads back what TMA wrote).  Each view is multiplied by the
 //     stacked taps [K(0,v); K(1,v); K(2,v)] (N = 192); the three 64-column results belong to the
 //     output rows r, r-1, r-2, whose accumulators sit next to each other in a ring of eight
 //     TMEM blocks.  An output row is complete after three input rows; the epilogue drains it,
-//     zeroes the block and stores.  The weights (72 KB) stay resident in shared memory.
+//     zeroes the block, and writes it through a swizzled staging tile that TMA stores (the mask
+//     source of backward-data arrives by TMA too).  The weights (72 KB) stay resident in shared
+//     memory.  A CTA owns one contiguous span of the flattened (strip, segment, row) space.
 // conv_wgrad_kernel
 //     dK[o,c,u,v] = sum_pixels dY[p,o] X[p + (u-1,v-1), c]: the three horizontal shifts of an X
-//     row are three TMA boxes (the W coordinate of a box start is free); two shifted copies
-//     form one M = 128 operand; all nine taps accumulate in TMEM for the whole kernel and each
-//     CTA writes one fp32 partial, summed in CTA order (= strip order) by wgrad_finish.
+//     row are again views of one 130-pixel box; two views one pixel apart form one M = 128
+//     operand (leading offset 128 bytes); all nine taps accumulate in TMEM for the whole kernel
+//     and each CTA writes one fp32 partial, summed in CTA order (= strip order) by wgrad_finish.
 #include <stdlib.h>
 
 #include <new>
@@ -54,10 +58,11 @@ constexpr int FWD_SMEM = FWD_W_BYTES + FWD1_STAGES * FWD1_ROW_BYTES + 4 * FWD_TI
 static_assert(FWD_SMEM <= 227 * 1024, "forward kernel's shared memory");
 constexpr int FWD_THREADS = 320;      // producer warp, MMA warp, 8 epilogue warps
 constexpr int WG_PIX = 128;           // pixels (reduction length) per backward-weight block
-constexpr int WG_XSTAGES = 2;          // X rows: 3 shifted copies of 16 KB each, each row used once
-constexpr int WG_YSTAGES = 4;          // dY rows: 16 KB each, plus 2 mirror slots
+constexpr int WG_XSTAGES = 4;          // X rows: one box of 130 pixels each (17 KB), each row used once
+constexpr int WG_YSTAGES = 6;          // dY rows: 16 KB each, plus 2 mirror slots
 constexpr int WG_CHUNK = WG_PIX * 128;
-constexpr int WG_SMEM = WG_XSTAGES * 3 * WG_CHUNK + (WG_YSTAGES + 2) * WG_CHUNK + 1024;
+constexpr int WG_XROW_BYTES = 17 * 1024;   // 130 x 128 B, padded to the swizzle span; the views may read one row past the box
+constexpr int WG_SMEM = WG_XSTAGES * WG_XROW_BYTES + (WG_YSTAGES + 2) * WG_CHUNK + 1024;
 constexpr int NUM_THREADS = 192;
 
 enum { MODE_RELU_STORE = 0, MODE_STORE_SSQ = 1, MODE_MASK = 2 };
@@ -512,7 +517,7 @@ __device__ __forceinline__ WgRun wg_run(const WgParams& p, long long pos, long l
   return r;
 }
 
-// One X row (three shifted copies) meets the up to three dY rows it contributes to in ONE
+// One X row (one box of 130 pixels, read through three shifted views) meets the up to three dY rows it contributes to in ONE
 // instruction group: B = [dY_{r-2} | dY_{r-1} | dY_r] (N = 64 per row, rows adjacent in the dY
 // ring), A = (shift 0 | shift 1) and (shift 2 | don't care), so tap (u, v) accumulates in
 // TMEM lanes (v, c) and columns (2 - u, o).  The dY ring mirrors its first two slots behind
@@ -526,8 +531,8 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   __shared__ int abort_flag;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t xring = base;                                    // slot = 3 chunks (shift 0,1,2)
-  const uint32_t yring = base + WG_XSTAGES * 3 * WG_CHUNK;        // WG_YSTAGES slots + 2 mirror slots
+  const uint32_t xring = base;                                    // slot = one 130-pixel box of an X row
+  const uint32_t yring = base + WG_XSTAGES * WG_XROW_BYTES;       // WG_YSTAGES slots + 2 mirror slots
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
@@ -574,9 +579,8 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           ok = mbar_wait(smem_u32(&xempty[xs]), xph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
           if (!ok) break;
           const uint32_t fb = smem_u32(&xfull[xs]);
-          mbar_expect_tx(fb, 3 * WG_CHUNK);
-          for (int v = 0; v < 3; ++v)
-            tma_load_4d(xring + (xs * 3 + v) * WG_CHUNK, &tmX, 0, x0 + v - 1, run.h0 + r, z, fb);
+          mbar_expect_tx(fb, (WG_PIX + 2) * 128);
+          tma_load_4d(xring + xs * WG_XROW_BYTES, &tmX, 0, x0 - 1, run.h0 + r, z, fb);
           if (++xs == WG_XSTAGES) { xs = 0; xph ^= 1u; }
         }
       }
@@ -610,9 +614,11 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           const uint32_t idesc = make_idesc(128, 64 * n, 1, 1);
           const int ys0 = (y_slot0 + i_lo) % WG_YSTAGES;       // window may run into the mirror slots
           const uint64_t bdesc = make_desc(yring + ys0 * WG_CHUNK, WG_CHUNK, 1024);
-          const uint32_t xa = xring + xw * 3 * WG_CHUNK;
-          const uint64_t a01 = make_desc(xa, WG_CHUNK, 1024);                 // lanes: (shift 0 | shift 1) x c
-          const uint64_t a2x = make_desc(xa + 2 * WG_CHUNK, WG_CHUNK, 1024);  // lanes: (shift 2 | don't care) x c
+          // The operand shifted by v pixels is the view of the box that starts v pixel rows (128 bytes) in; the
+          // two 64-channel chunks of an M = 128 operand are two such views, one row apart (leading offset 128).
+          const uint32_t xa = xring + xw * WG_XROW_BYTES;
+          const uint64_t a01 = make_desc(xa, 128, 1024);                      // lanes: (shift 0 | shift 1) x c
+          const uint64_t a2x = make_desc(xa + 2 * 128, 128, 1024);            // lanes: (shift 2 | don't care) x c
           for (int k = 0; k < ksteps; ++k) {
             tc_mma_bf16(tmem_base + b0 * 64, a01 + k * 128, bdesc + k * 128, idesc, 1u);
             tc_mma_bf16(tmem_base + 256 + b0 * 64, a2x + k * 128, bdesc + k * 128, idesc, 1u);
@@ -737,7 +743,7 @@ struct ConvNet {
   std::vector<bf16*> K, Wf, Wb;
   std::vector<float*> dK;
   std::vector<int> relu;
-  std::vector<CUtensorMap> act_fwd, act_wg, dY_fwd, dY_wg, wf_map, wb_map;
+  std::vector<CUtensorMap> act_fwd, dY_fwd, dY_wg, wf_map, wb_map;   // act_fwd / dY_fwd: 130-pixel boxes (also the X operand of backward-weight)
   std::vector<CUtensorMap> act_tile, dY_tile;     // [128 pixels][64 channels] boxes: TMA stores of outputs, mask rows
   float* wpart = nullptr;
   float* loss_part = nullptr;
@@ -811,12 +817,11 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   ok = ok && alloc(reinterpret_cast<void**>(&c->scratch_nchw), static_cast<size_t>(B) * C * H * W * 2);
   if (!ok) { conv_destroy(c); return MBD_E_ALLOC; }
   const int fwd_box = FWD1_BOX_PIX;
-  c->act_fwd.resize(L + 1); c->act_wg.resize(L + 1); c->dY_fwd.resize(L); c->dY_wg.resize(L);
+  c->act_fwd.resize(L + 1); c->dY_fwd.resize(L); c->dY_wg.resize(L);
   c->act_tile.resize(L + 1); c->dY_tile.resize(L);
   c->wf_map.resize(L); c->wb_map.resize(L);
   for (int i = 0; i <= L && ok; ++i)
-    ok = make_strip_map(&c->act_fwd[i], c->act[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->act_wg[i], c->act[i], W, c->R, c->Z, WG_PIX) &&
-         make_strip_map(&c->act_tile[i], c->act[i], W, c->R, c->Z, FWD_PIX);
+    ok = make_strip_map(&c->act_fwd[i], c->act[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->act_tile[i], c->act[i], W, c->R, c->Z, FWD_PIX);
   for (int i = 0; i < L && ok; ++i)
     ok = make_strip_map(&c->dY_fwd[i], c->dY[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->dY_wg[i], c->dY[i], W, c->R, c->Z, WG_PIX) &&
          make_strip_map(&c->dY_tile[i], c->dY[i], W, c->R, c->Z, FWD_PIX) &&
@@ -890,7 +895,7 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
     p.part = c->wpart; p.status = c->status;
     const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
     c->prof->begin(MBD_K_CONV_BWD_WEIGHT, 2.0 * c->B * c->H * c->W * 9.0 * C * C);
-    launch_pdl(conv_wgrad_kernel, dim3(grid), dim3(NUM_THREADS), WG_SMEM, c->stream, 1, c->act_wg[i], c->dY_wg[i], p);
+    launch_pdl(conv_wgrad_kernel, dim3(grid), dim3(NUM_THREADS), WG_SMEM, c->stream, 1, c->act_fwd[i], c->dY_wg[i], p);
     c->prof->end();
     c->prof->begin(MBD_K_REDUCE, (grid + 1.0) * 9 * C * C * 4.0);
     wgrad_finish_kernel<<<9 * C * C / 64, 256, 0, c->stream>>>(c->wpart, grid, fused ? nullptr : c->dK[i],
