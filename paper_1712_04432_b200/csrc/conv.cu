@@ -252,7 +252,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t w_smem = base;                         // 3 (v) x [192 rows (u, o) x 128 B]
-  const uint32_t ring = base + FWD_W_BYTES;             // slot = one input row (one box, or 3 shifted copies)
+  const uint32_t ring = base + FWD_W_BYTES;             // slot = one input row (one box of 130 pixels)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
