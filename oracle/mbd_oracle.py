@@ -19,7 +19,12 @@ none after the last layer; gradients are SUMS over the batch and the 1/B of
 Eq. 1 is applied once, in the update; softmax cross-entropy with natural log
 (sum over samples) or half sum of squares as the loss; dX_1 is not formed
 (Section 2.2: nothing is back-propagated beyond the first layer);
-convolution is cross-correlation with zero padding.
+convolution is cross-correlation with zero padding.  Where a fully connected
+layer follows a convolution (the integrated network of Section 2.4, Eq. 9:
+domain-parallel layers first, model-parallel layers after them), the
+activation [B, C, H, W] becomes the matrix with row index c*H*W + h*W + w
+(NCHW order, the layout of Section 2.2; a fully connected layer is the
+convolution whose kernel covers the whole input, end of Section 2.4).
 """
 from __future__ import annotations
 
@@ -52,6 +57,33 @@ class Conv3x3:
 def balanced_ranges(n: int, P: int):
     """Index ranges [floor(p n / P), floor((p+1) n / P)) for p = 0..P-1."""
     return [((p * n) // P, ((p + 1) * n) // P) for p in range(P)]
+
+
+def flatten_nchw(T):
+    """[B, C, H, W] -> the d x B matrix X with X[c*H*W + h*W + w, b] = T[b, c, h, w]:
+    the input of a fully connected layer that follows a convolution
+    (a fully connected layer = a convolution with k_h = X_H, k_w = X_W, Section 2.4)."""
+    T = np.asarray(T, F64)
+    return np.ascontiguousarray(T.reshape(T.shape[0], -1).T)
+
+
+def unflatten_nchw(M, shape):
+    """Inverse of `flatten_nchw`: d x B -> [B, C, H, W]."""
+    return np.ascontiguousarray(np.asarray(M, F64).T).reshape(shape)
+
+
+def _kept(A, lay, nxt, store):
+    """What is kept of Y_i as the input of the next layer: f(Y_i), storage-rounded,
+    flattened when a fully connected layer follows a convolution."""
+    A = _stored(relu(A) if lay.relu else A, store)
+    if A.ndim == 4 and isinstance(nxt, FC):
+        A = flatten_nchw(A)
+    return A
+
+
+def _below(dX, Y_prev):
+    """dX_i brought to the shape of the output of the layer below."""
+    return unflatten_nchw(dX, Y_prev.shape) if dX.ndim == 2 and Y_prev.ndim == 4 else dX
 
 
 # --------------------------------------------------------------------------
@@ -182,7 +214,7 @@ def forward(layers: Sequence, X1, store=None):
             Y = conv3x3(lay.K, Xs[i])
         Ys.append(Y)
         if i + 1 < len(layers):
-            Xs.append(_stored(relu(Y) if lay.relu else Y, store))
+            Xs.append(_kept(Y, lay, layers[i + 1], store))
     return Xs, Ys
 
 
@@ -218,6 +250,7 @@ def train_step(layers: Sequence, X1, labels, loss: str, eta: float, store=None):
             dWs[i] = conv3x3_dK(dYs[i], Xs[i])
         if i > 0:
             dXs[i] = fc_dX(lay.W, dYs[i]) if isinstance(lay, FC) else conv3x3_dX(lay.K, dYs[i])
+            dXs[i] = _below(dXs[i], Ys[i - 1])
             prev = layers[i - 1]
             dYs[i - 1] = dXs[i] * (Ys[i - 1] > 0.0) if prev.relu else dXs[i]
     new_W, new_b = [], []
@@ -369,13 +402,31 @@ def conv3x3_dK_strips(dY, X, P_r):
     return dK, parts
 
 
+def conv3x3_dK_grid(dY, X, P_r, P_c):
+    """Weight gradient of a domain-parallel layer on a P_r x P_c grid: process
+    (r, c) owns strip r of the samples of batch block c and forms one partial;
+    the all-reduce over all P = P_r P_c processes (last term of Eq. 9) adds them,
+    here in ascending c, then r.  Returns (dK, partials)."""
+    dY = np.asarray(dY, F64)
+    X = np.asarray(X, F64)
+    parts = []
+    for (c0, c1) in balanced_ranges(X.shape[0], P_c):
+        _, strip_parts = conv3x3_dK_strips(dY[c0:c1], X[c0:c1], P_r)
+        parts.extend(strip_parts)
+    dK = np.zeros_like(parts[0])
+    for part in parts:
+        dK = dK + part
+    return dK, parts
+
+
 def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
                        P_r: int, P_c: int, store=None):
     """The step of `train_step`, every contraction formed block by block over
     the P_r x P_c grid and every cross-block sum taken as P separate partials
     added in ascending block index.  FC layers split the model over P_r and the
-    batch over P_c; convolution layers split the image into P_r row strips
-    (P_c must be 1 for them)."""
+    batch over P_c; convolution layers split the image into P_r row strips and
+    the batch over P_c (Eq. 9: their weight gradient is summed over all
+    P = P_r P_c processes)."""
     L = len(layers)
     Xs = [np.asarray(X1, F64)]
     Ys = []
@@ -383,11 +434,10 @@ def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
         if isinstance(lay, FC):
             Y = fc_forward_blocked(lay.W, Xs[i], lay.b, P_r, P_c)
         else:
-            assert P_c == 1
             Y = conv3x3_strips(lay.K, Xs[i], P_r)
         Ys.append(Y)
         if i + 1 < L:
-            Xs.append(_stored(relu(Y) if lay.relu else Y, store))
+            Xs.append(_kept(Y, lay, layers[i + 1], store))
     B = _batch_of(Xs[0])
     J, per, dY_top = loss_and_top_grad(Ys[-1], loss, labels)
     dYs = [None] * L
@@ -405,12 +455,13 @@ def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
                     db = db + dYs[i][:, c0:c1].sum(axis=1)
                 dbs[i] = db
         else:
-            dWs[i], _ = conv3x3_dK_strips(dYs[i], Xs[i], P_r)
+            dWs[i], _ = conv3x3_dK_grid(dYs[i], Xs[i], P_r, P_c)
         if i > 0:
             if isinstance(lay, FC):
                 dXs[i], _ = fc_dX_blocked(lay.W, dYs[i], P_r, P_c)
             else:
                 dXs[i] = conv3x3_dX_strips(lay.K, dYs[i], P_r)
+            dXs[i] = _below(dXs[i], Ys[i - 1])
             prev = layers[i - 1]
             dYs[i - 1] = dXs[i] * (Ys[i - 1] > 0.0) if prev.relu else dXs[i]
     new_W, new_b = [], []

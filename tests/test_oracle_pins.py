@@ -376,3 +376,109 @@ def test_storage_rounding_only_touches_kept_activations():
     assert np.array_equal(c["Ys"][1], O.affine(layers[1].W, c["Xs"][1], layers[1].b))
     d = O.train_step_blocked(layers, X, labels, "softmax_ce", 0.01, 2, 2, store=q)
     assert all(relerr(x, y) < 1e-12 for x, y in zip(c["dWs"], d["dWs"]))
+
+
+# ---------------------------------------------------------------- convolutions followed by fully connected layers
+def mixed_case(seed=70, B=3, C=2, H=4, W=3, hidden=5, classes=4, relu_conv=True):
+    r = rng(seed)
+    layers = [O.Conv3x3(r.standard_normal((C, C, 3, 3)) / 3, relu=True),
+              O.Conv3x3(r.standard_normal((C, C, 3, 3)) / 3, relu=relu_conv),
+              O.FC(r.standard_normal((hidden, C * H * W)) / math.sqrt(C * H * W), 0.1 * r.standard_normal(hidden), relu=True),
+              O.FC(r.standard_normal((classes, hidden)) / math.sqrt(hidden), None, relu=False)]
+    X = r.standard_normal((B, C, H, W))
+    labels = r.integers(0, classes, B)
+    return layers, X, labels
+
+
+def test_flatten_is_nchw_order():
+    """Row c*H*W + h*W + w of the fully connected input is pixel (c, h, w): width runs
+    fastest, then height, then channels (Section 2.2)."""
+    B, C, H, W = 2, 3, 4, 5
+    T = rng(71).standard_normal((B, C, H, W))
+    M = O.flatten_nchw(T)
+    assert M.shape == (C * H * W, B)
+    for b in range(B):
+        for c in range(C):
+            for h in range(H):
+                for w in range(W):
+                    assert M[c * H * W + h * W + w, b] == T[b, c, h, w]
+    assert np.array_equal(O.unflatten_nchw(M, T.shape), T)
+
+
+def test_fc_after_conv_is_conv_covering_whole_input():
+    """A fully connected layer on the flattened activation equals the convolution whose kernel
+    covers the whole input (end of Section 2.4), evaluated with scalar loops."""
+    B, C, H, W, D = 2, 2, 3, 4, 3
+    r = rng(72)
+    T = r.standard_normal((B, C, H, W))
+    Wm = r.standard_normal((D, C * H * W))
+    Y = O.affine(Wm, O.flatten_nchw(T))
+    Kfull = Wm.reshape(D, C, H, W)
+    for b in range(B):
+        for o in range(D):
+            acc = 0.0
+            for c in range(C):
+                for h in range(H):
+                    for w in range(W):
+                        acc += Kfull[o, c, h, w] * T[b, c, h, w]
+            assert abs(acc - Y[o, b]) < 1e-12
+
+
+def test_mixed_stack_grads_by_central_differences():
+    seed = 70
+    while True:
+        layers, X, labels = mixed_case(seed)
+        if _no_kink(layers, X, 1e-4):
+            break
+        seed += 1
+    res = O.train_step(layers, X, labels, "softmax_ce", 0.0)
+    eps = 1e-6
+    checks = [(0, "K", (1, 0, 2, 1)), (0, "K", (0, 1, 0, 0)), (1, "K", (1, 1, 1, 2)), (1, "K", (0, 0, 2, 2)),
+              (2, "W", (3, 7)), (2, "W", (0, 23)), (3, "W", (2, 4)), (2, "b", (1,))]
+    for li, name, idx in checks:
+        arr = getattr(layers[li], name)
+        old = arr[idx]
+        arr[idx] = old + eps; Jp = O.total_loss(layers, X, labels, "softmax_ce")
+        arr[idx] = old - eps; Jm = O.total_loss(layers, X, labels, "softmax_ce")
+        arr[idx] = old
+        g = (Jp - Jm) / (2 * eps)
+        got = res["dbs"][li][idx] if name == "b" else res["dWs"][li][idx]
+        assert abs(g - got) < 1e-6 * max(1.0, abs(g)), (li, name, idx, g, got)
+    # dX of the first fully connected layer comes back in NCHW shape and feeds the convolution below it
+    assert res["dXs"][2].shape == X.shape and res["dYs"][1].shape == X.shape
+
+
+def test_mixed_stack_input_gradient_shape_and_mask():
+    layers, X, labels = mixed_case(73)
+    res = O.train_step(layers, X, labels, "softmax_ce", 0.0)
+    dX_fc = O.fc_dX(layers[2].W, res["dYs"][2])                      # d x B
+    assert np.array_equal(res["dXs"][2], O.unflatten_nchw(dX_fc, X.shape))
+    assert np.array_equal(res["dYs"][1], res["dXs"][2] * (res["Ys"][1] > 0))
+
+
+@pytest.mark.parametrize("grid", [(1, 1), (2, 1), (1, 3), (2, 3), (4, 2)])
+def test_mixed_blocked_step_equals_unblocked(grid):
+    layers, X, labels = mixed_case(74, B=6, H=8)
+    a = O.train_step(layers, X, labels, "softmax_ce", 0.01)
+    b = O.train_step_blocked(layers, X, labels, "softmax_ce", 0.01, *grid)
+    assert abs(a["J"] - b["J"]) < 1e-12 * abs(a["J"])
+    for i in range(4):
+        assert relerr(b["Ys"][i], a["Ys"][i]) < 1e-12
+        assert relerr(b["new_W"][i], a["new_W"][i]) < 1e-12
+        assert relerr(b["dWs"][i], a["dWs"][i]) < 1e-12
+    for i in range(1, 4):
+        assert relerr(b["dXs"][i], a["dXs"][i]) < 1e-12
+
+
+def test_conv_weight_gradient_partials_over_the_whole_grid():
+    """P_r x P_c partials, one per process, whose sum is the un-blocked gradient (last term of Eq. 9)."""
+    r = rng(75)
+    X = r.standard_normal((6, 3, 8, 5)); dY = r.standard_normal((6, 4, 8, 5))
+    for P_r, P_c in [(2, 3), (4, 2), (1, 6), (8, 1)]:
+        dK, parts = O.conv3x3_dK_grid(dY, X, P_r, P_c)
+        assert len(parts) == P_r * P_c
+        assert relerr(dK, O.conv3x3_dK(dY, X)) < 1e-13
+    # the partial of process (r=1, c=0) of a 2 x 3 grid: strip 1 of samples 0, 1
+    _, parts = O.conv3x3_dK_grid(dY, X, 2, 3)
+    Xz = X[0:2].copy(); dYz = dY[0:2].copy(); dYz[:, :, 0:4, :] = 0.0          # only output rows 4..7 contribute
+    assert relerr(parts[1], O.conv3x3_dK(dYz, Xz)) < 1e-13
