@@ -116,6 +116,9 @@ def pick_grid(w, arg):
 def workload_config(w, grid, max_partials):
     if w.kind == "fc":
         desc = f"{w.name}: FC stack {'-'.join(str(d) for d in w.dims)}, B={w.B}, ReLU, softmax-CE, {w.dtype}"
+    elif w.kind == "mixed":
+        desc = (f"{w.name}: {w.n_layers}x conv3x3 {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, then FC "
+                f"{'-'.join(str(d) for d in w.fc_dims)}, B={w.B}, ReLU, softmax-CE, {w.dtype}")
     else:
         desc = f"{w.name}: {w.n_layers}x conv3x3 {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, B={w.B}, half-SSQ, {w.dtype}"
     return dict(workload=desc, grid=f"{grid[0]}x{grid[1]}", max_partials=max_partials, batch=w.B,
@@ -139,6 +142,15 @@ def oracle_sample(w, inp):
         O.train_step(layers, X, labels, "softmax_ce", w.eta)
         dt = time.perf_counter() - t0
         return flops_per_sample * Bs, dt, f"whole {len(layers)}-layer network, first {Bs} of {w.B} samples, fp64 numpy"
+    if w.kind == "mixed":
+        Bs = min(w.B, 4)
+        layers = [O.Conv3x3(inp.Ws[i].astype(np.float64)) for i in range(w.n_layers)]
+        layers += [O.FC(inp.Ws[i].astype(np.float64), inp.bs[i].astype(np.float64)) for i in range(w.n_layers, w.L)]
+        X = inp.X[:Bs].astype(np.float64)
+        t0 = time.perf_counter()
+        O.train_step(layers, X, inp.labels[:Bs], "softmax_ce", w.eta)
+        dt = time.perf_counter() - t0
+        return I.step_flops(w) / w.B * Bs, dt, f"whole {w.L}-layer network, first {Bs} of {w.B} samples, fp64 numpy"
     C, H, Wd = w.dims
     Bs, Hs = 1, min(H, 56)
     layers = [O.Conv3x3(k.astype(np.float64)) for k in inp.Ws]
@@ -250,9 +262,17 @@ def run_ours(args):
             net.set_weights(i, dev(Wi), torch.from_numpy(inp.bs[i]).cuda())
         labels = torch.from_numpy(inp.labels).cuda()
         labels_host = torch.from_numpy(inp.labels).pin_memory()
+    elif w.kind == "mixed":
+        C_, H, Wd = w.dims
+        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd) + mbd.fc_layers(w.fc_dims, bias=True), w.B, grid[0], grid[1],
+                      mbd.BF16, mbd.LOSS_SOFTMAX_CE, args.max_partials)
+        for i, Wi in enumerate(inp.Ws):
+            net.set_weights(i, dev(Wi), None if inp.bs[i] is None else torch.from_numpy(inp.bs[i]).cuda())
+        labels = torch.from_numpy(inp.labels).cuda()
+        labels_host = torch.from_numpy(inp.labels).pin_memory()
     else:
         C_, H, Wd = w.dims
-        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd), w.B, grid[0], 1, mbd.BF16, mbd.LOSS_HALF_SSQ,
+        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd), w.B, grid[0], grid[1], mbd.BF16, mbd.LOSS_HALF_SSQ,
                       args.max_partials)
         for i, Ki in enumerate(inp.Ws):
             net.set_weights(i, dev(Ki))
@@ -364,6 +384,8 @@ def run_ours(args):
         peak = peaks["bf16_tflops_sustained"] if bf else 148 * 128 * 2 * 1.965e9 / 1e12
         if w.kind == "conv":
             kname = "conv_fwd_kernel (forward, backward-data) + conv_wgrad_kernel"
+        elif w.kind == "mixed":
+            kname = "conv_fwd_kernel + conv_wgrad_kernel (convolutions), gemm_tc_kernel (fully connected layers)"
         elif bf:
             kname = "gemm_tc_kernel (all three operand layouts)"
         else:

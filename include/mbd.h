@@ -107,10 +107,19 @@ enum {
  *                 the default (4); 1 never materialises; >= P materialises every
  *                 block's partial exactly as the paper's processes would hold it.
  *   cuda_stream   a cudaStream_t (may be NULL for the default stream).
- * MBD_E_GRID if P_r < 1, P_c < 1, P_c > B, P_r > min d_i over model-split layers,
- * a strip would be shorter than its halo, or P_c != 1 with a domain-split layer.
+ * Layer order (Section 2.4, Eq. 9): domain-split convolutions first (L_D), model-split
+ * fully connected layers after them (L_M); either group may be empty.  With both present
+ * the input is NCHW, the first fully connected layer reads the last convolution's output
+ * as [B, C*H*W] (row index c*H*W + h*W + w; its d_in must equal that), the loss is
+ * softmax-CE, the dtype bf16, and the public layer index counts the convolutions first.
+ * On a P_r x P_c grid a convolution is cut into P_r row strips and P_c batch blocks, a
+ * fully connected layer into P_r row blocks of W_i and the same P_c batch blocks.
+ * MBD_E_GRID if P_r < 1, P_c < 1, P_c > B, P_r > min d_i over model-split layers, or
+ * a strip would be shorter than its halo.
  * MBD_E_UNSUPPORTED for convolutions other than 3x3/s1/p1 with C_in = C_out = 64,
- * or bf16 FC dims that are not multiples of 8. */
+ * strips of unequal height, a convolution above a fully connected layer, half-SSQ with
+ * fully connected layers or softmax-CE without them, or bf16 FC dims that are not
+ * multiples of 8. */
 MBD_API mbd_status mbd_net_create(const mbd_layer* layers_host, int L, int64_t B, int P_r, int P_c,
                           int dtype, int loss, int max_partials, void* cuda_stream, mbd_net** out);
 MBD_API mbd_status mbd_net_destroy(mbd_net* net);

@@ -749,6 +749,7 @@ struct ConvNet {
   float* loss_part = nullptr;
   bf16* scratch_nchw = nullptr;
   int state = 0;                     // 0 idle, 1 forward done, 2 backward (gradients kept), 3 backward (fused)
+  bool fc_above = false;             // fully connected layers follow: no loss here, dY of the last layer comes from above
 };
 
 namespace {
@@ -786,7 +787,7 @@ void launch_stage_in(ConvNet* c, const bf16* nchw, bf16* strips) {
 }  // namespace
 
 mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int max_partials, int num_sms, int* status,
-                       cudaStream_t stream, Profiler* prof, ConvNet** out) {
+                       cudaStream_t stream, Profiler* prof, bool fc_above, ConvNet** out) {
   (void)max_partials;
   if (conv_init() != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
   const int H = layers[0].H, W = layers[0].W;
@@ -795,6 +796,7 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   if (!c) return MBD_E_ALLOC;
   c->L = L; c->B = B; c->H = H; c->W = W; c->P_r = P_r; c->Hs = H / P_r; c->R = c->Hs + 2; c->Z = B * P_r;
   c->num_sms = num_sms; c->grid = num_sms; c->status = status; c->stream = stream; c->prof = prof;
+  c->fc_above = fc_above;
   c->strip_elems = static_cast<size_t>(c->Z) * c->R * W * C;
   auto alloc = [&](void** p, size_t bytes) -> bool {
     if (cudaMalloc(p, bytes) != cudaSuccess) { (void)cudaGetLastError(); *p = nullptr; return false; }
@@ -807,7 +809,7 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   for (int i = 0; i <= L && ok; ++i) ok = alloc(reinterpret_cast<void**>(&c->act[i]), c->strip_elems * 2);
   for (int i = 0; i < L && ok; ++i) {
     c->relu[i] = layers[i].relu;
-    if (i < L - 1) ok = alloc(reinterpret_cast<void**>(&c->dY[i]), c->strip_elems * 2);
+    if (i < L - 1 || fc_above) ok = alloc(reinterpret_cast<void**>(&c->dY[i]), c->strip_elems * 2);
     else c->dY[i] = c->act[L];                       // half-SSQ loss: dY_L = Y_L
     ok = ok && alloc(reinterpret_cast<void**>(&c->K[i]), 9 * C * C * 2) && alloc(reinterpret_cast<void**>(&c->Wf[i]), 9 * C * C * 2) &&
          alloc(reinterpret_cast<void**>(&c->Wb[i]), 9 * C * C * 2) && alloc(reinterpret_cast<void**>(&c->dK[i]), 9 * C * C * 4);
@@ -835,7 +837,8 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
 void conv_destroy(ConvNet* c) {
   if (!c) return;
   for (size_t i = 0; i < c->act.size(); ++i) cudaFree(c->act[i]);
-  for (int i = 0; i + 1 < c->L; ++i) cudaFree(c->dY[i]);
+  for (int i = 0; i < c->L; ++i)
+    if (c->dY[i] != c->act[c->L]) cudaFree(c->dY[i]);
   for (int i = 0; i < c->L; ++i) { cudaFree(c->K[i]); cudaFree(c->Wf[i]); cudaFree(c->Wb[i]); cudaFree(c->dK[i]); }
   cudaFree(c->wpart); cudaFree(c->loss_part); cudaFree(c->scratch_nchw);
   (void)cudaGetLastError();
@@ -866,9 +869,9 @@ mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
     const bool last = i == c->L - 1;
     if (i > 0) launch_halo(c, c->act[i]);            // forward halo exchange (first halo term of Eq. 7)
     launch_fwd(c, MBD_K_CONV_FWD, c->act_fwd[i], c->wf_map[i], c->act[i + 1], c->act_tile[i + 1],
-               last ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK), nullptr, nullptr);
+               (last && !c->fc_above) ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK), nullptr, nullptr);
   }
-  if (loss_sum_dev) {
+  if (loss_sum_dev && !c->fc_above) {
     c->prof->begin(MBD_K_OTHER, c->grid * 32.0);
     if (sum_f32_launch(c->loss_part, c->grid * 8, 0.5f, loss_sum_dev, c->stream) != cudaSuccess) return MBD_E_CUDA;
     c->prof->end();
@@ -916,6 +919,25 @@ mbd_status conv_sgd_step(ConvNet* c, float eta) {
   }
   return MBD_OK;
 }
+
+// Between the domain-parallel and the model-parallel layers (Section 2.4): the strips of the last
+// convolution's output become the [B, C*H*W] matrix (NCHW order) the first fully connected layer reads,
+// and that layer's input gradient goes back into strips, its boundary rows also into the neighbours' halos.
+mbd_status conv_output_to_nchw(ConvNet* c, void* dst) {
+  dim3 g((c->W + 31) / 32, c->H, static_cast<unsigned>(c->B));
+  c->prof->begin(MBD_K_HALO, 2.0 * c->B * C * c->H * c->W * 2.0);
+  strips_to_nchw_kernel<<<g, 256, 0, c->stream>>>(c->act[c->L], static_cast<bf16*>(dst), c->H, c->W, c->P_r, c->Hs);
+  c->prof->end();
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+mbd_status conv_top_grad_from_nchw(ConvNet* c, const void* src) {
+  if (!c->fc_above) return MBD_E_STATE;
+  launch_stage_in(c, static_cast<const bf16*>(src), c->dY[c->L - 1]);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+int conv_last_relu(const ConvNet* c) { return c->relu[c->L - 1]; }
 
 mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t bytes) {
   const size_t nchw_bytes = conv_input_bytes(c);

@@ -10,7 +10,7 @@
 namespace mbd {
 struct ConvNet;
 mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int max_partials, int num_sms, int* status,
-                       cudaStream_t stream, Profiler* prof, ConvNet** out);
+                       cudaStream_t stream, Profiler* prof, bool fc_above, ConvNet** out);
 void conv_destroy(ConvNet* c);
 mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev);
 mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev);
@@ -20,4 +20,8 @@ mbd_status conv_sgd_step(ConvNet* c, float eta);
 mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t bytes);
 mbd_status conv_set_tensor(ConvNet* c, int which, int layer, const void* src, size_t bytes);
 size_t conv_input_bytes(const ConvNet* c);
+// fully connected layers above the convolutions: activation out / gradient in, [B, C*H*W] in NCHW order
+mbd_status conv_output_to_nchw(ConvNet* c, void* dst);
+mbd_status conv_top_grad_from_nchw(ConvNet* c, const void* src);
+int conv_last_relu(const ConvNet* c);
 }  // namespace mbd

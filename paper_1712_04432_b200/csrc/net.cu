@@ -38,7 +38,11 @@ struct Layer {
 }  // namespace
 
 struct mbd_net {
-  int L = 0;
+  int L = 0;                        // fully connected layers (n->layers); public layer index = Lc + index here
+  int Lc = 0;                       // convolution layers below them (n->conv)
+  bool mixed = false;               // convolutions first, fully connected layers after them (Section 2.4)
+  void* X_fc = nullptr;             // [B, C*H*W]: output of the last convolution in NCHW order = input of the first FC layer
+  void* dX_fc = nullptr;            // gradient w.r.t. X_fc after the mask of the last convolution's ReLU
   int64_t B = 0;
   int P_r = 1, P_c = 1, dtype = MBD_BF16, loss = 0, max_partials = 4;
   cudaStream_t stream = nullptr;
@@ -208,6 +212,8 @@ Epi fwd_epi(mbd_net* n, int i) {
 }
 Epi bwd_data_epi(mbd_net* n, int i) {
   Layer& l = n->layers[i];
+  if (i == 0)     // below the first fully connected layer sits the last convolution
+    return epi_mask(n->dX_fc, l.d_in, 1, conv_last_relu(n->conv) ? n->X_fc : nullptr, l.d_in);
   Layer& prev = n->layers[i - 1];
   return epi_mask(prev.dY, l.d_in, n->dtype == MBD_BF16, prev.spec.relu ? prev.act : nullptr, l.d_in);
 }
@@ -232,7 +238,7 @@ void free_net(mbd_net* n) {
     cudaFree(l.W); cudaFree(l.bias); cudaFree(l.dW); cudaFree(l.db); cudaFree(l.act); cudaFree(l.dY);
   }
   cudaFree(n->partials); cudaFree(n->colsum_scratch); cudaFree(n->per_sample); cudaFree(n->loss_dev);
-  cudaFree(n->status); cudaFree(n->X_stage); cudaFree(n->labels_stage);
+  cudaFree(n->status); cudaFree(n->X_stage); cudaFree(n->labels_stage); cudaFree(n->X_fc); cudaFree(n->dX_fc);
   for (int k = 0; k < 2; ++k) {
     cudaFree(n->X_in[k]); cudaFree(n->labels_in[k]);
     if (n->ev_copied[k]) cudaEventDestroy(n->ev_copied[k]);
@@ -266,21 +272,23 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   if (max_partials < 0) return MBD_E_INVALID;
   *out = nullptr;
   if (P_r < 1 || P_c < 1 || P_c > B) return MBD_E_GRID;
-  const bool is_conv = layers[0].kind == MBD_CONV3X3;
+  int Lc = 0;                                 // convolutions come first (L_D), fully connected layers after them (L_M)
+  while (Lc < L && layers[Lc].kind == MBD_CONV3X3) ++Lc;
+  const bool is_conv = Lc == L, mixed = Lc > 0 && Lc < L;
   for (int i = 0; i < L; ++i) {
     const mbd_layer& l = layers[i];
-    if ((l.kind == MBD_CONV3X3) != is_conv) return MBD_E_UNSUPPORTED;   // no mixed stacks yet
+    if (l.kind == MBD_CONV3X3 && i >= Lc) return MBD_E_UNSUPPORTED;      // a convolution above a fully connected layer
     if (l.kind == MBD_FC) {
       if (l.d_in < 1 || l.d_out < 1) return MBD_E_INVALID;
       if (l.split != MBD_SPLIT_MODEL) return MBD_E_INVALID;
-      if (i > 0 && l.d_in != layers[i - 1].d_out) return MBD_E_INVALID;
+      if (i > Lc && l.d_in != layers[i - 1].d_out) return MBD_E_INVALID;
+      if (i == Lc && mixed && l.d_in != static_cast<int64_t>(layers[0].C_out) * layers[0].H * layers[0].W) return MBD_E_INVALID;
       if (P_r > l.d_out) return MBD_E_GRID;
       if (dtype == MBD_BF16 && (l.d_in % 8 || l.d_out % 8)) return MBD_E_UNSUPPORTED;
       if (l.d_in > INT32_MAX || l.d_out > INT32_MAX || B > INT32_MAX) return MBD_E_UNSUPPORTED;
     } else if (l.kind == MBD_CONV3X3) {
       if (l.kh != 3 || l.kw != 3 || l.C_in != 64 || l.C_out != 64 || dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
       if (l.split != MBD_SPLIT_DOMAIN) return MBD_E_UNSUPPORTED;
-      if (P_c != 1) return MBD_E_GRID;
       if (l.H < 1 || l.W < 1 || P_r > l.H) return MBD_E_GRID;   // a strip needs >= 1 row (halo = 1)
       if (i > 0 && (l.H != layers[0].H || l.W != layers[0].W)) return MBD_E_INVALID;
     } else {
@@ -289,10 +297,12 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   }
   if (is_conv && loss != MBD_LOSS_HALF_SSQ) return MBD_E_UNSUPPORTED;
   if (!is_conv && loss != MBD_LOSS_SOFTMAX_CE) return MBD_E_UNSUPPORTED;
+  if (mixed && dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
 
   mbd_net* n = new (std::nothrow) mbd_net();
   if (!n) return MBD_E_ALLOC;
-  n->L = L; n->B = B; n->P_r = P_r; n->P_c = P_c; n->dtype = dtype; n->loss = loss;
+  n->L = L - Lc; n->Lc = Lc; n->mixed = mixed;
+  n->B = B; n->P_r = P_r; n->P_c = P_c; n->dtype = dtype; n->loss = loss;
   n->max_partials = max_partials == 0 ? 4 : max_partials;
   n->stream = static_cast<cudaStream_t>(cuda_stream);
   n->prof.stream = n->stream;
@@ -320,12 +330,16 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   ALLOC(n->loss_dev, sizeof(float));
   if (cudaMemsetAsync(n->status, 0, sizeof(int), n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
 
-  if (is_conv) {
-    st = conv_create(layers, L, B, P_r, n->max_partials, n->num_sms, n->status, n->stream, &n->prof, &n->conv);
+  if (Lc > 0) {
+    st = conv_create(layers, Lc, B, P_r, n->max_partials, n->num_sms, n->status, n->stream, &n->prof, mixed, &n->conv);
     if (st != MBD_OK) { free_net(n); return st; }
-    *out = n;
-    return MBD_OK;
+    if (is_conv) {
+      *out = n;
+      return MBD_OK;
+    }
   }
+  layers += Lc;                      // from here on: the fully connected layers
+  L -= Lc;
 
   const size_t es = n->elt();
   const int S_r = splits_for(P_r, n->max_partials), S_c = splits_for(P_c, n->max_partials);
@@ -352,22 +366,28 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
     }
     max_d = std::max(max_d, static_cast<size_t>(l.d_out));
   }
+  if (mixed) {
+    ALLOC(n->X_fc, static_cast<size_t>(B) * n->layers[0].d_in * es);
+    ALLOC(n->dX_fc, static_cast<size_t>(B) * n->layers[0].d_in * es);
+    n->X = n->X_fc;
+    n->X_mapped = n->X_fc;           // the plans below are built on the real input buffer
+  }
   if (dtype == MBD_BF16) {
     // Plan every contraction now (tile width, number of K pieces); the partial-sum workspace is
     // sized from the plans.  The first layer's maps are rebuilt once the caller's X is known.
     for (int i = 0; i < L; ++i) {
       Layer& l = n->layers[i];
-      const void* x_in = i > 0 ? n->layers[i - 1].act : l.W;       // placeholder address for layer 1
+      const void* x_in = i > 0 ? n->layers[i - 1].act : (mixed ? n->X_fc : l.W);   // placeholder address for layer 1
       const Epi ef = fwd_epi(n, i), ew = epi_sgd(l.W, l.d_in, 1, 0.f);
       st = prepare_tc(n, l.fwd, 0, B, l.d_out, l.d_in, x_in, l.d_in, l.W, l.d_in, 1, &ef);
-      if (st == MBD_OK && i > 0) {
+      if (st == MBD_OK && (i > 0 || mixed)) {
         const Epi ed = bwd_data_epi(n, i);
         st = prepare_tc(n, l.bwd_data, 1, B, l.d_in, l.d_out, l.dY, l.d_out, l.W, l.d_in, S_r, &ed);
       }
       if (st == MBD_OK) st = prepare_tc(n, l.bwd_weight, 2, l.d_out, l.d_in, B, l.dY, l.d_out, x_in, l.d_in, S_c, &ew);
       if (st != MBD_OK) { free_net(n); return st; }
       if (l.fwd.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.fwd.k_splits) * B * l.d_out);
-      if (i > 0 && l.bwd_data.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.bwd_data.k_splits) * B * l.d_in);
+      if ((i > 0 || mixed) && l.bwd_data.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.bwd_data.k_splits) * B * l.d_in);
       if (l.bwd_weight.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.bwd_weight.k_splits) * l.nW);
     }
   }
@@ -417,9 +437,9 @@ extern "C" mbd_status mbd_net_destroy(mbd_net* n) {
 }
 
 extern "C" mbd_status mbd_set_weights(mbd_net* n, int layer, const void* W_dev, const float* bias_dev) {
-  if (!n || !W_dev || layer < 0 || layer >= n->L) return MBD_E_INVALID;
-  if (n->is_conv) return conv_set_weights(n->conv, layer, W_dev);
-  Layer& l = n->layers[layer];
+  if (!n || !W_dev || layer < 0 || layer >= n->Lc + n->L) return MBD_E_INVALID;
+  if (layer < n->Lc) return bias_dev ? MBD_E_INVALID : conv_set_weights(n->conv, layer, W_dev);
+  Layer& l = n->layers[layer - n->Lc];
   CK(cudaMemcpyAsync(l.W, W_dev, l.nW * n->elt(), cudaMemcpyDeviceToDevice, n->stream));
   if (bias_dev) {
     if (!l.bias) return MBD_E_INVALID;
@@ -429,9 +449,9 @@ extern "C" mbd_status mbd_set_weights(mbd_net* n, int layer, const void* W_dev, 
 }
 
 extern "C" mbd_status mbd_get_weights(mbd_net* n, int layer, void* W_dev, float* bias_dev) {
-  if (!n || !W_dev || layer < 0 || layer >= n->L) return MBD_E_INVALID;
-  if (n->is_conv) return conv_get_weights(n->conv, layer, W_dev);
-  Layer& l = n->layers[layer];
+  if (!n || !W_dev || layer < 0 || layer >= n->Lc + n->L) return MBD_E_INVALID;
+  if (layer < n->Lc) return bias_dev ? MBD_E_INVALID : conv_get_weights(n->conv, layer, W_dev);
+  Layer& l = n->layers[layer - n->Lc];
   CK(cudaMemcpyAsync(W_dev, l.W, l.nW * n->elt(), cudaMemcpyDeviceToDevice, n->stream));
   if (bias_dev) {
     if (!l.bias) return MBD_E_INVALID;
@@ -448,9 +468,16 @@ extern "C" mbd_status mbd_forward(mbd_net* n, const void* X_dev, const int32_t* 
     return s;
   }
   if (!labels_dev) return MBD_E_INVALID;
-  n->X = X_dev;
+  mbd_status s;
+  if (n->mixed) {
+    // domain-parallel layers, then the activation leaves the strips as the [B, C*H*W] input of the model-parallel ones
+    if ((s = conv_forward(n->conv, X_dev, nullptr)) != MBD_OK) return s;
+    if ((s = conv_output_to_nchw(n->conv, n->X_fc)) != MBD_OK) return s;
+  } else {
+    n->X = X_dev;
+  }
   n->labels = labels_dev;
-  mbd_status s = map_input(n);
+  s = map_input(n);
   if (s != MBD_OK) return s;
   const int bf = n->dtype == MBD_BF16;
   for (int i = 0; i < n->L; ++i) {
@@ -515,7 +542,7 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
       n->prof.end();
       n->prof.total_launches += colsum_launches(n->B, l.d_out, n->num_sms) - 1;
     }
-    if (i > 0) {   // nothing is propagated below the first layer
+    if (i > 0 || n->mixed) {   // nothing is propagated below the first layer of the network
       const Epi e = bwd_data_epi(n, i);
       mbd_status s = run_gemm(n, l.bwd_data, 1, n->B, l.d_in, l.d_out, l.dY, l.d_out, l.W, l.d_in, S_r, e);
       if (s != MBD_OK) return s;
@@ -543,6 +570,12 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
     CK(cudaEventRecord(n->ev_join, n->aux));
     CK(cudaStreamWaitEvent(n->stream, n->ev_join, 0));
   }
+  if (n->mixed) {
+    // the gradient of the first fully connected layer's input goes back into strips and down the convolutions
+    mbd_status s = conv_top_grad_from_nchw(n->conv, n->dX_fc);
+    if (s == MBD_OK) s = conv_backward(n->conv, fused_eta);
+    if (s != MBD_OK) return s;
+  }
   n->state = fused ? ST_BWD_FUSED : ST_BWD_UNFUSED;
   return MBD_OK;
 }
@@ -556,6 +589,10 @@ extern "C" mbd_status mbd_sgd_step(mbd_net* n, float eta) {
     return s;
   }
   const float scale = -eta / static_cast<float>(n->B);
+  if (n->mixed) {
+    mbd_status s = conv_sgd_step(n->conv, eta);
+    if (s != MBD_OK) return s;
+  }
   for (int i = 0; i < n->L; ++i) {
     Layer& l = n->layers[i];
     n->prof.begin(MBD_K_SGD, static_cast<double>(l.nW) * (4.0 + 2.0 * n->elt()));
@@ -584,7 +621,7 @@ extern "C" mbd_status mbd_train_step(mbd_net* n, const void* X_dev, const int32_
   if (!same) {
     if (n->graph_exec) { cudaGraphExecDestroy(n->graph_exec); n->graph_exec = nullptr; }
     // first use of these buffers: build the tensor maps that refer to X outside the capture
-    n->X = X_dev;
+    if (!n->mixed) n->X = X_dev;
     mbd_status s = map_input(n);
     if (s != MBD_OK) return s;
     const int64_t launches_before = n->prof.total_launches;
@@ -616,9 +653,7 @@ extern "C" mbd_status mbd_train_step(mbd_net* n, const void* X_dev, const int32_
 extern "C" mbd_status mbd_train_step_host(mbd_net* n, const void* X_host, const int32_t* labels_host, float eta,
                                           float* loss_host) {
   if (!n || !X_host || !loss_host || eta <= 0.f) return MBD_E_INVALID;
-  size_t x_bytes;
-  if (n->is_conv) x_bytes = conv_input_bytes(n->conv);
-  else x_bytes = static_cast<size_t>(n->B) * n->layers[0].d_in * n->elt();
+  const size_t x_bytes = n->conv ? conv_input_bytes(n->conv) : static_cast<size_t>(n->B) * n->layers[0].d_in * n->elt();
   if (!n->X_stage) {
     mbd_status s = dev_alloc(&n->X_stage, x_bytes);
     if (s != MBD_OK) return s;
@@ -639,7 +674,7 @@ extern "C" mbd_status mbd_train_step_host(mbd_net* n, const void* X_host, const 
 
 namespace {
 size_t input_bytes(const mbd_net* n) {
-  return n->is_conv ? conv_input_bytes(n->conv) : static_cast<size_t>(n->B) * n->layers[0].d_in * n->elt();
+  return n->conv ? conv_input_bytes(n->conv) : static_cast<size_t>(n->B) * n->layers[0].d_in * n->elt();
 }
 
 mbd_status pipe_setup(mbd_net* n) {
@@ -703,6 +738,10 @@ extern "C" mbd_status mbd_train_step_host_end(mbd_net* n, float* loss_host) {
 extern "C" mbd_status mbd_get_tensor(mbd_net* n, int which, int layer, void* dst, size_t bytes) {
   if (!n || !dst) return MBD_E_INVALID;
   if (n->is_conv) return conv_get_tensor(n->conv, which, layer, dst, bytes);
+  if (n->mixed && which != MBD_T_LOSS && which != MBD_T_PARTIALS) {
+    if (layer >= 0 && layer < n->Lc) return conv_get_tensor(n->conv, which, layer, dst, bytes);
+    layer -= n->Lc;
+  }
   const void* src = nullptr;
   size_t size = 0;
   if (which == MBD_T_LOSS) {
@@ -730,6 +769,16 @@ extern "C" mbd_status mbd_get_tensor(mbd_net* n, int which, int layer, void* dst
 extern "C" mbd_status mbd_set_tensor(mbd_net* n, int which, int layer, const void* src, size_t bytes) {
   if (!n || !src) return MBD_E_INVALID;
   if (n->is_conv) return conv_set_tensor(n->conv, which, layer, src, bytes);
+  if (n->mixed) {
+    if (layer >= 0 && layer < n->Lc) {
+      const mbd_status s = conv_set_tensor(n->conv, which, layer, src, bytes);
+      // the last convolution's stored output is also the first fully connected layer's input
+      if (s == MBD_OK && which == MBD_T_ACT && layer == n->Lc - 1)
+        CK(cudaMemcpyAsync(n->X_fc, src, bytes, cudaMemcpyDeviceToDevice, n->stream));
+      return s;
+    }
+    layer -= n->Lc;
+  }
   if (layer < 0 || layer >= n->L) return MBD_E_INVALID;
   Layer& l = n->layers[layer];
   const bool last = layer == n->L - 1;

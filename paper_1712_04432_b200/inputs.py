@@ -45,8 +45,8 @@ def bits_to_f32(bits: np.ndarray) -> np.ndarray:
 @dataclass
 class Workload:
     name: str
-    kind: str                      # "fc" or "conv"
-    dims: Tuple[int, ...]          # fc: d_0..d_L ; conv: (C, H, W) with C_in == C_out
+    kind: str                      # "fc", "conv" or "mixed" (convolutions, then fully connected layers)
+    dims: Tuple[int, ...]          # fc: d_0..d_L ; conv, mixed: (C, H, W) with C_in == C_out
     B: int
     dtype: str                     # "f32" or "bf16"
     x_dist: str                    # "normal" or "relu_normal"
@@ -54,9 +54,12 @@ class Workload:
     eta: float = 0.01
     n_layers: int = 0
     grids: List[Tuple[int, int]] = field(default_factory=list)
+    fc_dims: Tuple[int, ...] = ()  # mixed: C*H*W -> ... -> classes above the n_layers convolutions
 
     @property
     def L(self) -> int:
+        if self.kind == "mixed":
+            return self.n_layers + len(self.fc_dims) - 1
         return self.n_layers if self.kind == "conv" else len(self.dims) - 1
 
 
@@ -75,6 +78,20 @@ WORKLOADS = {
 }
 
 
+def mixed_workload(C, H, W, n_conv, fc_dims, B, name="custom_mixed", grids=()) -> "Workload":
+    """n_conv 3x3 convolutions C -> C on H x W images, then a fully connected stack
+    C*H*W -> fc_dims[0] -> ... -> fc_dims[-1] with softmax cross-entropy."""
+    d = (int(C) * int(H) * int(W),) + tuple(int(x) for x in fc_dims)
+    return Workload(name, "mixed", (int(C), int(H), int(W)), int(B), "bf16", "normal", "softmax_ce",
+                    n_layers=int(n_conv), grids=list(grids), fc_dims=d)
+
+
+# Beyond the five configurations: the integrated network of Section 2.4 in miniature (convolutions on
+# row strips, a classifier head on row blocks of its matrices, one grid for both).
+WORKLOADS["mixed"] = mixed_workload(64, 56, 56, 2, (1024, 1024, 1000), 256, name="mixed",
+                                    grids=[(1, 1), (4, 4), (8, 1), (2, 8)])
+
+
 def fc_workload(dims, B, dtype="bf16", x_dist="normal", name="custom") -> Workload:
     return Workload(name, "fc", tuple(int(d) for d in dims), int(B), dtype, x_dist, "softmax_ce")
 
@@ -86,9 +103,9 @@ def conv_workload(C, H, W, B, n_layers=2, dtype="bf16", name="custom_conv") -> W
 
 @dataclass
 class Inputs:
-    X: np.ndarray                    # fc: [B, d_0] ; conv: [B, C, H, W]   (float32 values)
-    Ws: List[np.ndarray]             # fc: [d_i, d_{i-1}] ; conv: [C_out, C_in, 3, 3]
-    bs: List[Optional[np.ndarray]]   # zeros (fc) or None (conv)
+    X: np.ndarray                    # fc: [B, d_0] ; conv, mixed: [B, C, H, W]   (float32 values)
+    Ws: List[np.ndarray]             # fc: [d_i, d_{i-1}] ; conv: [C_out, C_in, 3, 3] ; mixed: the kernels, then the matrices
+    bs: List[Optional[np.ndarray]]   # zeros (fc layers) or None (conv layers)
     labels: Optional[np.ndarray]     # int32 [B] or None
 
 
@@ -118,12 +135,23 @@ def make_inputs(w: Workload, seed: int = 0) -> Inputs:
         K = rng.standard_normal((C, C, 3, 3), dtype=np.float32)
         K *= np.float32(np.sqrt(2.0 / (9 * C)))                  # N(0, 2/(9 C))
         Ws.append(rnd(K))
-    return Inputs(X, Ws, [None] * w.n_layers, None)
+    bs: List[Optional[np.ndarray]] = [None] * w.n_layers
+    if w.kind != "mixed":
+        return Inputs(X, Ws, bs, None)
+    d = w.fc_dims
+    for i in range(1, len(d)):
+        Wi = rng.standard_normal((d[i], d[i - 1]), dtype=np.float32)
+        Wi *= np.float32(1.0 / np.sqrt(d[i - 1]))
+        Ws.append(rnd(Wi))
+        bs.append(np.zeros(d[i], np.float32))
+    labels = rng.integers(0, d[-1], size=w.B, dtype=np.int64).astype(np.int32)
+    return Inputs(X, Ws, bs, labels)
 
 
 def step_flops(w: Workload) -> int:
     """2 x MACs of the dense contractions one step needs: forward and
-    backward-weight for every layer, backward-data for layers 2..L."""
+    backward-weight for every layer, backward-data for layers 2..L (layer 1 is the
+    first layer of the whole network)."""
     if w.kind == "fc":
         d = w.dims
         macs = 0
@@ -133,4 +161,8 @@ def step_flops(w: Workload) -> int:
         return 2 * macs
     C, H, Wd = w.dims
     per = w.B * H * Wd * C * C * 9
-    return 2 * per * (3 * w.n_layers - 1)
+    macs = per * (3 * w.n_layers - 1)
+    if w.kind == "mixed":
+        d = w.fc_dims
+        macs += sum(3 * w.B * d[i] * d[i - 1] for i in range(1, len(d)))
+    return 2 * macs

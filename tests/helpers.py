@@ -140,23 +140,25 @@ def compare_fc_step(g, o, tol, fused=False, tol_below_relu=None):
 # ---------------------------------------------------------------------------
 # convolution workloads
 # ---------------------------------------------------------------------------
-def oracle_conv_step(w, inp, strips=None):
+def oracle_conv_step(w, inp, strips=None, grid=None):
     """fp64 oracle step for a domain-parallel conv workload (NCHW); stored activations are
-    rounded to bf16 like the device's.  `strips` = P_r runs the strip / halo formulation."""
+    rounded to bf16 like the device's.  `strips` = P_r (or `grid` = (P_r, P_c)) runs the
+    strip / halo formulation."""
     from oracle import mbd_oracle as O
     layers = [O.Conv3x3(k.astype(np.float64), relu=True) for k in inp.Ws]
     X = inp.X.astype(np.float64)
-    if strips is None:
+    if strips is None and grid is None:
         return O.train_step(layers, X, None, "half_ssq", w.eta, store=bf16_store)
-    return O.train_step_blocked(layers, X, None, "half_ssq", w.eta, strips, 1, store=bf16_store)
+    P_r, P_c = grid if grid is not None else (strips, 1)
+    return O.train_step_blocked(layers, X, None, "half_ssq", w.eta, P_r, P_c, store=bf16_store)
 
 
-def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None):
+def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1):
     import torch
     from paper_1712_04432_b200 import mbd
     C_, H, Wd = w.dims
     L = w.n_layers
-    net = mbd.Net(mbd.conv_layers(L, C_, H, Wd), w.B, P_r, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+    net = mbd.Net(mbd.conv_layers(L, C_, H, Wd), w.B, P_r, P_c, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
     for i in range(L):
         net.set_weights(i, to_dev(inp.Ws[i], True))
     X = to_dev(inp.X, True)
@@ -202,5 +204,124 @@ def compare_conv_step(g, o, tol, fused=False, tol_below_relu=None):
         if not fused:
             chk(f"dK[{i}]", g["dW"][i], o["dWs"][i], tg)
         chk(f"K_new[{i}]", g["new_W"][i], o["new_W"][i], tol)
+    assert not bad, "rel. Frobenius error too large for %s: %s" % (bad, "; ".join(report))
+    return report
+
+
+# ---------------------------------------------------------------------------
+# convolutions followed by fully connected layers (Section 2.4)
+# ---------------------------------------------------------------------------
+def oracle_mixed_step(w, inp, blocked_grid=None):
+    """fp64 oracle step of a mixed workload: Conv3x3 layers on NCHW, then FC layers on the
+    flattened activation; stored activations rounded to bf16 like the device's."""
+    from oracle import mbd_oracle as O
+    Lc = w.n_layers
+    layers = [O.Conv3x3(inp.Ws[i].astype(np.float64), relu=True) for i in range(Lc)]
+    for i in range(Lc, w.L):
+        layers.append(O.FC(inp.Ws[i].astype(np.float64), inp.bs[i].astype(np.float64), relu=True))
+    X = inp.X.astype(np.float64)
+    if blocked_grid is None:
+        return O.train_step(layers, X, inp.labels, "softmax_ce", w.eta, store=bf16_store)
+    return O.train_step_blocked(layers, X, inp.labels, "softmax_ce", w.eta, *blocked_grid, store=bf16_store)
+
+
+def mixed_layers(w):
+    from paper_1712_04432_b200 import mbd
+    C_, H, Wd = w.dims
+    return mbd.conv_layers(w.n_layers, C_, H, Wd) + mbd.fc_layers(w.fc_dims, bias=True)
+
+
+def oracle_mixed_acts(o, w):
+    """The oracle's stored hidden activations in the device's layouts: NCHW for the outputs of
+    the convolutions, [B, d] for the outputs of the hidden fully connected layers."""
+    C_, H, Wd = w.dims
+    out = []
+    for i in range(w.L - 1):
+        x = o["Xs"][i + 1]
+        if i < w.n_layers:
+            x = x if x.ndim == 4 else np.ascontiguousarray(x.T).reshape(w.B, C_, H, Wd)
+        else:
+            x = x.T
+        out.append(np.ascontiguousarray(x, np.float32))
+    return out
+
+
+def gpu_mixed_step(w, inp, grid=(1, 1), max_partials=0, fused=False, force_acts=None):
+    """The same step through the C ABI; conv tensors come back NCHW, FC tensors [B, d]."""
+    import torch
+    from paper_1712_04432_b200 import mbd
+    L, Lc = w.L, w.n_layers
+    net = mbd.Net(mixed_layers(w), w.B, grid[0], grid[1], mbd.BF16, mbd.LOSS_SOFTMAX_CE, max_partials)
+    for i in range(L):
+        if i < Lc:
+            net.set_weights(i, to_dev(inp.Ws[i], True))
+        else:
+            net.set_weights(i, to_dev(inp.Ws[i], True), torch.from_numpy(inp.bs[i]).cuda())
+    X = to_dev(inp.X, True)
+    labels = torch.from_numpy(inp.labels).cuda()
+    J = torch.zeros(1, dtype=torch.float32, device="cuda")
+    out = {}
+    net.forward(X, labels, J)
+    out["act"] = [to_np(net.get_tensor(mbd.T_ACT, i)) for i in range(L)]
+    if force_acts is not None:
+        for i in range(L - 1):
+            net.set_tensor(mbd.T_ACT, i, to_dev(force_acts[i], True))
+    if fused:
+        net.backward(w.eta)
+    else:
+        net.backward(0.0)
+        out["dW"] = [to_np(net.get_tensor(mbd.T_DW, i)) for i in range(L)]
+        out["db"] = [to_np(net.get_tensor(mbd.T_DB, i)) if i >= Lc else None for i in range(L)]
+        net.sgd_step(w.eta)
+    net.poll()
+    out["J"] = float(J.item())
+    out["loss"] = to_np(net.get_tensor(mbd.T_LOSS))
+    out["dY"] = [to_np(net.get_tensor(mbd.T_DY, i)) for i in range(L)]
+    out["new_W"], out["new_b"] = [], []
+    for i in range(L):
+        if i < Lc:
+            out["new_W"].append(to_np(net.get_weights(i))); out["new_b"].append(None)
+        else:
+            a, b = net.get_weights(i, with_bias=True)
+            out["new_W"].append(to_np(a)); out["new_b"].append(to_np(b))
+    out["launches"] = net.launch_count
+    net.close()
+    return out
+
+
+def compare_mixed_step(g, o, w, tol, fused=False, tol_below_relu=None):
+    L, Lc = w.L, w.n_layers
+    C_, H, Wd = w.dims
+    report, bad = [], []
+    if tol_below_relu is None:
+        tol_below_relu = tol
+
+    def chk(name, got, ref, t):
+        e = rel_fro(got, ref)
+        report.append(f"{name}: {e:.3e}")
+        if e > t:
+            bad.append(name)
+
+    def dev_layout(a, i):
+        """oracle tensor of layer i's output side -> the device's layout"""
+        if i < Lc:
+            return a if a.ndim == 4 else np.ascontiguousarray(a.T).reshape(w.B, C_, H, Wd)
+        return a.T
+
+    assert abs(g["J"] - o["J"]) <= max(tol, 1e-4) * abs(o["J"]), (g["J"], o["J"])
+    chk("per-sample loss", g["loss"], o["per_sample"], tol)
+    for i in range(L):
+        ref_act = o["Ys"][i] if i == L - 1 else o["Xs"][i + 1]
+        chk(f"Y[{i}]", g["act"][i], dev_layout(ref_act, i), tol)
+        tg = tol if i == L - 1 else tol_below_relu
+        chk(f"dY[{i}]", g["dY"][i], dev_layout(o["dYs"][i], i), tg)
+        if not fused:
+            chk(f"dW[{i}]", g["dW"][i], o["dWs"][i], tg)
+            if i >= Lc:
+                chk(f"db[{i}]", g["db"][i], o["dbs"][i], tg)
+        chk(f"W_new[{i}]", g["new_W"][i], o["new_W"][i], tol)
+        if i >= Lc:
+            ref_b = o["new_b"][i]
+            assert np.abs(g["new_b"][i] - ref_b).max() <= tol * max(1.0, np.abs(ref_b).max()), f"b_new[{i}]"
     assert not bad, "rel. Frobenius error too large for %s: %s" % (bad, "; ".join(report))
     return report

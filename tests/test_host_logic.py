@@ -24,7 +24,7 @@ def test_grid_errors():
     assert create(fc, 8, 17, 1) == mbd.E_GRID         # more row blocks than neurons of the last layer
     conv = mbd.conv_layers(2, 64, 8, 16)
     assert create(conv, 4, 9, 1, loss=mbd.LOSS_HALF_SSQ) == mbd.E_GRID    # strips shorter than one row
-    assert create(conv, 4, 2, 2, loss=mbd.LOSS_HALF_SSQ) == mbd.E_GRID    # batch split with a domain layer
+    assert create(conv, 4, 2, 5, loss=mbd.LOSS_HALF_SSQ) == mbd.E_GRID    # more batch blocks than samples
 
 
 def test_invalid_and_unsupported():
@@ -39,6 +39,12 @@ def test_invalid_and_unsupported():
     conv5[0].kh = conv5[0].kw = 5
     assert create(conv5, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
     assert create(mbd.conv_layers(1, 64, 8, 16), 4, loss=mbd.LOSS_SOFTMAX_CE) == mbd.E_UNSUPPORTED
+    # convolutions first, fully connected layers after them
+    conv = mbd.conv_layers(1, 64, 8, 16)
+    assert create(mbd.fc_layers((64, 64 * 8 * 16)) + conv, 4) == mbd.E_UNSUPPORTED          # convolution above an FC layer
+    assert create(conv + mbd.fc_layers((64 * 8 * 16 - 8, 16)), 4) == mbd.E_INVALID          # d_in is not C*H*W
+    assert create(conv + mbd.fc_layers((64 * 8 * 16, 16)), 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
+    assert create(conv + mbd.fc_layers((64 * 8 * 16, 16)), 4, dtype=mbd.F32) == mbd.E_UNSUPPORTED
 
 
 def test_null_handles_are_rejected():

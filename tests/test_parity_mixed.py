@@ -1,0 +1,117 @@
+"""Parity of the integrated step of Section 2.4 (domain-parallel 3x3 convolutions first,
+model-parallel fully connected layers after them, one P_r x P_c grid for both, Eq. 9) with
+the fp64 oracle, through the C ABI; and of convolution stacks whose batch is split as well."""
+import numpy as np
+import pytest
+
+from paper_1712_04432_b200 import inputs as I
+from tests.helpers import (compare_conv_step, compare_mixed_step, gpu_conv_step, gpu_mixed_step, oracle_conv_step,
+                           oracle_mixed_acts, oracle_mixed_step, rel_fro)
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+TOL_FREE = 5e-2      # free-running gradients below a ReLU (see test_parity_fc.py)
+
+
+@pytest.fixture(scope="module")
+def small():
+    # 2 convolutions on 8 x 40 images (one ragged 40-pixel segment), then 20480 -> 256 -> 24
+    w = I.mixed_workload(64, 8, 40, 2, (256, 24), 6, name="mixed_small")
+    inp = I.make_inputs(w, seed=31)
+    return w, inp, oracle_mixed_step(w, inp)
+
+
+@pytest.mark.parametrize("grid", [(1, 1), (2, 1), (1, 3), (2, 3), (4, 2), (8, 6)])
+def test_small_all_grids(small, grid):
+    w, inp, o = small
+    g = gpu_mixed_step(w, inp, grid, force_acts=oracle_mixed_acts(o, w))
+    compare_mixed_step(g, o, w, TOL)
+    g = gpu_mixed_step(w, inp, grid)
+    compare_mixed_step(g, o, w, TOL, tol_below_relu=TOL_FREE)
+
+
+@pytest.mark.parametrize("grid,max_partials", [((1, 1), 1), ((2, 2), 4), ((4, 2), 2)])
+def test_small_fused_update(small, grid, max_partials):
+    w, inp, o = small
+    g = gpu_mixed_step(w, inp, grid, max_partials, fused=True, force_acts=oracle_mixed_acts(o, w))
+    compare_mixed_step(g, o, w, TOL, fused=True)
+
+
+def test_blocked_oracle_agrees(small):
+    w, inp, _ = small
+    ob = oracle_mixed_step(w, inp, blocked_grid=(4, 3))
+    g = gpu_mixed_step(w, inp, (4, 3), 4, force_acts=oracle_mixed_acts(ob, w))
+    compare_mixed_step(g, ob, w, TOL)
+
+
+def test_one_convolution_three_fc_layers_ragged():
+    # 28 rows (strips of 7), 130 pixels per row (two forward segments), 5 samples; FC 232960 -> 64 -> 32 -> 16
+    w = I.mixed_workload(64, 28, 130, 1, (64, 32, 16), 5, name="mixed_ragged")
+    inp = I.make_inputs(w, seed=32)
+    o = oracle_mixed_step(w, inp)
+    for grid in [(1, 1), (4, 5)]:
+        g = gpu_mixed_step(w, inp, grid, force_acts=oracle_mixed_acts(o, w))
+        compare_mixed_step(g, o, w, TOL)
+
+
+def test_train_step_graph_matches_separate_calls(small):
+    """mbd_train_step (captured graph, fused update) leaves the same weights, bit for bit, as
+    forward + backward(eta) issued one by one; and two steps change them twice."""
+    import torch
+    from paper_1712_04432_b200 import mbd
+    from tests.helpers import mixed_layers, to_dev
+    w, inp, _ = small
+    outs = []
+    for mode in ("calls", "graph"):
+        net = mbd.Net(mixed_layers(w), w.B, 2, 3, mbd.BF16, mbd.LOSS_SOFTMAX_CE, 0)
+        for i in range(w.L):
+            bias = None if i < w.n_layers else torch.from_numpy(inp.bs[i]).cuda()
+            net.set_weights(i, to_dev(inp.Ws[i], True), bias)
+        X = to_dev(inp.X, True)
+        labels = torch.from_numpy(inp.labels).cuda()
+        J = torch.zeros(1, dtype=torch.float32, device="cuda")
+        losses = []
+        for _ in range(2):
+            if mode == "calls":
+                net.forward(X, labels, J)
+                net.backward(w.eta)
+            else:
+                net.train_step(X, labels, w.eta, J)
+            net.poll()
+            losses.append(float(J.item()))
+        outs.append((losses, [net.get_weights(i).clone() for i in range(w.L)]))
+        net.close()
+    assert outs[0][0] == outs[1][0]
+    for a, b in zip(outs[0][1], outs[1][1]):
+        assert torch.equal(a, b)
+    assert outs[0][0][1] != outs[0][0][0]
+
+
+def test_host_step_of_a_mixed_stack(small):
+    import torch
+    from paper_1712_04432_b200 import mbd
+    from tests.helpers import mixed_layers, to_dev
+    w, inp, o = small
+    net = mbd.Net(mixed_layers(w), w.B, 2, 2, mbd.BF16, mbd.LOSS_SOFTMAX_CE, 0)
+    for i in range(w.L):
+        bias = None if i < w.n_layers else torch.from_numpy(inp.bs[i]).cuda()
+        net.set_weights(i, to_dev(inp.Ws[i], True), bias)
+    Xh = to_dev(inp.X, True).cpu().pin_memory()
+    lh = torch.from_numpy(inp.labels).pin_memory()
+    J = net.train_step_host(Xh, lh, w.eta)
+    net.poll()
+    assert abs(J - o["J"]) <= 1e-2 * abs(o["J"])
+    for i in range(w.L):
+        assert rel_fro(net.get_weights(i).float().cpu().numpy(), o["new_W"][i]) <= TOL
+    net.close()
+
+
+# ------------------------------------------------------------------ convolutions with a split batch
+@pytest.mark.parametrize("grid", [(1, 2), (2, 3), (4, 2)])
+def test_conv_stack_with_batch_blocks(grid):
+    w = I.conv_workload(64, 8, 40, 6, name="conv_pc")
+    inp = I.make_inputs(w, seed=33)
+    o = oracle_conv_step(w, inp, grid=grid)
+    hidden = [np.ascontiguousarray(x, np.float32) for x in o["Xs"][1:]]
+    g = gpu_conv_step(w, inp, grid[0], P_c=grid[1], force_acts=hidden)
+    compare_conv_step(g, o, TOL)
