@@ -68,23 +68,25 @@ constexpr int NUM_THREADS = 192;
 enum { MODE_RELU_STORE = 0, MODE_STORE_SSQ = 1, MODE_MASK = 2 };
 
 // ------------------------------------------------------------------------------ layout kernels
-// NCHW -> strips.  Block = (32-pixel segment, image row h, image b); 128 threads.  A row that
-// borders another strip is also written into that neighbour's halo row: this is the forward
-// halo exchange for the network input, fused into the staging pass.
+// NCHW -> strips.  Block = 32 consecutive pixels of one image's flattened (h, w) plane (so narrow
+// images fill their blocks too), all 64 channels; 128 threads.  A row that borders another strip is
+// also written into that neighbour's halo row: this is the forward halo exchange for the network
+// input (and the backward one for a gradient that arrives from above), fused into the staging pass.
 __global__ void __launch_bounds__(128)
 nchw_to_strips_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int H, int W, int P_r, int Hs) {
-  // 32 pixels x 64 channels per block; shared memory holds channel PAIRS as 32-bit words,
-  // [pixel][pair] with an odd pitch, so both phases are free of bank conflicts.
+  // shared memory holds channel PAIRS as 32-bit words, [pixel][pair] with an odd pitch, so both
+  // phases are free of bank conflicts.
   __shared__ uint32_t tile[32][33];
-  const int w0 = blockIdx.x * 32, h = blockIdx.y, b = blockIdx.z;
+  const int HW = H * W;
+  const int p0 = blockIdx.x * 32, b = blockIdx.y;
   const int t = threadIdx.x;
   {
-    const int cp = t >> 2, wq = (t & 3) * 8;          // channels 2cp, 2cp+1; pixels wq..wq+7
-    const bf16* p0 = src + ((static_cast<int64_t>(b) * C + 2 * cp) * H + h) * W + w0 + wq;
-    const bf16* p1 = p0 + static_cast<int64_t>(H) * W;
+    const int cp = t >> 2, wq = (t & 3) * 8;          // channels 2cp, 2cp+1; pixels p0+wq .. p0+wq+7
+    const bf16* q0 = src + (static_cast<int64_t>(b) * C + 2 * cp) * HW + p0 + wq;
+    const bf16* q1 = q0 + HW;
     uint16_t lo[8], hi[8];
-    if ((W & 7) == 0 && w0 + wq + 8 <= W) {
-      const uint4 a = __ldcs(reinterpret_cast<const uint4*>(p0)), c = __ldcs(reinterpret_cast<const uint4*>(p1));
+    if ((HW & 7) == 0 && p0 + wq + 8 <= HW) {
+      const uint4 a = __ldcs(reinterpret_cast<const uint4*>(q0)), c = __ldcs(reinterpret_cast<const uint4*>(q1));
       const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -94,24 +96,26 @@ nchw_to_strips_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int 
     } else {
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const bool in = w0 + wq + i < W;
-        lo[i] = in ? __bfloat16_as_ushort(p0[i]) : 0;
-        hi[i] = in ? __bfloat16_as_ushort(p1[i]) : 0;
+        const bool in = p0 + wq + i < HW;
+        lo[i] = in ? __bfloat16_as_ushort(q0[i]) : 0;
+        hi[i] = in ? __bfloat16_as_ushort(q1[i]) : 0;
       }
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) tile[wq + i][cp] = static_cast<uint32_t>(lo[i]) | (static_cast<uint32_t>(hi[i]) << 16);
   }
   __syncthreads();
-  const int px = t >> 2, cq = (t & 3) * 8;            // 8 words = channels 2cq .. 2cq+15 of pixel px
-  if (w0 + px >= W) return;
+  const int px = t >> 2, cq = (t & 3) * 8;            // 8 words = channels 2cq .. 2cq+15 of pixel p0+px
+  const int p = p0 + px;
+  if (p >= HW) return;
   uint4 v0, v1;
   v0.x = tile[px][cq + 0]; v0.y = tile[px][cq + 1]; v0.z = tile[px][cq + 2]; v0.w = tile[px][cq + 3];
   v1.x = tile[px][cq + 4]; v1.y = tile[px][cq + 5]; v1.z = tile[px][cq + 6]; v1.w = tile[px][cq + 7];
   const int R = Hs + 2;
+  const int h = p / W, w = p - h * W;
   const int s = h / Hs, r = h - s * Hs + 1;
   auto put = [&](int ss, int rr) {
-    bf16* q = dst + (((static_cast<int64_t>(b) * P_r + ss) * R + rr) * W + (w0 + px)) * C + 2 * cq;
+    bf16* q = dst + (((static_cast<int64_t>(b) * P_r + ss) * R + rr) * W + w) * C + 2 * cq;
     *reinterpret_cast<uint4*>(q) = v0;
     *reinterpret_cast<uint4*>(q + 8) = v1;
   };
@@ -120,28 +124,51 @@ nchw_to_strips_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int 
   if (r == Hs && s < P_r - 1) put(s + 1, 0);        // last row of a strip: upper halo of the strip below
 }
 
-// strips -> NCHW (read-back only).
-__global__ void __launch_bounds__(256)
+// strips -> NCHW: the mirror image (own rows only).  Used to hand the last convolution's output to the
+// fully connected layers above it, and for read-back.
+__global__ void __launch_bounds__(128)
 strips_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int H, int W, int P_r, int Hs) {
-  __shared__ bf16 tile[32][C + 2];
-  const int w0 = blockIdx.x * 32, h = blockIdx.y, b = blockIdx.z;
+  __shared__ uint32_t tile[32][33];
+  const int HW = H * W;
+  const int p0 = blockIdx.x * 32, b = blockIdx.y;
   const int t = threadIdx.x;
   const int R = Hs + 2;
-  const int s = h / Hs, r = h - s * Hs + 1;
   {
-    const int px = t >> 3, cq = (t & 7) * 8;
-    if (w0 + px < W) {
-      const bf16* q = src + (((static_cast<int64_t>(b) * P_r + s) * R + r) * W + (w0 + px)) * C + cq;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) tile[px][cq + i] = q[i];
+    const int px = t >> 2, cq = (t & 3) * 8;
+    const int p = p0 + px;
+    if (p < HW) {
+      const int h = p / W, w = p - h * W;
+      const int s = h / Hs, r = h - s * Hs + 1;
+      const bf16* q = src + (((static_cast<int64_t>(b) * P_r + s) * R + r) * W + w) * C + 2 * cq;
+      const uint4 v0 = *reinterpret_cast<const uint4*>(q), v1 = *reinterpret_cast<const uint4*>(q + 8);
+      tile[px][cq + 0] = v0.x; tile[px][cq + 1] = v0.y; tile[px][cq + 2] = v0.z; tile[px][cq + 3] = v0.w;
+      tile[px][cq + 4] = v1.x; tile[px][cq + 5] = v1.y; tile[px][cq + 6] = v1.z; tile[px][cq + 7] = v1.w;
     }
   }
   __syncthreads();
-  const int c = t >> 2, wq = (t & 3) * 8;
-  bf16* p = dst + ((static_cast<int64_t>(b) * C + c) * H + h) * W + w0 + wq;
+  const int cp = t >> 2, wq = (t & 3) * 8;            // channels 2cp, 2cp+1; pixels p0+wq .. p0+wq+7
+  if (p0 + wq >= HW) return;
+  uint32_t word[8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
-    if (w0 + wq + i < W) p[i] = tile[wq + i][c];
+  for (int i = 0; i < 8; ++i) word[i] = tile[wq + i][cp];
+  bf16* q0 = dst + (static_cast<int64_t>(b) * C + 2 * cp) * HW + p0 + wq;
+  bf16* q1 = q0 + HW;
+  if ((HW & 7) == 0 && p0 + wq + 8 <= HW) {
+    uint4 a, c;
+    a.x = (word[0] & 0xFFFFu) | (word[1] << 16); a.y = (word[2] & 0xFFFFu) | (word[3] << 16);
+    a.z = (word[4] & 0xFFFFu) | (word[5] << 16); a.w = (word[6] & 0xFFFFu) | (word[7] << 16);
+    c.x = (word[0] >> 16) | (word[1] & 0xFFFF0000u); c.y = (word[2] >> 16) | (word[3] & 0xFFFF0000u);
+    c.z = (word[4] >> 16) | (word[5] & 0xFFFF0000u); c.w = (word[6] >> 16) | (word[7] & 0xFFFF0000u);
+    *reinterpret_cast<uint4*>(q0) = a;
+    *reinterpret_cast<uint4*>(q1) = c;
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (p0 + wq + i < HW) {
+        q0[i] = __ushort_as_bfloat16(static_cast<uint16_t>(word[i] & 0xFFFFu));
+        q1[i] = __ushort_as_bfloat16(static_cast<uint16_t>(word[i] >> 16));
+      }
+  }
 }
 
 // Halo exchange between neighbouring strips of one tensor: the last own row of strip s becomes
@@ -778,7 +805,7 @@ void launch_halo(ConvNet* c, bf16* buf) {
 }
 
 void launch_stage_in(ConvNet* c, const bf16* nchw, bf16* strips) {
-  dim3 g((c->W + 31) / 32, c->H, static_cast<unsigned>(c->B));
+  dim3 g((c->H * c->W + 31) / 32, static_cast<unsigned>(c->B));
   c->prof->begin(MBD_K_HALO, 2.0 * c->B * C * c->H * c->W * 2.0);
   nchw_to_strips_kernel<<<g, 128, 0, c->stream>>>(nchw, strips, c->H, c->W, c->P_r, c->Hs);
   c->prof->end();
@@ -792,6 +819,7 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   if (conv_init() != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
   const int H = layers[0].H, W = layers[0].W;
   if (H % P_r != 0) return MBD_E_UNSUPPORTED;      // strips of equal height only
+  if (B > 65535 || static_cast<int64_t>(H) * W > INT32_MAX) return MBD_E_UNSUPPORTED;   // grid.y of the staging kernels
   ConvNet* c = new (std::nothrow) ConvNet();
   if (!c) return MBD_E_ALLOC;
   c->L = L; c->B = B; c->H = H; c->W = W; c->P_r = P_r; c->Hs = H / P_r; c->R = c->Hs + 2; c->Z = B * P_r;
@@ -924,9 +952,9 @@ mbd_status conv_sgd_step(ConvNet* c, float eta) {
 // convolution's output become the [B, C*H*W] matrix (NCHW order) the first fully connected layer reads,
 // and that layer's input gradient goes back into strips, its boundary rows also into the neighbours' halos.
 mbd_status conv_output_to_nchw(ConvNet* c, void* dst) {
-  dim3 g((c->W + 31) / 32, c->H, static_cast<unsigned>(c->B));
+  dim3 g((c->H * c->W + 31) / 32, static_cast<unsigned>(c->B));
   c->prof->begin(MBD_K_HALO, 2.0 * c->B * C * c->H * c->W * 2.0);
-  strips_to_nchw_kernel<<<g, 256, 0, c->stream>>>(c->act[c->L], static_cast<bf16*>(dst), c->H, c->W, c->P_r, c->Hs);
+  strips_to_nchw_kernel<<<g, 128, 0, c->stream>>>(c->act[c->L], static_cast<bf16*>(dst), c->H, c->W, c->P_r, c->Hs);
   c->prof->end();
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
@@ -954,8 +982,8 @@ mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t b
   if (layer < 0 || layer >= c->L || bytes != nchw_bytes) return MBD_E_INVALID;
   const bf16* src = which == MBD_T_ACT ? c->act[layer + 1] : which == MBD_T_DY ? c->dY[layer] : nullptr;
   if (!src) return MBD_E_INVALID;
-  dim3 g((c->W + 31) / 32, c->H, static_cast<unsigned>(c->B));
-  strips_to_nchw_kernel<<<g, 256, 0, c->stream>>>(src, static_cast<bf16*>(dst), c->H, c->W, c->P_r, c->Hs);
+  dim3 g((c->H * c->W + 31) / 32, static_cast<unsigned>(c->B));
+  strips_to_nchw_kernel<<<g, 128, 0, c->stream>>>(src, static_cast<bf16*>(dst), c->H, c->W, c->P_r, c->Hs);
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
@@ -963,7 +991,7 @@ mbd_status conv_set_tensor(ConvNet* c, int which, int layer, const void* src, si
   if (layer < 0 || layer >= c->L || bytes != conv_input_bytes(c)) return MBD_E_INVALID;
   bf16* dst = which == MBD_T_ACT ? c->act[layer + 1] : which == MBD_T_DY ? c->dY[layer] : nullptr;
   if (!dst) return MBD_E_INVALID;
-  dim3 g((c->W + 31) / 32, c->H, static_cast<unsigned>(c->B));
+  dim3 g((c->H * c->W + 31) / 32, static_cast<unsigned>(c->B));
   nchw_to_strips_kernel<<<g, 128, 0, c->stream>>>(static_cast<const bf16*>(src), dst, c->H, c->W, c->P_r, c->Hs);
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
