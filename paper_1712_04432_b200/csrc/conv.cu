@@ -233,7 +233,8 @@ wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ d
 // ------------------------------------------------------------------------------ forward kernel
 struct FwdParams {
   int W, Hs, R, nseg;
-  long long rows_total;   // output row segments: (strip z, segment, row) flattened with the row fastest
+  int pack, Z;            // narrow images: `pack` strips share one 128-pixel tile, 128 / pack pixels each (see below)
+  long long rows_total;   // output row segments: (strip group z, segment, row) flattened with the row fastest
   int mode;
   bf16* out;              // strips
   const bf16* mask_src;   // strips (MODE_MASK)
@@ -243,6 +244,13 @@ struct FwdParams {
 
 // A CTA owns a contiguous span of the flattened output rows and walks it as runs of rows of one
 // (strip, segment) column; a run of n output rows reads n + 2 input rows.
+//
+// Narrow images (W <= 62): a 128-pixel tile would be mostly padding, so `pack` = 2, 4 or 8 strips with
+// consecutive indices z share it.  Strip j of the group owns tile positions j*sub .. (j+1)*sub - 1,
+// sub = 128 / pack >= W + 2, and is loaded / stored by its own TMA box of `sub` pixels; its box starts at
+// pixel -1 like the wide one, so the shifted views still line up: position j*sub + i + v of the stage holds
+// pixel i + v - 1 of strip j, and what a view reads across a strip boundary only reaches outputs i >= W,
+// which are never stored.  `z` of a run is then the first strip of the group.
 struct FwdRun {
   int z, seg, h0, n;
 };
@@ -253,7 +261,7 @@ __device__ __forceinline__ FwdRun fwd_run(const FwdParams& p, long long pos, lon
   const long long left = end - pos;
   r.n = static_cast<int>(left < p.Hs - r.h0 ? left : p.Hs - r.h0);
   r.seg = static_cast<int>(col % p.nseg);
-  r.z = static_cast<int>(col / p.nseg);
+  r.z = static_cast<int>(col / p.nseg) * p.pack;
   return r;
 }
 
@@ -292,6 +300,13 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) tmem_alloc<512>(smem_u32(&tmem_base_slot));
+  if (p.pack > 1 && threadIdx.x >= 64 && threadIdx.x < 64 + FWD1_STAGES * 16) {
+    // packed stages: positions 128, 129 (read by the shifted views, written by no box) hold zeros
+    const int i = threadIdx.x - 64;
+    uint8_t* ring_gen = smem_raw + (ring - smem_u32(smem_raw));
+    *reinterpret_cast<uint4*>(ring_gen + (i >> 4) * FWD1_ROW_BYTES + FWD_PIX * 128 + (i & 15) * 16) = make_uint4(0, 0, 0, 0);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -316,8 +331,15 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
           if (!ok) break;
           const uint32_t fb = smem_u32(&full_bar[stage]);
-          mbar_expect_tx(fb, FWD1_BOX_PIX * 128);
-          tma_load_4d(ring + stage * FWD1_ROW_BYTES, &tmX, 0, run.seg * FWD_PIX - 1, run.h0 + r, run.z, fb);
+          if (p.pack == 1) {
+            mbar_expect_tx(fb, FWD1_BOX_PIX * 128);
+            tma_load_4d(ring + stage * FWD1_ROW_BYTES, &tmX, 0, run.seg * FWD_PIX - 1, run.h0 + r, run.z, fb);
+          } else {
+            const int sub_bytes = (FWD_PIX / p.pack) * 128;
+            mbar_expect_tx(fb, FWD_PIX * 128);
+            for (int j = 0; j < p.pack; ++j)      // a strip index beyond Z reads as zeros
+              tma_load_4d(ring + stage * FWD1_ROW_BYTES + j * sub_bytes, &tmX, 0, -1, run.h0 + r, run.z + j, fb);
+          }
           if (++stage == FWD1_STAGES) { stage = 0; phase ^= 1u; }
         }
         pos += run.n;
@@ -407,16 +429,19 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       auto row_coords = [&](int k, int& x0, int& row, int& z) {
         const long long pos = r0 + k;
         const long long col = pos / p.Hs;
-        z = static_cast<int>(col / p.nseg);
+        z = static_cast<int>(col / p.nseg) * p.pack;
         x0 = static_cast<int>(col % p.nseg) * FWD_PIX;
         row = static_cast<int>(pos - col * p.Hs) + 1;
       };
+      const int sub = FWD_PIX / p.pack;                   // tile positions per strip
+      const int sub_bytes = sub * 128;
       auto load_mask = [&](int k) {
         int x0, row, z;
         row_coords(k, x0, row, z);
         const uint32_t mb = smem_u32(&mask_full_bar[k & 1]);
         mbar_expect_tx(mb, FWD_TILE_BYTES);
-        tma_load_4d(stg_mask + (k & 1) * FWD_TILE_BYTES, &tmMask, 0, x0, row, z, mb);
+        for (int j = 0; j < p.pack; ++j)
+          tma_load_4d(stg_mask + (k & 1) * FWD_TILE_BYTES + j * sub_bytes, &tmMask, 0, x0, row, z + j, mb);
       };
       if (use_mask && issuer) {
         if (n_rows > 0) load_mask(0);
@@ -427,7 +452,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const int buf = g & 1;
         int x0, row, z;
         row_coords(g, x0, row, z);
-        const bool valid = x0 + pl < p.W;
+        const bool valid = p.pack == 1 ? x0 + pl < p.W : ((pl % sub) < p.W && z + pl / sub < p.Z);
         const int blk = acc_block(g);
         if (issuer) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store of row g - 2 has read this tile
         asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -494,10 +519,13 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         }
         if (!ok) break;
         if (issuer) {
-          asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
-                       ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(row), "r"(z),
-                         "r"(stg_out + buf * FWD_TILE_BYTES)
-                       : "memory");
+          for (int j = 0; j < p.pack; ++j) {           // one box per strip of the group; all of them in one bulk group
+            if (z + j >= p.Z) break;
+            asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+                         ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(row), "r"(z + j),
+                           "r"(stg_out + buf * FWD_TILE_BYTES + j * sub_bytes)
+                         : "memory");
+          }
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           if (use_mask && g + 2 < n_rows) load_mask(g + 2);
         }
@@ -523,7 +551,8 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 // ------------------------------------------------------------------------------ backward-weight kernel
 struct WgParams {
   int W, Hs, R, nseg;
-  long long rows_total;   // dY row segments: (strip z, segment, row) flattened with the row fastest
+  int pack;               // narrow images: strips per 128-pixel block, as in the forward kernel
+  long long rows_total;   // dY row segments: (strip group z, segment, row) flattened with the row fastest
   float* part;            // [gridDim.x][9][C][C]
   int* status;
 };
@@ -540,7 +569,7 @@ __device__ __forceinline__ WgRun wg_run(const WgParams& p, long long pos, long l
   const long long left = end - pos;
   r.n = static_cast<int>(left < p.Hs - r.h0 ? left : p.Hs - r.h0);
   r.seg = static_cast<int>(col % p.nseg);
-  r.z = static_cast<int>(col / p.nseg);
+  r.z = static_cast<int>(col / p.nseg) * p.pack;
   return r;
 }
 
@@ -571,6 +600,14 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) tmem_alloc<512>(smem_u32(&tmem_base_slot));
+  if (p.pack > 1 && threadIdx.x >= 64) {
+    // packed X stages: the pixel rows behind position 127 (read by the shifted views, written by no box)
+    // must be finite, since they meet the zero-filled tail of the dY block in the reduction
+    uint8_t* ring_gen = smem_raw + (xring - smem_u32(smem_raw));
+    for (int i = threadIdx.x - 64; i < WG_XSTAGES * 64; i += NUM_THREADS - 64)
+      *reinterpret_cast<uint4*>(ring_gen + (i >> 6) * WG_XROW_BYTES + WG_PIX * 128 + (i & 63) * 16) = make_uint4(0, 0, 0, 0);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -584,6 +621,7 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 
   if (warp == 0) {
     if (lane == 0) {
+      const int sub_bytes = (WG_PIX / p.pack) * 128;
       int xs = 0, ys = 0;
       uint32_t xph = 0, yph = 0;
       bool ok = true;
@@ -599,15 +637,23 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             const uint32_t fy = smem_u32(&yfull[ys]);
             const bool mirrored = ys < 2;
             mbar_expect_tx(fy, mirrored ? 2 * WG_CHUNK : WG_CHUNK);
-            tma_load_4d(yring + ys * WG_CHUNK, &tmY, 0, x0, run.h0 + r + 1, z, fy);
-            if (mirrored) tma_load_4d(yring + (WG_YSTAGES + ys) * WG_CHUNK, &tmY, 0, x0, run.h0 + r + 1, z, fy);
+            for (int j = 0; j < p.pack; ++j) {     // one box per strip of the group (pixels beyond W and strips beyond Z read as zeros)
+              tma_load_4d(yring + ys * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, run.h0 + r + 1, z + j, fy);
+              if (mirrored) tma_load_4d(yring + (WG_YSTAGES + ys) * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, run.h0 + r + 1, z + j, fy);
+            }
             if (++ys == WG_YSTAGES) { ys = 0; yph ^= 1u; }
           }
           ok = mbar_wait(smem_u32(&xempty[xs]), xph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
           if (!ok) break;
           const uint32_t fb = smem_u32(&xfull[xs]);
-          mbar_expect_tx(fb, (WG_PIX + 2) * 128);
-          tma_load_4d(xring + xs * WG_XROW_BYTES, &tmX, 0, x0 - 1, run.h0 + r, z, fb);
+          if (p.pack == 1) {
+            mbar_expect_tx(fb, (WG_PIX + 2) * 128);
+            tma_load_4d(xring + xs * WG_XROW_BYTES, &tmX, 0, x0 - 1, run.h0 + r, z, fb);
+          } else {
+            mbar_expect_tx(fb, WG_PIX * 128);
+            for (int j = 0; j < p.pack; ++j)
+              tma_load_4d(xring + xs * WG_XROW_BYTES + j * sub_bytes, &tmX, 0, -1, run.h0 + r, z + j, fb);
+          }
           if (++xs == WG_XSTAGES) { xs = 0; xph ^= 1u; }
         }
       }
@@ -622,7 +668,7 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       for (long long pos = r0; pos < r1 && ok;) {
         const WgRun run = wg_run(p, pos, r1);
         pos += run.n;
-        const int npx = min(WG_PIX, p.W - run.seg * WG_PIX);
+        const int npx = p.pack > 1 ? WG_PIX : min(WG_PIX, p.W - run.seg * WG_PIX);
         const int ksteps = (npx + UMMA_K - 1) / UMMA_K;
         int yhave = 0;
         for (int r = 0; r < run.n + 2 && ok; ++r) {
@@ -760,6 +806,7 @@ bool make_weight_map(CUtensorMap* tm, const void* base) {
 
 struct ConvNet {
   int L = 0, H = 0, W = 0, P_r = 1, Hs = 0, R = 0, num_sms = 148, grid = 148;
+  int pack = 1;                      // strips per 128-pixel tile (narrow images: 2, 4 or 8)
   int64_t B = 0, Z = 0;
   size_t strip_elems = 0;
   int* status = nullptr;
@@ -786,7 +833,8 @@ void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w
   FwdParams p;
   p.W = c->W; p.Hs = c->Hs; p.R = c->R;
   p.nseg = (c->W + FWD_PIX - 1) / FWD_PIX;
-  p.rows_total = static_cast<long long>(c->Z) * p.nseg * c->Hs;
+  p.pack = c->pack; p.Z = static_cast<int>(c->Z);
+  p.rows_total = ((c->Z + c->pack - 1) / c->pack) * p.nseg * c->Hs;
   p.mode = mode; p.out = out; p.mask_src = mask; p.loss_part = c->loss_part; p.status = c->status;
   const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
   if (mode == MODE_STORE_SSQ) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 8, c->stream);
@@ -846,15 +894,21 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   ok = ok && alloc(reinterpret_cast<void**>(&c->loss_part), sizeof(float) * c->grid * 8);
   ok = ok && alloc(reinterpret_cast<void**>(&c->scratch_nchw), static_cast<size_t>(B) * C * H * W * 2);
   if (!ok) { conv_destroy(c); return MBD_E_ALLOC; }
-  const int fwd_box = FWD1_BOX_PIX;
+  // narrow images: as many strips per 128-pixel tile as fit with their two border pixels
+  c->pack = W + 2 <= 16 ? 8 : W + 2 <= 32 ? 4 : W + 2 <= 64 ? 2 : 1;
+  if (getenv("MBD_CONV_NO_PACK")) c->pack = 1;       // tuning knob
+  if (c->Z > INT32_MAX - 8) { conv_destroy(c); return MBD_E_UNSUPPORTED; }
+  const int sub = FWD_PIX / c->pack;
+  const int fwd_box = c->pack > 1 ? sub : FWD1_BOX_PIX;
+  const int tile_box = c->pack > 1 ? sub : FWD_PIX;
   c->act_fwd.resize(L + 1); c->dY_fwd.resize(L); c->dY_wg.resize(L);
   c->act_tile.resize(L + 1); c->dY_tile.resize(L);
   c->wf_map.resize(L); c->wb_map.resize(L);
   for (int i = 0; i <= L && ok; ++i)
-    ok = make_strip_map(&c->act_fwd[i], c->act[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->act_tile[i], c->act[i], W, c->R, c->Z, FWD_PIX);
+    ok = make_strip_map(&c->act_fwd[i], c->act[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->act_tile[i], c->act[i], W, c->R, c->Z, tile_box);
   for (int i = 0; i < L && ok; ++i)
-    ok = make_strip_map(&c->dY_fwd[i], c->dY[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->dY_wg[i], c->dY[i], W, c->R, c->Z, WG_PIX) &&
-         make_strip_map(&c->dY_tile[i], c->dY[i], W, c->R, c->Z, FWD_PIX) &&
+    ok = make_strip_map(&c->dY_fwd[i], c->dY[i], W, c->R, c->Z, fwd_box) && make_strip_map(&c->dY_wg[i], c->dY[i], W, c->R, c->Z, tile_box) &&
+         make_strip_map(&c->dY_tile[i], c->dY[i], W, c->R, c->Z, tile_box) &&
          make_weight_map(&c->wf_map[i], c->Wf[i]) && make_weight_map(&c->wb_map[i], c->Wb[i]);
   if (!ok) { conv_destroy(c); return MBD_E_CUDA; }
   if (cudaStreamSynchronize(stream) != cudaSuccess) { conv_destroy(c); return MBD_E_CUDA; }
@@ -922,7 +976,8 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
     WgParams p;
     p.W = c->W; p.Hs = c->Hs; p.R = c->R;
     p.nseg = (c->W + WG_PIX - 1) / WG_PIX;
-    p.rows_total = static_cast<long long>(c->Z) * p.nseg * c->Hs;
+    p.pack = c->pack;
+    p.rows_total = ((c->Z + c->pack - 1) / c->pack) * p.nseg * c->Hs;
     p.part = c->wpart; p.status = c->status;
     const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
     c->prof->begin(MBD_K_CONV_BWD_WEIGHT, 2.0 * c->B * c->H * c->W * 9.0 * C * C);

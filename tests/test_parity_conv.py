@@ -84,3 +84,17 @@ def test_full_workload_32_images_two_strips():
     o = oracle_conv_step(w, inp)
     g = gpu_conv_step(w, inp, 2, force_acts=stored_hidden(o))
     compare_conv_step(g, o, TOL)
+
+
+@pytest.mark.parametrize("H,W,B,P_r", [(8, 62, 3, 1), (8, 56, 4, 2), (8, 30, 5, 2), (6, 14, 3, 3), (8, 7, 2, 1),
+                                       (4, 1, 9, 1), (8, 63, 2, 2)])
+@pytest.mark.parametrize("fused", [False, True])
+def test_narrow_images_share_tiles(H, W, B, P_r, fused):
+    """Images of at most 62 / 30 / 14 pixels per row put 2 / 4 / 8 strips into one 128-pixel tile; strip
+    counts that do not fill the last group, the widest image of each class, and the first width that
+    does not pack."""
+    w = I.conv_workload(64, H, W, B, name=f"conv_narrow_{W}")
+    inp = I.make_inputs(w, seed=40 + W)
+    o = oracle_conv_step(w, inp)
+    g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o))
+    compare_conv_step(g, o, TOL, fused)
