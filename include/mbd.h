@@ -248,7 +248,9 @@ MBD_API mbd_status mbd_poll_status(mbd_net* net);
  * every launch is bracketed by two events; mbd_profile_read waits for the stream and returns,
  * for one class, the summed duration (ms), the number of launches and the summed ALGORITHMIC
  * work of those launches: flops (2 M N K) for the contraction classes, bytes for the others.
- * mbd_profile_enable(net, 1) also clears the counters. */
+ * mbd_profile_enable(net, 1) also clears the counters.  MBD_K_HALO: the passes between NCHW and the
+ * strip layout (they also fill the halo rows of what they write; the halo rows of a tensor a
+ * convolution produces are stored by that convolution's epilogue and have no launch of their own). */
 enum {
   MBD_K_GEMM_FWD = 0, MBD_K_GEMM_BWD_DATA = 1, MBD_K_GEMM_BWD_WEIGHT = 2, MBD_K_REDUCE = 3,
   MBD_K_SOFTMAX = 4, MBD_K_COLSUM = 5, MBD_K_SGD = 6, MBD_K_HALO = 7, MBD_K_CONV_FWD = 8,

@@ -1,8 +1,10 @@
 // Domain-parallel 3x3 convolution stack (Section 2.2 and 2.4 of the paper): every image is
-// cut into P_r row strips; a strip owner holds its rows plus one halo row per neighbour,
-// exchanged before each convolution that needs them (forward: X halos, backward-data: dY
-// halos); the weight gradient is formed as per-owner partial sums that are then added (the
-// all-reduce over the strips, third term of Eq. 7).
+// cut into P_r row strips; a strip owner holds its rows plus one halo row per neighbour
+// (forward: X halos, backward-data: dY halos).  The exchange is fused into whatever produces a
+// tensor: the convolution epilogue stores a strip's first / last row a second time, into the
+// neighbouring strip's halo row (one more TMA store of the same staging tile), and the staging pass
+// from NCHW does the same.  The weight gradient is formed as per-owner partial sums that are then
+// added (the all-reduce over the strips, third term of Eq. 7).
 //
 // Layout in HBM: every activation / gradient tensor lives as "strips": [Z = B*P_r][R = Hs+2]
 // [W][C = 64] bf16 (channels innermost), row 0 and row Hs+1 of a strip being the halo rows
@@ -171,24 +173,6 @@ strips_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int 
   }
 }
 
-// Halo exchange between neighbouring strips of one tensor: the last own row of strip s becomes
-// the upper halo of strip s+1 and the first own row of strip s+1 the lower halo of strip s.
-// grid = (B * (P_r - 1), 2 directions); one boundary row = W*C bf16, copied with 16-byte accesses.
-__global__ void __launch_bounds__(256)
-halo_stage_kernel(bf16* __restrict__ buf, int W, int P_r, int Hs) {
-  const int R = Hs + 2;
-  const int b = blockIdx.x / (P_r - 1), s = blockIdx.x % (P_r - 1);
-  const int64_t row = static_cast<int64_t>(W) * C;           // elements per row
-  const int64_t z0 = (static_cast<int64_t>(b) * P_r + s) * R, z1 = z0 + R;
-  const bf16* src;
-  bf16* dst;
-  if (blockIdx.y == 0) { src = buf + (z0 + Hs) * row; dst = buf + (z1 + 0) * row; }
-  else { src = buf + (z1 + 1) * row; dst = buf + (z0 + Hs + 1) * row; }
-  const uint4* s4 = reinterpret_cast<const uint4*>(src);
-  uint4* d4 = reinterpret_cast<uint4*>(dst);
-  for (int64_t i = threadIdx.x; i < row / 8; i += 256) d4[i] = s4[i];
-}
-
 // Canonical K[o][c][u][v] -> forward operand Wf[v][(u,o)][c] and backward-data operand
 // Wb[v'][(u',c)][o] = K[o][c][2-u'][2-v'] (taps flipped, channels swapped).
 __global__ void pack_weights_kernel(const bf16* __restrict__ K, bf16* __restrict__ Wf, bf16* __restrict__ Wb) {
@@ -234,6 +218,7 @@ wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ d
 struct FwdParams {
   int W, Hs, R, nseg;
   int pack, Z;            // narrow images: `pack` strips share one 128-pixel tile, 128 / pack pixels each (see below)
+  int P_r;                // strips per image: a boundary row is also stored into the neighbouring strip's halo row
   long long rows_total;   // output row segments: (strip group z, segment, row) flattened with the row fastest
   int mode;
   bf16* out;              // strips
@@ -272,6 +257,8 @@ __device__ __forceinline__ FwdRun fwd_run(const FwdParams& p, long long pos, lon
 // every MMA accumulates.
 __device__ __forceinline__ int acc_block(int g) { return 7 - (g & 7); }
 
+// PACKED: several strips per tile (narrow images); the wide instantiation keeps its single box per row.
+template <bool PACKED>
 __global__ void __launch_bounds__(FWD_THREADS, 1)
 conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
                 const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmMask, const FwdParams p) {
@@ -289,6 +276,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const uint32_t w_smem = base;                         // 3 (v) x [192 rows (u, o) x 128 B]
   const uint32_t ring = base + FWD_W_BYTES;             // slot = one input row (one box of 130 pixels)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int pack = PACKED ? p.pack : 1;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < FWD1_STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
@@ -300,7 +288,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) tmem_alloc<512>(smem_u32(&tmem_base_slot));
-  if (p.pack > 1 && threadIdx.x >= 64 && threadIdx.x < 64 + FWD1_STAGES * 16) {
+  if (pack > 1 && threadIdx.x >= 64 && threadIdx.x < 64 + FWD1_STAGES * 16) {
     // packed stages: positions 128, 129 (read by the shifted views, written by no box) hold zeros
     const int i = threadIdx.x - 64;
     uint8_t* ring_gen = smem_raw + (ring - smem_u32(smem_raw));
@@ -331,13 +319,13 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
           if (!ok) break;
           const uint32_t fb = smem_u32(&full_bar[stage]);
-          if (p.pack == 1) {
+          if (pack == 1) {
             mbar_expect_tx(fb, FWD1_BOX_PIX * 128);
             tma_load_4d(ring + stage * FWD1_ROW_BYTES, &tmX, 0, run.seg * FWD_PIX - 1, run.h0 + r, run.z, fb);
           } else {
-            const int sub_bytes = (FWD_PIX / p.pack) * 128;
+            const int sub_bytes = (FWD_PIX / pack) * 128;
             mbar_expect_tx(fb, FWD_PIX * 128);
-            for (int j = 0; j < p.pack; ++j)      // a strip index beyond Z reads as zeros
+            for (int j = 0; j < pack; ++j)      // a strip index beyond Z reads as zeros
               tma_load_4d(ring + stage * FWD1_ROW_BYTES + j * sub_bytes, &tmX, 0, -1, run.h0 + r, run.z + j, fb);
           }
           if (++stage == FWD1_STAGES) { stage = 0; phase ^= 1u; }
@@ -426,33 +414,45 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       const bool use_mask = p.mode == MODE_MASK && p.mask_src != nullptr;
       const bool issuer = warp == 2 && lane == 0;
       const int n_rows = static_cast<int>(r1 - r0);
-      auto row_coords = [&](int k, int& x0, int& row, int& z) {
-        const long long pos = r0 + k;
+      // Position of an output row in the flattened (strip group, segment, row) space, advanced row by row
+      // (no divisions inside the loop): `cur` is the row being drained, `ahead` the one whose mask is loaded.
+      struct Pos { int x0, row, z; };
+      auto pos_at = [&](long long pos) {
         const long long col = pos / p.Hs;
-        z = static_cast<int>(col / p.nseg) * p.pack;
-        x0 = static_cast<int>(col % p.nseg) * FWD_PIX;
-        row = static_cast<int>(pos - col * p.Hs) + 1;
+        Pos q;
+        q.z = static_cast<int>(col / p.nseg) * pack;
+        q.x0 = static_cast<int>(col % p.nseg) * FWD_PIX;
+        q.row = static_cast<int>(pos - col * p.Hs) + 1;
+        return q;
       };
-      const int sub = FWD_PIX / p.pack;                   // tile positions per strip
+      auto advance = [&](Pos& q) {
+        if (++q.row > p.Hs) {
+          q.row = 1;
+          q.x0 += FWD_PIX;
+          if (q.x0 >= p.nseg * FWD_PIX) { q.x0 = 0; q.z += pack; }
+        }
+      };
+      const int sub = FWD_PIX / pack;                   // tile positions per strip
       const int sub_bytes = sub * 128;
-      auto load_mask = [&](int k) {
-        int x0, row, z;
-        row_coords(k, x0, row, z);
+      auto load_mask = [&](int k, const Pos& q) {
         const uint32_t mb = smem_u32(&mask_full_bar[k & 1]);
         mbar_expect_tx(mb, FWD_TILE_BYTES);
-        for (int j = 0; j < p.pack; ++j)
-          tma_load_4d(stg_mask + (k & 1) * FWD_TILE_BYTES + j * sub_bytes, &tmMask, 0, x0, row, z + j, mb);
+        for (int j = 0; j < pack; ++j)
+          tma_load_4d(stg_mask + (k & 1) * FWD_TILE_BYTES + j * sub_bytes, &tmMask, 0, q.x0, q.row, q.z + j, mb);
       };
+      Pos cur = pos_at(r0), ahead = cur;
       if (use_mask && issuer) {
-        if (n_rows > 0) load_mask(0);
-        if (n_rows > 1) load_mask(1);
+        if (n_rows > 0) load_mask(0, ahead);
+        advance(ahead);
+        if (n_rows > 1) load_mask(1, ahead);
+        advance(ahead);
       }
       const int cell0 = half * 4;                         // first 16-byte cell of this thread's channels
-      for (; g < n_rows; ++g) {
+      const int pl_sub = PACKED ? pl % sub : pl, pl_strip = PACKED ? pl / sub : 0;
+      for (; g < n_rows; ++g, advance(cur)) {
         const int buf = g & 1;
-        int x0, row, z;
-        row_coords(g, x0, row, z);
-        const bool valid = p.pack == 1 ? x0 + pl < p.W : ((pl % sub) < p.W && z + pl / sub < p.Z);
+        const int x0 = cur.x0, row = cur.row, z = cur.z;
+        const bool valid = PACKED ? (pl_sub < p.W && z + pl_strip < p.Z) : x0 + pl < p.W;
         const int blk = acc_block(g);
         if (issuer) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store of row g - 2 has read this tile
         asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -519,15 +519,26 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         }
         if (!ok) break;
         if (issuer) {
-          for (int j = 0; j < p.pack; ++j) {           // one box per strip of the group; all of them in one bulk group
-            if (z + j >= p.Z) break;
+          for (int j = 0; j < pack; ++j) {           // one box per strip of the group; all of them in one bulk group
+            const int zj = z + j;
+            if (zj >= p.Z) break;
+            const uint32_t src = stg_out + buf * FWD_TILE_BYTES + j * sub_bytes;
             asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
-                         ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(row), "r"(z + j),
-                           "r"(stg_out + buf * FWD_TILE_BYTES + j * sub_bytes)
+                         ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(row), "r"(zj), "r"(src)
                          : "memory");
+            // Halo exchange (Section 2.2), fused: the first / last own row of a strip is also the lower / upper
+            // halo row of the strip above / below it in the same image.
+            if (row == 1 && p.P_r > 1 && zj % p.P_r > 0)
+              asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+                           ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(p.Hs + 1), "r"(zj - 1), "r"(src)
+                           : "memory");
+            if (row == p.Hs && p.P_r > 1 && zj % p.P_r < p.P_r - 1)
+              asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+                           ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(0), "r"(zj + 1), "r"(src)
+                           : "memory");
           }
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-          if (use_mask && g + 2 < n_rows) load_mask(g + 2);
+          if (use_mask && g + 2 < n_rows) { load_mask(g + 2, ahead); advance(ahead); }
         }
       }
       if (issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // stores done before the CTA exits
@@ -773,7 +784,8 @@ cudaError_t conv_init() {
   cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
   if (e != cudaSuccess) return e;
   if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
-  if ((e = cudaFuncSetAttribute(conv_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(conv_fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(conv_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM)) != cudaSuccess) return e;
   g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   return cudaSuccess;
@@ -833,22 +845,17 @@ void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w
   FwdParams p;
   p.W = c->W; p.Hs = c->Hs; p.R = c->R;
   p.nseg = (c->W + FWD_PIX - 1) / FWD_PIX;
-  p.pack = c->pack; p.Z = static_cast<int>(c->Z);
+  p.pack = c->pack; p.Z = static_cast<int>(c->Z); p.P_r = c->P_r;
   p.rows_total = ((c->Z + c->pack - 1) / c->pack) * p.nseg * c->Hs;
   p.mode = mode; p.out = out; p.mask_src = mask; p.loss_part = c->loss_part; p.status = c->status;
   const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
   if (mode == MODE_STORE_SSQ) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 8, c->stream);
   const double flops = 2.0 * c->B * c->H * c->W * 9.0 * C * C;
   c->prof->begin(cls, flops);
-  launch_pdl(conv_fwd_kernel, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, out_tile, mask_tile ? *mask_tile : out_tile, p);
-  c->prof->end();
-}
-
-void launch_halo(ConvNet* c, bf16* buf) {
-  if (c->P_r < 2) return;
-  dim3 g(static_cast<unsigned>(c->B * (c->P_r - 1)), 2);
-  c->prof->begin(MBD_K_HALO, 2.0 * 2.0 * c->B * (c->P_r - 1) * c->W * C * 2.0);
-  halo_stage_kernel<<<g, 256, 0, c->stream>>>(buf, c->W, c->P_r, c->Hs);
+  if (c->pack > 1)
+    launch_pdl(conv_fwd_kernel<true>, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, out_tile, mask_tile ? *mask_tile : out_tile, p);
+  else
+    launch_pdl(conv_fwd_kernel<false>, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, out_tile, mask_tile ? *mask_tile : out_tile, p);
   c->prof->end();
 }
 
@@ -949,7 +956,8 @@ mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
   }
   for (int i = 0; i < c->L; ++i) {
     const bool last = i == c->L - 1;
-    if (i > 0) launch_halo(c, c->act[i]);            // forward halo exchange (first halo term of Eq. 7)
+    // forward halo exchange (first halo term of Eq. 7): the kernel that produced act[i] (or the staging pass,
+    // for the network input) has already stored its boundary rows into the neighbouring strips' halo rows
     launch_fwd(c, MBD_K_CONV_FWD, c->act_fwd[i], c->wf_map[i], c->act[i + 1], c->act_tile[i + 1],
                (last && !c->fc_above) ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK), nullptr, nullptr);
   }
@@ -969,7 +977,7 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
   for (int i = c->L - 1; i >= 0; --i) {
     if (i > 0) {
       // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0]
-      launch_halo(c, c->dY[i]);
+      // (the producer of dY_i has stored its boundary rows into the neighbours' halo rows)
       launch_fwd(c, MBD_K_CONV_BWD_DATA, c->dY_fwd[i], c->wb_map[i], c->dY[i - 1], c->dY_tile[i - 1], MODE_MASK,
                  c->relu[i - 1] ? c->act[i] : nullptr, c->relu[i - 1] ? &c->act_tile[i] : nullptr);
     }
