@@ -185,9 +185,11 @@ __global__ void pack_weights_kernel(const bf16* __restrict__ K, bf16* __restrict
 }
 
 // Sum of the per-CTA partials [G][9][c][o] in CTA order, into canonical [o][c][u][v]:
-// either stored (dK) or applied as K += scale * dK (Eq. 1).
+// either stored (dK) or applied as K += scale * dK (Eq. 1); the updated weight also goes into the
+// two operand layouts the next step's kernels read (see pack_weights_kernel).
 __global__ void __launch_bounds__(256)
-wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ dK, bf16* __restrict__ K, float scale) {
+wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ dK, bf16* __restrict__ K,
+                    bf16* __restrict__ Wf, bf16* __restrict__ Wb, float scale) {
   // 64 outputs per block; four thread groups each add a contiguous quarter of the CTA partials in
   // ascending order, and the four sub-sums are added in ascending order too (a fixed order).
   __shared__ float sub[4][64];
@@ -211,7 +213,13 @@ wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ d
   const int t = i / (C * C), c = (i / C) % C, o = i % C;
   const int e = (o * C + c) * 9 + t;
   if (dK) dK[e] = s;
-  if (K) K[e] = __float2bfloat16_rn(fmaf(scale, s, __bfloat162float(K[e])));
+  if (K) {
+    const bf16 k = __float2bfloat16_rn(fmaf(scale, s, __bfloat162float(K[e])));
+    const int u = t / 3, v = t - 3 * u;
+    K[e] = k;
+    Wf[((v * 3 + u) * C + o) * C + c] = k;
+    Wb[(((2 - v) * 3 + (2 - u)) * C + c) * C + o] = k;
+  }
 }
 
 // ------------------------------------------------------------------------------ forward kernel
@@ -934,9 +942,18 @@ void conv_destroy(ConvNet* c) {
   delete c;
 }
 
+namespace {
+mbd_status launch_pack(ConvNet* c, int layer) {
+  c->prof->begin(MBD_K_OTHER, 9.0 * C * C * 6.0);
+  pack_weights_kernel<<<(9 * C * C + 255) / 256, 256, 0, c->stream>>>(c->K[layer], c->Wf[layer], c->Wb[layer]);
+  c->prof->end();
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+}  // namespace
+
 mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev) {
   if (cudaMemcpyAsync(c->K[layer], K_dev, 9 * C * C * 2, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) return MBD_E_CUDA;
-  return MBD_OK;
+  return launch_pack(c, layer);
 }
 
 mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev) {
@@ -947,13 +964,9 @@ mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev) {
 size_t conv_input_bytes(const ConvNet* c) { return static_cast<size_t>(c->B) * C * c->H * c->W * 2; }
 
 mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
-  // stage the input into strips (with its halo rows) and pack the current weights
+  // stage the input into strips (with its halo rows); the operand layouts of the weights are kept current
+  // by whatever changes the weights (conv_set_weights, the fused update, conv_sgd_step)
   launch_stage_in(c, static_cast<const bf16*>(X_nchw), c->act[0]);
-  for (int i = 0; i < c->L; ++i) {
-    c->prof->begin(MBD_K_OTHER, 9.0 * C * C * 6.0);
-    pack_weights_kernel<<<(9 * C * C + 255) / 256, 256, 0, c->stream>>>(c->K[i], c->Wf[i], c->Wb[i]);
-    c->prof->end();
-  }
   for (int i = 0; i < c->L; ++i) {
     const bool last = i == c->L - 1;
     // forward halo exchange (first halo term of Eq. 7): the kernel that produced act[i] (or the staging pass,
@@ -993,7 +1006,7 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
     c->prof->end();
     c->prof->begin(MBD_K_REDUCE, (grid + 1.0) * 9 * C * C * 4.0);
     wgrad_finish_kernel<<<9 * C * C / 64, 256, 0, c->stream>>>(c->wpart, grid, fused ? nullptr : c->dK[i],
-                                                                      fused ? c->K[i] : nullptr, scale);
+                                                                      fused ? c->K[i] : nullptr, c->Wf[i], c->Wb[i], scale);
     c->prof->end();
   }
   if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
@@ -1007,6 +1020,7 @@ mbd_status conv_sgd_step(ConvNet* c, float eta) {
     c->prof->begin(MBD_K_SGD, 9.0 * C * C * 8.0);
     if (sgd_update_launch(c->K[i], 1, c->dK[i], 9 * C * C, scale, c->num_sms, c->stream) != cudaSuccess) return MBD_E_CUDA;
     c->prof->end();
+    if (launch_pack(c, i) != MBD_OK) return MBD_E_CUDA;
   }
   return MBD_OK;
 }

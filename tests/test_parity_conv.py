@@ -98,3 +98,48 @@ def test_narrow_images_share_tiles(H, W, B, P_r, fused):
     o = oracle_conv_step(w, inp)
     g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o))
     compare_conv_step(g, o, TOL, fused)
+
+
+@pytest.mark.parametrize("mode", ["fused", "unfused", "graph"])
+def test_second_step_uses_the_updated_kernels(mode):
+    """Two steps in a row against two oracle steps: the operand layouts the convolution kernels read are
+    refreshed by whatever updates the weights (fused update, mbd_sgd_step), also under graph replay."""
+    import torch
+    from oracle import mbd_oracle as O
+    from paper_1712_04432_b200 import mbd
+    from tests.helpers import bf16_store, to_dev, to_np
+    w = I.conv_workload(64, 8, 40, 2, name="conv_two_steps")
+    w.eta = 2e-5
+    inp = I.make_inputs(w, seed=61)
+    layers = [O.Conv3x3(k.astype(np.float64), relu=True) for k in inp.Ws]
+    X = inp.X.astype(np.float64)
+    o1 = O.train_step(layers, X, None, "half_ssq", w.eta, store=bf16_store)
+    # the device keeps its weights in bf16: the second oracle step starts from the rounded update
+    layers2 = [O.Conv3x3(bf16_store(k), relu=True) for k in o1["new_W"]]
+    o2 = O.train_step(layers2, X, None, "half_ssq", w.eta, store=bf16_store)
+    assert abs(o2["J"] - o1["J"]) > 1e-3 * abs(o1["J"])          # the step is large enough to be seen
+
+    net = mbd.Net(mbd.conv_layers(2, 64, 8, 40), w.B, 2, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+    for i in range(2):
+        net.set_weights(i, to_dev(inp.Ws[i], True))
+    Xd = to_dev(inp.X, True)
+    J = torch.zeros(1, dtype=torch.float32, device="cuda")
+    Js = []
+    for _ in range(2):
+        if mode == "graph":
+            net.train_step(Xd, None, w.eta, J)
+        else:
+            net.forward(Xd, None, J)
+            if mode == "fused":
+                net.backward(w.eta)
+            else:
+                net.backward(0.0)
+                net.sgd_step(w.eta)
+        net.poll()
+        Js.append(float(J.item()))
+    assert abs(Js[0] - o1["J"]) <= 1e-2 * abs(o1["J"])
+    assert abs(Js[1] - o2["J"]) <= 1e-2 * abs(o2["J"])
+    assert abs(Js[1] - o2["J"]) < 0.2 * abs(o2["J"] - o1["J"])    # and it is the second step's loss, not the first's
+    for i in range(2):
+        assert rel_fro(to_np(net.get_weights(i)), o2["new_W"][i]) <= TOL
+    net.close()
