@@ -5,6 +5,7 @@ a profiler (small, self-terminating):
     python -m paper_1712_04432_b200.profile_case gemm_bwd_weight --size 4096
     python -m paper_1712_04432_b200.profile_case reduce --size 8192 --splits 2
     python -m paper_1712_04432_b200.profile_case conv --batch 4 --strips 4
+    python -m paper_1712_04432_b200.profile_case conv --batch 64 --strips 2 --image 56
     python -m paper_1712_04432_b200.profile_case fc --batch 8192 --dims 1024,8192
 
 gemm_*: one tensor-core contraction of size^3 in the operand layout of that product.
@@ -13,7 +14,7 @@ reduce: a split contraction followed by the partial-sum reduction (the reduction
 fc:     `launches` training steps of a small fully connected net (softmax, bias-gradient and
         update kernels at a size where their DRAM figures mean something).
 conv:   `launches` training steps of the two-layer 3x3 convolution stack on `batch` images of
-64 x 224 x 224, cut into `strips` row strips.
+64 x image x image (default 224), cut into `strips` row strips.
 """
 import argparse
 
@@ -28,6 +29,7 @@ def main():
     ap.add_argument("--dims", default="1024,8192")
     ap.add_argument("--batch", type=int, default=4)
     ap.add_argument("--strips", type=int, default=4)
+    ap.add_argument("--image", type=int, default=224)
     ap.add_argument("--size", type=int, default=8192)
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--splits", type=int, default=2)
@@ -74,11 +76,11 @@ def fc_case(a):
 
 def conv_case(a):
     g = torch.Generator(device="cuda").manual_seed(0)
-    net = mbd.Net(mbd.conv_layers(2, 64, 224, 224), a.batch, a.strips, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+    net = mbd.Net(mbd.conv_layers(2, 64, a.image, a.image), a.batch, a.strips, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
     for i in range(2):
         K = (torch.randn((64, 64, 3, 3), generator=g, device="cuda") * (2.0 / 576) ** 0.5).to(torch.bfloat16)
         net.set_weights(i, K)
-    X = torch.randn((a.batch, 64, 224, 224), generator=g, device="cuda").to(torch.bfloat16)
+    X = torch.randn((a.batch, 64, a.image, a.image), generator=g, device="cuda").to(torch.bfloat16)
     J = torch.zeros(1, device="cuda")
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
@@ -89,7 +91,7 @@ def conv_case(a):
     ev1.record()
     torch.cuda.synchronize()
     net.poll()
-    print(f"conv batch={a.batch} strips={a.strips}: {ev0.elapsed_time(ev1) / a.launches:.3f} ms per step, J = {J.item():.4e}")
+    print(f"conv batch={a.batch} image={a.image} strips={a.strips}: {ev0.elapsed_time(ev1) / a.launches:.3f} ms per step, J = {J.item():.4e}")
 
 
 if __name__ == "__main__":
