@@ -116,7 +116,8 @@ enum {
  * fully connected layer into P_r row blocks of W_i and the same P_c batch blocks.
  * MBD_E_GRID if P_r < 1, P_c < 1, P_c > B, P_r > min d_i over model-split layers, or
  * a strip would be shorter than its halo.
- * MBD_E_UNSUPPORTED for convolutions other than 3x3/s1/p1 with C_in = C_out = 64,
+ * MBD_E_UNSUPPORTED for convolutions other than 3x3 or 1x1, stride 1, "same" zero padding,
+ * C_in = C_out = 64 (kind MBD_CONV3X3 with kh = kw = 1 is the 1x1 case, weights [C_out][C_in]),
  * strips of unequal height, a convolution above a fully connected layer, half-SSQ with
  * fully connected layers or softmax-CE without them, or bf16 FC dims that are not
  * multiples of 8. */

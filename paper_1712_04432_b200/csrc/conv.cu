@@ -184,12 +184,25 @@ __global__ void pack_weights_kernel(const bf16* __restrict__ K, bf16* __restrict
   Wb[(((2 - v) * 3 + (2 - u)) * C + c) * C + o] = k;
 }
 
+// A 1 x 1 convolution (the case that needs no halo, remark after Eq. 7) runs through the same kernels as
+// a 3 x 3 kernel whose eight outer taps are zero and stay zero: its [o][c] weights live in the centre tap.
+__global__ void embed_1x1_kernel(const bf16* __restrict__ K1, bf16* __restrict__ K) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= C * C * 9) return;
+  K[i] = (i % 9) == 4 ? K1[i / 9] : __float2bfloat16_rn(0.f);
+}
+template <typename T>
+__global__ void extract_1x1_kernel(const T* __restrict__ K, T* __restrict__ K1) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < C * C) K1[i] = K[i * 9 + 4];
+}
+
 // Sum of the per-CTA partials [G][9][c][o] in CTA order, into canonical [o][c][u][v]:
 // either stored (dK) or applied as K += scale * dK (Eq. 1); the updated weight also goes into the
 // two operand layouts the next step's kernels read (see pack_weights_kernel).
 __global__ void __launch_bounds__(256)
 wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ dK, bf16* __restrict__ K,
-                    bf16* __restrict__ Wf, bf16* __restrict__ Wb, float scale) {
+                    bf16* __restrict__ Wf, bf16* __restrict__ Wb, float scale, int centre_only) {
   // 64 outputs per block; four thread groups each add a contiguous quarter of the CTA partials in
   // ascending order, and the four sub-sums are added in ascending order too (a fixed order).
   __shared__ float sub[4][64];
@@ -212,6 +225,10 @@ wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ d
   s = ((sub[0][j] + sub[1][j]) + sub[2][j]) + sub[3][j];
   const int t = i / (C * C), c = (i / C) % C, o = i % C;
   const int e = (o * C + c) * 9 + t;
+  if (centre_only && t != 4) {       // the outer taps of a 1 x 1 layer are not parameters: no gradient, no update
+    if (dK) dK[e] = 0.f;
+    return;
+  }
   if (dK) dK[e] = s;
   if (K) {
     const bf16 k = __float2bfloat16_rn(fmaf(scale, s, __bfloat162float(K[e])));
@@ -837,6 +854,7 @@ struct ConvNet {
   std::vector<bf16*> K, Wf, Wb;
   std::vector<float*> dK;
   std::vector<int> relu;
+  std::vector<int> k1;               // 1 x 1 layer: weights in the centre tap, outer taps zero
   std::vector<CUtensorMap> act_fwd, dY_fwd, dY_wg, wf_map, wb_map;   // act_fwd / dY_fwd: 130-pixel boxes (also the X operand of backward-weight)
   std::vector<CUtensorMap> act_tile, dY_tile;     // [128 pixels][64 channels] boxes: TMA stores of outputs, mask rows
   float* wpart = nullptr;
@@ -848,7 +866,7 @@ struct ConvNet {
 
 namespace {
 
-void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w, bf16* out, const CUtensorMap& out_tile, int mode,
+void launch_fwd(ConvNet* c, int cls, int layer, const CUtensorMap& in, const CUtensorMap& w, bf16* out, const CUtensorMap& out_tile, int mode,
                 const bf16* mask, const CUtensorMap* mask_tile) {
   FwdParams p;
   p.W = c->W; p.Hs = c->Hs; p.R = c->R;
@@ -858,7 +876,7 @@ void launch_fwd(ConvNet* c, int cls, const CUtensorMap& in, const CUtensorMap& w
   p.mode = mode; p.out = out; p.mask_src = mask; p.loss_part = c->loss_part; p.status = c->status;
   const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
   if (mode == MODE_STORE_SSQ) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 8, c->stream);
-  const double flops = 2.0 * c->B * c->H * c->W * 9.0 * C * C;
+  const double flops = 2.0 * c->B * c->H * c->W * (c->k1[layer] ? 1.0 : 9.0) * C * C;   // the method's flops, not the kernel's
   c->prof->begin(cls, flops);
   if (c->pack > 1)
     launch_pdl(conv_fwd_kernel<true>, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, out_tile, mask_tile ? *mask_tile : out_tile, p);
@@ -897,9 +915,11 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   c->act.assign(L + 1, nullptr); c->dY.assign(L, nullptr);
   c->K.assign(L, nullptr); c->Wf.assign(L, nullptr); c->Wb.assign(L, nullptr); c->dK.assign(L, nullptr);
   c->relu.resize(L);
+  c->k1.resize(L);
   for (int i = 0; i <= L && ok; ++i) ok = alloc(reinterpret_cast<void**>(&c->act[i]), c->strip_elems * 2);
   for (int i = 0; i < L && ok; ++i) {
     c->relu[i] = layers[i].relu;
+    c->k1[i] = layers[i].kh == 1;
     if (i < L - 1 || fc_above) ok = alloc(reinterpret_cast<void**>(&c->dY[i]), c->strip_elems * 2);
     else c->dY[i] = c->act[L];                       // half-SSQ loss: dY_L = Y_L
     ok = ok && alloc(reinterpret_cast<void**>(&c->K[i]), 9 * C * C * 2) && alloc(reinterpret_cast<void**>(&c->Wf[i]), 9 * C * C * 2) &&
@@ -952,11 +972,20 @@ mbd_status launch_pack(ConvNet* c, int layer) {
 }  // namespace
 
 mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev) {
-  if (cudaMemcpyAsync(c->K[layer], K_dev, 9 * C * C * 2, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) return MBD_E_CUDA;
+  if (c->k1[layer]) {
+    embed_1x1_kernel<<<(9 * C * C + 255) / 256, 256, 0, c->stream>>>(static_cast<const bf16*>(K_dev), c->K[layer]);
+    if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
+  } else if (cudaMemcpyAsync(c->K[layer], K_dev, 9 * C * C * 2, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) {
+    return MBD_E_CUDA;
+  }
   return launch_pack(c, layer);
 }
 
 mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev) {
+  if (c->k1[layer]) {
+    extract_1x1_kernel<bf16><<<(C * C + 255) / 256, 256, 0, c->stream>>>(c->K[layer], static_cast<bf16*>(K_dev));
+    return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+  }
   if (cudaMemcpyAsync(K_dev, c->K[layer], 9 * C * C * 2, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) return MBD_E_CUDA;
   return MBD_OK;
 }
@@ -971,7 +1000,7 @@ mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
     const bool last = i == c->L - 1;
     // forward halo exchange (first halo term of Eq. 7): the kernel that produced act[i] (or the staging pass,
     // for the network input) has already stored its boundary rows into the neighbouring strips' halo rows
-    launch_fwd(c, MBD_K_CONV_FWD, c->act_fwd[i], c->wf_map[i], c->act[i + 1], c->act_tile[i + 1],
+    launch_fwd(c, MBD_K_CONV_FWD, i, c->act_fwd[i], c->wf_map[i], c->act[i + 1], c->act_tile[i + 1],
                (last && !c->fc_above) ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK), nullptr, nullptr);
   }
   if (loss_sum_dev && !c->fc_above) {
@@ -991,7 +1020,7 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
     if (i > 0) {
       // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0]
       // (the producer of dY_i has stored its boundary rows into the neighbours' halo rows)
-      launch_fwd(c, MBD_K_CONV_BWD_DATA, c->dY_fwd[i], c->wb_map[i], c->dY[i - 1], c->dY_tile[i - 1], MODE_MASK,
+      launch_fwd(c, MBD_K_CONV_BWD_DATA, i, c->dY_fwd[i], c->wb_map[i], c->dY[i - 1], c->dY_tile[i - 1], MODE_MASK,
                  c->relu[i - 1] ? c->act[i] : nullptr, c->relu[i - 1] ? &c->act_tile[i] : nullptr);
     }
     WgParams p;
@@ -1001,12 +1030,12 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
     p.rows_total = ((c->Z + c->pack - 1) / c->pack) * p.nseg * c->Hs;
     p.part = c->wpart; p.status = c->status;
     const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
-    c->prof->begin(MBD_K_CONV_BWD_WEIGHT, 2.0 * c->B * c->H * c->W * 9.0 * C * C);
+    c->prof->begin(MBD_K_CONV_BWD_WEIGHT, 2.0 * c->B * c->H * c->W * (c->k1[i] ? 1.0 : 9.0) * C * C);
     launch_pdl(conv_wgrad_kernel, dim3(grid), dim3(NUM_THREADS), WG_SMEM, c->stream, 1, c->act_fwd[i], c->dY_wg[i], p);
     c->prof->end();
     c->prof->begin(MBD_K_REDUCE, (grid + 1.0) * 9 * C * C * 4.0);
     wgrad_finish_kernel<<<9 * C * C / 64, 256, 0, c->stream>>>(c->wpart, grid, fused ? nullptr : c->dK[i],
-                                                                      fused ? c->K[i] : nullptr, c->Wf[i], c->Wb[i], scale);
+                                                                      fused ? c->K[i] : nullptr, c->Wf[i], c->Wb[i], scale, c->k1[i]);
     c->prof->end();
   }
   if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
@@ -1047,7 +1076,13 @@ int conv_last_relu(const ConvNet* c) { return c->relu[c->L - 1]; }
 mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t bytes) {
   const size_t nchw_bytes = conv_input_bytes(c);
   if (which == MBD_T_DW) {
-    if (layer < 0 || layer >= c->L || bytes != 9 * C * C * 4) return MBD_E_INVALID;
+    if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
+    if (c->k1[layer]) {
+      if (bytes != C * C * 4) return MBD_E_INVALID;
+      extract_1x1_kernel<float><<<(C * C + 255) / 256, 256, 0, c->stream>>>(c->dK[layer], static_cast<float*>(dst));
+      return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+    }
+    if (bytes != 9 * C * C * 4) return MBD_E_INVALID;
     if (cudaMemcpyAsync(dst, c->dK[layer], bytes, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) return MBD_E_CUDA;
     return MBD_OK;
   }

@@ -287,7 +287,8 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
       if (dtype == MBD_BF16 && (l.d_in % 8 || l.d_out % 8)) return MBD_E_UNSUPPORTED;
       if (l.d_in > INT32_MAX || l.d_out > INT32_MAX || B > INT32_MAX) return MBD_E_UNSUPPORTED;
     } else if (l.kind == MBD_CONV3X3) {
-      if (l.kh != 3 || l.kw != 3 || l.C_in != 64 || l.C_out != 64 || dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
+      const bool k3 = l.kh == 3 && l.kw == 3, k1 = l.kh == 1 && l.kw == 1;     // stride 1, "same" padding
+      if (!(k3 || k1) || l.C_in != 64 || l.C_out != 64 || dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
       if (l.split != MBD_SPLIT_DOMAIN) return MBD_E_UNSUPPORTED;
       if (l.H < 1 || l.W < 1 || P_r > l.H) return MBD_E_GRID;   // a strip needs >= 1 row (halo = 1)
       if (i > 0 && (l.H != layers[0].H || l.W != layers[0].W)) return MBD_E_INVALID;

@@ -55,6 +55,10 @@ class Workload:
     n_layers: int = 0
     grids: List[Tuple[int, int]] = field(default_factory=list)
     fc_dims: Tuple[int, ...] = ()  # mixed: C*H*W -> ... -> classes above the n_layers convolutions
+    ksizes: Tuple[int, ...] = ()   # conv, mixed: kernel size (3 or 1) per convolution; empty = all 3 x 3
+
+    def ksize(self, i: int) -> int:
+        return self.ksizes[i] if self.ksizes else 3
 
     @property
     def L(self) -> int:
@@ -78,12 +82,12 @@ WORKLOADS = {
 }
 
 
-def mixed_workload(C, H, W, n_conv, fc_dims, B, name="custom_mixed", grids=()) -> "Workload":
+def mixed_workload(C, H, W, n_conv, fc_dims, B, name="custom_mixed", grids=(), ksizes=()) -> "Workload":
     """n_conv 3x3 convolutions C -> C on H x W images, then a fully connected stack
     C*H*W -> fc_dims[0] -> ... -> fc_dims[-1] with softmax cross-entropy."""
     d = (int(C) * int(H) * int(W),) + tuple(int(x) for x in fc_dims)
     return Workload(name, "mixed", (int(C), int(H), int(W)), int(B), "bf16", "normal", "softmax_ce",
-                    n_layers=int(n_conv), grids=list(grids), fc_dims=d)
+                    n_layers=int(n_conv), grids=list(grids), fc_dims=d, ksizes=tuple(ksizes))
 
 
 # Beyond the five configurations: the integrated network of Section 2.4 in miniature (convolutions on
@@ -96,9 +100,9 @@ def fc_workload(dims, B, dtype="bf16", x_dist="normal", name="custom") -> Worklo
     return Workload(name, "fc", tuple(int(d) for d in dims), int(B), dtype, x_dist, "softmax_ce")
 
 
-def conv_workload(C, H, W, B, n_layers=2, dtype="bf16", name="custom_conv") -> Workload:
+def conv_workload(C, H, W, B, n_layers=2, dtype="bf16", name="custom_conv", ksizes=()) -> Workload:
     return Workload(name, "conv", (int(C), int(H), int(W)), int(B), dtype, "normal",
-                    "half_ssq", n_layers=n_layers)
+                    "half_ssq", n_layers=n_layers, ksizes=tuple(ksizes))
 
 
 @dataclass
@@ -131,9 +135,10 @@ def make_inputs(w: Workload, seed: int = 0) -> Inputs:
     C, H, Wd = w.dims
     X = rnd(rng.standard_normal((w.B, C, H, Wd), dtype=np.float32))
     Ws = []
-    for _ in range(w.n_layers):
-        K = rng.standard_normal((C, C, 3, 3), dtype=np.float32)
-        K *= np.float32(np.sqrt(2.0 / (9 * C)))                  # N(0, 2/(9 C))
+    for i in range(w.n_layers):
+        k = w.ksize(i)
+        K = rng.standard_normal((C, C, k, k), dtype=np.float32)
+        K *= np.float32(np.sqrt(2.0 / (k * k * C)))              # N(0, 2/(k^2 C))
         Ws.append(rnd(K))
     bs: List[Optional[np.ndarray]] = [None] * w.n_layers
     if w.kind != "mixed":
@@ -160,8 +165,10 @@ def step_flops(w: Workload) -> int:
             macs += (3 if i >= 2 else 2) * per
         return 2 * macs
     C, H, Wd = w.dims
-    per = w.B * H * Wd * C * C * 9
-    macs = per * (3 * w.n_layers - 1)
+    macs = 0
+    for i in range(w.n_layers):
+        per = w.B * H * Wd * C * C * w.ksize(i) ** 2
+        macs += (3 if i >= 1 else 2) * per
     if w.kind == "mixed":
         d = w.fc_dims
         macs += sum(3 * w.B * d[i] * d[i - 1] for i in range(1, len(d)))

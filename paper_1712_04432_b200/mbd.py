@@ -133,10 +133,13 @@ def fc_layers(dims: Sequence[int], bias: bool = True, relu: bool = True) -> List
                   d_out=int(dims[i])) for i in range(1, len(dims))]
 
 
-def conv_layers(n: int, C_: int, H: int, W: int, relu: bool = True) -> List[Layer]:
-    """n domain-split 3x3 convolution layers C -> C on H x W images."""
+def conv_layers(n: int, C_: int, H: int, W: int, relu: bool = True, k=3) -> List[Layer]:
+    """n domain-split convolution layers C -> C on H x W images; `k` is the kernel size (3 or 1),
+    one value for all layers or one per layer."""
+    ks = [k] * n if isinstance(k, int) else list(k)
+    assert len(ks) == n
     return [Layer(kind=CONV3X3, split=SPLIT_DOMAIN, relu=int(relu), bias=0, d_in=C_ * H * W, d_out=C_ * H * W,
-                  C_in=C_, C_out=C_, H=H, W=W, kh=3, kw=3) for _ in range(n)]
+                  C_in=C_, C_out=C_, H=H, W=W, kh=ks[i], kw=ks[i]) for i in range(n)]
 
 
 def _layer_array(layers: Sequence[Layer]):
@@ -232,7 +235,7 @@ class Net:
 
     def _wshape(self, i):
         l = self.layers[i]
-        return (l.C_out, l.C_in, 3, 3) if l.kind == CONV3X3 else (l.d_out, l.d_in)
+        return (l.C_out, l.C_in, l.kh, l.kw) if l.kind == CONV3X3 else (l.d_out, l.d_in)
 
     def close(self):
         if self._h:

@@ -140,12 +140,28 @@ def compare_fc_step(g, o, tol, fused=False, tol_below_relu=None):
 # ---------------------------------------------------------------------------
 # convolution workloads
 # ---------------------------------------------------------------------------
+def oracle_kernel(K):
+    """The oracle's 3 x 3 layer for a device kernel: a 1 x 1 kernel [O, C, 1, 1] is the 3 x 3 kernel whose
+    centre tap holds it and whose other taps are zero (the same correlation)."""
+    K = np.asarray(K, np.float64)
+    if K.shape[2] == 3:
+        return K
+    K3 = np.zeros(K.shape[:2] + (3, 3), np.float64)
+    K3[:, :, 1, 1] = K[:, :, 0, 0]
+    return K3
+
+
+def like_device(ref, got):
+    """Oracle weight / gradient of a convolution in the device's shape: the centre tap for a 1 x 1 layer."""
+    ref = np.asarray(ref)
+    return ref[:, :, 1:2, 1:2] if (ref.ndim == 4 and got.shape[-1] == 1 and ref.shape[-1] == 3) else ref
+
 def oracle_conv_step(w, inp, strips=None, grid=None):
     """fp64 oracle step for a domain-parallel conv workload (NCHW); stored activations are
     rounded to bf16 like the device's.  `strips` = P_r (or `grid` = (P_r, P_c)) runs the
     strip / halo formulation."""
     from oracle import mbd_oracle as O
-    layers = [O.Conv3x3(k.astype(np.float64), relu=True) for k in inp.Ws]
+    layers = [O.Conv3x3(oracle_kernel(k), relu=True) for k in inp.Ws]
     X = inp.X.astype(np.float64)
     if strips is None and grid is None:
         return O.train_step(layers, X, None, "half_ssq", w.eta, store=bf16_store)
@@ -158,7 +174,8 @@ def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1):
     from paper_1712_04432_b200 import mbd
     C_, H, Wd = w.dims
     L = w.n_layers
-    net = mbd.Net(mbd.conv_layers(L, C_, H, Wd), w.B, P_r, P_c, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+    net = mbd.Net(mbd.conv_layers(L, C_, H, Wd, k=[w.ksize(i) for i in range(L)]), w.B, P_r, P_c, mbd.BF16,
+                  mbd.LOSS_HALF_SSQ, 0)
     for i in range(L):
         net.set_weights(i, to_dev(inp.Ws[i], True))
     X = to_dev(inp.X, True)
@@ -202,8 +219,8 @@ def compare_conv_step(g, o, tol, fused=False, tol_below_relu=None):
         tg = tol if i == L - 1 else tol_below_relu
         chk(f"dY[{i}]", g["dY"][i], o["dYs"][i], tg)
         if not fused:
-            chk(f"dK[{i}]", g["dW"][i], o["dWs"][i], tg)
-        chk(f"K_new[{i}]", g["new_W"][i], o["new_W"][i], tol)
+            chk(f"dK[{i}]", g["dW"][i], like_device(o["dWs"][i], g["dW"][i]), tg)
+        chk(f"K_new[{i}]", g["new_W"][i], like_device(o["new_W"][i], g["new_W"][i]), tol)
     assert not bad, "rel. Frobenius error too large for %s: %s" % (bad, "; ".join(report))
     return report
 
@@ -216,7 +233,7 @@ def oracle_mixed_step(w, inp, blocked_grid=None):
     flattened activation; stored activations rounded to bf16 like the device's."""
     from oracle import mbd_oracle as O
     Lc = w.n_layers
-    layers = [O.Conv3x3(inp.Ws[i].astype(np.float64), relu=True) for i in range(Lc)]
+    layers = [O.Conv3x3(oracle_kernel(inp.Ws[i]), relu=True) for i in range(Lc)]
     for i in range(Lc, w.L):
         layers.append(O.FC(inp.Ws[i].astype(np.float64), inp.bs[i].astype(np.float64), relu=True))
     X = inp.X.astype(np.float64)
@@ -228,7 +245,7 @@ def oracle_mixed_step(w, inp, blocked_grid=None):
 def mixed_layers(w):
     from paper_1712_04432_b200 import mbd
     C_, H, Wd = w.dims
-    return mbd.conv_layers(w.n_layers, C_, H, Wd) + mbd.fc_layers(w.fc_dims, bias=True)
+    return mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.ksize(i) for i in range(w.n_layers)]) + mbd.fc_layers(w.fc_dims, bias=True)
 
 
 def oracle_mixed_acts(o, w):
@@ -316,10 +333,10 @@ def compare_mixed_step(g, o, w, tol, fused=False, tol_below_relu=None):
         tg = tol if i == L - 1 else tol_below_relu
         chk(f"dY[{i}]", g["dY"][i], dev_layout(o["dYs"][i], i), tg)
         if not fused:
-            chk(f"dW[{i}]", g["dW"][i], o["dWs"][i], tg)
+            chk(f"dW[{i}]", g["dW"][i], like_device(o["dWs"][i], g["dW"][i]), tg)
             if i >= Lc:
                 chk(f"db[{i}]", g["db"][i], o["dbs"][i], tg)
-        chk(f"W_new[{i}]", g["new_W"][i], o["new_W"][i], tol)
+        chk(f"W_new[{i}]", g["new_W"][i], like_device(o["new_W"][i], g["new_W"][i]), tol)
         if i >= Lc:
             ref_b = o["new_b"][i]
             assert np.abs(g["new_b"][i] - ref_b).max() <= tol * max(1.0, np.abs(ref_b).max()), f"b_new[{i}]"

@@ -38,6 +38,10 @@ def test_invalid_and_unsupported():
     conv5 = mbd.conv_layers(1, 64, 8, 16)
     conv5[0].kh = conv5[0].kw = 5
     assert create(conv5, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
+    conv13 = mbd.conv_layers(1, 64, 8, 16)
+    conv13[0].kh = 1                                                                       # 1 x 3: neither 3 x 3 nor 1 x 1
+    assert create(conv13, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
+    assert create(mbd.conv_layers(2, 64, 8, 16, k=[3, 1]), 4, loss=mbd.LOSS_HALF_SSQ) in (mbd.OK, mbd.E_CUDA)   # valid; E_CUDA only without a device
     assert create(mbd.conv_layers(1, 64, 8, 16), 4, loss=mbd.LOSS_SOFTMAX_CE) == mbd.E_UNSUPPORTED
     # convolutions first, fully connected layers after them
     conv = mbd.conv_layers(1, 64, 8, 16)

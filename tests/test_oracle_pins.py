@@ -482,3 +482,19 @@ def test_conv_weight_gradient_partials_over_the_whole_grid():
     _, parts = O.conv3x3_dK_grid(dY, X, 2, 3)
     Xz = X[0:2].copy(); dYz = dY[0:2].copy(); dYz[:, :, 0:4, :] = 0.0          # only output rows 4..7 contribute
     assert relerr(parts[1], O.conv3x3_dK(dYz, Xz)) < 1e-13
+
+
+def test_centre_tap_gradient_is_the_per_pixel_outer_product_sum():
+    """The gradient of the centre tap is the fully connected weight gradient with every pixel as a sample
+    (the 1 x 1 convolution singled out after Eq. 7): sum over b, h, w of dY[b, o, h, w] X[b, c, h, w]."""
+    K, X, dY = conv_case(seed=76)
+    dK = O.conv3x3_dK(dY, X)
+    B, C_, H, W = X.shape
+    for o_ in range(dY.shape[1]):
+        for c in range(C_):
+            acc = 0.0
+            for b in range(B):
+                for h in range(H):
+                    for w in range(W):
+                        acc += dY[b, o_, h, w] * X[b, c, h, w]
+            assert abs(acc - dK[o_, c, 1, 1]) < 1e-11

@@ -143,3 +143,18 @@ def test_second_step_uses_the_updated_kernels(mode):
     for i in range(2):
         assert rel_fro(to_np(net.get_weights(i)), o2["new_W"][i]) <= TOL
     net.close()
+
+
+@pytest.mark.parametrize("ksizes", [(3, 1, 3), (1, 3), (1, 1), (3, 1)])
+@pytest.mark.parametrize("P_r", [1, 4])
+@pytest.mark.parametrize("fused", [False, True])
+def test_one_by_one_layers(ksizes, P_r, fused):
+    """1 x 1 convolutions (the layers that need no halo, remark after Eq. 7) between, below and above
+    3 x 3 ones; weights, gradients and updates are [C_out, C_in, 1, 1] at the boundary."""
+    w = I.conv_workload(64, 8, 130, 3, n_layers=len(ksizes), name="conv_1x1", ksizes=ksizes)
+    inp = I.make_inputs(w, seed=70 + len(ksizes) + ksizes[0])
+    assert [k.shape[-1] for k in inp.Ws] == list(ksizes)
+    o = oracle_conv_step(w, inp)
+    g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o))
+    assert [a.shape[-1] for a in g["new_W"]] == list(ksizes)
+    compare_conv_step(g, o, TOL, fused)

@@ -115,3 +115,12 @@ def test_conv_stack_with_batch_blocks(grid):
     hidden = [np.ascontiguousarray(x, np.float32) for x in o["Xs"][1:]]
     g = gpu_conv_step(w, inp, grid[0], P_c=grid[1], force_acts=hidden)
     compare_conv_step(g, o, TOL)
+
+
+def test_one_by_one_convolution_below_fully_connected_layers():
+    w = I.mixed_workload(64, 8, 40, 2, (128, 16), 6, name="mixed_1x1", ksizes=(3, 1))
+    inp = I.make_inputs(w, seed=34)
+    o = oracle_mixed_step(w, inp)
+    for grid, fused in [((1, 1), False), ((4, 3), True)]:
+        g = gpu_mixed_step(w, inp, grid, 4, fused=fused, force_acts=oracle_mixed_acts(o, w))
+        compare_mixed_step(g, o, w, TOL, fused)
