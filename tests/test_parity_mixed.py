@@ -124,3 +124,26 @@ def test_one_by_one_convolution_below_fully_connected_layers():
     for grid, fused in [((1, 1), False), ((4, 3), True)]:
         g = gpu_mixed_step(w, inp, grid, 4, fused=fused, force_acts=oracle_mixed_acts(o, w))
         compare_mixed_step(g, o, w, TOL, fused)
+
+
+@pytest.mark.parametrize("case", range(8))
+def test_seeded_random_integrated_stacks(case):
+    """Depth of both groups, kernel sizes, image shape (from one pixel column groups of eight strips per tile
+    to two segments per row), batch, grid, number of materialised partials and fused / un-fused update drawn
+    from a seeded generator."""
+    r = np.random.default_rng(5000 + case)
+    n_conv = int(r.integers(1, 4))
+    ksizes = tuple(int(k) for k in r.choice([1, 3], size=n_conv))
+    H = int(r.choice([4, 6, 8, 12]))
+    W = int(r.choice([int(r.integers(3, 15)), int(r.integers(15, 31)), int(r.integers(31, 63)), int(r.integers(63, 150))]))
+    B = int(r.integers(1, 8))
+    fc = tuple(8 * int(r.integers(1, 13)) for _ in range(int(r.integers(1, 4))))
+    P_r = int(r.choice([p for p in range(1, H + 1) if H % p == 0 and p <= min(fc)]))
+    P_c = int(r.integers(1, B + 1))
+    mp = int(r.choice([1, 2, 4, 64]))
+    fused = bool(r.integers(0, 2))
+    w = I.mixed_workload(64, H, W, n_conv, fc, B, name=f"mixed_random{case}", ksizes=ksizes)
+    inp = I.make_inputs(w, seed=200 + case)
+    o = oracle_mixed_step(w, inp)
+    g = gpu_mixed_step(w, inp, (P_r, P_c), mp, fused=fused, force_acts=oracle_mixed_acts(o, w))
+    compare_mixed_step(g, o, w, TOL, fused)
