@@ -96,7 +96,8 @@ enum {
   MBD_T_DW = 2,       /* dW_i, float, weight shape (valid after mbd_backward(net, 0))        */
   MBD_T_DB = 3,       /* db_i, float [d_i]                                                   */
   MBD_T_LOSS = 4,     /* per-sample loss, float [B] (softmax-CE); layer ignored              */
-  MBD_T_PARTIALS = 5  /* fp32 partial-sum workspace as left by the LAST reduction executed   */
+  MBD_T_PARTIALS = 5, /* fp32 partial-sum workspace as left by the LAST reduction executed   */
+  MBD_T_MASTER = 6    /* fp32 master weights, weight shape (get only; after mbd_enable_master_weights) */
 };
 
 /* Section 2.3 / 2.4.  Builds the plan for an L-layer network on batch B over a
@@ -124,6 +125,14 @@ enum {
 MBD_API mbd_status mbd_net_create(const mbd_layer* layers_host, int L, int64_t B, int P_r, int P_c,
                           int dtype, int loss, int max_partials, void* cuda_stream, mbd_net** out);
 MBD_API mbd_status mbd_net_destroy(mbd_net* net);
+
+/* Optional, bf16 networks: keep an fp32 master copy of every weight.  Eq. 1 is then applied to the
+ * master (w32 += -(eta/B) dW, from the fp32 gradient) and the bf16 weights the contractions read are
+ * the rounded master, so updates below half a bf16 ulp accumulate instead of being lost.  Costs
+ * 4 + 4 + 2 bytes of update traffic per weight plus the fp32 gradient instead of 2 + 2 (the update
+ * leaves the contraction's epilogue).  The masters start from the current weights and follow every
+ * later mbd_set_weights.  MBD_E_UNSUPPORTED for an fp32 network (its weights are fp32 already). */
+MBD_API mbd_status mbd_enable_master_weights(mbd_net* net);
 
 /* Copy weights (network dtype) and bias (float, may be NULL) device -> library / back. */
 MBD_API mbd_status mbd_set_weights(mbd_net* net, int layer, const void* W_dev, const float* bias_dev);

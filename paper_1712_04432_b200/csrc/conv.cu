@@ -202,7 +202,7 @@ __global__ void extract_1x1_kernel(const T* __restrict__ K, T* __restrict__ K1) 
 // two operand layouts the next step's kernels read (see pack_weights_kernel).
 __global__ void __launch_bounds__(256)
 wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ dK, bf16* __restrict__ K,
-                    bf16* __restrict__ Wf, bf16* __restrict__ Wb, float scale, int centre_only) {
+                    bf16* __restrict__ Wf, bf16* __restrict__ Wb, float* __restrict__ K32, float scale, int centre_only) {
   // 64 outputs per block; four thread groups each add a contiguous quarter of the CTA partials in
   // ascending order, and the four sub-sums are added in ascending order too (a fixed order).
   __shared__ float sub[4][64];
@@ -231,7 +231,14 @@ wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ d
   }
   if (dK) dK[e] = s;
   if (K) {
-    const bf16 k = __float2bfloat16_rn(fmaf(scale, s, __bfloat162float(K[e])));
+    bf16 k;
+    if (K32) {                       // fp32 master weights: the bf16 kernel is the rounded master
+      const float m = fmaf(scale, s, K32[e]);
+      K32[e] = m;
+      k = __float2bfloat16_rn(m);
+    } else {
+      k = __float2bfloat16_rn(fmaf(scale, s, __bfloat162float(K[e])));
+    }
     const int u = t / 3, v = t - 3 * u;
     K[e] = k;
     Wf[((v * 3 + u) * C + o) * C + c] = k;
@@ -853,6 +860,7 @@ struct ConvNet {
   std::vector<bf16*> dY;             // dY[i]: gradient w.r.t. the output of layer i; dY[L-1] == act[L]
   std::vector<bf16*> K, Wf, Wb;
   std::vector<float*> dK;
+  std::vector<float*> K32;           // fp32 master weights (empty unless enabled)
   std::vector<int> relu;
   std::vector<int> k1;               // 1 x 1 layer: weights in the centre tap, outer taps zero
   std::vector<CUtensorMap> act_fwd, dY_fwd, dY_wg, wf_map, wb_map;   // act_fwd / dY_fwd: 130-pixel boxes (also the X operand of backward-weight)
@@ -957,6 +965,7 @@ void conv_destroy(ConvNet* c) {
   for (int i = 0; i < c->L; ++i)
     if (c->dY[i] != c->act[c->L]) cudaFree(c->dY[i]);
   for (int i = 0; i < c->L; ++i) { cudaFree(c->K[i]); cudaFree(c->Wf[i]); cudaFree(c->Wb[i]); cudaFree(c->dK[i]); }
+  for (float* m : c->K32) cudaFree(m);
   cudaFree(c->wpart); cudaFree(c->loss_part); cudaFree(c->scratch_nchw);
   (void)cudaGetLastError();
   delete c;
@@ -978,7 +987,23 @@ mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev) {
   } else if (cudaMemcpyAsync(c->K[layer], K_dev, 9 * C * C * 2, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) {
     return MBD_E_CUDA;
   }
+  if (!c->K32.empty() && widen_bf16_launch(c->K[layer], c->K32[layer], 9 * C * C, c->num_sms, c->stream) != cudaSuccess) return MBD_E_CUDA;
   return launch_pack(c, layer);
+}
+
+mbd_status conv_enable_master(ConvNet* c) {
+  if (!c->K32.empty()) return MBD_OK;
+  std::vector<float*> m(c->L, nullptr);
+  for (int i = 0; i < c->L; ++i) {
+    if (cudaMalloc(reinterpret_cast<void**>(&m[i]), 9 * C * C * 4) != cudaSuccess ||
+        widen_bf16_launch(c->K[i], m[i], 9 * C * C, c->num_sms, c->stream) != cudaSuccess) {
+      (void)cudaGetLastError();
+      for (float* q : m) cudaFree(q);
+      return MBD_E_ALLOC;
+    }
+  }
+  c->K32 = m;
+  return MBD_OK;
 }
 
 mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev) {
@@ -1035,7 +1060,8 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
     c->prof->end();
     c->prof->begin(MBD_K_REDUCE, (grid + 1.0) * 9 * C * C * 4.0);
     wgrad_finish_kernel<<<9 * C * C / 64, 256, 0, c->stream>>>(c->wpart, grid, fused ? nullptr : c->dK[i],
-                                                                      fused ? c->K[i] : nullptr, c->Wf[i], c->Wb[i], scale, c->k1[i]);
+                                                                      fused ? c->K[i] : nullptr, c->Wf[i], c->Wb[i],
+                                                                      c->K32.empty() ? nullptr : c->K32[i], scale, c->k1[i]);
     c->prof->end();
   }
   if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
@@ -1047,7 +1073,9 @@ mbd_status conv_sgd_step(ConvNet* c, float eta) {
   const float scale = -eta / static_cast<float>(c->B);
   for (int i = 0; i < c->L; ++i) {
     c->prof->begin(MBD_K_SGD, 9.0 * C * C * 8.0);
-    if (sgd_update_launch(c->K[i], 1, c->dK[i], 9 * C * C, scale, c->num_sms, c->stream) != cudaSuccess) return MBD_E_CUDA;
+    const cudaError_t e = c->K32.empty() ? sgd_update_launch(c->K[i], 1, c->dK[i], 9 * C * C, scale, c->num_sms, c->stream)
+                                         : sgd_master_update_launch(c->K32[i], c->K[i], c->dK[i], 9 * C * C, scale, c->num_sms, c->stream);
+    if (e != cudaSuccess) return MBD_E_CUDA;
     c->prof->end();
     if (launch_pack(c, i) != MBD_OK) return MBD_E_CUDA;
   }
@@ -1075,15 +1103,17 @@ int conv_last_relu(const ConvNet* c) { return c->relu[c->L - 1]; }
 
 mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t bytes) {
   const size_t nchw_bytes = conv_input_bytes(c);
-  if (which == MBD_T_DW) {
+  if (which == MBD_T_DW || which == MBD_T_MASTER) {
     if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
+    if (which == MBD_T_MASTER && c->K32.empty()) return MBD_E_STATE;
+    const float* src32 = which == MBD_T_DW ? c->dK[layer] : c->K32[layer];
     if (c->k1[layer]) {
       if (bytes != C * C * 4) return MBD_E_INVALID;
-      extract_1x1_kernel<float><<<(C * C + 255) / 256, 256, 0, c->stream>>>(c->dK[layer], static_cast<float*>(dst));
+      extract_1x1_kernel<float><<<(C * C + 255) / 256, 256, 0, c->stream>>>(src32, static_cast<float*>(dst));
       return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
     }
     if (bytes != 9 * C * C * 4) return MBD_E_INVALID;
-    if (cudaMemcpyAsync(dst, c->dK[layer], bytes, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) return MBD_E_CUDA;
+    if (cudaMemcpyAsync(dst, src32, bytes, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) return MBD_E_CUDA;
     return MBD_OK;
   }
   if (which == MBD_T_PARTIALS) {

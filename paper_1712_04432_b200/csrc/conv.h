@@ -24,4 +24,5 @@ size_t conv_input_bytes(const ConvNet* c);
 mbd_status conv_output_to_nchw(ConvNet* c, void* dst);
 mbd_status conv_top_grad_from_nchw(ConvNet* c, const void* src);
 int conv_last_relu(const ConvNet* c);
+mbd_status conv_enable_master(ConvNet* c);     // fp32 master weights from now on
 }  // namespace mbd

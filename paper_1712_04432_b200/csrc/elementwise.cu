@@ -310,6 +310,39 @@ sgd_update_scalar(void* __restrict__ w, int w_bf16, const float* __restrict__ g,
   }
 }
 
+// Eq. 1 on fp32 master weights: w32 += scale * g, and the bf16 working copy the contractions read is the
+// rounded master (updates smaller than half a bf16 ulp are kept in the master instead of being lost).
+__global__ void __launch_bounds__(256)
+sgd_master_update_kernel(float* __restrict__ w32, __nv_bfloat16* __restrict__ w, const float* __restrict__ g, int64_t n,
+                         float scale) {
+  pdl_wait();
+  const int64_t n4 = n >> 2;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n4;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const float4 a = __ldcs(reinterpret_cast<const float4*>(g + i * 4));
+    float4 m = *reinterpret_cast<const float4*>(w32 + i * 4);
+    m.x = fmaf(scale, a.x, m.x); m.y = fmaf(scale, a.y, m.y); m.z = fmaf(scale, a.z, m.z); m.w = fmaf(scale, a.w, m.w);
+    *reinterpret_cast<float4*>(w32 + i * 4) = m;
+    uint2 o;
+    o.x = pack_bf16x2(m.x, m.y);
+    o.y = pack_bf16x2(m.z, m.w);
+    *reinterpret_cast<uint2*>(w + i * 4) = o;
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (n & 3)) {          // tail
+    const int64_t i = (n4 << 2) + threadIdx.x;
+    const float m = fmaf(scale, g[i], w32[i]);
+    w32[i] = m;
+    w[i] = __float2bfloat16_rn(m);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+widen_bf16_kernel(const __nv_bfloat16* __restrict__ w, float* __restrict__ w32, int64_t n) {
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x)
+    w32[i] = __bfloat162float(w[i]);
+}
+
 int grid_for(int64_t work_items, int num_sms, int per_sm) {
   int64_t blocks = (work_items + 255) / 256;
   const int64_t cap = static_cast<int64_t>(num_sms) * per_sm;
@@ -374,6 +407,17 @@ cudaError_t sgd_update_launch(void* w, int w_bf16, const float* g, int64_t n, fl
     return launch_pdl(sgd_update_bf16_vec8, dim3(grid_for(n / 8, num_sms, 8)), dim3(256), 0, stream, 0, reinterpret_cast<__nv_bfloat16*>(w), g, n / 8, scale);
   }
   return launch_pdl(sgd_update_scalar, dim3(grid_for(n, num_sms, 8)), dim3(256), 0, stream, 0, w, w_bf16, g, n, scale);
+}
+
+cudaError_t sgd_master_update_launch(float* w32, void* w_bf16, const float* g, int64_t n, float scale, int num_sms,
+                                     cudaStream_t stream) {
+  return launch_pdl(sgd_master_update_kernel, dim3(grid_for((n + 3) / 4, num_sms, 8)), dim3(256), 0, stream, 0, w32,
+                    reinterpret_cast<__nv_bfloat16*>(w_bf16), g, n, scale);
+}
+
+cudaError_t widen_bf16_launch(const void* w_bf16, float* w32, int64_t n, int num_sms, cudaStream_t stream) {
+  widen_bf16_kernel<<<grid_for(n, num_sms, 8), 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(w_bf16), w32, n);
+  return cudaGetLastError();
 }
 
 }  // namespace mbd

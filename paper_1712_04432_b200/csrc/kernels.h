@@ -142,6 +142,11 @@ int colsum_launches(int64_t M, int64_t N, int num_sms);    // kernels one colsum
 cudaError_t sgd_update_launch(void* w, int w_bf16, const float* g, int64_t n, float scale,
                               int num_sms, cudaStream_t stream);
 
+// fp32 master weights: w32[i] += scale * g[i]; w_bf16[i] = round(w32[i]).  widen: w32[i] = w_bf16[i].
+cudaError_t sgd_master_update_launch(float* w32, void* w_bf16, const float* g, int64_t n, float scale,
+                                     int num_sms, cudaStream_t stream);
+cudaError_t widen_bf16_launch(const void* w_bf16, float* w32, int64_t n, int num_sms, cudaStream_t stream);
+
 // ---- per-class event timing (host) ---------------------------------------------------------
 struct Profiler {
   static constexpr int NCLS = 12;

@@ -29,6 +29,7 @@ struct Layer {
   void* W = nullptr;
   float* bias = nullptr;
   float* dW = nullptr;
+  float* W32 = nullptr;  // fp32 master weights (optional)
   float* db = nullptr;
   void* act = nullptr;   // stored forward output [B, d_out]; float logits for the last FC layer
   void* dY = nullptr;    // [B, d_out] activation dtype
@@ -49,6 +50,7 @@ struct mbd_net {
   int num_sms = 148;
   int device = 0;
   bool is_conv = false;
+  bool master = false;              // fp32 master weights: the update leaves the contraction's epilogue
   std::vector<Layer> layers;
   float* partials = nullptr;
   size_t partial_elems = 0;
@@ -235,7 +237,7 @@ mbd_status map_input(mbd_net* n) {
 void free_net(mbd_net* n) {
   if (!n) return;
   for (Layer& l : n->layers) {
-    cudaFree(l.W); cudaFree(l.bias); cudaFree(l.dW); cudaFree(l.db); cudaFree(l.act); cudaFree(l.dY);
+    cudaFree(l.W); cudaFree(l.bias); cudaFree(l.dW); cudaFree(l.db); cudaFree(l.act); cudaFree(l.dY); cudaFree(l.W32);
   }
   cudaFree(n->partials); cudaFree(n->colsum_scratch); cudaFree(n->per_sample); cudaFree(n->loss_dev);
   cudaFree(n->status); cudaFree(n->X_stage); cudaFree(n->labels_stage); cudaFree(n->X_fc); cudaFree(n->dX_fc);
@@ -442,10 +444,29 @@ extern "C" mbd_status mbd_set_weights(mbd_net* n, int layer, const void* W_dev, 
   if (layer < n->Lc) return bias_dev ? MBD_E_INVALID : conv_set_weights(n->conv, layer, W_dev);
   Layer& l = n->layers[layer - n->Lc];
   CK(cudaMemcpyAsync(l.W, W_dev, l.nW * n->elt(), cudaMemcpyDeviceToDevice, n->stream));
+  if (l.W32) CK(widen_bf16_launch(l.W, l.W32, l.nW, n->num_sms, n->stream));
   if (bias_dev) {
     if (!l.bias) return MBD_E_INVALID;
     CK(cudaMemcpyAsync(l.bias, bias_dev, l.d_out * sizeof(float), cudaMemcpyDeviceToDevice, n->stream));
   }
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_enable_master_weights(mbd_net* n) {
+  if (!n) return MBD_E_INVALID;
+  if (n->dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
+  if (n->master) return MBD_OK;
+  if (n->conv) {
+    const mbd_status s = conv_enable_master(n->conv);
+    if (s != MBD_OK) return s;
+  }
+  for (Layer& l : n->layers) {
+    const mbd_status s = dev_alloc(reinterpret_cast<void**>(&l.W32), l.nW * sizeof(float));
+    if (s != MBD_OK) return s;
+    CK(widen_bf16_launch(l.W, l.W32, l.nW, n->num_sms, n->stream));
+  }
+  n->master = true;
+  if (n->graph_exec) { cudaGraphExecDestroy(n->graph_exec); n->graph_exec = nullptr; }   // the step's launches change
   return MBD_OK;
 }
 
@@ -548,7 +569,9 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
       mbd_status s = run_gemm(n, l.bwd_data, 1, n->B, l.d_in, l.d_out, l.dY, l.d_out, l.W, l.d_in, S_r, e);
       if (s != MBD_OK) return s;
     }
-    const Epi e = fused ? epi_sgd(l.W, l.d_in, bf, scale) : epi_act(l.dW, l.d_in, 0, nullptr, 0);
+    // with master weights the gradient is materialised and Eq. 1 is applied to the master by its own kernel
+    const bool in_epilogue = fused && !n->master;
+    const Epi e = in_epilogue ? epi_sgd(l.W, l.d_in, bf, scale) : epi_act(l.dW, l.d_in, 0, nullptr, 0);
     cudaStream_t ws = nullptr;
     if (n->overlap_dw) {
       // dY_i is final and the last reader of the old W_i has been enqueued: dW_i may start beside
@@ -561,6 +584,12 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
     mbd_status s = run_gemm(n, l.bwd_weight, 2, l.d_out, l.d_in, n->B, l.dY, l.d_out, layer_input(n, i), l.d_in, S_c, e, ws,
                             ws ? n->partials_dw : nullptr);
     if (s != MBD_OK) return s;
+    if (fused && n->master) {
+      cudaStream_t us = ws ? ws : n->stream;
+      n->prof.begin(MBD_K_SGD, static_cast<double>(l.nW) * 14.0, us);
+      CK(sgd_master_update_launch(l.W32, l.W, l.dW, l.nW, scale, n->num_sms, us));
+      n->prof.end();
+    }
   }
   if (dw_forked) {
     CK(cudaEventRecord(n->ev_wjoin, n->wstream));
@@ -596,8 +625,9 @@ extern "C" mbd_status mbd_sgd_step(mbd_net* n, float eta) {
   }
   for (int i = 0; i < n->L; ++i) {
     Layer& l = n->layers[i];
-    n->prof.begin(MBD_K_SGD, static_cast<double>(l.nW) * (4.0 + 2.0 * n->elt()));
-    CK(sgd_update_launch(l.W, n->dtype == MBD_BF16, l.dW, l.nW, scale, n->num_sms, n->stream));
+    n->prof.begin(MBD_K_SGD, static_cast<double>(l.nW) * (n->master ? 14.0 : 4.0 + 2.0 * n->elt()));
+    if (n->master) CK(sgd_master_update_launch(l.W32, l.W, l.dW, l.nW, scale, n->num_sms, n->stream));
+    else CK(sgd_update_launch(l.W, n->dtype == MBD_BF16, l.dW, l.nW, scale, n->num_sms, n->stream));
     n->prof.end();
     if (l.bias) {
       n->prof.begin(MBD_K_SGD, static_cast<double>(l.d_out) * 12.0);
@@ -758,6 +788,7 @@ extern "C" mbd_status mbd_get_tensor(mbd_net* n, int which, int layer, void* dst
       case MBD_T_ACT: src = l.act; size = static_cast<size_t>(n->B) * l.d_out * (last ? sizeof(float) : n->elt()); break;
       case MBD_T_DY: src = l.dY; size = static_cast<size_t>(n->B) * l.d_out * n->elt(); break;
       case MBD_T_DW: src = l.dW; size = l.nW * sizeof(float); break;
+      case MBD_T_MASTER: src = l.W32; size = l.nW * sizeof(float); break;
       case MBD_T_DB: src = l.db; size = l.d_out * sizeof(float); break;
       default: return MBD_E_INVALID;
     }

@@ -18,7 +18,7 @@ FC, CONV3X3 = 0, 1
 SPLIT_MODEL, SPLIT_DOMAIN = 0, 1
 F32, BF16 = 0, 1
 LOSS_SOFTMAX_CE, LOSS_HALF_SSQ = 0, 1
-T_ACT, T_DY, T_DW, T_DB, T_LOSS, T_PARTIALS = range(6)
+T_ACT, T_DY, T_DW, T_DB, T_LOSS, T_PARTIALS, T_MASTER = range(7)
 
 KERNEL_CLASSES = ["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce_partials", "softmax_xent", "colsum",
                   "sgd_update", "halo_stage", "conv_fwd", "conv_bwd_data", "conv_bwd_weight", "other"]
@@ -27,7 +27,8 @@ EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weig
            "mbd_backward", "mbd_sgd_step", "mbd_train_step", "mbd_train_step_host", "mbd_comm_words", "mbd_get_tensor",
            "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_gemm_bf16_noalloc", "mbd_selftest_timeout", "mbd_strerror",
            "mbd_train_step_host_begin", "mbd_train_step_host_end",
-           "mbd_comm_time", "mbd_redistribute_time", "mbd_total_time", "mbd_grid_table", "mbd_choose_grid"]
+           "mbd_comm_time", "mbd_redistribute_time", "mbd_total_time", "mbd_grid_table", "mbd_choose_grid",
+           "mbd_enable_master_weights"]
 
 
 class MbdError(RuntimeError):
@@ -105,6 +106,7 @@ def lib():
         L.mbd_get_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
         L.mbd_set_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
         L.mbd_poll_status.argtypes = [vp]
+        L.mbd_enable_master_weights.argtypes = [vp]
         L.mbd_profile_enable.argtypes = [vp, i32]
         L.mbd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double)]
         L.mbd_launch_count.argtypes = [vp]
@@ -269,6 +271,10 @@ class Net:
         self._keep = [X, labels, loss_out]      # the library reads X again during backward
         _check(lib().mbd_forward(self._h, _ptr(X), _ptr(labels), _ptr(loss_out)), "mbd_forward")
 
+    def enable_master_weights(self):
+        """fp32 master copies of all weights from now on (see include/mbd.h)."""
+        _check(lib().mbd_enable_master_weights(self._h), "mbd_enable_master_weights")
+
     def backward(self, fused_eta: float = 0.0):
         _check(lib().mbd_backward(self._h, float(fused_eta)), "mbd_backward")
 
@@ -311,7 +317,7 @@ class Net:
                 (t.float32 if (last and not conv) else self.act_dtype)
         elif which == T_DY:
             shape, dt = ((self.B, l.C_out, l.H, l.W) if conv else (self.B, l.d_out)), self.act_dtype
-        elif which == T_DW:
+        elif which in (T_DW, T_MASTER):
             shape, dt = self._wshape(layer), t.float32
         elif which == T_DB:
             shape, dt = (l.d_out,), t.float32

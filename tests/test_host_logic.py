@@ -57,6 +57,7 @@ def test_null_handles_are_rejected():
     assert L.mbd_backward(None, 0.0) == mbd.E_INVALID
     assert L.mbd_sgd_step(None, 0.1) == mbd.E_INVALID
     assert L.mbd_poll_status(None) == mbd.E_INVALID
+    assert L.mbd_enable_master_weights(None) == mbd.E_INVALID
     assert L.mbd_launch_count(None) == -1
     assert L.mbd_net_destroy(None) == mbd.E_INVALID
 
