@@ -285,6 +285,42 @@ MBD_API mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, c
                          int64_t lda, const void* B_dev, int64_t ldb, float* D_dev, int64_t ldd,
                          int k_splits, float* partials_dev, void* cuda_stream);
 
+/* ---- Block operations for a multi-process driver of the grid (Section 2.3; Appendix A.1 / A.2) ----
+ * What one process (r, c) does between two collectives, on caller-owned device buffers: a block product
+ * with its tail operation fused, the tail operation applied to a sum that a collective delivered, and
+ * the loss.  Every call enqueues on cuda_stream and returns after the stream has drained (MBD_E_TIMEOUT
+ * if a bounded wait inside a kernel gave up).
+ *
+ * mbd_tail: what happens to a finished fp32 element acc at (m, n):
+ *   MBD_TAIL_STORE  out = acc (+ bias_dev[n]); relu != 0: max(., 0)
+ *   MBD_TAIL_MASK   out = (mask_dev == NULL || mask_dev[m, n] > 0) ? acc : 0      (ReLU derivative)
+ *   MBD_TAIL_SGD    out = out + scale * acc                                          (Eq. 1, scale = -eta/B)
+ * out_dev is [M, ldo] bf16 (out_bf16 != 0) or float; mask_dev has out's element type and ldmask.
+ * Leading dimensions in elements, multiples of 8 for the contraction (as for mbd_gemm_bf16). */
+enum { MBD_TAIL_STORE = 0, MBD_TAIL_MASK = 1, MBD_TAIL_SGD = 2 };
+typedef struct {
+  int32_t op, out_bf16, relu, reserved;
+  void* out_dev;
+  int64_t ldo;
+  const float* bias_dev;
+  const void* mask_dev;
+  int64_t ldmask;
+  float scale;
+} mbd_tail;
+
+/* One block product (variants and operand layouts of mbd_gemm_bf16, K not split) with `tail` fused. */
+MBD_API mbd_status mbd_block_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, const void* A_dev,
+                               int64_t lda, const void* B_dev, int64_t ldb, const mbd_tail* tail,
+                               void* cuda_stream);
+/* sum_{s < S} parts_dev[s] (planes of M x N floats, ascending s), then `tail`.  S = 1 applies the tail
+ * operation to a sum that is already complete (e.g. after an all-reduce). */
+MBD_API mbd_status mbd_block_reduce(const float* parts_dev, int S, int64_t M, int64_t N, const mbd_tail* tail,
+                            void* cuda_stream);
+/* Softmax cross-entropy of float logits [B, d]: per_sample_dev[b] = loss of sample b (natural log),
+ * dY_dev [B, d] = softmax - onehot (bf16 if dY_bf16 != 0, else float).  labels_dev: int32 in [0, d). */
+MBD_API mbd_status mbd_softmax_xent(const float* logits_dev, int64_t B, int64_t d, const int32_t* labels_dev,
+                            void* dY_dev, int dY_bf16, float* per_sample_dev, void* cuda_stream);
+
 /* Failure-detection self test: launches one small kernel whose only job is to wait, with a
  * limit of `limit_ms` milliseconds, on a barrier that nothing will ever signal.  The kernel
  * gives up when the limit runs out, records a status code and returns normally; the call then

@@ -1,0 +1,173 @@
+"""One training step of a fully connected stack executed for real over a P_r x P_c grid of PROCESSES
+(Section 2.3, Fig. 5; Appendix A.1 / A.2): process (r, c) owns the row block W_i(r, :) of every weight
+matrix and the batch block c of the samples.
+
+    forward    Y_i(r, c) = W_i(r, :) X_i(:, c)                   block product, ReLU fused
+               all-gather over the P_r group                     -> X_{i+1}(:, c)              Eq. 8, term 1
+    backward   dX_i partial = W_i(r, :)^T dY_i(r, c)             block product, fp32
+               all-reduce over the P_r group, ReLU mask          -> dY_{i-1}(:, c)             Eq. 8, term 2
+               dW_i(r, :) partial = dY_i(r, c) X_i(:, c)^T       block product, fp32
+               all-reduce over the P_c group, Eq. 1              -> W_i(r, :) updated          Eq. 8, term 3
+
+Every arithmetic step runs in the library's kernels (mbd_block_gemm_bf16, mbd_block_reduce,
+mbd_softmax_xent); torch.distributed only moves the blocks.  With the "nccl" backend the collectives run
+on the device buffers; with "gloo" (tests: several processes sharing one GPU) they go through host copies.
+The words every collective moves per process are counted from the buffers actually exchanged, so that
+they can be compared with mbd_comm_words.
+
+Rank layout: rank = c * P_r + r.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Sequence
+
+from . import mbd
+
+
+def grid_coords(rank: int, P_r: int, P_c: int):
+    assert 0 <= rank < P_r * P_c
+    return rank % P_r, rank // P_r
+
+
+class GridComm:
+    """The two process groups of one rank and the collectives of the step, with word accounting.
+
+    Words per process follow the bandwidth-optimal algorithms the paper assumes: an all-gather over p
+    processes of n words each receives (p - 1) n; an all-reduce of n words moves 2 (p - 1) / p * n."""
+
+    def __init__(self, P_r: int, P_c: int, via_host: bool = False):
+        import torch.distributed as dist
+        self.dist = dist
+        self.P_r, self.P_c = P_r, P_c
+        assert dist.get_world_size() == P_r * P_c
+        self.rank = dist.get_rank()
+        self.r, self.c = grid_coords(self.rank, P_r, P_c)
+        self.via_host = via_host
+        # every process must create every group, in the same order
+        self.row_group = self.col_group = None
+        for c in range(P_c):
+            g = dist.new_group([c * P_r + r for r in range(P_r)])
+            if c == self.c:
+                self.row_group = g
+        for r in range(P_r):
+            g = dist.new_group([c * P_r + r for c in range(P_c)])
+            if r == self.r:
+                self.col_group = g
+        self.words: Dict[str, float] = {"allgather_y": 0.0, "allreduce_dx": 0.0, "allreduce_dw": 0.0}
+
+    def all_gather_cols(self, block, out, kind="allgather_y"):
+        """out[:, r' * n : (r' + 1) * n] = block of process r' of the P_r group, for every r'."""
+        import torch
+        p, n = self.P_r, block.shape[1]
+        assert out.shape[1] == p * n and out.shape[0] == block.shape[0]
+        if p == 1:
+            out.copy_(block)
+            return out
+        src = block.contiguous()
+        if self.via_host:
+            src = src.cpu()
+        parts = [torch.empty_like(src) for _ in range(p)]
+        self.dist.all_gather(parts, src, group=self.row_group)
+        for j in range(p):
+            out[:, j * n:(j + 1) * n].copy_(parts[j])
+        self.words[kind] += (p - 1) * block.numel()
+        return out
+
+    def all_reduce_(self, t, over: str, kind: str):
+        """In-place sum of a contiguous float tensor over the P_r ("rows") or the P_c ("cols") group."""
+        p, g = (self.P_r, self.row_group) if over == "rows" else (self.P_c, self.col_group)
+        if p == 1:
+            return t
+        assert t.is_contiguous()
+        if self.via_host:
+            h = t.cpu()
+            self.dist.all_reduce(h, group=g)
+            t.copy_(h)
+        else:
+            self.dist.all_reduce(t, group=g)
+        self.words[kind] += 2.0 * (p - 1) / p * t.numel()
+        return t
+
+
+class GridFC:
+    """One process's share of a fully connected stack d_0 -> ... -> d_L (ReLU between layers, softmax
+    cross-entropy on top, no bias): W_i(r, :) in bf16, and the step over its batch block."""
+
+    def __init__(self, dims: Sequence[int], B: int, comm: GridComm, device="cuda"):
+        import torch
+        self.t = torch
+        self.dims = [int(d) for d in dims]
+        self.L = len(self.dims) - 1
+        self.B = int(B)
+        self.comm = comm
+        P_r, P_c = comm.P_r, comm.P_c
+        if self.B % P_c:
+            raise ValueError("the batch must divide into P_c equal blocks")
+        for d in self.dims[1:]:
+            if d % P_r or (d // P_r) % 8:
+                raise ValueError("every d_i must divide into P_r row blocks whose height is a multiple of 8")
+        if self.dims[0] % 8:
+            raise ValueError("d_0 must be a multiple of 8")
+        self.m = self.B // P_c
+        self.device = device
+        self.W: List = [torch.zeros((self.dims[i + 1] // P_r, self.dims[i]), dtype=torch.bfloat16, device=device)
+                        for i in range(self.L)]
+        self.dW: List = [None] * self.L            # summed fp32 gradients of the last step (kept for inspection)
+
+    def rows(self, i: int):
+        """Row range of W_i (0-based layer i) this process owns."""
+        h = self.dims[i + 1] // self.comm.P_r
+        return self.comm.r * h, (self.comm.r + 1) * h
+
+    def set_weights(self, i: int, W_full):
+        """Takes this process's row block out of the full matrix [d_{i+1}, d_i] (bf16, any device)."""
+        a, b = self.rows(i)
+        self.W[i].copy_(W_full[a:b])
+
+    def step(self, X_c, labels_c, eta: float):
+        """One step on the batch block X_c [B / P_c, d_0] (bf16), labels_c int32.  Returns the sum of the
+        losses of this block; the logits are kept in self.logits."""
+        t, comm = self.t, self.comm
+        m, L = self.m, self.L
+        assert tuple(X_c.shape) == (m, self.dims[0]) and X_c.dtype == t.bfloat16
+        acts = [X_c.contiguous()]
+        # ---- forward: block product, then the all-gather over the P_r group (Appendix A.1)
+        for i in range(L):
+            last = i == L - 1
+            h = self.dims[i + 1] // comm.P_r
+            blk = t.empty((m, h), dtype=t.float32 if last else t.bfloat16, device=self.device)
+            mbd.block_gemm(0, acts[i], self.W[i], blk, mbd.TAIL_STORE, relu=not last)
+            full = t.empty((m, self.dims[i + 1]), dtype=blk.dtype, device=self.device)
+            comm.all_gather_cols(blk, full)
+            acts.append(full)
+        self.logits = acts[L]
+        # ---- loss and top gradient (every process of a P_r group holds the full logits of its samples)
+        dY = t.empty((m, self.dims[L]), dtype=t.bfloat16, device=self.device)
+        per = t.empty((m,), dtype=t.float32, device=self.device)
+        mbd.softmax_xent(self.logits, labels_c, dY, per)
+        loss = float(per.double().sum().item())
+        # ---- backward (Appendix A.2)
+        scale = -float(eta) / self.B
+        for i in range(L - 1, -1, -1):
+            a, b = self.rows(i)
+            dY_r = dY[:, a:b]                                           # dY_i(r, c): this process's rows of layer i's output
+            dY_prev = None
+            if i > 0:
+                part = t.empty((m, self.dims[i]), dtype=t.float32, device=self.device)
+                mbd.block_gemm(1, dY_r, self.W[i], part, mbd.TAIL_STORE)       # W_i(r, :)^T dY_i(r, c), one summand
+                comm.all_reduce_(part, "rows", "allreduce_dx")
+                dY_prev = t.empty((m, self.dims[i]), dtype=t.bfloat16, device=self.device)
+                mbd.block_reduce(part, dY_prev, mbd.TAIL_MASK, mask=acts[i])   # ReLU derivative from the stored X_i
+            g = t.empty((b - a, self.dims[i]), dtype=t.float32, device=self.device)
+            mbd.block_gemm(2, dY_r, acts[i], g, mbd.TAIL_STORE)                # dY_i(r, c) X_i(:, c)^T, one summand
+            comm.all_reduce_(g, "cols", "allreduce_dw")
+            self.dW[i] = g
+            mbd.block_reduce(g, self.W[i], mbd.TAIL_SGD, scale=scale)          # Eq. 1 on the owned rows
+            dY = dY_prev
+        return loss
+
+
+def expected_words(dims: Sequence[int], B: int, P_r: int, P_c: int) -> Dict[str, int]:
+    """Per-process totals of mbd_comm_words for the stack (Eq. 8)."""
+    rows = mbd.comm_words(mbd.fc_layers(dims, bias=False), B, P_r, P_c)
+    return {k: sum(r[k] for r in rows) for k in ("allgather_y", "allreduce_dx", "allreduce_dw")}

@@ -28,7 +28,7 @@ EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weig
            "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_gemm_bf16_noalloc", "mbd_selftest_timeout", "mbd_strerror",
            "mbd_train_step_host_begin", "mbd_train_step_host_end",
            "mbd_comm_time", "mbd_redistribute_time", "mbd_total_time", "mbd_grid_table", "mbd_choose_grid",
-           "mbd_enable_master_weights"]
+           "mbd_enable_master_weights", "mbd_block_gemm_bf16", "mbd_block_reduce", "mbd_softmax_xent"]
 
 
 class MbdError(RuntimeError):
@@ -42,6 +42,16 @@ class Layer(C.Structure):
                 ("d_in", C.c_int64), ("d_out", C.c_int64),
                 ("C_in", C.c_int32), ("C_out", C.c_int32), ("H", C.c_int32), ("W", C.c_int32),
                 ("kh", C.c_int32), ("kw", C.c_int32)]
+
+
+TAIL_STORE, TAIL_MASK, TAIL_SGD = range(3)
+
+
+class Tail(C.Structure):
+    """mbd_tail: the operation applied to a finished fp32 block (see include/mbd.h)."""
+    _fields_ = [("op", C.c_int32), ("out_bf16", C.c_int32), ("relu", C.c_int32), ("reserved", C.c_int32),
+                ("out_dev", C.c_void_p), ("ldo", C.c_int64), ("bias_dev", C.c_void_p), ("mask_dev", C.c_void_p),
+                ("ldmask", C.c_int64), ("scale", C.c_float)]
 
 
 class Words(C.Structure):
@@ -107,6 +117,9 @@ def lib():
         L.mbd_set_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
         L.mbd_poll_status.argtypes = [vp]
         L.mbd_enable_master_weights.argtypes = [vp]
+        L.mbd_block_gemm_bf16.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, C.POINTER(Tail), vp]
+        L.mbd_block_reduce.argtypes = [vp, i32, i64, i64, C.POINTER(Tail), vp]
+        L.mbd_softmax_xent.argtypes = [vp, i64, i64, vp, vp, i32, vp, vp]
         L.mbd_profile_enable.argtypes = [vp, i32]
         L.mbd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double)]
         L.mbd_launch_count.argtypes = [vp]
@@ -374,6 +387,64 @@ def gemm_bf16(variant: int, A, B, k_splits: int = 1, return_partials: bool = Fal
                              k_splits, _ptr(parts), C.c_void_p(torch.cuda.current_stream().cuda_stream))
     _check(st, "mbd_gemm_bf16")
     return (D, parts) if return_partials else D
+
+
+def _tail(op: int, out, relu: bool = False, bias=None, mask=None, scale: float = 0.0) -> Tail:
+    import torch
+    assert out.is_cuda and out.stride(-1) == 1 and out.dtype in (torch.bfloat16, torch.float32)
+    if mask is not None:
+        assert mask.dtype == out.dtype and mask.stride(-1) == 1
+    return Tail(op, int(out.dtype == torch.bfloat16), int(relu), 0, out.data_ptr(), out.stride(0),
+                None if bias is None else bias.data_ptr(), None if mask is None else mask.data_ptr(),
+                0 if mask is None else mask.stride(0), float(scale))
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def block_gemm(variant: int, A, B, out, op: int = TAIL_STORE, relu: bool = False, bias=None, mask=None, scale: float = 0.0):
+    """mbd_block_gemm_bf16: one block product into `out` ([M, N] view, bf16 or float, row stride free) with the
+    tail operation fused.  variant 0: A[M,K], B[N,K];  1: A[M,K], B[K,N];  2: A[K,M], B[K,N] (row strides free)."""
+    import torch
+    assert A.is_cuda and B.is_cuda and A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16
+    assert A.stride(1) == 1 and B.stride(1) == 1
+    if variant == 0:
+        M, K = A.shape; N = B.shape[0]; assert B.shape[1] == K
+    elif variant == 1:
+        M, K = A.shape; N = B.shape[1]; assert B.shape[0] == K
+    else:
+        K, M = A.shape; N = B.shape[1]; assert B.shape[0] == K
+    assert tuple(out.shape) == (M, N)
+    t = _tail(op, out, relu, bias, mask, scale)
+    _check(lib().mbd_block_gemm_bf16(variant, M, N, K, _ptr(A), A.stride(0), _ptr(B), B.stride(0), C.byref(t), _stream()),
+           "mbd_block_gemm_bf16")
+    return out
+
+
+def block_reduce(parts, out, op: int = TAIL_STORE, relu: bool = False, bias=None, mask=None, scale: float = 0.0):
+    """mbd_block_reduce: sum of the S dense float planes parts[S, M, N] (or one plane [M, N]) in ascending
+    order, then the tail operation into `out`."""
+    import torch
+    assert parts.is_cuda and parts.dtype == torch.float32 and parts.is_contiguous()
+    if parts.dim() == 2:
+        parts = parts.unsqueeze(0)
+    S, M, N = parts.shape
+    assert tuple(out.shape) == (M, N)
+    t = _tail(op, out, relu, bias, mask, scale)
+    _check(lib().mbd_block_reduce(_ptr(parts), S, M, N, C.byref(t), _stream()), "mbd_block_reduce")
+    return out
+
+
+def softmax_xent(logits, labels, dY, per_sample):
+    """mbd_softmax_xent: per-sample loss and dY = softmax - onehot of float logits [B, d]."""
+    import torch
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
+    assert labels.dtype == torch.int32 and labels.is_cuda and dY.is_contiguous() and per_sample.dtype == torch.float32
+    Bn, d = logits.shape
+    _check(lib().mbd_softmax_xent(_ptr(logits), Bn, d, _ptr(labels), _ptr(dY), int(dY.dtype == torch.bfloat16),
+                                  _ptr(per_sample), _stream()), "mbd_softmax_xent")
 
 
 def selftest_timeout(limit_ms: int = 50) -> int:
