@@ -288,8 +288,11 @@ MBD_API mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, c
 /* ---- Block operations for a multi-process driver of the grid (Section 2.3; Appendix A.1 / A.2) ----
  * What one process (r, c) does between two collectives, on caller-owned device buffers: a block product
  * with its tail operation fused, the tail operation applied to a sum that a collective delivered, and
- * the loss.  Every call enqueues on cuda_stream and returns after the stream has drained (MBD_E_TIMEOUT
- * if a bounded wait inside a kernel gave up).
+ * the loss.  All of them enqueue on cuda_stream.  mbd_block_gemm_bf16 with status_dev == NULL, and the
+ * other two with sync != 0, return after the stream has drained (MBD_E_TIMEOUT if a bounded wait inside a
+ * kernel gave up); with a caller-owned, zero-initialised device word status_dev (resp. sync == 0) they only
+ * enqueue, so that a driver can overlap them with its collectives on other streams -- the caller then reads
+ * the word when it likes: non-zero means a bounded wait gave up and the results are not valid.
  *
  * mbd_tail: what happens to a finished fp32 element acc at (m, n):
  *   MBD_TAIL_STORE  out = acc (+ bias_dev[n]); relu != 0: max(., 0)
@@ -311,15 +314,15 @@ typedef struct {
 /* One block product (variants and operand layouts of mbd_gemm_bf16, K not split) with `tail` fused. */
 MBD_API mbd_status mbd_block_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, const void* A_dev,
                                int64_t lda, const void* B_dev, int64_t ldb, const mbd_tail* tail,
-                               void* cuda_stream);
+                               int32_t* status_dev, void* cuda_stream);
 /* sum_{s < S} parts_dev[s] (planes of M x N floats, ascending s), then `tail`.  S = 1 applies the tail
  * operation to a sum that is already complete (e.g. after an all-reduce). */
 MBD_API mbd_status mbd_block_reduce(const float* parts_dev, int S, int64_t M, int64_t N, const mbd_tail* tail,
-                            void* cuda_stream);
+                            int sync, void* cuda_stream);
 /* Softmax cross-entropy of float logits [B, d]: per_sample_dev[b] = loss of sample b (natural log),
  * dY_dev [B, d] = softmax - onehot (bf16 if dY_bf16 != 0, else float).  labels_dev: int32 in [0, d). */
 MBD_API mbd_status mbd_softmax_xent(const float* logits_dev, int64_t B, int64_t d, const int32_t* labels_dev,
-                            void* dY_dev, int dY_bf16, float* per_sample_dev, void* cuda_stream);
+                            void* dY_dev, int dY_bf16, float* per_sample_dev, int sync, void* cuda_stream);
 
 /* Failure-detection self test: launches one small kernel whose only job is to wait, with a
  * limit of `limit_ms` milliseconds, on a barrier that nothing will ever signal.  The kernel

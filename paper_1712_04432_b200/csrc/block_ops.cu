@@ -2,8 +2,9 @@
 // between two collectives (Section 2.3; Appendix A.1 / A.2) -- a block product with its tail operation
 // fused, the tail operation applied to a sum that arrived from a collective, and the loss.  They let a
 // multi-process driver run the grid for real, every arithmetic step in these kernels and only the
-// exchange outside.  Each call enqueues on the given stream and waits for it (the status word of the
-// bounded waits is read back), so it is a building block, not the fast path of a single GPU.
+// exchange outside.  With a caller-owned status word a call only enqueues (the caller reads the word when it
+// likes: non-zero = a bounded wait gave up); without one the call allocates a word, waits for the stream and
+// reports what it found.
 #include "../../include/mbd.h"
 #include "kernels.h"
 
@@ -48,7 +49,8 @@ struct StatusWord {
 }  // namespace
 
 extern "C" mbd_status mbd_block_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
-                                          const void* Bm, int64_t ldb, const mbd_tail* tail, void* cuda_stream) {
+                                          const void* Bm, int64_t ldb, const mbd_tail* tail, int32_t* status_dev,
+                                          void* cuda_stream) {
   Epi epi;
   if (!A || !Bm || variant < 0 || variant > 2 || M < 1 || N < 1 || K < 1 || !to_epi(tail, &epi)) return MBD_E_INVALID;
   if (lda % 8 || ldb % 8 || epi.ldo % 8 || N % 8 || (epi.mask && epi.ldmask % 8)) return MBD_E_UNSUPPORTED;
@@ -60,7 +62,8 @@ extern "C" mbd_status mbd_block_gemm_bf16(int variant, int64_t M, int64_t N, int
     return MBD_E_CUDA;
   }
   StatusWord st;
-  if (!st.alloc(stream)) return MBD_E_ALLOC;
+  if (status_dev) st.dev = status_dev;
+  else if (!st.alloc(stream)) return MBD_E_ALLOC;
   TcGemm g{};
   g.variant = variant;
   g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
@@ -73,17 +76,22 @@ extern "C" mbd_status mbd_block_gemm_bf16(int variant, int64_t M, int64_t N, int
     g.partials = nullptr;
     if (tc_gemm_launch(g, stream) != cudaSuccess) ret = MBD_E_CUDA;
   }
+  if (status_dev) {                      // enqueue-only: the caller owns and reads the status word
+    if (ret != MBD_OK) (void)cudaGetLastError();
+    return ret;
+  }
   return st.finish(stream, ret);
 }
 
 extern "C" mbd_status mbd_block_reduce(const float* parts, int S, int64_t M, int64_t N, const mbd_tail* tail,
-                                       void* cuda_stream) {
+                                       int sync, void* cuda_stream) {
   Epi epi;
   if (!parts || S < 1 || M < 1 || N < 1 || !to_epi(tail, &epi)) return MBD_E_INVALID;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-      reduce_partials_launch(parts, S, M, N, epi, sms, stream) != cudaSuccess || cudaStreamSynchronize(stream) != cudaSuccess) {
+      reduce_partials_launch(parts, S, M, N, epi, sms, stream) != cudaSuccess ||
+      (sync && cudaStreamSynchronize(stream) != cudaSuccess)) {
     (void)cudaGetLastError();
     return MBD_E_CUDA;
   }
@@ -91,11 +99,11 @@ extern "C" mbd_status mbd_block_reduce(const float* parts, int S, int64_t M, int
 }
 
 extern "C" mbd_status mbd_softmax_xent(const float* logits, int64_t B, int64_t d, const int32_t* labels, void* dY,
-                                       int dY_bf16, float* per_sample, void* cuda_stream) {
+                                       int dY_bf16, float* per_sample, int sync, void* cuda_stream) {
   if (!logits || !labels || !dY || !per_sample || B < 1 || d < 1) return MBD_E_INVALID;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   if (softmax_xent_launch(logits, B, d, labels, dY, dY_bf16 != 0, per_sample, stream) != cudaSuccess ||
-      cudaStreamSynchronize(stream) != cudaSuccess) {
+      (sync && cudaStreamSynchronize(stream) != cudaSuccess)) {
     (void)cudaGetLastError();
     return MBD_E_CUDA;
   }

@@ -10,7 +10,8 @@ matrix and the batch block c of the samples.
                all-reduce over the P_c group, Eq. 1              -> W_i(r, :) updated          Eq. 8, term 3
 
 Every arithmetic step runs in the library's kernels (mbd_block_gemm_bf16, mbd_block_reduce,
-mbd_softmax_xent); torch.distributed only moves the blocks.  With the "nccl" backend the collectives run
+mbd_softmax_xent, all enqueue-only here: one status word is read at the end of the step);
+torch.distributed only moves the blocks.  With the "nccl" backend the collectives run
 on the device buffers; with "gloo" (tests: several processes sharing one GPU) they go through host copies.
 The words every collective moves per process are counted from the buffers actually exchanged, so that
 they can be compared with mbd_comm_words.
@@ -113,6 +114,7 @@ class GridFC:
         self.W: List = [torch.zeros((self.dims[i + 1] // P_r, self.dims[i]), dtype=torch.bfloat16, device=device)
                         for i in range(self.L)]
         self.dW: List = [None] * self.L            # summed fp32 gradients of the last step (kept for inspection)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)   # bounded-wait status word of the block products
 
     def rows(self, i: int):
         """Row range of W_i (0-based layer i) this process owns."""
@@ -136,7 +138,7 @@ class GridFC:
             last = i == L - 1
             h = self.dims[i + 1] // comm.P_r
             blk = t.empty((m, h), dtype=t.float32 if last else t.bfloat16, device=self.device)
-            mbd.block_gemm(0, acts[i], self.W[i], blk, mbd.TAIL_STORE, relu=not last)
+            mbd.block_gemm(0, acts[i], self.W[i], blk, mbd.TAIL_STORE, relu=not last, status=self.status)
             full = t.empty((m, self.dims[i + 1]), dtype=blk.dtype, device=self.device)
             comm.all_gather_cols(blk, full)
             acts.append(full)
@@ -144,7 +146,7 @@ class GridFC:
         # ---- loss and top gradient (every process of a P_r group holds the full logits of its samples)
         dY = t.empty((m, self.dims[L]), dtype=t.bfloat16, device=self.device)
         per = t.empty((m,), dtype=t.float32, device=self.device)
-        mbd.softmax_xent(self.logits, labels_c, dY, per)
+        mbd.softmax_xent(self.logits, labels_c, dY, per, sync=False)
         loss = float(per.double().sum().item())
         # ---- backward (Appendix A.2)
         scale = -float(eta) / self.B
@@ -154,16 +156,19 @@ class GridFC:
             dY_prev = None
             if i > 0:
                 part = t.empty((m, self.dims[i]), dtype=t.float32, device=self.device)
-                mbd.block_gemm(1, dY_r, self.W[i], part, mbd.TAIL_STORE)       # W_i(r, :)^T dY_i(r, c), one summand
+                mbd.block_gemm(1, dY_r, self.W[i], part, mbd.TAIL_STORE, status=self.status)       # W_i(r, :)^T dY_i(r, c), one summand
                 comm.all_reduce_(part, "rows", "allreduce_dx")
                 dY_prev = t.empty((m, self.dims[i]), dtype=t.bfloat16, device=self.device)
-                mbd.block_reduce(part, dY_prev, mbd.TAIL_MASK, mask=acts[i])   # ReLU derivative from the stored X_i
+                mbd.block_reduce(part, dY_prev, mbd.TAIL_MASK, mask=acts[i], sync=False)   # ReLU derivative from the stored X_i
             g = t.empty((b - a, self.dims[i]), dtype=t.float32, device=self.device)
-            mbd.block_gemm(2, dY_r, acts[i], g, mbd.TAIL_STORE)                # dY_i(r, c) X_i(:, c)^T, one summand
+            mbd.block_gemm(2, dY_r, acts[i], g, mbd.TAIL_STORE, status=self.status)                # dY_i(r, c) X_i(:, c)^T, one summand
             comm.all_reduce_(g, "cols", "allreduce_dw")
             self.dW[i] = g
-            mbd.block_reduce(g, self.W[i], mbd.TAIL_SGD, scale=scale)          # Eq. 1 on the owned rows
+            mbd.block_reduce(g, self.W[i], mbd.TAIL_SGD, scale=scale, sync=False)          # Eq. 1 on the owned rows
             dY = dY_prev
+        if int(self.status.item()) != 0:             # (synchronises) a bounded wait inside a product gave up
+            self.status.zero_()
+            raise mbd.MbdError(mbd.E_TIMEOUT, "grid step")
         return loss
 
 

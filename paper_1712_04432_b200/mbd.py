@@ -117,9 +117,9 @@ def lib():
         L.mbd_set_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
         L.mbd_poll_status.argtypes = [vp]
         L.mbd_enable_master_weights.argtypes = [vp]
-        L.mbd_block_gemm_bf16.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, C.POINTER(Tail), vp]
-        L.mbd_block_reduce.argtypes = [vp, i32, i64, i64, C.POINTER(Tail), vp]
-        L.mbd_softmax_xent.argtypes = [vp, i64, i64, vp, vp, i32, vp, vp]
+        L.mbd_block_gemm_bf16.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, C.POINTER(Tail), vp, vp]
+        L.mbd_block_reduce.argtypes = [vp, i32, i64, i64, C.POINTER(Tail), i32, vp]
+        L.mbd_softmax_xent.argtypes = [vp, i64, i64, vp, vp, i32, vp, i32, vp]
         L.mbd_profile_enable.argtypes = [vp, i32]
         L.mbd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double)]
         L.mbd_launch_count.argtypes = [vp]
@@ -404,9 +404,11 @@ def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def block_gemm(variant: int, A, B, out, op: int = TAIL_STORE, relu: bool = False, bias=None, mask=None, scale: float = 0.0):
+def block_gemm(variant: int, A, B, out, op: int = TAIL_STORE, relu: bool = False, bias=None, mask=None, scale: float = 0.0,
+               status=None):
     """mbd_block_gemm_bf16: one block product into `out` ([M, N] view, bf16 or float, row stride free) with the
-    tail operation fused.  variant 0: A[M,K], B[N,K];  1: A[M,K], B[K,N];  2: A[K,M], B[K,N] (row strides free)."""
+    tail operation fused.  variant 0: A[M,K], B[N,K];  1: A[M,K], B[K,N];  2: A[K,M], B[K,N] (row strides free).
+    `status` (int32 CUDA tensor of one zero): enqueue only; otherwise the call waits for the stream."""
     import torch
     assert A.is_cuda and B.is_cuda and A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16
     assert A.stride(1) == 1 and B.stride(1) == 1
@@ -418,12 +420,13 @@ def block_gemm(variant: int, A, B, out, op: int = TAIL_STORE, relu: bool = False
         K, M = A.shape; N = B.shape[1]; assert B.shape[0] == K
     assert tuple(out.shape) == (M, N)
     t = _tail(op, out, relu, bias, mask, scale)
-    _check(lib().mbd_block_gemm_bf16(variant, M, N, K, _ptr(A), A.stride(0), _ptr(B), B.stride(0), C.byref(t), _stream()),
-           "mbd_block_gemm_bf16")
+    _check(lib().mbd_block_gemm_bf16(variant, M, N, K, _ptr(A), A.stride(0), _ptr(B), B.stride(0), C.byref(t),
+                                     _ptr(status), _stream()), "mbd_block_gemm_bf16")
     return out
 
 
-def block_reduce(parts, out, op: int = TAIL_STORE, relu: bool = False, bias=None, mask=None, scale: float = 0.0):
+def block_reduce(parts, out, op: int = TAIL_STORE, relu: bool = False, bias=None, mask=None, scale: float = 0.0,
+                 sync: bool = True):
     """mbd_block_reduce: sum of the S dense float planes parts[S, M, N] (or one plane [M, N]) in ascending
     order, then the tail operation into `out`."""
     import torch
@@ -433,18 +436,18 @@ def block_reduce(parts, out, op: int = TAIL_STORE, relu: bool = False, bias=None
     S, M, N = parts.shape
     assert tuple(out.shape) == (M, N)
     t = _tail(op, out, relu, bias, mask, scale)
-    _check(lib().mbd_block_reduce(_ptr(parts), S, M, N, C.byref(t), _stream()), "mbd_block_reduce")
+    _check(lib().mbd_block_reduce(_ptr(parts), S, M, N, C.byref(t), int(sync), _stream()), "mbd_block_reduce")
     return out
 
 
-def softmax_xent(logits, labels, dY, per_sample):
+def softmax_xent(logits, labels, dY, per_sample, sync: bool = True):
     """mbd_softmax_xent: per-sample loss and dY = softmax - onehot of float logits [B, d]."""
     import torch
     assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
     assert labels.dtype == torch.int32 and labels.is_cuda and dY.is_contiguous() and per_sample.dtype == torch.float32
     Bn, d = logits.shape
     _check(lib().mbd_softmax_xent(_ptr(logits), Bn, d, _ptr(labels), _ptr(dY), int(dY.dtype == torch.bfloat16),
-                                  _ptr(per_sample), _stream()), "mbd_softmax_xent")
+                                  _ptr(per_sample), int(sync), _stream()), "mbd_softmax_xent")
 
 
 def selftest_timeout(limit_ms: int = 50) -> int:

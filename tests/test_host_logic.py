@@ -69,3 +69,13 @@ def test_no_silent_fallback_without_a_gpu():
     # valid arguments, but no device: the library reports a CUDA error instead of computing elsewhere
     assert create(mbd.fc_layers((64, 32, 16)), 8) == mbd.E_CUDA
     assert create(mbd.fc_layers((64, 32, 16)), 8, dtype=mbd.F32) == mbd.E_CUDA
+
+
+def test_block_calls_reject_bad_arguments():
+    import ctypes as C
+    from paper_1712_04432_b200 import mbd
+    L = mbd.lib()
+    t = mbd.Tail(mbd.TAIL_STORE, 0, 0, 0, None, 8, None, None, 0, 0.0)          # no output buffer
+    assert L.mbd_block_gemm_bf16(0, 8, 8, 8, None, 8, None, 8, C.byref(t), None, None) == mbd.E_INVALID
+    assert L.mbd_block_reduce(None, 1, 8, 8, C.byref(t), 1, None) == mbd.E_INVALID
+    assert L.mbd_softmax_xent(None, 1, 8, None, None, 0, None, 1, None) == mbd.E_INVALID
