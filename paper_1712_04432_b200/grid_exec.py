@@ -89,6 +89,28 @@ class GridComm:
         self.words[kind] += 2.0 * (p - 1) / p * t.numel()
         return t
 
+    def all_reduce_start(self, t, over: str, kind: str):
+        """Starts the in-place sum of `t` and returns a handle for all_reduce_finish; what is enqueued or
+        computed in between runs beside the exchange (Section 3: the all-reduce of dW_i can hide behind the
+        products of the layers below)."""
+        p, g = (self.P_r, self.row_group) if over == "rows" else (self.P_c, self.col_group)
+        if p == 1:
+            return (t, None, None)
+        assert t.is_contiguous()
+        self.words[kind] += 2.0 * (p - 1) / p * t.numel()
+        if self.via_host:
+            h = t.cpu()
+            return (t, h, self.dist.all_reduce(h, group=g, async_op=True))
+        return (t, None, self.dist.all_reduce(t, group=g, async_op=True))
+
+    def all_reduce_finish(self, handle):
+        t, h, work = handle
+        if work is not None:
+            work.wait()                  # nccl: the current stream waits; gloo: the host waits
+            if h is not None:
+                t.copy_(h)
+        return t
+
 
 class GridFC:
     """One process's share of a fully connected stack d_0 -> ... -> d_L (ReLU between layers, softmax
@@ -115,6 +137,13 @@ class GridFC:
                         for i in range(self.L)]
         self.dW: List = [None] * self.L            # summed fp32 gradients of the last step (kept for inspection)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)   # bounded-wait status word of the block products
+
+    def _update(self, pending, scale: float):
+        """Waits for the all-reduce of dW_i started earlier and applies Eq. 1 to the owned rows."""
+        i, handle = pending
+        g = self.comm.all_reduce_finish(handle)
+        self.dW[i] = g
+        mbd.block_reduce(g, self.W[i], mbd.TAIL_SGD, scale=scale, sync=False)
 
     def rows(self, i: int):
         """Row range of W_i (0-based layer i) this process owns."""
@@ -150,6 +179,7 @@ class GridFC:
         loss = float(per.double().sum().item())
         # ---- backward (Appendix A.2)
         scale = -float(eta) / self.B
+        pending = None                                                  # the all-reduce of the layer above, in flight
         for i in range(L - 1, -1, -1):
             a, b = self.rows(i)
             dY_r = dY[:, a:b]                                           # dY_i(r, c): this process's rows of layer i's output
@@ -162,10 +192,12 @@ class GridFC:
                 mbd.block_reduce(part, dY_prev, mbd.TAIL_MASK, mask=acts[i], sync=False)   # ReLU derivative from the stored X_i
             g = t.empty((b - a, self.dims[i]), dtype=t.float32, device=self.device)
             mbd.block_gemm(2, dY_r, acts[i], g, mbd.TAIL_STORE, status=self.status)                # dY_i(r, c) X_i(:, c)^T, one summand
-            comm.all_reduce_(g, "cols", "allreduce_dw")
-            self.dW[i] = g
-            mbd.block_reduce(g, self.W[i], mbd.TAIL_SGD, scale=scale, sync=False)          # Eq. 1 on the owned rows
+            handle = comm.all_reduce_start(g, "cols", "allreduce_dw")          # runs beside the products of layer i - 1
+            if pending is not None:
+                self._update(pending, scale)
+            pending = (i, handle)
             dY = dY_prev
+        self._update(pending, scale)
         if int(self.status.item()) != 0:             # (synchronises) a bounded wait inside a product gave up
             self.status.zero_()
             raise mbd.MbdError(mbd.E_TIMEOUT, "grid step")
