@@ -29,7 +29,12 @@ __device__ __forceinline__ void epi_apply1(const Epi& e, int64_t m, int64_t n, f
     if (e.out_bf16) reinterpret_cast<__nv_bfloat16*>(e.out)[m * e.ldo + n] = __float2bfloat16_rn(v);
     else reinterpret_cast<float*>(e.out)[m * e.ldo + n] = v;
   } else {  // EPI_SGD
-    if (e.out_bf16) {
+    if (e.out_bf16 && e.master) {
+      float* w32 = e.master + m * e.ldo + n;
+      const float v = fmaf(e.scale, acc, *w32);
+      *w32 = v;
+      reinterpret_cast<__nv_bfloat16*>(e.out)[m * e.ldo + n] = __float2bfloat16_rn(v);
+    } else if (e.out_bf16) {
       __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(e.out) + m * e.ldo + n;
       *w = __float2bfloat16_rn(fmaf(e.scale, acc, __bfloat162float(*w)));
     } else {
@@ -72,7 +77,15 @@ __device__ __forceinline__ void epi_apply8(const Epi& e, int64_t m, int64_t n0, 
       }
     }
   } else {  // EPI_SGD: read-modify-write of the weights
-    if (e.out_bf16) {
+    if (e.out_bf16 && e.master) {   // fp32 master weights: update the master, the bf16 copy is its rounding
+      float* x = e.master + m * e.ldo + n0;
+      const float4 a = *reinterpret_cast<const float4*>(x), b = *reinterpret_cast<const float4*>(x + 4);
+      const float xs[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = fmaf(e.scale, v[i], xs[i]);
+      *reinterpret_cast<float4*>(x) = make_float4(v[0], v[1], v[2], v[3]);
+      *reinterpret_cast<float4*>(x + 4) = make_float4(v[4], v[5], v[6], v[7]);
+    } else if (e.out_bf16) {
       uint4* p = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(e.out) + m * e.ldo + n0);
       const uint4 q = *p;
       const uint32_t w[4] = {q.x, q.y, q.z, q.w};

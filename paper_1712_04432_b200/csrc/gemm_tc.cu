@@ -413,7 +413,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       __syncwarp();
     } else {
     const bool prefetch = p.S == 1 && p.epi.out_bf16 &&
-                          (p.epi.op == EPI_SGD || (p.epi.op == EPI_MASK && p.epi.mask != nullptr));
+                          ((p.epi.op == EPI_SGD && p.epi.master == nullptr) ||      // master weights: shared tail, no prefetch
+                           (p.epi.op == EPI_MASK && p.epi.mask != nullptr));
     const __nv_bfloat16* pre_src = p.epi.op == EPI_SGD ? reinterpret_cast<const __nv_bfloat16*>(p.epi.out)
                                                        : reinterpret_cast<const __nv_bfloat16*>(p.epi.mask);
     const int64_t pre_ld = p.epi.op == EPI_SGD ? p.epi.ldo : p.epi.ldmask;
@@ -704,7 +705,7 @@ cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
   p.epi = g.epi;
   p.status = g.status;
   p.te = g.te && g.epi.op == g.te_epi.op && g.epi.out == g.te_epi.out && g.epi.out_bf16 && g.epi.mask == g.te_epi.mask &&
-         g.epi.ldo == g.te_epi.ldo && g.k_splits == 1;
+         g.epi.ldo == g.te_epi.ldo && g.k_splits == 1 && !g.epi.master;   // the TMA epilogue has no master path
   if (g.variant == 0) return launch_t<0, 0>(g, p, stream);
   if (g.variant == 1) return launch_t<0, 1>(g, p, stream);
   return launch_t<1, 1>(g, p, stream);

@@ -66,7 +66,7 @@ enum : int {
 enum EpiOp : int {
   EPI_ACT = 0,    // v = acc (+ bias[n]); relu ? max(v,0) : v; store (bf16 or f32)
   EPI_MASK = 1,   // v = (mask == null || mask[m,n] > 0) ? acc : 0; store (bf16 or f32)
-  EPI_SGD = 2     // out[m,n] = out[m,n] + scale * acc   (Eq. 1 with scale = -eta/B)
+  EPI_SGD = 2     // out[m,n] = out[m,n] + scale * acc   (Eq. 1 with scale = -eta/B); see Epi::master
 };
 
 struct Epi {
@@ -79,6 +79,8 @@ struct Epi {
   const void* mask;    // [M, ldmask] in out's dtype, or null
   int64_t ldmask;
   float scale;
+  float* master;       // EPI_SGD on bf16 weights: fp32 master copy [M, ldo] (null: none).  The update is applied
+                       // to the master and `out` receives the rounded master.
 };
 
 // ---- tcgen05 GEMM -----------------------------------------------------------

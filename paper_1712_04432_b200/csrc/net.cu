@@ -141,9 +141,9 @@ Epi epi_mask(void* out, int64_t ldo, int out_bf16, const void* mask, int64_t ldm
   e.op = EPI_MASK; e.out_bf16 = out_bf16; e.out = out; e.ldo = ldo; e.mask = mask; e.ldmask = ldmask;
   return e;
 }
-Epi epi_sgd(void* w, int64_t ldo, int out_bf16, float scale) {
+Epi epi_sgd(void* w, int64_t ldo, int out_bf16, float scale, float* master = nullptr) {
   Epi e{};
-  e.op = EPI_SGD; e.out_bf16 = out_bf16; e.out = w; e.ldo = ldo; e.scale = scale;
+  e.op = EPI_SGD; e.out_bf16 = out_bf16; e.out = w; e.ldo = ldo; e.scale = scale; e.master = master;
   return e;
 }
 
@@ -569,9 +569,13 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
       mbd_status s = run_gemm(n, l.bwd_data, 1, n->B, l.d_in, l.d_out, l.dY, l.d_out, l.W, l.d_in, S_r, e);
       if (s != MBD_OK) return s;
     }
-    // with master weights the gradient is materialised and Eq. 1 is applied to the master by its own kernel
-    const bool in_epilogue = fused && !n->master;
-    const Epi e = in_epilogue ? epi_sgd(l.W, l.d_in, bf, scale) : epi_act(l.dW, l.d_in, 0, nullptr, 0);
+    // With master weights: a split product updates the fp32 master in the tail of its reduction (which streams
+    // the sum through registers anyway); an unsplit one materialises the gradient and a streaming kernel applies
+    // Eq. 1 to the master (measured equal to doing it in the product's epilogue, whose loads would be exposed).
+    const bool master_tail = fused && n->master && bf && l.bwd_weight.k_splits > 1;
+    const bool master_kernel = fused && n->master && !master_tail;
+    const Epi e = (fused && !master_kernel) ? epi_sgd(l.W, l.d_in, bf, scale, master_tail ? l.W32 : nullptr)
+                                            : epi_act(l.dW, l.d_in, 0, nullptr, 0);
     cudaStream_t ws = nullptr;
     if (n->overlap_dw) {
       // dY_i is final and the last reader of the old W_i has been enqueued: dW_i may start beside
@@ -584,7 +588,7 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
     mbd_status s = run_gemm(n, l.bwd_weight, 2, l.d_out, l.d_in, n->B, l.dY, l.d_out, layer_input(n, i), l.d_in, S_c, e, ws,
                             ws ? n->partials_dw : nullptr);
     if (s != MBD_OK) return s;
-    if (fused && n->master) {
+    if (master_kernel) {
       cudaStream_t us = ws ? ws : n->stream;
       n->prof.begin(MBD_K_SGD, static_cast<double>(l.nW) * 14.0, us);
       CK(sgd_master_update_launch(l.W32, l.W, l.dW, l.nW, scale, n->num_sms, us));
