@@ -608,7 +608,7 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
   {
     double best = 1e30;
     int best_bn = 128, best_mh = 1, best_x = 1, best_pair = 0;
-    const int x_max = g.allow_extra_split ? 8 : 1;
+    const int x_max = g.allow_extra_split ? 32 : 1;
     for (int cand = 0; cand < 4; ++cand) {           // 0: 128-row tiles, 1: 256-row tiles, 2: CTA pairs, 3: pairs of 256-row CTAs
       const int mh = (cand == 1 || cand == 3) ? 2 : 1;
       const bool pair = cand >= 2;
