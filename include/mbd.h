@@ -324,6 +324,26 @@ MBD_API mbd_status mbd_block_reduce(const float* parts_dev, int S, int64_t M, in
 MBD_API mbd_status mbd_softmax_xent(const float* logits_dev, int64_t B, int64_t d, const int32_t* labels_dev,
                             void* dY_dev, int dY_bf16, float* per_sample_dev, int sync, void* cuda_stream);
 
+/* ---- The convolution step piece by piece, for a driver with one process per row strip (Section 2.2) ----
+ * A process holds its strip of every image as a network of its own (H = its rows) and exchanges the
+ * strips' outer rows with its neighbours between the pieces: mbd_conv_stage_input, then per layer
+ * [outer halo rows of the layer's input, if its kernel is 3x3] mbd_conv_forward_layer; backward per layer
+ * from the top [outer halo rows of dY_layer, if 3x3 and layer > 0] mbd_conv_backward_layer (the gradient
+ * with respect to the layer's input, then the layer's weight gradient).  mbd_forward / mbd_backward are
+ * exactly these pieces in a row.  Pure convolution stacks only (MBD_E_UNSUPPORTED otherwise).
+ *
+ * mbd_conv_outer_rows: rows_dev is [B][W][C] bf16 (bytes = B*W*C*2).  set == 0 reads the first (side 0) or
+ * last (side 1) OWN row of every image of the tensor -- what the process above / below needs as its halo
+ * row; set != 0 writes the upper (side 0) or lower (side 1) HALO row, which is zero (the image border)
+ * unless written.  which = MBD_T_ACT (output of `layer`; layer -1 = the staged input) or MBD_T_DY.
+ * mbd_set_tensor(MBD_T_DW) on a convolution stack replaces the materialised weight gradient (e.g. by its
+ * sum over all processes) before mbd_sgd_step. */
+MBD_API mbd_status mbd_conv_stage_input(mbd_net* net, const void* X_dev);
+MBD_API mbd_status mbd_conv_forward_layer(mbd_net* net, int layer, float* loss_sum_dev);
+MBD_API mbd_status mbd_conv_backward_layer(mbd_net* net, int layer, float fused_eta);
+MBD_API mbd_status mbd_conv_outer_rows(mbd_net* net, int which, int layer, int side, void* rows_dev,
+                               size_t bytes, int set);
+
 /* Failure-detection self test: launches one small kernel whose only job is to wait, with a
  * limit of `limit_ms` milliseconds, on a barrier that nothing will ever signal.  The kernel
  * gives up when the limit runs out, records a status code and returns normally; the call then

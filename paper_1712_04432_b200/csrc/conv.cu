@@ -197,6 +197,24 @@ __global__ void extract_1x1_kernel(const T* __restrict__ K, T* __restrict__ K1) 
   if (i < C * C) K1[i] = K[i * 9 + 4];
 }
 
+__global__ void embed_1x1_f32_kernel(const float* __restrict__ g1, float* __restrict__ g) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < C * C * 9) g[i] = (i % 9) == 4 ? g1[i / 9] : 0.f;
+}
+
+// One row of every image between the strips tensor and a dense [B][W][C] buffer (see conv_outer_rows).
+__global__ void __launch_bounds__(256)
+outer_rows_kernel(bf16* __restrict__ buf, bf16* __restrict__ rows, int W, int P_r, int R, int strip, int row, int set) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;      // 16-byte piece inside the row
+  const int per_image = W * C / 8;
+  if (i >= per_image) return;
+  const int b = blockIdx.y;
+  uint4* in_strips = reinterpret_cast<uint4*>(buf + ((static_cast<int64_t>(b) * P_r + strip) * R + row) * W * C) + i;
+  uint4* in_rows = reinterpret_cast<uint4*>(rows + static_cast<int64_t>(b) * W * C) + i;
+  if (set) *in_strips = *in_rows;
+  else *in_rows = *in_strips;
+}
+
 // Sum of the per-CTA partials [G][9][c][o] in CTA order, into canonical [o][c][u][v]:
 // either stored (dK) or applied as K += scale * dK (Eq. 1); the updated weight also goes into the
 // two operand layouts the next step's kernels read (see pack_weights_kernel).
@@ -1017,31 +1035,43 @@ mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev) {
 
 size_t conv_input_bytes(const ConvNet* c) { return static_cast<size_t>(c->B) * C * c->H * c->W * 2; }
 
-mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
-  // stage the input into strips (with its halo rows); the operand layouts of the weights are kept current
-  // by whatever changes the weights (conv_set_weights, the fused update, conv_sgd_step)
+// The step, piece by piece (a multi-process driver exchanges the image's outer halo rows between the pieces;
+// conv_forward / conv_backward below are these pieces in a row).
+mbd_status conv_stage_input(ConvNet* c, const void* X_nchw) {
+  // the input goes into strips (with the halo rows between its own strips); the operand layouts of the weights
+  // are kept current by whatever changes the weights (conv_set_weights, the fused update, conv_sgd_step)
   launch_stage_in(c, static_cast<const bf16*>(X_nchw), c->act[0]);
-  for (int i = 0; i < c->L; ++i) {
-    const bool last = i == c->L - 1;
-    // forward halo exchange (first halo term of Eq. 7): the kernel that produced act[i] (or the staging pass,
-    // for the network input) has already stored its boundary rows into the neighbouring strips' halo rows
-    launch_fwd(c, MBD_K_CONV_FWD, i, c->act_fwd[i], c->wf_map[i], c->act[i + 1], c->act_tile[i + 1],
-               (last && !c->fc_above) ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK), nullptr, nullptr);
-  }
-  if (loss_sum_dev && !c->fc_above) {
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+mbd_status conv_forward_layer(ConvNet* c, int i, float* loss_sum_dev) {
+  if (i < 0 || i >= c->L) return MBD_E_INVALID;
+  const bool last = i == c->L - 1;
+  // forward halo exchange (first halo term of Eq. 7): the kernel that produced act[i] (or the staging pass,
+  // for the network input) has already stored its boundary rows into the neighbouring strips' halo rows
+  launch_fwd(c, MBD_K_CONV_FWD, i, c->act_fwd[i], c->wf_map[i], c->act[i + 1], c->act_tile[i + 1],
+             (last && !c->fc_above) ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK), nullptr, nullptr);
+  if (last && loss_sum_dev && !c->fc_above) {
     c->prof->begin(MBD_K_OTHER, c->grid * 32.0);
     if (sum_f32_launch(c->loss_part, c->grid * 8, 0.5f, loss_sum_dev, c->stream) != cudaSuccess) return MBD_E_CUDA;
     c->prof->end();
   }
   if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
-  c->state = 1;
+  if (last) c->state = 1;
   return MBD_OK;
 }
 
-mbd_status conv_backward(ConvNet* c, float fused_eta) {
+mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
+  mbd_status s = conv_stage_input(c, X_nchw);
+  for (int i = 0; i < c->L && s == MBD_OK; ++i) s = conv_forward_layer(c, i, loss_sum_dev);
+  return s;
+}
+
+mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta) {
+  if (i < 0 || i >= c->L) return MBD_E_INVALID;
   const bool fused = fused_eta > 0.f;
   const float scale = -fused_eta / static_cast<float>(c->B);
-  for (int i = c->L - 1; i >= 0; --i) {
+  {
     if (i > 0) {
       // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0]
       // (the producer of dY_i has stored its boundary rows into the neighbours' halo rows)
@@ -1065,8 +1095,41 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
     c->prof->end();
   }
   if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
-  c->state = fused ? 3 : 2;
+  if (i == 0) c->state = fused ? 3 : 2;
   return MBD_OK;
+}
+
+mbd_status conv_backward(ConvNet* c, float fused_eta) {
+  mbd_status s = MBD_OK;
+  for (int i = c->L - 1; i >= 0 && s == MBD_OK; --i) s = conv_backward_layer(c, i, fused_eta);
+  return s;
+}
+
+// The outer rows of every image: its first / last own row (what a neighbouring process needs as a halo row) is
+// read out, or its upper / lower halo row (zero unless a neighbour supplies it) is written.  `side` 0 = top,
+// 1 = bottom; the row buffer is [B][W][C] bf16.  which / layer as in conv_get_tensor; layer -1 = the staged input.
+mbd_status conv_outer_rows(ConvNet* c, int which, int layer, int side, void* rows, size_t bytes, int set) {
+  if (layer < -1 || layer >= c->L || (side != 0 && side != 1)) return MBD_E_INVALID;
+  if (bytes != static_cast<size_t>(c->B) * c->W * C * 2) return MBD_E_INVALID;
+  bf16* buf = which == MBD_T_ACT ? c->act[layer + 1] : (which == MBD_T_DY && layer >= 0) ? c->dY[layer] : nullptr;
+  if (!buf) return MBD_E_INVALID;
+  const int strip = side == 0 ? 0 : c->P_r - 1;
+  const int row = set ? (side == 0 ? 0 : c->Hs + 1) : (side == 0 ? 1 : c->Hs);
+  const int per_image = c->W * C / 8;                       // 16-byte pieces per row
+  dim3 g((per_image + 255) / 256, static_cast<unsigned>(c->B));
+  outer_rows_kernel<<<g, 256, 0, c->stream>>>(buf, static_cast<bf16*>(rows), c->W, c->P_r, c->R, strip, row, set);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+mbd_status conv_set_dw(ConvNet* c, int layer, const void* src, size_t bytes) {
+  if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
+  if (c->k1[layer]) {
+    if (bytes != C * C * 4) return MBD_E_INVALID;
+    embed_1x1_f32_kernel<<<(9 * C * C + 255) / 256, 256, 0, c->stream>>>(static_cast<const float*>(src), c->dK[layer]);
+    return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+  }
+  if (bytes != 9 * C * C * 4) return MBD_E_INVALID;
+  return cudaMemcpyAsync(c->dK[layer], src, bytes, cudaMemcpyDeviceToDevice, c->stream) == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
 mbd_status conv_sgd_step(ConvNet* c, float eta) {

@@ -804,7 +804,7 @@ extern "C" mbd_status mbd_get_tensor(mbd_net* n, int which, int layer, void* dst
 
 extern "C" mbd_status mbd_set_tensor(mbd_net* n, int which, int layer, const void* src, size_t bytes) {
   if (!n || !src) return MBD_E_INVALID;
-  if (n->is_conv) return conv_set_tensor(n->conv, which, layer, src, bytes);
+  if (n->is_conv) return which == MBD_T_DW ? conv_set_dw(n->conv, layer, src, bytes) : conv_set_tensor(n->conv, which, layer, src, bytes);
   if (n->mixed) {
     if (layer >= 0 && layer < n->Lc) {
       const mbd_status s = conv_set_tensor(n->conv, which, layer, src, bytes);
@@ -826,6 +826,39 @@ extern "C" mbd_status mbd_set_tensor(mbd_net* n, int which, int layer, const voi
   if (bytes != size) return MBD_E_INVALID;
   CK(cudaMemcpyAsync(dst, src, size, cudaMemcpyDeviceToDevice, n->stream));
   return MBD_OK;
+}
+
+// ---- the convolution step piece by piece (pure convolution stacks; one process per strip, Section 2.2) ----
+extern "C" mbd_status mbd_conv_stage_input(mbd_net* n, const void* X_dev) {
+  if (!n || !X_dev) return MBD_E_INVALID;
+  if (!n->is_conv) return MBD_E_UNSUPPORTED;
+  n->state = ST_IDLE;
+  return conv_stage_input(n->conv, X_dev);
+}
+
+extern "C" mbd_status mbd_conv_forward_layer(mbd_net* n, int layer, float* loss_sum_dev) {
+  if (!n) return MBD_E_INVALID;
+  if (!n->is_conv) return MBD_E_UNSUPPORTED;
+  if (layer < 0 || layer >= n->Lc) return MBD_E_INVALID;
+  const mbd_status s = conv_forward_layer(n->conv, layer, loss_sum_dev);
+  if (s == MBD_OK && layer == n->Lc - 1) n->state = ST_FWD;
+  return s;
+}
+
+extern "C" mbd_status mbd_conv_backward_layer(mbd_net* n, int layer, float fused_eta) {
+  if (!n || fused_eta < 0.f) return MBD_E_INVALID;
+  if (!n->is_conv) return MBD_E_UNSUPPORTED;
+  if (layer < 0 || layer >= n->Lc) return MBD_E_INVALID;
+  if (n->state != ST_FWD) return MBD_E_STATE;
+  const mbd_status s = conv_backward_layer(n->conv, layer, fused_eta);
+  if (s == MBD_OK && layer == 0) n->state = fused_eta > 0.f ? ST_BWD_FUSED : ST_BWD_UNFUSED;
+  return s;
+}
+
+extern "C" mbd_status mbd_conv_outer_rows(mbd_net* n, int which, int layer, int side, void* rows_dev, size_t bytes, int set) {
+  if (!n || !rows_dev) return MBD_E_INVALID;
+  if (!n->is_conv) return MBD_E_UNSUPPORTED;
+  return conv_outer_rows(n->conv, which, layer, side, rows_dev, bytes, set);
 }
 
 extern "C" mbd_status mbd_poll_status(mbd_net* n) {

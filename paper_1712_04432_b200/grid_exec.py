@@ -17,6 +17,10 @@ The words every collective moves per process are counted from the buffers actual
 they can be compared with mbd_comm_words.
 
 Rank layout: rank = c * P_r + r.
+
+GridConv runs stacks of convolutions the same way under domain + batch parallelism (Section 2.2): one
+process per row strip, halo rows exchanged with the neighbouring processes before every 3 x 3 layer,
+weight gradients summed over all processes.
 """
 from __future__ import annotations
 
@@ -202,6 +206,96 @@ class GridFC:
             self.status.zero_()
             raise mbd.MbdError(mbd.E_TIMEOUT, "grid step")
         return loss
+
+
+class GridConv:
+    """One process's share of a stack of 64-channel convolutions under domain + batch parallelism
+    (Section 2.2, Eq. 7 / Eq. 9): strip r (H / P_r rows) of the images of batch block c, held as a network of
+    its own.  Before every 3 x 3 layer the strips' outer rows are exchanged with the processes above and
+    below (a 1 x 1 layer needs none); the weight gradients are summed over all P processes.  Loss: half the
+    sum of squares of the last layer's output."""
+
+    def __init__(self, ksizes: Sequence[int], C_: int, H: int, W: int, B: int, comm: GridComm):
+        import torch
+        self.t = torch
+        self.comm = comm
+        P_r, P_c = comm.P_r, comm.P_c
+        if H % P_r or B % P_c:
+            raise ValueError("H must divide into P_r strips and the batch into P_c blocks")
+        self.ksizes = [int(k) for k in ksizes]
+        self.L = len(self.ksizes)
+        self.C, self.Hs, self.W, self.m = int(C_), H // P_r, int(W), B // P_c
+        self.net = mbd.Net(mbd.conv_layers(self.L, C_, self.Hs, W, k=self.ksizes), self.m, 1, 1, mbd.BF16,
+                           mbd.LOSS_HALF_SSQ, 0)
+        comm.words.setdefault("halo_fwd", 0.0)
+        comm.words.setdefault("halo_bwd", 0.0)
+        self.dK: List = [None] * self.L
+
+    def set_weights(self, i: int, K):
+        self.net.set_weights(i, K)
+
+    def _exchange(self, which: int, layer: int, kind: str):
+        """First own rows go to the process above, last own rows to the process below; what arrives becomes
+        this strip's halo rows.  Counted as the paper counts it: one boundary of (B / P_c) W C words."""
+        comm, dist, t = self.comm, self.comm.dist, self.t
+        if comm.P_r == 1:
+            return
+        up = comm.rank - 1 if comm.r > 0 else None
+        down = comm.rank + 1 if comm.r < comm.P_r - 1 else None
+        ops, got = [], {}
+        for side, peer in ((0, up), (1, down)):
+            if peer is None:
+                continue
+            out = self.net.conv_outer_rows(which, layer, side)
+            if comm.via_host:
+                out = out.cpu()
+            inc = t.empty_like(out)
+            got[side] = inc
+            ops.append(dist.P2POp(dist.isend, out, peer))
+            ops.append(dist.P2POp(dist.irecv, inc, peer))
+        for req in dist.batch_isend_irecv(ops):
+            req.wait()
+        for side, inc in got.items():
+            self.net.conv_outer_rows(which, layer, side, rows=inc.cuda() if comm.via_host else inc)
+        comm.words[kind] += self.m * self.W * self.C
+
+    def step(self, X_local, eta: float):
+        """One step on this process's strip X_local [B / P_c, C, H / P_r, W] (bf16).  Returns its share of J."""
+        t, net, comm, L = self.t, self.net, self.comm, self.L
+        J = t.zeros(1, dtype=t.float32, device="cuda")
+        net.conv_stage_input(X_local)
+        for i in range(L):
+            if self.ksizes[i] == 3:
+                self._exchange(mbd.T_ACT, i - 1, "halo_fwd")        # halo rows of the layer's input (Eq. 7, term 1)
+            net.conv_forward_layer(i, J if i == L - 1 else None)
+        for i in range(L - 1, -1, -1):
+            if i > 0 and self.ksizes[i] == 3:
+                self._exchange(mbd.T_DY, i, "halo_bwd")             # halo rows of dY_i (Eq. 7, term 2)
+            net.conv_backward_layer(i, 0.0)
+        P = comm.P_r * comm.P_c
+        for i in range(L):                                            # all-reduce over all P processes (Eq. 7, term 3)
+            g = net.get_tensor(mbd.T_DW, i)
+            if P > 1:
+                if comm.via_host:
+                    h = g.cpu()
+                    comm.dist.all_reduce(h)
+                    g.copy_(h)
+                else:
+                    comm.dist.all_reduce(g)
+                comm.words["allreduce_dw"] += 2.0 * (P - 1) / P * g.numel()
+                net.set_tensor(mbd.T_DW, i, g)
+            self.dK[i] = g
+        net.sgd_step(eta / comm.P_c)          # the library divides by its own batch B / P_c: eta / B in total
+        net.poll()
+        return float(J.item())
+
+
+def expected_conv_words(ksizes: Sequence[int], C_: int, H: int, W: int, B: int, P_r: int, P_c: int) -> Dict[str, int]:
+    """Per-process totals of mbd_comm_words (Eq. 9 with all layers in L_D).  The backward halo term is summed
+    over the layers above the first: the formula counts it for every layer, the first layer needs no dX."""
+    rows = mbd.comm_words(mbd.conv_layers(len(ksizes), C_, H, W, k=list(ksizes)), B, P_r, P_c)
+    return {"halo_fwd": sum(r["halo_fwd"] for r in rows), "halo_bwd": sum(r["halo_bwd"] for r in rows[1:]),
+            "allreduce_dw": sum(r["allreduce_dw"] for r in rows)}
 
 
 def expected_words(dims: Sequence[int], B: int, P_r: int, P_c: int) -> Dict[str, int]:

@@ -28,7 +28,8 @@ EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weig
            "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_gemm_bf16_noalloc", "mbd_selftest_timeout", "mbd_strerror",
            "mbd_train_step_host_begin", "mbd_train_step_host_end",
            "mbd_comm_time", "mbd_redistribute_time", "mbd_total_time", "mbd_grid_table", "mbd_choose_grid",
-           "mbd_enable_master_weights", "mbd_block_gemm_bf16", "mbd_block_reduce", "mbd_softmax_xent"]
+           "mbd_enable_master_weights", "mbd_block_gemm_bf16", "mbd_block_reduce", "mbd_softmax_xent",
+           "mbd_conv_stage_input", "mbd_conv_forward_layer", "mbd_conv_backward_layer", "mbd_conv_outer_rows"]
 
 
 class MbdError(RuntimeError):
@@ -120,6 +121,10 @@ def lib():
         L.mbd_block_gemm_bf16.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, C.POINTER(Tail), vp, vp]
         L.mbd_block_reduce.argtypes = [vp, i32, i64, i64, C.POINTER(Tail), i32, vp]
         L.mbd_softmax_xent.argtypes = [vp, i64, i64, vp, vp, i32, vp, i32, vp]
+        L.mbd_conv_stage_input.argtypes = [vp, vp]
+        L.mbd_conv_forward_layer.argtypes = [vp, i32, vp]
+        L.mbd_conv_backward_layer.argtypes = [vp, i32, f32]
+        L.mbd_conv_outer_rows.argtypes = [vp, i32, i32, i32, vp, C.c_size_t, i32]
         L.mbd_profile_enable.argtypes = [vp, i32]
         L.mbd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double)]
         L.mbd_launch_count.argtypes = [vp]
@@ -283,6 +288,31 @@ class Net:
             assert labels.is_cuda and labels.dtype == self._torch.int32 and labels.is_contiguous()
         self._keep = [X, labels, loss_out]      # the library reads X again during backward
         _check(lib().mbd_forward(self._h, _ptr(X), _ptr(labels), _ptr(loss_out)), "mbd_forward")
+
+    # -- the convolution step piece by piece (see include/mbd.h)
+    def conv_stage_input(self, X):
+        assert X.is_cuda and X.is_contiguous() and X.dtype == self.act_dtype
+        self._keep = [X]
+        _check(lib().mbd_conv_stage_input(self._h, _ptr(X)), "mbd_conv_stage_input")
+
+    def conv_forward_layer(self, layer: int, loss_out=None):
+        _check(lib().mbd_conv_forward_layer(self._h, layer, _ptr(loss_out)), "mbd_conv_forward_layer")
+
+    def conv_backward_layer(self, layer: int, fused_eta: float = 0.0):
+        _check(lib().mbd_conv_backward_layer(self._h, layer, float(fused_eta)), "mbd_conv_backward_layer")
+
+    def conv_outer_rows(self, which: int, layer: int, side: int, rows=None):
+        """rows None: returns the first (side 0) / last (side 1) own row of every image, [B, W, C] bf16;
+        otherwise writes `rows` into the upper / lower halo row."""
+        t = self._torch
+        l = self.layers[0]
+        get = rows is None
+        if get:
+            rows = t.empty((self.B, l.W, l.C_out), dtype=t.bfloat16, device="cuda")
+        assert rows.is_cuda and rows.is_contiguous() and rows.dtype == t.bfloat16
+        _check(lib().mbd_conv_outer_rows(self._h, which, layer, side, _ptr(rows), rows.numel() * 2, int(not get)),
+               "mbd_conv_outer_rows")
+        return rows
 
     def enable_master_weights(self):
         """fp32 master copies of all weights from now on (see include/mbd.h)."""

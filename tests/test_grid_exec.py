@@ -142,3 +142,70 @@ def test_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, P_r, P_c):
             assert rel_fro(z[f"W{i}"], o["new_W"][i][rows]) < 1e-2, (rank, i)
         assert json.loads(str(z["words"])) == json.loads(str(z["want"]))          # Eq. 8, per process
     assert abs(loss - o["J"]) < 1e-2 * abs(o["J"])
+
+
+CONV_WORKER = r'''
+import json, os, sys
+sys.path.insert(0, %(root)r)
+import numpy as np
+import torch, torch.distributed as dist
+from paper_1712_04432_b200 import inputs as I, mbd
+from paper_1712_04432_b200.grid_exec import GridComm, GridConv, expected_conv_words
+from tests.helpers import to_dev
+torch.cuda.set_device(0)
+dist.init_process_group("gloo")
+P_r, P_c = %(P_r)d, %(P_c)d
+ksizes, H, W, B, eta, out_dir = %(ksizes)r, %(H)d, %(W)d, %(B)d, %(eta)r, %(out)r
+comm = GridComm(P_r, P_c, via_host=True)
+w = I.conv_workload(64, H, W, B, n_layers=len(ksizes), ksizes=ksizes)
+inp = I.make_inputs(w, seed=%(seed)d)                      # every process draws the same tensors and takes its block
+net = GridConv(ksizes, 64, H, W, B, comm)
+for i in range(len(ksizes)):
+    net.set_weights(i, to_dev(inp.Ws[i], True))
+m, Hs = B // P_c, H // P_r
+X_local = to_dev(np.ascontiguousarray(inp.X[comm.c * m:(comm.c + 1) * m, :, comm.r * Hs:(comm.r + 1) * Hs, :]), True)
+loss = net.step(X_local, eta)
+torch.cuda.synchronize()
+L = len(ksizes)
+np.savez(os.path.join(out_dir, "rank%%d.npz" %% dist.get_rank()), r=comm.r, c=comm.c, loss=loss,
+         Y=net.net.get_tensor(mbd.T_ACT, L - 1).float().cpu().numpy(),
+         dY0=net.net.get_tensor(mbd.T_DY, 0).float().cpu().numpy(),
+         **{"K%%d" %% i: net.net.get_weights(i).float().cpu().numpy() for i in range(L)},
+         **{"dK%%d" %% i: net.dK[i].cpu().numpy() for i in range(L)},
+         words=json.dumps({k: int(round(v)) for k, v in comm.words.items() if k in ("halo_fwd", "halo_bwd", "allreduce_dw")}),
+         want=json.dumps(expected_conv_words(ksizes, 64, H, W, B, P_r, P_c)))
+dist.barrier()
+dist.destroy_process_group()
+'''
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("P_r,P_c,ksizes", [(2, 1, (3, 3)), (2, 2, (3, 1, 3)), (4, 1, (3, 3, 3)), (1, 2, (3, 3))])
+def test_convolution_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, P_r, P_c, ksizes):
+    from paper_1712_04432_b200 import inputs as I
+    from tests.helpers import like_device, oracle_conv_step, rel_fro
+    H, W, B, eta, seed = 16, 40, 4, 2e-5, 92
+    script = tmp_path / "conv_worker.py"
+    script.write_text(CONV_WORKER % {"root": ROOT, "P_r": P_r, "P_c": P_c, "ksizes": list(ksizes), "H": H, "W": W, "B": B,
+                                     "eta": eta, "out": str(tmp_path), "seed": seed})
+    r = _torchrun(script, P_r * P_c, 29571 + P_r + 2 * P_c)
+    assert r.returncode == 0, (r.stdout[-1500:], r.stderr[-3000:])
+
+    w = I.conv_workload(64, H, W, B, n_layers=len(ksizes), ksizes=ksizes)
+    w.eta = eta
+    inp = I.make_inputs(w, seed=seed)
+    o = oracle_conv_step(w, inp)
+    L, m, Hs = len(ksizes), B // P_c, H // P_r
+    loss = 0.0
+    for rank in range(P_r * P_c):
+        z = np.load(tmp_path / f"rank{rank}.npz")
+        rr, cc = int(z["r"]), int(z["c"])
+        loss += float(z["loss"])
+        own = (slice(cc * m, (cc + 1) * m), slice(None), slice(rr * Hs, (rr + 1) * Hs), slice(None))
+        assert rel_fro(z["Y"], o["Ys"][L - 1][own]) < 1e-2, rank                 # this strip of the last layer's output
+        assert rel_fro(z["dY0"], o["dYs"][0][own]) < 5e-2, rank                  # ... and of the gradient that reached layer 1
+        for i in range(L):
+            assert rel_fro(z[f"dK{i}"], like_device(o["dWs"][i], z[f"dK{i}"])) < (1e-2 if i == L - 1 else 5e-2), (rank, i)
+            assert rel_fro(z[f"K{i}"], like_device(o["new_W"][i], z[f"K{i}"])) < 1e-2, (rank, i)
+        assert json.loads(str(z["words"])) == json.loads(str(z["want"]))        # Eq. 9's terms for domain layers, per process
+    assert abs(loss - o["J"]) < 1e-2 * abs(o["J"])
