@@ -64,7 +64,11 @@ typedef enum {
 enum { MBD_FC = 0, MBD_CONV3X3 = 1 };                 /* mbd_layer.kind                      */
 enum { MBD_SPLIT_MODEL = 0, MBD_SPLIT_DOMAIN = 1 };   /* mbd_layer.split: L_M or L_D, Eq. 9  */
 enum { MBD_F32 = 0, MBD_BF16 = 1 };                   /* dtype                               */
-enum { MBD_LOSS_SOFTMAX_CE = 0, MBD_LOSS_HALF_SSQ = 1 };
+enum { MBD_LOSS_SOFTMAX_CE = 0, MBD_LOSS_HALF_SSQ = 1,
+       MBD_LOSS_NONE = 2 };   /* convolution stacks only: no loss here.  The last layer applies its ReLU like
+                                 any other, and the caller supplies dJ/dY of the last layer with
+                                 mbd_set_tensor(MBD_T_DY, L-1) between the forward and the backward pass
+                                 (the stack is the lower part of a larger network). */
 
 /* One layer.  FC: d_in, d_out.  Convolution (3x3, stride 1, zero pad 1, NCHW):
  * C_in, C_out, H, W, kh = kw = 3; d_in = C_in*H*W, d_out = C_out*H*W (Eq. 2).

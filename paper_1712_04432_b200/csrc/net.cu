@@ -270,7 +270,7 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
                                      int max_partials, void* cuda_stream, mbd_net** out) {
   if (!layers || !out || L < 1 || B < 1) return MBD_E_INVALID;
   if (dtype != MBD_F32 && dtype != MBD_BF16) return MBD_E_INVALID;
-  if (loss != MBD_LOSS_SOFTMAX_CE && loss != MBD_LOSS_HALF_SSQ) return MBD_E_INVALID;
+  if (loss != MBD_LOSS_SOFTMAX_CE && loss != MBD_LOSS_HALF_SSQ && loss != MBD_LOSS_NONE) return MBD_E_INVALID;
   if (max_partials < 0) return MBD_E_INVALID;
   *out = nullptr;
   if (P_r < 1 || P_c < 1 || P_c > B) return MBD_E_GRID;
@@ -298,7 +298,7 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
       return MBD_E_INVALID;
     }
   }
-  if (is_conv && loss != MBD_LOSS_HALF_SSQ) return MBD_E_UNSUPPORTED;
+  if (is_conv && loss != MBD_LOSS_HALF_SSQ && loss != MBD_LOSS_NONE) return MBD_E_UNSUPPORTED;
   if (!is_conv && loss != MBD_LOSS_SOFTMAX_CE) return MBD_E_UNSUPPORTED;
   if (mixed && dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
 
@@ -334,7 +334,8 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   if (cudaMemsetAsync(n->status, 0, sizeof(int), n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
 
   if (Lc > 0) {
-    st = conv_create(layers, Lc, B, P_r, n->max_partials, n->num_sms, n->status, n->stream, &n->prof, mixed, &n->conv);
+    st = conv_create(layers, Lc, B, P_r, n->max_partials, n->num_sms, n->status, n->stream, &n->prof,
+                     mixed || loss == MBD_LOSS_NONE, &n->conv);
     if (st != MBD_OK) { free_net(n); return st; }
     if (is_conv) {
       *out = n;

@@ -159,9 +159,11 @@ class GridFC:
         a, b = self.rows(i)
         self.W[i].copy_(W_full[a:b])
 
-    def step(self, X_c, labels_c, eta: float):
+    def step(self, X_c, labels_c, eta: float, input_is_relu_output: bool = False):
         """One step on the batch block X_c [B / P_c, d_0] (bf16), labels_c int32.  Returns the sum of the
-        losses of this block; the logits are kept in self.logits."""
+        losses of this block; the logits are kept in self.logits.  `input_is_relu_output`: the stack sits on
+        top of other layers whose ReLU output X_c is -- the gradient with respect to X_c is then formed as
+        well (masked by [X_c > 0]) and kept in self.dX0."""
         t, comm = self.t, self.comm
         m, L = self.m, self.L
         assert tuple(X_c.shape) == (m, self.dims[0]) and X_c.dtype == t.bfloat16
@@ -188,7 +190,7 @@ class GridFC:
             a, b = self.rows(i)
             dY_r = dY[:, a:b]                                           # dY_i(r, c): this process's rows of layer i's output
             dY_prev = None
-            if i > 0:
+            if i > 0 or input_is_relu_output:
                 part = t.empty((m, self.dims[i]), dtype=t.float32, device=self.device)
                 mbd.block_gemm(1, dY_r, self.W[i], part, mbd.TAIL_STORE, status=self.status)       # W_i(r, :)^T dY_i(r, c), one summand
                 comm.all_reduce_(part, "rows", "allreduce_dx")
@@ -201,6 +203,7 @@ class GridFC:
                 self._update(pending, scale)
             pending = (i, handle)
             dY = dY_prev
+        self.dX0 = dY                                                   # None unless input_is_relu_output
         self._update(pending, scale)
         if int(self.status.item()) != 0:             # (synchronises) a bounded wait inside a product gave up
             self.status.zero_()
@@ -215,18 +218,19 @@ class GridConv:
     below (a 1 x 1 layer needs none); the weight gradients are summed over all P processes.  Loss: half the
     sum of squares of the last layer's output."""
 
-    def __init__(self, ksizes: Sequence[int], C_: int, H: int, W: int, B: int, comm: GridComm):
+    def __init__(self, ksizes: Sequence[int], C_: int, H: int, W: int, B: int, comm: GridComm,
+                 loss: int = mbd.LOSS_HALF_SSQ):
         import torch
         self.t = torch
         self.comm = comm
+        self.loss = loss
         P_r, P_c = comm.P_r, comm.P_c
         if H % P_r or B % P_c:
             raise ValueError("H must divide into P_r strips and the batch into P_c blocks")
         self.ksizes = [int(k) for k in ksizes]
         self.L = len(self.ksizes)
         self.C, self.Hs, self.W, self.m = int(C_), H // P_r, int(W), B // P_c
-        self.net = mbd.Net(mbd.conv_layers(self.L, C_, self.Hs, W, k=self.ksizes), self.m, 1, 1, mbd.BF16,
-                           mbd.LOSS_HALF_SSQ, 0)
+        self.net = mbd.Net(mbd.conv_layers(self.L, C_, self.Hs, W, k=self.ksizes), self.m, 1, 1, mbd.BF16, loss, 0)
         comm.words.setdefault("halo_fwd", 0.0)
         comm.words.setdefault("halo_bwd", 0.0)
         self.dK: List = [None] * self.L
@@ -261,13 +265,24 @@ class GridConv:
 
     def step(self, X_local, eta: float):
         """One step on this process's strip X_local [B / P_c, C, H / P_r, W] (bf16).  Returns its share of J."""
-        t, net, comm, L = self.t, self.net, self.comm, self.L
+        J = self.forward(X_local)
+        self.backward(eta)
+        return J
+
+    def forward(self, X_local):
+        t, net, L = self.t, self.net, self.L
         J = t.zeros(1, dtype=t.float32, device="cuda")
         net.conv_stage_input(X_local)
         for i in range(L):
             if self.ksizes[i] == 3:
                 self._exchange(mbd.T_ACT, i - 1, "halo_fwd")        # halo rows of the layer's input (Eq. 7, term 1)
             net.conv_forward_layer(i, J if i == L - 1 else None)
+        return float(J.item()) if self.loss == mbd.LOSS_HALF_SSQ else 0.0
+
+    def backward(self, eta: float):
+        """Backward pass and update.  With LOSS_NONE the gradient of the last layer's output must have been
+        set before (net.set_tensor(T_DY, L - 1, ...))."""
+        t, net, comm, L = self.t, self.net, self.comm, self.L
         for i in range(L - 1, -1, -1):
             if i > 0 and self.ksizes[i] == 3:
                 self._exchange(mbd.T_DY, i, "halo_bwd")             # halo rows of dY_i (Eq. 7, term 2)
@@ -287,7 +302,38 @@ class GridConv:
             self.dK[i] = g
         net.sgd_step(eta / comm.P_c)          # the library divides by its own batch B / P_c: eta / B in total
         net.poll()
-        return float(J.item())
+
+
+class GridMixed:
+    """The integrated network of Section 2.4 over processes: convolutions with the P_r groups splitting the
+    domain (GridConv), then fully connected layers with the same groups splitting the model (GridFC), one
+    P_r x P_c grid (Eq. 9).  Between the two the strips of the last convolution's output are all-gathered
+    over the P_r group into the [B / P_c, C H W] input every process of the group needs (the re-distribution
+    of Section 2.1, Eq. 6), and the gradient of that input goes back to the strips' owners without
+    communication: after the all-reduce of the first fully connected layer every process holds all of it."""
+
+    def __init__(self, ksizes: Sequence[int], C_: int, H: int, W: int, fc_dims: Sequence[int], B: int, comm: GridComm):
+        self.comm = comm
+        self.C, self.H, self.W = int(C_), int(H), int(W)
+        self.conv = GridConv(ksizes, C_, H, W, B, comm, loss=mbd.LOSS_NONE)
+        self.fc = GridFC([C_ * H * W] + [int(d) for d in fc_dims], B, comm)
+        comm.words.setdefault("redistribute", 0.0)
+
+    def step(self, X_local, labels_c, eta: float):
+        import torch
+        comm, conv = self.comm, self.conv
+        m, Hs, L = conv.m, conv.Hs, conv.L
+        conv.forward(X_local)
+        strip = conv.net.get_tensor(mbd.T_ACT, L - 1)                       # [m, C, Hs, W], after the ReLU
+        # all-gather of the strips over the P_r group; strip r' lands in rows r' Hs .. of every channel
+        gathered = torch.empty((m, comm.P_r, self.C * Hs * self.W), dtype=strip.dtype, device=strip.device)
+        comm.all_gather_cols(strip.view(m, -1), gathered.view(m, -1), kind="redistribute")
+        X_fc = gathered.view(m, comm.P_r, self.C, Hs, self.W).permute(0, 2, 1, 3, 4).reshape(m, -1).contiguous()
+        loss = self.fc.step(X_fc, labels_c, eta, input_is_relu_output=True)
+        dX = self.fc.dX0.view(m, self.C, self.H, self.W)[:, :, comm.r * Hs:(comm.r + 1) * Hs, :].contiguous()
+        conv.net.set_tensor(mbd.T_DY, L - 1, dX)
+        conv.backward(eta)
+        return loss
 
 
 def expected_conv_words(ksizes: Sequence[int], C_: int, H: int, W: int, B: int, P_r: int, P_c: int) -> Dict[str, int]:
@@ -296,6 +342,19 @@ def expected_conv_words(ksizes: Sequence[int], C_: int, H: int, W: int, B: int, 
     rows = mbd.comm_words(mbd.conv_layers(len(ksizes), C_, H, W, k=list(ksizes)), B, P_r, P_c)
     return {"halo_fwd": sum(r["halo_fwd"] for r in rows), "halo_bwd": sum(r["halo_bwd"] for r in rows[1:]),
             "allreduce_dw": sum(r["allreduce_dw"] for r in rows)}
+
+
+def expected_mixed_words(ksizes: Sequence[int], C_: int, H: int, W: int, fc_dims: Sequence[int], B: int, P_r: int,
+                         P_c: int) -> Dict[str, int]:
+    """Per-process totals of mbd_comm_words for the integrated stack (Eq. 9), plus the re-distribution between
+    the two groups of layers (Eq. 6 on the grid: (B / P_c) (P_r - 1) / P_r d words), which Eq. 9 leaves out."""
+    layers = mbd.conv_layers(len(ksizes), C_, H, W, k=list(ksizes)) + mbd.fc_layers([C_ * H * W] + list(fc_dims), bias=False)
+    rows = mbd.comm_words(layers, B, P_r, P_c)
+    n = len(ksizes)
+    return {"halo_fwd": sum(r["halo_fwd"] for r in rows), "halo_bwd": sum(r["halo_bwd"] for r in rows[1:]),
+            "allgather_y": sum(r["allgather_y"] for r in rows), "allreduce_dx": sum(r["allreduce_dx"] for r in rows),
+            "allreduce_dw": sum(r["allreduce_dw"] for r in rows),
+            "redistribute": (B // P_c) * (P_r - 1) * (C_ * H * W // P_r)}
 
 
 def expected_words(dims: Sequence[int], B: int, P_r: int, P_c: int) -> Dict[str, int]:

@@ -17,7 +17,7 @@ OK, E_INVALID, E_GRID, E_ALLOC, E_CUDA, E_STATE, E_TIMEOUT, E_UNSUPPORTED, E_TOO
 FC, CONV3X3 = 0, 1
 SPLIT_MODEL, SPLIT_DOMAIN = 0, 1
 F32, BF16 = 0, 1
-LOSS_SOFTMAX_CE, LOSS_HALF_SSQ = 0, 1
+LOSS_SOFTMAX_CE, LOSS_HALF_SSQ, LOSS_NONE = 0, 1, 2
 T_ACT, T_DY, T_DW, T_DB, T_LOSS, T_PARTIALS, T_MASTER = range(7)
 
 KERNEL_CLASSES = ["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce_partials", "softmax_xent", "colsum",

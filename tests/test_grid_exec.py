@@ -209,3 +209,80 @@ def test_convolution_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, 
             assert rel_fro(z[f"K{i}"], like_device(o["new_W"][i], z[f"K{i}"])) < 1e-2, (rank, i)
         assert json.loads(str(z["words"])) == json.loads(str(z["want"]))        # Eq. 9's terms for domain layers, per process
     assert abs(loss - o["J"]) < 1e-2 * abs(o["J"])
+
+
+MIXED_WORKER = r'''
+import json, os, sys
+sys.path.insert(0, %(root)r)
+import numpy as np
+import torch, torch.distributed as dist
+from paper_1712_04432_b200 import inputs as I, mbd
+from paper_1712_04432_b200.grid_exec import GridComm, GridMixed, expected_mixed_words
+from tests.helpers import to_dev
+torch.cuda.set_device(0)
+dist.init_process_group("gloo")
+P_r, P_c = %(P_r)d, %(P_c)d
+ksizes, H, W, fc, B, eta, out_dir = %(ksizes)r, %(H)d, %(W)d, %(fc)r, %(B)d, %(eta)r, %(out)r
+comm = GridComm(P_r, P_c, via_host=True)
+w = I.mixed_workload(64, H, W, len(ksizes), fc, B, ksizes=ksizes)
+inp = I.make_inputs(w, seed=%(seed)d)
+net = GridMixed(ksizes, 64, H, W, fc, B, comm)
+Lc = len(ksizes)
+for i in range(Lc):
+    net.conv.set_weights(i, to_dev(inp.Ws[i], True))
+for i in range(len(fc)):
+    net.fc.set_weights(i, to_dev(inp.Ws[Lc + i], True))
+m, Hs = B // P_c, H // P_r
+X_local = to_dev(np.ascontiguousarray(inp.X[comm.c * m:(comm.c + 1) * m, :, comm.r * Hs:(comm.r + 1) * Hs, :]), True)
+labels_c = torch.from_numpy(inp.labels[comm.c * m:(comm.c + 1) * m]).cuda()
+loss = net.step(X_local, labels_c, eta)
+torch.cuda.synchronize()
+np.savez(os.path.join(out_dir, "rank%%d.npz" %% dist.get_rank()), r=comm.r, c=comm.c, loss=loss,
+         logits=net.fc.logits.float().cpu().numpy(),
+         **{"K%%d" %% i: net.conv.net.get_weights(i).float().cpu().numpy() for i in range(Lc)},
+         **{"dK%%d" %% i: net.conv.dK[i].cpu().numpy() for i in range(Lc)},
+         **{"W%%d" %% i: net.fc.W[i].float().cpu().numpy() for i in range(len(fc))},
+         **{"dW%%d" %% i: net.fc.dW[i].cpu().numpy() for i in range(len(fc))},
+         words=json.dumps({k: int(round(v)) for k, v in comm.words.items()}),
+         want=json.dumps(expected_mixed_words(ksizes, 64, H, W, fc, B, P_r, P_c)))
+dist.barrier()
+dist.destroy_process_group()
+'''
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("P_r,P_c,ksizes", [(2, 2, (3, 3)), (4, 1, (3, 1)), (1, 2, (3,)), (2, 1, (1, 3))])
+def test_integrated_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, P_r, P_c, ksizes):
+    """Eq. 9 executed: domain-split convolutions, the re-distribution of Eq. 6, model-split fully connected layers."""
+    from paper_1712_04432_b200 import inputs as I
+    from tests.helpers import like_device, oracle_mixed_step, rel_fro
+    H, W, fc, B, eta, seed = 8, 40, [64, 32], 4, 0.02, 93
+    script = tmp_path / "mixed_worker.py"
+    script.write_text(MIXED_WORKER % {"root": ROOT, "P_r": P_r, "P_c": P_c, "ksizes": list(ksizes), "H": H, "W": W, "fc": fc,
+                                      "B": B, "eta": eta, "out": str(tmp_path), "seed": seed})
+    r = _torchrun(script, P_r * P_c, 29591 + P_r + 2 * P_c)
+    assert r.returncode == 0, (r.stdout[-1500:], r.stderr[-3000:])
+
+    w = I.mixed_workload(64, H, W, len(ksizes), fc, B, ksizes=ksizes)
+    w.eta = eta
+    inp = I.make_inputs(w, seed=seed)
+    o = oracle_mixed_step(w, inp)
+    Lc, Lf, m = len(ksizes), len(fc), B // P_c
+    dims = [64 * H * W] + fc
+    loss = 0.0
+    for rank in range(P_r * P_c):
+        z = np.load(tmp_path / f"rank{rank}.npz")
+        rr, cc = int(z["r"]), int(z["c"])
+        if rr == 0:
+            loss += float(z["loss"])
+        assert rel_fro(z["logits"], o["Ys"][-1].T[cc * m:(cc + 1) * m]) < 1e-2, rank
+        for i in range(Lc):
+            assert rel_fro(z[f"dK{i}"], like_device(o["dWs"][i], z[f"dK{i}"])) < 5e-2, (rank, i)
+            assert rel_fro(z[f"K{i}"], like_device(o["new_W"][i], z[f"K{i}"])) < 1e-2, (rank, i)
+        for i in range(Lf):
+            h = dims[i + 1] // P_r
+            rows = slice(rr * h, (rr + 1) * h)
+            assert rel_fro(z[f"dW{i}"], o["dWs"][Lc + i][rows]) < (1e-2 if i == Lf - 1 else 5e-2), (rank, i)
+            assert rel_fro(z[f"W{i}"], o["new_W"][Lc + i][rows]) < 1e-2, (rank, i)
+        assert json.loads(str(z["words"])) == json.loads(str(z["want"]))
+    assert abs(loss - o["J"]) < 1e-2 * abs(o["J"])

@@ -43,6 +43,8 @@ def test_invalid_and_unsupported():
     assert create(conv13, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
     assert create(mbd.conv_layers(2, 64, 8, 16, k=[3, 1]), 4, loss=mbd.LOSS_HALF_SSQ) in (mbd.OK, mbd.E_CUDA)   # valid; E_CUDA only without a device
     assert create(mbd.conv_layers(1, 64, 8, 16), 4, loss=mbd.LOSS_SOFTMAX_CE) == mbd.E_UNSUPPORTED
+    assert create(fc, 8, loss=mbd.LOSS_NONE) == mbd.E_UNSUPPORTED                          # "no loss" is for convolution stacks
+    assert create(mbd.conv_layers(1, 64, 8, 16), 4, loss=mbd.LOSS_NONE) in (mbd.OK, mbd.E_CUDA)
     # convolutions first, fully connected layers after them
     conv = mbd.conv_layers(1, 64, 8, 16)
     assert create(mbd.fc_layers((64, 64 * 8 * 16)) + conv, 4) == mbd.E_UNSUPPORTED          # convolution above an FC layer
@@ -58,6 +60,10 @@ def test_null_handles_are_rejected():
     assert L.mbd_sgd_step(None, 0.1) == mbd.E_INVALID
     assert L.mbd_poll_status(None) == mbd.E_INVALID
     assert L.mbd_enable_master_weights(None) == mbd.E_INVALID
+    assert L.mbd_conv_stage_input(None, None) == mbd.E_INVALID
+    assert L.mbd_conv_forward_layer(None, 0, None) == mbd.E_INVALID
+    assert L.mbd_conv_backward_layer(None, 0, 0.0) == mbd.E_INVALID
+    assert L.mbd_conv_outer_rows(None, 0, 0, 0, None, 0, 0) == mbd.E_INVALID
     assert L.mbd_launch_count(None) == -1
     assert L.mbd_net_destroy(None) == mbd.E_INVALID
 
