@@ -361,3 +361,79 @@ def expected_words(dims: Sequence[int], B: int, P_r: int, P_c: int) -> Dict[str,
     """Per-process totals of mbd_comm_words for the stack (Eq. 8)."""
     rows = mbd.comm_words(mbd.fc_layers(dims, bias=False), B, P_r, P_c)
     return {k: sum(r[k] for r in rows) for k in ("allgather_y", "allreduce_dx", "allreduce_dw")}
+
+
+def main(argv=None):
+    """Runs a few steps of a fully connected stack over a P_r x P_c grid of processes (launch with torchrun,
+    one process per grid position) and prints one JSON line from rank 0: time per step (slowest rank), the
+    words each process moved against Eq. 8, and what the alpha-beta model predicts for them.
+
+        python -m torch.distributed.run --nproc-per-node 4 --master-addr 127.0.0.1 \\
+            -m paper_1712_04432_b200.grid_exec --grid 2x2 --dims 1024,1024,512 --batch 256 --backend nccl
+    """
+    import argparse
+    import json
+    import os
+    import time
+
+    import torch
+    import torch.distributed as dist
+
+    from . import inputs as I
+
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--grid", default="2x1", help="P_r x P_c")
+    ap.add_argument("--dims", default="1024,1024,512")
+    ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--eta", type=float, default=0.01)
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"],
+                    help="gloo: collectives through host copies (several processes may then share one GPU)")
+    a = ap.parse_args(argv)
+    P_r, P_c = (int(x) for x in a.grid.lower().split("x"))
+    dims = [int(d) for d in a.dims.split(",")]
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local % torch.cuda.device_count())
+    dist.init_process_group(a.backend)
+    comm = GridComm(P_r, P_c, via_host=a.backend == "gloo")
+    w = I.fc_workload(dims, a.batch, "bf16", "relu_normal")
+    inp = I.make_inputs(w, seed=0)
+
+    def dev(x):
+        return torch.from_numpy(I.bf16_bits(x).view("int16")).cuda().view(torch.bfloat16)
+
+    net = GridFC(dims, a.batch, comm)
+    for i in range(len(dims) - 1):
+        net.set_weights(i, dev(inp.Ws[i]))
+    m = a.batch // P_c
+    X_c = dev(inp.X[comm.c * m:(comm.c + 1) * m])
+    labels_c = torch.from_numpy(inp.labels[comm.c * m:(comm.c + 1) * m]).cuda()
+    net.step(X_c, labels_c, a.eta)                                   # warm-up
+    for k in comm.words:
+        comm.words[k] = 0.0
+    dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    loss = 0.0
+    for _ in range(a.steps):
+        loss = net.step(X_c, labels_c, a.eta)
+    torch.cuda.synchronize()
+    dt = torch.tensor([(time.perf_counter() - t0) / a.steps], dtype=torch.float64)
+    if a.backend == "nccl":
+        dt = dt.cuda()
+    dist.all_reduce(dt, op=dist.ReduceOp.MAX)
+    if dist.get_rank() == 0:
+        layers = mbd.fc_layers(dims, bias=False)
+        model = mbd.comm_time(layers, a.batch, P_r, P_c, mbd.MACHINE_B200_NVLINK5)
+        print(json.dumps({
+            "grid": f"{P_r}x{P_c}", "dims": dims, "batch": a.batch, "backend": a.backend, "steps": a.steps,
+            "ms_per_step": float(dt.item()) * 1e3, "loss_block_0": loss,
+            "words_per_process_per_step": {k: v / a.steps for k, v in comm.words.items()},
+            "eq8_words_per_process": expected_words(dims, a.batch, P_r, P_c),
+            "alpha_beta_seconds_nvlink5": sum(sum(t.values()) for t in model)}), flush=True)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

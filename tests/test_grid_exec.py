@@ -286,3 +286,16 @@ def test_integrated_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, P
             assert rel_fro(z[f"W{i}"], o["new_W"][Lc + i][rows]) < 1e-2, (rank, i)
         assert json.loads(str(z["words"])) == json.loads(str(z["want"]))
     assert abs(loss - o["J"]) < 1e-2 * abs(o["J"])
+
+
+@pytest.mark.gpu
+def test_command_line_driver_prints_words_equal_to_eq8():
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="2")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
+           "--master-port", "29611", "-m", "paper_1712_04432_b200.grid_exec", "--grid", "2x1", "--dims", "256,128,64",
+           "--batch", "32", "--steps", "2", "--backend", "gloo"]
+    r = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, (r.stdout[-1500:], r.stderr[-3000:])
+    d = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
+    assert {k: int(round(v)) for k, v in d["words_per_process_per_step"].items()} == d["eq8_words_per_process"]
+    assert d["ms_per_step"] > 0 and d["alpha_beta_seconds_nvlink5"] > 0
