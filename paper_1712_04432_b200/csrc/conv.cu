@@ -1071,29 +1071,27 @@ mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta) {
   if (i < 0 || i >= c->L) return MBD_E_INVALID;
   const bool fused = fused_eta > 0.f;
   const float scale = -fused_eta / static_cast<float>(c->B);
-  {
-    if (i > 0) {
-      // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0]
-      // (the producer of dY_i has stored its boundary rows into the neighbours' halo rows)
-      launch_fwd(c, MBD_K_CONV_BWD_DATA, i, c->dY_fwd[i], c->wb_map[i], c->dY[i - 1], c->dY_tile[i - 1], MODE_MASK,
-                 c->relu[i - 1] ? c->act[i] : nullptr, c->relu[i - 1] ? &c->act_tile[i] : nullptr);
-    }
-    WgParams p;
-    p.W = c->W; p.Hs = c->Hs; p.R = c->R;
-    p.nseg = (c->W + WG_PIX - 1) / WG_PIX;
-    p.pack = c->pack;
-    p.rows_total = ((c->Z + c->pack - 1) / c->pack) * p.nseg * c->Hs;
-    p.part = c->wpart; p.status = c->status;
-    const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
-    c->prof->begin(MBD_K_CONV_BWD_WEIGHT, 2.0 * c->B * c->H * c->W * (c->k1[i] ? 1.0 : 9.0) * C * C);
-    launch_pdl(conv_wgrad_kernel, dim3(grid), dim3(NUM_THREADS), WG_SMEM, c->stream, 1, c->act_fwd[i], c->dY_wg[i], p);
-    c->prof->end();
-    c->prof->begin(MBD_K_REDUCE, (grid + 1.0) * 9 * C * C * 4.0);
-    wgrad_finish_kernel<<<9 * C * C / 64, 256, 0, c->stream>>>(c->wpart, grid, fused ? nullptr : c->dK[i],
-                                                                      fused ? c->K[i] : nullptr, c->Wf[i], c->Wb[i],
-                                                                      c->K32.empty() ? nullptr : c->K32[i], scale, c->k1[i]);
-    c->prof->end();
+  if (i > 0) {
+    // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0]
+    // (the producer of dY_i has stored its boundary rows into the neighbours' halo rows)
+    launch_fwd(c, MBD_K_CONV_BWD_DATA, i, c->dY_fwd[i], c->wb_map[i], c->dY[i - 1], c->dY_tile[i - 1], MODE_MASK,
+               c->relu[i - 1] ? c->act[i] : nullptr, c->relu[i - 1] ? &c->act_tile[i] : nullptr);
   }
+  WgParams p;
+  p.W = c->W; p.Hs = c->Hs; p.R = c->R;
+  p.nseg = (c->W + WG_PIX - 1) / WG_PIX;
+  p.pack = c->pack;
+  p.rows_total = ((c->Z + c->pack - 1) / c->pack) * p.nseg * c->Hs;
+  p.part = c->wpart; p.status = c->status;
+  const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
+  c->prof->begin(MBD_K_CONV_BWD_WEIGHT, 2.0 * c->B * c->H * c->W * (c->k1[i] ? 1.0 : 9.0) * C * C);
+  launch_pdl(conv_wgrad_kernel, dim3(grid), dim3(NUM_THREADS), WG_SMEM, c->stream, 1, c->act_fwd[i], c->dY_wg[i], p);
+  c->prof->end();
+  c->prof->begin(MBD_K_REDUCE, (grid + 1.0) * 9 * C * C * 4.0);
+  wgrad_finish_kernel<<<9 * C * C / 64, 256, 0, c->stream>>>(c->wpart, grid, fused ? nullptr : c->dK[i],
+                                                                    fused ? c->K[i] : nullptr, c->Wf[i], c->Wb[i],
+                                                                    c->K32.empty() ? nullptr : c->K32[i], scale, c->k1[i]);
+  c->prof->end();
   if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
   if (i == 0) c->state = fused ? 3 : 2;
   return MBD_OK;
