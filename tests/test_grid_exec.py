@@ -14,6 +14,7 @@ import numpy as np
 import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+_PORTS = iter(range(29541, 29700))          # a fresh rendezvous port for every launch
 
 COMM_WORKER = r'''
 import json, sys
@@ -100,7 +101,7 @@ def _torchrun(script, nproc, port, timeout=600):
 def test_groups_placement_sums_and_word_counts(tmp_path, P_r, P_c):
     script = tmp_path / "comm_worker.py"
     script.write_text(COMM_WORKER % {"root": ROOT, "P_r": P_r, "P_c": P_c, "dims": [64, 32, 48, 16], "B": 12})
-    r = _torchrun(script, P_r * P_c, 29541 + P_r)
+    r = _torchrun(script, P_r * P_c, next(_PORTS))
     assert r.returncode == 0, r.stderr[-3000:]
     d = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
     assert d["ok"], d
@@ -116,7 +117,7 @@ def test_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, P_r, P_c):
     script = tmp_path / "step_worker.py"
     script.write_text(STEP_WORKER % {"root": ROOT, "P_r": P_r, "P_c": P_c, "dims": dims, "B": B, "eta": eta,
                                      "out": str(tmp_path), "seed": seed})
-    r = _torchrun(script, P_r * P_c, 29551 + P_r + 2 * P_c)
+    r = _torchrun(script, P_r * P_c, next(_PORTS))
     assert r.returncode == 0, (r.stdout[-1500:], r.stderr[-3000:])
 
     w = I.fc_workload(dims, B, "bf16", "relu_normal")
@@ -188,7 +189,7 @@ def test_convolution_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, 
     script = tmp_path / "conv_worker.py"
     script.write_text(CONV_WORKER % {"root": ROOT, "P_r": P_r, "P_c": P_c, "ksizes": list(ksizes), "H": H, "W": W, "B": B,
                                      "eta": eta, "out": str(tmp_path), "seed": seed})
-    r = _torchrun(script, P_r * P_c, 29571 + P_r + 2 * P_c)
+    r = _torchrun(script, P_r * P_c, next(_PORTS))
     assert r.returncode == 0, (r.stdout[-1500:], r.stderr[-3000:])
 
     w = I.conv_workload(64, H, W, B, n_layers=len(ksizes), ksizes=ksizes)
@@ -260,7 +261,7 @@ def test_integrated_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, P
     script = tmp_path / "mixed_worker.py"
     script.write_text(MIXED_WORKER % {"root": ROOT, "P_r": P_r, "P_c": P_c, "ksizes": list(ksizes), "H": H, "W": W, "fc": fc,
                                       "B": B, "eta": eta, "out": str(tmp_path), "seed": seed})
-    r = _torchrun(script, P_r * P_c, 29591 + P_r + 2 * P_c)
+    r = _torchrun(script, P_r * P_c, next(_PORTS))
     assert r.returncode == 0, (r.stdout[-1500:], r.stderr[-3000:])
 
     w = I.mixed_workload(64, H, W, len(ksizes), fc, B, ksizes=ksizes)
@@ -292,7 +293,7 @@ def test_integrated_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, P
 def test_command_line_driver_prints_words_equal_to_eq8():
     env = dict(os.environ, MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="2")
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
-           "--master-port", "29611", "-m", "paper_1712_04432_b200.grid_exec", "--grid", "2x1", "--dims", "256,128,64",
+           "--master-port", str(next(_PORTS)), "-m", "paper_1712_04432_b200.grid_exec", "--grid", "2x1", "--dims", "256,128,64",
            "--batch", "32", "--steps", "2", "--backend", "gloo"]
     r = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, (r.stdout[-1500:], r.stderr[-3000:])
