@@ -427,7 +427,9 @@ def run_ours(args):
                 frac_of_burst_peak=flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"] if bf else None,
                 kernels=kernels, dominant_kernel_class=dom, loss_last=loss_last,
                 launch_mode="CUDA graph replay (mbd_train_step)" if use_graph else "direct launches",
-                ms_per_step_direct=prof_ms if use_graph else None)
+                ms_per_step_direct=prof_ms if use_graph else None,
+                ms_per_step_median=float(np.median(per_step)), ms_per_step_min=float(min(per_step)),
+                ms_per_step_max=float(max(per_step)))
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
