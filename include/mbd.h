@@ -249,9 +249,11 @@ MBD_API mbd_status mbd_choose_grid(const mbd_layer* layers_host, int L, int64_t 
 /* Copy an internal tensor to dst_dev; `bytes` must equal the tensor's size. */
 MBD_API mbd_status mbd_get_tensor(mbd_net* net, int which, int layer, void* dst_dev, size_t bytes);
 
-/* Overwrite an internal tensor (MBD_T_ACT or MBD_T_DY) from src_dev, same shapes and types
- * as mbd_get_tensor.  A test hook: writing the stored activations between mbd_forward and
- * mbd_backward fixes the ReLU decisions [X_{i+1} > 0] the backward pass will take. */
+/* Overwrite an internal tensor (MBD_T_ACT or MBD_T_DY; MBD_T_DW on a convolution stack) from
+ * src_dev, same shapes and types as mbd_get_tensor.  Writing the stored activations between
+ * mbd_forward and mbd_backward fixes the ReLU decisions [X_{i+1} > 0] the backward pass will take
+ * (the parity tests do); MBD_T_DY of the last layer is how a MBD_LOSS_NONE stack receives its top
+ * gradient; MBD_T_DW is how a multi-process driver puts back a summed weight gradient. */
 MBD_API mbd_status mbd_set_tensor(mbd_net* net, int which, int layer, const void* src_dev, size_t bytes);
 
 /* Waits for the stream and reads the device status word: MBD_OK, or MBD_E_TIMEOUT if
