@@ -158,3 +158,52 @@ def test_one_by_one_layers(ksizes, P_r, fused):
     g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o))
     assert [a.shape[-1] for a in g["new_W"]] == list(ksizes)
     compare_conv_step(g, o, TOL, fused)
+
+
+def test_step_piece_by_piece_equals_the_whole_step():
+    """mbd_forward / mbd_backward are the stepped calls in a row: same loss and, bit for bit, the same updated
+    kernels; and halo rows written from outside are what the next layer reads (a strip cut out of a taller image
+    gives the rows the whole image gives)."""
+    import torch
+    from paper_1712_04432_b200 import mbd
+    from tests.helpers import to_dev, to_np
+    w = I.conv_workload(64, 12, 40, 3, name="conv_steps")
+    inp = I.make_inputs(w, seed=62)
+    X = to_dev(inp.X, True)
+    res = []
+    for stepped in (False, True):
+        net = mbd.Net(mbd.conv_layers(2, 64, 12, 40), w.B, 3, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+        for i in range(2):
+            net.set_weights(i, to_dev(inp.Ws[i], True))
+        J = torch.zeros(1, dtype=torch.float32, device="cuda")
+        if stepped:
+            net.conv_stage_input(X)
+            net.conv_forward_layer(0)
+            net.conv_forward_layer(1, J)
+            net.conv_backward_layer(1, 1e-5)
+            net.conv_backward_layer(0, 1e-5)
+        else:
+            net.forward(X, None, J)
+            net.backward(1e-5)
+        net.poll()
+        res.append((float(J.item()), [net.get_weights(i).clone() for i in range(2)], net.get_tensor(mbd.T_ACT, 0).clone()))
+        net.close()
+    assert res[0][0] == res[1][0]
+    for a, b in zip(res[0][1], res[1][1]):
+        assert torch.equal(a, b)
+    # rows 4..7 of the 12-row images as a network of their own, with rows 3 and 8 supplied as halo rows
+    sub = mbd.Net(mbd.conv_layers(1, 64, 4, 40), w.B, 1, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+    sub.set_weights(0, to_dev(inp.Ws[0], True))
+    sub.conv_stage_input(X[:, :, 4:8, :].contiguous())
+    nhwc = X.permute(0, 2, 3, 1).contiguous()                                  # [B, H, W, C]
+    sub.conv_outer_rows(mbd.T_ACT, -1, 0, rows=nhwc[:, 3].contiguous())
+    sub.conv_outer_rows(mbd.T_ACT, -1, 1, rows=nhwc[:, 8].contiguous())
+    assert torch.equal(sub.conv_outer_rows(mbd.T_ACT, -1, 0), nhwc[:, 4].contiguous())   # first own row read back
+    sub.conv_forward_layer(0)
+    sub.poll()
+    y_sub = to_np(sub.get_tensor(mbd.T_ACT, 0))                                # raw output of the last layer
+    ref = inp.Ws[0].astype(np.float64)
+    from oracle import mbd_oracle as O
+    y_ref = O.conv3x3(ref, inp.X.astype(np.float64))[:, :, 4:8, :]
+    assert rel_fro(y_sub, y_ref) < TOL
+    sub.close()
