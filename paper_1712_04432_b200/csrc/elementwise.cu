@@ -245,7 +245,7 @@ sum_f32_kernel(const float* __restrict__ x, int64_t n, float scale, float* __res
 // Stage 1: grid (ceil(N/256), row_splits); 256 threads = 8 warps; a lane owns 8 consecutive
 // columns (one 16-byte load per row for bf16), a warp 256 columns, the 8 warps stride over the
 // rows of this split.  Every warp stores its own partial row, scratch[(split * 8 + warp)][N];
-// stage 2 adds the 8 * row_splits rows in order.  No shared memory: the CTAs fit on an SM next
+// stage 2 adds the 8 * row_splits rows in a fixed order.  No shared memory: the CTAs fit on an SM next
 // to a resident tensor-core GEMM CTA, so the kernel can run on the side stream under a product.
 template <bool BF16>
 __global__ void __launch_bounds__(256)
@@ -287,24 +287,36 @@ colsum_stage1(const void* __restrict__ dY, int64_t M, int64_t N, int row_splits,
     if (n0 + i < N) dst[i] = a[i];
 }
 
+// Stage 2: a warp owns 4 columns; the partial rows of a column are shared out over 8 lanes (contiguous row
+// ranges, each added in row order with eight loads in flight) and the 8 sub-sums are gathered by shuffles and
+// added in lane order: a fixed order, a chain of rows / 64 dependent iterations instead of rows / 8, and still
+// no shared memory (see stage 1).
 __global__ void __launch_bounds__(256)
-colsum_stage2(const float* __restrict__ scratch, int row_splits, int64_t N, float* __restrict__ db,
+colsum_stage2(const float* __restrict__ scratch, int rows, int64_t N, float* __restrict__ db,
               float* __restrict__ bias, float scale) {
   pdl_wait();                            // everything this kernel reads or overwrites comes from earlier kernels
-  const int64_t n = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
-  if (n >= N) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int col = lane & 3, grp = lane >> 2;
+  const int64_t n = (blockIdx.x * 8ll + warp) * 4 + col;
+  const int r0 = (grp * rows) / 8, r1 = ((grp + 1) * rows) / 8;
   float s = 0.f;
-  int r = 0;
-  for (; r + 8 <= row_splits; r += 8) {        // eight loads in flight, added in row order
-    float v[8];
+  if (n < N) {
+    int r = r0;
+    for (; r + 8 <= r1; r += 8) {
+      float v[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) v[j] = scratch[static_cast<int64_t>(r + j) * N + n];
+      for (int j = 0; j < 8; ++j) v[j] = scratch[static_cast<int64_t>(r + j) * N + n];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) s += v[j];
+      for (int j = 0; j < 8; ++j) s += v[j];
+    }
+    for (; r < r1; ++r) s += scratch[static_cast<int64_t>(r) * N + n];
   }
-  for (; r < row_splits; ++r) s += scratch[static_cast<int64_t>(r) * N + n];
-  if (db) db[n] = s;
-  if (bias) bias[n] = fmaf(scale, s, bias[n]);
+  float total = 0.f;
+#pragma unroll
+  for (int g = 0; g < 8; ++g) total += __shfl_sync(0xffffffffu, s, g * 4 + col);   // ascending group order
+  if (grp != 0 || n >= N) return;
+  if (db) db[n] = total;
+  if (bias) bias[n] = fmaf(scale, total, bias[n]);
 }
 
 // ------------------------------------------------------------------ SGD update (Eq. 1)
@@ -431,7 +443,7 @@ cudaError_t colsum_launch(const void* dY, int dy_bf16, int64_t M, int64_t N, flo
   cudaError_t e = dy_bf16 ? launch_pdl(colsum_stage1<true>, g1, dim3(256), 0, stream, 0, dY, M, N, row_splits, scratch)
                           : launch_pdl(colsum_stage1<false>, g1, dim3(256), 0, stream, 0, dY, M, N, row_splits, scratch);
   if (e != cudaSuccess) return e;
-  return launch_pdl(colsum_stage2, dim3(static_cast<unsigned>((N + 255) / 256)), dim3(256), 0, stream, 0, static_cast<const float*>(scratch),
+  return launch_pdl(colsum_stage2, dim3(static_cast<unsigned>((N + 31) / 32)), dim3(256), 0, stream, 0, static_cast<const float*>(scratch),
                     row_splits * 8, N, db, bias, scale);
 }
 
