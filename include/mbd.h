@@ -13,12 +13,15 @@
  * (the paper's all-reduces) are taken on the device: consecutive logical
  * blocks are either chained in the tensor-memory accumulator or written as
  * fp32 partials and added, in ascending block order, by a reduction kernel.
+ * The last part of this file holds the calls a multi-process driver needs to
+ * run the same grid with one process per position (block operations, the
+ * convolution step piece by piece).
  *
  * Conventions
  *   - Every pointer named *_dev is DEVICE memory, every *_host is HOST memory.
  *   - Activations are [B, d] row-major (row = sample = one column of the
  *     paper's X_i); weights are [d_i, d_{i-1}] row-major; convolution input is
- *     NCHW, its kernel [C_out, C_in, 3, 3].
+ *     NCHW, its kernel [C_out, C_in, 3, 3] (or [C_out, C_in, 1, 1]).
  *   - dtype MBD_BF16: X, W, activations and dY are bfloat16 bit patterns,
  *     accumulation, logits, loss, partials, dW, biases are float.
  *     dtype MBD_F32: everything float (no tensor cores; the <=1e-5 check mode).
@@ -26,8 +29,9 @@
  *     column sums use a side stream of the library that is forked from and joined
  *     back into that stream inside mbd_backward; the pipelined host step copies
  *     its batches on a copy stream of the library); nothing synchronises except
- *     mbd_poll_status, mbd_train_step_host, mbd_train_step_host_end and creation /
- *     destruction.  The library owns weights, activations, gradients and
+ *     mbd_poll_status, mbd_train_step_host, mbd_train_step_host_end, creation /
+ *     destruction, and the stand-alone calls that say so (mbd_gemm_bf16*, the block
+ *     operations in their synchronous form).  The library owns weights, activations, gradients and
  *     workspace; the caller owns every buffer it passes in.
  *   - Errors are return codes; nothing aborts, throws or traps.
  */
