@@ -110,11 +110,19 @@ enum {
 
 /* Section 2.3 / 2.4.  Builds the plan for an L-layer network on batch B over a
  * logical P_r x P_c grid and allocates all device state (weights start at zero).
- *   max_partials  how many fp32 partial sums a reduction over P blocks may
- *                 materialise: S = min(P, max_partials) partials, each chaining
+ *   max_partials  how many separate fp32 partial sums a reduction over P blocks is
+ *                 formed from: S = min(P, max_partials) partials, each chaining
  *                 P/S consecutive logical blocks in the accumulator; 0 selects
- *                 the default (4); 1 never materialises; >= P materialises every
- *                 block's partial exactly as the paper's processes would hold it.
+ *                 the default (4); 1 never leaves the accumulator; >= P keeps every
+ *                 block's partial as a plane of its own, exactly as the paper's
+ *                 processes would hold it, and a reduction kernel adds the planes.
+ *                 With 1 < S < P the partials are intermediate: they are either
+ *                 written as S planes and reduced the same way, or (two pieces, or
+ *                 more output tiles than SMs) added as a running sum inside the
+ *                 product -- the CTA that finishes piece s of a tile adds it to the
+ *                 sum of pieces 0..s-1 that the CTA before it left in one fp32 plane
+ *                 and the last one applies the tail operation.  Both forms add in
+ *                 ascending block order and give bit-identical results.
  *   cuda_stream   a cudaStream_t (may be NULL for the default stream).
  * Layer order (Section 2.4, Eq. 9): domain-split convolutions first (L_D), model-split
  * fully connected layers after them (L_M); either group may be empty.  With both present
@@ -283,6 +291,19 @@ MBD_API mbd_status mbd_profile_read(mbd_net* net, int kclass, double* ms_total, 
 /* Kernels launched by this network since creation (host counter). */
 MBD_API int64_t mbd_launch_count(const mbd_net* net);
 
+/* How one of the three products of Section 1 is launched for fully connected layer `layer` (public
+ * index) of a bf16 network: product 0 = forward, 1 = backward-data, 2 = backward-weight.  Lets a test
+ * or a benchmark state which kernel variant it ran.  tile_m x tile_n is the output tile of one work
+ * unit (of the CTA pair when cta_pair != 0); k_pieces the number of fp32 partial sums the K range is
+ * cut into (the grid's S = min(P, max_partials) times any further cut the planner added); running_sum != 0:
+ * the pieces are added inside the product's own epilogue (see max_partials of mbd_net_create), otherwise
+ * k_pieces > 1 means a reduce_partials launch follows; tma_epilogue != 0: the tail operation the plan was made for (bias +
+ * ReLU, ReLU mask, fused update) moves its global data by TMA; ctas: CTAs launched.
+ * MBD_E_UNSUPPORTED for fp32 networks and convolution layers, MBD_E_INVALID for a product the layer
+ * does not have (backward-data of the network's first layer). */
+typedef struct { int32_t tile_m, tile_n, cta_pair, k_pieces, tma_epilogue, ctas, running_sum, reserved; } mbd_plan;
+MBD_API mbd_status mbd_get_plan(const mbd_net* net, int layer, int product, mbd_plan* out_host);
+
 /* Stand-alone dense contraction on the tensor cores, used by the unit tests:
  *   variant 0 (forward)          D[M,N] = A[M,K]   * B[N,K]^T   A, B row-major, K contiguous
  *   variant 1 (backward-data)    D[M,N] = A[M,K]   * B[K,N]     B row-major, N contiguous
@@ -290,7 +311,8 @@ MBD_API int64_t mbd_launch_count(const mbd_net* net);
  * bf16 inputs, fp32 accumulation.  The K range is cut into k_splits balanced pieces;
  * k_splits == 1 writes D_dev [M,N] float directly, otherwise partials_dev
  * [k_splits][M][N] float receives the pieces and D_dev their sum (ascending order).
- * Leading dimensions are in elements and, like M/N/K offsets, multiples of 8. */
+ * Leading dimensions are in elements and, like M/N/K offsets, multiples of 8; every base pointer is
+ * 16-byte aligned (MBD_E_UNSUPPORTED otherwise: nothing is launched). */
 MBD_API mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, const void* A_dev,
                          int64_t lda, const void* B_dev, int64_t ldb, float* D_dev, int64_t ldd,
                          int k_splits, float* partials_dev, void* cuda_stream);
@@ -309,7 +331,10 @@ MBD_API mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K, c
  *   MBD_TAIL_MASK   out = (mask_dev == NULL || mask_dev[m, n] > 0) ? acc : 0      (ReLU derivative)
  *   MBD_TAIL_SGD    out = out + scale * acc                                          (Eq. 1, scale = -eta/B)
  * out_dev is [M, ldo] bf16 (out_bf16 != 0) or float; mask_dev has out's element type and ldmask.
- * Leading dimensions in elements, multiples of 8 for the contraction (as for mbd_gemm_bf16). */
+ * Leading dimensions in elements, multiples of 8 for the contraction, and its bases (operands, out, mask,
+ * bias) 16-byte aligned (MBD_E_UNSUPPORTED otherwise, nothing is launched).  mbd_block_reduce and
+ * mbd_softmax_xent accept any alignment: they move 16 bytes per access when bases and leading dimensions
+ * allow it and fall back to element-wise kernels otherwise. */
 enum { MBD_TAIL_STORE = 0, MBD_TAIL_MASK = 1, MBD_TAIL_SGD = 2 };
 typedef struct {
   int32_t op, out_bf16, relu, reserved;
@@ -330,7 +355,9 @@ MBD_API mbd_status mbd_block_gemm_bf16(int variant, int64_t M, int64_t N, int64_
 MBD_API mbd_status mbd_block_reduce(const float* parts_dev, int S, int64_t M, int64_t N, const mbd_tail* tail,
                             int sync, void* cuda_stream);
 /* Softmax cross-entropy of float logits [B, d]: per_sample_dev[b] = loss of sample b (natural log),
- * dY_dev [B, d] = softmax - onehot (bf16 if dY_bf16 != 0, else float).  labels_dev: int32 in [0, d). */
+ * dY_dev [B, d] = softmax - onehot (bf16 if dY_bf16 != 0, else float).  labels_dev: int32 in [0, d); a label
+ * outside that range is never used as an index: the sample's loss comes back as NaN and its dY row is the
+ * plain softmax (mbd_forward treats labels the same way). */
 MBD_API mbd_status mbd_softmax_xent(const float* logits_dev, int64_t B, int64_t d, const int32_t* labels_dev,
                             void* dY_dev, int dY_bf16, float* per_sample_dev, int sync, void* cuda_stream);
 
@@ -371,11 +398,14 @@ MBD_API mbd_status mbd_selftest_timeout(int limit_ms, void* cuda_stream);
  * library's device image (present on every GPU that loads the library, until exit) and the
  * call makes no cudaMalloc / cudaFree nor any other allocating call.
  *   - MBD_E_TOO_LARGE if min(k_splits, ceil(K/64)) * M * N exceeds 4 Mi floats (k_splits > 1).
- *   - The first call on each device looks up the array's device address (that device must be
- *     current, as for every call); make that first call before starting any stream capture.
+ *   - The first call on each device looks up the array's device address and opts the kernels into
+ *     their shared-memory size on that device (the device must be current, as for every call); make
+ *     that first call before starting any stream capture.
  *   - All calls on a device share the one array, which keeps the previous call's contents; the
  *     entry clears what has to start at zero.  Calls whose GPU work overlaps -- different
- *     streams or threads -- race on it: serialise them.  The call returns after its work is done. */
+ *     streams or threads -- race on it: serialise them.  The call waits for cuda_stream (it reads the
+ *     status word back) and returns after its work is done.
+ *   - Bases 16-byte aligned, leading dimensions multiples of 8 (MBD_E_UNSUPPORTED otherwise). */
 MBD_API mbd_status mbd_gemm_bf16_noalloc(int variant, int64_t M, int64_t N, int64_t K, const void* A_dev,
                                  int64_t lda, const void* B_dev, int64_t ldb, float* D_dev, int64_t ldd,
                                  int k_splits, void* cuda_stream);

@@ -28,6 +28,8 @@ bool to_epi(const mbd_tail* t, Epi* e) {
   return true;
 }
 
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
 struct StatusWord {
   int* dev = nullptr;
   bool alloc(cudaStream_t s) {
@@ -54,6 +56,8 @@ extern "C" mbd_status mbd_block_gemm_bf16(int variant, int64_t M, int64_t N, int
   Epi epi;
   if (!A || !Bm || variant < 0 || variant > 2 || M < 1 || N < 1 || K < 1 || !to_epi(tail, &epi)) return MBD_E_INVALID;
   if (lda % 8 || ldb % 8 || epi.ldo % 8 || N % 8 || (epi.mask && epi.ldmask % 8)) return MBD_E_UNSUPPORTED;
+  // TMA and the 16-byte accesses of the epilogue need 16-byte aligned bases (a view may start anywhere)
+  if (!aligned16(A) || !aligned16(Bm) || !aligned16(epi.out) || !aligned16(epi.mask) || !aligned16(epi.bias)) return MBD_E_UNSUPPORTED;
   if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return MBD_E_UNSUPPORTED;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   int dev = 0, sms = 0;

@@ -136,7 +136,8 @@ softmax_xent_kernel(const float* __restrict__ logits, int64_t d, const int32_t* 
     if (dy_bf16) reinterpret_cast<__nv_bfloat16*>(dY)[b * d + k] = __float2bfloat16_rn(g);
     else reinterpret_cast<float*>(dY)[b * d + k] = g;
   }
-  if (tid == 0) per_sample[b] = mx + logf(sum) - row[label];
+  // a label outside [0, d) is never used as an index: the sample's loss is reported as NaN
+  if (tid == 0) per_sample[b] = (label >= 0 && label < d) ? mx + logf(sum) - row[label] : __int_as_float(0x7fc00000);
 }
 
 // Same, with the whole row held in registers (VPT values per thread): one pass over HBM.
@@ -222,7 +223,7 @@ softmax_xent_reg_kernel(const float* __restrict__ logits, int64_t d, const int32
       }
     }
   }
-  if (tid == 0) per_sample[b] = mx + logf(sum) - row[label];
+  if (tid == 0) per_sample[b] = (label >= 0 && label < d) ? mx + logf(sum) - row[label] : __int_as_float(0x7fc00000);
 }
 
 // ------------------------------------------------------------------ fixed-order sum
@@ -386,6 +387,8 @@ widen_bf16_kernel(const __nv_bfloat16* __restrict__ w, float* __restrict__ w32, 
     w32[i] = __bfloat162float(w[i]);
 }
 
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
 int grid_for(int64_t work_items, int num_sms, int per_sm) {
   int64_t blocks = (work_items + 255) / 256;
   const int64_t cap = static_cast<int64_t>(num_sms) * per_sm;
@@ -398,7 +401,10 @@ int grid_for(int64_t work_items, int num_sms, int per_sm) {
 
 cudaError_t reduce_partials_launch(const float* parts, int S, int64_t M, int64_t N, const Epi& epi, int num_sms,
                                    cudaStream_t stream) {
-  const bool vec = (N % 8 == 0) && (epi.ldo % 8 == 0) && (epi.mask == nullptr || epi.ldmask % 8 == 0);
+  // 16-byte accesses need 16-byte aligned bases as well as leading dimensions that are multiples of 8; a
+  // caller's view that starts at an odd offset goes through the element-wise kernel instead
+  const bool vec = (N % 8 == 0) && (epi.ldo % 8 == 0) && (epi.mask == nullptr || epi.ldmask % 8 == 0) &&
+                   aligned16(parts) && aligned16(epi.out) && aligned16(epi.mask) && aligned16(epi.bias) && aligned16(epi.master);
   if (vec) {
     // two planes of at least 8 MB: the two-piece kernel; small or many-plane sums: the plain one
     if (S == 2 && M * N >= (2 << 20))
@@ -411,7 +417,7 @@ cudaError_t reduce_partials_launch(const float* parts, int S, int64_t M, int64_t
 cudaError_t softmax_xent_launch(const float* logits, int64_t B, int64_t d, const int32_t* labels, void* dY,
                                 int dy_bf16, float* per_sample, cudaStream_t stream) {
   const unsigned nb = static_cast<unsigned>(B);
-  const bool vec = d % 4 == 0;
+  const bool vec = d % 4 == 0 && aligned16(logits) && aligned16(dY);
   if (d <= 64) return launch_pdl(softmax_xent_reg_kernel<1, 2, false>, dim3(nb), dim3(32), 0, stream, 0, logits, d, labels, dY, dy_bf16, per_sample);
   if (d <= 1024 && vec) return launch_pdl(softmax_xent_reg_kernel<4, 8, true>, dim3(nb), dim3(128), 0, stream, 0, logits, d, labels, dY, dy_bf16, per_sample);
   if (d <= 1024) return launch_pdl(softmax_xent_reg_kernel<4, 8, false>, dim3(nb), dim3(128), 0, stream, 0, logits, d, labels, dY, dy_bf16, per_sample);

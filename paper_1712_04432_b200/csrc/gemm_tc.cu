@@ -91,6 +91,8 @@ struct Params {
   Epi epi;
   int* status;
   int te;                 // epilogue moves its global data with TMA through shared memory
+  int fix;                // running sum: piece s adds its accumulator to the sum pieces 0..s-1 left in `partials`
+  int* flags;             // fix: one word per (tile, CTA of the pair, 128-row half, epilogue warp); zero between launches
 };
 
 struct Work {
@@ -99,19 +101,63 @@ struct Work {
 
 __device__ __forceinline__ Work decode_work(const Params& p, int w) {
   const int num_tiles = p.tiles_m * p.tiles_n;
-  Work o;
-  o.s = w / num_tiles;
-  const int t = w - o.s * num_tiles;
   const int per_group = p.group_m * p.tiles_n;
-  const int g = t / per_group;
-  const int first_m = g * p.group_m;
-  const int gsize = min(p.tiles_m - first_m, p.group_m);
-  const int r = t - g * per_group;
-  o.tm = first_m + r % gsize;
-  o.tn = r / gsize;
+  Work o;
+  if (p.fix) {
+    // Running sum: the pieces of a raster group follow one another (all tiles of the group for piece 0,
+    // then for piece 1, ...), so that piece s of a tile finds the sum of pieces 0..s-1 still in L2 and
+    // the unit it depends on always has a smaller index than itself.
+    const int span = per_group * p.S;
+    int g = w / span;
+    const int full = p.tiles_m / p.group_m;
+    if (g > full) g = full;                    // the last, shorter group
+    const int first_m = g * p.group_m;
+    const int gsize = min(p.tiles_m - first_m, p.group_m);
+    const int gtiles = gsize * p.tiles_n;
+    int r = w - g * span;
+    o.s = r / gtiles;
+    r -= o.s * gtiles;
+    o.tm = first_m + r % gsize;
+    o.tn = r / gsize;
+  } else {
+    o.s = w / num_tiles;
+    const int t = w - o.s * num_tiles;
+    const int g = t / per_group;
+    const int first_m = g * p.group_m;
+    const int gsize = min(p.tiles_m - first_m, p.group_m);
+    const int r = t - g * per_group;
+    o.tm = first_m + r % gsize;
+    o.tn = r / gsize;
+  }
   o.kb0 = static_cast<int>((static_cast<long long>(o.s) * p.kb_total) / p.S);
   o.kb1 = static_cast<int>((static_cast<long long>(o.s + 1) * p.kb_total) / p.S);
   return o;
+}
+
+// Running-sum hand-over between the pieces of one tile (different CTAs, same launch): the warp that wrote
+// its part of the sum publishes `value` with release semantics; the warp of the next piece that owns the
+// same rows and columns waits for it (bounded, like every wait here) before it reads them.
+__device__ __forceinline__ void flag_publish(int* flag, int value) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
+}
+__device__ __forceinline__ int flag_read(const int* flag) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+  return v;
+}
+static __device__ __noinline__ bool flag_wait(const int* flag, int value, volatile int* abort_flag, int* status) {
+  const unsigned long long t0 = globaltimer_ns();
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (flag_read(flag) == value) return true;
+    if (*abort_flag) return false;
+    if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+      *abort_flag = 1;
+      atomicCAS(status, 0, DEV_TIMEOUT_RUNNING_SUM);
+      return false;
+    }
+    __nanosleep(200);
+  }
 }
 
 // MH = number of 128-row halves of the CTA tile (1: 128 x BN, 2: 256 x BN).  The 256-row tile
@@ -425,11 +471,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int acc = it % ACC_BUFS;
       const uint32_t acc_phase = (it / ACC_BUFS) & 1u;
       const int64_t nbase = static_cast<int64_t>(wk.tn) * BN + half * HC;
-      float* part = p.S > 1 ? p.partials + static_cast<int64_t>(wk.s) * p.M * p.N : nullptr;
+      const bool fix = p.fix != 0;
+      const bool fix_first = wk.s == 0, fix_last = wk.s == p.S - 1;
+      float* part = p.S > 1 ? (fix ? p.partials : p.partials + static_cast<int64_t>(wk.s) * p.M * p.N) : nullptr;
 #pragma unroll 1
       for (int h = 0; h < MH; ++h) {
       const int64_t m = static_cast<int64_t>(wk.tm) * TILE_M + rank * BMT + h * 128 + q * 32 + lane;
       const bool row_ok = m < p.M;
+      int* flag = nullptr;
+      if (fix) flag = p.flags + (((static_cast<int64_t>(wk.tm) * p.tiles_n + wk.tn) * 2 + rank) * 2 + h) * 8 + (warp - 2);
       uint4 pre[NV];
       if (prefetch) {
 #pragma unroll
@@ -444,11 +494,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!ok) break;
         tc_fence_after();
       }
+      if (fix && !fix_first) {                   // the sum of pieces 0..s-1 of these rows and columns is complete
+        if (lane == 0) ok = flag_wait(flag, wk.s, abortp, p.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_COLS + h * BN + half * HC;
 #pragma unroll
       for (int c = 0; c < HC / 32; ++c) {
         uint32_t r[32];
         tc_ld32(taddr + c * 32, r);
+        // running sum of the earlier pieces, requested under the TMEM load; it borrows the registers of the
+        // prefetch array, which an unsplit product uses and a split one does not
+        if (fix && !fix_first && row_ok) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int64_t n = nbase + c * 32 + j * 8;
+            if (n < p.N) {
+              pre[2 * j] = __ldcg(reinterpret_cast<const uint4*>(part + m * p.N + n));
+              pre[2 * j + 1] = __ldcg(reinterpret_cast<const uint4*>(part + m * p.N + n + 4));
+            }
+          }
+        }
         tc_wait_ld();
         if (h == MH - 1 && c == HC / 32 - 1) {     // accumulator fully in registers: hand it back
           tc_fence_before();
@@ -466,7 +533,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               float v[8];
 #pragma unroll
               for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j * 8 + i]);
-              if (part) {
+              if (fix) {
+                if (!fix_first) {                 // ascending order: (sum of the earlier pieces) + this piece
+                  const uint4 r0 = pre[2 * j], r1 = pre[2 * j + 1];
+                  v[0] = __uint_as_float(r0.x) + v[0]; v[1] = __uint_as_float(r0.y) + v[1];
+                  v[2] = __uint_as_float(r0.z) + v[2]; v[3] = __uint_as_float(r0.w) + v[3];
+                  v[4] = __uint_as_float(r1.x) + v[4]; v[5] = __uint_as_float(r1.y) + v[5];
+                  v[6] = __uint_as_float(r1.z) + v[6]; v[7] = __uint_as_float(r1.w) + v[7];
+                }
+                if (!fix_last) {
+                  float* dst = part + m * p.N + n;
+                  __stcg(reinterpret_cast<float4*>(dst), make_float4(v[0], v[1], v[2], v[3]));
+                  __stcg(reinterpret_cast<float4*>(dst + 4), make_float4(v[4], v[5], v[6], v[7]));
+                } else {
+                  epi_apply8(p.epi, m, n, v);
+                }
+              } else if (part) {
                 float* dst = part + m * p.N + n;
                 *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
                 *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
@@ -495,6 +577,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               }
             }
           }
+        }
+      }
+      if (fix) {
+        if (!fix_last) {
+          __threadfence();                       // this lane's part of the sum is visible device-wide ...
+          __syncwarp();
+          if (lane == 0) flag_publish(flag, wk.s + 1);      // ... before the next piece is told so
+        } else if (lane == 0) {
+          *flag = 0;                             // consumed: the word is zero again for the next launch
         }
       }
       }   // h
@@ -532,7 +623,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
-bool g_init_done = false;
+// The opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of each kernel.
+constexpr int MAX_DEVICES = 64;
+bool g_attr_done[MAX_DEVICES] = {false};
 
 // 2-D bf16 tensor map: `inner` contiguous elements per row, `rows` rows `ld` elements apart.
 cudaError_t make_map(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t rows, uint64_t ld,
@@ -573,17 +666,23 @@ cudaError_t launch_t(const TcGemm& g, const Params& p, cudaStream_t stream) {
 }  // namespace
 
 cudaError_t tc_gemm_init() {
-  if (g_init_done) return cudaSuccess;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
-  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  if (g_attr_done[dev]) return cudaSuccess;
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
   if ((e = set_attr<0, 0>()) != cudaSuccess) return e;
   if ((e = set_attr<0, 1>()) != cudaSuccess) return e;
   if ((e = set_attr<1, 1>()) != cudaSuccess) return e;
-  g_init_done = true;
+  g_attr_done[dev] = true;
   return cudaSuccess;
 }
 
@@ -675,6 +774,14 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
   if (!b_mn) e = make_map(&g.tmB, B, g.K, g.N, ldb, BK, g.pair ? g.BN / 2 : g.BN);    // B[N,K]
   else e = make_map(&g.tmB, B, g.N, g.K, ldb, 64, BK);             // B[K,N]
   if (e != cudaSuccess) return e;
+  // Running sum instead of S planes and a reduction launch: when the pieces of a tile are far apart in the
+  // work order (more tiles than CTA slots), or there are just two of them.
+  {
+    const long long tiles = 1ll * tiles_m * tiles_n;
+    const int slots = g.pair ? num_sms / 2 : num_sms;
+    g.fix = g.allow_fix && g.k_splits > 1 && (g.k_splits == 2 || tiles >= slots) ? 1 : 0;
+    g.flag_words = g.fix ? tiles * 32 : 0;
+  }
   // TMA epilogue: bf16 output of an unsplit contraction on 128-row tiles
   g.te = 0;
   g.tmOut = g.tmA;
@@ -702,6 +809,8 @@ cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
   p.group_m = 8;                        // m-tiles per raster group (L2 reuse of the B operand)
   if (const char* ev = getenv("MBD_TC_GROUP_M")) { const int gm = atoi(ev); if (gm >= 1) p.group_m = gm; }
   p.partials = g.partials;
+  p.fix = g.fix && g.flags != nullptr;
+  p.flags = g.flags;
   p.epi = g.epi;
   p.status = g.status;
   p.te = g.te && g.epi.op == g.te_epi.op && g.epi.out == g.te_epi.out && g.epi.out_bf16 && g.epi.mask == g.te_epi.mask &&

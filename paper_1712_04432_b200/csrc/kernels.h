@@ -59,7 +59,8 @@ enum : int {
   DEV_TIMEOUT_MMA_FULL = 102,   // MMA issuer waited too long for operands
   DEV_TIMEOUT_MMA_TMEM = 103,   // MMA issuer waited too long for a drained accumulator
   DEV_TIMEOUT_EPILOGUE = 104,   // epilogue waited too long for a finished accumulator
-  DEV_SMEM_MISALIGNED = 105     // dynamic shared memory did not start on a 1024-byte boundary; nothing ran
+  DEV_SMEM_MISALIGNED = 105,    // dynamic shared memory did not start on a 1024-byte boundary; nothing ran
+  DEV_TIMEOUT_RUNNING_SUM = 106 // epilogue waited too long for the earlier pieces' sum of its tile
 };
 
 // What happens to a finished fp32 accumulator element acc at (m, n).
@@ -97,6 +98,11 @@ struct TcGemm {
   int MH;               // CTA tile height in units of 128 rows: 1 or 2
   int pair;             // two CTAs of a cluster share one 256 x 256 tile (cta_group::2)
   int allow_extra_split; // the planner may cut K further than asked (its pieces go through the same reduction)
+  int allow_fix;        // in: the S pieces need not be kept as S planes
+  int fix;              // out: pieces are added as a running sum in the epilogue (one plane in `partials`, words in
+                        // `flags`), in ascending order like the reduction kernel; no reduction launch follows
+  long long flag_words; // out: ints `flags` must hold (zero-initialised; the kernel leaves them zero)
+  int* flags;
   int M, N, K;
   int k_splits;         // S >= 1; S > 1 writes partials[S][M][N] (fp32) and skips the epilogue op
   float* partials;
@@ -112,7 +118,7 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
                             int num_sms, const Epi* te_epi);
 cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream);
 cudaError_t selftest_timeout_launch(int* status, int limit_ms, cudaStream_t stream);
-cudaError_t tc_gemm_init();   // driver entry point lookup + kernel attributes; idempotent
+cudaError_t tc_gemm_init();   // driver entry point lookup + kernel attributes of the current device; idempotent per device
 
 // ---- fp32 SIMT GEMM (check mode) ----------------------------------------------
 struct SimtGemm {

@@ -55,6 +55,7 @@ struct mbd_net {
   float* partials = nullptr;
   size_t partial_elems = 0;
   float* colsum_scratch = nullptr;
+  float* colsum_scratch_aux = nullptr;   // the side stream's own: sums on the two streams are not ordered
   // The bias gradients (column sums of dY_i) are small and independent of the contractions of
   // their layer: they run on a side stream, forked after dY_i exists and joined at the end of
   // the backward pass, next to the persistent GEMM CTAs (the column-sum kernels use no shared
@@ -73,6 +74,11 @@ struct mbd_net {
   std::vector<cudaEvent_t> ev_dx;           // per layer: dY_i final and W_i no longer read
   cudaEvent_t ev_wjoin = nullptr;
   float* partials_dw = nullptr;             // partials of the backward-weight products when they run beside the others
+  // Running sums (a product's pieces added in its own epilogue instead of a reduction launch) hand over
+  // through one word per (tile, epilogue warp); products that can run at the same time have words of their own.
+  int* fix_flags = nullptr;
+  int* fix_flags_dw = nullptr;
+  size_t fix_words = 0, fix_words_dw = 0;
   size_t last_dw_elems = 0;
   bool last_red_dw = false;                 // the last reduction executed used partials_dw
   cudaEvent_t ev_loss = nullptr;            // forward done -> the sum of the per-sample losses may start
@@ -159,10 +165,11 @@ mbd_status run_gemm(mbd_net* n, TcGemm& tc, int variant, int64_t M, int64_t N, i
   if (n->dtype == MBD_BF16) {
     tc.epi = epi;
     tc.partials = parts;
+    tc.flags = own_parts ? n->fix_flags_dw : n->fix_flags;
     n->prof.begin(MBD_K_GEMM_FWD + variant, flops, stream);
     CK(tc_gemm_launch(tc, stream));
     n->prof.end();
-    S = tc.k_splits;
+    S = tc.fix ? 1 : tc.k_splits;          // a running sum leaves nothing to reduce
   } else {
     SimtGemm g{};
     g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
@@ -199,6 +206,11 @@ mbd_status prepare_tc(mbd_net* n, TcGemm& g, int variant, int64_t M, int64_t N, 
   g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
   g.k_splits = S;
   g.allow_extra_split = variant != 2;     // forward and backward-data: small outputs, cheap partials
+  // max_partials >= P asks for every process's partial as a plane of its own (Appendix A.2 as the paper's
+  // processes hold it); otherwise the pieces are intermediate and may be folded into a running sum
+  const int P = variant == 1 ? n->P_r : variant == 2 ? n->P_c : 1;
+  static const bool no_fix = getenv("MBD_NO_FIXUP") != nullptr;      // tuning knob: always S planes + reduction launch
+  g.allow_fix = !no_fix && (P == 1 || S < P);
   g.status = n->status;
   CK(tc_gemm_prepare(g, A, lda, Bm, ldb, n->num_sms, te_epi));
   return MBD_OK;
@@ -239,7 +251,7 @@ void free_net(mbd_net* n) {
   for (Layer& l : n->layers) {
     cudaFree(l.W); cudaFree(l.bias); cudaFree(l.dW); cudaFree(l.db); cudaFree(l.act); cudaFree(l.dY); cudaFree(l.W32);
   }
-  cudaFree(n->partials); cudaFree(n->colsum_scratch); cudaFree(n->per_sample); cudaFree(n->loss_dev);
+  cudaFree(n->partials); cudaFree(n->colsum_scratch); cudaFree(n->colsum_scratch_aux); cudaFree(n->per_sample); cudaFree(n->loss_dev);
   cudaFree(n->status); cudaFree(n->X_stage); cudaFree(n->labels_stage); cudaFree(n->X_fc); cudaFree(n->dX_fc);
   for (int k = 0; k < 2; ++k) {
     cudaFree(n->X_in[k]); cudaFree(n->labels_in[k]);
@@ -257,7 +269,7 @@ void free_net(mbd_net* n) {
   for (cudaEvent_t e : n->ev_dx) if (e) cudaEventDestroy(e);
   if (n->ev_wjoin) cudaEventDestroy(n->ev_wjoin);
   if (n->wstream) cudaStreamDestroy(n->wstream);
-  cudaFree(n->partials_dw);
+  cudaFree(n->partials_dw); cudaFree(n->fix_flags); cudaFree(n->fix_flags_dw);
   if (n->aux) cudaStreamDestroy(n->aux);
   n->prof.destroy();
   (void)cudaGetLastError();
@@ -390,9 +402,12 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
       }
       if (st == MBD_OK) st = prepare_tc(n, l.bwd_weight, 2, l.d_out, l.d_in, B, l.dY, l.d_out, x_in, l.d_in, S_c, &ew);
       if (st != MBD_OK) { free_net(n); return st; }
-      if (l.fwd.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.fwd.k_splits) * B * l.d_out);
-      if ((i > 0 || mixed) && l.bwd_data.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.bwd_data.k_splits) * B * l.d_in);
-      if (l.bwd_weight.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(l.bwd_weight.k_splits) * l.nW);
+      auto planes = [](const TcGemm& g) { return static_cast<size_t>(g.fix ? 1 : g.k_splits); };
+      if (l.fwd.k_splits > 1) part_elems = std::max(part_elems, planes(l.fwd) * B * l.d_out);
+      if ((i > 0 || mixed) && l.bwd_data.k_splits > 1) part_elems = std::max(part_elems, planes(l.bwd_data) * B * l.d_in);
+      if (l.bwd_weight.k_splits > 1) part_elems = std::max(part_elems, planes(l.bwd_weight) * l.nW);
+      n->fix_words = std::max(n->fix_words, static_cast<size_t>(std::max(l.fwd.flag_words, l.bwd_weight.flag_words)));
+      if (i > 0 || mixed) n->fix_words = std::max(n->fix_words, static_cast<size_t>(l.bwd_data.flag_words));
     }
   }
   n->partial_elems = part_elems;
@@ -405,13 +420,23 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
     for (int i = 0; i < L && small; ++i) {
       const Layer& l = n->layers[i];
       if (2.0 * static_cast<double>(l.nW) * static_cast<double>(B) > 2e11) small = false;
-      if (l.bwd_weight.k_splits > 1) dw_elems = std::max(dw_elems, static_cast<size_t>(l.bwd_weight.k_splits) * l.nW);
+      if (l.bwd_weight.k_splits > 1) dw_elems = std::max(dw_elems, static_cast<size_t>(l.bwd_weight.fix ? 1 : l.bwd_weight.k_splits) * l.nW);
+      n->fix_words_dw = std::max(n->fix_words_dw, static_cast<size_t>(l.bwd_weight.flag_words));
     }
     n->overlap_dw = small;
     if (small && dw_elems) ALLOC(n->partials_dw, dw_elems * sizeof(float));
     n->last_dw_elems = dw_elems;
+    if (n->fix_words) {
+      ALLOC(n->fix_flags, n->fix_words * sizeof(int));
+      if (cudaMemsetAsync(n->fix_flags, 0, n->fix_words * sizeof(int), n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
+    }
+    if (small && n->fix_words_dw) {
+      ALLOC(n->fix_flags_dw, n->fix_words_dw * sizeof(int));
+      if (cudaMemsetAsync(n->fix_flags_dw, 0, n->fix_words_dw * sizeof(int), n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
+    }
   }
   ALLOC(n->colsum_scratch, static_cast<size_t>(8 * 32) * max_d * sizeof(float));
+  ALLOC(n->colsum_scratch_aux, static_cast<size_t>(8 * 32) * max_d * sizeof(float));
   ALLOC(n->per_sample, B * sizeof(float));
 #undef ALLOC
   {
@@ -560,7 +585,7 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
         forked = true;
       }
       n->prof.begin(MBD_K_COLSUM, static_cast<double>(n->B) * l.d_out * (bf ? 2.0 : 4.0), cs);
-      CK(colsum_launch(l.dY, bf, n->B, l.d_out, n->colsum_scratch, colsum_row_splits(n->B, l.d_out, n->num_sms), fused ? nullptr : l.db,
+      CK(colsum_launch(l.dY, bf, n->B, l.d_out, cs == n->aux ? n->colsum_scratch_aux : n->colsum_scratch, colsum_row_splits(n->B, l.d_out, n->num_sms), fused ? nullptr : l.db,
                        fused ? l.bias : nullptr, scale, cs));
       n->prof.end();
       n->prof.total_launches += colsum_launches(n->B, l.d_out, n->num_sms) - 1;
@@ -869,12 +894,34 @@ extern "C" mbd_status mbd_poll_status(mbd_net* n) {
   CK(cudaMemcpy(&h, n->status, sizeof(int), cudaMemcpyDeviceToHost));
   if (h != 0) {
     CK(cudaMemset(n->status, 0, sizeof(int)));
+    // a kernel that gave up may have left hand-over words of a running sum behind
+    if (n->fix_flags) CK(cudaMemset(n->fix_flags, 0, n->fix_words * sizeof(int)));
+    if (n->fix_flags_dw) CK(cudaMemset(n->fix_flags_dw, 0, n->fix_words_dw * sizeof(int)));
     return h == DEV_SMEM_MISALIGNED ? MBD_E_CUDA : MBD_E_TIMEOUT;
   }
   return MBD_OK;
 }
 
 extern "C" int64_t mbd_launch_count(const mbd_net* n) { return n ? n->prof.total_launches : -1; }
+
+extern "C" mbd_status mbd_get_plan(const mbd_net* n, int layer, int product, mbd_plan* out) {
+  if (!n || !out || product < 0 || product > 2) return MBD_E_INVALID;
+  if (layer < 0 || layer >= n->Lc + n->L) return MBD_E_INVALID;
+  if (n->dtype != MBD_BF16 || layer < n->Lc) return MBD_E_UNSUPPORTED;
+  const int i = layer - n->Lc;
+  if (product == 1 && i == 0 && !n->mixed) return MBD_E_INVALID;
+  const Layer& l = n->layers[i];
+  const TcGemm& g = product == 0 ? l.fwd : product == 1 ? l.bwd_data : l.bwd_weight;
+  out->tile_m = 128 * g.MH * (g.pair ? 2 : 1);
+  out->tile_n = g.BN;
+  out->cta_pair = g.pair;
+  out->k_pieces = g.k_splits;
+  out->tma_epilogue = g.te;
+  out->ctas = g.grid;
+  out->running_sum = g.fix;
+  out->reserved = 0;
+  return MBD_OK;
+}
 
 extern "C" mbd_status mbd_profile_enable(mbd_net* n, int on) {
   if (!n) return MBD_E_INVALID;
@@ -897,6 +944,8 @@ extern "C" mbd_status mbd_gemm_bf16(int variant, int64_t M, int64_t N, int64_t K
                                     void* cuda_stream) {
   if (!A || !Bm || !D || variant < 0 || variant > 2 || M < 1 || N < 1 || K < 1 || k_splits < 1) return MBD_E_INVALID;
   if (lda % 8 || ldb % 8 || ldd % 8 || N % 8) return MBD_E_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(Bm) | reinterpret_cast<uintptr_t>(D) |
+       reinterpret_cast<uintptr_t>(partials)) & 15u) return MBD_E_UNSUPPORTED;      // 16-byte aligned bases
   if (k_splits > 1 && !partials) return MBD_E_INVALID;
   if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return MBD_E_UNSUPPORTED;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -1,8 +1,11 @@
 // mbd_gemm_bf16_noalloc: the split-K tensor-core contraction of mbd_gemm_bf16 for callers
-// that must not allocate device memory -- code running between the capture calls of a
-// stream, inside a memory-pool-managed service whose allocator is the only permitted
-// one, or on a device whose memory is fully handed out already.  The fp32 partial sums
-// and the status word live in a fixed array that is part of this library's device image.
+// that must not allocate device memory -- a service whose own memory pool was handed the
+// whole GPU at start-up and is the only allocator permitted, or a plug-in called on a
+// device whose memory is fully given out already, where cudaMalloc would fail or stall.
+// The fp32 partial sums and the status word live in a fixed array that is part of this
+// library's device image.  The call waits for the stream before it returns (it reads the
+// status word back); the first call on a device also looks up the arrays' device addresses
+// and sets the kernels' shared-memory attribute for that device.
 #include "../../include/mbd.h"
 #include "kernels.h"
 
@@ -41,6 +44,8 @@ extern "C" mbd_status mbd_gemm_bf16_noalloc(int variant, int64_t M, int64_t N, i
   if (!A || !Bm || !D || variant < 0 || variant > 2 || M < 1 || N < 1 || K < 1 || k_splits < 1) return MBD_E_INVALID;
   if (lda % 8 || ldb % 8 || ldd % 8 || N % 8) return MBD_E_UNSUPPORTED;
   if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return MBD_E_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(Bm) | reinterpret_cast<uintptr_t>(D)) & 15u)
+    return MBD_E_UNSUPPORTED;                              // TMA and the 16-byte stores need 16-byte aligned bases
   const int64_t kb = (K + 63) / 64;
   const int64_t S = k_splits < kb ? k_splits : kb;
   if (S > 1 && static_cast<unsigned __int128>(S) * M * N > SCRATCH_FLOATS) return MBD_E_TOO_LARGE;

@@ -29,7 +29,8 @@ EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weig
            "mbd_train_step_host_begin", "mbd_train_step_host_end",
            "mbd_comm_time", "mbd_redistribute_time", "mbd_total_time", "mbd_grid_table", "mbd_choose_grid",
            "mbd_enable_master_weights", "mbd_block_gemm_bf16", "mbd_block_reduce", "mbd_softmax_xent",
-           "mbd_conv_stage_input", "mbd_conv_forward_layer", "mbd_conv_backward_layer", "mbd_conv_outer_rows"]
+           "mbd_conv_stage_input", "mbd_conv_forward_layer", "mbd_conv_backward_layer", "mbd_conv_outer_rows",
+           "mbd_get_plan"]
 
 
 class MbdError(RuntimeError):
@@ -53,6 +54,12 @@ class Tail(C.Structure):
     _fields_ = [("op", C.c_int32), ("out_bf16", C.c_int32), ("relu", C.c_int32), ("reserved", C.c_int32),
                 ("out_dev", C.c_void_p), ("ldo", C.c_int64), ("bias_dev", C.c_void_p), ("mask_dev", C.c_void_p),
                 ("ldmask", C.c_int64), ("scale", C.c_float)]
+
+
+class Plan(C.Structure):
+    """mbd_plan: how one product of a layer is launched (see include/mbd.h)."""
+    _fields_ = [("tile_m", C.c_int32), ("tile_n", C.c_int32), ("cta_pair", C.c_int32), ("k_pieces", C.c_int32),
+                ("tma_epilogue", C.c_int32), ("ctas", C.c_int32), ("running_sum", C.c_int32), ("reserved", C.c_int32)]
 
 
 class Words(C.Structure):
@@ -129,6 +136,7 @@ def lib():
         L.mbd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double)]
         L.mbd_launch_count.argtypes = [vp]
         L.mbd_launch_count.restype = i64
+        L.mbd_get_plan.argtypes = [vp, i32, i32, C.POINTER(Plan)]
         L.mbd_gemm_bf16.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp, vp]
         L.mbd_gemm_bf16_noalloc.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
         L.mbd_selftest_timeout.argtypes = [i32, vp]
@@ -397,6 +405,12 @@ class Net:
     @property
     def launch_count(self) -> int:
         return int(lib().mbd_launch_count(self._h))
+
+    def plan(self, layer: int, product: int) -> Dict[str, int]:
+        """mbd_get_plan: tile shape, CTA pair, pieces of K, TMA epilogue, CTAs of product 0 / 1 / 2 of a layer."""
+        p = Plan()
+        _check(lib().mbd_get_plan(self._h, layer, product, C.byref(p)), "mbd_get_plan")
+        return {k: int(getattr(p, k)) for k, _ in Plan._fields_}
 
 
 def gemm_bf16(variant: int, A, B, k_splits: int = 1, return_partials: bool = False):

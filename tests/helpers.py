@@ -41,21 +41,48 @@ def bf16_store(A):
     return I.round_to_bf16(np.asarray(A, np.float32)).astype(np.float64)
 
 
-def oracle_fc_step(w, inp, blocked_grid=None, exact=False):
+def oracle_fc_step(w, inp, blocked_grid=None, exact=False, eta=None):
     """fp64 oracle step for a fully connected workload (paper orientation: d x B).
     bf16 workloads round the STORED activations to bf16 unless `exact`."""
     from oracle import mbd_oracle as O
     store = bf16_store if (w.dtype == "bf16" and not exact) else None
+    eta = w.eta if eta is None else eta
     L = len(inp.Ws)
     layers = [O.FC(inp.Ws[i].astype(np.float64), None if inp.bs[i] is None else inp.bs[i].astype(np.float64),
                    relu=True) for i in range(L)]
     X1 = inp.X.astype(np.float64).T
     if blocked_grid is None:
-        return O.train_step(layers, X1, inp.labels, "softmax_ce", w.eta, store=store)
-    return O.train_step_blocked(layers, X1, inp.labels, "softmax_ce", w.eta, *blocked_grid, store=store)
+        return O.train_step(layers, X1, inp.labels, "softmax_ce", eta, store=store)
+    return O.train_step_blocked(layers, X1, inp.labels, "softmax_ce", eta, *blocked_grid, store=store)
 
 
-def gpu_fc_step(w, inp, grid=(1, 1), max_partials=0, fused=False, force_acts=None):
+def update_sized_eta(o, Ws, B, ratio=1.0):
+    """A learning rate at which Eq. 1 moves every weight matrix by at least `ratio` of its own norm:
+    eta = ratio * B * max_i ||W_i|| / ||dW_i||.  At the workloads' eta = 0.01 a step moves the weights by
+    1e-4 .. 5e-4 of their norm, less than one bf16 rounding of the weights themselves (1e-3), so a
+    comparison of updated bf16 weights cannot tell an update from no update; at this eta it can."""
+    worst = max(np.linalg.norm(_oracle_shape(Ws[i])) / np.linalg.norm(o["dWs"][i]) for i in range(len(Ws)))
+    return float(ratio * B * worst)
+
+
+def _oracle_shape(W):
+    """A weight array as the oracle holds it (a 1 x 1 kernel is the centre tap of a 3 x 3 one)."""
+    W = np.asarray(W, np.float64)
+    return oracle_kernel(W) if W.ndim == 4 else W
+
+
+def oracle_with_eta(o, Ws, bs, B, eta):
+    """The oracle's result for another learning rate: only Eq. 1 depends on eta, so the updated weights
+    are re-formed from the oracle's own gradients with the oracle's own update."""
+    from oracle import mbd_oracle as O
+    o2 = dict(o)
+    o2["new_W"] = [O.sgd(_oracle_shape(Ws[i]), o["dWs"][i], eta, B) for i in range(len(Ws))]
+    o2["new_b"] = [None if (bs[i] is None or o["dbs"][i] is None) else O.sgd(np.asarray(bs[i], np.float64), o["dbs"][i], eta, B)
+                   for i in range(len(Ws))]
+    return o2
+
+
+def gpu_fc_step(w, inp, grid=(1, 1), max_partials=0, fused=False, force_acts=None, eta=None):
     """The same step through the C ABI.  Returns numpy fp64 arrays in the GPU's
     [B, d] / [d_out, d_in] layouts.  `force_acts` (list of [B, d_i] arrays for the hidden
     layers, bf16-exact) overwrites the stored activations after the forward pass, so that
@@ -64,6 +91,7 @@ def gpu_fc_step(w, inp, grid=(1, 1), max_partials=0, fused=False, force_acts=Non
     from paper_1712_04432_b200 import mbd
     bf = w.dtype == "bf16"
     L = len(inp.Ws)
+    eta = w.eta if eta is None else eta
     net = mbd.Net(mbd.fc_layers(w.dims, bias=True), w.B, grid[0], grid[1], mbd.BF16 if bf else mbd.F32,
                   mbd.LOSS_SOFTMAX_CE, max_partials)
     for i in range(L):
@@ -78,12 +106,12 @@ def gpu_fc_step(w, inp, grid=(1, 1), max_partials=0, fused=False, force_acts=Non
         for i in range(L - 1):
             net.set_tensor(mbd.T_ACT, i, to_dev(force_acts[i], bf))
     if fused:
-        net.backward(w.eta)
+        net.backward(eta)
     else:
         net.backward(0.0)
         out["dW"] = [to_np(net.get_tensor(mbd.T_DW, i)) for i in range(L)]
         out["db"] = [to_np(net.get_tensor(mbd.T_DB, i)) for i in range(L)]
-        net.sgd_step(w.eta)
+        net.sgd_step(eta)
     net.poll()
     out["J"] = float(J.item())
     out["loss"] = to_np(net.get_tensor(mbd.T_LOSS))
@@ -101,10 +129,35 @@ def oracle_hidden_acts(o):
     return [np.ascontiguousarray(x.T, np.float32) for x in o["Xs"][1:]]
 
 
-def compare_fc_step(g, o, tol, fused=False, tol_below_relu=None):
+BF16_ROUNDING_RMS = 2.0 ** -9 / np.sqrt(3.0)     # rms relative error of one round-to-nearest to bfloat16
+FP32_ROUNDING_RMS = 2.0 ** -24 / np.sqrt(3.0)
+
+
+def update_checks(chk, g, o, init_W, init_b, tols, bf16, require_sized):
+    """Eq. 1 itself: the step that was applied, W_new - W_0 (and b_new - b_0), against the oracle's, relative
+    to the size of the STEP, not of the weights.  Stored weights carry the rounding of W_new, which is
+    BF16_ROUNDING_RMS (or FP32_ROUNDING_RMS) * ||W_new|| whatever the step was; it is added to the tolerance,
+    so the check is sharp exactly when the step is comparable to the weights (`require_sized` demands that)."""
+    for i in range(len(init_W)):
+        w0 = np.asarray(init_W[i], np.float64)
+        step_o = np.asarray(o["new_W"][i], np.float64) - w0
+        rms = BF16_ROUNDING_RMS if bf16 else FP32_ROUNDING_RMS
+        noise = 1.5 * rms * np.linalg.norm(o["new_W"][i]) / max(np.linalg.norm(step_o), 1e-300)
+        if require_sized:
+            assert noise <= 0.5 * tols[i], f"layer {i}: the step is too small against the weights for a sharp check"
+        chk(f"W_new[{i}] - W_0[{i}]", g["new_W"][i] - w0, step_o, tols[i] + noise)
+        if init_b is not None and init_b[i] is not None and o["new_b"][i] is not None:
+            b0 = np.asarray(init_b[i], np.float64)
+            if np.linalg.norm(o["new_b"][i] - b0) > 0:
+                chk(f"b_new[{i}] - b_0[{i}]", g["new_b"][i] - b0, o["new_b"][i] - b0, tols[i])
+
+
+def compare_fc_step(g, o, tol, fused=False, tol_below_relu=None, init=None, bf16=True, require_sized=False, errors=None):
     """Element-by-element comparison, tensor by tensor; returns the worst relative
     Frobenius error.  `tol_below_relu` (default `tol`) applies to the gradients that sit
-    below a ReLU decision: dY_i, dW_i, db_i of every layer but the last."""
+    below a ReLU decision: dY_i, dW_i, db_i of every layer but the last.  `init` (the Inputs the
+    step started from) adds the comparison of the applied update itself (see `update_checks`).
+    `errors` (a dict) receives every measured error by tensor name."""
     L = len(o["Ys"])
     worst = 0.0
     report = []
@@ -116,6 +169,8 @@ def compare_fc_step(g, o, tol, fused=False, tol_below_relu=None):
         nonlocal worst
         e = rel_fro(got, ref)
         worst = max(worst, e)
+        if errors is not None:
+            errors[name] = e
         report.append(f"{name}: {e:.3e}")
         if e > (tol if t is None else t):
             bad.append(name)
@@ -130,9 +185,12 @@ def compare_fc_step(g, o, tol, fused=False, tol_below_relu=None):
         if not fused:
             chk(f"dW[{i}]", g["dW"][i], o["dWs"][i], tg)
             chk(f"db[{i}]", g["db"][i], o["dbs"][i], tg)
-        chk(f"W_new[{i}]", g["new_W"][i], o["new_W"][i])
+        chk(f"W_new[{i}]", g["new_W"][i], o["new_W"][i], tg)
         ref_b = o["new_b"][i]
-        assert np.abs(g["new_b"][i] - ref_b).max() <= tol * max(1.0, np.abs(ref_b).max()), f"b_new[{i}]"
+        assert np.abs(g["new_b"][i] - ref_b).max() <= tg * max(1.0, np.abs(ref_b).max()), f"b_new[{i}]"
+    if init is not None:
+        update_checks(chk, g, o, init.Ws, init.bs, [tol if i == L - 1 else tol_below_relu for i in range(L)], bf16,
+                      require_sized)
     assert not bad, "rel. Frobenius error too large for %s: %s" % (bad, "; ".join(report))
     return worst
 
@@ -156,24 +214,26 @@ def like_device(ref, got):
     ref = np.asarray(ref)
     return ref[:, :, 1:2, 1:2] if (ref.ndim == 4 and got.shape[-1] == 1 and ref.shape[-1] == 3) else ref
 
-def oracle_conv_step(w, inp, strips=None, grid=None):
+def oracle_conv_step(w, inp, strips=None, grid=None, eta=None):
     """fp64 oracle step for a domain-parallel conv workload (NCHW); stored activations are
     rounded to bf16 like the device's.  `strips` = P_r (or `grid` = (P_r, P_c)) runs the
     strip / halo formulation."""
     from oracle import mbd_oracle as O
     layers = [O.Conv3x3(oracle_kernel(k), relu=True) for k in inp.Ws]
     X = inp.X.astype(np.float64)
+    eta = w.eta if eta is None else eta
     if strips is None and grid is None:
-        return O.train_step(layers, X, None, "half_ssq", w.eta, store=bf16_store)
+        return O.train_step(layers, X, None, "half_ssq", eta, store=bf16_store)
     P_r, P_c = grid if grid is not None else (strips, 1)
-    return O.train_step_blocked(layers, X, None, "half_ssq", w.eta, P_r, P_c, store=bf16_store)
+    return O.train_step_blocked(layers, X, None, "half_ssq", eta, P_r, P_c, store=bf16_store)
 
 
-def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1):
+def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1, eta=None):
     import torch
     from paper_1712_04432_b200 import mbd
     C_, H, Wd = w.dims
     L = w.n_layers
+    eta = w.eta if eta is None else eta
     net = mbd.Net(mbd.conv_layers(L, C_, H, Wd, k=[w.ksize(i) for i in range(L)]), w.B, P_r, P_c, mbd.BF16,
                   mbd.LOSS_HALF_SSQ, 0)
     for i in range(L):
@@ -187,11 +247,11 @@ def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1):
         for i in range(L - 1):
             net.set_tensor(mbd.T_ACT, i, to_dev(force_acts[i], True))
     if fused:
-        net.backward(w.eta)
+        net.backward(eta)
     else:
         net.backward(0.0)
         out["dW"] = [to_np(net.get_tensor(mbd.T_DW, i)) for i in range(L)]
-        net.sgd_step(w.eta)
+        net.sgd_step(eta)
     net.poll()
     out["J"] = float(J.item())
     out["dY"] = [to_np(net.get_tensor(mbd.T_DY, i)) for i in range(L)]
@@ -201,7 +261,7 @@ def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1):
     return out
 
 
-def compare_conv_step(g, o, tol, fused=False, tol_below_relu=None):
+def compare_conv_step(g, o, tol, fused=False, tol_below_relu=None, init=None, require_sized=False):
     L = len(o["Ys"])
     report, bad = [], []
     if tol_below_relu is None:
@@ -220,7 +280,13 @@ def compare_conv_step(g, o, tol, fused=False, tol_below_relu=None):
         chk(f"dY[{i}]", g["dY"][i], o["dYs"][i], tg)
         if not fused:
             chk(f"dK[{i}]", g["dW"][i], like_device(o["dWs"][i], g["dW"][i]), tg)
-        chk(f"K_new[{i}]", g["new_W"][i], like_device(o["new_W"][i], g["new_W"][i]), tol)
+        chk(f"K_new[{i}]", g["new_W"][i], like_device(o["new_W"][i], g["new_W"][i]), tg)
+    if init is not None:
+        od = dict(o)
+        od["new_W"] = [like_device(o["new_W"][i], g["new_W"][i]) for i in range(L)]
+        od["new_b"] = [None] * L
+        update_checks(chk, g, od, init.Ws, None, [tol if i == L - 1 else tol_below_relu for i in range(L)], True,
+                      require_sized)
     assert not bad, "rel. Frobenius error too large for %s: %s" % (bad, "; ".join(report))
     return report
 
@@ -228,7 +294,7 @@ def compare_conv_step(g, o, tol, fused=False, tol_below_relu=None):
 # ---------------------------------------------------------------------------
 # convolutions followed by fully connected layers (Section 2.4)
 # ---------------------------------------------------------------------------
-def oracle_mixed_step(w, inp, blocked_grid=None):
+def oracle_mixed_step(w, inp, blocked_grid=None, eta=None):
     """fp64 oracle step of a mixed workload: Conv3x3 layers on NCHW, then FC layers on the
     flattened activation; stored activations rounded to bf16 like the device's."""
     from oracle import mbd_oracle as O
@@ -237,9 +303,10 @@ def oracle_mixed_step(w, inp, blocked_grid=None):
     for i in range(Lc, w.L):
         layers.append(O.FC(inp.Ws[i].astype(np.float64), inp.bs[i].astype(np.float64), relu=True))
     X = inp.X.astype(np.float64)
+    eta = w.eta if eta is None else eta
     if blocked_grid is None:
-        return O.train_step(layers, X, inp.labels, "softmax_ce", w.eta, store=bf16_store)
-    return O.train_step_blocked(layers, X, inp.labels, "softmax_ce", w.eta, *blocked_grid, store=bf16_store)
+        return O.train_step(layers, X, inp.labels, "softmax_ce", eta, store=bf16_store)
+    return O.train_step_blocked(layers, X, inp.labels, "softmax_ce", eta, *blocked_grid, store=bf16_store)
 
 
 def mixed_layers(w):
@@ -263,11 +330,12 @@ def oracle_mixed_acts(o, w):
     return out
 
 
-def gpu_mixed_step(w, inp, grid=(1, 1), max_partials=0, fused=False, force_acts=None):
+def gpu_mixed_step(w, inp, grid=(1, 1), max_partials=0, fused=False, force_acts=None, eta=None):
     """The same step through the C ABI; conv tensors come back NCHW, FC tensors [B, d]."""
     import torch
     from paper_1712_04432_b200 import mbd
     L, Lc = w.L, w.n_layers
+    eta = w.eta if eta is None else eta
     net = mbd.Net(mixed_layers(w), w.B, grid[0], grid[1], mbd.BF16, mbd.LOSS_SOFTMAX_CE, max_partials)
     for i in range(L):
         if i < Lc:
@@ -284,12 +352,12 @@ def gpu_mixed_step(w, inp, grid=(1, 1), max_partials=0, fused=False, force_acts=
         for i in range(L - 1):
             net.set_tensor(mbd.T_ACT, i, to_dev(force_acts[i], True))
     if fused:
-        net.backward(w.eta)
+        net.backward(eta)
     else:
         net.backward(0.0)
         out["dW"] = [to_np(net.get_tensor(mbd.T_DW, i)) for i in range(L)]
         out["db"] = [to_np(net.get_tensor(mbd.T_DB, i)) if i >= Lc else None for i in range(L)]
-        net.sgd_step(w.eta)
+        net.sgd_step(eta)
     net.poll()
     out["J"] = float(J.item())
     out["loss"] = to_np(net.get_tensor(mbd.T_LOSS))
@@ -306,7 +374,7 @@ def gpu_mixed_step(w, inp, grid=(1, 1), max_partials=0, fused=False, force_acts=
     return out
 
 
-def compare_mixed_step(g, o, w, tol, fused=False, tol_below_relu=None):
+def compare_mixed_step(g, o, w, tol, fused=False, tol_below_relu=None, init=None, require_sized=False):
     L, Lc = w.L, w.n_layers
     C_, H, Wd = w.dims
     report, bad = [], []
@@ -336,9 +404,14 @@ def compare_mixed_step(g, o, w, tol, fused=False, tol_below_relu=None):
             chk(f"dW[{i}]", g["dW"][i], like_device(o["dWs"][i], g["dW"][i]), tg)
             if i >= Lc:
                 chk(f"db[{i}]", g["db"][i], o["dbs"][i], tg)
-        chk(f"W_new[{i}]", g["new_W"][i], like_device(o["new_W"][i], g["new_W"][i]), tol)
+        chk(f"W_new[{i}]", g["new_W"][i], like_device(o["new_W"][i], g["new_W"][i]), tg)
         if i >= Lc:
             ref_b = o["new_b"][i]
-            assert np.abs(g["new_b"][i] - ref_b).max() <= tol * max(1.0, np.abs(ref_b).max()), f"b_new[{i}]"
+            assert np.abs(g["new_b"][i] - ref_b).max() <= tg * max(1.0, np.abs(ref_b).max()), f"b_new[{i}]"
+    if init is not None:
+        od = dict(o)
+        od["new_W"] = [like_device(o["new_W"][i], g["new_W"][i]) for i in range(L)]
+        update_checks(chk, g, od, init.Ws, init.bs, [tol if i == L - 1 else tol_below_relu for i in range(L)], True,
+                      require_sized)
     assert not bad, "rel. Frobenius error too large for %s: %s" % (bad, "; ".join(report))
     return report

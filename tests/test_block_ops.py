@@ -75,3 +75,38 @@ def test_block_reduce_and_softmax():
     mbd.softmax_xent(torch.from_numpy(logits).cuda(), torch.from_numpy(labels).cuda(), dY, per)
     J, per_ref, dY_ref = O.softmax_ce(logits.astype(np.float64).T, labels)
     assert rel_fro(to_np(per), per_ref) < 1e-5 and rel_fro(to_np(dY), dY_ref.T) < 1e-5
+
+
+def test_views_at_odd_offsets_take_the_element_wise_kernels():
+    # mbd_block_reduce and mbd_softmax_xent move 16 bytes per access only when every base is 16-byte aligned;
+    # a view that starts 4 bytes into a buffer (leading dimension still a multiple of 8) gives the same values
+    import torch
+    from paper_1712_04432_b200 import mbd
+    r = np.random.default_rng(8)
+    S, M, N = 2, 16, 40
+    parts = r.standard_normal((S, M, N)).astype(np.float32)
+    mask = r.standard_normal((M, N)).astype(np.float32)
+    buf = torch.zeros(M * N + 8, dtype=torch.float32, device="cuda")
+    out = buf[1:1 + M * N].view(M, N)                                   # 4 bytes past a 16-byte boundary
+    mbuf = torch.zeros(M * N + 8, dtype=torch.float32, device="cuda")
+    mview = mbuf[3:3 + M * N].view(M, N)
+    mview.copy_(torch.from_numpy(mask))
+    mbd.block_reduce(torch.from_numpy(parts).cuda(), out, mbd.TAIL_MASK, mask=mview)
+    assert np.array_equal(to_np(out), ((parts[0] + parts[1]) * (mask > 0)).astype(np.float64))
+    assert float(buf[0]) == 0 and not buf[1 + M * N:].any()
+    # softmax on a logits view at an odd offset, with one label out of range: NaN loss for that sample only
+    Bn, d = 6, 40
+    logits = r.standard_normal((Bn, d)).astype(np.float32)
+    lbuf = torch.zeros(Bn * d + 8, dtype=torch.float32, device="cuda")
+    lview = lbuf[1:1 + Bn * d].view(Bn, d)
+    lview.copy_(torch.from_numpy(logits))
+    labels = np.array([0, 5, 39, 40, -1, 7], np.int32)
+    dY = torch.empty((Bn, d), dtype=torch.float32, device="cuda")
+    per = torch.empty(Bn, dtype=torch.float32, device="cuda")
+    mbd.softmax_xent(lview, torch.from_numpy(labels).cuda(), dY, per)
+    p = np.exp(logits - logits.max(1, keepdims=True)); p /= p.sum(1, keepdims=True)
+    per_h = to_np(per)
+    assert np.isnan(per_h[3]) and np.isnan(per_h[4]) and not np.isnan(per_h[[0, 1, 2, 5]]).any()
+    for b in (0, 1, 2, 5):
+        assert abs(per_h[b] + np.log(p[b, labels[b]])) < 1e-5
+    assert np.allclose(to_np(dY)[3], p[3], atol=1e-6) and np.allclose(to_np(dY)[4], p[4], atol=1e-6)

@@ -139,7 +139,7 @@ def test_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, P_r, P_c):
         for i in range(L):
             h = dims[i + 1] // P_r
             rows = slice(rr * h, (rr + 1) * h)
-            assert rel_fro(z[f"dW{i}"], o["dWs"][i][rows]) < (1e-2 if i == L - 1 else 5e-2), (rank, i)
+            assert rel_fro(z[f"dW{i}"], o["dWs"][i][rows]) < 1e-2, (rank, i)
             assert rel_fro(z[f"W{i}"], o["new_W"][i][rows]) < 1e-2, (rank, i)
         assert json.loads(str(z["words"])) == json.loads(str(z["want"]))          # Eq. 8, per process
     assert abs(loss - o["J"]) < 1e-2 * abs(o["J"])
@@ -204,9 +204,9 @@ def test_convolution_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, 
         loss += float(z["loss"])
         own = (slice(cc * m, (cc + 1) * m), slice(None), slice(rr * Hs, (rr + 1) * Hs), slice(None))
         assert rel_fro(z["Y"], o["Ys"][L - 1][own]) < 1e-2, rank                 # this strip of the last layer's output
-        assert rel_fro(z["dY0"], o["dYs"][0][own]) < 5e-2, rank                  # ... and of the gradient that reached layer 1
+        assert rel_fro(z["dY0"], o["dYs"][0][own]) < 1e-2, rank                  # ... and of the gradient that reached layer 1
         for i in range(L):
-            assert rel_fro(z[f"dK{i}"], like_device(o["dWs"][i], z[f"dK{i}"])) < (1e-2 if i == L - 1 else 5e-2), (rank, i)
+            assert rel_fro(z[f"dK{i}"], like_device(o["dWs"][i], z[f"dK{i}"])) < 1e-2, (rank, i)
             assert rel_fro(z[f"K{i}"], like_device(o["new_W"][i], z[f"K{i}"])) < 1e-2, (rank, i)
         assert json.loads(str(z["words"])) == json.loads(str(z["want"]))        # Eq. 9's terms for domain layers, per process
     assert abs(loss - o["J"]) < 1e-2 * abs(o["J"])
@@ -278,12 +278,12 @@ def test_integrated_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, P
             loss += float(z["loss"])
         assert rel_fro(z["logits"], o["Ys"][-1].T[cc * m:(cc + 1) * m]) < 1e-2, rank
         for i in range(Lc):
-            assert rel_fro(z[f"dK{i}"], like_device(o["dWs"][i], z[f"dK{i}"])) < 5e-2, (rank, i)
+            assert rel_fro(z[f"dK{i}"], like_device(o["dWs"][i], z[f"dK{i}"])) < 1e-2, (rank, i)
             assert rel_fro(z[f"K{i}"], like_device(o["new_W"][i], z[f"K{i}"])) < 1e-2, (rank, i)
         for i in range(Lf):
             h = dims[i + 1] // P_r
             rows = slice(rr * h, (rr + 1) * h)
-            assert rel_fro(z[f"dW{i}"], o["dWs"][Lc + i][rows]) < (1e-2 if i == Lf - 1 else 5e-2), (rank, i)
+            assert rel_fro(z[f"dW{i}"], o["dWs"][Lc + i][rows]) < 1e-2, (rank, i)
             assert rel_fro(z[f"W{i}"], o["new_W"][Lc + i][rows]) < 1e-2, (rank, i)
         assert json.loads(str(z["words"])) == json.loads(str(z["want"]))
     assert abs(loss - o["J"]) < 1e-2 * abs(o["J"])

@@ -85,3 +85,24 @@ def test_block_calls_reject_bad_arguments():
     assert L.mbd_block_gemm_bf16(0, 8, 8, 8, None, 8, None, 8, C.byref(t), None, None) == mbd.E_INVALID
     assert L.mbd_block_reduce(None, 1, 8, 8, C.byref(t), 1, None) == mbd.E_INVALID
     assert L.mbd_softmax_xent(None, 1, 8, None, None, 0, None, 1, None) == mbd.E_INVALID
+
+
+def test_misaligned_bases_are_rejected_before_anything_is_launched():
+    # The contraction moves its operands by TMA and its results by 16-byte stores: a view that starts
+    # at an odd offset (leading dimension still a multiple of 8) gets a return code, never a launch.
+    # The addresses are made up and never dereferenced: the checks run before any CUDA call.
+    L = mbd.lib()
+    ok, odd = 0x7000000000, 0x7000000000 + 4
+    args = lambda A, B, D: (0, 64, 64, 64, C.c_void_p(A), 64, C.c_void_p(B), 64, C.c_void_p(D), 64, 1)
+    for A, B, D in [(odd, ok, ok), (ok, odd, ok), (ok, ok, odd)]:
+        assert L.mbd_gemm_bf16(*args(A, B, D), None, None) == mbd.E_UNSUPPORTED
+        assert L.mbd_gemm_bf16_noalloc(*args(A, B, D), None) == mbd.E_UNSUPPORTED
+    for field in ("out", "mask", "bias"):
+        t = mbd.Tail(mbd.TAIL_MASK, 1, 0, 0, odd if field == "out" else ok, 64, odd if field == "bias" else None,
+                     odd if field == "mask" else None, 64, 0.0)
+        assert L.mbd_block_gemm_bf16(0, 64, 64, 64, C.c_void_p(ok), 64, C.c_void_p(ok), 64, C.byref(t), None, None) == mbd.E_UNSUPPORTED
+
+
+def test_plan_query_rejects_bad_arguments():
+    p = mbd.Plan()
+    assert mbd.lib().mbd_get_plan(None, 0, 0, C.byref(p)) == mbd.E_INVALID

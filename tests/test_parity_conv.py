@@ -5,11 +5,11 @@ import numpy as np
 import pytest
 
 from paper_1712_04432_b200 import inputs as I
-from tests.helpers import compare_conv_step, gpu_conv_step, oracle_conv_step, rel_fro
+from tests.helpers import compare_conv_step, gpu_conv_step, oracle_conv_step, oracle_with_eta, rel_fro, update_sized_eta
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-2
-TOL_FREE = 5e-2      # free-running gradients below a ReLU (see test_parity_fc.py)
+TOL_FREE = 1e-2      # free-running (ReLU decisions on the device's own stored activations): measured 1.9e-3 at worst, no flips
 
 
 def stored_hidden(o):
@@ -77,13 +77,23 @@ def test_full_resolution_two_images(P_r):
     compare_conv_step(g, o, TOL)
 
 
-def test_full_workload_32_images_two_strips():
-    # the benchmark's launch configuration: 32 images of 64 x 224 x 224, two strips per image
+@pytest.fixture(scope="module")
+def cfg4_full():
     w = I.WORKLOADS["cfg4"]
     inp = I.make_inputs(w, seed=0)
     o = oracle_conv_step(w, inp)
-    g = gpu_conv_step(w, inp, 2, force_acts=stored_hidden(o))
-    compare_conv_step(g, o, TOL)
+    # a learning rate at which Eq. 1 moves both kernels by at least their own norm (see helpers.update_checks)
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    return w, inp, oracle_with_eta(o, inp.Ws, inp.bs, w.B, eta), eta
+
+
+@pytest.mark.parametrize("P_r,fused", [(1, False), (2, True), (4, True), (8, True)])
+def test_full_workload_32_images_every_strip_count(cfg4_full, P_r, fused):
+    # the whole workload -- 32 images of 64 x 224 x 224 -- on every strip count it lists; two strips with the fused
+    # update is the benchmark's launch configuration
+    w, inp, o, eta = cfg4_full
+    g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o), eta=eta)
+    compare_conv_step(g, o, TOL, fused, init=inp, require_sized=True)
 
 
 @pytest.mark.parametrize("H,W,B,P_r", [(8, 62, 3, 1), (8, 56, 4, 2), (8, 30, 5, 2), (6, 14, 3, 3), (8, 7, 2, 1),

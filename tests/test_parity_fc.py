@@ -5,18 +5,22 @@ import numpy as np
 import pytest
 
 from paper_1712_04432_b200 import inputs as I
-from tests.helpers import compare_fc_step, gpu_fc_step, oracle_fc_step, oracle_hidden_acts, rel_fro
+from tests.helpers import (compare_fc_step, gpu_fc_step, oracle_fc_step, oracle_hidden_acts, oracle_with_eta, rel_fro,
+                           update_sized_eta)
 
 pytestmark = pytest.mark.gpu
 
 TOL_F32 = 1e-5     # fp32 check mode
 TOL_BF16 = 1e-2    # bf16 storage, fp32 accumulation
-# Free-running bf16 step, gradients below a ReLU: fp32 (device) and fp64 (oracle) sums round a
-# few stored activations to neighbouring bf16 values, which moves a few pre-activations of the
-# next layer across zero; a flipped mask element is wrong by its full size, so a fraction f of
-# flips costs about sqrt(f) (f ~ 1e-4 at K = 25088 gives ~1.3e-2).  With the ReLU decisions
-# forced to the oracle's stored activations the plain 1e-2 holds.
-TOL_BF16_FREE = 5e-2
+# Free-running bf16 step (the device takes its ReLU decisions on its own stored activations).  fp32 (device)
+# and fp64 (oracle) sums round a few stored activations to neighbouring bf16 values, which moves a few
+# pre-activations of the next layer across zero; a flipped mask element is wrong by its full size, so a
+# fraction f of flips costs about sqrt(f).  Measured, worst tensor below a ReLU, every grid of each case:
+# 2.6e-3 (small_bf16, no flips), 6.0e-3 (cfg2, f = 1.3e-5 in layer 2), 1.09e-2 (cfg3, K = 25088, f = 6.6e-5).
+# So every case but cfg3 meets the plain 1e-2 free-running as well; cfg3 gets 1.5 x its measured error, and
+# meets 1e-2 with the ReLU decisions forced to the oracle's stored activations.
+TOL_BF16_FREE = 1e-2
+TOL_BF16_FREE_CFG3 = 1.65e-2
 
 
 @pytest.fixture(scope="module")
@@ -58,15 +62,23 @@ def small_bf16():
     return w, inp, oracle_fc_step(w, inp)
 
 
+def sized(w, inp, o):
+    """The oracle's step at a learning rate that moves every weight matrix by at least its own norm, so
+    that the comparison of the applied update is sharp on bf16 weights (see helpers.update_checks)."""
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    return oracle_with_eta(o, inp.Ws, inp.bs, w.B, eta), eta
+
+
 @pytest.mark.parametrize("grid,mp", [((1, 1), 0), ((8, 1), 8), ((1, 8), 8), ((2, 4), 4), ((4, 2), 1), ((16, 16), 2),
                                      ((3, 5), 8)])
 @pytest.mark.parametrize("fused", [False, True])
 def test_small_bf16_grids(small_bf16, grid, mp, fused):
     w, inp, o = small_bf16
-    g = gpu_fc_step(w, inp, grid, max_partials=mp, fused=fused)
-    compare_fc_step(g, o, TOL_BF16, fused, tol_below_relu=TOL_BF16_FREE)
-    g = gpu_fc_step(w, inp, grid, max_partials=mp, fused=fused, force_acts=oracle_hidden_acts(o))
-    compare_fc_step(g, o, TOL_BF16, fused)
+    o, eta = sized(w, inp, o)
+    g = gpu_fc_step(w, inp, grid, max_partials=mp, fused=fused, eta=eta)
+    compare_fc_step(g, o, TOL_BF16, fused, tol_below_relu=TOL_BF16_FREE, init=inp)
+    g = gpu_fc_step(w, inp, grid, max_partials=mp, fused=fused, force_acts=oracle_hidden_acts(o), eta=eta)
+    compare_fc_step(g, o, TOL_BF16, fused, init=inp, require_sized=True)
 
 
 def test_small_bf16_against_unrounded_oracle(small_bf16):
@@ -83,7 +95,7 @@ def test_small_bf16_against_unrounded_oracle(small_bf16):
     assert rel_fro(g["dY"][2], o["dYs"][2].T) < TOL_BF16       # top gradient: no mask above it
     assert rel_fro(g["dW"][2], o["dWs"][2]) < TOL_BF16
     for i in range(2):
-        assert rel_fro(g["dW"][i], o["dWs"][i]) < 0.1
+        assert rel_fro(g["dW"][i], o["dWs"][i]) < 5e-2      # measured 3.3e-2: the unrounded oracle decides many ReLUs differently
 
 
 def test_small_bf16_against_blocked_oracle(small_bf16):
@@ -117,13 +129,16 @@ def test_run_to_run_bitwise_reproducible(small_bf16):
 def test_full_size_fc_workloads(name, grid, mp):
     w = I.WORKLOADS[name]
     inp = I.make_inputs(w, seed=0)
-    o = oracle_fc_step(w, inp)
-    g = gpu_fc_step(w, inp, grid, max_partials=mp)
-    compare_fc_step(g, o, TOL_BF16, tol_below_relu=TOL_BF16_FREE)
-    g = gpu_fc_step(w, inp, grid, max_partials=mp, force_acts=oracle_hidden_acts(o))
-    compare_fc_step(g, o, TOL_BF16)
-    gf = gpu_fc_step(w, inp, grid, max_partials=mp, fused=True)
-    compare_fc_step(gf, o, TOL_BF16, fused=True, tol_below_relu=TOL_BF16_FREE)
+    o, eta = sized(w, inp, oracle_fc_step(w, inp))
+    g = gpu_fc_step(w, inp, grid, max_partials=mp, eta=eta)
+    free = TOL_BF16_FREE_CFG3 if name == "cfg3" else TOL_BF16_FREE
+    compare_fc_step(g, o, TOL_BF16, tol_below_relu=free, init=inp)
+    g = gpu_fc_step(w, inp, grid, max_partials=mp, force_acts=oracle_hidden_acts(o), eta=eta)
+    compare_fc_step(g, o, TOL_BF16, init=inp, require_sized=True)
+    gf = gpu_fc_step(w, inp, grid, max_partials=mp, fused=True, force_acts=oracle_hidden_acts(o), eta=eta)
+    compare_fc_step(gf, o, TOL_BF16, fused=True, init=inp, require_sized=True)
+    gf = gpu_fc_step(w, inp, grid, max_partials=mp, fused=True)                    # the workload's own eta, free-running
+    compare_fc_step(gf, oracle_with_eta(o, inp.Ws, inp.bs, w.B, w.eta), TOL_BF16, fused=True, tol_below_relu=free)
 
 
 @pytest.mark.parametrize("case", range(10))
@@ -143,7 +158,8 @@ def test_seeded_random_networks_and_grids(case):
     inp = I.make_inputs(w, seed=100 + case)
     o = oracle_fc_step(w, inp)
     if dtype == "f32":
-        compare_fc_step(gpu_fc_step(w, inp, (P_r, P_c), max_partials=mp, fused=fused), o, TOL_F32, fused)
+        compare_fc_step(gpu_fc_step(w, inp, (P_r, P_c), max_partials=mp, fused=fused), o, TOL_F32, fused, init=inp, bf16=False)
     else:
-        g = gpu_fc_step(w, inp, (P_r, P_c), max_partials=mp, fused=fused, force_acts=oracle_hidden_acts(o))
-        compare_fc_step(g, o, TOL_BF16, fused)
+        o, eta = sized(w, inp, o)
+        g = gpu_fc_step(w, inp, (P_r, P_c), max_partials=mp, fused=fused, force_acts=oracle_hidden_acts(o), eta=eta)
+        compare_fc_step(g, o, TOL_BF16, fused, init=inp, require_sized=True)
