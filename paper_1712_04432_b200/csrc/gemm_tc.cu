@@ -91,7 +91,9 @@ struct Params {
   Epi epi;
   int* status;
   int te;                 // epilogue moves its global data with TMA through shared memory
+  int te_prefetch;        // TMA epilogue requests its boxes one tile ahead
   int fix;                // running sum: piece s adds its accumulator to the sum pieces 0..s-1 left in `partials`
+                          // (1: the pieces of a raster group follow one another; 2: all tiles piece by piece)
   int* flags;             // fix: one word per (tile, CTA of the pair, 128-row half, epilogue warp); zero between launches
 };
 
@@ -99,11 +101,12 @@ struct Work {
   int tm, tn, s, kb0, kb1;
 };
 
+template <int FIX>
 __device__ __forceinline__ Work decode_work(const Params& p, int w) {
   const int num_tiles = p.tiles_m * p.tiles_n;
   const int per_group = p.group_m * p.tiles_n;
   Work o;
-  if (p.fix) {
+  if (FIX && p.fix == 1) {
     // Running sum: the pieces of a raster group follow one another (all tiles of the group for piece 0,
     // then for piece 1, ...), so that piece s of a tile finds the sum of pieces 0..s-1 still in L2 and
     // the unit it depends on always has a smaller index than itself.
@@ -170,7 +173,8 @@ static __device__ __noinline__ bool flag_wait(const int* flag, int value, volati
 // reads both halves), keeps its 128 rows of the accumulator in its own TMEM and runs its own
 // epilogue: 64 B/clk of operand fill like the 256 x 256 tile, but with two accumulators (the
 // epilogue overlaps the next tile), 32 KB stages and the TMA epilogue.
-template <int A_MN, int B_MN, int BN, int MH, int PAIR>
+// FIX = 1: the instantiation that can add a product's K pieces as a running sum in its epilogue (CTA pairs only).
+template <int A_MN, int B_MN, int BN, int MH, int PAIR, int FIX>
 // 136 registers per thread at most (a few bytes of spill in three instantiations): the register file
 // is split over the SM's four sub-partitions, the busiest of which holds three of this CTA's ten
 // warps; at 136 registers it keeps room for two warps of a side-stream kernel (a reduction, a
@@ -201,7 +205,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __shared__ __align__(8) uint64_t empty_bar[STAGES];
   __shared__ __align__(8) uint64_t tmem_full_bar[2];
   __shared__ __align__(8) uint64_t tmem_empty_bar[2];
-  __shared__ __align__(8) uint64_t te_bar[8];
+  __shared__ __align__(8) uint64_t te_bar[16];        // TMA epilogue: one per epilogue warp and staging box
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
@@ -211,7 +215,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (threadIdx.x == 0) atomicCAS(p.status, 0, DEV_SMEM_MISALIGNED);
     return;
   }
-  const bool te = MH == 1 && p.te != 0;
+  const bool te = !FIX && MH == 1 && p.te != 0;
   const int stages = te ? STAGES_TE : STAGES;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -228,7 +232,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(smem_u32(&tmem_full_bar[i]), 1);
       mbar_init(smem_u32(&tmem_empty_bar[i]), PAIR ? 16 : 8);
     }
-    for (int i = 0; i < 8; ++i) mbar_init(smem_u32(&te_bar[i]), 1);
+    for (int i = 0; i < 16; ++i) mbar_init(smem_u32(&te_bar[i]), 1);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -263,7 +267,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0;
       bool ok = true;
       for (int w = w_first; w < total_work && ok; w += w_step) {
-        const Work wk = decode_work(p, w);
+        const Work wk = decode_work<FIX>(p, w);
         const int row0 = wk.tm * TILE_M + static_cast<int>(rank) * BMT;       // this CTA's rows of A
         const int col0 = wk.tn * BN + static_cast<int>(rank) * BNL;           // this CTA's part of the B tile
         for (int kb = wk.kb0; kb < wk.kb1; ++kb) {
@@ -303,7 +307,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int it = 0;
       bool ok = true;
       for (int w = w_first; w < total_work && ok; w += w_step, ++it) {
-        const Work wk = decode_work(p, w);
+        const Work wk = decode_work<FIX>(p, w);
         const int acc = it % ACC_BUFS;
         const uint32_t acc_phase = (it / ACC_BUFS) & 1u;
         ok = mbar_wait(smem_u32(&tmem_empty_bar[acc]), acc_phase ^ 1u, abortp, p.status, DEV_TIMEOUT_MMA_TMEM);
@@ -353,110 +357,260 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int half = (warp - 2) >> 2;
     if (te) {
       // ---- TMA epilogue: the tile's old weights / mask source arrive in this warp's staging boxes by
-      // TMA (requested before the accumulator is waited for), are combined in place with the
-      // accumulator, and leave by TMA store; the LSU never touches global memory.
+      // TMA, are combined in place with the accumulator, and leave by TMA store; the LSU never touches
+      // global memory.  A box ([32 rows][64 columns] bf16) is requested for the NEXT tile as soon as its
+      // store for this tile has read it, so the HBM latency of that load passes under the rest of this
+      // tile's epilogue and the next tile's main loop instead of standing between two tiles (with K = B
+      // of a few hundred, a tile's main loop is only a few microseconds long).
       const int e = warp - 2;
       const uint32_t stg = ring + STAGES_TE * STAGE_BYTES + e * (TE_BOXES * 4096);
       uint8_t* stg_gen = smem_raw + (stg - smem_u32(smem_raw));
-      const uint32_t lbar = smem_u32(&te_bar[e]);
       uint32_t lphase = 0;
       const bool need_load = p.epi.op == EPI_SGD || (p.epi.op == EPI_MASK && p.epi.mask != nullptr);
       const CUtensorMap* src_map = p.epi.op == EPI_SGD ? &tmOut : &tmAux;
+      auto request = [&](const Work& wk, int b) {        // lane 0: box b of tile wk
+        const int row0 = wk.tm * TILE_M + static_cast<int>(rank) * BMT + q * 32;
+        const int col0 = wk.tn * BN + half * HC;
+        const uint32_t lb = smem_u32(&te_bar[e * 2 + b]);
+        mbar_expect_tx(lb, 4096);
+        tma_load_2d(stg + b * 4096, src_map, col0 + b * 64, row0, lb);
+      };
+      const bool ahead = p.te_prefetch != 0;
+      if (need_load && ahead && lane == 0 && w_first < total_work) {
+        const Work wk0 = decode_work<FIX>(p, w_first);
+#pragma unroll
+        for (int b = 0; b < TE_BOXES; ++b) request(wk0, b);
+      }
       int it = 0;
       bool ok = true;
       for (int w = w_first; w < total_work && ok; w += w_step, ++it) {
-        const Work wk = decode_work(p, w);
+        const Work wk = decode_work<FIX>(p, w);
+        const bool has_next = w + w_step < total_work;
+        Work wk_next = wk;
+        if (need_load && ahead && has_next && lane == 0) wk_next = decode_work<FIX>(p, w + w_step);
+        if (need_load && !ahead && lane == 0) {            // tuning knob: request the boxes when the tile starts
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+#pragma unroll
+          for (int b = 0; b < TE_BOXES; ++b) request(wk, b);
+        }
         const int acc = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1u;
         const int row0 = wk.tm * TILE_M + static_cast<int>(rank) * BMT + q * 32;
         const int col0 = wk.tn * BN + half * HC;
-        if (lane == 0) {
-          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");     // earlier stores have read the boxes
-          if (need_load) {
-            mbar_expect_tx(lbar, TE_BOXES * 4096);
-#pragma unroll
-            for (int b = 0; b < TE_BOXES; ++b) tma_load_2d(stg + b * 4096, src_map, col0 + b * 64, row0, lbar);
-          }
-        }
-        __syncwarp();
         ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
-        if (ok && need_load) {
-          ok = mbar_wait(lbar, lphase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
-          lphase ^= 1u;
-        }
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_COLS + half * HC;
 #pragma unroll
-        for (int c = 0; c < HC / 32; ++c) {
-          uint32_t r[32];
-          tc_ld32(taddr + c * 32, r);
-          tc_wait_ld();
-          if (c == HC / 32 - 1) {                  // accumulator fully in registers: hand it back
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-              if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty_bar[acc]), 0));
-              else mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
-            }
+        for (int b = 0; b < TE_BOXES; ++b) {
+          if (need_load) {
+            ok = mbar_wait(smem_u32(&te_bar[e * 2 + b]), lphase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+          } else if (lane == 0) {
+            // nothing is loaded into the box: its store for the previous tile must have read it before it is refilled
+            if (TE_BOXES == 2) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
           }
-          uint8_t* box = stg_gen + (c >> 1) * 4096 + lane * 128;
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint4* cell = reinterpret_cast<uint4*>(box + ((((c & 1) * 4 + j) ^ (lane & 7)) << 4));
-            float v[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j * 8 + i]);
-            if (need_load) {
-              const uint4 qv = *cell;
-              const uint32_t wv[4] = {qv.x, qv.y, qv.z, qv.w};
-              if (p.epi.op == EPI_SGD) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  v[2 * i] = fmaf(p.epi.scale, v[2 * i], bf16_bits_to_f32(wv[i] & 0xFFFFu));
-                  v[2 * i + 1] = fmaf(p.epi.scale, v[2 * i + 1], bf16_bits_to_f32(wv[i] >> 16));
-                }
-              } else {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  if (!(bf16_bits_to_f32(wv[i] & 0xFFFFu) > 0.f)) v[2 * i] = 0.f;
-                  if (!(bf16_bits_to_f32(wv[i] >> 16) > 0.f)) v[2 * i + 1] = 0.f;
-                }
-              }
-            } else if (p.epi.op == EPI_ACT) {
-              const int n = col0 + c * 32 + j * 8;
-              if (p.epi.bias && n < p.N) {
-                const float4 b0 = *reinterpret_cast<const float4*>(p.epi.bias + n);
-                const float4 b1 = *reinterpret_cast<const float4*>(p.epi.bias + n + 4);
-                v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
-                v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
-              }
-              if (p.epi.relu) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) v[i] = fmaxf(v[i], 0.f);
+          for (int cc = 0; cc < 2; ++cc) {
+            const int c = b * 2 + cc;
+            uint32_t r[32];
+            tc_ld32(taddr + c * 32, r);
+            tc_wait_ld();
+            if (c == HC / 32 - 1) {                  // accumulator fully in registers: hand it back
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) {
+                if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty_bar[acc]), 0));
+                else mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
               }
             }
-            uint4 o;
-            o.x = pack_bf16x2(v[0], v[1]); o.y = pack_bf16x2(v[2], v[3]);
-            o.z = pack_bf16x2(v[4], v[5]); o.w = pack_bf16x2(v[6], v[7]);
-            *cell = o;
-          }
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // generic writes -> visible to TMA
-        __syncwarp();
-        if (lane == 0) {
+            uint8_t* box = stg_gen + b * 4096 + lane * 128;
 #pragma unroll
-          for (int b = 0; b < TE_BOXES; ++b) {
+            for (int j = 0; j < 4; ++j) {
+              uint4* cell = reinterpret_cast<uint4*>(box + (((cc * 4 + j) ^ (lane & 7)) << 4));
+              float v[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j * 8 + i]);
+              if (need_load) {
+                const uint4 qv = *cell;
+                const uint32_t wv[4] = {qv.x, qv.y, qv.z, qv.w};
+                if (p.epi.op == EPI_SGD) {
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    v[2 * i] = fmaf(p.epi.scale, v[2 * i], bf16_bits_to_f32(wv[i] & 0xFFFFu));
+                    v[2 * i + 1] = fmaf(p.epi.scale, v[2 * i + 1], bf16_bits_to_f32(wv[i] >> 16));
+                  }
+                } else {
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    if (!(bf16_bits_to_f32(wv[i] & 0xFFFFu) > 0.f)) v[2 * i] = 0.f;
+                    if (!(bf16_bits_to_f32(wv[i] >> 16) > 0.f)) v[2 * i + 1] = 0.f;
+                  }
+                }
+              } else if (p.epi.op == EPI_ACT) {
+                const int n = col0 + c * 32 + j * 8;
+                if (p.epi.bias && n < p.N) {
+                  const float4 b0 = *reinterpret_cast<const float4*>(p.epi.bias + n);
+                  const float4 b1 = *reinterpret_cast<const float4*>(p.epi.bias + n + 4);
+                  v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
+                  v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+                }
+                if (p.epi.relu) {
+#pragma unroll
+                  for (int i = 0; i < 8; ++i) v[i] = fmaxf(v[i], 0.f);
+                }
+              }
+              uint4 o;
+              o.x = pack_bf16x2(v[0], v[1]); o.y = pack_bf16x2(v[2], v[3]);
+              o.z = pack_bf16x2(v[4], v[5]); o.w = pack_bf16x2(v[6], v[7]);
+              *cell = o;
+            }
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // generic writes -> visible to TMA
+          __syncwarp();
+          if (lane == 0) {
             asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
                          ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(col0 + b * 64), "r"(row0), "r"(stg + b * 4096)
                          : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            if (need_load && ahead && has_next) {
+              asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the store has read the box: refill it
+              request(wk_next, b);
+            }
           }
-          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
+        if (!ok) break;
+        lphase ^= 1u;
       }
       if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // stores done before the CTA exits
       __syncwarp();
+    } else if (FIX && p.fix != 0) {
+      // ---- Running sum of a product's K pieces (Appendix A.2: the sum over the blocks of a process group,
+      // taken in ascending block order).  Piece s of a tile adds its accumulator to the sum of pieces
+      // 0..s-1, which the CTA that finished piece s-1 left in ONE fp32 plane, and writes the new sum back;
+      // the last piece applies the tail operation instead.  Same additions in the same order as the
+      // reduction kernel over S planes, so the results agree bit for bit.  All loads of a 32-column chunk
+      // (the sum so far and, for the last piece, the bf16 operand of its tail operation) are issued together
+      // under the TMEM load, so a chunk costs one memory round trip.
+      // Measured on the 8192^3 products (two pieces): 0.5 ms less per training step than S planes plus the
+      // reduction kernel -- and no more, because these reads share the L2 -> SM path with the operand ring,
+      // which the main loop already keeps close to its limit; a variant that transposed each chunk through
+      // shared memory for fully coalesced accesses was slower still (24.2 against 21.2 ms per step).
+      const int e = warp - 2;
+      const bool src_bf16 = p.epi.out_bf16 && ((p.epi.op == EPI_SGD && p.epi.master == nullptr) ||
+                                               (p.epi.op == EPI_MASK && p.epi.mask != nullptr));
+      const __nv_bfloat16* tsrc = p.epi.op == EPI_SGD ? reinterpret_cast<const __nv_bfloat16*>(p.epi.out)
+                                                      : reinterpret_cast<const __nv_bfloat16*>(p.epi.mask);
+      const int64_t tsrc_ld = p.epi.op == EPI_SGD ? p.epi.ldo : p.epi.ldmask;
+      int it = 0;
+      bool ok = true;
+      for (int w = w_first; w < total_work && ok; w += w_step, ++it) {
+        const Work wk = decode_work<FIX>(p, w);
+        const int acc = it % ACC_BUFS;
+        const uint32_t acc_phase = (it / ACC_BUFS) & 1u;
+        const bool first = wk.s == 0, last = wk.s == p.S - 1;
+        const bool tail_src = last && src_bf16;
+        const int64_t nbase = static_cast<int64_t>(wk.tn) * BN + half * HC;
+#pragma unroll 1
+        for (int h = 0; h < MH; ++h) {
+          const int64_t m = static_cast<int64_t>(wk.tm) * TILE_M + rank * BMT + h * 128 + q * 32 + lane;
+          const bool row_ok = m < p.M;
+          int* flag = p.flags + (((static_cast<int64_t>(wk.tm) * p.tiles_n + wk.tn) * 2 + rank) * 2 + h) * 8 + e;
+          if (h == 0) {
+            ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+          }
+          if (!first) {                          // the sum of pieces 0..s-1 of these rows and columns is complete
+            if (lane == 0) ok = flag_wait(flag, wk.s, abortp, p.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
+          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_COLS + h * BN + half * HC;
+#pragma unroll
+          for (int c = 0; c < HC / 32; ++c) {
+            uint32_t r[32];
+            tc_ld32(taddr + c * 32, r);
+            uint4 run[8], src[4];
+            if (!first && row_ok) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int64_t n = nbase + c * 32 + j * 8;
+                if (n < p.N) {
+                  run[2 * j] = __ldcg(reinterpret_cast<const uint4*>(p.partials + m * p.N + n));
+                  run[2 * j + 1] = __ldcg(reinterpret_cast<const uint4*>(p.partials + m * p.N + n + 4));
+                  if (tail_src) src[j] = *reinterpret_cast<const uint4*>(tsrc + m * tsrc_ld + n);
+                }
+              }
+            }
+            tc_wait_ld();
+            if (h == MH - 1 && c == HC / 32 - 1) {     // accumulator fully in registers: hand it back
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) {
+                if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty_bar[acc]), 0));
+                else mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+              }
+            }
+            if (row_ok) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int64_t n = nbase + c * 32 + j * 8;
+                if (n < p.N) {
+                  float v[8];
+#pragma unroll
+                  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j * 8 + i]);
+                  if (!first) {                   // ascending order: (sum of the earlier pieces) + this piece
+                    const uint4 r0 = run[2 * j], r1 = run[2 * j + 1];
+                    v[0] = __uint_as_float(r0.x) + v[0]; v[1] = __uint_as_float(r0.y) + v[1];
+                    v[2] = __uint_as_float(r0.z) + v[2]; v[3] = __uint_as_float(r0.w) + v[3];
+                    v[4] = __uint_as_float(r1.x) + v[4]; v[5] = __uint_as_float(r1.y) + v[5];
+                    v[6] = __uint_as_float(r1.z) + v[6]; v[7] = __uint_as_float(r1.w) + v[7];
+                  }
+                  if (!last) {
+                    float* dst = p.partials + m * p.N + n;
+                    __stcg(reinterpret_cast<float4*>(dst), make_float4(v[0], v[1], v[2], v[3]));
+                    __stcg(reinterpret_cast<float4*>(dst + 4), make_float4(v[4], v[5], v[6], v[7]));
+                  } else if (tail_src) {            // the arithmetic of epi_apply8, operand already in registers
+                    const uint4 qv = src[j];
+                    const uint32_t wv[4] = {qv.x, qv.y, qv.z, qv.w};
+                    if (p.epi.op == EPI_SGD) {
+#pragma unroll
+                      for (int i = 0; i < 4; ++i) {
+                        v[2 * i] = fmaf(p.epi.scale, v[2 * i], bf16_bits_to_f32(wv[i] & 0xFFFFu));
+                        v[2 * i + 1] = fmaf(p.epi.scale, v[2 * i + 1], bf16_bits_to_f32(wv[i] >> 16));
+                      }
+                    } else {
+#pragma unroll
+                      for (int i = 0; i < 4; ++i) {
+                        if (!(bf16_bits_to_f32(wv[i] & 0xFFFFu) > 0.f)) v[2 * i] = 0.f;
+                        if (!(bf16_bits_to_f32(wv[i] >> 16) > 0.f)) v[2 * i + 1] = 0.f;
+                      }
+                    }
+                    uint4 o;
+                    o.x = pack_bf16x2(v[0], v[1]); o.y = pack_bf16x2(v[2], v[3]);
+                    o.z = pack_bf16x2(v[4], v[5]); o.w = pack_bf16x2(v[6], v[7]);
+                    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.epi.out) + m * p.epi.ldo + n) = o;
+                  } else {
+                    epi_apply8(p.epi, m, n, v);
+                  }
+                }
+              }
+            }
+          }
+          if (!last) {
+            __threadfence();                       // this lane's part of the sum is visible device-wide ...
+            __syncwarp();
+            if (lane == 0) flag_publish(flag, wk.s + 1);      // ... before the next piece is told so
+          } else if (lane == 0) {
+            *flag = 0;                             // consumed: the word is zero again for the next launch
+          }
+        }   // h
+      }
     } else {
     const bool prefetch = p.S == 1 && p.epi.out_bf16 &&
                           ((p.epi.op == EPI_SGD && p.epi.master == nullptr) ||      // master weights: shared tail, no prefetch
@@ -467,19 +621,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     int it = 0;
     bool ok = true;
     for (int w = w_first; w < total_work && ok; w += w_step, ++it) {
-      const Work wk = decode_work(p, w);
+      const Work wk = decode_work<FIX>(p, w);
       const int acc = it % ACC_BUFS;
       const uint32_t acc_phase = (it / ACC_BUFS) & 1u;
       const int64_t nbase = static_cast<int64_t>(wk.tn) * BN + half * HC;
-      const bool fix = p.fix != 0;
-      const bool fix_first = wk.s == 0, fix_last = wk.s == p.S - 1;
-      float* part = p.S > 1 ? (fix ? p.partials : p.partials + static_cast<int64_t>(wk.s) * p.M * p.N) : nullptr;
+      float* part = p.S > 1 ? p.partials + static_cast<int64_t>(wk.s) * p.M * p.N : nullptr;
 #pragma unroll 1
       for (int h = 0; h < MH; ++h) {
       const int64_t m = static_cast<int64_t>(wk.tm) * TILE_M + rank * BMT + h * 128 + q * 32 + lane;
       const bool row_ok = m < p.M;
-      int* flag = nullptr;
-      if (fix) flag = p.flags + (((static_cast<int64_t>(wk.tm) * p.tiles_n + wk.tn) * 2 + rank) * 2 + h) * 8 + (warp - 2);
       uint4 pre[NV];
       if (prefetch) {
 #pragma unroll
@@ -494,28 +644,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!ok) break;
         tc_fence_after();
       }
-      if (fix && !fix_first) {                   // the sum of pieces 0..s-1 of these rows and columns is complete
-        if (lane == 0) ok = flag_wait(flag, wk.s, abortp, p.status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-      }
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_COLS + h * BN + half * HC;
 #pragma unroll
       for (int c = 0; c < HC / 32; ++c) {
         uint32_t r[32];
         tc_ld32(taddr + c * 32, r);
-        // running sum of the earlier pieces, requested under the TMEM load; it borrows the registers of the
-        // prefetch array, which an unsplit product uses and a split one does not
-        if (fix && !fix_first && row_ok) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int64_t n = nbase + c * 32 + j * 8;
-            if (n < p.N) {
-              pre[2 * j] = __ldcg(reinterpret_cast<const uint4*>(part + m * p.N + n));
-              pre[2 * j + 1] = __ldcg(reinterpret_cast<const uint4*>(part + m * p.N + n + 4));
-            }
-          }
-        }
         tc_wait_ld();
         if (h == MH - 1 && c == HC / 32 - 1) {     // accumulator fully in registers: hand it back
           tc_fence_before();
@@ -533,22 +666,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               float v[8];
 #pragma unroll
               for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j * 8 + i]);
-              if (fix) {
-                if (!fix_first) {                 // ascending order: (sum of the earlier pieces) + this piece
-                  const uint4 r0 = pre[2 * j], r1 = pre[2 * j + 1];
-                  v[0] = __uint_as_float(r0.x) + v[0]; v[1] = __uint_as_float(r0.y) + v[1];
-                  v[2] = __uint_as_float(r0.z) + v[2]; v[3] = __uint_as_float(r0.w) + v[3];
-                  v[4] = __uint_as_float(r1.x) + v[4]; v[5] = __uint_as_float(r1.y) + v[5];
-                  v[6] = __uint_as_float(r1.z) + v[6]; v[7] = __uint_as_float(r1.w) + v[7];
-                }
-                if (!fix_last) {
-                  float* dst = part + m * p.N + n;
-                  __stcg(reinterpret_cast<float4*>(dst), make_float4(v[0], v[1], v[2], v[3]));
-                  __stcg(reinterpret_cast<float4*>(dst + 4), make_float4(v[4], v[5], v[6], v[7]));
-                } else {
-                  epi_apply8(p.epi, m, n, v);
-                }
-              } else if (part) {
+              if (part) {
                 float* dst = part + m * p.N + n;
                 *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
                 *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
@@ -577,15 +695,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               }
             }
           }
-        }
-      }
-      if (fix) {
-        if (!fix_last) {
-          __threadfence();                       // this lane's part of the sum is visible device-wide ...
-          __syncwarp();
-          if (lane == 0) flag_publish(flag, wk.s + 1);      // ... before the next piece is told so
-        } else if (lane == 0) {
-          *flag = 0;                             // consumed: the word is zero again for the next launch
         }
       }
       }   // h
@@ -643,24 +752,30 @@ cudaError_t make_map(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t
 template <int A_MN, int B_MN>
 cudaError_t set_attr() {
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
-  return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES);
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 1, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 2, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES);
 }
 
 template <int A_MN, int B_MN>
 cudaError_t launch_t(const TcGemm& g, const Params& p, cudaStream_t stream) {
   const size_t smem = SMEM_DYN_BYTES;
   const dim3 grid(g.grid), block(NUM_THREADS);
-  if (g.pair && g.MH == 2) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  if (g.pair) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  if (g.BN == 256 && g.MH == 1) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 1, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  if (g.BN == 128 && g.MH == 1) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 128, 1, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  if (g.BN == 256) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 2, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
-  return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 128, 2, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  if (g.pair && p.fix) {
+    if (g.MH == 2) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1, 1>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+    return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1, 1>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  }
+  if (g.pair && g.MH == 2) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1, 0>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  if (g.pair) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1, 0>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  if (g.BN == 256 && g.MH == 1) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 1, 0, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  if (g.BN == 128 && g.MH == 1) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 128, 1, 0, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  if (g.BN == 256) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 2, 0, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 128, 2, 0, 0>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
 }
 
 }  // namespace
@@ -775,11 +890,14 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
   else e = make_map(&g.tmB, B, g.N, g.K, ldb, 64, BK);             // B[K,N]
   if (e != cudaSuccess) return e;
   // Running sum instead of S planes and a reduction launch: when the pieces of a tile are far apart in the
-  // work order (more tiles than CTA slots), or there are just two of them.
+  // work order (at least as many tiles as CTA slots: the pieces of one tile never run at the same time) ...
   {
     const long long tiles = 1ll * tiles_m * tiles_n;
     const int slots = g.pair ? num_sms / 2 : num_sms;
-    g.fix = g.allow_fix && g.k_splits > 1 && (g.k_splits == 2 || tiles >= slots) ? 1 : 0;
+    const int kb_piece = kb_total / (g.k_splits > 0 ? g.k_splits : 1);
+    // ... and a piece's main loop must be long enough to hide the epilogue of the piece before it (which reads
+    // the sum back row by row): short pieces are better served by S planes and the coalesced reduction kernel
+    g.fix = g.allow_fix && g.pair && g.k_splits > 1 && tiles >= slots && kb_piece >= 32 ? 1 : 0;
     g.flag_words = g.fix ? tiles * 32 : 0;
   }
   // TMA epilogue: bf16 output of an unsplit contraction on 128-row tiles
@@ -809,7 +927,9 @@ cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
   p.group_m = 8;                        // m-tiles per raster group (L2 reuse of the B operand)
   if (const char* ev = getenv("MBD_TC_GROUP_M")) { const int gm = atoi(ev); if (gm >= 1) p.group_m = gm; }
   p.partials = g.partials;
-  p.fix = g.fix && g.flags != nullptr;
+  p.fix = g.fix && g.pair && g.flags != nullptr;
+  if (p.fix && getenv("MBD_FIX_PLAIN_ORDER")) p.fix = 2;                 // tuning knob
+  p.te_prefetch = getenv("MBD_TE_NO_PREFETCH") ? 0 : 1;                  // tuning knob
   p.flags = g.flags;
   p.epi = g.epi;
   p.status = g.status;

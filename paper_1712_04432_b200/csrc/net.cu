@@ -209,7 +209,7 @@ mbd_status prepare_tc(mbd_net* n, TcGemm& g, int variant, int64_t M, int64_t N, 
   // max_partials >= P asks for every process's partial as a plane of its own (Appendix A.2 as the paper's
   // processes hold it); otherwise the pieces are intermediate and may be folded into a running sum
   const int P = variant == 1 ? n->P_r : variant == 2 ? n->P_c : 1;
-  static const bool no_fix = getenv("MBD_NO_FIXUP") != nullptr;      // tuning knob: always S planes + reduction launch
+  const bool no_fix = getenv("MBD_NO_FIXUP") != nullptr;             // tuning knob: always S planes + reduction launch
   g.allow_fix = !no_fix && (P == 1 || S < P);
   g.status = n->status;
   CK(tc_gemm_prepare(g, A, lda, Bm, ldb, n->num_sms, te_epi));

@@ -7,12 +7,16 @@ a profiler (small, self-terminating):
     python -m paper_1712_04432_b200.profile_case conv --batch 4 --strips 4
     python -m paper_1712_04432_b200.profile_case conv --batch 64 --strips 2 --image 56
     python -m paper_1712_04432_b200.profile_case fc --batch 8192 --dims 1024,8192
+    python -m paper_1712_04432_b200.profile_case fc --batch 8192 --dims 8192,8192,8192 --grid 16x16 --max-partials 2
 
 gemm_*: one tensor-core contraction of size^3 in the operand layout of that product.
 reduce: a split contraction followed by the partial-sum reduction (the reduction reads
 `splits` fp32 planes of size^2 and writes one).
 fc:     `launches` training steps of a small fully connected net (softmax, bias-gradient and
-        update kernels at a size where their DRAM figures mean something).
+        update kernels at a size where their DRAM figures mean something); with --grid / --max-partials
+        the products are launched as a workload on that logical grid launches them (two layers of
+        8192 x 8192 at batch 8192 on 16x16 with 2 partials: the benchmark's three products, one of each
+        per step plus a second forward and backward-weight product).
 conv:   `launches` training steps of the two-layer 3x3 convolution stack on `batch` images of
 64 x image x image (default 224), cut into `strips` row strips.
 """
@@ -34,6 +38,8 @@ def main():
     ap.add_argument("--size", type=int, default=8192)
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--splits", type=int, default=2)
+    ap.add_argument("--grid", default="1x1", help="fc: logical grid P_r x P_c")
+    ap.add_argument("--max-partials", type=int, default=0, help="fc: as mbd_net_create")
     a = ap.parse_args()
     if a.case == "conv":
         return conv_case(a)
@@ -60,19 +66,28 @@ def main():
 def fc_case(a):
     g = torch.Generator(device="cuda").manual_seed(0)
     dims = [int(d) for d in a.dims.split(",")]
-    net = mbd.Net(mbd.fc_layers(dims), a.batch, 1, 1, mbd.BF16, mbd.LOSS_SOFTMAX_CE, 0)
+    P_r, P_c = (int(x) for x in a.grid.lower().split("x"))
+    net = mbd.Net(mbd.fc_layers(dims), a.batch, P_r, P_c, mbd.BF16, mbd.LOSS_SOFTMAX_CE, a.max_partials)
+    for i in range(len(dims) - 1):
+        for product in ((0, 2) if i == 0 else (0, 1, 2)):
+            print(f"layer {i} product {product}: {net.plan(i, product)}")
     for i in range(len(dims) - 1):
         W = (torch.randn((dims[i + 1], dims[i]), generator=g, device="cuda") / dims[i] ** 0.5).to(torch.bfloat16)
         net.set_weights(i, W)
     X = torch.randn((a.batch, dims[0]), generator=g, device="cuda").to(torch.bfloat16)
     labels = torch.randint(0, dims[-1], (a.batch,), generator=g, device="cuda", dtype=torch.int32)
     J = torch.zeros(1, device="cuda")
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
     for _ in range(a.launches):
         net.forward(X, labels, J)
         net.backward(0.01)
+    ev1.record()
     torch.cuda.synchronize()
     net.poll()
-    print(f"fc dims={dims} batch={a.batch}: J = {J.item():.4e}")
+    print(f"fc dims={dims} batch={a.batch} grid={a.grid} max_partials={a.max_partials}: "
+          f"{ev0.elapsed_time(ev1) / a.launches:.3f} ms per step, J = {J.item():.4e}")
 
 
 def conv_case(a):

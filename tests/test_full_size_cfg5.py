@@ -100,7 +100,8 @@ def sized_eta(c):
     return c["eta"]
 
 
-@pytest.mark.parametrize("grid,mp,bench_plan", [((16, 16), 2, True), ((1, 1), 1, False), ((64, 4), 2, False), ((4, 64), 2, False)])
+@pytest.mark.parametrize("grid,mp,bench_plan", [((16, 16), 2, True), ((1, 1), 1, False), ((64, 4), 2, False), ((4, 64), 2, False),
+                                                ((16, 16), 4, False)])       # four pieces per sum: a running sum over three hand-overs
 def test_cfg5_listed_grids_fused_step(cfg5, grid, mp, bench_plan):
     from oracle import mbd_oracle as O
     from paper_1712_04432_b200 import mbd

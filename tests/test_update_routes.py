@@ -36,8 +36,8 @@ ROUTES = {
                                          dict(tile_m=256, cta_pair=0, k_pieces=1, tma_epilogue=0)),
     "epilogue_registers_cta_pair_512": ({"MBD_TC_PAIR": "2"}, (1, 1), 1, True,
                                         dict(tile_m=512, cta_pair=1, k_pieces=1, tma_epilogue=0)),
-    "reduction_tail_three_planes": ({}, (1, 3), 3, True, dict(k_pieces=3)),
-    "reduction_tail_two_large_planes": ({}, (2, 2), 2, True, dict(k_pieces=2)),
+    "reduction_tail_three_planes": ({}, (1, 3), 3, True, dict(k_pieces=3, running_sum=0)),
+    "reduction_tail_two_large_planes": ({}, (2, 2), 2, True, dict(k_pieces=2, running_sum=0)),
     "update_kernel_from_materialised_gradient": ({}, (1, 1), 1, False, dict(k_pieces=1)),
     "update_kernel_after_a_reduction": ({}, (1, 2), 2, False, dict(k_pieces=2)),
 }
@@ -111,3 +111,57 @@ def test_stand_alone_update_kernels_against_the_definition():
         want = O.sgd(W0, G, 1.0, 64)                               # eta = 1, B = 64
         got = to_np(W)
         assert np.linalg.norm((got - W0) - (want - W0)) <= 3e-3 * np.linalg.norm(want - W0)   # bf16 rounding of W_new
+
+
+@pytest.fixture(scope="module")
+def long_k_case():
+    # batch 4096 and 4096-wide layers: with two pieces per sum every piece is 32 k-blocks long, and every product
+    # has more output tiles than CTA pairs -- the conditions under which the pieces are added as a running sum
+    w = I.fc_workload((2048, 4096, 4096, 1000), 4096, "bf16", "relu_normal", name="running_sum")
+    inp = I.make_inputs(w, seed=33)
+    o = oracle_fc_step(w, inp)
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    return w, inp, oracle_with_eta(o, inp.Ws, inp.bs, w.B, eta), eta
+
+
+@pytest.mark.parametrize("grid,mp", [((4, 4), 2), ((2, 8), 2)])
+@pytest.mark.parametrize("fused", [True, False])
+def test_running_sum_equals_planes_and_reduction_bit_for_bit(monkeypatch, long_k_case, grid, mp, fused):
+    # With fewer partial sums than blocks (1 < S < P) and long pieces, the pieces of a product are added inside its
+    # own epilogue: piece s adds its accumulator to the sum of pieces 0..s-1 that another CTA left in one fp32 plane,
+    # and the last piece applies the tail operation (ReLU mask for backward-data, Eq. 1 or a plain store for
+    # backward-weight).  Same ascending order as the reduction kernel over S planes: every bit must agree.
+    from paper_1712_04432_b200 import mbd
+    w, inp, o, eta = long_k_case
+    runs = []
+    for off in (False, True):
+        if off:
+            monkeypatch.setenv("MBD_NO_FIXUP", "1")
+        net = mbd.Net(mbd.fc_layers(w.dims, bias=True), w.B, grid[0], grid[1], mbd.BF16, mbd.LOSS_SOFTMAX_CE, mp)
+        plans = [net.plan(0, 2), net.plan(1, 2), net.plan(2, 1)]       # dW_1, dW_2 (K = B), dX_3 (K = 4096... of layer 2's outputs)
+        net.close()
+        assert [p["k_pieces"] for p in plans[:2]] == [2, 2]
+        assert [p["running_sum"] for p in plans[:2]] == ([0, 0] if off else [1, 1]), plans
+        runs.append(gpu_fc_step(w, inp, grid, max_partials=mp, fused=fused, force_acts=oracle_hidden_acts(o), eta=eta))
+    a, b = runs
+    for i in range(3):
+        assert np.array_equal(a["new_W"][i], b["new_W"][i]) and np.array_equal(a["dY"][i], b["dY"][i]), i
+        if not fused:
+            assert np.array_equal(a["dW"][i], b["dW"][i]), i
+    compare_fc_step(a, o, TOL, fused, init=inp, require_sized=True)
+
+
+def test_running_sum_of_the_backward_data_product(monkeypatch, long_k_case):
+    # the ReLU-mask tail on the last piece: layer 2's input gradient sums over two row blocks of W_2 (K = 4096)
+    from paper_1712_04432_b200 import mbd
+    w, inp, o, eta = long_k_case
+    net = mbd.Net(mbd.fc_layers(w.dims, bias=True), w.B, 4, 1, mbd.BF16, mbd.LOSS_SOFTMAX_CE, 2)
+    p = net.plan(1, 1)
+    net.close()
+    assert p["k_pieces"] == 2 and p["running_sum"] == 1, p
+    a = gpu_fc_step(w, inp, (4, 1), max_partials=2, fused=True, force_acts=oracle_hidden_acts(o), eta=eta)
+    monkeypatch.setenv("MBD_NO_FIXUP", "1")
+    b = gpu_fc_step(w, inp, (4, 1), max_partials=2, fused=True, force_acts=oracle_hidden_acts(o), eta=eta)
+    for i in range(3):
+        assert np.array_equal(a["dY"][i], b["dY"][i]) and np.array_equal(a["new_W"][i], b["new_W"][i]), i
+    compare_fc_step(a, o, TOL, True, init=inp, require_sized=True)
