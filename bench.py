@@ -47,6 +47,10 @@ def parse_args():
     ap.add_argument("--grid", default=None, help="P_r x P_c, e.g. 16x16 (default: the workload's second grid)")
     ap.add_argument("--max-partials", type=int, default=2)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--mode", default="logical", choices=["logical", "grid"],
+                    help="logical (default): the P_r x P_c grid as logical blocks on every GPU (replicas for N > 1).  "
+                         "grid: one PROCESS per grid position (P_r * P_c = N, --grid required for N > 1), collectives "
+                         "over NCCL; fully connected workloads only")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -122,7 +126,8 @@ def workload_config(w, grid, max_partials):
         desc = (f"{w.name}: {w.n_layers}x conv3x3 {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, then FC "
                 f"{'-'.join(str(d) for d in w.fc_dims)}, B={w.B}, ReLU, softmax-CE, {w.dtype}")
     else:
-        desc = f"{w.name}: {w.n_layers}x conv3x3 {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, B={w.B}, half-SSQ, {w.dtype}"
+        ks = "x".join(str(w.ksize(0)) * 2)
+        desc = f"{w.name}: {w.n_layers}x conv{ks} {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, B={w.B}, half-SSQ, {w.dtype}"
     return dict(workload=desc, grid=f"{grid[0]}x{grid[1]}", max_partials=max_partials, batch=w.B,
                 l2="weights + activations per step exceed the 126 MB L2 (no flush needed)"
                 if I.step_flops(w) > 1e12 else "L2 flushed by a 256 MB write between steps")
@@ -155,12 +160,20 @@ def oracle_sample(w, inp):
         return I.step_flops(w) / w.B * Bs, dt, f"whole {w.L}-layer network, first {Bs} of {w.B} samples, fp64 numpy"
     C, H, Wd = w.dims
     Bs, Hs = 1, min(H, 56)
-    layers = [O.Conv3x3(k.astype(np.float64)) for k in inp.Ws]
+    def as3x3(k):          # the oracle's layer is 3 x 3: a 1 x 1 kernel is its centre tap
+        k = k.astype(np.float64)
+        if k.shape[-1] == 3:
+            return k
+        k3 = np.zeros(k.shape[:2] + (3, 3))
+        k3[:, :, 1, 1] = k[:, :, 0, 0]
+        return k3
+
+    layers = [O.Conv3x3(as3x3(k)) for k in inp.Ws]
     X = inp.X[:Bs, :, :Hs, :].astype(np.float64)
     t0 = time.perf_counter()
     O.train_step(layers, X, None, "half_ssq", w.eta)
     dt = time.perf_counter() - t0
-    flops = 2.0 * Bs * Hs * Wd * C * C * 9 * (3 * w.n_layers - 1)
+    flops = I.step_flops(w) / w.B / H * Bs * Hs          # the method's flops for these rows (1 x 1 layers: one tap)
     return flops, dt, f"{w.n_layers} conv layers on {Bs} image(s), first {Hs} rows, fp64 numpy"
 
 
@@ -274,8 +287,8 @@ def run_ours(args):
         labels_host = torch.from_numpy(inp.labels).pin_memory()
     else:
         C_, H, Wd = w.dims
-        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd), w.B, grid[0], grid[1], mbd.BF16, mbd.LOSS_HALF_SSQ,
-                      args.max_partials)
+        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.ksize(i) for i in range(w.n_layers)]), w.B, grid[0], grid[1],
+                      mbd.BF16, mbd.LOSS_HALF_SSQ, args.max_partials)
         for i, Ki in enumerate(inp.Ws):
             net.set_weights(i, dev(Ki))
         labels = labels_host = None
@@ -368,6 +381,33 @@ def run_ours(args):
         h2d = X_host.numel() * X_host.element_size() + (labels_host.numel() * 4 if labels_host is not None else 0)
         e2e = dict(value=aggregate_tflops(flops, world, dt * 1e3), unit="TFLOP/s", h2d_bytes_per_step=int(h2d), d2h_bytes_per_step=4,
                    ms_per_step=dt * 1e3)
+    # ---- the partial-sum reduction kernel on its own (outside the timed region): with few partial sums per
+    # reduction the step adds them inside the products' epilogues and never launches it, so its HBM rate is
+    # measured here, on two fp32 planes of the workload's largest weight matrix with the update of Eq. 1 as tail
+    reduce_probe = None
+    if rank == 0 and bf and w.kind == "fc":
+        d_out, d_in = max(((w.dims[i + 1], w.dims[i]) for i in range(len(w.dims) - 1)), key=lambda t: t[0] * t[1])
+        parts = torch.randn((2, d_out, d_in), dtype=torch.float32, device="cuda")
+        Wp = torch.randn((d_out, d_in), dtype=torch.float32, device="cuda").to(torch.bfloat16)
+        reps = 5
+        for _ in range(2):
+            mbd.block_reduce(parts, Wp, mbd.TAIL_SGD, scale=-1e-6, sync=False)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a_, b_ in ev:
+            if flush is not None:
+                flush.fill_(1)
+            a_.record()
+            mbd.block_reduce(parts, Wp, mbd.TAIL_SGD, scale=-1e-6, sync=False)
+            b_.record()
+        torch.cuda.synchronize()
+        r_ms = sum(a_.elapsed_time(b_) for a_, b_ in ev) / reps
+        r_bytes = d_out * d_in * (2 * 4 + 2 + 2)          # two fp32 planes read, bf16 weights read and written
+        peaks_ = measured_peaks()
+        reduce_probe = dict(kernel="reduce_partials_vec8_two_planes + Eq. 1 tail" if d_out * d_in >= (2 << 20) else "reduce_partials_vec8 + Eq. 1 tail",
+                            shape=[2, d_out, d_in], ms=r_ms, algorithmic_bytes=r_bytes, achieved=r_bytes / (r_ms * 1e-3) / 1e9,
+                            peak=peaks_["hbm_gbs"], unit="GB/s", frac=r_bytes / (r_ms * 1e-3) / 1e9 / peaks_["hbm_gbs"],
+                            peak_kind=f"{peaks_['source']} copy bandwidth")
+        del parts, Wp
     clocks = sampler.stop() if rank == 0 else None
     if rank != 0:
         if world > 1:
@@ -401,7 +441,12 @@ def run_ours(args):
                                   "derived fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x 1965 MHz",
                         frac_of_burst=ach / peaks["bf16_tflops"] if bf else None,
                         launches=g_n, avg_launch_ms=g_ms / g_n, flops_per_launch=g_fl / g_n,
-                        share_of_step=g_ms / (prof_ms * args.steps), traffic=TRAFFIC.get(w.name),
+                        share_of_step=g_ms / (prof_ms * args.steps),
+                        traffic=(traffic_for(w, grid, args.max_partials) or {}).get("per_launch_mean"),
+                        traffic_detail=traffic_for(w, grid, args.max_partials),
+                        note="with few partial sums per reduction the backward products add their K pieces in their own "
+                             "epilogue: the flops counted here are the products' alone, the time includes that reduction"
+                             if bf and w.kind == "fc" else None,
                         timed_in="second pass, direct launches" if use_graph else "the timed region")
     kernels = {k: dict(ms_per_step=v["ms"] / args.steps, launches_per_step=v["launches"] / args.steps,
                        rate=(v["work"] / (v["ms"] * 1e-3) / (1e12 if (k.startswith("gemm") or k.startswith("conv_")) else 1e9))
@@ -425,7 +470,7 @@ def run_ours(args):
                 clocks=clocks, e2e=e2e,
                 gpu_launches=int(launches) * world, roofline=roofline, cpu_baseline=cpu,
                 frac_of_burst_peak=flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"] if bf else None,
-                kernels=kernels, dominant_kernel_class=dom, loss_last=loss_last,
+                kernels=kernels, reduce_partials_probe=reduce_probe, dominant_kernel_class=dom, loss_last=loss_last,
                 launch_mode="CUDA graph replay (mbd_train_step)" if use_graph else "direct launches",
                 ms_per_step_direct=prof_ms if use_graph else None,
                 ms_per_step_median=float(np.median(per_step)), ms_per_step_min=float(min(per_step)),
@@ -435,15 +480,98 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# DRAM bytes per launch of the dominant kernel from an ncu capture (see profiles/); null until captured.
-# cfg5: gemm_tc_kernel at 8192^3, dram__bytes_read.sum + dram__bytes_write.sum of one launch
-# (profiles/gemm_tc_kernel_8192cubed.md; the captured launch wrote an fp32 result).
-TRAFFIC = {"cfg5": 1.06e9}
+# ------------------------------------------------------------------------------ the grid over processes
+def run_grid(args):
+    """Section 2.3 for real: rank (r, c) of a P_r x P_c grid of processes owns W_i(r, :) and batch block c; block
+    products with their tail operations in the library's kernels, all-gather / all-reduce over NCCL.  Strong
+    scaling: the workload is fixed, the grid divides it.  Prints ms per step (slowest rank, CUDA events), the
+    words every process moved per step against mbd_comm_words (Eq. 8), and the alpha-beta model's time for them."""
+    import torch
+    import torch.distributed as dist
+    from paper_1712_04432_b200 import mbd
+    from paper_1712_04432_b200.grid_exec import GridComm, GridFC, expected_words
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29511")
+    os.environ.setdefault("RANK", "0")
+    os.environ.setdefault("WORLD_SIZE", "1")
+    torch.cuda.set_device(local)
+    dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    w = I.WORKLOADS[args.workload]
+    if w.kind != "fc" or w.dtype != "bf16":
+        raise SystemExit("--mode grid runs the bf16 fully connected workloads (cfg2, cfg3, cfg5)")
+    P_r, P_c = (int(x) for x in args.grid.lower().split("x")) if args.grid else (world, 1)
+    if P_r * P_c != world:
+        raise SystemExit(f"--grid {P_r}x{P_c} needs {P_r * P_c} processes, got {world}")
+    comm = GridComm(P_r, P_c)
+    net = GridFC(w.dims, w.B, comm)
+    inp = I.make_inputs(w, seed=0)             # every process draws the same tensors and keeps its blocks
+
+    def dev(a):
+        return torch.from_numpy(I.bf16_bits(np.ascontiguousarray(a, np.float32)).view(np.int16)).cuda().view(torch.bfloat16)
+
+    for i in range(len(w.dims) - 1):
+        a, b = net.rows(i)
+        net.W[i].copy_(dev(inp.Ws[i][a:b]))
+    m = w.B // P_c
+    X_c = dev(inp.X[comm.c * m:(comm.c + 1) * m])
+    labels_c = torch.from_numpy(inp.labels[comm.c * m:(comm.c + 1) * m]).cuda()
+    del inp
+    for _ in range(max(args.warmup, 3)):
+        net.step(X_c, labels_c, w.eta)
+    for k in comm.words:
+        comm.words[k] = 0.0
+    dist.barrier()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    loss = 0.0
+    for _ in range(args.steps):
+        loss = net.step(X_c, labels_c, w.eta)
+    ev1.record()
+    torch.cuda.synchronize()
+    dist.barrier()
+    ms = max_over_ranks(ev0.elapsed_time(ev1) / args.steps, world)
+    if rank == 0:
+        flops = float(I.step_flops(w))
+        model = mbd.comm_time(mbd.fc_layers(w.dims, bias=False), w.B, P_r, P_c, mbd.MACHINE_B200_NVLINK5)
+        line = dict(metric=METRIC, value=flops / (ms * 1e-3) / 1e12, unit="TFLOP/s", n_gpus=world, steps=args.steps,
+                    warmup=max(args.warmup, 3), ms_per_step=ms, higher_is_better=True, scaling="strong", vs_baseline=None,
+                    dtype=w.dtype, data="synthetic",
+                    config=dict(workload=workload_config(w, (P_r, P_c), 0)["workload"], grid=f"{P_r}x{P_c}",
+                                mode="one process per grid position, NCCL collectives", batch=w.B),
+                    words_per_process_per_step={k: v / args.steps for k, v in comm.words.items()},
+                    eq8_words_per_process=expected_words(w.dims, w.B, P_r, P_c),
+                    alpha_beta_seconds_nvlink5=sum(sum(t.values()) for t in model), loss_block_0=loss)
+        print(json.dumps(line), flush=True)
+    dist.destroy_process_group()
+
+
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of
+# the same three products in the same plan: profiles/gemm_tc_kernel_8192_step_products.md).  gemm_tc_kernel is
+# launched 23 times per step of cfg5 on 16x16 with 2 partials: 8 forward products (0.944 GB each), 7 backward-data
+# (1.604 GB) and 8 backward-weight products (1.585 GB) whose two K pieces are added as a running sum in the
+# epilogue (one fp32 plane written and read back inside the launch).  Other plans have no capture: null.
+TRAFFIC_CFG5_16X16_2 = dict(per_launch_mean=(8 * 0.944e9 + 7 * 1.604e9 + 8 * 1.585e9) / 23,
+                            forward=0.944e9, backward_data=1.604e9, backward_weight=1.585e9,
+                            algorithmic=dict(forward=384e6, backward_data=384e6 + 134e6, backward_weight=384e6 + 134e6),
+                            source="profiles/gemm_tc_kernel_8192_step_products.md")
+
+
+def traffic_for(w, grid, max_partials):
+    if w.name == "cfg5" and tuple(grid) == (16, 16) and max_partials == 2 and not os.environ.get("MBD_NO_FIXUP"):
+        return TRAFFIC_CFG5_16X16_2
+    return None
 
 
 if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.mode == "grid":
+        run_grid(a)
     else:
         run_ours(a)

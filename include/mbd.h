@@ -117,8 +117,8 @@ enum {
  *                 block's partial as a plane of its own, exactly as the paper's
  *                 processes would hold it, and a reduction kernel adds the planes.
  *                 With 1 < S < P the partials are intermediate: they are either
- *                 written as S planes and reduced the same way, or (two pieces, or
- *                 more output tiles than SMs) added as a running sum inside the
+ *                 written as S planes and reduced the same way, or (two long pieces
+ *                 of a product with more output tiles than SMs) added as a running sum inside the
  *                 product -- the CTA that finishes piece s of a tile adds it to the
  *                 sum of pieces 0..s-1 that the CTA before it left in one fp32 plane
  *                 and the last one applies the tail operation.  Both forms add in
@@ -129,13 +129,14 @@ enum {
  * the input is NCHW, the first fully connected layer reads the last convolution's output
  * as [B, C*H*W] (row index c*H*W + h*W + w; its d_in must equal that), the loss is
  * softmax-CE, the dtype bf16, and the public layer index counts the convolutions first.
- * On a P_r x P_c grid a convolution is cut into P_r row strips and P_c batch blocks, a
+ * On a P_r x P_c grid a convolution is cut into P_r row strips (the balanced ranges
+ * [floor(s H / P_r), floor((s + 1) H / P_r)): heights differ by at most one row) and P_c batch blocks, a
  * fully connected layer into P_r row blocks of W_i and the same P_c batch blocks.
  * MBD_E_GRID if P_r < 1, P_c < 1, P_c > B, P_r > min d_i over model-split layers, or
  * a strip would be shorter than its halo.
  * MBD_E_UNSUPPORTED for convolutions other than 3x3 or 1x1, stride 1, "same" zero padding,
  * C_in = C_out = 64 (kind MBD_CONV3X3 with kh = kw = 1 is the 1x1 case, weights [C_out][C_in]),
- * strips of unequal height, a convolution above a fully connected layer, half-SSQ with
+ * a convolution above a fully connected layer, half-SSQ with
  * fully connected layers or softmax-CE without them, or bf16 FC dims that are not
  * multiples of 8. */
 MBD_API mbd_status mbd_net_create(const mbd_layer* layers_host, int L, int64_t B, int P_r, int P_c,

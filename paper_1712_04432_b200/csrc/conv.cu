@@ -69,6 +69,16 @@ constexpr int NUM_THREADS = 192;
 
 enum { MODE_RELU_STORE = 0, MODE_STORE_SSQ = 1, MODE_MASK = 2 };
 
+// Strips of an image of H rows are the balanced ranges [floor(s H / P), floor((s + 1) H / P)): their heights differ by
+// at most one.  Every strip is stored with the layout of the tallest one, Hs = ceil(H / P) own rows between two halo
+// rows; a shorter strip keeps its lower halo row right behind its last own row (row index height + 1 = Hs), and its
+// row Hs + 1 is never written and stays zero.  The kernels walk Hs rows per strip: what they compute for the one
+// dead row of a short strip is not stored, and where a dead row would be read as data (the dY rows of the
+// backward-weight product) the all-zero row Hs + 1 is read in its place.
+__host__ __device__ __forceinline__ int strip_first(int s, int H, int P) { return static_cast<int>((static_cast<long long>(s) * H) / P); }
+__host__ __device__ __forceinline__ int strip_height(int s, int H, int P) { return strip_first(s + 1, H, P) - strip_first(s, H, P); }
+__host__ __device__ __forceinline__ int strip_of_row(int h, int H, int P) { return static_cast<int>(((static_cast<long long>(h) + 1) * P - 1) / H); }
+
 // ------------------------------------------------------------------------------ layout kernels
 // NCHW -> strips.  Block = 32 consecutive pixels of one image's flattened (h, w) plane (so narrow
 // images fill their blocks too), all 64 channels; 128 threads.  A row that borders another strip is
@@ -115,15 +125,15 @@ nchw_to_strips_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int 
   v1.x = tile[px][cq + 4]; v1.y = tile[px][cq + 5]; v1.z = tile[px][cq + 6]; v1.w = tile[px][cq + 7];
   const int R = Hs + 2;
   const int h = p / W, w = p - h * W;
-  const int s = h / Hs, r = h - s * Hs + 1;
+  const int s = strip_of_row(h, H, P_r), r = h - strip_first(s, H, P_r) + 1;
   auto put = [&](int ss, int rr) {
     bf16* q = dst + (((static_cast<int64_t>(b) * P_r + ss) * R + rr) * W + w) * C + 2 * cq;
     *reinterpret_cast<uint4*>(q) = v0;
     *reinterpret_cast<uint4*>(q + 8) = v1;
   };
   put(s, r);
-  if (r == 1 && s > 0) put(s - 1, Hs + 1);          // first row of a strip: lower halo of the strip above
-  if (r == Hs && s < P_r - 1) put(s + 1, 0);        // last row of a strip: upper halo of the strip below
+  if (r == 1 && s > 0) put(s - 1, strip_height(s - 1, H, P_r) + 1);          // first row of a strip: lower halo of the strip above
+  if (r == strip_height(s, H, P_r) && s < P_r - 1) put(s + 1, 0);            // last row of a strip: upper halo of the strip below
 }
 
 // strips -> NCHW: the mirror image (own rows only).  Used to hand the last convolution's output to the
@@ -140,7 +150,7 @@ strips_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int 
     const int p = p0 + px;
     if (p < HW) {
       const int h = p / W, w = p - h * W;
-      const int s = h / Hs, r = h - s * Hs + 1;
+      const int s = strip_of_row(h, H, P_r), r = h - strip_first(s, H, P_r) + 1;
       const bf16* q = src + (((static_cast<int64_t>(b) * P_r + s) * R + r) * W + w) * C + 2 * cq;
       const uint4 v0 = *reinterpret_cast<const uint4*>(q), v1 = *reinterpret_cast<const uint4*>(q + 8);
       tile[px][cq + 0] = v0.x; tile[px][cq + 1] = v0.y; tile[px][cq + 2] = v0.z; tile[px][cq + 3] = v0.w;
@@ -267,8 +277,10 @@ wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ d
 // ------------------------------------------------------------------------------ forward kernel
 struct FwdParams {
   int W, Hs, R, nseg;
+  int H;                  // image rows: strip s of an image owns strip_height(s, H, P_r) <= Hs of the Hs row slots
   int pack, Z;            // narrow images: `pack` strips share one 128-pixel tile, 128 / pack pixels each (see below)
   int P_r;                // strips per image: a boundary row is also stored into the neighbouring strip's halo row
+  int k1;                 // 1 x 1 layer: an output row reads its own input row only, through the centre tap only
   long long rows_total;   // output row segments: (strip group z, segment, row) flattened with the row fastest
   int mode;
   bf16* out;              // strips
@@ -365,18 +377,21 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       bool ok = true;
       for (long long pos = r0; pos < r1 && ok;) {
         const FwdRun run = fwd_run(p, pos, r1);
-        for (int r = 0; r < run.n + 2; ++r) {
+        // 3 x 3: a run of n output rows reads n + 2 input rows, from the row above its first one on;
+        // 1 x 1: its own n rows (row index + 1: row 0 of a strip is the upper halo row)
+        const int n_in = p.k1 ? run.n : run.n + 2, row_in0 = p.k1 ? run.h0 + 1 : run.h0;
+        for (int r = 0; r < n_in; ++r) {
           ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
           if (!ok) break;
           const uint32_t fb = smem_u32(&full_bar[stage]);
           if (pack == 1) {
             mbar_expect_tx(fb, FWD1_BOX_PIX * 128);
-            tma_load_4d(ring + stage * FWD1_ROW_BYTES, &tmX, 0, run.seg * FWD_PIX - 1, run.h0 + r, run.z, fb);
+            tma_load_4d(ring + stage * FWD1_ROW_BYTES, &tmX, 0, run.seg * FWD_PIX - 1, row_in0 + r, run.z, fb);
           } else {
             const int sub_bytes = (FWD_PIX / pack) * 128;
             mbar_expect_tx(fb, FWD_PIX * 128);
             for (int j = 0; j < pack; ++j)      // a strip index beyond Z reads as zeros
-              tma_load_4d(ring + stage * FWD1_ROW_BYTES + j * sub_bytes, &tmX, 0, -1, run.h0 + r, run.z + j, fb);
+              tma_load_4d(ring + stage * FWD1_ROW_BYTES + j * sub_bytes, &tmX, 0, -1, row_in0 + r, run.z + j, fb);
           }
           if (++stage == FWD1_STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -391,6 +406,29 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       int g0 = 0;              // output rows of earlier runs of this CTA
       for (long long pos = r0; pos < r1 && ok;) {
         const FwdRun run = fwd_run(p, pos, r1);
+        if (p.k1) {
+          // 1 x 1 layer (the layer that needs no halo, remark after Eq. 7): output row r is the product of input
+          // row r with the centre tap alone -- one view (shifted by one pixel: the box starts at pixel -1), N = 64
+          for (int r = 0; r < run.n && ok; ++r) {
+            const int g = g0 + r, blk = acc_block(g);
+            ok = mbar_wait(smem_u32(&acc_empty_bar[blk]), (g >> 3) & 1u, abortp, p.status, DEV_TIMEOUT_MMA_TMEM);
+            if (!ok) break;
+            ok = mbar_wait(smem_u32(&full_bar[stage]), phase, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t adesc = make_desc(ring + stage * FWD1_ROW_BYTES + 128, 16, 1024);
+            const uint64_t bdesc = make_desc(w_smem + 192 * 128 + 64 * 128, 16, 1024);       // tap (u, v) = (1, 1)
+            const uint32_t idesc = make_idesc(128, 64, 0, 0);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) tc_mma_bf16(tmem_base + blk * 64, adesc + k * 2, bdesc + k * 2, idesc, 1u);
+            tc_commit(smem_u32(&empty_bar[stage]));
+            if (++stage == FWD1_STAGES) { stage = 0; phase ^= 1u; }
+            tc_commit(smem_u32(&acc_full_bar[blk]));
+          }
+          g0 += run.n;
+          pos += run.n;
+          continue;
+        }
         for (int r = 0; r < run.n + 2 && ok; ++r) {
           if (r < run.n) {     // this input row opens output row r: its block must be drained and zeroed
             const int g = g0 + r;
@@ -502,7 +540,9 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       for (; g < n_rows; ++g, advance(cur)) {
         const int buf = g & 1;
         const int x0 = cur.x0, row = cur.row, z = cur.z;
-        const bool valid = PACKED ? (pl_sub < p.W && z + pl_strip < p.Z) : x0 + pl < p.W;
+        // (a row beyond its strip's height is the dead row of a short strip: computed, never stored or counted)
+        const bool valid = (PACKED ? (pl_sub < p.W && z + pl_strip < p.Z) : x0 + pl < p.W) &&
+                           row <= strip_height((z + pl_strip) % p.P_r, p.H, p.P_r);
         const int blk = acc_block(g);
         if (issuer) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store of row g - 2 has read this tile
         asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -572,6 +612,8 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           for (int j = 0; j < pack; ++j) {           // one box per strip of the group; all of them in one bulk group
             const int zj = z + j;
             if (zj >= p.Z) break;
+            const int hs_j = strip_height(zj % p.P_r, p.H, p.P_r);
+            if (row > hs_j) continue;                  // dead row of a short strip
             const uint32_t src = stg_out + buf * FWD_TILE_BYTES + j * sub_bytes;
             asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
                          ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(row), "r"(zj), "r"(src)
@@ -580,9 +622,9 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             // halo row of the strip above / below it in the same image.
             if (row == 1 && p.P_r > 1 && zj % p.P_r > 0)
               asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
-                           ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(p.Hs + 1), "r"(zj - 1), "r"(src)
+                           ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(strip_height(zj % p.P_r - 1, p.H, p.P_r) + 1), "r"(zj - 1), "r"(src)
                            : "memory");
-            if (row == p.Hs && p.P_r > 1 && zj % p.P_r < p.P_r - 1)
+            if (row == hs_j && p.P_r > 1 && zj % p.P_r < p.P_r - 1)
               asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
                            ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(0), "r"(zj + 1), "r"(src)
                            : "memory");
@@ -612,7 +654,9 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 // ------------------------------------------------------------------------------ backward-weight kernel
 struct WgParams {
   int W, Hs, R, nseg;
+  int H, P_r;             // image rows and strips per image (heights of the strips: see strip_height)
   int pack;               // narrow images: strips per 128-pixel block, as in the forward kernel
+  int k1;                 // 1 x 1 layer: a dY row meets its own X row only, and only the centre tap is formed
   long long rows_total;   // dY row segments: (strip group z, segment, row) flattened with the row fastest
   float* part;            // [gridDim.x][9][C][C]
   int* status;
@@ -691,16 +735,20 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         pos += run.n;
         const int z = run.z;
         const int x0 = run.seg * WG_PIX;
-        for (int r = 0; r < run.n + 2 && ok; ++r) {
+        // 3 x 3: n dY rows meet n + 2 X rows (from the row above the first one on); 1 x 1: their own n X rows
+        const int n_x = p.k1 ? run.n : run.n + 2, xrow0 = p.k1 ? run.h0 + 1 : run.h0;
+        for (int r = 0; r < n_x && ok; ++r) {
           if (r < run.n) {
             ok = mbar_wait(smem_u32(&yempty[ys]), yph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
             if (!ok) break;
             const uint32_t fy = smem_u32(&yfull[ys]);
-            const bool mirrored = ys < 2;
+            const bool mirrored = ys < 2 && !p.k1;       // (a 1 x 1 layer reads one dY row at a time: no window)
             mbar_expect_tx(fy, mirrored ? 2 * WG_CHUNK : WG_CHUNK);
             for (int j = 0; j < p.pack; ++j) {     // one box per strip of the group (pixels beyond W and strips beyond Z read as zeros)
-              tma_load_4d(yring + ys * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, run.h0 + r + 1, z + j, fy);
-              if (mirrored) tma_load_4d(yring + (WG_YSTAGES + ys) * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, run.h0 + r + 1, z + j, fy);
+              // the dead row of a short strip holds the neighbour's row (it is that strip's halo row): read the all-zero row instead
+              const int yrow = run.h0 + r + 1 > strip_height((z + j) % p.P_r, p.H, p.P_r) ? p.Hs + 1 : run.h0 + r + 1;
+              tma_load_4d(yring + ys * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, yrow, z + j, fy);
+              if (mirrored) tma_load_4d(yring + (WG_YSTAGES + ys) * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, yrow, z + j, fy);
             }
             if (++ys == WG_YSTAGES) { ys = 0; yph ^= 1u; }
           }
@@ -709,11 +757,11 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           const uint32_t fb = smem_u32(&xfull[xs]);
           if (p.pack == 1) {
             mbar_expect_tx(fb, (WG_PIX + 2) * 128);
-            tma_load_4d(xring + xs * WG_XROW_BYTES, &tmX, 0, x0 - 1, run.h0 + r, z, fb);
+            tma_load_4d(xring + xs * WG_XROW_BYTES, &tmX, 0, x0 - 1, xrow0 + r, z, fb);
           } else {
             mbar_expect_tx(fb, WG_PIX * 128);
             for (int j = 0; j < p.pack; ++j)
-              tma_load_4d(xring + xs * WG_XROW_BYTES + j * sub_bytes, &tmX, 0, -1, run.h0 + r, z + j, fb);
+              tma_load_4d(xring + xs * WG_XROW_BYTES + j * sub_bytes, &tmX, 0, -1, xrow0 + r, z + j, fb);
           }
           if (++xs == WG_XSTAGES) { xs = 0; xph ^= 1u; }
         }
@@ -732,6 +780,27 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         const int npx = p.pack > 1 ? WG_PIX : min(WG_PIX, p.W - run.seg * WG_PIX);
         const int ksteps = (npx + UMMA_K - 1) / UMMA_K;
         int yhave = 0;
+        if (p.k1) {
+          // 1 x 1 layer: dY row r meets X row r; the operand (shift 0 | shift 1) carries the centre tap in its upper
+          // 64 lanes (the lower ones form a tap that is thrown away), the result sits in column block 1 (u = 1)
+          for (int r = 0; r < run.n && ok; ++r) {
+            ok = mbar_wait(smem_u32(&yfull[yw]), ywph, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
+            if (!ok) break;
+            ok = mbar_wait(smem_u32(&xfull[xw]), xwph, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t idesc = make_idesc(128, 64, 1, 1);
+            const uint64_t bdesc = make_desc(yring + yw * WG_CHUNK, WG_CHUNK, 1024);
+            const uint64_t a01 = make_desc(xring + xw * WG_XROW_BYTES, 128, 1024);
+            for (int k = 0; k < ksteps; ++k) tc_mma_bf16(tmem_base + 64, a01 + k * 128, bdesc + k * 128, idesc, 1u);
+            tc_commit(smem_u32(&xempty[xw]));
+            tc_commit(smem_u32(&yempty[yw]));
+            if (++xw == WG_XSTAGES) { xw = 0; xwph ^= 1u; }
+            if (++yw == WG_YSTAGES) { yw = 0; ywph ^= 1u; }
+          }
+          y_slot0 = (y_slot0 + run.n) % WG_YSTAGES;
+          continue;
+        }
         for (int r = 0; r < run.n + 2 && ok; ++r) {
           const int i_hi = min(r, run.n - 1), i_lo = max(0, r - 2);
           while (yhave <= i_hi && ok) {
@@ -895,9 +964,10 @@ namespace {
 void launch_fwd(ConvNet* c, int cls, int layer, const CUtensorMap& in, const CUtensorMap& w, bf16* out, const CUtensorMap& out_tile, int mode,
                 const bf16* mask, const CUtensorMap* mask_tile) {
   FwdParams p;
-  p.W = c->W; p.Hs = c->Hs; p.R = c->R;
+  p.W = c->W; p.Hs = c->Hs; p.R = c->R; p.H = c->H;
   p.nseg = (c->W + FWD_PIX - 1) / FWD_PIX;
   p.pack = c->pack; p.Z = static_cast<int>(c->Z); p.P_r = c->P_r;
+  p.k1 = c->k1[layer] && !getenv("MBD_CONV_1X1_AS_3X3");       // tuning knob: a 1 x 1 layer through all nine taps
   p.rows_total = ((c->Z + c->pack - 1) / c->pack) * p.nseg * c->Hs;
   p.mode = mode; p.out = out; p.mask_src = mask; p.loss_part = c->loss_part; p.status = c->status;
   const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
@@ -925,11 +995,10 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   (void)max_partials;
   if (conv_init() != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
   const int H = layers[0].H, W = layers[0].W;
-  if (H % P_r != 0) return MBD_E_UNSUPPORTED;      // strips of equal height only
   if (B > 65535 || static_cast<int64_t>(H) * W > INT32_MAX) return MBD_E_UNSUPPORTED;   // grid.y of the staging kernels
   ConvNet* c = new (std::nothrow) ConvNet();
   if (!c) return MBD_E_ALLOC;
-  c->L = L; c->B = B; c->H = H; c->W = W; c->P_r = P_r; c->Hs = H / P_r; c->R = c->Hs + 2; c->Z = B * P_r;
+  c->L = L; c->B = B; c->H = H; c->W = W; c->P_r = P_r; c->Hs = (H + P_r - 1) / P_r; c->R = c->Hs + 2; c->Z = B * P_r;
   c->num_sms = num_sms; c->grid = num_sms; c->status = status; c->stream = stream; c->prof = prof;
   c->fc_above = fc_above;
   c->strip_elems = static_cast<size_t>(c->Z) * c->R * W * C;
@@ -1078,9 +1147,10 @@ mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta) {
                c->relu[i - 1] ? c->act[i] : nullptr, c->relu[i - 1] ? &c->act_tile[i] : nullptr);
   }
   WgParams p;
-  p.W = c->W; p.Hs = c->Hs; p.R = c->R;
+  p.W = c->W; p.Hs = c->Hs; p.R = c->R; p.H = c->H; p.P_r = c->P_r;
   p.nseg = (c->W + WG_PIX - 1) / WG_PIX;
   p.pack = c->pack;
+  p.k1 = c->k1[i] && !getenv("MBD_CONV_1X1_AS_3X3");
   p.rows_total = ((c->Z + c->pack - 1) / c->pack) * p.nseg * c->Hs;
   p.part = c->wpart; p.status = c->status;
   const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
@@ -1112,7 +1182,8 @@ mbd_status conv_outer_rows(ConvNet* c, int which, int layer, int side, void* row
   bf16* buf = which == MBD_T_ACT ? c->act[layer + 1] : (which == MBD_T_DY && layer >= 0) ? c->dY[layer] : nullptr;
   if (!buf) return MBD_E_INVALID;
   const int strip = side == 0 ? 0 : c->P_r - 1;
-  const int row = set ? (side == 0 ? 0 : c->Hs + 1) : (side == 0 ? 1 : c->Hs);
+  const int hs_last = strip_height(c->P_r - 1, c->H, c->P_r);      // the bottom strip may be shorter than the row slots
+  const int row = set ? (side == 0 ? 0 : hs_last + 1) : (side == 0 ? 1 : hs_last);
   const int per_image = c->W * C / 8;                       // 16-byte pieces per row
   dim3 g((per_image + 255) / 256, static_cast<unsigned>(c->B));
   outer_rows_kernel<<<g, 256, 0, c->stream>>>(buf, static_cast<bf16*>(rows), c->W, c->P_r, c->R, strip, row, set);

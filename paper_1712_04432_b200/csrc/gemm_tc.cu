@@ -897,7 +897,10 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
     const int kb_piece = kb_total / (g.k_splits > 0 ? g.k_splits : 1);
     // ... and a piece's main loop must be long enough to hide the epilogue of the piece before it (which reads
     // the sum back row by row): short pieces are better served by S planes and the coalesced reduction kernel
-    g.fix = g.allow_fix && g.pair && g.k_splits > 1 && tiles >= slots && kb_piece >= 32 ? 1 : 0;
+    // ... and there must be just two of them: with more, most epilogues read a plane back and the step loses
+    // (cfg5 with four pieces: 27 ms against 21 ms with two); the kernel itself handles any S.
+    const bool two = g.k_splits == 2 || (g.k_splits > 2 && getenv("MBD_FIX_ANY_S") != nullptr);     // tuning knob
+    g.fix = g.allow_fix && g.pair && two && tiles >= slots && kb_piece >= 32 ? 1 : 0;
     g.flag_words = g.fix ? tiles * 32 : 0;
   }
   // TMA epilogue: bf16 output of an unsplit contraction on 128-row tiles

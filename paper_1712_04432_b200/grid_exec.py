@@ -60,21 +60,26 @@ class GridComm:
                 self.col_group = g
         self.words: Dict[str, float] = {"allgather_y": 0.0, "allreduce_dx": 0.0, "allreduce_dw": 0.0}
 
-    def all_gather_cols(self, block, out, kind="allgather_y"):
-        """out[:, r' * n : (r' + 1) * n] = block of process r' of the P_r group, for every r'."""
+    def all_gather_cols(self, block, out, kind="allgather_y", scratch=None):
+        """out[:, r' * n : (r' + 1) * n] = block of process r' of the P_r group, for every r'.
+
+        One collective into one buffer [P_r, m, n] (`scratch`, allocated here if not given) and one strided
+        copy that puts block r' into its columns of `out` [m, P_r n]."""
         import torch
-        p, n = self.P_r, block.shape[1]
-        assert out.shape[1] == p * n and out.shape[0] == block.shape[0]
+        p, (m, n) = self.P_r, block.shape
+        assert out.shape[1] == p * n and out.shape[0] == m and out.is_contiguous()
         if p == 1:
             out.copy_(block)
             return out
         src = block.contiguous()
         if self.via_host:
             src = src.cpu()
-        parts = [torch.empty_like(src) for _ in range(p)]
-        self.dist.all_gather(parts, src, group=self.row_group)
-        for j in range(p):
-            out[:, j * n:(j + 1) * n].copy_(parts[j])
+            buf = torch.empty((p, m, n), dtype=src.dtype)
+        else:
+            buf = scratch if scratch is not None else torch.empty((p, m, n), dtype=src.dtype, device=src.device)
+        assert tuple(buf.shape) == (p, m, n) and buf.is_contiguous()
+        self.dist.all_gather_into_tensor(buf.view(p * m, n), src, group=self.row_group)
+        out.view(m, p, n).copy_(buf.permute(1, 0, 2))
         self.words[kind] += (p - 1) * block.numel()
         return out
 
@@ -140,7 +145,27 @@ class GridFC:
         self.W: List = [torch.zeros((self.dims[i + 1] // P_r, self.dims[i]), dtype=torch.bfloat16, device=device)
                         for i in range(self.L)]
         self.dW: List = [None] * self.L            # summed fp32 gradients of the last step (kept for inspection)
-        self.status = torch.zeros(1, dtype=torch.int32, device=device)   # bounded-wait status word of the block products
+        # Every buffer of a step is allocated once, here: per layer the block product's output, the landing buffer
+        # of the all-gather, the gathered activation, the fp32 summand of dX and of dW, the masked gradient.
+        m, L, d = self.m, self.L, self.dims
+        f32, bf = torch.float32, torch.bfloat16
+
+        def buf(shape, dtype):
+            return torch.empty(shape, dtype=dtype, device=device)
+
+        self._blk = [buf((m, d[i + 1] // P_r), f32 if i == L - 1 else bf) for i in range(L)]
+        self._gat = [buf((P_r, m, d[i + 1] // P_r), f32 if i == L - 1 else bf) if P_r > 1 else None for i in range(L)]
+        self._act = [None] + [buf((m, d[i + 1]), f32 if i == L - 1 else bf) for i in range(L)]
+        self._part = [buf((m, d[i]), f32) for i in range(L)]
+        self._dYprev = [buf((m, d[i]), bf) for i in range(L)]
+        self._g = [buf((d[i + 1] // P_r, d[i]), f32) for i in range(L)]
+        self._dYtop = buf((m, d[L]), bf)
+        self._per = buf((m,), f32)
+        # word 0: bounded-wait status of the block products; word 1: the bits of this block's loss sum.  Read
+        # back together, once, at the end of a step.
+        self._tail = torch.zeros(2, dtype=torch.int32, device=device)
+        self.status = self._tail[0:1]
+        self._loss = self._tail[1:2].view(torch.float32)
 
     def _update(self, pending, scale: float):
         """Waits for the all-reduce of dW_i started earlier and applies Eq. 1 to the owned rows."""
@@ -167,48 +192,50 @@ class GridFC:
         t, comm = self.t, self.comm
         m, L = self.m, self.L
         assert tuple(X_c.shape) == (m, self.dims[0]) and X_c.dtype == t.bfloat16
-        acts = [X_c.contiguous()]
+        acts = self._act
+        acts[0] = X_c.contiguous()
         # ---- forward: block product, then the all-gather over the P_r group (Appendix A.1)
         for i in range(L):
             last = i == L - 1
-            h = self.dims[i + 1] // comm.P_r
-            blk = t.empty((m, h), dtype=t.float32 if last else t.bfloat16, device=self.device)
-            mbd.block_gemm(0, acts[i], self.W[i], blk, mbd.TAIL_STORE, relu=not last, status=self.status)
-            full = t.empty((m, self.dims[i + 1]), dtype=blk.dtype, device=self.device)
-            comm.all_gather_cols(blk, full)
-            acts.append(full)
+            mbd.block_gemm(0, acts[i], self.W[i], self._blk[i], mbd.TAIL_STORE, relu=not last, status=self.status)
+            comm.all_gather_cols(self._blk[i], acts[i + 1], scratch=self._gat[i])
         self.logits = acts[L]
-        # ---- loss and top gradient (every process of a P_r group holds the full logits of its samples)
-        dY = t.empty((m, self.dims[L]), dtype=t.bfloat16, device=self.device)
-        per = t.empty((m,), dtype=t.float32, device=self.device)
-        mbd.softmax_xent(self.logits, labels_c, dY, per, sync=False)
-        loss = float(per.double().sum().item())
+        # ---- loss and top gradient (every process of a P_r group holds the full logits of its samples); the
+        # block's losses are added, in sample order, by the library's reduction (S = m planes of one element)
+        dY = self._dYtop
+        mbd.softmax_xent(self.logits, labels_c, dY, self._per, sync=False)
+        mbd.block_reduce(self._per.view(m, 1, 1), self._loss.view(1, 1), mbd.TAIL_STORE, sync=False)
         # ---- backward (Appendix A.2)
         scale = -float(eta) / self.B
-        pending = None                                                  # the all-reduce of the layer above, in flight
+        pending = None                                                  # the all-reduce of dW of the layer above, in flight
         for i in range(L - 1, -1, -1):
             a, b = self.rows(i)
             dY_r = dY[:, a:b]                                           # dY_i(r, c): this process's rows of layer i's output
-            dY_prev = None
-            if i > 0 or input_is_relu_output:
-                part = t.empty((m, self.dims[i]), dtype=t.float32, device=self.device)
+            need_dx = i > 0 or input_is_relu_output
+            hx = None
+            if need_dx:
+                part = self._part[i]
                 mbd.block_gemm(1, dY_r, self.W[i], part, mbd.TAIL_STORE, status=self.status)       # W_i(r, :)^T dY_i(r, c), one summand
-                comm.all_reduce_(part, "rows", "allreduce_dx")
-                dY_prev = t.empty((m, self.dims[i]), dtype=t.bfloat16, device=self.device)
-                mbd.block_reduce(part, dY_prev, mbd.TAIL_MASK, mask=acts[i], sync=False)   # ReLU derivative from the stored X_i
-            g = t.empty((b - a, self.dims[i]), dtype=t.float32, device=self.device)
+                hx = comm.all_reduce_start(part, "rows", "allreduce_dx")          # in flight beside the dW product below
+            g = self._g[i]
             mbd.block_gemm(2, dY_r, acts[i], g, mbd.TAIL_STORE, status=self.status)                # dY_i(r, c) X_i(:, c)^T, one summand
             handle = comm.all_reduce_start(g, "cols", "allreduce_dw")          # runs beside the products of layer i - 1
             if pending is not None:
                 self._update(pending, scale)
             pending = (i, handle)
+            dY_prev = None
+            if need_dx:
+                part = comm.all_reduce_finish(hx)
+                dY_prev = self._dYprev[i]
+                mbd.block_reduce(part, dY_prev, mbd.TAIL_MASK, mask=acts[i], sync=False)   # ReLU derivative from the stored X_i
             dY = dY_prev
         self.dX0 = dY                                                   # None unless input_is_relu_output
         self._update(pending, scale)
-        if int(self.status.item()) != 0:             # (synchronises) a bounded wait inside a product gave up
-            self.status.zero_()
+        tail = self._tail.cpu()                      # (synchronises) status word and loss in one copy
+        if int(tail[0]) != 0:                        # a bounded wait inside a product gave up
+            self._tail.zero_()
             raise mbd.MbdError(mbd.E_TIMEOUT, "grid step")
-        return loss
+        return float(tail[1:2].view(t.float32).item())
 
 
 class GridConv:
@@ -225,11 +252,13 @@ class GridConv:
         self.comm = comm
         self.loss = loss
         P_r, P_c = comm.P_r, comm.P_c
-        if H % P_r or B % P_c:
-            raise ValueError("H must divide into P_r strips and the batch into P_c blocks")
+        if B % P_c or P_r > H:
+            raise ValueError("the batch must divide into P_c blocks and every strip needs a row")
         self.ksizes = [int(k) for k in ksizes]
         self.L = len(self.ksizes)
-        self.C, self.Hs, self.W, self.m = int(C_), H // P_r, int(W), B // P_c
+        # strip r of the image: the balanced range of rows [floor(r H / P_r), floor((r + 1) H / P_r))
+        self.h0, self.h1 = (comm.r * H) // P_r, ((comm.r + 1) * H) // P_r
+        self.C, self.Hs, self.W, self.m = int(C_), self.h1 - self.h0, int(W), B // P_c
         self.net = mbd.Net(mbd.conv_layers(self.L, C_, self.Hs, W, k=self.ksizes), self.m, 1, 1, mbd.BF16, loss, 0)
         comm.words.setdefault("halo_fwd", 0.0)
         comm.words.setdefault("halo_bwd", 0.0)
@@ -315,6 +344,8 @@ class GridMixed:
     def __init__(self, ksizes: Sequence[int], C_: int, H: int, W: int, fc_dims: Sequence[int], B: int, comm: GridComm):
         self.comm = comm
         self.C, self.H, self.W = int(C_), int(H), int(W)
+        if H % comm.P_r:
+            raise ValueError("the all-gather between the convolutions and the fully connected layers wants equal strips")
         self.conv = GridConv(ksizes, C_, H, W, B, comm, loss=mbd.LOSS_NONE)
         self.fc = GridFC([C_ * H * W] + [int(d) for d in fc_dims], B, comm)
         comm.words.setdefault("redistribute", 0.0)

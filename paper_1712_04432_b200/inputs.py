@@ -96,6 +96,11 @@ WORKLOADS["mixed"] = mixed_workload(64, 56, 56, 2, (1024, 1024, 1000), 256, name
                                     grids=[(1, 1), (4, 4), (8, 1), (2, 8)])
 
 
+# The layers the paper singles out as needing no halo exchange (remark after Eq. 7): cfg4's stack with 1 x 1 kernels.
+WORKLOADS["conv1x1"] = Workload("conv1x1", "conv", (64, 224, 224), 32, "bf16", "normal", "half_ssq", eta=1e-7,
+                                n_layers=2, grids=[(1, 1), (2, 1), (4, 1), (8, 1)], ksizes=(1, 1))
+
+
 def fc_workload(dims, B, dtype="bf16", x_dist="normal", name="custom") -> Workload:
     return Workload(name, "fc", tuple(int(d) for d in dims), int(B), dtype, x_dist, "softmax_ce")
 

@@ -100,14 +100,21 @@ def sized_eta(c):
     return c["eta"]
 
 
-@pytest.mark.parametrize("grid,mp,bench_plan", [((16, 16), 2, True), ((1, 1), 1, False), ((64, 4), 2, False), ((4, 64), 2, False),
-                                                ((16, 16), 4, False)])       # four pieces per sum: a running sum over three hand-overs
-def test_cfg5_listed_grids_fused_step(cfg5, grid, mp, bench_plan):
+@pytest.mark.parametrize("grid,mp,bench_plan,any_s", [((16, 16), 2, True, False), ((1, 1), 1, False, False), ((64, 4), 2, False, False),
+                                                      ((4, 64), 2, False, False),
+                                                      ((16, 16), 4, False, False),     # four planes and the reduction kernel
+                                                      ((16, 16), 4, False, True)])     # four pieces as a running sum (tuning knob)
+def test_cfg5_listed_grids_fused_step(monkeypatch, cfg5, grid, mp, bench_plan, any_s):
     from oracle import mbd_oracle as O
     from paper_1712_04432_b200 import mbd
     c, o = cfg5, cfg5["o"]
     eta = sized_eta(c)
+    if any_s:
+        monkeypatch.setenv("MBD_FIX_ANY_S", "1")
     net = make_net(c, grid, mp)
+    if mp == 4:
+        p = net.plan(3, 2)
+        assert (p["k_pieces"], p["running_sum"]) == (4, 1 if any_s else 0), p
     if bench_plan:
         # what `bench.py` launches by default: unsplit forward products on 512 x 256 CTA-pair tiles, both backward
         # products cut in two pieces on 256 x 256 CTA-pair tiles, the pieces added as a running sum in the epilogue

@@ -163,8 +163,8 @@ inp = I.make_inputs(w, seed=%(seed)d)                      # every process draws
 net = GridConv(ksizes, 64, H, W, B, comm)
 for i in range(len(ksizes)):
     net.set_weights(i, to_dev(inp.Ws[i], True))
-m, Hs = B // P_c, H // P_r
-X_local = to_dev(np.ascontiguousarray(inp.X[comm.c * m:(comm.c + 1) * m, :, comm.r * Hs:(comm.r + 1) * Hs, :]), True)
+m = B // P_c
+X_local = to_dev(np.ascontiguousarray(inp.X[comm.c * m:(comm.c + 1) * m, :, net.h0:net.h1, :]), True)
 loss = net.step(X_local, eta)
 torch.cuda.synchronize()
 L = len(ksizes)
@@ -181,11 +181,12 @@ dist.destroy_process_group()
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("P_r,P_c,ksizes", [(2, 1, (3, 3)), (2, 2, (3, 1, 3)), (4, 1, (3, 3, 3)), (1, 2, (3, 3))])
-def test_convolution_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, P_r, P_c, ksizes):
+@pytest.mark.parametrize("P_r,P_c,ksizes,H", [(2, 1, (3, 3), 16), (2, 2, (3, 1, 3), 16), (4, 1, (3, 3, 3), 16), (1, 2, (3, 3), 16),
+                                              (3, 1, (3, 3), 10)])       # 10 rows on 3 processes: strips of 3, 3 and 4 rows
+def test_convolution_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, P_r, P_c, ksizes, H):
     from paper_1712_04432_b200 import inputs as I
     from tests.helpers import like_device, oracle_conv_step, rel_fro
-    H, W, B, eta, seed = 16, 40, 4, 2e-5, 92
+    W, B, eta, seed = 40, 4, 2e-5, 92
     script = tmp_path / "conv_worker.py"
     script.write_text(CONV_WORKER % {"root": ROOT, "P_r": P_r, "P_c": P_c, "ksizes": list(ksizes), "H": H, "W": W, "B": B,
                                      "eta": eta, "out": str(tmp_path), "seed": seed})
@@ -196,13 +197,13 @@ def test_convolution_step_over_a_grid_of_processes_matches_the_oracle(tmp_path, 
     w.eta = eta
     inp = I.make_inputs(w, seed=seed)
     o = oracle_conv_step(w, inp)
-    L, m, Hs = len(ksizes), B // P_c, H // P_r
+    L, m = len(ksizes), B // P_c
     loss = 0.0
     for rank in range(P_r * P_c):
         z = np.load(tmp_path / f"rank{rank}.npz")
         rr, cc = int(z["r"]), int(z["c"])
         loss += float(z["loss"])
-        own = (slice(cc * m, (cc + 1) * m), slice(None), slice(rr * Hs, (rr + 1) * Hs), slice(None))
+        own = (slice(cc * m, (cc + 1) * m), slice(None), slice((rr * H) // P_r, ((rr + 1) * H) // P_r), slice(None))
         assert rel_fro(z["Y"], o["Ys"][L - 1][own]) < 1e-2, rank                 # this strip of the last layer's output
         assert rel_fro(z["dY0"], o["dYs"][0][own]) < 1e-2, rank                  # ... and of the gradient that reached layer 1
         for i in range(L):

@@ -170,6 +170,47 @@ def test_one_by_one_layers(ksizes, P_r, fused):
     compare_conv_step(g, o, TOL, fused)
 
 
+@pytest.mark.parametrize("H,W,B,P_r,ksizes", [(10, 40, 2, 3, (3, 3)), (7, 130, 3, 2, (3, 3, 3)), (9, 64, 2, 4, (3, 1, 3)), (28, 130, 2, 5, (3, 3)),
+                                              (10, 30, 5, 3, (3, 3)), (11, 14, 3, 4, (1, 3)), (5, 224, 1, 5, (3, 3)), (13, 40, 2, 7, (3, 3))])
+@pytest.mark.parametrize("fused", [False, True])
+def test_strips_of_unequal_height(H, W, B, P_r, ksizes, fused):
+    """H is not a multiple of P_r: the strips are the balanced ranges [floor(s H / P_r), floor((s + 1) H / P_r)), one row
+    apart in height (heights 4, 3, 3 for 10 rows on 3 strips; down to single-row strips) -- on wide, ragged and
+    tile-sharing narrow images, with 1 x 1 layers in between; against the whole-image oracle and the oracle that
+    forms the same strips with their halo rows."""
+    w = I.conv_workload(64, H, W, B, n_layers=len(ksizes), name="conv_unequal", ksizes=ksizes)
+    inp = I.make_inputs(w, seed=90 + H + W)
+    o = oracle_conv_step(w, inp)
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    o = oracle_with_eta(o, inp.Ws, inp.bs, w.B, eta)
+    g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o), eta=eta)
+    compare_conv_step(g, o, TOL, fused, init=inp, require_sized=True)
+    assert abs(g["J"] - o["J"]) <= 1e-3 * abs(o["J"])            # the dead row of a short strip is not counted in the loss
+    if not fused:
+        ob = oracle_with_eta(oracle_conv_step(w, inp, strips=P_r), inp.Ws, inp.bs, w.B, eta)
+        compare_conv_step(g, ob, TOL)
+        one = gpu_conv_step(w, inp, 1, force_acts=stored_hidden(o), eta=eta)      # one strip: the same sums in another order
+        for i in range(len(ksizes)):
+            assert np.array_equal(g["act"][i], one["act"][i]) and np.array_equal(g["dY"][i], one["dY"][i]), i
+
+
+@pytest.mark.parametrize("H,W,B,P_r,ksizes", [(8, 130, 3, 2, (1, 3, 1)), (8, 30, 5, 2, (1, 1)), (6, 14, 3, 3, (3, 1)), (12, 224, 2, 3, (1,))])
+def test_one_by_one_layers_have_a_path_of_their_own(monkeypatch, H, W, B, P_r, ksizes):
+    """A 1 x 1 layer reads one input row per output row and forms one tap (remark after Eq. 7: the layer that needs no
+    halo); run instead as a 3 x 3 layer whose outer taps are zero it adds exact zeros to the same sums in the same
+    order, so the two ways must agree bit for bit -- on wide, ragged and tile-sharing narrow images."""
+    w = I.conv_workload(64, H, W, B, n_layers=len(ksizes), name="conv_1x1_path", ksizes=ksizes)
+    inp = I.make_inputs(w, seed=80 + W)
+    o = oracle_conv_step(w, inp)
+    a = gpu_conv_step(w, inp, P_r, force_acts=stored_hidden(o))
+    compare_conv_step(a, o, TOL)
+    monkeypatch.setenv("MBD_CONV_1X1_AS_3X3", "1")
+    b = gpu_conv_step(w, inp, P_r, force_acts=stored_hidden(o))
+    for i in range(len(ksizes)):
+        assert np.array_equal(a["act"][i], b["act"][i]) and np.array_equal(a["dY"][i], b["dY"][i]), i
+        assert np.array_equal(a["dW"][i], b["dW"][i]) and np.array_equal(a["new_W"][i], b["new_W"][i]), i
+
+
 def test_step_piece_by_piece_equals_the_whole_step():
     """mbd_forward / mbd_backward are the stepped calls in a row: same loss and, bit for bit, the same updated
     kernels; and halo rows written from outside are what the next layer reads (a strip cut out of a taller image

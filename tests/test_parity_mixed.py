@@ -62,6 +62,18 @@ def test_one_convolution_three_fc_layers_ragged():
         compare_mixed_step(g, o, w, TOL)
 
 
+def test_unequal_strips_under_fully_connected_layers():
+    # 10 rows on 3 and 4 strips (heights 4, 3, 3 and 3, 2, 3, 2), batch split as well; then 25600 -> 64 -> 16
+    w = I.mixed_workload(64, 10, 40, 2, (64, 16), 6, name="mixed_unequal")
+    inp = I.make_inputs(w, seed=34)
+    o = oracle_mixed_step(w, inp)
+    for grid in [(3, 2), (4, 3)]:
+        g = gpu_mixed_step(w, inp, grid, 4, force_acts=oracle_mixed_acts(o, w))
+        compare_mixed_step(g, o, w, TOL)
+        g = gpu_mixed_step(w, inp, grid, 4, fused=True, force_acts=oracle_mixed_acts(o, w))
+        compare_mixed_step(g, o, w, TOL, fused=True)
+
+
 def test_train_step_graph_matches_separate_calls(small):
     """mbd_train_step (captured graph, fused update) leaves the same weights, bit for bit, as
     forward + backward(eta) issued one by one; and two steps change them twice."""
