@@ -375,10 +375,22 @@ MBD_API mbd_status mbd_softmax_xent(const float* logits_dev, int64_t B, int64_t 
  * row; set != 0 writes the upper (side 0) or lower (side 1) HALO row, which is zero (the image border)
  * unless written.  which = MBD_T_ACT (output of `layer`; layer -1 = the staged input) or MBD_T_DY.
  * mbd_set_tensor(MBD_T_DW) on a convolution stack replaces the materialised weight gradient (e.g. by its
- * sum over all processes) before mbd_sgd_step. */
+ * sum over all processes) before mbd_sgd_step.
+ *
+ * Section 2.2's overlap of the halo exchange with the interior computation: the _rows forms compute part of a
+ * layer.  MBD_ROWS_INTERIOR = the own rows 2 .. H - 1, which read no halo row of the layer's input (forward) or of
+ * dY_layer (backward): they can be enqueued while the halo rows are still travelling; MBD_ROWS_BOUNDARY = rows 1 and
+ * H, after the halo rows have been written -- and, in the backward form, the layer's weight gradient (and update)
+ * after them.  A 1x1 layer reads no halo: all of its rows are interior, its boundary call only finishes the layer.
+ * INTERIOR then BOUNDARY leaves bit for bit the tensors MBD_ROWS_ALL (= the plain call) leaves (the loss sum adds
+ * the same squares in another order).  One strip per network only
+ * (P_r = 1: the network of one process), MBD_E_UNSUPPORTED otherwise. */
+enum { MBD_ROWS_ALL = 0, MBD_ROWS_INTERIOR = 1, MBD_ROWS_BOUNDARY = 2 };
 MBD_API mbd_status mbd_conv_stage_input(mbd_net* net, const void* X_dev);
 MBD_API mbd_status mbd_conv_forward_layer(mbd_net* net, int layer, float* loss_sum_dev);
 MBD_API mbd_status mbd_conv_backward_layer(mbd_net* net, int layer, float fused_eta);
+MBD_API mbd_status mbd_conv_forward_layer_rows(mbd_net* net, int layer, int rows, float* loss_sum_dev);
+MBD_API mbd_status mbd_conv_backward_layer_rows(mbd_net* net, int layer, int rows, float fused_eta);
 MBD_API mbd_status mbd_conv_outer_rows(mbd_net* net, int which, int layer, int side, void* rows_dev,
                                size_t bytes, int set);
 

@@ -281,6 +281,8 @@ struct FwdParams {
   int pack, Z;            // narrow images: `pack` strips share one 128-pixel tile, 128 / pack pixels each (see below)
   int P_r;                // strips per image: a boundary row is also stored into the neighbouring strip's halo row
   int k1;                 // 1 x 1 layer: an output row reads its own input row only, through the centre tap only
+  int row_lo, nrows;      // the own rows this launch computes: row_lo .. row_lo + nrows - 1 (1-based; all of them: 1, Hs)
+  int loss_add;           // MODE_STORE_SSQ: add to the per-CTA loss partials instead of overwriting them
   long long rows_total;   // output row segments: (strip group z, segment, row) flattened with the row fastest
   int mode;
   bf16* out;              // strips
@@ -302,11 +304,12 @@ struct FwdRun {
   int z, seg, h0, n;
 };
 __device__ __forceinline__ FwdRun fwd_run(const FwdParams& p, long long pos, long long end) {
-  const long long col = pos / p.Hs;
+  const long long col = pos / p.nrows;
   FwdRun r;
-  r.h0 = static_cast<int>(pos - col * p.Hs);
+  const int k = static_cast<int>(pos - col * p.nrows);       // position inside the launch's row range
+  r.h0 = p.row_lo - 1 + k;
   const long long left = end - pos;
-  r.n = static_cast<int>(left < p.Hs - r.h0 ? left : p.Hs - r.h0);
+  r.n = static_cast<int>(left < p.nrows - k ? left : p.nrows - k);
   r.seg = static_cast<int>(col % p.nseg);
   r.z = static_cast<int>(col / p.nseg) * p.pack;
   return r;
@@ -506,16 +509,16 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       // (no divisions inside the loop): `cur` is the row being drained, `ahead` the one whose mask is loaded.
       struct Pos { int x0, row, z; };
       auto pos_at = [&](long long pos) {
-        const long long col = pos / p.Hs;
+        const long long col = pos / p.nrows;
         Pos q;
         q.z = static_cast<int>(col / p.nseg) * pack;
         q.x0 = static_cast<int>(col % p.nseg) * FWD_PIX;
-        q.row = static_cast<int>(pos - col * p.Hs) + 1;
+        q.row = static_cast<int>(pos - col * p.nrows) + p.row_lo;
         return q;
       };
       auto advance = [&](Pos& q) {
-        if (++q.row > p.Hs) {
-          q.row = 1;
+        if (++q.row >= p.row_lo + p.nrows) {
+          q.row = p.row_lo;
           q.x0 += FWD_PIX;
           if (q.x0 >= p.nseg * FWD_PIX) { q.x0 = 0; q.z += pack; }
         }
@@ -638,7 +641,10 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     if (p.mode == MODE_STORE_SSQ) {
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, o);
-      if (lane == 0) p.loss_part[blockIdx.x * 8 + (warp - 2)] = ssq;
+      if (lane == 0) {
+        float* slot = p.loss_part + blockIdx.x * 8 + (warp - 2);
+        *slot = p.loss_add ? *slot + ssq : ssq;
+      }
     }
   }
 
@@ -961,18 +967,22 @@ struct ConvNet {
 
 namespace {
 
+// row_lo / nrows: the own rows to compute (default: all Hs of them); loss_add: see FwdParams
 void launch_fwd(ConvNet* c, int cls, int layer, const CUtensorMap& in, const CUtensorMap& w, bf16* out, const CUtensorMap& out_tile, int mode,
-                const bf16* mask, const CUtensorMap* mask_tile) {
+                const bf16* mask, const CUtensorMap* mask_tile, int row_lo = 1, int nrows = -1, int loss_add = 0) {
   FwdParams p;
+  if (nrows < 0) nrows = c->Hs;
+  if (nrows == 0) return;
+  p.row_lo = row_lo; p.nrows = nrows; p.loss_add = loss_add;
   p.W = c->W; p.Hs = c->Hs; p.R = c->R; p.H = c->H;
   p.nseg = (c->W + FWD_PIX - 1) / FWD_PIX;
   p.pack = c->pack; p.Z = static_cast<int>(c->Z); p.P_r = c->P_r;
   p.k1 = c->k1[layer] && !getenv("MBD_CONV_1X1_AS_3X3");       // tuning knob: a 1 x 1 layer through all nine taps
-  p.rows_total = ((c->Z + c->pack - 1) / c->pack) * p.nseg * c->Hs;
+  p.rows_total = ((c->Z + c->pack - 1) / c->pack) * p.nseg * nrows;
   p.mode = mode; p.out = out; p.mask_src = mask; p.loss_part = c->loss_part; p.status = c->status;
   const int grid = p.rows_total < c->grid ? static_cast<int>(p.rows_total) : c->grid;
-  if (mode == MODE_STORE_SSQ) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 8, c->stream);
-  const double flops = 2.0 * c->B * c->H * c->W * (c->k1[layer] ? 1.0 : 9.0) * C * C;   // the method's flops, not the kernel's
+  if (mode == MODE_STORE_SSQ && !loss_add) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 8, c->stream);
+  const double flops = 2.0 * c->B * c->H * c->W * (c->k1[layer] ? 1.0 : 9.0) * C * C * nrows / c->Hs;   // the method's flops, not the kernel's
   c->prof->begin(cls, flops);
   if (c->pack > 1)
     launch_pdl(conv_fwd_kernel<true>, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, out_tile, mask_tile ? *mask_tile : out_tile, p);
@@ -1113,13 +1123,40 @@ mbd_status conv_stage_input(ConvNet* c, const void* X_nchw) {
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
-mbd_status conv_forward_layer(ConvNet* c, int i, float* loss_sum_dev) {
+namespace {
+// Section 2.2: "the halo exchange can be overlapped with the interior computation".  With one strip per network
+// (a process of a multi-process driver) the rows 2 .. Hs - 1 of a 3 x 3 layer's output read no halo row: they
+// are the interior, computable while the halo rows travel; rows 1 and Hs are the boundary.  A 1 x 1 layer reads
+// no halo at all: all of its rows are interior.  Calls `launch(row_lo, nrows, first)` for the ranges of `rows`.
+template <typename F>
+void for_rows(const ConvNet* c, int layer, int rows, F launch) {
+  const int Hs = c->Hs;
+  if (rows == MBD_ROWS_ALL) { launch(1, Hs, true); return; }
+  if (c->k1[layer]) {
+    if (rows == MBD_ROWS_INTERIOR) launch(1, Hs, true);
+    return;
+  }
+  if (rows == MBD_ROWS_INTERIOR) {
+    if (Hs > 2) launch(2, Hs - 2, true);
+  } else {
+    launch(1, 1, Hs <= 2);                     // with no interior rows the boundary launch is the first one
+    if (Hs > 1) launch(Hs, 1, false);
+  }
+}
+}  // namespace
+
+mbd_status conv_forward_layer(ConvNet* c, int i, float* loss_sum_dev, int rows) {
   if (i < 0 || i >= c->L) return MBD_E_INVALID;
+  if (rows != MBD_ROWS_ALL && (c->P_r != 1 || (rows != MBD_ROWS_INTERIOR && rows != MBD_ROWS_BOUNDARY))) return MBD_E_UNSUPPORTED;
   const bool last = i == c->L - 1;
   // forward halo exchange (first halo term of Eq. 7): the kernel that produced act[i] (or the staging pass,
   // for the network input) has already stored its boundary rows into the neighbouring strips' halo rows
-  launch_fwd(c, MBD_K_CONV_FWD, i, c->act_fwd[i], c->wf_map[i], c->act[i + 1], c->act_tile[i + 1],
-             (last && !c->fc_above) ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK), nullptr, nullptr);
+  const int mode = (last && !c->fc_above) ? MODE_STORE_SSQ : (c->relu[i] ? MODE_RELU_STORE : MODE_MASK);
+  for_rows(c, i, rows, [&](int row_lo, int nrows, bool first) {
+    launch_fwd(c, MBD_K_CONV_FWD, i, c->act_fwd[i], c->wf_map[i], c->act[i + 1], c->act_tile[i + 1], mode, nullptr, nullptr,
+               row_lo, nrows, first ? 0 : 1);          // a later launch of the same layer adds to the loss partials
+  });
+  if (rows == MBD_ROWS_INTERIOR) return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;   // the boundary rows complete the layer
   if (last && loss_sum_dev && !c->fc_above) {
     c->prof->begin(MBD_K_OTHER, c->grid * 32.0);
     if (sum_f32_launch(c->loss_part, c->grid * 8, 0.5f, loss_sum_dev, c->stream) != cudaSuccess) return MBD_E_CUDA;
@@ -1132,20 +1169,24 @@ mbd_status conv_forward_layer(ConvNet* c, int i, float* loss_sum_dev) {
 
 mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
   mbd_status s = conv_stage_input(c, X_nchw);
-  for (int i = 0; i < c->L && s == MBD_OK; ++i) s = conv_forward_layer(c, i, loss_sum_dev);
+  for (int i = 0; i < c->L && s == MBD_OK; ++i) s = conv_forward_layer(c, i, loss_sum_dev, MBD_ROWS_ALL);
   return s;
 }
 
-mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta) {
+mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta, int rows) {
   if (i < 0 || i >= c->L) return MBD_E_INVALID;
+  if (rows != MBD_ROWS_ALL && (c->P_r != 1 || (rows != MBD_ROWS_INTERIOR && rows != MBD_ROWS_BOUNDARY))) return MBD_E_UNSUPPORTED;
   const bool fused = fused_eta > 0.f;
   const float scale = -fused_eta / static_cast<float>(c->B);
   if (i > 0) {
     // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0]
     // (the producer of dY_i has stored its boundary rows into the neighbours' halo rows)
-    launch_fwd(c, MBD_K_CONV_BWD_DATA, i, c->dY_fwd[i], c->wb_map[i], c->dY[i - 1], c->dY_tile[i - 1], MODE_MASK,
-               c->relu[i - 1] ? c->act[i] : nullptr, c->relu[i - 1] ? &c->act_tile[i] : nullptr);
+    for_rows(c, i, rows, [&](int row_lo, int nrows, bool) {
+      launch_fwd(c, MBD_K_CONV_BWD_DATA, i, c->dY_fwd[i], c->wb_map[i], c->dY[i - 1], c->dY_tile[i - 1], MODE_MASK,
+                 c->relu[i - 1] ? c->act[i] : nullptr, c->relu[i - 1] ? &c->act_tile[i] : nullptr, row_lo, nrows);
+    });
   }
+  if (rows == MBD_ROWS_INTERIOR) return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;   // the weight gradient follows the boundary rows
   WgParams p;
   p.W = c->W; p.Hs = c->Hs; p.R = c->R; p.H = c->H; p.P_r = c->P_r;
   p.nseg = (c->W + WG_PIX - 1) / WG_PIX;
@@ -1169,7 +1210,7 @@ mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta) {
 
 mbd_status conv_backward(ConvNet* c, float fused_eta) {
   mbd_status s = MBD_OK;
-  for (int i = c->L - 1; i >= 0 && s == MBD_OK; --i) s = conv_backward_layer(c, i, fused_eta);
+  for (int i = c->L - 1; i >= 0 && s == MBD_OK; --i) s = conv_backward_layer(c, i, fused_eta, MBD_ROWS_ALL);
   return s;
 }
 

@@ -27,8 +27,9 @@ int conv_last_relu(const ConvNet* c);
 mbd_status conv_enable_master(ConvNet* c);     // fp32 master weights from now on
 // the step piece by piece, and the outer rows of the images (for a driver with one process per strip)
 mbd_status conv_stage_input(ConvNet* c, const void* X_nchw);
-mbd_status conv_forward_layer(ConvNet* c, int layer, float* loss_sum_dev);
-mbd_status conv_backward_layer(ConvNet* c, int layer, float fused_eta);
+// rows: MBD_ROWS_ALL, or (one strip per network only) MBD_ROWS_INTERIOR / MBD_ROWS_BOUNDARY -- see include/mbd.h
+mbd_status conv_forward_layer(ConvNet* c, int layer, float* loss_sum_dev, int rows);
+mbd_status conv_backward_layer(ConvNet* c, int layer, float fused_eta, int rows);
 mbd_status conv_outer_rows(ConvNet* c, int which, int layer, int side, void* rows, size_t bytes, int set);
 mbd_status conv_set_dw(ConvNet* c, int layer, const void* src, size_t bytes);
 }  // namespace mbd

@@ -862,23 +862,31 @@ extern "C" mbd_status mbd_conv_stage_input(mbd_net* n, const void* X_dev) {
   return conv_stage_input(n->conv, X_dev);
 }
 
-extern "C" mbd_status mbd_conv_forward_layer(mbd_net* n, int layer, float* loss_sum_dev) {
+extern "C" mbd_status mbd_conv_forward_layer_rows(mbd_net* n, int layer, int rows, float* loss_sum_dev) {
   if (!n) return MBD_E_INVALID;
   if (!n->is_conv) return MBD_E_UNSUPPORTED;
-  if (layer < 0 || layer >= n->Lc) return MBD_E_INVALID;
-  const mbd_status s = conv_forward_layer(n->conv, layer, loss_sum_dev);
-  if (s == MBD_OK && layer == n->Lc - 1) n->state = ST_FWD;
+  if (layer < 0 || layer >= n->Lc || rows < MBD_ROWS_ALL || rows > MBD_ROWS_BOUNDARY) return MBD_E_INVALID;
+  const mbd_status s = conv_forward_layer(n->conv, layer, loss_sum_dev, rows);
+  if (s == MBD_OK && layer == n->Lc - 1 && rows != MBD_ROWS_INTERIOR) n->state = ST_FWD;
+  return s;
+}
+
+extern "C" mbd_status mbd_conv_forward_layer(mbd_net* n, int layer, float* loss_sum_dev) {
+  return mbd_conv_forward_layer_rows(n, layer, MBD_ROWS_ALL, loss_sum_dev);
+}
+
+extern "C" mbd_status mbd_conv_backward_layer_rows(mbd_net* n, int layer, int rows, float fused_eta) {
+  if (!n || fused_eta < 0.f) return MBD_E_INVALID;
+  if (!n->is_conv) return MBD_E_UNSUPPORTED;
+  if (layer < 0 || layer >= n->Lc || rows < MBD_ROWS_ALL || rows > MBD_ROWS_BOUNDARY) return MBD_E_INVALID;
+  if (n->state != ST_FWD) return MBD_E_STATE;
+  const mbd_status s = conv_backward_layer(n->conv, layer, fused_eta, rows);
+  if (s == MBD_OK && layer == 0 && rows != MBD_ROWS_INTERIOR) n->state = fused_eta > 0.f ? ST_BWD_FUSED : ST_BWD_UNFUSED;
   return s;
 }
 
 extern "C" mbd_status mbd_conv_backward_layer(mbd_net* n, int layer, float fused_eta) {
-  if (!n || fused_eta < 0.f) return MBD_E_INVALID;
-  if (!n->is_conv) return MBD_E_UNSUPPORTED;
-  if (layer < 0 || layer >= n->Lc) return MBD_E_INVALID;
-  if (n->state != ST_FWD) return MBD_E_STATE;
-  const mbd_status s = conv_backward_layer(n->conv, layer, fused_eta);
-  if (s == MBD_OK && layer == 0) n->state = fused_eta > 0.f ? ST_BWD_FUSED : ST_BWD_UNFUSED;
-  return s;
+  return mbd_conv_backward_layer_rows(n, layer, MBD_ROWS_ALL, fused_eta);
 }
 
 extern "C" mbd_status mbd_conv_outer_rows(mbd_net* n, int which, int layer, int side, void* rows_dev, size_t bytes, int set) {

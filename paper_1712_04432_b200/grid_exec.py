@@ -267,12 +267,12 @@ class GridConv:
     def set_weights(self, i: int, K):
         self.net.set_weights(i, K)
 
-    def _exchange(self, which: int, layer: int, kind: str):
-        """First own rows go to the process above, last own rows to the process below; what arrives becomes
-        this strip's halo rows.  Counted as the paper counts it: one boundary of (B / P_c) W C words."""
+    def _exchange_start(self, which: int, layer: int, kind: str):
+        """First own rows go to the process above, last own rows to the process below (started here, not waited
+        for).  Counted as the paper counts it: one boundary of (B / P_c) W C words."""
         comm, dist, t = self.comm, self.comm.dist, self.t
         if comm.P_r == 1:
-            return
+            return None
         up = comm.rank - 1 if comm.r > 0 else None
         down = comm.rank + 1 if comm.r < comm.P_r - 1 else None
         ops, got = [], {}
@@ -286,11 +286,18 @@ class GridConv:
             got[side] = inc
             ops.append(dist.P2POp(dist.isend, out, peer))
             ops.append(dist.P2POp(dist.irecv, inc, peer))
-        for req in dist.batch_isend_irecv(ops):
+        comm.words[kind] += self.m * self.W * self.C
+        return (dist.batch_isend_irecv(ops), got, which, layer)
+
+    def _exchange_finish(self, handle):
+        """What arrived becomes this strip's halo rows."""
+        if handle is None:
+            return
+        reqs, got, which, layer = handle
+        for req in reqs:
             req.wait()
         for side, inc in got.items():
-            self.net.conv_outer_rows(which, layer, side, rows=inc.cuda() if comm.via_host else inc)
-        comm.words[kind] += self.m * self.W * self.C
+            self.net.conv_outer_rows(which, layer, side, rows=inc.cuda() if self.comm.via_host else inc)
 
     def step(self, X_local, eta: float):
         """One step on this process's strip X_local [B / P_c, C, H / P_r, W] (bf16).  Returns its share of J."""
@@ -303,9 +310,16 @@ class GridConv:
         J = t.zeros(1, dtype=t.float32, device="cuda")
         net.conv_stage_input(X_local)
         for i in range(L):
-            if self.ksizes[i] == 3:
-                self._exchange(mbd.T_ACT, i - 1, "halo_fwd")        # halo rows of the layer's input (Eq. 7, term 1)
-            net.conv_forward_layer(i, J if i == L - 1 else None)
+            loss_out = J if i == L - 1 else None
+            if self.ksizes[i] == 3 and self.comm.P_r > 1:
+                # halo rows of the layer's input (Eq. 7, term 1) travel while the rows that need none are computed
+                # (Section 2.2: "the halo exchange can be overlapped with the interior computation")
+                h = self._exchange_start(mbd.T_ACT, i - 1, "halo_fwd")
+                net.conv_forward_layer(i, None, rows=mbd.ROWS_INTERIOR)
+                self._exchange_finish(h)
+                net.conv_forward_layer(i, loss_out, rows=mbd.ROWS_BOUNDARY)
+            else:
+                net.conv_forward_layer(i, loss_out)
         return float(J.item()) if self.loss == mbd.LOSS_HALF_SSQ else 0.0
 
     def backward(self, eta: float):
@@ -313,9 +327,13 @@ class GridConv:
         set before (net.set_tensor(T_DY, L - 1, ...))."""
         t, net, comm, L = self.t, self.net, self.comm, self.L
         for i in range(L - 1, -1, -1):
-            if i > 0 and self.ksizes[i] == 3:
-                self._exchange(mbd.T_DY, i, "halo_bwd")             # halo rows of dY_i (Eq. 7, term 2)
-            net.conv_backward_layer(i, 0.0)
+            if i > 0 and self.ksizes[i] == 3 and comm.P_r > 1:
+                h = self._exchange_start(mbd.T_DY, i, "halo_bwd")   # halo rows of dY_i (Eq. 7, term 2), in flight beside
+                net.conv_backward_layer(i, 0.0, rows=mbd.ROWS_INTERIOR)     # the interior rows of the input gradient
+                self._exchange_finish(h)
+                net.conv_backward_layer(i, 0.0, rows=mbd.ROWS_BOUNDARY)     # its boundary rows, then the weight gradient
+            else:
+                net.conv_backward_layer(i, 0.0)
         P = comm.P_r * comm.P_c
         for i in range(L):                                            # all-reduce over all P processes (Eq. 7, term 3)
             g = net.get_tensor(mbd.T_DW, i)

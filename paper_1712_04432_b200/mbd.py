@@ -19,6 +19,7 @@ SPLIT_MODEL, SPLIT_DOMAIN = 0, 1
 F32, BF16 = 0, 1
 LOSS_SOFTMAX_CE, LOSS_HALF_SSQ, LOSS_NONE = 0, 1, 2
 T_ACT, T_DY, T_DW, T_DB, T_LOSS, T_PARTIALS, T_MASTER = range(7)
+ROWS_ALL, ROWS_INTERIOR, ROWS_BOUNDARY = range(3)
 
 KERNEL_CLASSES = ["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce_partials", "softmax_xent", "colsum",
                   "sgd_update", "halo_stage", "conv_fwd", "conv_bwd_data", "conv_bwd_weight", "other"]
@@ -30,7 +31,7 @@ EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weig
            "mbd_comm_time", "mbd_redistribute_time", "mbd_total_time", "mbd_grid_table", "mbd_choose_grid",
            "mbd_enable_master_weights", "mbd_block_gemm_bf16", "mbd_block_reduce", "mbd_softmax_xent",
            "mbd_conv_stage_input", "mbd_conv_forward_layer", "mbd_conv_backward_layer", "mbd_conv_outer_rows",
-           "mbd_get_plan"]
+           "mbd_get_plan", "mbd_conv_forward_layer_rows", "mbd_conv_backward_layer_rows"]
 
 
 class MbdError(RuntimeError):
@@ -131,6 +132,8 @@ def lib():
         L.mbd_conv_stage_input.argtypes = [vp, vp]
         L.mbd_conv_forward_layer.argtypes = [vp, i32, vp]
         L.mbd_conv_backward_layer.argtypes = [vp, i32, f32]
+        L.mbd_conv_forward_layer_rows.argtypes = [vp, i32, i32, vp]
+        L.mbd_conv_backward_layer_rows.argtypes = [vp, i32, i32, f32]
         L.mbd_conv_outer_rows.argtypes = [vp, i32, i32, i32, vp, C.c_size_t, i32]
         L.mbd_profile_enable.argtypes = [vp, i32]
         L.mbd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double)]
@@ -303,11 +306,12 @@ class Net:
         self._keep = [X]
         _check(lib().mbd_conv_stage_input(self._h, _ptr(X)), "mbd_conv_stage_input")
 
-    def conv_forward_layer(self, layer: int, loss_out=None):
-        _check(lib().mbd_conv_forward_layer(self._h, layer, _ptr(loss_out)), "mbd_conv_forward_layer")
+    def conv_forward_layer(self, layer: int, loss_out=None, rows: int = ROWS_ALL):
+        """rows: ROWS_ALL, or ROWS_INTERIOR (the rows that read no halo row) / ROWS_BOUNDARY (the rest), see include/mbd.h"""
+        _check(lib().mbd_conv_forward_layer_rows(self._h, layer, rows, _ptr(loss_out)), "mbd_conv_forward_layer_rows")
 
-    def conv_backward_layer(self, layer: int, fused_eta: float = 0.0):
-        _check(lib().mbd_conv_backward_layer(self._h, layer, float(fused_eta)), "mbd_conv_backward_layer")
+    def conv_backward_layer(self, layer: int, fused_eta: float = 0.0, rows: int = ROWS_ALL):
+        _check(lib().mbd_conv_backward_layer_rows(self._h, layer, rows, float(fused_eta)), "mbd_conv_backward_layer_rows")
 
     def conv_outer_rows(self, which: int, layer: int, side: int, rows=None):
         """rows None: returns the first (side 0) / last (side 1) own row of every image, [B, W, C] bf16;

@@ -258,3 +258,55 @@ def test_step_piece_by_piece_equals_the_whole_step():
     y_ref = O.conv3x3(ref, inp.X.astype(np.float64))[:, :, 4:8, :]
     assert rel_fro(y_sub, y_ref) < TOL
     sub.close()
+
+
+@pytest.mark.parametrize("H,ksizes", [(12, (3, 3, 3)), (3, (3, 3)), (2, (3, 3)), (1, (3, 3)), (9, (3, 1, 3)), (5, (1, 1))])
+def test_interior_and_boundary_rows_equal_the_whole_layer(H, ksizes):
+    """Section 2.2: the rows of a strip that read no halo row (2 .. H - 1) can be computed while the halo rows travel.
+    Every layer run as INTERIOR rows, then BOUNDARY rows -- forward and backward -- must leave, bit for bit, what the
+    whole-layer calls leave: outputs, propagated gradients, kernel gradients (and the same loss up to the order in
+    which the squares are added).  Strips of 1, 2 and 3 rows have
+    no or one interior row; a 1 x 1 layer is all interior."""
+    import torch
+    from paper_1712_04432_b200 import mbd
+    from tests.helpers import to_dev
+    L = len(ksizes)
+    w = I.conv_workload(64, H, 130, 3, n_layers=L, name="conv_rows", ksizes=ksizes)
+    inp = I.make_inputs(w, seed=63 + H)
+    X = to_dev(inp.X, True)
+    res = []
+    for split in (False, True):
+        net = mbd.Net(mbd.conv_layers(L, 64, H, 130, k=list(ksizes)), w.B, 1, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+        for i in range(L):
+            net.set_weights(i, to_dev(inp.Ws[i], True))
+        J = torch.zeros(1, dtype=torch.float32, device="cuda")
+        net.conv_stage_input(X)
+        for i in range(L):
+            out = J if i == L - 1 else None
+            if split:
+                net.conv_forward_layer(i, None, rows=mbd.ROWS_INTERIOR)
+                net.conv_forward_layer(i, out, rows=mbd.ROWS_BOUNDARY)
+            else:
+                net.conv_forward_layer(i, out)
+        for i in range(L - 1, -1, -1):
+            if split:
+                net.conv_backward_layer(i, 0.0, rows=mbd.ROWS_INTERIOR)
+                net.conv_backward_layer(i, 0.0, rows=mbd.ROWS_BOUNDARY)
+            else:
+                net.conv_backward_layer(i, 0.0)
+        net.poll()
+        res.append(dict(J=float(J.item()), act=[net.get_tensor(mbd.T_ACT, i).clone() for i in range(L)],
+                        dY=[net.get_tensor(mbd.T_DY, i).clone() for i in range(L)],
+                        dK=[net.get_tensor(mbd.T_DW, i).clone() for i in range(L)]))
+        net.close()
+    a, b = res
+    assert a["J"] > 0 and abs(a["J"] - b["J"]) <= 1e-5 * a["J"]       # the same squares, added in another order
+    for i in range(L):
+        assert torch.equal(a["act"][i], b["act"][i]) and torch.equal(a["dY"][i], b["dY"][i]) and torch.equal(a["dK"][i], b["dK"][i]), i
+    # more than one strip per network has no such split
+    net = mbd.Net(mbd.conv_layers(1, 64, 8, 40), 2, 2, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+    net.conv_stage_input(to_dev(np.zeros((2, 64, 8, 40), np.float32), True))
+    with pytest.raises(mbd.MbdError) as e:
+        net.conv_forward_layer(0, None, rows=mbd.ROWS_INTERIOR)
+    assert e.value.status == mbd.E_UNSUPPORTED
+    net.close()
