@@ -66,7 +66,11 @@ typedef enum {
 } mbd_status;
 
 enum { MBD_FC = 0, MBD_CONV3X3 = 1 };                 /* mbd_layer.kind                      */
-enum { MBD_SPLIT_MODEL = 0, MBD_SPLIT_DOMAIN = 1 };   /* mbd_layer.split: L_M or L_D, Eq. 9  */
+enum { MBD_SPLIT_MODEL = 0, MBD_SPLIT_DOMAIN = 1,     /* mbd_layer.split: L_M or L_D, Eq. 9  */
+       MBD_SPLIT_BATCH = 2 };  /* Section 3's improved case: this layer runs batch-parallel on a 1 x P grid
+                                  (P = P_r P_c) whatever the grid of the other layers -- "we force P_r = 1,
+                                  P_c = P for the convolutional layers and use varying P_r x P_c grids for the
+                                  fully connected layers"; convolution layers only, and all of them alike */
 enum { MBD_F32 = 0, MBD_BF16 = 1 };                   /* dtype                               */
 enum { MBD_LOSS_SOFTMAX_CE = 0, MBD_LOSS_HALF_SSQ = 1,
        MBD_LOSS_NONE = 2 };   /* convolution stacks only: no loss here.  The last layer applies its ReLU like
@@ -91,7 +95,9 @@ typedef struct {
   int64_t allgather_y;   /* Eq. 8 term 1:  B/P_c (P_r-1)/P_r d_i                    */
   int64_t allreduce_dx;  /* Eq. 8 term 2:  2 B/P_c (P_r-1)/P_r d_{i-1}, 0 for i = 1 */
   int64_t allreduce_dw;  /* Eq. 8 term 3:  2 (P_c-1)/P_c |W_i|/P_r ; Eq. 9 term 6:  */
-                         /*                2 (P-1)/P |W_i| for a domain-split layer */
+                         /*                2 (P-1)/P |W_i| for a domain-split layer; */
+                         /* Eq. 4: the same 2 (P-1)/P |W_i| for a batch-split layer  */
+                         /* (its only term)                                          */
   int64_t halo_fwd;      /* Eq. 9 term 4:  B/P_c X_W X_C floor(k_h/2), 0 if P_r = 1 */
   int64_t halo_bwd;      /* Eq. 9 term 5:  B/P_c Y_W Y_C floor(k_h/2), 0 if P_r = 1 */
 } mbd_words;
@@ -132,8 +138,10 @@ enum {
  * On a P_r x P_c grid a convolution is cut into P_r row strips (the balanced ranges
  * [floor(s H / P_r), floor((s + 1) H / P_r)): heights differ by at most one row) and P_c batch blocks, a
  * fully connected layer into P_r row blocks of W_i and the same P_c batch blocks.
- * MBD_E_GRID if P_r < 1, P_c < 1, P_c > B, P_r > min d_i over model-split layers, or
- * a strip would be shorter than its halo.
+ * MBD_E_GRID if P_r < 1, P_c < 1, P_c > B, P_r > min d_i over model-split layers,
+ * a strip would be shorter than its halo, or (batch-split convolutions) P_r P_c > B.
+ * Batch-split convolutions (MBD_SPLIT_BATCH) are cut into P_r P_c batch blocks and no strips; between them
+ * and the fully connected layers on P_r x P_c lies the re-distribution of Eq. 6 (mbd_redistribute_time).
  * MBD_E_UNSUPPORTED for convolutions other than 3x3 or 1x1, stride 1, "same" zero padding,
  * C_in = C_out = 64 (kind MBD_CONV3X3 with kh = kw = 1 is the 1x1 case, weights [C_out][C_in]),
  * a convolution above a fully connected layer, half-SSQ with

@@ -78,12 +78,17 @@ def layer_words(layers: Sequence[Dict], B: int, P_r: int, P_c: int) -> List[Dict
     Layers with split == "model" (set L_M) contribute the all-gather of Y, the
     all-reduce of dX and the all-reduce of dW over P_c; layers with
     split == "domain" (set L_D) contribute the two halo exchanges and the
-    all-reduce of dW over all P = P_r P_c processes."""
+    all-reduce of dW over all P = P_r P_c processes; layers with
+    split == "batch" are forced onto a 1 x P grid (Section 3: "we force P_r = 1,
+    P_c = P for the convolutional layers") and contribute Eq. 4's all-reduce."""
     P = P_r * P_c
     rows = []
     for i, l in enumerate(layers):
         row = dict(allgather_y=0, allreduce_dx=0, allreduce_dw=0, halo_fwd=0, halo_bwd=0)
-        if l.get("split", "model") == "model":
+        if l.get("split", "model") == "batch":
+            # Section 3, improved case: the layer runs on a 1 x P grid (pure batch parallelism): Eq. 4's term
+            row["allreduce_dw"] = _int(Fraction(2 * (P - 1) * n_weights(l), P))
+        elif l.get("split", "model") == "model":
             row["allgather_y"] = _int(Fraction(B * (P_r - 1) * d_out(l), P_r * P_c))
             if i >= 1:
                 row["allreduce_dx"] = _int(Fraction(2 * B * (P_r - 1) * d_in(l), P_r * P_c))

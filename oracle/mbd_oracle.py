@@ -49,9 +49,13 @@ class FC:
 
 @dataclass
 class Conv3x3:
-    """3x3, stride 1, zero-pad 1 convolution: K is [C_out, C_in, 3, 3]."""
+    """3x3, stride 1, zero-pad 1 convolution: K is [C_out, C_in, 3, 3].
+    split (used by the blocked step only): "domain" = row strips over the P_r groups (Section 2.2 / 2.4);
+    "batch" = the layer forced onto a 1 x P grid, P = P_r P_c (Section 3's improved case: pure batch
+    parallelism in the convolutional layers, P_r x P_c grids in the fully connected ones)."""
     K: np.ndarray
     relu: bool = True
+    split: str = "domain"
 
 
 def balanced_ranges(n: int, P: int):
@@ -426,7 +430,8 @@ def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
     added in ascending block index.  FC layers split the model over P_r and the
     batch over P_c; convolution layers split the image into P_r row strips and
     the batch over P_c (Eq. 9: their weight gradient is summed over all
-    P = P_r P_c processes)."""
+    P = P_r P_c processes); convolution layers with split == "batch" are cut into
+    P_r P_c batch blocks and no strips (Section 3's improved case)."""
     L = len(layers)
     Xs = [np.asarray(X1, F64)]
     Ys = []
@@ -434,7 +439,7 @@ def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
         if isinstance(lay, FC):
             Y = fc_forward_blocked(lay.W, Xs[i], lay.b, P_r, P_c)
         else:
-            Y = conv3x3_strips(lay.K, Xs[i], P_r)
+            Y = conv3x3_strips(lay.K, Xs[i], 1 if lay.split == "batch" else P_r)
         Ys.append(Y)
         if i + 1 < L:
             Xs.append(_kept(Y, lay, layers[i + 1], store))
@@ -454,13 +459,15 @@ def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
                 for (c0, c1) in balanced_ranges(B, P_c):
                     db = db + dYs[i][:, c0:c1].sum(axis=1)
                 dbs[i] = db
+        elif lay.split == "batch":
+            dWs[i], _ = conv3x3_dK_grid(dYs[i], Xs[i], 1, P_r * P_c)      # one partial per process of the 1 x P grid
         else:
             dWs[i], _ = conv3x3_dK_grid(dYs[i], Xs[i], P_r, P_c)
         if i > 0:
             if isinstance(lay, FC):
                 dXs[i], _ = fc_dX_blocked(lay.W, dYs[i], P_r, P_c)
             else:
-                dXs[i] = conv3x3_dX_strips(lay.K, dYs[i], P_r)
+                dXs[i] = conv3x3_dX_strips(lay.K, dYs[i], 1 if lay.split == "batch" else P_r)
             dXs[i] = _below(dXs[i], Ys[i - 1])
             prev = layers[i - 1]
             dYs[i - 1] = dXs[i] * (Ys[i - 1] > 0.0) if prev.relu else dXs[i]

@@ -61,7 +61,9 @@ def layer_messages(layers: Sequence[Dict], P_r: int, P_c: int) -> List[Dict[str,
     rows = []
     for i, l in enumerate(layers):
         row = dict.fromkeys(TERMS, 0)
-        if l.get("split", "model") == "model":
+        if l.get("split", "model") == "batch":      # forced onto 1 x P (Section 3's improved case): Eq. 4's all-reduce alone
+            row["allreduce_dw"] = 2 * ceil_log2(P)
+        elif l.get("split", "model") == "model":
             row["allgather_y"] = ceil_log2(P_r)
             if i >= 1:
                 row["allreduce_dx"] = 2 * ceil_log2(P_r)
@@ -81,7 +83,9 @@ def layer_words_exact(layers: Sequence[Dict], B: int, P_r: int, P_c: int) -> Lis
     rows = []
     for i, l in enumerate(layers):
         row = dict.fromkeys(TERMS, Fraction(0))
-        if l.get("split", "model") == "model":
+        if l.get("split", "model") == "batch":
+            row["allreduce_dw"] = 2 * Fraction(P - 1, P) * n_weights(l)
+        elif l.get("split", "model") == "model":
             row["allgather_y"] = Fraction(B, P_c) * Fraction(P_r - 1, P_r) * d_out(l)
             if i >= 1:
                 row["allreduce_dx"] = 2 * Fraction(B, P_c) * Fraction(P_r - 1, P_r) * d_in(l)
@@ -175,6 +179,9 @@ def grid_feasible(layers: Sequence[Dict], B: int, P_r: int, P_c: int) -> bool:
     for l in layers:
         if l.get("split", "model") == "model":
             if P_r > d_out(l):
+                return False
+        elif l.get("split") == "batch":
+            if P_r * P_c > B:
                 return False
         elif P_r > l["H"]:
             return False

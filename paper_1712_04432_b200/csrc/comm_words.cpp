@@ -54,6 +54,10 @@ extern "C" mbd_status mbd_comm_words(const mbd_layer* layers, int L, int64_t B, 
         ok = ok && ceil_div_to_i64(static_cast<i128>(B) * l.W * l.C_out * (l.kh / 2), P_c, &w.halo_bwd);
       }
       ok = ok && ceil_div_to_i64(static_cast<i128>(2) * (P - 1) * nW, P, &w.allreduce_dw);
+    } else if (l.split == MBD_SPLIT_BATCH) {
+      if (P > static_cast<i128>(B)) return MBD_E_GRID;      // one sample per process at least
+      // Section 3's improved case: the layer is batch-parallel on 1 x P; its one term is Eq. 4's all-reduce over all P
+      ok = ok && ceil_div_to_i64(static_cast<i128>(2) * (P - 1) * nW, P, &w.allreduce_dw);
     } else {
       return MBD_E_INVALID;
     }

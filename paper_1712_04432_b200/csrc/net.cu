@@ -303,8 +303,13 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
     } else if (l.kind == MBD_CONV3X3) {
       const bool k3 = l.kh == 3 && l.kw == 3, k1 = l.kh == 1 && l.kw == 1;     // stride 1, "same" padding
       if (!(k3 || k1) || l.C_in != 64 || l.C_out != 64 || dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
-      if (l.split != MBD_SPLIT_DOMAIN) return MBD_E_UNSUPPORTED;
-      if (l.H < 1 || l.W < 1 || P_r > l.H) return MBD_E_GRID;   // a strip needs >= 1 row (halo = 1)
+      if (l.split != MBD_SPLIT_DOMAIN && l.split != MBD_SPLIT_BATCH) return MBD_E_UNSUPPORTED;
+      if (l.split != layers[0].split) return MBD_E_UNSUPPORTED;          // all convolutions split alike
+      if (l.split == MBD_SPLIT_BATCH) {                                  // 1 x P: one sample per process at least
+        if (l.H < 1 || l.W < 1 || static_cast<int64_t>(P_r) * P_c > B) return MBD_E_GRID;
+      } else if (l.H < 1 || l.W < 1 || P_r > l.H) {
+        return MBD_E_GRID;   // a strip needs >= 1 row (halo = 1)
+      }
       if (i > 0 && (l.H != layers[0].H || l.W != layers[0].W)) return MBD_E_INVALID;
     } else {
       return MBD_E_INVALID;
@@ -346,7 +351,8 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   if (cudaMemsetAsync(n->status, 0, sizeof(int), n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
 
   if (Lc > 0) {
-    st = conv_create(layers, Lc, B, P_r, n->max_partials, n->num_sms, n->status, n->stream, &n->prof,
+    // batch-split convolutions (Section 3's improved case) run on 1 x P: no strips, whatever P_r is
+    st = conv_create(layers, Lc, B, layers[0].split == MBD_SPLIT_BATCH ? 1 : P_r, n->max_partials, n->num_sms, n->status, n->stream, &n->prof,
                      mixed || loss == MBD_LOSS_NONE, &n->conv);
     if (st != MBD_OK) { free_net(n); return st; }
     if (is_conv) {

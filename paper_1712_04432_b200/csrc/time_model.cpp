@@ -66,6 +66,8 @@ mbd_status layer_row(const mbd_layer& l, int split, bool first, double B, int P_
     t->allreduce_dw = 2.0 * (m.alpha * ceil_log2(static_cast<long long>(P_r) * P_c) + m.beta * ((P - 1.0) / P) * d.nW);
     return MBD_OK;
   }
+  if (split == MBD_SPLIT_BATCH)   // forced onto 1 x P (Section 3's improved case): only dW moves, over all P processes
+    return layer_row(l, MBD_SPLIT_MODEL, first, B, 1, P_r * P_c, m, t);
   return MBD_E_INVALID;
 }
 
@@ -77,6 +79,8 @@ bool feasible(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, bool 
     if (l.split == MBD_SPLIT_MODEL) {
       const double dout = l.kind == MBD_FC ? static_cast<double>(l.d_out) : static_cast<double>(l.H) * l.W * l.C_out;
       if (static_cast<double>(P_r) > dout) return false;
+    } else if (l.split == MBD_SPLIT_BATCH) {
+      if (static_cast<int64_t>(P_r) * P_c > B) return false;
     } else if (P_r > l.H) {
       return false;
     }

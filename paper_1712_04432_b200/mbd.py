@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libmbd.so")
 
 OK, E_INVALID, E_GRID, E_ALLOC, E_CUDA, E_STATE, E_TIMEOUT, E_UNSUPPORTED, E_TOO_LARGE = range(9)
 FC, CONV3X3 = 0, 1
-SPLIT_MODEL, SPLIT_DOMAIN = 0, 1
+SPLIT_MODEL, SPLIT_DOMAIN, SPLIT_BATCH = 0, 1, 2
 F32, BF16 = 0, 1
 LOSS_SOFTMAX_CE, LOSS_HALF_SSQ, LOSS_NONE = 0, 1, 2
 T_ACT, T_DY, T_DW, T_DB, T_LOSS, T_PARTIALS, T_MASTER = range(7)
@@ -164,12 +164,13 @@ def fc_layers(dims: Sequence[int], bias: bool = True, relu: bool = True) -> List
                   d_out=int(dims[i])) for i in range(1, len(dims))]
 
 
-def conv_layers(n: int, C_: int, H: int, W: int, relu: bool = True, k=3) -> List[Layer]:
-    """n domain-split convolution layers C -> C on H x W images; `k` is the kernel size (3 or 1),
-    one value for all layers or one per layer."""
+def conv_layers(n: int, C_: int, H: int, W: int, relu: bool = True, k=3, split: int = SPLIT_DOMAIN) -> List[Layer]:
+    """n convolution layers C -> C on H x W images, domain-split (row strips) or, with split=SPLIT_BATCH,
+    batch-parallel on 1 x P (Section 3's improved case); `k` is the kernel size (3 or 1), one value for all
+    layers or one per layer."""
     ks = [k] * n if isinstance(k, int) else list(k)
     assert len(ks) == n
-    return [Layer(kind=CONV3X3, split=SPLIT_DOMAIN, relu=int(relu), bias=0, d_in=C_ * H * W, d_out=C_ * H * W,
+    return [Layer(kind=CONV3X3, split=split, relu=int(relu), bias=0, d_in=C_ * H * W, d_out=C_ * H * W,
                   C_in=C_, C_out=C_, H=H, W=W, kh=ks[i], kw=ks[i]) for i in range(n)]
 
 

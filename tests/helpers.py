@@ -294,12 +294,12 @@ def compare_conv_step(g, o, tol, fused=False, tol_below_relu=None, init=None, re
 # ---------------------------------------------------------------------------
 # convolutions followed by fully connected layers (Section 2.4)
 # ---------------------------------------------------------------------------
-def oracle_mixed_step(w, inp, blocked_grid=None, eta=None):
+def oracle_mixed_step(w, inp, blocked_grid=None, eta=None, conv_split="domain"):
     """fp64 oracle step of a mixed workload: Conv3x3 layers on NCHW, then FC layers on the
     flattened activation; stored activations rounded to bf16 like the device's."""
     from oracle import mbd_oracle as O
     Lc = w.n_layers
-    layers = [O.Conv3x3(oracle_kernel(inp.Ws[i]), relu=True) for i in range(Lc)]
+    layers = [O.Conv3x3(oracle_kernel(inp.Ws[i]), relu=True, split=conv_split) for i in range(Lc)]
     for i in range(Lc, w.L):
         layers.append(O.FC(inp.Ws[i].astype(np.float64), inp.bs[i].astype(np.float64), relu=True))
     X = inp.X.astype(np.float64)
@@ -309,10 +309,11 @@ def oracle_mixed_step(w, inp, blocked_grid=None, eta=None):
     return O.train_step_blocked(layers, X, inp.labels, "softmax_ce", eta, *blocked_grid, store=bf16_store)
 
 
-def mixed_layers(w):
+def mixed_layers(w, conv_split=None):
     from paper_1712_04432_b200 import mbd
     C_, H, Wd = w.dims
-    return mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.ksize(i) for i in range(w.n_layers)]) + mbd.fc_layers(w.fc_dims, bias=True)
+    split = mbd.SPLIT_DOMAIN if conv_split in (None, "domain") else mbd.SPLIT_BATCH
+    return mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.ksize(i) for i in range(w.n_layers)], split=split) + mbd.fc_layers(w.fc_dims, bias=True)
 
 
 def oracle_mixed_acts(o, w):
@@ -330,13 +331,13 @@ def oracle_mixed_acts(o, w):
     return out
 
 
-def gpu_mixed_step(w, inp, grid=(1, 1), max_partials=0, fused=False, force_acts=None, eta=None):
+def gpu_mixed_step(w, inp, grid=(1, 1), max_partials=0, fused=False, force_acts=None, eta=None, conv_split=None):
     """The same step through the C ABI; conv tensors come back NCHW, FC tensors [B, d]."""
     import torch
     from paper_1712_04432_b200 import mbd
     L, Lc = w.L, w.n_layers
     eta = w.eta if eta is None else eta
-    net = mbd.Net(mixed_layers(w), w.B, grid[0], grid[1], mbd.BF16, mbd.LOSS_SOFTMAX_CE, max_partials)
+    net = mbd.Net(mixed_layers(w, conv_split), w.B, grid[0], grid[1], mbd.BF16, mbd.LOSS_SOFTMAX_CE, max_partials)
     for i in range(L):
         if i < Lc:
             net.set_weights(i, to_dev(inp.Ws[i], True))

@@ -34,7 +34,7 @@ def _as_layers(rows):
         if l["kind"] == "fc":
             out.append(mbd.Layer(kind=mbd.FC, split=mbd.SPLIT_MODEL, relu=1, bias=1, d_in=l["d_in"], d_out=l["d_out"]))
         else:
-            out.append(mbd.Layer(kind=mbd.CONV3X3, split=mbd.SPLIT_DOMAIN if l["split"] == "domain" else mbd.SPLIT_MODEL,
+            out.append(mbd.Layer(kind=mbd.CONV3X3, split={"domain": mbd.SPLIT_DOMAIN, "batch": mbd.SPLIT_BATCH}.get(l["split"], mbd.SPLIT_MODEL),
                                  relu=1, bias=0, d_in=l["C_in"] * l["H"] * l["W"], d_out=l["C_out"] * l["H"] * l["W"],
                                  C_in=l["C_in"], C_out=l["C_out"], H=l["H"], W=l["W"], kh=l["kh"], kw=l["kw"]))
     return out
@@ -58,6 +58,22 @@ def test_comm_words_match_oracle_on_odd_grids(P_r, P_c):
     assert mbd.comm_words(_as_layers(conv), 30, P_r, P_c) == CW.layer_words(conv, 30, P_r, P_c)
     convm = [dict(kind="conv", split="model", C_in=8, C_out=24, H=13, W=13, kh=3, kw=3)] * 2
     assert mbd.comm_words(_as_layers(convm), 30, P_r, P_c) == CW.layer_words(convm, 30, P_r, P_c)
+
+
+@pytest.mark.parametrize("P_r,P_c", [(1, 1), (4, 4), (2, 8), (16, 1), (3, 5)])
+def test_comm_words_of_batch_parallel_convolutions(P_r, P_c):
+    # Section 3's improved case: the convolutions forced onto 1 x P, the fully connected layers on P_r x P_c
+    net = [dict(kind="conv", split="batch", C_in=64, C_out=64, H=56, W=56, kh=3, kw=3),
+           dict(kind="conv", split="batch", C_in=64, C_out=64, H=56, W=56, kh=1, kw=1),
+           dict(kind="fc", split="model", d_in=64 * 56 * 56, d_out=1024), dict(kind="fc", split="model", d_in=1024, d_out=1000)]
+    got = mbd.comm_words(_as_layers(net), 256, P_r, P_c)
+    assert got == CW.layer_words(net, 256, P_r, P_c)
+    # the convolutions move what Eq. 4 moves on P processes, and nothing else
+    assert sum(sum(r.values()) for r in got[:2]) == CW.eq4_batch_words(net[:2], P_r * P_c)
+    assert all(r["halo_fwd"] == r["halo_bwd"] == r["allgather_y"] == r["allreduce_dx"] == 0 for r in got[:2])
+    with pytest.raises(mbd.MbdError) as e:
+        mbd.comm_words(_as_layers(net), 12, 4, 4)            # 16 processes, 12 samples
+    assert e.value.status == mbd.E_GRID
 
 
 def test_comm_words_rejects_bad_arguments():

@@ -126,3 +126,18 @@ def test_pure_schemes_bracket_the_mixed_grids_at_small_batch():
     t = {g: CW.total_words(layers, 256, *g) for g in [(8, 1), (1, 8), (2, 4), (4, 2)]}
     assert t[(8, 1)] < t[(4, 2)] < t[(2, 4)] < t[(1, 8)]
     assert t[(8, 1)] == 5729024 and t[(1, 8)] == 102588416
+
+
+def test_batch_split_layers_move_what_Eq4_moves_on_all_processes():
+    # Section 3's improved case ("we force P_r = 1, P_c = P for the convolutional layers"): whatever the grid
+    # of the other layers, a batch-split layer contributes Eq. 4's term for P = P_r P_c processes and no other:
+    # by hand for |W| = 9*64*64 = 36864 on 4 x 2: 2 * 7/8 * 36864 = 64512
+    conv = dict(kind="conv", split="batch", C_in=64, C_out=64, H=56, W=56, kh=3, kw=3)
+    row = CW.layer_words([conv], 32, 4, 2)[0]
+    assert row == dict(allgather_y=0, allreduce_dx=0, allreduce_dw=64512, halo_fwd=0, halo_bwd=0)
+    for P_r, P_c in [(1, 8), (8, 1), (2, 4), (16, 2)]:
+        rows = CW.layer_words([conv, conv], 64, P_r, P_c)
+        assert sum(sum(r.values()) for r in rows) == CW.eq4_batch_words([conv, conv], P_r * P_c)
+        # the same layer on a 1 x P grid as a model-split layer: Eq. 8 with P_r = 1 leaves that one term as well
+        as_model = CW.layer_words([dict(conv, split="model")] * 2, 64, 1, P_r * P_c)
+        assert rows == as_model

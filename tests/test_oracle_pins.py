@@ -470,6 +470,27 @@ def test_mixed_blocked_step_equals_unblocked(grid):
         assert relerr(b["dXs"][i], a["dXs"][i]) < 1e-12
 
 
+@pytest.mark.parametrize("grid", [(2, 3), (3, 2), (6, 1), (1, 6)])
+def test_batch_split_convolutions_in_the_blocked_step(grid):
+    """Section 3's improved case: convolutions on 1 x P, fully connected layers on P_r x P_c.  Re-blocking changes no
+    sum (the step equals the un-blocked one), and the convolutions' weight gradient is formed from P = P_r P_c
+    per-process partials over batch blocks of whole images -- what a 1 x P grid of the domain-split form gives."""
+    import dataclasses
+    layers, X, labels = mixed_case(77, B=6, H=8)
+    batch = [dataclasses.replace(l, split="batch") if isinstance(l, O.Conv3x3) else l for l in layers]
+    a = O.train_step(layers, X, labels, "softmax_ce", 0.01)
+    b = O.train_step_blocked(batch, X, labels, "softmax_ce", 0.01, *grid)
+    assert abs(a["J"] - b["J"]) < 1e-12 * abs(a["J"])
+    for i in range(4):
+        assert relerr(b["Ys"][i], a["Ys"][i]) < 1e-12 and relerr(b["dWs"][i], a["dWs"][i]) < 1e-12
+        assert relerr(b["new_W"][i], a["new_W"][i]) < 1e-12
+    P = grid[0] * grid[1]
+    c = O.train_step_blocked(layers[:2], X, None, "half_ssq", 0.01, 1, P)      # the two convolutions alone, domain form on 1 x P
+    d = O.train_step_blocked(batch[:2], X, None, "half_ssq", 0.01, *grid)      # ... and batch-split on the P_r x P_c grid
+    for i in range(2):
+        assert np.array_equal(c["dWs"][i], d["dWs"][i]) and np.array_equal(c["Ys"][i], d["Ys"][i])
+
+
 def test_conv_weight_gradient_partials_over_the_whole_grid():
     """P_r x P_c partials, one per process, whose sum is the un-blocked gradient (last term of Eq. 9)."""
     r = rng(75)

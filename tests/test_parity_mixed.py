@@ -74,6 +74,25 @@ def test_unequal_strips_under_fully_connected_layers():
         compare_mixed_step(g, o, w, TOL, fused=True)
 
 
+@pytest.mark.parametrize("grid", [(2, 3), (3, 2), (6, 1)])
+def test_batch_parallel_convolutions_under_model_parallel_layers(small, grid):
+    """Section 3's improved case: the convolutions forced onto a 1 x P grid (pure batch parallelism: no strips, one
+    weight-gradient partial per process), the fully connected layers on P_r x P_c.  Against the oracle that forms
+    exactly those blocks; 6 samples on 6 processes is the limit (one sample per process), 12 processes are refused."""
+    from paper_1712_04432_b200 import mbd
+    w, inp, _ = small
+    ob = oracle_mixed_step(w, inp, blocked_grid=grid, conv_split="batch")
+    eta = update_sized_eta(ob, inp.Ws, w.B)
+    ob = oracle_with_eta(ob, inp.Ws, inp.bs, w.B, eta)
+    for fused in (False, True):
+        g = gpu_mixed_step(w, inp, grid, 4, fused=fused, force_acts=oracle_mixed_acts(ob, w), eta=eta, conv_split="batch")
+        compare_mixed_step(g, ob, w, TOL, fused=fused, init=inp, require_sized=True)
+    from tests.helpers import mixed_layers
+    with pytest.raises(mbd.MbdError) as e:
+        mbd.Net(mixed_layers(w, "batch"), w.B, 4, 3, mbd.BF16, mbd.LOSS_SOFTMAX_CE, 0)
+    assert e.value.status == mbd.E_GRID
+
+
 def test_train_step_graph_matches_separate_calls(small):
     """mbd_train_step (captured graph, fused update) leaves the same weights, bit for bit, as
     forward + backward(eta) issued one by one; and two steps change them twice."""

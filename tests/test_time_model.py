@@ -49,6 +49,25 @@ def test_comm_time_matches_oracle_term_by_term(kind):
                 assert close(g[k], w[k]), (rows, B, P_r, P_c, k, g[k], w[k])
 
 
+def test_batch_parallel_convolutions_equal_their_own_1xP_grid():
+    # Section 3's improved case, two ways: the layer marked batch-split on the network's P_r x P_c grid, and the same
+    # layer as a model-split layer on a grid of its own, 1 x P (the oracle's per-layer form, written separately)
+    r = random.Random(7)
+    for _ in range(40):
+        rows = random_net(r, "mixed")
+        B = r.choice([64, 328, 2048])
+        P_r, P_c = r.choice([1, 2, 4, 8]), r.choice([1, 2, 4, 8])
+        a, b = r.choice(MACHINES)
+        batch = [dict(l, split="batch") if l["kind"] == "conv" else l for l in rows]
+        got = mbd.comm_time(_as_layers(batch), B, P_r, P_c, (a, b))
+        grids = [(1, P_r * P_c) if l["kind"] == "conv" else (P_r, P_c) for l in rows]
+        want = T.per_layer_times(rows, B, grids, a, b)
+        same = T.layer_times(batch, B, P_r, P_c, a, b)
+        for g, w, s in zip(got, want, same):
+            for k in T.TERMS:
+                assert close(g[k], w[k]) and close(s[k], w[k]), (rows, B, P_r, P_c, k, g[k], w[k], s[k])
+
+
 def test_redistribution_and_total_time():
     for B, pr, pc, d in [(256, 8, 1, 4096), (2048, 16, 32, 9216), (64, 1, 64, 100), (30, 3, 5, 7)]:
         for a, b in MACHINES:
