@@ -78,6 +78,18 @@ enum { MODE_RELU_STORE = 0, MODE_STORE_SSQ = 1, MODE_MASK = 2 };
 __host__ __device__ __forceinline__ int strip_first(int s, int H, int P) { return static_cast<int>((static_cast<long long>(s) * H) / P); }
 __host__ __device__ __forceinline__ int strip_height(int s, int H, int P) { return strip_first(s + 1, H, P) - strip_first(s, H, P); }
 __host__ __device__ __forceinline__ int strip_of_row(int h, int H, int P) { return static_cast<int>(((static_cast<long long>(h) + 1) * P - 1) / H); }
+// The same inside the kernels, where they sit on the epilogue's critical path: strips of equal height (H = Hs P, the
+// common case) need no division by P at all, the others one in 32 bits (H P < 2^31 is checked when the network is made).
+__device__ __forceinline__ bool strips_uneven(int H, int P, int Hs) { return Hs * P != H; }
+__device__ __forceinline__ int strip_first(int s, int H, int P, int Hs) {
+  return !strips_uneven(H, P, Hs) ? s * Hs : static_cast<int>(static_cast<unsigned>(s * H) / static_cast<unsigned>(P));
+}
+__device__ __forceinline__ int strip_height(int s, int H, int P, int Hs) {
+  return !strips_uneven(H, P, Hs) ? Hs : strip_first(s + 1, H, P, Hs) - strip_first(s, H, P, Hs);
+}
+__device__ __forceinline__ int strip_of_row(int h, int H, int P, int Hs) {
+  return !strips_uneven(H, P, Hs) ? h / Hs : static_cast<int>(static_cast<unsigned>((h + 1) * P - 1) / static_cast<unsigned>(H));
+}
 
 // ------------------------------------------------------------------------------ layout kernels
 // NCHW -> strips.  Block = 32 consecutive pixels of one image's flattened (h, w) plane (so narrow
@@ -125,15 +137,15 @@ nchw_to_strips_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int 
   v1.x = tile[px][cq + 4]; v1.y = tile[px][cq + 5]; v1.z = tile[px][cq + 6]; v1.w = tile[px][cq + 7];
   const int R = Hs + 2;
   const int h = p / W, w = p - h * W;
-  const int s = strip_of_row(h, H, P_r), r = h - strip_first(s, H, P_r) + 1;
+  const int s = strip_of_row(h, H, P_r, Hs), r = h - strip_first(s, H, P_r, Hs) + 1;
   auto put = [&](int ss, int rr) {
     bf16* q = dst + (((static_cast<int64_t>(b) * P_r + ss) * R + rr) * W + w) * C + 2 * cq;
     *reinterpret_cast<uint4*>(q) = v0;
     *reinterpret_cast<uint4*>(q + 8) = v1;
   };
   put(s, r);
-  if (r == 1 && s > 0) put(s - 1, strip_height(s - 1, H, P_r) + 1);          // first row of a strip: lower halo of the strip above
-  if (r == strip_height(s, H, P_r) && s < P_r - 1) put(s + 1, 0);            // last row of a strip: upper halo of the strip below
+  if (r == 1 && s > 0) put(s - 1, strip_height(s - 1, H, P_r, Hs) + 1);          // first row of a strip: lower halo of the strip above
+  if (r == strip_height(s, H, P_r, Hs) && s < P_r - 1) put(s + 1, 0);            // last row of a strip: upper halo of the strip below
 }
 
 // strips -> NCHW: the mirror image (own rows only).  Used to hand the last convolution's output to the
@@ -150,7 +162,7 @@ strips_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, int 
     const int p = p0 + px;
     if (p < HW) {
       const int h = p / W, w = p - h * W;
-      const int s = strip_of_row(h, H, P_r), r = h - strip_first(s, H, P_r) + 1;
+      const int s = strip_of_row(h, H, P_r, Hs), r = h - strip_first(s, H, P_r, Hs) + 1;
       const bf16* q = src + (((static_cast<int64_t>(b) * P_r + s) * R + r) * W + w) * C + 2 * cq;
       const uint4 v0 = *reinterpret_cast<const uint4*>(q), v1 = *reinterpret_cast<const uint4*>(q + 8);
       tile[px][cq + 0] = v0.x; tile[px][cq + 1] = v0.y; tile[px][cq + 2] = v0.z; tile[px][cq + 3] = v0.w;
@@ -523,6 +535,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           if (q.x0 >= p.nseg * FWD_PIX) { q.x0 = 0; q.z += pack; }
         }
       };
+      const bool uneven = strips_uneven(p.H, p.P_r, p.Hs);
       const int sub = FWD_PIX / pack;                   // tile positions per strip
       const int sub_bytes = sub * 128;
       auto load_mask = [&](int k, const Pos& q) {
@@ -545,7 +558,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const int x0 = cur.x0, row = cur.row, z = cur.z;
         // (a row beyond its strip's height is the dead row of a short strip: computed, never stored or counted)
         const bool valid = (PACKED ? (pl_sub < p.W && z + pl_strip < p.Z) : x0 + pl < p.W) &&
-                           row <= strip_height((z + pl_strip) % p.P_r, p.H, p.P_r);
+                           (row < p.Hs || !uneven || row <= strip_height((z + pl_strip) % p.P_r, p.H, p.P_r, p.Hs));
         const int blk = acc_block(g);
         if (issuer) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store of row g - 2 has read this tile
         asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -615,7 +628,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           for (int j = 0; j < pack; ++j) {           // one box per strip of the group; all of them in one bulk group
             const int zj = z + j;
             if (zj >= p.Z) break;
-            const int hs_j = strip_height(zj % p.P_r, p.H, p.P_r);
+            const int hs_j = uneven ? strip_height(zj % p.P_r, p.H, p.P_r, p.Hs) : p.Hs;
             if (row > hs_j) continue;                  // dead row of a short strip
             const uint32_t src = stg_out + buf * FWD_TILE_BYTES + j * sub_bytes;
             asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
@@ -625,7 +638,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             // halo row of the strip above / below it in the same image.
             if (row == 1 && p.P_r > 1 && zj % p.P_r > 0)
               asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
-                           ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(strip_height(zj % p.P_r - 1, p.H, p.P_r) + 1), "r"(zj - 1), "r"(src)
+                           ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(strip_height(zj % p.P_r - 1, p.H, p.P_r, p.Hs) + 1), "r"(zj - 1), "r"(src)
                            : "memory");
             if (row == hs_j && p.P_r > 1 && zj % p.P_r < p.P_r - 1)
               asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
@@ -752,7 +765,8 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             mbar_expect_tx(fy, mirrored ? 2 * WG_CHUNK : WG_CHUNK);
             for (int j = 0; j < p.pack; ++j) {     // one box per strip of the group (pixels beyond W and strips beyond Z read as zeros)
               // the dead row of a short strip holds the neighbour's row (it is that strip's halo row): read the all-zero row instead
-              const int yrow = run.h0 + r + 1 > strip_height((z + j) % p.P_r, p.H, p.P_r) ? p.Hs + 1 : run.h0 + r + 1;
+              const int yrow = run.h0 + r + 1 == p.Hs && strips_uneven(p.H, p.P_r, p.Hs) && p.Hs > strip_height((z + j) % p.P_r, p.H, p.P_r, p.Hs)
+                                   ? p.Hs + 1 : run.h0 + r + 1;
               tma_load_4d(yring + ys * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, yrow, z + j, fy);
               if (mirrored) tma_load_4d(yring + (WG_YSTAGES + ys) * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, yrow, z + j, fy);
             }
@@ -1006,6 +1020,7 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
   if (conv_init() != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
   const int H = layers[0].H, W = layers[0].W;
   if (B > 65535 || static_cast<int64_t>(H) * W > INT32_MAX) return MBD_E_UNSUPPORTED;   // grid.y of the staging kernels
+  if ((static_cast<int64_t>(H) + 1) * P_r > INT32_MAX) return MBD_E_UNSUPPORTED;               // 32-bit strip arithmetic in the kernels
   ConvNet* c = new (std::nothrow) ConvNet();
   if (!c) return MBD_E_ALLOC;
   c->L = L; c->B = B; c->H = H; c->W = W; c->P_r = P_r; c->Hs = (H + P_r - 1) / P_r; c->R = c->Hs + 2; c->Z = B * P_r;
