@@ -306,8 +306,9 @@ MBD_API int64_t mbd_launch_count(const mbd_net* net);
  * unit (of the CTA pair when cta_pair != 0); k_pieces the number of fp32 partial sums the K range is
  * cut into (the grid's S = min(P, max_partials) times any further cut the planner added); running_sum != 0:
  * the pieces are added inside the product's own epilogue (see max_partials of mbd_net_create), otherwise
- * k_pieces > 1 means a reduce_partials launch follows; tma_epilogue != 0: the tail operation the plan was made for (bias +
- * ReLU, ReLU mask, fused update) moves its global data by TMA; ctas: CTAs launched.
+ * k_pieces > 1 means a reduce_partials launch follows; tma_epilogue = 1: the tail operation the plan was made for (bias +
+ * ReLU, ReLU mask, fused update) moves its global data by TMA; tma_epilogue = 2: the k_pieces fp32 partial sums are
+ * stored by TMA (short pieces on 128-row tiles); ctas: CTAs launched.
  * MBD_E_UNSUPPORTED for fp32 networks and convolution layers, MBD_E_INVALID for a product the layer
  * does not have (backward-data of the network's first layer). */
 typedef struct { int32_t tile_m, tile_n, cta_pair, k_pieces, tma_epilogue, ctas, running_sum, reserved; } mbd_plan;

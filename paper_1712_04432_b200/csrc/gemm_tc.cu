@@ -194,6 +194,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   constexpr int TE_BOXES = BN / 128;
   constexpr int TE_BYTES = 8 * TE_BOXES * 4096;
   constexpr int STAGES_TE = (RING_MAX_BYTES - TE_BYTES) / STAGE_BYTES;
+  // fp32 planes by TMA (p.te == 2): two boxes of [32 rows][32 columns] fp32 per epilogue warp
+  constexpr int STAGES_TEP = (RING_MAX_BYTES - 8 * 2 * 4096) / STAGE_BYTES;
   constexpr int ACC_COLS = MH * BN;                           // TMEM columns of one tile
   constexpr int ACC_BUFS = ACC_COLS * 2 <= 512 ? 2 : 1;
   constexpr int TMEM_COLS = ACC_COLS * ACC_BUFS;
@@ -216,7 +218,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     return;
   }
   const bool te = !FIX && MH == 1 && p.te != 0;
-  const int stages = te ? STAGES_TE : STAGES;
+  const int stages = te ? (p.te == 2 ? STAGES_TEP : STAGES_TE) : STAGES;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;        // 0 = the CTA that issues the MMAs
@@ -355,7 +357,63 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     constexpr int NV = HC / 8;                    // 16-byte vectors per thread and tile
     const int q = warp & 3;
     const int half = (warp - 2) >> 2;
-    if (te) {
+    if (te && p.te == 2) {
+      // ---- One piece of a sum over K, kept as an fp32 plane of its own (Appendix A.2: the partial result a
+      // process holds before the all-reduce): the accumulator leaves through two 128B-swizzled staging boxes of
+      // [32 rows][32 columns] per warp and TMA stores into partials[s][M][N] (a 3-D map, so a tile's rows
+      // beyond M are clipped instead of landing in the next plane).  With a K range of a few k-blocks per
+      // piece the epilogue is most of a tile's time, and row-per-lane stores of 16 bytes keep the LSU busy
+      // for 32 cycles each; the bulk store takes the LSU out of the path.
+      const int e = warp - 2;
+      const uint32_t stg = ring + STAGES_TEP * STAGE_BYTES + e * (2 * 4096);
+      uint8_t* stg_gen = smem_raw + (stg - smem_u32(smem_raw));
+      int it = 0, nb = 0;
+      bool ok = true;
+      for (int w = w_first; w < total_work && ok; w += w_step, ++it) {
+        const Work wk = decode_work<FIX>(p, w);
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1u;
+        const int row0 = wk.tm * TILE_M + static_cast<int>(rank) * BMT + q * 32;
+        const int col0 = wk.tn * BN + half * HC;
+        ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_COLS + half * HC;
+#pragma unroll
+        for (int c = 0; c < HC / 32; ++c, ++nb) {
+          uint32_t r[32];
+          tc_ld32(taddr + c * 32, r);
+          // the store that used this box two chunks ago has read it
+          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          __syncwarp();
+          tc_wait_ld();
+          if (c == HC / 32 - 1) {                    // accumulator fully in registers: hand it back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+              if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty_bar[acc]), 0));
+              else mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+            }
+          }
+          uint8_t* box = stg_gen + (nb & 1) * 4096 + lane * 128;
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<uint4*>(box + ((j ^ (lane & 7)) << 4)) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // generic writes -> visible to TMA
+          __syncwarp();
+          if (lane == 0) {
+            asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                         ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(col0 + c * 32), "r"(row0), "r"(wk.s),
+                           "r"(stg + (nb & 1) * 4096)
+                         : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+        }
+      }
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // stores done before the CTA exits
+      __syncwarp();
+    } else if (te) {
       // ---- TMA epilogue: the tile's old weights / mask source arrive in this warp's staging boxes by
       // TMA, are combined in place with the accumulator, and leave by TMA store; the LSU never touches
       // global memory.  A box ([32 rows][64 columns] bf16) is requested for the NEXT tile as soon as its
@@ -749,6 +807,18 @@ cudaError_t make_map(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// 3-D fp32 tensor map over partials[S][M][N]; box = [1][32 rows][32 columns] (128 bytes per row, 128B-swizzled).
+cudaError_t make_planes_map(CUtensorMap* tm, const float* base, uint64_t N, uint64_t M, uint64_t S) {
+  const cuuint64_t dims[3] = {N, M, S};
+  const cuuint64_t strides[2] = {N * 4, N * M * 4};
+  const cuuint32_t box[3] = {32, 32, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 template <int A_MN, int B_MN>
 cudaError_t set_attr() {
   cudaError_t e;
@@ -903,6 +973,14 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
     g.fix = g.allow_fix && g.pair && two && tiles >= slots && kb_piece >= 32 ? 1 : 0;
     g.flag_words = g.fix ? tiles * 32 : 0;
   }
+  // S planes of short pieces on 128-row tiles leave by TMA store: a piece of fewer than 32 k-blocks is over before
+  // its predecessor's row-per-lane stores are (measured: batch-512 backward-weight products in 16 pieces of 8
+  // k-blocks 0.49 -> 0.31 ms); long pieces hide those stores and keep the two extra ring stages instead
+  // (8192-deep pieces of 64 k-blocks on CTA pairs: 2.5 % slower with the bulk stores).  The map is made at launch.
+  {
+    const int kb_piece = kb_total / (g.k_splits > 0 ? g.k_splits : 1);
+    g.te_planes = g.k_splits > 1 && !g.fix && g.MH == 1 && (g.N & 3) == 0 && kb_piece < 32 && !getenv("MBD_TC_NO_TE");
+  }
   // TMA epilogue: bf16 output of an unsplit contraction on 128-row tiles
   g.te = 0;
   g.tmOut = g.tmA;
@@ -938,6 +1016,20 @@ cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
   p.status = g.status;
   p.te = g.te && g.epi.op == g.te_epi.op && g.epi.out == g.te_epi.out && g.epi.out_bf16 && g.epi.mask == g.te_epi.mask &&
          g.epi.ldo == g.te_epi.ldo && g.k_splits == 1 && !g.epi.master;   // the TMA epilogue has no master path
+  // S planes on 128-row tiles: stored by TMA when the planes can be described by a tensor map
+  if (g.te_planes && g.k_splits > 1 && !p.fix && g.partials && (reinterpret_cast<uintptr_t>(g.partials) & 15u) == 0) {
+    if (g.planes_base != g.partials) {
+      const cudaError_t e = make_planes_map(&g.tmPlanes, g.partials, g.N, g.M, g.k_splits);
+      if (e != cudaSuccess) return e;
+      g.planes_base = g.partials;
+    }
+    p.te = 2;
+    TcGemm h = g;
+    h.tmOut = g.tmPlanes;
+    if (g.variant == 0) return launch_t<0, 0>(h, p, stream);
+    if (g.variant == 1) return launch_t<0, 1>(h, p, stream);
+    return launch_t<1, 1>(h, p, stream);
+  }
   if (g.variant == 0) return launch_t<0, 0>(g, p, stream);
   if (g.variant == 1) return launch_t<0, 1>(g, p, stream);
   return launch_t<1, 1>(g, p, stream);

@@ -92,6 +92,7 @@ struct TcGemm {
   CUtensorMap tmA, tmB;
   CUtensorMap tmOut, tmAux;   // output / mask-source maps of the TMA epilogue (valid when te)
   int te;                     // plan allows the TMA epilogue for te_epi
+  int te_planes;              // out: the S > 1 fp32 planes leave through TMA stores (short pieces on 128-row tiles)
   Epi te_epi;
   int variant;
   int BN;               // CTA tile width: 256 or 128
@@ -109,6 +110,10 @@ struct TcGemm {
   Epi epi;
   int* status;
   int grid;
+  // fp32 planes written by TMA (k_splits > 1 on 128-row tiles): the map over partials[S][M][N], encoded at the
+  // first launch that sees `partials` (the workspace is the caller's and is known only then)
+  mutable CUtensorMap tmPlanes;
+  mutable const float* planes_base = nullptr;
 };
 
 // Fills tmA/tmB/BN/grid.  Returns cudaSuccess or an error.

@@ -930,7 +930,7 @@ extern "C" mbd_status mbd_get_plan(const mbd_net* n, int layer, int product, mbd
   out->tile_n = g.BN;
   out->cta_pair = g.pair;
   out->k_pieces = g.k_splits;
-  out->tma_epilogue = g.te;
+  out->tma_epilogue = g.te_planes ? 2 : g.te;
   out->ctas = g.grid;
   out->running_sum = g.fix;
   out->reserved = 0;

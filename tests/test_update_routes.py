@@ -95,6 +95,25 @@ def test_fused_update_equals_unfused_update_bit_for_bit(monkeypatch, net_case, e
         assert np.array_equal(a["new_b"][i], b["new_b"][i]), f"b[{i}]"
 
 
+def test_planes_stored_by_tma_equal_planes_stored_from_registers(monkeypatch, net_case):
+    # Short pieces of a sum over K leave the product as fp32 planes through TMA stores (a 3-D map over
+    # partials[S][M][N]: rows of a ragged last tile -- M = 1000 here -- must be clipped, not land in the next
+    # plane); the same planes written by the epilogue's own stores must agree bit for bit, and so must
+    # everything computed from them.
+    w, inp, o, eta = net_case
+    grid, mp = (2, 3), 3
+    plans = _plan_of(w, grid, mp)
+    assert [(q["k_pieces"], q["tma_epilogue"]) for q in plans] == [(3, 2)] * 3, plans
+    a = gpu_fc_step(w, inp, grid, max_partials=mp, fused=False, force_acts=oracle_hidden_acts(o), eta=eta)
+    monkeypatch.setenv("MBD_TC_NO_TE", "1")
+    assert all(q["tma_epilogue"] == 0 for q in _plan_of(w, grid, mp))
+    b = gpu_fc_step(w, inp, grid, max_partials=mp, fused=False, force_acts=oracle_hidden_acts(o), eta=eta)
+    for i in range(3):
+        assert np.array_equal(a["dW"][i], b["dW"][i]) and np.array_equal(a["dY"][i], b["dY"][i]), i
+        assert np.array_equal(a["new_W"][i], b["new_W"][i]), i
+    compare_fc_step(a, o, TOL, False, init=inp, require_sized=True)
+
+
 def test_stand_alone_update_kernels_against_the_definition():
     # mbd_block_reduce with the SGD tail on one complete plane is Eq. 1 applied to a given gradient: bf16 weights
     # through the 16-byte path and (with a width that is not a multiple of 8) the element-wise path
