@@ -127,8 +127,11 @@ enum {
  *                 of a product with more output tiles than SMs) added as a running sum inside the
  *                 product -- the CTA that finishes piece s of a tile adds it to the
  *                 sum of pieces 0..s-1 that the CTA before it left in one fp32 plane
- *                 and the last one applies the tail operation.  Both forms add in
- *                 ascending block order and give bit-identical results.
+ *                 and the last one applies the tail operation -- or (two or four short
+ *                 pieces) kept as S accumulators of one tile in tensor memory, which the
+ *                 product's epilogue adds before its tail operation.  All three forms add
+ *                 in ascending block order and give bit-identical results; mbd_get_plan
+ *                 tells which one a product uses.
  *   cuda_stream   a cudaStream_t (may be NULL for the default stream).
  * Layer order (Section 2.4, Eq. 9): domain-split convolutions first (L_D), model-split
  * fully connected layers after them (L_M); either group may be empty.  With both present
@@ -305,7 +308,8 @@ MBD_API int64_t mbd_launch_count(const mbd_net* net);
  * or a benchmark state which kernel variant it ran.  tile_m x tile_n is the output tile of one work
  * unit (of the CTA pair when cta_pair != 0); k_pieces the number of fp32 partial sums the K range is
  * cut into (the grid's S = min(P, max_partials) times any further cut the planner added); running_sum != 0:
- * the pieces are added inside the product's own epilogue (see max_partials of mbd_net_create), otherwise
+ * the pieces are added inside the product's own epilogue (see max_partials of mbd_net_create; 1: as a running sum
+ * through one fp32 plane, 2: as accumulators of their own in tensor memory), otherwise
  * k_pieces > 1 means a reduce_partials launch follows; tma_epilogue = 1: the tail operation the plan was made for (bias +
  * ReLU, ReLU mask, fused update) moves its global data by TMA; tma_epilogue = 2: the k_pieces fp32 partial sums are
  * stored by TMA (short pieces on 128-row tiles); ctas: CTAs launched.

@@ -95,18 +95,34 @@ struct Params {
   int fix;                // running sum: piece s adds its accumulator to the sum pieces 0..s-1 left in `partials`
                           // (1: the pieces of a raster group follow one another; 2: all tiles piece by piece)
   int* flags;             // fix: one word per (tile, CTA of the pair, 128-row half, epilogue warp); zero between launches
+  int join;               // > 1: a tile's `join` K pieces are accumulators of their own in tensor memory, added in the epilogue
 };
 
 struct Work {
   int tm, tn, s, kb0, kb1;
 };
 
+// Joined pieces: r (piece 0's 32 columns of this lane's row) += the same columns of pieces 1 .. join-1, in
+// ascending order, each from the accumulator `stride` TMEM columns further on.
+__device__ __forceinline__ void add_joined_pieces(uint32_t taddr, int join, int stride, uint32_t* r) {
+  for (int s = 1; s < join; ++s) {
+#pragma unroll
+    for (int o = 0; o < 32; o += 8) {          // eight columns at a time: the caller's registers are nearly all taken
+      uint32_t t[8];
+      tc::tc_ld8(taddr + s * stride + o, t);
+      tc::tc_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 8; ++i) r[o + i] = __float_as_uint(__uint_as_float(r[o + i]) + __uint_as_float(t[i]));
+    }
+  }
+}
+
 template <int FIX>
 __device__ __forceinline__ Work decode_work(const Params& p, int w) {
   const int num_tiles = p.tiles_m * p.tiles_n;
   const int per_group = p.group_m * p.tiles_n;
   Work o;
-  if (FIX && p.fix == 1) {
+  if (FIX == 1 && p.fix == 1) {
     // Running sum: the pieces of a raster group follow one another (all tiles of the group for piece 0,
     // then for piece 1, ...), so that piece s of a tile finds the sum of pieces 0..s-1 still in L2 and
     // the unit it depends on always has a smaller index than itself.
@@ -174,6 +190,9 @@ static __device__ __noinline__ bool flag_wait(const int* flag, int value, volati
 // epilogue: 64 B/clk of operand fill like the 256 x 256 tile, but with two accumulators (the
 // epilogue overlaps the next tile), 32 KB stages and the TMA epilogue.
 // FIX = 1: the instantiation that can add a product's K pieces as a running sum in its epilogue (CTA pairs only).
+// FIX = 2: the instantiation that keeps a tile's K pieces as accumulators of their own in tensor memory (p.join).
+// Both are kept apart so that the FIX = 0 instantiations compile to the code they had (a run-time branch in the
+// shared epilogue cost 3 - 4 % of a cfg2 / cfg3 step).
 template <int A_MN, int B_MN, int BN, int MH, int PAIR, int FIX>
 // 136 registers per thread at most (a few bytes of spill in three instantiations): the register file
 // is split over the SM's four sub-partitions, the busiest of which holds three of this CTA's ten
@@ -217,7 +236,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (threadIdx.x == 0) atomicCAS(p.status, 0, DEV_SMEM_MISALIGNED);
     return;
   }
-  const bool te = !FIX && MH == 1 && p.te != 0;
+  const bool te = FIX != 1 && MH == 1 && p.te != 0;
+  // Joined pieces (p.join = 2 or 4): the K range of a tile is cut into p.join pieces, each accumulated in TMEM
+  // columns of its own; the epilogue adds them in ascending order -- the sum the reduction kernel would form over
+  // p.join planes, without the planes.  The accumulators of one tile then take p.join * ACC_COLS columns.
+  constexpr bool JOIN = FIX == 2 && ACC_COLS <= 256;           // (a tile that fills tensor memory has no room for a second piece)
+  const int join = JOIN ? p.join : 1;
+  const int acc_stride = join * ACC_COLS;
+  const int acc_bufs = JOIN && join > 1 ? (2 * acc_stride <= 512 ? 2 : 1) : ACC_BUFS;
+  const int tmem_cols = JOIN && join > 1 ? 512 : TMEM_COLS;
   const int stages = te ? (p.te == 2 ? STAGES_TEP : STAGES_TE) : STAGES;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -241,11 +268,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 1) {
     if (PAIR) {
       asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                   "r"(TMEM_COLS) : "memory");
+                   "r"(tmem_cols) : "memory");
       asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     } else {
       asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                   "r"(TMEM_COLS) : "memory");
+                   "r"(tmem_cols) : "memory");
       asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
   }
@@ -310,13 +337,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       for (int w = w_first; w < total_work && ok; w += w_step, ++it) {
         const Work wk = decode_work<FIX>(p, w);
-        const int acc = it % ACC_BUFS;
-        const uint32_t acc_phase = (it / ACC_BUFS) & 1u;
+        const int acc = it % acc_bufs;
+        const uint32_t acc_phase = (it / acc_bufs) & 1u;
         ok = mbar_wait(smem_u32(&tmem_empty_bar[acc]), acc_phase ^ 1u, abortp, p.status, DEV_TIMEOUT_MMA_TMEM);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
+        uint32_t d_tmem = tmem_base + acc * acc_stride;
+        int piece = 0, piece_kb0 = wk.kb0;                 // joined pieces: the balanced ranges of the K blocks
         for (int kb = wk.kb0; kb < wk.kb1; ++kb) {
+          if (JOIN && join > 1 && kb == static_cast<int>((static_cast<long long>(piece + 1) * p.kb_total) / join)) {
+            ++piece;
+            piece_kb0 = kb;
+            d_tmem += ACC_COLS;
+          }
           ok = mbar_wait(smem_u32(&full_bar[stage]), phase, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
           if (!ok) break;
           tc_fence_after();
@@ -332,9 +365,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
             for (int h = 0; h < MH; ++h) {
               if (PAIR) tc_mma_bf16_pair(d_tmem + h * BN, adesc + h * A_HALF + k * A_STEP, bdesc + k * B_STEP, IDESC,
-                                         (kb > wk.kb0 || k > 0) ? 1u : 0u);
+                                         (kb > piece_kb0 || k > 0) ? 1u : 0u);
               else tc_mma_bf16(d_tmem + h * BN, adesc + h * A_HALF + k * A_STEP, bdesc + k * B_STEP, IDESC,
-                               (kb > wk.kb0 || k > 0) ? 1u : 0u);
+                               (kb > piece_kb0 || k > 0) ? 1u : 0u);
             }
           }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
@@ -451,15 +484,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int b = 0; b < TE_BOXES; ++b) request(wk, b);
         }
-        const int acc = it & 1;
-        const uint32_t acc_phase = (it >> 1) & 1u;
+        const int acc = it % acc_bufs;
+        const uint32_t acc_phase = (it / acc_bufs) & 1u;
         const int row0 = wk.tm * TILE_M + static_cast<int>(rank) * BMT + q * 32;
         const int col0 = wk.tn * BN + half * HC;
         ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_COLS + half * HC;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * acc_stride + half * HC;
 #pragma unroll
         for (int b = 0; b < TE_BOXES; ++b) {
           if (need_load) {
@@ -477,6 +510,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t r[32];
             tc_ld32(taddr + c * 32, r);
             tc_wait_ld();
+            if (JOIN && join > 1) add_joined_pieces(taddr + c * 32, join, ACC_COLS, r);
             if (c == HC / 32 - 1) {                  // accumulator fully in registers: hand it back
               tc_fence_before();
               __syncwarp();
@@ -545,7 +579,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
       if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // stores done before the CTA exits
       __syncwarp();
-    } else if (FIX && p.fix != 0) {
+    } else if (FIX == 1 && p.fix != 0) {
       // ---- Running sum of a product's K pieces (Appendix A.2: the sum over the blocks of a process group,
       // taken in ascending block order).  Piece s of a tile adds its accumulator to the sum of pieces
       // 0..s-1, which the CTA that finished piece s-1 left in ONE fp32 plane, and writes the new sum back;
@@ -669,6 +703,53 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }   // h
       }
+    } else if (JOIN && join > 1) {
+      // ---- Joined pieces without the TMA epilogue (fp32 results, ragged leading dimensions, 256-row tiles): each
+      // 32-column chunk is the ascending sum of the tile's accumulators, then the tail operation from registers.
+      int it = 0;
+      bool ok = true;
+      for (int w = w_first; w < total_work && ok; w += w_step, ++it) {
+        const Work wk = decode_work<FIX>(p, w);
+        const int acc = it % acc_bufs;
+        const uint32_t acc_phase = (it / acc_bufs) & 1u;
+        const int64_t nbase = static_cast<int64_t>(wk.tn) * BN + half * HC;
+        ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_phase, abortp, p.status, DEV_TIMEOUT_EPILOGUE);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll 1
+        for (int h = 0; h < MH; ++h) {
+          const int64_t m = static_cast<int64_t>(wk.tm) * TILE_M + rank * BMT + h * 128 + q * 32 + lane;
+          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * acc_stride + h * BN + half * HC;
+#pragma unroll 1
+          for (int c = 0; c < HC / 32; ++c) {
+            uint32_t r[32];
+            tc_ld32(taddr + c * 32, r);
+            tc_wait_ld();
+            add_joined_pieces(taddr + c * 32, join, ACC_COLS, r);
+            if (h == MH - 1 && c == HC / 32 - 1) {     // accumulators fully in registers: hand them back
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) {
+                if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty_bar[acc]), 0));
+                else mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+              }
+            }
+            if (m < p.M) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int64_t n = nbase + c * 32 + j * 8;
+                if (n < p.N) {
+                  float v[8];
+#pragma unroll
+                  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j * 8 + i]);
+                  epi_apply8(p.epi, m, n, v);
+                }
+              }
+            }
+          }
+        }
+      }
     } else {
     const bool prefetch = p.S == 1 && p.epi.out_bf16 &&
                           ((p.epi.op == EPI_SGD && p.epi.master == nullptr) ||      // master weights: shared tail, no prefetch
@@ -766,8 +847,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
-    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
   }
 }
 
@@ -829,6 +910,10 @@ cudaError_t set_attr() {
   if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 256, 1, 0, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 1, 0, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 2, 0, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES)) != cudaSuccess) return e;
   return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, 128, 2, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_BYTES);
 }
 
@@ -839,6 +924,12 @@ cudaError_t launch_t(const TcGemm& g, const Params& p, cudaStream_t stream) {
   if (g.pair && p.fix) {
     if (g.MH == 2) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1, 1>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
     return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1, 1>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+  }
+  if (p.join > 1) {        // (the planner admits only these four shapes)
+    if (g.pair) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1, 2>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+    if (g.BN == 256) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 1, 0, 2>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+    if (g.MH == 1) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 128, 1, 0, 2>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
+    return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 128, 2, 0, 2>, grid, block, smem, stream, 1, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
   }
   if (g.pair && g.MH == 2) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 2, 1, 0>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
   if (g.pair) return launch_pdl(gemm_tc_kernel<A_MN, B_MN, 256, 1, 1, 0>, grid, block, smem, stream, 2, g.tmA, g.tmB, g.tmOut, g.tmAux, p);
@@ -889,16 +980,24 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
   // costs fp32 partial traffic and the reduction launch.  Checked against measurements: 8192^3 picks
   // 256 x 256 (1236 -> 1445 TFLOP/s), the batch-512 forward product 512 x 4096 x 25088 picks
   // 256 x 256 with K cut in 4; short-K and split products pick CTA pairs (cta_group::2).
+  // Short pieces whose planes nobody asked to see may stay in tensor memory (`join`): the tile's K range is
+  // walked piece by piece into accumulators of their own, and the epilogue adds them in ascending order -- the
+  // sum of the reduction kernel over the same pieces, bit for bit, with no fp32 plane crossing HBM.  Needs
+  // k_splits x (tile's TMEM columns) <= 512; measured: cfg3 1x16 (two pieces of 4 k-blocks) 0.67 -> 0.34 ms per step.
+  const bool join_ok = g.allow_fix && (g.k_splits == 2 || g.k_splits == 4) && !getenv("MBD_NO_JOIN") &&
+                       (kb_total / g.k_splits < 32 || getenv("MBD_JOIN_ANY"));        // tuning knobs
+  g.join = 1;
   {
     double best = 1e30;
-    int best_bn = 128, best_mh = 1, best_x = 1, best_pair = 0;
+    int best_bn = 128, best_mh = 1, best_x = 1, best_pair = 0, best_join = 0;
     const int x_max = g.allow_extra_split ? 32 : 1;
     for (int cand = 0; cand < 4; ++cand) {           // 0: 128-row tiles, 1: 256-row tiles, 2: CTA pairs, 3: pairs of 256-row CTAs
       const int mh = (cand == 1 || cand == 3) ? 2 : 1;
       const bool pair = cand >= 2;
       for (int bn = pair ? 256 : 128; bn <= 256; bn += 128) {
-        for (int x = 1; x <= x_max; x *= 2) {
-          const long long S = 1ll * g.k_splits * x;
+        for (int jn = 0; jn <= (join_ok && g.k_splits * mh * bn <= 512 ? 1 : 0); ++jn) {
+        for (int x = 1; x <= (jn ? 1 : x_max); x *= 2) {
+          const long long S = jn ? 1 : 1ll * g.k_splits * x;
           if (S > kb_total || (x > 1 && kb_total / S < 8)) continue;
           const double kb = static_cast<double>(kb_total) / S;
           const int tile_m = 128 * mh * (pair ? 2 : 1);
@@ -911,20 +1010,25 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
           const double mma = 4.0 * mh * ((pair ? 256 : bn) / 2) / eff;
           const double fill = (pair ? 128.0 * mh + 128.0 : 128.0 * mh + bn) * 128.0 / 70.0;
           const double mainloop = kb * (mma > fill ? mma : fill);
-          const double epi = 2500.0 * mh * bn / 256.0 * (S > 1 ? 2.0 : 1.0);
+          const double epi = 2500.0 * mh * bn / 256.0 * (S > 1 ? 2.0 : 1.0) * (jn ? 1.0 + 0.25 * (g.k_splits - 1) : 1.0);
+          // (joined pieces take the shape the unsplit product would: a CTA pair whose two pieces fill tensor memory
+          // measured 14 % faster than 128 x 128 tiles with room for two sets on the batch-512 product, 4 % slower on
+          // the batch-256 one -- the model's epilogue estimate cannot tell them apart)
           const bool overlapped = mh * bn <= 256;        // two accumulators fit in TMEM
           double unit = overlapped ? (mainloop > epi ? mainloop : epi) : mainloop + epi;
           double t = waves * unit + 4000.0;
-          if (S > 1 && x > 1) {          // the reduction exists anyway when the grid itself splits K
+          if (S > 1 && (x > 1 || join_ok)) {   // the reduction exists anyway when the grid itself splits K and must keep planes
             const double bytes = (static_cast<double>(S) + 1.0) * g.M * g.N * 4.0;
             t += (5e-6 + bytes / 5.5e12) * 1.9e9;
           }
-          if (t < best) { best = t; best_bn = bn; best_mh = mh; best_x = x; best_pair = pair ? 1 : 0; }
+          if (t < best) { best = t; best_bn = bn; best_mh = mh; best_x = x; best_pair = pair ? 1 : 0; best_join = jn; }
+        }
         }
       }
     }
     g.BN = best_bn; g.MH = best_mh; g.pair = best_pair;
     g.k_splits *= best_x;
+    if (best_join) { g.join = g.k_splits; g.k_splits = 1; }
   }
   if (const char* ev = getenv("MBD_TC_MH")) {          // tuning knobs
     const int mh = atoi(ev);
@@ -940,9 +1044,11 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
     else if (atoi(ev) == 0) g.pair = 0;
   }
   if (g.pair) g.BN = 256;
+  if (g.join > 1 && g.join * g.MH * g.BN > 512) { g.k_splits = g.join; g.join = 1; }     // a forced tile shape without room
   if (getenv("MBD_TC_DEBUG"))
-    fprintf(stderr, "tc_gemm_prepare: variant %d  M %d N %d K %d  pieces of K %d  ->  %d x %d tile%s\n", g.variant, g.M, g.N,
-            g.K, g.k_splits, 128 * g.MH * (g.pair ? 2 : 1), g.BN, g.pair ? " (CTA pair)" : "");
+    fprintf(stderr, "tc_gemm_prepare: variant %d  M %d N %d K %d  pieces of K %d%s  ->  %d x %d tile%s\n", g.variant, g.M, g.N,
+            g.K, g.join > 1 ? g.join : g.k_splits, g.join > 1 ? " (joined in tensor memory)" : "", 128 * g.MH * (g.pair ? 2 : 1),
+            g.BN, g.pair ? " (CTA pair)" : "");
   const int bmt = BM * g.MH * (g.pair ? 2 : 1);        // rows of one work unit's tile
   const int tiles_m = (g.M + bmt - 1) / bmt;
   const int tiles_n = (g.N + g.BN - 1) / g.BN;
@@ -1012,6 +1118,7 @@ cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
   if (p.fix && getenv("MBD_FIX_PLAIN_ORDER")) p.fix = 2;                 // tuning knob
   p.te_prefetch = getenv("MBD_TE_NO_PREFETCH") ? 0 : 1;                  // tuning knob
   p.flags = g.flags;
+  p.join = g.join > 1 ? g.join : 1;
   p.epi = g.epi;
   p.status = g.status;
   p.te = g.te && g.epi.op == g.te_epi.op && g.epi.out == g.te_epi.out && g.epi.out_bf16 && g.epi.mask == g.te_epi.mask &&

@@ -102,6 +102,8 @@ struct TcGemm {
   int allow_fix;        // in: the S pieces need not be kept as S planes
   int fix;              // out: pieces are added as a running sum in the epilogue (one plane in `partials`, words in
                         // `flags`), in ascending order like the reduction kernel; no reduction launch follows
+  int join;             // out: > 1: that many pieces of K are accumulators of their own in tensor memory, added in ascending order by
+                        // the epilogue (k_splits is 1 then: nothing is written to `partials`, no reduction launch follows)
   long long flag_words; // out: ints `flags` must hold (zero-initialised; the kernel leaves them zero)
   int* flags;
   int M, N, K;

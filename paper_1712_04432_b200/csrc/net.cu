@@ -929,10 +929,10 @@ extern "C" mbd_status mbd_get_plan(const mbd_net* n, int layer, int product, mbd
   out->tile_m = 128 * g.MH * (g.pair ? 2 : 1);
   out->tile_n = g.BN;
   out->cta_pair = g.pair;
-  out->k_pieces = g.k_splits;
+  out->k_pieces = g.join > 1 ? g.join : g.k_splits;
   out->tma_epilogue = g.te_planes ? 2 : g.te;
   out->ctas = g.grid;
-  out->running_sum = g.fix;
+  out->running_sum = g.join > 1 ? 2 : g.fix;
   out->reserved = 0;
   return MBD_OK;
 }

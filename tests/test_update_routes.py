@@ -114,6 +114,27 @@ def test_planes_stored_by_tma_equal_planes_stored_from_registers(monkeypatch, ne
     compare_fc_step(a, o, TOL, False, init=inp, require_sized=True)
 
 
+@pytest.mark.parametrize("grid,mp", [((1, 4), 2), ((4, 8), 4), ((8, 1), 2), ((4, 4), 2)])
+@pytest.mark.parametrize("fused", [True, False])
+def test_pieces_joined_in_tensor_memory_equal_planes_and_reduction(monkeypatch, net_case, grid, mp, fused):
+    # Fewer partial sums than blocks (1 < S < P) and short pieces: the S pieces of a tile are accumulators of their
+    # own in tensor memory and the product's epilogue adds them in ascending order before its tail operation.
+    # Same pieces, same order as S fp32 planes and the reduction kernel: every bit must agree.
+    w, inp, o, eta = net_case
+    if grid[1] > 1:
+        plans = _plan_of(w, grid, mp)
+        assert [(q["k_pieces"], q["running_sum"]) for q in plans] == [(mp, 2)] * 3, plans
+    a = gpu_fc_step(w, inp, grid, max_partials=mp, fused=fused, force_acts=oracle_hidden_acts(o), eta=eta)
+    monkeypatch.setenv("MBD_NO_JOIN", "1")
+    assert all(q["running_sum"] == 0 for q in _plan_of(w, grid, mp))
+    b = gpu_fc_step(w, inp, grid, max_partials=mp, fused=fused, force_acts=oracle_hidden_acts(o), eta=eta)
+    for i in range(3):
+        assert np.array_equal(a["dY"][i], b["dY"][i]) and np.array_equal(a["new_W"][i], b["new_W"][i]), i
+        if not fused:
+            assert np.array_equal(a["dW"][i], b["dW"][i]), i
+    compare_fc_step(a, o, TOL, fused, init=inp, require_sized=True)
+
+
 def test_stand_alone_update_kernels_against_the_definition():
     # mbd_block_reduce with the SGD tail on one complete plane is Eq. 1 applied to a given gradient: bf16 weights
     # through the 16-byte path and (with a width that is not a multiple of 8) the element-wise path
