@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="cfg5", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--momentum", type=float, default=None,
+                    help="heavy-ball momentum with this mu (the update becomes a kernel of its own); not the default")
     ap.add_argument("--master-weights", action="store_true",
                     help="keep fp32 master weights (the update leaves the contraction's epilogue); not the default")
     ap.add_argument("--grid", default=None, help="P_r x P_c, e.g. 16x16 (default: the workload's second grid)")
@@ -294,6 +296,8 @@ def run_ours(args):
         labels = labels_host = None
     if args.master_weights:
         net.enable_master_weights()
+    if args.momentum is not None:
+        net.enable_momentum(args.momentum)
     X = dev(inp.X)
     X_host = X.cpu().pin_memory()
     J = torch.zeros(1, dtype=torch.float32, device="cuda")
@@ -466,7 +470,8 @@ def run_ours(args):
     line = dict(metric=METRIC, value=aggregate_tflops(flops, world, ms), unit="TFLOP/s", n_gpus=world,
                 steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=ms, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype=w.dtype, data="synthetic",
-                config=dict(workload_config(w, grid, args.max_partials), **({"master_weights": True} if args.master_weights else {})),
+                config=dict(workload_config(w, grid, args.max_partials), **({"master_weights": True} if args.master_weights else {}),
+                            **({"momentum": args.momentum} if args.momentum is not None else {})),
                 clocks=clocks, e2e=e2e,
                 gpu_launches=int(launches) * world, roofline=roofline, cpu_baseline=cpu,
                 frac_of_burst_peak=flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"] if bf else None,

@@ -111,7 +111,9 @@ enum {
   MBD_T_DB = 3,       /* db_i, float [d_i]                                                   */
   MBD_T_LOSS = 4,     /* per-sample loss, float [B] (softmax-CE); layer ignored              */
   MBD_T_PARTIALS = 5, /* fp32 partial-sum workspace as left by the LAST reduction executed   */
-  MBD_T_MASTER = 6    /* fp32 master weights, weight shape (get only; after mbd_enable_master_weights) */
+  MBD_T_MASTER = 6,   /* fp32 master weights, weight shape (get only; after mbd_enable_master_weights) */
+  MBD_T_VELOCITY = 7, /* momentum velocity of W_i, float, weight shape (get only; after mbd_enable_momentum) */
+  MBD_T_VELOCITY_BIAS = 8 /* momentum velocity of b_i, float [d_i] (fully connected layers with a bias)    */
 };
 
 /* Section 2.3 / 2.4.  Builds the plan for an L-layer network on batch B over a
@@ -161,6 +163,16 @@ MBD_API mbd_status mbd_net_destroy(mbd_net* net);
  * leaves the contraction's epilogue).  The masters start from the current weights and follow every
  * later mbd_set_weights.  MBD_E_UNSUPPORTED for an fp32 network (its weights are fp32 already). */
 MBD_API mbd_status mbd_enable_master_weights(mbd_net* net);
+
+/* Optional: heavy-ball momentum in place of the plain step of Eq. 1 (Section 2: SGD stands for any first-order
+ * method; forward pass, back-propagation and their communication are the same).  Per parameter
+ *     v <- mu v + dW / B ,   w <- w - eta v ,        0 <= mu < 1, v = 0 when this call returns;
+ * mu = 0 is Eq. 1.  The velocities are fp32 (4 more bytes per parameter, biases included).  The update no longer
+ * rides in a product's epilogue or a reduction's tail: with fused_eta > 0 mbd_backward materialises dW_i (as with
+ * fused_eta = 0) and one streaming kernel per layer applies the two lines above -- to the fp32 master when
+ * master weights are on, the bf16 weights being its rounding.  mbd_sgd_step does the same from the stored
+ * gradients.  Calling it again resets the velocities and sets a new mu.  MBD_E_INVALID for mu outside [0, 1). */
+MBD_API mbd_status mbd_enable_momentum(mbd_net* net, float mu);
 
 /* Copy weights (network dtype) and bias (float, may be NULL) device -> library / back. */
 MBD_API mbd_status mbd_set_weights(mbd_net* net, int layer, const void* W_dev, const float* bias_dev);

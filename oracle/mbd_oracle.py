@@ -189,6 +189,13 @@ def sgd(w, dw, eta, B):
     return np.asarray(w, F64) - (eta / B) * np.asarray(dw, F64)
 
 
+def sgd_momentum(w, v, dw, eta, B, mu):
+    """Heavy-ball momentum, the first-order method beside Eq. 1 (Section 2: the paper writes SGD for any
+    of them).  v <- mu v + dw / B, w <- w - eta v; returns (w_new, v_new).  mu = 0 is Eq. 1."""
+    v_new = mu * np.asarray(v, F64) + np.asarray(dw, F64) / B
+    return np.asarray(w, F64) - eta * v_new, v_new
+
+
 # --------------------------------------------------------------------------
 # one training step, un-blocked
 # --------------------------------------------------------------------------

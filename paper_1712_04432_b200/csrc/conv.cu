@@ -968,6 +968,8 @@ struct ConvNet {
   std::vector<bf16*> K, Wf, Wb;
   std::vector<float*> dK;
   std::vector<float*> K32;           // fp32 master weights (empty unless enabled)
+  std::vector<float*> Vk;            // momentum: velocities of the kernels (empty unless enabled), canonical [o][c][3][3]
+  float mu = 0.f;
   std::vector<int> relu;
   std::vector<int> k1;               // 1 x 1 layer: weights in the centre tap, outer taps zero
   std::vector<CUtensorMap> act_fwd, dY_fwd, dY_wg, wf_map, wb_map;   // act_fwd / dY_fwd: 130-pixel boxes (also the X operand of backward-weight)
@@ -1078,6 +1080,7 @@ void conv_destroy(ConvNet* c) {
     if (c->dY[i] != c->act[c->L]) cudaFree(c->dY[i]);
   for (int i = 0; i < c->L; ++i) { cudaFree(c->K[i]); cudaFree(c->Wf[i]); cudaFree(c->Wb[i]); cudaFree(c->dK[i]); }
   for (float* m : c->K32) cudaFree(m);
+  for (float* m : c->Vk) cudaFree(m);
   cudaFree(c->wpart); cudaFree(c->loss_part); cudaFree(c->scratch_nchw);
   (void)cudaGetLastError();
   delete c;
@@ -1117,6 +1120,36 @@ mbd_status conv_enable_master(ConvNet* c) {
   c->K32 = m;
   return MBD_OK;
 }
+
+mbd_status conv_enable_momentum(ConvNet* c, float mu) {
+  if (c->Vk.empty()) {
+    std::vector<float*> v(c->L, nullptr);
+    for (int i = 0; i < c->L; ++i) {
+      if (cudaMalloc(reinterpret_cast<void**>(&v[i]), 9 * C * C * 4) != cudaSuccess) {
+        (void)cudaGetLastError();
+        for (float* q : v) cudaFree(q);
+        return MBD_E_ALLOC;
+      }
+    }
+    c->Vk = v;
+  }
+  for (int i = 0; i < c->L; ++i)
+    if (cudaMemsetAsync(c->Vk[i], 0, 9 * C * C * 4, c->stream) != cudaSuccess) return MBD_E_CUDA;
+  c->mu = mu;
+  return MBD_OK;
+}
+
+namespace {
+// momentum update of layer i from its materialised gradient, then the two operand layouts of the new weights
+mbd_status momentum_update(ConvNet* c, int i, float eta) {
+  c->prof->begin(MBD_K_SGD, 9.0 * C * C * 14.0);
+  const cudaError_t e = sgd_momentum_update_launch(c->K[i], 1, c->K32.empty() ? nullptr : c->K32[i], c->Vk[i], c->dK[i], 9 * C * C, c->mu,
+                                                   1.f / static_cast<float>(c->B), eta, c->num_sms, c->stream);
+  c->prof->end();
+  if (e != cudaSuccess) return MBD_E_CUDA;
+  return launch_pack(c, i);
+}
+}  // namespace
 
 mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev) {
   if (c->k1[layer]) {
@@ -1191,7 +1224,8 @@ mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
 mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta, int rows) {
   if (i < 0 || i >= c->L) return MBD_E_INVALID;
   if (rows != MBD_ROWS_ALL && (c->P_r != 1 || (rows != MBD_ROWS_INTERIOR && rows != MBD_ROWS_BOUNDARY))) return MBD_E_UNSUPPORTED;
-  const bool fused = fused_eta > 0.f;
+  const bool momentum = !c->Vk.empty();
+  const bool fused = fused_eta > 0.f && !momentum;       // momentum: the gradient first, then the update kernel
   const float scale = -fused_eta / static_cast<float>(c->B);
   if (i > 0) {
     // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0]
@@ -1219,7 +1253,8 @@ mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta, int rows) {
                                                                     c->K32.empty() ? nullptr : c->K32[i], scale, c->k1[i]);
   c->prof->end();
   if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
-  if (i == 0) c->state = fused ? 3 : 2;
+  if (momentum && fused_eta > 0.f && momentum_update(c, i, fused_eta) != MBD_OK) return MBD_E_CUDA;
+  if (i == 0) c->state = fused_eta > 0.f ? 3 : 2;
   return MBD_OK;
 }
 
@@ -1260,6 +1295,10 @@ mbd_status conv_set_dw(ConvNet* c, int layer, const void* src, size_t bytes) {
 mbd_status conv_sgd_step(ConvNet* c, float eta) {
   const float scale = -eta / static_cast<float>(c->B);
   for (int i = 0; i < c->L; ++i) {
+    if (!c->Vk.empty()) {
+      if (momentum_update(c, i, eta) != MBD_OK) return MBD_E_CUDA;
+      continue;
+    }
     c->prof->begin(MBD_K_SGD, 9.0 * C * C * 8.0);
     const cudaError_t e = c->K32.empty() ? sgd_update_launch(c->K[i], 1, c->dK[i], 9 * C * C, scale, c->num_sms, c->stream)
                                          : sgd_master_update_launch(c->K32[i], c->K[i], c->dK[i], 9 * C * C, scale, c->num_sms, c->stream);
@@ -1291,10 +1330,11 @@ int conv_last_relu(const ConvNet* c) { return c->relu[c->L - 1]; }
 
 mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t bytes) {
   const size_t nchw_bytes = conv_input_bytes(c);
-  if (which == MBD_T_DW || which == MBD_T_MASTER) {
+  if (which == MBD_T_DW || which == MBD_T_MASTER || which == MBD_T_VELOCITY) {
     if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
     if (which == MBD_T_MASTER && c->K32.empty()) return MBD_E_STATE;
-    const float* src32 = which == MBD_T_DW ? c->dK[layer] : c->K32[layer];
+    if (which == MBD_T_VELOCITY && c->Vk.empty()) return MBD_E_STATE;
+    const float* src32 = which == MBD_T_DW ? c->dK[layer] : which == MBD_T_MASTER ? c->K32[layer] : c->Vk[layer];
     if (c->k1[layer]) {
       if (bytes != C * C * 4) return MBD_E_INVALID;
       extract_1x1_kernel<float><<<(C * C + 255) / 256, 256, 0, c->stream>>>(src32, static_cast<float*>(dst));

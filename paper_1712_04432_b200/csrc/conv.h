@@ -25,6 +25,7 @@ mbd_status conv_output_to_nchw(ConvNet* c, void* dst);
 mbd_status conv_top_grad_from_nchw(ConvNet* c, const void* src);
 int conv_last_relu(const ConvNet* c);
 mbd_status conv_enable_master(ConvNet* c);     // fp32 master weights from now on
+mbd_status conv_enable_momentum(ConvNet* c, float mu);   // heavy-ball momentum from now on (velocities start at zero)
 // the step piece by piece, and the outer rows of the images (for a driver with one process per strip)
 mbd_status conv_stage_input(ConvNet* c, const void* X_nchw);
 // rows: MBD_ROWS_ALL, or (one strip per network only) MBD_ROWS_INTERIOR / MBD_ROWS_BOUNDARY -- see include/mbd.h

@@ -453,6 +453,36 @@ cudaError_t colsum_launch(const void* dY, int dy_bf16, int64_t M, int64_t N, flo
                     row_splits * 8, N, db, bias, scale);
 }
 
+// Heavy-ball momentum, the first-order method next to plain SGD (Section 2: the analysis holds for any of them):
+//   v <- mu v + g / B ;  w <- w - eta v        (v starts at zero; mu = 0 is Eq. 1)
+// on fp32 weights, bf16 weights (one rounding of the new weight) or an fp32 master whose rounding is the bf16 copy.
+__global__ void __launch_bounds__(256)
+sgd_momentum_update_kernel(void* __restrict__ w, int w_bf16, float* __restrict__ w32, float* __restrict__ v,
+                           const float* __restrict__ g, int64_t n, float mu, float inv_B, float eta) {
+  pdl_wait();
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const float vel = fmaf(mu, v[i], g[i] * inv_B);
+    v[i] = vel;
+    if (w_bf16) {
+      __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(w) + i;
+      const float old = w32 ? w32[i] : __bfloat162float(*p);
+      const float nw = fmaf(-eta, vel, old);
+      if (w32) w32[i] = nw;
+      *p = __float2bfloat16_rn(nw);
+    } else {
+      float* p = reinterpret_cast<float*>(w) + i;
+      *p = fmaf(-eta, vel, *p);
+    }
+  }
+}
+
+cudaError_t sgd_momentum_update_launch(void* w, int w_bf16, float* w32, float* v, const float* g, int64_t n, float mu,
+                                       float inv_B, float eta, int num_sms, cudaStream_t stream) {
+  return launch_pdl(sgd_momentum_update_kernel, dim3(grid_for(n, num_sms, 8)), dim3(256), 0, stream, 0, w, w_bf16, w32, v, g, n,
+                    mu, inv_B, eta);
+}
+
 cudaError_t sgd_update_launch(void* w, int w_bf16, const float* g, int64_t n, float scale, int num_sms,
                               cudaStream_t stream) {
   if (w_bf16 && n % 8 == 0) {

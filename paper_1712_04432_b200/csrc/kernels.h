@@ -157,6 +157,9 @@ int colsum_launches(int64_t M, int64_t N, int num_sms);    // kernels one colsum
 cudaError_t sgd_update_launch(void* w, int w_bf16, const float* g, int64_t n, float scale,
                               int num_sms, cudaStream_t stream);
 
+// Heavy-ball momentum: v = mu v + g inv_B; w -= eta v (w fp32, bf16, or bf16 copy of the fp32 master w32).
+cudaError_t sgd_momentum_update_launch(void* w, int w_bf16, float* w32, float* v, const float* g, int64_t n, float mu,
+                                       float inv_B, float eta, int num_sms, cudaStream_t stream);
 // fp32 master weights: w32[i] += scale * g[i]; w_bf16[i] = round(w32[i]).  widen: w32[i] = w_bf16[i].
 cudaError_t sgd_master_update_launch(float* w32, void* w_bf16, const float* g, int64_t n, float scale,
                                      int num_sms, cudaStream_t stream);

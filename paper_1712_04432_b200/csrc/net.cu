@@ -30,6 +30,8 @@ struct Layer {
   float* bias = nullptr;
   float* dW = nullptr;
   float* W32 = nullptr;  // fp32 master weights (optional)
+  float* V = nullptr;    // momentum: velocity of W (optional), fp32
+  float* Vb = nullptr;   // momentum: velocity of the bias
   float* db = nullptr;
   void* act = nullptr;   // stored forward output [B, d_out]; float logits for the last FC layer
   void* dY = nullptr;    // [B, d_out] activation dtype
@@ -51,6 +53,8 @@ struct mbd_net {
   int device = 0;
   bool is_conv = false;
   bool master = false;              // fp32 master weights: the update leaves the contraction's epilogue
+  bool momentum = false;            // heavy-ball momentum: the update is a kernel of its own after the gradient
+  float mu = 0.f;
   std::vector<Layer> layers;
   float* partials = nullptr;
   size_t partial_elems = 0;
@@ -249,7 +253,7 @@ mbd_status map_input(mbd_net* n) {
 void free_net(mbd_net* n) {
   if (!n) return;
   for (Layer& l : n->layers) {
-    cudaFree(l.W); cudaFree(l.bias); cudaFree(l.dW); cudaFree(l.db); cudaFree(l.act); cudaFree(l.dY); cudaFree(l.W32);
+    cudaFree(l.W); cudaFree(l.bias); cudaFree(l.dW); cudaFree(l.db); cudaFree(l.act); cudaFree(l.dY); cudaFree(l.W32); cudaFree(l.V); cudaFree(l.Vb);
   }
   cudaFree(n->partials); cudaFree(n->colsum_scratch); cudaFree(n->colsum_scratch_aux); cudaFree(n->per_sample); cudaFree(n->loss_dev);
   cudaFree(n->status); cudaFree(n->X_stage); cudaFree(n->labels_stage); cudaFree(n->X_fc); cudaFree(n->dX_fc);
@@ -502,6 +506,27 @@ extern "C" mbd_status mbd_enable_master_weights(mbd_net* n) {
   return MBD_OK;
 }
 
+extern "C" mbd_status mbd_enable_momentum(mbd_net* n, float mu) {
+  if (!n || !(mu >= 0.f && mu < 1.f)) return MBD_E_INVALID;
+  if (n->conv) {
+    const mbd_status s = conv_enable_momentum(n->conv, mu);
+    if (s != MBD_OK) return s;
+  }
+  for (Layer& l : n->layers) {
+    if (!l.V) {
+      mbd_status s = dev_alloc(reinterpret_cast<void**>(&l.V), l.nW * sizeof(float));
+      if (s == MBD_OK && l.bias) s = dev_alloc(reinterpret_cast<void**>(&l.Vb), l.d_out * sizeof(float));
+      if (s != MBD_OK) return s;
+    }
+    CK(cudaMemsetAsync(l.V, 0, l.nW * sizeof(float), n->stream));
+    if (l.Vb) CK(cudaMemsetAsync(l.Vb, 0, l.d_out * sizeof(float), n->stream));
+  }
+  n->momentum = true;
+  n->mu = mu;
+  if (n->graph_exec) { cudaGraphExecDestroy(n->graph_exec); n->graph_exec = nullptr; }   // the step's launches change
+  return MBD_OK;
+}
+
 extern "C" mbd_status mbd_get_weights(mbd_net* n, int layer, void* W_dev, float* bias_dev) {
   if (!n || !W_dev || layer < 0 || layer >= n->Lc + n->L) return MBD_E_INVALID;
   if (layer < n->Lc) return bias_dev ? MBD_E_INVALID : conv_get_weights(n->conv, layer, W_dev);
@@ -591,10 +616,16 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
         forked = true;
       }
       n->prof.begin(MBD_K_COLSUM, static_cast<double>(n->B) * l.d_out * (bf ? 2.0 : 4.0), cs);
-      CK(colsum_launch(l.dY, bf, n->B, l.d_out, cs == n->aux ? n->colsum_scratch_aux : n->colsum_scratch, colsum_row_splits(n->B, l.d_out, n->num_sms), fused ? nullptr : l.db,
-                       fused ? l.bias : nullptr, scale, cs));
+      const bool fused_b = fused && !n->momentum;          // momentum: db first, then the update kernel
+      CK(colsum_launch(l.dY, bf, n->B, l.d_out, cs == n->aux ? n->colsum_scratch_aux : n->colsum_scratch, colsum_row_splits(n->B, l.d_out, n->num_sms), fused_b ? nullptr : l.db,
+                       fused_b ? l.bias : nullptr, scale, cs));
       n->prof.end();
       n->prof.total_launches += colsum_launches(n->B, l.d_out, n->num_sms) - 1;
+      if (fused && n->momentum) {
+        n->prof.begin(MBD_K_SGD, static_cast<double>(l.d_out) * 20.0, cs);
+        CK(sgd_momentum_update_launch(l.bias, 0, nullptr, l.Vb, l.db, l.d_out, n->mu, 1.f / static_cast<float>(n->B), fused_eta, n->num_sms, cs));
+        n->prof.end();
+      }
     }
     if (i > 0 || n->mixed) {   // nothing is propagated below the first layer of the network
       const Epi e = bwd_data_epi(n, i);
@@ -604,8 +635,8 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
     // With master weights: a split product updates the fp32 master in the tail of its reduction (which streams
     // the sum through registers anyway); an unsplit one materialises the gradient and a streaming kernel applies
     // Eq. 1 to the master (measured equal to doing it in the product's epilogue, whose loads would be exposed).
-    const bool master_tail = fused && n->master && bf && l.bwd_weight.k_splits > 1;
-    const bool master_kernel = fused && n->master && !master_tail;
+    const bool master_tail = fused && n->master && !n->momentum && bf && l.bwd_weight.k_splits > 1;
+    const bool master_kernel = fused && (n->master || n->momentum) && !master_tail;     // momentum: always a kernel of its own
     const Epi e = (fused && !master_kernel) ? epi_sgd(l.W, l.d_in, bf, scale, master_tail ? l.W32 : nullptr)
                                             : epi_act(l.dW, l.d_in, 0, nullptr, 0);
     cudaStream_t ws = nullptr;
@@ -622,8 +653,11 @@ extern "C" mbd_status mbd_backward(mbd_net* n, float fused_eta) {
     if (s != MBD_OK) return s;
     if (master_kernel) {
       cudaStream_t us = ws ? ws : n->stream;
-      n->prof.begin(MBD_K_SGD, static_cast<double>(l.nW) * 14.0, us);
-      CK(sgd_master_update_launch(l.W32, l.W, l.dW, l.nW, scale, n->num_sms, us));
+      n->prof.begin(MBD_K_SGD, static_cast<double>(l.nW) * (n->momentum ? 12.0 + 2.0 * n->elt() + (l.W32 ? 8.0 : 0.0) : 14.0), us);
+      if (n->momentum)
+        CK(sgd_momentum_update_launch(l.W, bf, l.W32, l.V, l.dW, l.nW, n->mu, 1.f / static_cast<float>(n->B), fused_eta, n->num_sms, us));
+      else
+        CK(sgd_master_update_launch(l.W32, l.W, l.dW, l.nW, scale, n->num_sms, us));
       n->prof.end();
     }
   }
@@ -662,12 +696,15 @@ extern "C" mbd_status mbd_sgd_step(mbd_net* n, float eta) {
   for (int i = 0; i < n->L; ++i) {
     Layer& l = n->layers[i];
     n->prof.begin(MBD_K_SGD, static_cast<double>(l.nW) * (n->master ? 14.0 : 4.0 + 2.0 * n->elt()));
-    if (n->master) CK(sgd_master_update_launch(l.W32, l.W, l.dW, l.nW, scale, n->num_sms, n->stream));
+    const float inv_B = 1.f / static_cast<float>(n->B);
+    if (n->momentum) CK(sgd_momentum_update_launch(l.W, n->dtype == MBD_BF16, l.W32, l.V, l.dW, l.nW, n->mu, inv_B, eta, n->num_sms, n->stream));
+    else if (n->master) CK(sgd_master_update_launch(l.W32, l.W, l.dW, l.nW, scale, n->num_sms, n->stream));
     else CK(sgd_update_launch(l.W, n->dtype == MBD_BF16, l.dW, l.nW, scale, n->num_sms, n->stream));
     n->prof.end();
     if (l.bias) {
       n->prof.begin(MBD_K_SGD, static_cast<double>(l.d_out) * 12.0);
-      CK(sgd_update_launch(l.bias, 0, l.db, l.d_out, scale, n->num_sms, n->stream));
+      if (n->momentum) CK(sgd_momentum_update_launch(l.bias, 0, nullptr, l.Vb, l.db, l.d_out, n->mu, inv_B, eta, n->num_sms, n->stream));
+      else CK(sgd_update_launch(l.bias, 0, l.db, l.d_out, scale, n->num_sms, n->stream));
       n->prof.end();
     }
   }
@@ -825,6 +862,8 @@ extern "C" mbd_status mbd_get_tensor(mbd_net* n, int which, int layer, void* dst
       case MBD_T_DY: src = l.dY; size = static_cast<size_t>(n->B) * l.d_out * n->elt(); break;
       case MBD_T_DW: src = l.dW; size = l.nW * sizeof(float); break;
       case MBD_T_MASTER: src = l.W32; size = l.nW * sizeof(float); break;
+      case MBD_T_VELOCITY: src = l.V; size = l.nW * sizeof(float); break;
+      case MBD_T_VELOCITY_BIAS: src = l.Vb; size = l.d_out * sizeof(float); break;
       case MBD_T_DB: src = l.db; size = l.d_out * sizeof(float); break;
       default: return MBD_E_INVALID;
     }

@@ -18,7 +18,7 @@ FC, CONV3X3 = 0, 1
 SPLIT_MODEL, SPLIT_DOMAIN, SPLIT_BATCH = 0, 1, 2
 F32, BF16 = 0, 1
 LOSS_SOFTMAX_CE, LOSS_HALF_SSQ, LOSS_NONE = 0, 1, 2
-T_ACT, T_DY, T_DW, T_DB, T_LOSS, T_PARTIALS, T_MASTER = range(7)
+T_ACT, T_DY, T_DW, T_DB, T_LOSS, T_PARTIALS, T_MASTER, T_VELOCITY, T_VELOCITY_BIAS = range(9)
 ROWS_ALL, ROWS_INTERIOR, ROWS_BOUNDARY = range(3)
 
 KERNEL_CLASSES = ["gemm_fwd", "gemm_bwd_data", "gemm_bwd_weight", "reduce_partials", "softmax_xent", "colsum",
@@ -29,7 +29,7 @@ EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weig
            "mbd_set_tensor", "mbd_poll_status", "mbd_profile_enable", "mbd_profile_read", "mbd_launch_count", "mbd_gemm_bf16", "mbd_gemm_bf16_noalloc", "mbd_selftest_timeout", "mbd_strerror",
            "mbd_train_step_host_begin", "mbd_train_step_host_end",
            "mbd_comm_time", "mbd_redistribute_time", "mbd_total_time", "mbd_grid_table", "mbd_choose_grid",
-           "mbd_enable_master_weights", "mbd_block_gemm_bf16", "mbd_block_reduce", "mbd_softmax_xent",
+           "mbd_enable_master_weights", "mbd_enable_momentum", "mbd_block_gemm_bf16", "mbd_block_reduce", "mbd_softmax_xent",
            "mbd_conv_stage_input", "mbd_conv_forward_layer", "mbd_conv_backward_layer", "mbd_conv_outer_rows",
            "mbd_get_plan", "mbd_conv_forward_layer_rows", "mbd_conv_backward_layer_rows"]
 
@@ -126,6 +126,7 @@ def lib():
         L.mbd_set_tensor.argtypes = [vp, i32, i32, vp, C.c_size_t]
         L.mbd_poll_status.argtypes = [vp]
         L.mbd_enable_master_weights.argtypes = [vp]
+        L.mbd_enable_momentum.argtypes = [vp, C.c_float]
         L.mbd_block_gemm_bf16.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, C.POINTER(Tail), vp, vp]
         L.mbd_block_reduce.argtypes = [vp, i32, i64, i64, C.POINTER(Tail), i32, vp]
         L.mbd_softmax_xent.argtypes = [vp, i64, i64, vp, vp, i32, vp, i32, vp]
@@ -331,6 +332,10 @@ class Net:
         """fp32 master copies of all weights from now on (see include/mbd.h)."""
         _check(lib().mbd_enable_master_weights(self._h), "mbd_enable_master_weights")
 
+    def enable_momentum(self, mu: float):
+        """Heavy-ball momentum from now on, velocities zero (see include/mbd.h)."""
+        _check(lib().mbd_enable_momentum(self._h, float(mu)), "mbd_enable_momentum")
+
     def backward(self, fused_eta: float = 0.0):
         _check(lib().mbd_backward(self._h, float(fused_eta)), "mbd_backward")
 
@@ -373,9 +378,9 @@ class Net:
                 (t.float32 if (last and not conv) else self.act_dtype)
         elif which == T_DY:
             shape, dt = ((self.B, l.C_out, l.H, l.W) if conv else (self.B, l.d_out)), self.act_dtype
-        elif which in (T_DW, T_MASTER):
+        elif which in (T_DW, T_MASTER, T_VELOCITY):
             shape, dt = self._wshape(layer), t.float32
-        elif which == T_DB:
+        elif which in (T_DB, T_VELOCITY_BIAS):
             shape, dt = (l.d_out,), t.float32
         elif which == T_LOSS:
             shape, dt = (self.B,), t.float32

@@ -226,6 +226,45 @@ def test_sgd_descends():
     assert O.total_loss(new_layers, X, labels, "softmax_ce") < J0
 
 
+# ---------------------------------------------------------------- momentum (the first-order method beside Eq. 1)
+def test_momentum_with_mu_zero_is_eq1_and_constant_gradient_sums_a_geometric_series():
+    r = rng(33)
+    w, g = r.standard_normal((4, 3)), r.standard_normal((4, 3))
+    w1, v1 = O.sgd_momentum(w, np.zeros_like(w), g, 0.1, 8, 0.0)
+    assert np.array_equal(w1, O.sgd(w, g, 0.1, 8)) and np.array_equal(v1, g / 8)
+    # the same gradient k times: v_k = (1 + mu + ... + mu^(k-1)) g / B = (1 - mu^k) / (1 - mu) g / B
+    mu, eta, B = 0.9, 0.05, 8
+    wk, vk = w, np.zeros_like(w)
+    total = np.zeros_like(w)
+    for k in range(1, 7):
+        wk, vk = O.sgd_momentum(wk, vk, g, eta, B, mu)
+        assert np.allclose(vk, (1 - mu ** k) / (1 - mu) * g / B, atol=1e-15)
+        total += vk
+        assert np.allclose(wk, w - eta * total, atol=1e-15)
+
+
+def test_momentum_on_a_quadratic_follows_the_two_term_recurrence():
+    # J(w) = a w^2 / 2 with "batch" 1: w_{k+1} = (1 + mu - eta a) w_k - mu w_{k-1}, whose solution is a combination
+    # of the powers of the roots of z^2 - (1 + mu - eta a) z + mu = 0 (complex here: a damped oscillation of
+    # modulus sqrt(mu) per step)
+    a, eta, mu = 2.0, 0.3, 0.64
+    w, v = np.array([1.0]), np.array([0.0])
+    traj = [w.copy()]
+    for _ in range(12):
+        w, v = O.sgd_momentum(w, v, a * w, eta, 1, mu)
+        traj.append(w.copy())
+    t = np.array(traj)[:, 0]
+    c = 1 + mu - eta * a
+    for k in range(1, 12):
+        assert abs(t[k + 1] - (c * t[k] - mu * t[k - 1])) < 1e-14
+    z = np.roots([1.0, -c, mu])
+    assert np.iscomplex(z[0]) and abs(abs(z[0]) - np.sqrt(mu)) < 1e-12
+    # w_0 = 1, w_1 = 1 - eta a: fit the two coefficients, check the closed form at every later step
+    A = np.linalg.solve(np.array([[1, 1], [z[0], z[1]]]), np.array([t[0], t[1]], complex))
+    for k in range(13):
+        assert abs((A[0] * z[0] ** k + A[1] * z[1] ** k).real - t[k]) < 1e-12
+
+
 # ---------------------------------------------------------------- grid invariance
 @pytest.mark.parametrize("grid", [(1, 1), (2, 2), (4, 1), (1, 4), (3, 5), (8, 1), (1, 8), (2, 4)])
 def test_blocked_step_equals_unblocked(grid):
