@@ -36,7 +36,8 @@ def dW_outer_sum(dY, X):
 
 
 def conv3x3(K, X):
-    """Y[b][o][h][w] = sum_{c,u,v} K[o][c][u][v] X[b][c][h+u-1][w+v-1]."""
+    """Y[b][o][h][w] = sum_{c,u,v} K[o][c][u][v] X[b][c][h+u-p_h][w+v-p_w], p = floor(k/2) (k_h, k_w odd)."""
+    KH, KW = len(K[0][0]), len(K[0][0][0])
     B, C, H, W = len(X), len(X[0]), len(X[0][0]), len(X[0][0][0])
     O = len(K)
     Y = [[[[0.0] * W for _ in range(H)] for _ in range(O)] for _ in range(B)]
@@ -46,9 +47,9 @@ def conv3x3(K, X):
                 for w in range(W):
                     s = 0.0
                     for c in range(C):
-                        for u in range(3):
-                            for v in range(3):
-                                hh, ww = h + u - 1, w + v - 1
+                        for u in range(KH):
+                            for v in range(KW):
+                                hh, ww = h + u - KH // 2, w + v - KW // 2
                                 if 0 <= hh < H and 0 <= ww < W:
                                     s += K[o][c][u][v] * X[b][c][hh][ww]
                     Y[b][o][h][w] = s
@@ -60,6 +61,7 @@ def conv3x3_dX(K, dY):
     position it came from."""
     B, O, H, W = len(dY), len(dY[0]), len(dY[0][0]), len(dY[0][0][0])
     C = len(K[0])
+    KH, KW = len(K[0][0]), len(K[0][0][0])
     dX = [[[[0.0] * W for _ in range(H)] for _ in range(C)] for _ in range(B)]
     for b in range(B):
         for o in range(O):
@@ -67,27 +69,28 @@ def conv3x3_dX(K, dY):
                 for w in range(W):
                     g = dY[b][o][h][w]
                     for c in range(C):
-                        for u in range(3):
-                            for v in range(3):
-                                hh, ww = h + u - 1, w + v - 1
+                        for u in range(KH):
+                            for v in range(KW):
+                                hh, ww = h + u - KH // 2, w + v - KW // 2
                                 if 0 <= hh < H and 0 <= ww < W:
                                     dX[b][c][hh][ww] += K[o][c][u][v] * g
     return dX
 
 
-def conv3x3_dK(dY, X):
+def conv3x3_dK(dY, X, ksize=(3, 3)):
+    KH, KW = ksize
     B, C, H, W = len(X), len(X[0]), len(X[0][0]), len(X[0][0][0])
     O = len(dY[0])
-    dK = [[[[0.0] * 3 for _ in range(3)] for _ in range(C)] for _ in range(O)]
+    dK = [[[[0.0] * KW for _ in range(KH)] for _ in range(C)] for _ in range(O)]
     for b in range(B):
         for o in range(O):
             for h in range(H):
                 for w in range(W):
                     g = dY[b][o][h][w]
                     for c in range(C):
-                        for u in range(3):
-                            for v in range(3):
-                                hh, ww = h + u - 1, w + v - 1
+                        for u in range(KH):
+                            for v in range(KW):
+                                hh, ww = h + u - KH // 2, w + v - KW // 2
                                 if 0 <= hh < H and 0 <= ww < W:
                                     dK[o][c][u][v] += g * X[b][c][hh][ww]
     return dK

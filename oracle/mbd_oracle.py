@@ -49,7 +49,8 @@ class FC:
 
 @dataclass
 class Conv3x3:
-    """3x3, stride 1, zero-pad 1 convolution: K is [C_out, C_in, 3, 3].
+    """k_h x k_w (both odd; 3 x 3 in the listed workloads), stride 1, zero-pad floor(k/2) convolution:
+    K is [C_out, C_in, k_h, k_w].
     split (used by the blocked step only): "domain" = row strips over the P_r groups (Section 2.2 / 2.4);
     "batch" = the layer forced onto a 1 x P grid, P = P_r P_c (Section 3's improved case: pure batch
     parallelism in the convolutional layers, P_r x P_c grids in the fully connected ones)."""
@@ -115,46 +116,59 @@ def fc_dW(dY, X):
     return np.asarray(dY, F64) @ np.asarray(X, F64).T
 
 
+def _pads(K):
+    """Rows / columns of zero padding per side of a k_h x k_w kernel (odd sizes): floor(k/2), which is also the
+    number of halo rows a strip needs from each neighbour (Section 2.2)."""
+    kh, kw = K.shape[2], K.shape[3]
+    assert kh % 2 == 1 and kw % 2 == 1
+    return kh // 2, kw // 2
+
+
 def conv3x3(K, X):
-    """Y[b,o,h,w] = sum_{c,u,v} K[o,c,u,v] X[b,c,h+u-1,w+v-1], zero outside."""
+    """Y[b,o,h,w] = sum_{c,u,v} K[o,c,u,v] X[b,c,h+u-p_h,w+v-p_w], zero outside; p = floor(k/2)
+    (for the 3 x 3 kernels of the listed workloads: h+u-1, w+v-1)."""
     K = np.asarray(K, F64)
     X = np.asarray(X, F64)
+    ph, pw = _pads(K)
     B, C, H, W = X.shape
-    Xp = np.zeros((B, C, H + 2, W + 2), F64)
-    Xp[:, :, 1:H + 1, 1:W + 1] = X
+    Xp = np.zeros((B, C, H + 2 * ph, W + 2 * pw), F64)
+    Xp[:, :, ph:H + ph, pw:W + pw] = X
     Y = np.zeros((B, K.shape[0], H, W), F64)
-    for u in range(3):
-        for v in range(3):
+    for u in range(K.shape[2]):
+        for v in range(K.shape[3]):
             Y += np.einsum("oc,bchw->bohw", K[:, :, u, v], Xp[:, :, u:u + H, v:v + W], optimize=True)
     return Y
 
 
 def conv3x3_dX(K, dY):
-    """dX[b,c,h,w] = sum_{o,u,v} K[o,c,u,v] dY[b,o,h-u+1,w-v+1], zero outside."""
+    """dX[b,c,h,w] = sum_{o,u,v} K[o,c,u,v] dY[b,o,h-u+p_h,w-v+p_w], zero outside."""
     K = np.asarray(K, F64)
     dY = np.asarray(dY, F64)
+    ph, pw = _pads(K)
     B, O, H, W = dY.shape
-    dYp = np.zeros((B, O, H + 2, W + 2), F64)
-    dYp[:, :, 1:H + 1, 1:W + 1] = dY
+    dYp = np.zeros((B, O, H + 2 * ph, W + 2 * pw), F64)
+    dYp[:, :, ph:H + ph, pw:W + pw] = dY
     dX = np.zeros((B, K.shape[1], H, W), F64)
-    for u in range(3):
-        for v in range(3):
-            # index h-u+1 in dY  ==  (h-u+2) in the padded array
+    for u in range(K.shape[2]):
+        for v in range(K.shape[3]):
+            # index h-u+p_h in dY  ==  (h-u+2 p_h) in the padded array
             dX += np.einsum("oc,bohw->bchw", K[:, :, u, v],
-                            dYp[:, :, 2 - u:2 - u + H, 2 - v:2 - v + W], optimize=True)
+                            dYp[:, :, 2 * ph - u:2 * ph - u + H, 2 * pw - v:2 * pw - v + W], optimize=True)
     return dX
 
 
-def conv3x3_dK(dY, X):
-    """dK[o,c,u,v] = sum_{b,h,w} dY[b,o,h,w] X[b,c,h+u-1,w+v-1]."""
+def conv3x3_dK(dY, X, ksize=(3, 3)):
+    """dK[o,c,u,v] = sum_{b,h,w} dY[b,o,h,w] X[b,c,h+u-p_h,w+v-p_w]; ksize = (k_h, k_w), both odd."""
     dY = np.asarray(dY, F64)
     X = np.asarray(X, F64)
+    kh, kw = ksize
+    ph, pw = kh // 2, kw // 2
     B, C, H, W = X.shape
-    Xp = np.zeros((B, C, H + 2, W + 2), F64)
-    Xp[:, :, 1:H + 1, 1:W + 1] = X
-    dK = np.zeros((dY.shape[1], C, 3, 3), F64)
-    for u in range(3):
-        for v in range(3):
+    Xp = np.zeros((B, C, H + 2 * ph, W + 2 * pw), F64)
+    Xp[:, :, ph:H + ph, pw:W + pw] = X
+    dK = np.zeros((dY.shape[1], C, kh, kw), F64)
+    for u in range(kh):
+        for v in range(kw):
             dK[:, :, u, v] = np.einsum("bohw,bchw->oc", dY, Xp[:, :, u:u + H, v:v + W], optimize=True)
     return dK
 
@@ -258,7 +272,7 @@ def train_step(layers: Sequence, X1, labels, loss: str, eta: float, store=None):
             dWs[i] = fc_dW(dYs[i], Xs[i])
             dbs[i] = dYs[i].sum(axis=1) if lay.b is not None else None
         else:
-            dWs[i] = conv3x3_dK(dYs[i], Xs[i])
+            dWs[i] = conv3x3_dK(dYs[i], Xs[i], lay.K.shape[2:])
         if i > 0:
             dXs[i] = fc_dX(lay.W, dYs[i]) if isinstance(lay, FC) else conv3x3_dX(lay.K, dYs[i])
             dXs[i] = _below(dXs[i], Ys[i - 1])
@@ -335,43 +349,45 @@ def fc_dW_blocked(dY, X, P_r, P_c):
     return dW, parts
 
 
-def strip_with_halo(T, h0, h1):
-    """Rows [h0-1, h1+1) of an NCHW tensor as a strip owner sees them after
-    the halo exchange (Section 2.2): its own rows plus one boundary row copied
-    from each neighbour; zero rows where there is no neighbour."""
+def strip_with_halo(T, h0, h1, halo=1):
+    """Rows [h0-halo, h1+halo) of an NCHW tensor as a strip owner sees them after the halo exchange
+    (Section 2.2): its own rows plus `halo` = floor(k_h/2) boundary rows copied from the strips above and
+    below; zero rows where the image ends."""
     B, C, H, W = T.shape
-    S = np.zeros((B, C, h1 - h0 + 2, W), F64)
-    S[:, :, 1:1 + (h1 - h0), :] = T[:, :, h0:h1, :]
-    if h0 > 0:
-        S[:, :, 0, :] = T[:, :, h0 - 1, :]       # copy of the upper neighbour's last row
-    if h1 < H:
-        S[:, :, -1, :] = T[:, :, h1, :]          # copy of the lower neighbour's first row
+    S = np.zeros((B, C, h1 - h0 + 2 * halo, W), F64)
+    S[:, :, halo:halo + (h1 - h0), :] = T[:, :, h0:h1, :]
+    for j in range(1, halo + 1):
+        if h0 - j >= 0:
+            S[:, :, halo - j, :] = T[:, :, h0 - j, :]              # row j above the strip: a neighbour's
+        if h1 - 1 + j < H:
+            S[:, :, halo + (h1 - h0) - 1 + j, :] = T[:, :, h1 - 1 + j, :]      # row j below it
     return S
 
 
 def _conv_rows_valid(K, S):
-    """Correlate a haloed strip S [B,C,hs+2,W]: zero padding in W only, the
+    """Correlate a haloed strip S [B,C,hs+2 p_h,W]: zero padding in W only, the
     halo rows supply the H neighbours.  Output [B,O,hs,W]."""
+    ph, pw = _pads(K)
     B, C, Hh, W = S.shape
-    hs = Hh - 2
-    Sp = np.zeros((B, C, Hh, W + 2), F64)
-    Sp[:, :, :, 1:W + 1] = S
+    hs = Hh - 2 * ph
+    Sp = np.zeros((B, C, Hh, W + 2 * pw), F64)
+    Sp[:, :, :, pw:W + pw] = S
     Y = np.zeros((B, K.shape[0], hs, W), F64)
-    for u in range(3):
-        for v in range(3):
+    for u in range(K.shape[2]):
+        for v in range(K.shape[3]):
             Y += np.einsum("oc,bchw->bohw", K[:, :, u, v], Sp[:, :, u:u + hs, v:v + W], optimize=True)
     return Y
 
 
 def conv3x3_strips(K, X, P_r):
     """Domain-parallel forward: each of P_r strips correlates its own rows
-    after receiving one halo row per neighbour (Section 2.2, Eq. 7)."""
+    after receiving floor(k_h/2) halo rows per neighbour (Section 2.2, Eq. 7)."""
     K = np.asarray(K, F64)
     X = np.asarray(X, F64)
     B, C, H, W = X.shape
     Y = np.empty((B, K.shape[0], H, W), F64)
     for (h0, h1) in balanced_ranges(H, P_r):
-        Y[:, :, h0:h1, :] = _conv_rows_valid(K, strip_with_halo(X, h0, h1))
+        Y[:, :, h0:h1, :] = _conv_rows_valid(K, strip_with_halo(X, h0, h1, _pads(K)[0]))
     return Y
 
 
@@ -384,26 +400,28 @@ def conv3x3_dX_strips(K, dY, P_r):
     B, O, H, W = dY.shape
     dX = np.empty((B, K.shape[1], H, W), F64)
     for (h0, h1) in balanced_ranges(H, P_r):
-        dX[:, :, h0:h1, :] = _conv_rows_valid(Kt, strip_with_halo(dY, h0, h1))
+        dX[:, :, h0:h1, :] = _conv_rows_valid(Kt, strip_with_halo(dY, h0, h1, _pads(K)[0]))
     return dX
 
 
-def conv3x3_dK_strips(dY, X, P_r):
+def conv3x3_dK_strips(dY, X, P_r, ksize=(3, 3)):
     """Each strip forms a partial dK from its own output rows and its haloed
     input; the all-reduce over the strips adds them in ascending order
     (third term of Eq. 7).  Returns (dK, partials)."""
     dY = np.asarray(dY, F64)
     X = np.asarray(X, F64)
+    kh, kw = ksize
+    ph, pw = kh // 2, kw // 2
     B, C, H, W = X.shape
     parts = []
     for (h0, h1) in balanced_ranges(H, P_r):
-        S = strip_with_halo(X, h0, h1)
+        S = strip_with_halo(X, h0, h1, ph)
         hs = h1 - h0
-        Sp = np.zeros((B, C, hs + 2, W + 2), F64)
-        Sp[:, :, :, 1:W + 1] = S
-        part = np.zeros((dY.shape[1], C, 3, 3), F64)
-        for u in range(3):
-            for v in range(3):
+        Sp = np.zeros((B, C, hs + 2 * ph, W + 2 * pw), F64)
+        Sp[:, :, :, pw:W + pw] = S
+        part = np.zeros((dY.shape[1], C, kh, kw), F64)
+        for u in range(kh):
+            for v in range(kw):
                 part[:, :, u, v] = np.einsum("bohw,bchw->oc", dY[:, :, h0:h1, :],
                                              Sp[:, :, u:u + hs, v:v + W], optimize=True)
         parts.append(part)
@@ -413,7 +431,7 @@ def conv3x3_dK_strips(dY, X, P_r):
     return dK, parts
 
 
-def conv3x3_dK_grid(dY, X, P_r, P_c):
+def conv3x3_dK_grid(dY, X, P_r, P_c, ksize=(3, 3)):
     """Weight gradient of a domain-parallel layer on a P_r x P_c grid: process
     (r, c) owns strip r of the samples of batch block c and forms one partial;
     the all-reduce over all P = P_r P_c processes (last term of Eq. 9) adds them,
@@ -422,7 +440,7 @@ def conv3x3_dK_grid(dY, X, P_r, P_c):
     X = np.asarray(X, F64)
     parts = []
     for (c0, c1) in balanced_ranges(X.shape[0], P_c):
-        _, strip_parts = conv3x3_dK_strips(dY[c0:c1], X[c0:c1], P_r)
+        _, strip_parts = conv3x3_dK_strips(dY[c0:c1], X[c0:c1], P_r, ksize)
         parts.extend(strip_parts)
     dK = np.zeros_like(parts[0])
     for part in parts:
@@ -467,9 +485,9 @@ def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
                     db = db + dYs[i][:, c0:c1].sum(axis=1)
                 dbs[i] = db
         elif lay.split == "batch":
-            dWs[i], _ = conv3x3_dK_grid(dYs[i], Xs[i], 1, P_r * P_c)      # one partial per process of the 1 x P grid
+            dWs[i], _ = conv3x3_dK_grid(dYs[i], Xs[i], 1, P_r * P_c, lay.K.shape[2:])      # one partial per process of the 1 x P grid
         else:
-            dWs[i], _ = conv3x3_dK_grid(dYs[i], Xs[i], P_r, P_c)
+            dWs[i], _ = conv3x3_dK_grid(dYs[i], Xs[i], P_r, P_c, lay.K.shape[2:])
         if i > 0:
             if isinstance(lay, FC):
                 dXs[i], _ = fc_dX_blocked(lay.W, dYs[i], P_r, P_c)

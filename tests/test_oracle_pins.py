@@ -312,6 +312,57 @@ def test_conv_matches_scalar_loops():
     assert relerr(O.conv3x3_dK(dY, X), np.array(brute.conv3x3_dK(dY.tolist(), X.tolist()))) < 1e-14
 
 
+@pytest.mark.parametrize("ksize", [(5, 5), (1, 7), (7, 3), (1, 1)])
+def test_conv_of_other_odd_kernel_sizes(ksize):
+    # k_h x k_w kernels with floor(k/2) rows / columns of zero padding: scalar loops, the adjoint identities
+    # <Y, conv(K, X)> = <conv_dX(K, Y), X> = <conv_dK(Y, X), K>, a 3 x 3 kernel embedded in the centre of the larger
+    # one gives the 3 x 3 result, and strips with floor(k_h/2) halo rows (Section 2.2) reproduce the whole image
+    kh, kw = ksize
+    r = rng(58)
+    K, X, dY = r.standard_normal((4, 3, kh, kw)), r.standard_normal((2, 3, 9, 8)), r.standard_normal((2, 4, 9, 8))
+    Y = O.conv3x3(K, X)
+    assert relerr(Y, np.array(brute.conv3x3(K.tolist(), X.tolist()))) < 1e-14
+    assert relerr(O.conv3x3_dX(K, dY), np.array(brute.conv3x3_dX(K.tolist(), dY.tolist()))) < 1e-14
+    assert relerr(O.conv3x3_dK(dY, X, ksize), np.array(brute.conv3x3_dK(dY.tolist(), X.tolist(), ksize))) < 1e-14
+    lhs = float(np.sum(dY * Y))
+    assert abs(lhs - float(np.sum(O.conv3x3_dX(K, dY) * X))) < 1e-11 * abs(lhs)
+    assert abs(lhs - float(np.sum(O.conv3x3_dK(dY, X, ksize) * K))) < 1e-11 * abs(lhs)
+    if kh >= 3 and kw >= 3:
+        K3 = r.standard_normal((4, 3, 3, 3))
+        Kbig = np.zeros((4, 3, kh, kw)); Kbig[:, :, kh // 2 - 1:kh // 2 + 2, kw // 2 - 1:kw // 2 + 2] = K3
+        assert relerr(O.conv3x3(Kbig, X), O.conv3x3(K3, X)) < 1e-14
+    for P_r in (1, 2, 3, 4):
+        assert relerr(O.conv3x3_strips(K, X, P_r), Y) < 1e-14
+        assert relerr(O.conv3x3_dX_strips(K, dY, P_r), O.conv3x3_dX(K, dY)) < 1e-14
+        dK, parts = O.conv3x3_dK_grid(dY, X, P_r, 2, ksize)
+        assert len(parts) == 2 * P_r and relerr(dK, O.conv3x3_dK(dY, X, ksize)) < 1e-13
+    # a strip's halo holds exactly floor(k_h/2) rows of each neighbour
+    S = O.strip_with_halo(X, 3, 6, kh // 2)
+    assert S.shape[2] == 3 + 2 * (kh // 2)
+    assert np.array_equal(S[:, :, 0], X[:, :, 3 - kh // 2]) and np.array_equal(S[:, :, -1], X[:, :, 5 + kh // 2])
+
+
+def test_wide_kernel_tap_direction_and_finite_differences():
+    # tap (u, v) = (0, 0) of a 5 x 5 kernel reads the input two rows up and two columns left of the output position
+    X = np.zeros((1, 1, 5, 5)); X[0, 0, 2, 2] = 1.0
+    K = np.zeros((1, 1, 5, 5)); K[0, 0, 0, 0] = 3.0
+    Y = O.conv3x3(K, X)
+    assert Y[0, 0, 4, 4] == 3.0 and np.count_nonzero(Y) == 1
+    # the gradients of J = sum(Y^2)/2 through a 5 x 3 layer by central differences
+    r = rng(59)
+    K, X = r.standard_normal((2, 2, 5, 3)) / 3, r.standard_normal((1, 2, 6, 5))
+    J = lambda K_, X_: 0.5 * float(np.sum(O.conv3x3(K_, X_) ** 2))
+    Y = O.conv3x3(K, X)
+    dK, dX = O.conv3x3_dK(Y, X, (5, 3)), O.conv3x3_dX(K, Y)
+    eps = 1e-6
+    for idx in [(0, 1, 0, 0), (1, 0, 4, 2), (1, 1, 2, 1)]:
+        Kp, Km = K.copy(), K.copy(); Kp[idx] += eps; Km[idx] -= eps
+        assert abs((J(Kp, X) - J(Km, X)) / (2 * eps) - dK[idx]) < 1e-6 * max(1.0, abs(dK[idx]))
+    for idx in [(0, 0, 0, 0), (0, 1, 5, 4), (0, 1, 3, 2)]:
+        Xp, Xm = X.copy(), X.copy(); Xp[idx] += eps; Xm[idx] -= eps
+        assert abs((J(K, Xp) - J(K, Xm)) / (2 * eps) - dX[idx]) < 1e-6 * max(1.0, abs(dX[idx]))
+
+
 def test_conv_centre_tap_is_per_pixel_fc():
     # a kernel with only its centre tap is the 1x1 convolution: Y[:, :, h, w] = M X[:, :, h, w]
     K, X, _ = conv_case(seed=51)
