@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmbd.so")
-SOURCES = ["net.cu", "gemm_tc.cu", "gemm_simt.cu", "elementwise.cu", "conv.cu", "comm_words.cpp", "time_model.cpp", "profiler.cpp", "noalloc.cu", "block_ops.cu"]
+SOURCES = ["net.cu", "gemm_tc.cu", "gemm_simt.cu", "elementwise.cu", "conv.cu", "conv_general.cu", "comm_words.cpp", "time_model.cpp", "profiler.cpp", "noalloc.cu", "block_ops.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--use_fast_math=false"]
 

@@ -34,6 +34,7 @@
 #include <vector>
 
 #include "conv.h"
+#include "conv_general.h"
 #include "epi.cuh"
 #include "tc_common.cuh"
 
@@ -967,6 +968,7 @@ struct ConvNet {
   std::vector<bf16*> dY;             // dY[i]: gradient w.r.t. the output of layer i; dY[L-1] == act[L]
   std::vector<bf16*> K, Wf, Wb;
   std::vector<float*> dK;
+  GenConv* gen = nullptr;            // layers these kernels do not cover: every call is forwarded (conv_general.cu)
   std::vector<float*> K32;           // fp32 master weights (empty unless enabled)
   std::vector<float*> Vk;            // momentum: velocities of the kernels (empty unless enabled), canonical [o][c][3][3]
   float mu = 0.f;
@@ -1016,9 +1018,17 @@ void launch_stage_in(ConvNet* c, const bf16* nchw, bf16* strips) {
 
 }  // namespace
 
-mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int max_partials, int num_sms, int* status,
+mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, int max_partials, int num_sms, int* status,
                        cudaStream_t stream, Profiler* prof, bool fc_above, ConvNet** out) {
-  (void)max_partials;
+  if (gconv_needed(layers, L)) {
+    ConvNet* c = new (std::nothrow) ConvNet();
+    if (!c) return MBD_E_ALLOC;
+    const mbd_status s = gconv_create(layers, L, B, P_r, P_c, max_partials, num_sms, status, stream, prof, fc_above, &c->gen);
+    if (s != MBD_OK) { delete c; return s; }
+    c->L = L; c->B = B;
+    *out = c;
+    return MBD_OK;
+  }
   if (conv_init() != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
   const int H = layers[0].H, W = layers[0].W;
   if (B > 65535 || static_cast<int64_t>(H) * W > INT32_MAX) return MBD_E_UNSUPPORTED;   // grid.y of the staging kernels
@@ -1074,6 +1084,7 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int m
 }
 
 void conv_destroy(ConvNet* c) {
+  if (c && c->gen) { gconv_destroy(c->gen); delete c; return; }
   if (!c) return;
   for (size_t i = 0; i < c->act.size(); ++i) cudaFree(c->act[i]);
   for (int i = 0; i < c->L; ++i)
@@ -1096,6 +1107,7 @@ mbd_status launch_pack(ConvNet* c, int layer) {
 }  // namespace
 
 mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev) {
+  if (c->gen) return gconv_set_weights(c->gen, layer, K_dev);
   if (c->k1[layer]) {
     embed_1x1_kernel<<<(9 * C * C + 255) / 256, 256, 0, c->stream>>>(static_cast<const bf16*>(K_dev), c->K[layer]);
     if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
@@ -1107,6 +1119,7 @@ mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev) {
 }
 
 mbd_status conv_enable_master(ConvNet* c) {
+  if (c->gen) return MBD_E_UNSUPPORTED;
   if (!c->K32.empty()) return MBD_OK;
   std::vector<float*> m(c->L, nullptr);
   for (int i = 0; i < c->L; ++i) {
@@ -1122,6 +1135,7 @@ mbd_status conv_enable_master(ConvNet* c) {
 }
 
 mbd_status conv_enable_momentum(ConvNet* c, float mu) {
+  if (c->gen) return MBD_E_UNSUPPORTED;
   if (c->Vk.empty()) {
     std::vector<float*> v(c->L, nullptr);
     for (int i = 0; i < c->L; ++i) {
@@ -1152,6 +1166,7 @@ mbd_status momentum_update(ConvNet* c, int i, float eta) {
 }  // namespace
 
 mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev) {
+  if (c->gen) return gconv_get_weights(c->gen, layer, K_dev);
   if (c->k1[layer]) {
     extract_1x1_kernel<bf16><<<(C * C + 255) / 256, 256, 0, c->stream>>>(c->K[layer], static_cast<bf16*>(K_dev));
     return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
@@ -1160,11 +1175,12 @@ mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev) {
   return MBD_OK;
 }
 
-size_t conv_input_bytes(const ConvNet* c) { return static_cast<size_t>(c->B) * C * c->H * c->W * 2; }
+size_t conv_input_bytes(const ConvNet* c) { return c->gen ? gconv_input_bytes(c->gen) : static_cast<size_t>(c->B) * C * c->H * c->W * 2; }
 
 // The step, piece by piece (a multi-process driver exchanges the image's outer halo rows between the pieces;
 // conv_forward / conv_backward below are these pieces in a row).
 mbd_status conv_stage_input(ConvNet* c, const void* X_nchw) {
+  if (c->gen) return gconv_stage_input(c->gen, X_nchw);
   // the input goes into strips (with the halo rows between its own strips); the operand layouts of the weights
   // are kept current by whatever changes the weights (conv_set_weights, the fused update, conv_sgd_step)
   launch_stage_in(c, static_cast<const bf16*>(X_nchw), c->act[0]);
@@ -1194,6 +1210,7 @@ void for_rows(const ConvNet* c, int layer, int rows, F launch) {
 }  // namespace
 
 mbd_status conv_forward_layer(ConvNet* c, int i, float* loss_sum_dev, int rows) {
+  if (c->gen) return rows == MBD_ROWS_ALL ? gconv_forward_layer(c->gen, i, loss_sum_dev) : MBD_E_UNSUPPORTED;
   if (i < 0 || i >= c->L) return MBD_E_INVALID;
   if (rows != MBD_ROWS_ALL && (c->P_r != 1 || (rows != MBD_ROWS_INTERIOR && rows != MBD_ROWS_BOUNDARY))) return MBD_E_UNSUPPORTED;
   const bool last = i == c->L - 1;
@@ -1216,12 +1233,14 @@ mbd_status conv_forward_layer(ConvNet* c, int i, float* loss_sum_dev, int rows) 
 }
 
 mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
+  if (c->gen) return gconv_forward(c->gen, X_nchw, loss_sum_dev);
   mbd_status s = conv_stage_input(c, X_nchw);
   for (int i = 0; i < c->L && s == MBD_OK; ++i) s = conv_forward_layer(c, i, loss_sum_dev, MBD_ROWS_ALL);
   return s;
 }
 
 mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta, int rows) {
+  if (c->gen) return rows == MBD_ROWS_ALL ? gconv_backward_layer(c->gen, i, fused_eta) : MBD_E_UNSUPPORTED;
   if (i < 0 || i >= c->L) return MBD_E_INVALID;
   if (rows != MBD_ROWS_ALL && (c->P_r != 1 || (rows != MBD_ROWS_INTERIOR && rows != MBD_ROWS_BOUNDARY))) return MBD_E_UNSUPPORTED;
   const bool momentum = !c->Vk.empty();
@@ -1259,6 +1278,7 @@ mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta, int rows) {
 }
 
 mbd_status conv_backward(ConvNet* c, float fused_eta) {
+  if (c->gen) return gconv_backward(c->gen, fused_eta);
   mbd_status s = MBD_OK;
   for (int i = c->L - 1; i >= 0 && s == MBD_OK; --i) s = conv_backward_layer(c, i, fused_eta, MBD_ROWS_ALL);
   return s;
@@ -1268,6 +1288,7 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
 // read out, or its upper / lower halo row (zero unless a neighbour supplies it) is written.  `side` 0 = top,
 // 1 = bottom; the row buffer is [B][W][C] bf16.  which / layer as in conv_get_tensor; layer -1 = the staged input.
 mbd_status conv_outer_rows(ConvNet* c, int which, int layer, int side, void* rows, size_t bytes, int set) {
+  if (c->gen) return MBD_E_UNSUPPORTED;
   if (layer < -1 || layer >= c->L || (side != 0 && side != 1)) return MBD_E_INVALID;
   if (bytes != static_cast<size_t>(c->B) * c->W * C * 2) return MBD_E_INVALID;
   bf16* buf = which == MBD_T_ACT ? c->act[layer + 1] : (which == MBD_T_DY && layer >= 0) ? c->dY[layer] : nullptr;
@@ -1282,6 +1303,7 @@ mbd_status conv_outer_rows(ConvNet* c, int which, int layer, int side, void* row
 }
 
 mbd_status conv_set_dw(ConvNet* c, int layer, const void* src, size_t bytes) {
+  if (c->gen) return gconv_set_dw(c->gen, layer, src, bytes);
   if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
   if (c->k1[layer]) {
     if (bytes != C * C * 4) return MBD_E_INVALID;
@@ -1293,6 +1315,7 @@ mbd_status conv_set_dw(ConvNet* c, int layer, const void* src, size_t bytes) {
 }
 
 mbd_status conv_sgd_step(ConvNet* c, float eta) {
+  if (c->gen) return gconv_sgd_step(c->gen, eta);
   const float scale = -eta / static_cast<float>(c->B);
   for (int i = 0; i < c->L; ++i) {
     if (!c->Vk.empty()) {
@@ -1313,6 +1336,7 @@ mbd_status conv_sgd_step(ConvNet* c, float eta) {
 // convolution's output become the [B, C*H*W] matrix (NCHW order) the first fully connected layer reads,
 // and that layer's input gradient goes back into strips, its boundary rows also into the neighbours' halos.
 mbd_status conv_output_to_nchw(ConvNet* c, void* dst) {
+  if (c->gen) return gconv_output_to_nchw(c->gen, dst);
   dim3 g((c->H * c->W + 31) / 32, static_cast<unsigned>(c->B));
   c->prof->begin(MBD_K_HALO, 2.0 * c->B * C * c->H * c->W * 2.0);
   strips_to_nchw_kernel<<<g, 128, 0, c->stream>>>(c->act[c->L], static_cast<bf16*>(dst), c->H, c->W, c->P_r, c->Hs);
@@ -1321,14 +1345,16 @@ mbd_status conv_output_to_nchw(ConvNet* c, void* dst) {
 }
 
 mbd_status conv_top_grad_from_nchw(ConvNet* c, const void* src) {
+  if (c->gen) return gconv_top_grad_from_nchw(c->gen, src);
   if (!c->fc_above) return MBD_E_STATE;
   launch_stage_in(c, static_cast<const bf16*>(src), c->dY[c->L - 1]);
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
-int conv_last_relu(const ConvNet* c) { return c->relu[c->L - 1]; }
+int conv_last_relu(const ConvNet* c) { return c->gen ? gconv_last_relu(c->gen) : c->relu[c->L - 1]; }
 
 mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t bytes) {
+  if (c->gen) return gconv_get_tensor(c->gen, which, layer, dst, bytes);
   const size_t nchw_bytes = conv_input_bytes(c);
   if (which == MBD_T_DW || which == MBD_T_MASTER || which == MBD_T_VELOCITY) {
     if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
@@ -1358,6 +1384,7 @@ mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t b
 }
 
 mbd_status conv_set_tensor(ConvNet* c, int which, int layer, const void* src, size_t bytes) {
+  if (c->gen) return gconv_set_tensor(c->gen, which, layer, src, bytes);
   if (layer < 0 || layer >= c->L || bytes != conv_input_bytes(c)) return MBD_E_INVALID;
   bf16* dst = which == MBD_T_ACT ? c->act[layer + 1] : which == MBD_T_DY ? c->dY[layer] : nullptr;
   if (!dst) return MBD_E_INVALID;

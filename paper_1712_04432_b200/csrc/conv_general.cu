@@ -1,0 +1,500 @@
+// General domain-parallel convolution layers (Section 2.2 / 2.4): any odd k_h x k_w up to 7 x 7, stride 1, zero
+// padding floor(k/2), C_in and C_out multiples of 8, row strips with floor(k_h/2) halo rows.  The layers with 64
+// channels and 3 x 3 / 1 x 1 kernels have kernels of their own (conv.cu); everything else runs here, on the
+// tensor-core contraction kernel of the fully connected layers (gemm_tc.cu) fed with shifted views.
+//
+// Layout.  Every activation / gradient tensor is pixel-major with its zero padding stored:
+//     T[z][r][x][c],  z = b P_r + s (image b, strip s),  r in [0, Hs + 2 ph),  x in [0, W + 2 pw),  c in [0, C)
+// ph, pw = the largest floor(k_h/2), floor(k_w/2) of the network.  Rows ph .. ph+Hs-1 and columns pw .. pw+W-1 are
+// the strip's own pixels; the other columns are zero; the other rows are the halo rows -- copies of the
+// neighbouring strips' boundary rows (the halo exchange of Section 2.2, here a copy kernel), zero where the image
+// ends.  With p the flattened pixel index (z, r, x), tap (u, v) of a layer reads pixel p + (u - kh/2) Wp + (v - kw/2):
+// a convolution is a contraction over (tap, channel) whose operand tiles are row-shifted views of ONE 2-D tensor
+// [pixels][channels] -- no patch matrix is ever formed.  The products compute every pixel position, padding
+// included (a few per cent of extra rows); a small kernel then restores the zeros and the halo rows.
+//     forward         Y[p][o]      = sum_{t,c} X[p + off_t][c] Wm[o][t][c]
+//     backward-data   dX[p][c]     = sum_{t,o} dY[p - off_t][o] Wm[o][t][c]        (then the ReLU mask)
+//     backward-weight dWm[o][t][c] = sum_p dY[p][o] X[p + off_t][c]   (dY zero outside the strips' own pixels)
+// Wm[o][t][c] is the kernel K[o][c][u][v] with t = u k_w + v and the channel index padded to a multiple of 64 (zero
+// weights, which stay zero: their gradient is a sum of zero-filled operand columns).  The weight gradient is a
+// contraction over ALL pixels: its K range is cut by the planner into enough pieces to fill the SMs, the grid's
+// S = min(P, max_partials) partial sums being the first cut.
+#include "conv_general.h"
+
+#include <algorithm>
+#include <cstdlib>
+#include <new>
+#include <vector>
+
+namespace mbd {
+
+typedef __nv_bfloat16 bf16;
+
+namespace {
+
+struct Geo {
+  int B, H, W, P_r, Hs, R, Wp, ph, pw;
+  long long Z, Ptot;
+};
+
+// ------------------------------------------------------------------------------ layout kernels
+// NCHW -> pixel-major (own pixels only; padding and halos are the business of pad_fix_kernel).
+// One thread per (pixel, 8 channels): eight reads that are coalesced across the warp (consecutive w), one 16-byte store.
+__global__ void __launch_bounds__(256)
+nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C) {
+  const int c8 = C / 8;
+  const long long total = static_cast<long long>(g.B) * g.H * g.W * c8;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
+    const int w = static_cast<int>(i % g.W);
+    long long q = i / g.W;
+    const int h = static_cast<int>(q % g.H); q /= g.H;
+    const int cg = static_cast<int>(q % c8);
+    const int b = static_cast<int>(q / c8);
+    const int s = h / g.Hs, r = h - s * g.Hs + g.ph;
+    uint16_t v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      v[j] = __bfloat16_as_ushort(src[((static_cast<long long>(b) * C + cg * 8 + j) * g.H + h) * g.W + w]);
+    uint4 o;
+    o.x = v[0] | (static_cast<uint32_t>(v[1]) << 16); o.y = v[2] | (static_cast<uint32_t>(v[3]) << 16);
+    o.z = v[4] | (static_cast<uint32_t>(v[5]) << 16); o.w = v[6] | (static_cast<uint32_t>(v[7]) << 16);
+    const long long p = ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w + g.pw;
+    *reinterpret_cast<uint4*>(dst + p * C + cg * 8) = o;
+  }
+}
+
+template <typename T>   // T = bf16 (activations, gradients)
+__global__ void __launch_bounds__(256)
+pix_to_nchw_kernel(const T* __restrict__ src, T* __restrict__ dst, Geo g, int C) {
+  const long long total = static_cast<long long>(g.B) * C * g.H * g.W;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
+    const int w = static_cast<int>(i % g.W);
+    long long q = i / g.W;
+    const int h = static_cast<int>(q % g.H); q /= g.H;
+    const int c = static_cast<int>(q % C);
+    const int b = static_cast<int>(q / C);
+    const int s = h / g.Hs, r = h - s * g.Hs + g.ph;
+    const long long p = ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w + g.pw;
+    dst[i] = src[p * C + c];
+  }
+}
+
+// Everything that is not a strip's own pixel: the padding columns and the image's outer rows become zero; a halo
+// row becomes the copy of the neighbouring strip's boundary row (fill_halos) -- the halo exchange of Section 2.2:
+// floor(k_h/2) rows per neighbour and direction -- or zero (a gradient about to enter the weight-gradient sum, whose
+// pixels must each be counted once).  One thread per 16 bytes of the tensor; own pixels are left alone.
+__global__ void __launch_bounds__(256)
+pad_fix_kernel(bf16* __restrict__ T, Geo g, int C, int fill_halos) {
+  const int c8 = C / 8;
+  const long long total = g.Ptot * c8;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
+    const int cg = static_cast<int>(i % c8);
+    const long long p = i / c8;
+    const int x = static_cast<int>(p % g.Wp);
+    const long long zr = p / g.Wp;
+    const int r = static_cast<int>(zr % g.R);
+    const long long z = zr / g.R;
+    const bool own_col = x >= g.pw && x < g.pw + g.W;
+    const bool own_row = r >= g.ph && r < g.ph + g.Hs;
+    if (own_col && own_row) continue;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (fill_halos && own_col && !own_row) {
+      const int s = static_cast<int>(z % g.P_r);
+      if (r < g.ph && s > 0)                        // rows above the strip: the last rows of the strip above
+        v = *reinterpret_cast<const uint4*>(T + ((((z - 1) * g.R) + r + g.Hs) * g.Wp + x) * C + cg * 8);
+      else if (r >= g.ph + g.Hs && s < g.P_r - 1)   // rows below it: the first rows of the strip below
+        v = *reinterpret_cast<const uint4*>(T + ((((z + 1) * g.R) + r - g.Hs) * g.Wp + x) * C + cg * 8);
+    }
+    *reinterpret_cast<uint4*>(T + p * C + cg * 8) = v;
+  }
+}
+
+// Per-CTA sums of squares of a bf16 tensor (padding is zero, so the whole buffer may be summed); fixed order.
+__global__ void __launch_bounds__(256)
+ssq_partial_kernel(const bf16* __restrict__ T, long long n8, float* __restrict__ part) {
+  float s = 0.f;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n8; i += gridDim.x * 256ll) {
+    const uint4 q = *reinterpret_cast<const uint4*>(T + i * 8);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float a = __uint_as_float(w[j] << 16), b = __uint_as_float(w[j] & 0xFFFF0000u);
+      s = fmaf(a, a, s);
+      s = fmaf(b, b, s);
+    }
+  }
+  __shared__ float sh[256];
+  sh[threadIdx.x] = s;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) part[blockIdx.x] = sh[0];
+}
+
+// Public kernel K[o][c][u][v]  <->  internal Wm[o][t = u kw + v][c padded to Cp].
+__global__ void pack_w_kernel(const bf16* __restrict__ K, bf16* __restrict__ Wm, int Cout, int Cin, int taps, int Cp) {
+  const long long n = static_cast<long long>(Cout) * taps * Cp;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
+    const int c = static_cast<int>(i % Cp);
+    const int t = static_cast<int>((i / Cp) % taps);
+    const int o = static_cast<int>(i / (static_cast<long long>(Cp) * taps));
+    Wm[i] = c < Cin ? K[(static_cast<long long>(o) * Cin + c) * taps + t] : __float2bfloat16(0.f);
+  }
+}
+template <typename T>
+__global__ void unpack_w_kernel(const T* __restrict__ Wm, T* __restrict__ K, int Cout, int Cin, int taps, int Cp) {
+  const long long n = static_cast<long long>(Cout) * Cin * taps;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
+    const int t = static_cast<int>(i % taps);
+    const int c = static_cast<int>((i / taps) % Cin);
+    const int o = static_cast<int>(i / (static_cast<long long>(taps) * Cin));
+    K[i] = Wm[(static_cast<long long>(o) * taps + t) * Cp + c];
+  }
+}
+__global__ void pack_dw_kernel(const float* __restrict__ K, float* __restrict__ Wm, int Cout, int Cin, int taps, int Cp) {
+  const long long n = static_cast<long long>(Cout) * taps * Cp;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
+    const int c = static_cast<int>(i % Cp);
+    const int t = static_cast<int>((i / Cp) % taps);
+    const int o = static_cast<int>(i / (static_cast<long long>(Cp) * taps));
+    Wm[i] = c < Cin ? K[(static_cast<long long>(o) * Cin + c) * taps + t] : 0.f;
+  }
+}
+
+int grid_1d(long long n, int num_sms) {
+  const long long b = (n + 255) / 256;
+  const long long cap = static_cast<long long>(num_sms) * 16;
+  return static_cast<int>(std::max(1ll, std::min(b, cap)));
+}
+int round64(int c) { return (c + 63) / 64 * 64; }
+
+}  // namespace
+
+struct GenConv {
+  int L = 0;
+  Geo g{};
+  int P = 1, S = 1;                       // processes of the grid; fp32 partial sums per weight gradient asked for
+  std::vector<int> Cin, Cout, kh, kw, relu, taps, Cp;
+  std::vector<bf16*> act, dY, Wm;
+  std::vector<float*> dWm;
+  std::vector<TcGemm> fwd, bwd_data, bwd_weight;
+  float* partials = nullptr;
+  float* loss_part = nullptr;
+  int loss_grid = 0;
+  int* status = nullptr;
+  cudaStream_t stream = nullptr;
+  Profiler* prof = nullptr;
+  int num_sms = 148;
+  bool fc_above = false;
+};
+
+namespace {
+
+Epi make_epi_act(void* out, int64_t ldo, int out_bf16, int relu) {
+  Epi e{};
+  e.op = EPI_ACT; e.out_bf16 = out_bf16; e.out = out; e.ldo = ldo; e.relu = relu;
+  return e;
+}
+Epi make_epi_mask(void* out, int64_t ldo, const void* mask, int64_t ldmask) {
+  Epi e{};
+  e.op = EPI_MASK; e.out_bf16 = 1; e.out = out; e.ldo = ldo; e.mask = mask; e.ldmask = ldmask;
+  return e;
+}
+Epi make_epi_sgd(void* w, int64_t ldo, float scale) {
+  Epi e{};
+  e.op = EPI_SGD; e.out_bf16 = 1; e.out = w; e.ldo = ldo; e.scale = scale;
+  return e;
+}
+
+// One product and, when its K range was cut into planes, their reduction with the tail operation.
+mbd_status run(GenConv* c, TcGemm& t, int cls, double flops, const Epi& epi) {
+  t.epi = epi;
+  t.partials = c->partials;
+  t.flags = nullptr;
+  c->prof->begin(cls, flops, c->stream);
+  if (tc_gemm_launch(t, c->stream) != cudaSuccess) return MBD_E_CUDA;
+  c->prof->end();
+  if (t.k_splits > 1) {
+    const double esz = epi.out_bf16 ? 2.0 : 4.0;
+    c->prof->begin(MBD_K_REDUCE, static_cast<double>(t.M) * t.N * (4.0 * t.k_splits + 2.0 * esz), c->stream);
+    if (reduce_partials_launch(c->partials, t.k_splits, t.M, t.N, epi, c->num_sms, c->stream) != cudaSuccess) return MBD_E_CUDA;
+    c->prof->end();
+  }
+  return MBD_OK;
+}
+
+void pad_fix(GenConv* c, bf16* T, int C, bool fill_halos) {
+  c->prof->begin(MBD_K_HALO, static_cast<double>(c->g.Ptot - static_cast<long long>(c->g.Z) * c->g.Hs * c->g.W) * C * 2.0, c->stream);
+  pad_fix_kernel<<<grid_1d(c->g.Ptot * (C / 8), c->num_sms), 256, 0, c->stream>>>(T, c->g, C, fill_halos ? 1 : 0);
+  c->prof->end();
+}
+
+void set_shift(TcGemm& t, int mode, int taps, int blocks, int Cp, int kh, int kw, int Wp) {
+  t.cv.mode = mode; t.cv.taps = taps; t.cv.blocks = blocks; t.cv.Cp = Cp;
+  for (int u = 0; u < kh; ++u)
+    for (int v = 0; v < kw; ++v) t.cv.off[u * kw + v] = (u - kh / 2) * Wp + (v - kw / 2);
+}
+
+}  // namespace
+
+bool gconv_needed(const mbd_layer* layers, int L) {
+  if (getenv("MBD_CONV_GENERAL")) return true;        // tuning knob: the listed 64-channel layers through this path too
+  for (int i = 0; i < L; ++i) {
+    const mbd_layer& l = layers[i];
+    const bool k3 = l.kh == 3 && l.kw == 3, k1 = l.kh == 1 && l.kw == 1;
+    if (!(k3 || k1) || l.C_in != 64 || l.C_out != 64) return true;
+  }
+  return false;
+}
+
+void gconv_destroy(GenConv* c) {
+  if (!c) return;
+  for (size_t i = 0; i < c->act.size(); ++i) cudaFree(c->act[i]);
+  for (size_t i = 0; i < c->dY.size(); ++i)
+    if (c->dY[i] && (c->act.size() <= static_cast<size_t>(c->L) || c->dY[i] != c->act[c->L])) cudaFree(c->dY[i]);
+  for (bf16* p : c->Wm) cudaFree(p);
+  for (float* p : c->dWm) cudaFree(p);
+  cudaFree(c->partials); cudaFree(c->loss_part);
+  delete c;
+}
+
+mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, int max_partials, int num_sms, int* status,
+                        cudaStream_t stream, Profiler* prof, bool fc_above, GenConv** out) {
+  if (tc_gemm_init() != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
+  const int H = layers[0].H, W = layers[0].W;
+  int ph = 0, pw = 0;
+  for (int i = 0; i < L; ++i) {
+    const mbd_layer& l = layers[i];
+    if (l.kh < 1 || l.kw < 1 || l.kh > 7 || l.kw > 7 || l.kh % 2 == 0 || l.kw % 2 == 0) return MBD_E_UNSUPPORTED;
+    if (l.C_in < 8 || l.C_out < 8 || l.C_in % 8 || l.C_out % 8) return MBD_E_UNSUPPORTED;       // 16-byte rows for TMA
+    if (i > 0 && l.C_in != layers[i - 1].C_out) return MBD_E_INVALID;
+    ph = std::max(ph, l.kh / 2); pw = std::max(pw, l.kw / 2);
+  }
+  if (H % P_r != 0) return MBD_E_UNSUPPORTED;            // strips of equal height on this path
+  const int Hs = H / P_r;
+  if (P_r > 1 && Hs < ph) return MBD_E_GRID;             // a halo row must come from the adjacent strip
+  GenConv* c = new (std::nothrow) GenConv();
+  if (!c) return MBD_E_ALLOC;
+  c->L = L; c->status = status; c->stream = stream; c->prof = prof; c->num_sms = num_sms; c->fc_above = fc_above;
+  Geo& g = c->g;
+  g.B = static_cast<int>(B); g.H = H; g.W = W; g.P_r = P_r; g.Hs = Hs; g.ph = ph; g.pw = pw;
+  g.R = Hs + 2 * ph; g.Wp = W + 2 * pw; g.Z = B * P_r; g.Ptot = g.Z * g.R * g.Wp;
+  if (B > INT32_MAX / std::max(1, P_r) || g.Ptot > INT32_MAX - 512) { delete c; return MBD_E_UNSUPPORTED; }   // TMA coordinates are 32-bit
+  c->P = P_r * P_c;
+  c->S = max_partials < 1 ? 1 : std::min(c->P, max_partials);
+  auto alloc = [&](void** p, size_t bytes) -> bool {
+    if (cudaMalloc(p, bytes) != cudaSuccess) { (void)cudaGetLastError(); *p = nullptr; return false; }
+    return cudaMemsetAsync(*p, 0, bytes, stream) == cudaSuccess;
+  };
+  bool ok = true;
+  c->act.assign(L + 1, nullptr); c->dY.assign(L, nullptr); c->Wm.assign(L, nullptr); c->dWm.assign(L, nullptr);
+  c->fwd.resize(L); c->bwd_data.resize(L); c->bwd_weight.resize(L);
+  for (int i = 0; i < L; ++i) {
+    const mbd_layer& l = layers[i];
+    c->Cin.push_back(l.C_in); c->Cout.push_back(l.C_out); c->kh.push_back(l.kh); c->kw.push_back(l.kw);
+    // the output of the last layer of a convolution-only network goes into the half-SSQ loss as it is
+    c->relu.push_back((i == L - 1 && !fc_above) ? 0 : l.relu);
+    c->taps.push_back(l.kh * l.kw); c->Cp.push_back(round64(l.C_in));
+  }
+  // (a slack of one tile of rows behind every tensor is not needed: rows outside a tensor map read as zero)
+  for (int i = 0; i <= L && ok; ++i) {
+    const int C = i == 0 ? c->Cin[0] : c->Cout[i - 1];
+    ok = alloc(reinterpret_cast<void**>(&c->act[i]), static_cast<size_t>(g.Ptot) * C * 2);
+  }
+  for (int i = 0; i < L && ok; ++i) {
+    if (i < L - 1 || fc_above) ok = alloc(reinterpret_cast<void**>(&c->dY[i]), static_cast<size_t>(g.Ptot) * c->Cout[i] * 2);
+    else c->dY[i] = c->act[L];                       // half-SSQ loss: dY_L = Y_L
+    const size_t nw = static_cast<size_t>(c->Cout[i]) * c->taps[i] * c->Cp[i];
+    ok = ok && alloc(reinterpret_cast<void**>(&c->Wm[i]), nw * 2) && alloc(reinterpret_cast<void**>(&c->dWm[i]), nw * 4);
+  }
+  c->loss_grid = num_sms * 4;
+  ok = ok && alloc(reinterpret_cast<void**>(&c->loss_part), sizeof(float) * c->loss_grid);
+  if (!ok) { gconv_destroy(c); return MBD_E_ALLOC; }
+  size_t part_elems = 0;
+  for (int i = 0; i < L; ++i) {
+    const int Cin = c->Cin[i], Cout = c->Cout[i], taps = c->taps[i], Cp = c->Cp[i], Cop = round64(Cout);
+    const int ldw = taps * Cp;
+    // forward
+    TcGemm& f = c->fwd[i];
+    f = TcGemm{};
+    f.variant = 0; f.M = static_cast<int>(g.Ptot); f.N = Cout; f.K = taps * Cp; f.k_splits = 1; f.status = status;
+    set_shift(f, 1, taps, Cp / 64, Cp, c->kh[i], c->kw[i], g.Wp);
+    f.cv_a_inner = Cin;
+    const Epi ef = make_epi_act(c->act[i + 1], Cout, 1, c->relu[i]);
+    if (tc_gemm_prepare(f, c->act[i], Cin, c->Wm[i], ldw, num_sms, &ef) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
+    // backward-data
+    if (i > 0) {
+      TcGemm& d = c->bwd_data[i];
+      d = TcGemm{};
+      d.variant = 1; d.M = static_cast<int>(g.Ptot); d.N = Cin; d.K = taps * Cop; d.k_splits = 1; d.status = status;
+      set_shift(d, 2, taps, Cop / 64, Cp, c->kh[i], c->kw[i], g.Wp);
+      d.cv_a_inner = Cout; d.cv_b_inner = ldw; d.cv_b_rows = Cout;
+      const Epi ed = make_epi_mask(c->dY[i - 1], Cin, c->relu[i - 1] ? c->act[i] : nullptr, Cin);
+      if (tc_gemm_prepare(d, c->dY[i], Cout, c->Wm[i], ldw, num_sms, &ed) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
+    }
+    // backward-weight: few output tiles, a very long K (all pixels): the planner cuts K to fill the SMs
+    TcGemm& w = c->bwd_weight[i];
+    w = TcGemm{};
+    w.variant = 2; w.M = Cout; w.N = ldw; w.K = static_cast<int>(g.Ptot); w.k_splits = c->S; w.status = status;
+    w.allow_extra_split = 1;
+    set_shift(w, 3, taps, 0, Cp, c->kh[i], c->kw[i], g.Wp);
+    w.cv_b_inner = Cin; w.cv_b_rows = g.Ptot;
+    const Epi ew = make_epi_sgd(c->Wm[i], ldw, 0.f);
+    if (tc_gemm_prepare(w, c->dY[i], Cout, c->act[i], Cin, num_sms, &ew) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
+    if (w.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(w.k_splits) * Cout * ldw);
+  }
+  if (part_elems && !alloc(reinterpret_cast<void**>(&c->partials), part_elems * 4)) { gconv_destroy(c); return MBD_E_ALLOC; }
+  if (cudaStreamSynchronize(stream) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
+  *out = c;
+  return MBD_OK;
+}
+
+size_t gconv_input_bytes(const GenConv* c) { return static_cast<size_t>(c->g.B) * c->Cin[0] * c->g.H * c->g.W * 2; }
+int gconv_last_relu(const GenConv* c) { return c->relu[c->L - 1]; }
+
+mbd_status gconv_set_weights(GenConv* c, int i, const void* K_dev) {
+  const long long n = static_cast<long long>(c->Cout[i]) * c->taps[i] * c->Cp[i];
+  pack_w_kernel<<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(static_cast<const bf16*>(K_dev), c->Wm[i], c->Cout[i], c->Cin[i], c->taps[i], c->Cp[i]);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+mbd_status gconv_get_weights(GenConv* c, int i, void* K_dev) {
+  const long long n = static_cast<long long>(c->Cout[i]) * c->Cin[i] * c->taps[i];
+  unpack_w_kernel<bf16><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(c->Wm[i], static_cast<bf16*>(K_dev), c->Cout[i], c->Cin[i], c->taps[i], c->Cp[i]);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+namespace {
+void stage(GenConv* c, const bf16* nchw, bf16* dst, int C, bool fill_halos) {
+  const long long n = static_cast<long long>(c->g.B) * c->g.H * c->g.W * (C / 8);
+  c->prof->begin(MBD_K_HALO, 2.0 * c->g.B * C * c->g.H * c->g.W * 2.0, c->stream);
+  nchw_to_pix_kernel<<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(nchw, dst, c->g, C);
+  c->prof->end();
+  pad_fix(c, dst, C, fill_halos);
+}
+void unstage(GenConv* c, const bf16* src, bf16* nchw, int C) {
+  const long long n = static_cast<long long>(c->g.B) * C * c->g.H * c->g.W;
+  c->prof->begin(MBD_K_HALO, 2.0 * n * 2.0, c->stream);
+  pix_to_nchw_kernel<bf16><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(src, nchw, c->g, C);
+  c->prof->end();
+}
+}  // namespace
+
+mbd_status gconv_stage_input(GenConv* c, const void* X_nchw) {
+  stage(c, static_cast<const bf16*>(X_nchw), c->act[0], c->Cin[0], true);     // the forward halo exchange of the input rides along
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+mbd_status gconv_forward_layer(GenConv* c, int i, float* loss_sum_dev) {
+  if (i < 0 || i >= c->L) return MBD_E_INVALID;
+  const bool last = i == c->L - 1;
+  const double flops = 2.0 * c->g.B * c->g.H * c->g.W * c->taps[i] * c->Cin[i] * c->Cout[i];     // the method's flops
+  const Epi e = make_epi_act(c->act[i + 1], c->Cout[i], 1, c->relu[i]);
+  mbd_status s = run(c, c->fwd[i], MBD_K_CONV_FWD, flops, e);
+  if (s != MBD_OK) return s;
+  // the output's halo exchange for the next layer (first halo term of Eq. 7); the last output is the top gradient of
+  // the half-SSQ loss and enters the weight-gradient sum: zeros outside the strips' own pixels
+  pad_fix(c, c->act[i + 1], c->Cout[i], !last);
+  if (last && loss_sum_dev && !c->fc_above) {
+    const long long n8 = c->g.Ptot * c->Cout[i] / 8;
+    c->prof->begin(MBD_K_OTHER, static_cast<double>(n8) * 16.0, c->stream);
+    ssq_partial_kernel<<<c->loss_grid, 256, 0, c->stream>>>(c->act[i + 1], n8, c->loss_part);
+    if (sum_f32_launch(c->loss_part, c->loss_grid, 0.5f, loss_sum_dev, c->stream) != cudaSuccess) return MBD_E_CUDA;
+    c->prof->end();
+  }
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+mbd_status gconv_forward(GenConv* c, const void* X_nchw, float* loss_sum_dev) {
+  mbd_status s = gconv_stage_input(c, X_nchw);
+  for (int i = 0; i < c->L && s == MBD_OK; ++i) s = gconv_forward_layer(c, i, loss_sum_dev);
+  return s;
+}
+
+mbd_status gconv_backward_layer(GenConv* c, int i, float fused_eta) {
+  if (i < 0 || i >= c->L) return MBD_E_INVALID;
+  const bool fused = fused_eta > 0.f;
+  const float scale = -fused_eta / static_cast<float>(c->g.B);
+  const double flops = 2.0 * c->g.B * c->g.H * c->g.W * c->taps[i] * c->Cin[i] * c->Cout[i];
+  const int ldw = c->taps[i] * c->Cp[i];
+  if (i > 0) {
+    // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0] -- with the
+    // weights as they are BEFORE this step's update, so this product comes first
+    if (c->g.P_r > 1) pad_fix(c, c->dY[i], c->Cout[i], true);
+    const Epi ed = make_epi_mask(c->dY[i - 1], c->Cin[i], c->relu[i - 1] ? c->act[i] : nullptr, c->Cin[i]);
+    mbd_status s = run(c, c->bwd_data[i], MBD_K_CONV_BWD_DATA, flops, ed);
+    if (s != MBD_OK) return s;
+    pad_fix(c, c->dY[i - 1], c->Cin[i], false);
+    if (c->g.P_r > 1) pad_fix(c, c->dY[i], c->Cout[i], false);      // the halo copies must not enter the sum below
+  }
+  // dY_i is zero outside the strips' own pixels here: every pixel enters the weight gradient once (the sum over the
+  // strips and batch blocks is the all-reduce over all P processes, last term of Eq. 9)
+  const Epi ew = fused ? make_epi_sgd(c->Wm[i], ldw, scale) : make_epi_act(c->dWm[i], ldw, 0, 0);
+  const mbd_status s = run(c, c->bwd_weight[i], MBD_K_CONV_BWD_WEIGHT, flops, ew);
+  if (s != MBD_OK) return s;
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+mbd_status gconv_backward(GenConv* c, float fused_eta) {
+  mbd_status s = MBD_OK;
+  for (int i = c->L - 1; i >= 0 && s == MBD_OK; --i) s = gconv_backward_layer(c, i, fused_eta);
+  return s;
+}
+
+mbd_status gconv_sgd_step(GenConv* c, float eta) {
+  const float scale = -eta / static_cast<float>(c->g.B);
+  for (int i = 0; i < c->L; ++i) {
+    const long long n = static_cast<long long>(c->Cout[i]) * c->taps[i] * c->Cp[i];
+    c->prof->begin(MBD_K_SGD, static_cast<double>(n) * 8.0, c->stream);
+    if (sgd_update_launch(c->Wm[i], 1, c->dWm[i], n, scale, c->num_sms, c->stream) != cudaSuccess) return MBD_E_CUDA;
+    c->prof->end();
+  }
+  return MBD_OK;
+}
+
+mbd_status gconv_output_to_nchw(GenConv* c, void* dst) {
+  unstage(c, c->act[c->L], static_cast<bf16*>(dst), c->Cout[c->L - 1]);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+mbd_status gconv_top_grad_from_nchw(GenConv* c, const void* src) {
+  if (!c->fc_above) return MBD_E_STATE;
+  stage(c, static_cast<const bf16*>(src), c->dY[c->L - 1], c->Cout[c->L - 1], false);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+mbd_status gconv_get_tensor(GenConv* c, int which, int layer, void* dst, size_t bytes) {
+  if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
+  if (which == MBD_T_DW) {
+    const long long n = static_cast<long long>(c->Cout[layer]) * c->Cin[layer] * c->taps[layer];
+    if (bytes != static_cast<size_t>(n) * 4) return MBD_E_INVALID;
+    unpack_w_kernel<float><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(c->dWm[layer], static_cast<float*>(dst), c->Cout[layer], c->Cin[layer],
+                                                                          c->taps[layer], c->Cp[layer]);
+    return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+  }
+  if (which != MBD_T_ACT && which != MBD_T_DY) return MBD_E_INVALID;
+  const int C = c->Cout[layer];
+  if (bytes != static_cast<size_t>(c->g.B) * C * c->g.H * c->g.W * 2) return MBD_E_INVALID;
+  unstage(c, which == MBD_T_ACT ? c->act[layer + 1] : c->dY[layer], static_cast<bf16*>(dst), C);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+mbd_status gconv_set_tensor(GenConv* c, int which, int layer, const void* src, size_t bytes) {
+  if (layer < 0 || layer >= c->L || which != MBD_T_ACT) return MBD_E_INVALID;
+  const int C = c->Cout[layer];
+  if (bytes != static_cast<size_t>(c->g.B) * C * c->g.H * c->g.W * 2) return MBD_E_INVALID;
+  stage(c, static_cast<const bf16*>(src), c->act[layer + 1], C, layer + 1 < c->L);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+mbd_status gconv_set_dw(GenConv* c, int layer, const void* src, size_t bytes) {
+  if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
+  const long long n = static_cast<long long>(c->Cout[layer]) * c->taps[layer] * c->Cp[layer];
+  if (bytes != static_cast<size_t>(c->Cout[layer]) * c->Cin[layer] * c->taps[layer] * 4) return MBD_E_INVALID;
+  pack_dw_kernel<<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(static_cast<const float*>(src), c->dWm[layer], c->Cout[layer], c->Cin[layer],
+                                                                c->taps[layer], c->Cp[layer]);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+}  // namespace mbd

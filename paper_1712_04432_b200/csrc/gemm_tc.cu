@@ -96,6 +96,7 @@ struct Params {
                           // (1: the pieces of a raster group follow one another; 2: all tiles piece by piece)
   int* flags;             // fix: one word per (tile, CTA of the pair, 128-row half, epilogue warp); zero between launches
   int join;               // > 1: a tile's `join` K pieces are accumulators of their own in tensor memory, added in the epilogue
+  ConvShift cv;           // cv.mode != 0: operand tiles are shifted views (see ConvShift)
 };
 
 struct Work {
@@ -312,17 +313,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (PAIR) tma_load_2d_pair(dst, tm, x, y, fb);
             else tma_load_2d(dst, tm, x, y, fb);
           };
-          if (A_MN == 0) {
-            load(sa, &tmA, kb * BK, row0);
+          if (p.cv.mode == 0) {
+            if (A_MN == 0) {
+              load(sa, &tmA, kb * BK, row0);
+            } else {
+#pragma unroll
+              for (int c = 0; c < BMT / 64; ++c) load(sa + c * (64 * BK * 2), &tmA, row0 + c * 64, kb * BK);
+            }
+            if (B_MN == 0) {
+              load(sb, &tmB, kb * BK, col0);
+            } else {
+#pragma unroll
+              for (int c = 0; c < BNL / 64; ++c) load(sb + c * (64 * BK * 2), &tmB, col0 + c * 64, kb * BK);
+            }
+          } else if (A_MN == 0) {
+            // convolution, forward (B K-major) or backward-data (B MN-major): k-block = (tap, 64-channel block)
+            const int t = kb / p.cv.blocks, cb = kb - t * p.cv.blocks;
+            load(sa, &tmA, cb * 64, B_MN == 0 ? row0 + p.cv.off[t] : row0 - p.cv.off[t]);
+            if (B_MN == 0) {
+              load(sb, &tmB, kb * BK, col0);
+            } else {
+#pragma unroll
+              for (int c = 0; c < BNL / 64; ++c) load(sb + c * (64 * BK * 2), &tmB, t * p.cv.Cp + col0 + c * 64, cb * 64);
+            }
           } else {
+            // convolution, backward-weight: K = pixels; an output column chunk = (tap, 64 input channels)
 #pragma unroll
             for (int c = 0; c < BMT / 64; ++c) load(sa + c * (64 * BK * 2), &tmA, row0 + c * 64, kb * BK);
-          }
-          if (B_MN == 0) {
-            load(sb, &tmB, kb * BK, col0);
-          } else {
 #pragma unroll
-            for (int c = 0; c < BNL / 64; ++c) load(sb + c * (64 * BK * 2), &tmB, col0 + c * 64, kb * BK);
+            for (int c = 0; c < BNL / 64; ++c) {
+              const int n0 = col0 + c * 64;
+              int t = n0 / p.cv.Cp;
+              if (t >= p.cv.taps) t = p.cv.taps - 1;        // columns beyond N: loaded from somewhere valid, never stored
+              load(sb + c * (64 * BK * 2), &tmB, n0 - t * p.cv.Cp, kb * BK + p.cv.off[t]);
+            }
           }
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
@@ -1059,10 +1083,12 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
     g.grid = static_cast<int>(2 * pairs);
   }
   const bool a_mn = g.variant == 2, b_mn = g.variant >= 1;
-  if (!a_mn) e = make_map(&g.tmA, A, g.K, g.M, lda, BK, BM * g.MH);   // A[M,K]: inner = K; box = the rows one CTA loads
+  if (g.cv.mode != 0 && g.cv.mode != g.variant + 1) return cudaErrorInvalidValue;
+  if (!a_mn) e = make_map(&g.tmA, A, g.cv.mode ? g.cv_a_inner : g.K, g.M, lda, BK, BM * g.MH);   // A[M,K]: inner = K; box = the rows one CTA loads
   else e = make_map(&g.tmA, A, g.M, g.K, lda, 64, BK);             // A[K,M]: inner = M, one 64-wide chunk per box
   if (e != cudaSuccess) return e;
   if (!b_mn) e = make_map(&g.tmB, B, g.K, g.N, ldb, BK, g.pair ? g.BN / 2 : g.BN);    // B[N,K]
+  else if (g.cv.mode) e = make_map(&g.tmB, B, g.cv_b_inner, g.cv_b_rows, ldb, 64, BK);     // the tensor as stored; the kernel shifts
   else e = make_map(&g.tmB, B, g.N, g.K, ldb, 64, BK);             // B[K,N]
   if (e != cudaSuccess) return e;
   // Running sum instead of S planes and a reduction launch: when the pieces of a tile are far apart in the
@@ -1119,6 +1145,7 @@ cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
   p.te_prefetch = getenv("MBD_TE_NO_PREFETCH") ? 0 : 1;                  // tuning knob
   p.flags = g.flags;
   p.join = g.join > 1 ? g.join : 1;
+  p.cv = g.cv;
   p.epi = g.epi;
   p.status = g.status;
   p.te = g.te && g.epi.op == g.te_epi.op && g.epi.out == g.te_epi.out && g.epi.out_bf16 && g.epi.mask == g.te_epi.mask &&

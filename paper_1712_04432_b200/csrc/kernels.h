@@ -88,6 +88,18 @@ struct Epi {
 // variant 0: D[M,N] = A[M,K] B[N,K]^T      (A, B K-contiguous)          forward
 // variant 1: D[M,N] = A[M,K] B[K,N]        (B N-contiguous)             backward-data
 // variant 2: D[M,N] = A[K,M]^T B[K,N]      (A M-contiguous, B N-cont.)  backward-weight
+// A convolution of k_h x k_w taps on tensors stored pixel-major ([pixels][channels], zero padding stored) is a
+// contraction whose operand tiles are views of the same tensor shifted by whole pixel rows: tap t reads pixel
+// p + off[t].  mode 1 (forward, variant 0): K index = (tap, input channel), padded to `Cp` per tap; the A tile of
+// k-block (t, cb) starts at row m0 + off[t], column 64 cb.  mode 2 (backward-data, variant 1): K index = (tap,
+// output channel); A tile at row m0 - off[t]; the B tile is rows 64 ob.. of the weight matrix [C_out][taps Cp] at
+// column t Cp + n0.  mode 3 (backward-weight, variant 2): K = pixels; the B chunk of output columns n0.. = (tap t,
+// channels n0 - t Cp ..) starts at pixel row k0 + off[t].  Rows outside the tensor read as zero (TMA fill).
+struct ConvShift {
+  int mode, taps, blocks, Cp;      // blocks: 64-wide k-blocks per tap (modes 1, 2)
+  int off[49];
+};
+
 struct TcGemm {
   CUtensorMap tmA, tmB;
   CUtensorMap tmOut, tmAux;   // output / mask-source maps of the TMA epilogue (valid when te)
@@ -116,6 +128,10 @@ struct TcGemm {
   // first launch that sees `partials` (the workspace is the caller's and is known only then)
   mutable CUtensorMap tmPlanes;
   mutable const float* planes_base = nullptr;
+  // Convolution as a contraction over shifted views (set before tc_gemm_prepare; cv.mode = 0: a plain product)
+  ConvShift cv = {};
+  int64_t cv_a_inner = 0;      // modes 1, 2: channels per pixel of the A tensor (its rows are pixels)
+  int64_t cv_b_inner = 0, cv_b_rows = 0;   // modes 2, 3: extent of the B tensor as stored (inner, rows)
 };
 
 // Fills tmA/tmB/BN/grid.  Returns cudaSuccess or an error.

@@ -300,19 +300,21 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
       if (l.d_in < 1 || l.d_out < 1) return MBD_E_INVALID;
       if (l.split != MBD_SPLIT_MODEL) return MBD_E_INVALID;
       if (i > Lc && l.d_in != layers[i - 1].d_out) return MBD_E_INVALID;
-      if (i == Lc && mixed && l.d_in != static_cast<int64_t>(layers[0].C_out) * layers[0].H * layers[0].W) return MBD_E_INVALID;
+      if (i == Lc && mixed && l.d_in != static_cast<int64_t>(layers[Lc - 1].C_out) * layers[0].H * layers[0].W) return MBD_E_INVALID;
       if (P_r > l.d_out) return MBD_E_GRID;
       if (dtype == MBD_BF16 && (l.d_in % 8 || l.d_out % 8)) return MBD_E_UNSUPPORTED;
       if (l.d_in > INT32_MAX || l.d_out > INT32_MAX || B > INT32_MAX) return MBD_E_UNSUPPORTED;
     } else if (l.kind == MBD_CONV3X3) {
-      const bool k3 = l.kh == 3 && l.kw == 3, k1 = l.kh == 1 && l.kw == 1;     // stride 1, "same" padding
-      if (!(k3 || k1) || l.C_in != 64 || l.C_out != 64 || dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
+      // stride 1, "same" padding; odd kernel sizes up to 7, channel counts that are multiples of 8
+      if (l.kh < 1 || l.kw < 1 || l.kh > 7 || l.kw > 7 || l.kh % 2 == 0 || l.kw % 2 == 0 || dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
+      if (l.C_in < 8 || l.C_out < 8 || l.C_in % 8 || l.C_out % 8) return MBD_E_UNSUPPORTED;
+      if (i > 0 && l.C_in != layers[i - 1].C_out) return MBD_E_INVALID;
       if (l.split != MBD_SPLIT_DOMAIN && l.split != MBD_SPLIT_BATCH) return MBD_E_UNSUPPORTED;
       if (l.split != layers[0].split) return MBD_E_UNSUPPORTED;          // all convolutions split alike
       if (l.split == MBD_SPLIT_BATCH) {                                  // 1 x P: one sample per process at least
         if (l.H < 1 || l.W < 1 || static_cast<int64_t>(P_r) * P_c > B) return MBD_E_GRID;
-      } else if (l.H < 1 || l.W < 1 || P_r > l.H) {
-        return MBD_E_GRID;   // a strip needs >= 1 row (halo = 1)
+      } else if (l.H < 1 || l.W < 1 || P_r > l.H || (P_r > 1 && l.H / P_r < l.kh / 2)) {
+        return MBD_E_GRID;   // a strip needs >= 1 row, and its halo rows come from the adjacent strip only
       }
       if (i > 0 && (l.H != layers[0].H || l.W != layers[0].W)) return MBD_E_INVALID;
     } else {
@@ -356,7 +358,8 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
 
   if (Lc > 0) {
     // batch-split convolutions (Section 3's improved case) run on 1 x P: no strips, whatever P_r is
-    st = conv_create(layers, Lc, B, layers[0].split == MBD_SPLIT_BATCH ? 1 : P_r, n->max_partials, n->num_sms, n->status, n->stream, &n->prof,
+    const bool batch_split = layers[0].split == MBD_SPLIT_BATCH;
+    st = conv_create(layers, Lc, B, batch_split ? 1 : P_r, batch_split ? P_r * P_c : P_c, n->max_partials, n->num_sms, n->status, n->stream, &n->prof,
                      mixed || loss == MBD_LOSS_NONE, &n->conv);
     if (st != MBD_OK) { free_net(n); return st; }
     if (is_conv) {

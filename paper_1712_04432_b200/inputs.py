@@ -55,10 +55,21 @@ class Workload:
     n_layers: int = 0
     grids: List[Tuple[int, int]] = field(default_factory=list)
     fc_dims: Tuple[int, ...] = ()  # mixed: C*H*W -> ... -> classes above the n_layers convolutions
-    ksizes: Tuple[int, ...] = ()   # conv, mixed: kernel size (3 or 1) per convolution; empty = all 3 x 3
+    ksizes: Tuple = ()             # conv, mixed: kernel size per convolution, k or (k_h, k_w); empty = all 3 x 3
+    channels: Tuple[int, ...] = () # conv: C_0 .. C_L (layer i maps C_{i-1} -> C_i); empty = dims[0] everywhere
 
     def ksize(self, i: int) -> int:
-        return self.ksizes[i] if self.ksizes else 3
+        k = self.ksizes[i] if self.ksizes else 3
+        assert isinstance(k, int)
+        return k
+
+    def kshape(self, i: int) -> Tuple[int, int]:
+        k = self.ksizes[i] if self.ksizes else 3
+        return (k, k) if isinstance(k, int) else (int(k[0]), int(k[1]))
+
+    def chan(self, i: int) -> int:
+        """Channels of tensor i (0 = the input)."""
+        return self.channels[i] if self.channels else self.dims[0]
 
     @property
     def L(self) -> int:
@@ -105,9 +116,12 @@ def fc_workload(dims, B, dtype="bf16", x_dist="normal", name="custom") -> Worklo
     return Workload(name, "fc", tuple(int(d) for d in dims), int(B), dtype, x_dist, "softmax_ce")
 
 
-def conv_workload(C, H, W, B, n_layers=2, dtype="bf16", name="custom_conv", ksizes=()) -> Workload:
+def conv_workload(C, H, W, B, n_layers=2, dtype="bf16", name="custom_conv", ksizes=(), channels=()) -> Workload:
+    """`channels` = (C_0, .., C_L) for layers that change the channel count (then C = C_0)."""
+    if channels:
+        assert len(channels) == n_layers + 1 and channels[0] == C
     return Workload(name, "conv", (int(C), int(H), int(W)), int(B), dtype, "normal",
-                    "half_ssq", n_layers=n_layers, ksizes=tuple(ksizes))
+                    "half_ssq", n_layers=n_layers, ksizes=tuple(ksizes), channels=tuple(int(c) for c in channels))
 
 
 @dataclass
@@ -141,9 +155,9 @@ def make_inputs(w: Workload, seed: int = 0) -> Inputs:
     X = rnd(rng.standard_normal((w.B, C, H, Wd), dtype=np.float32))
     Ws = []
     for i in range(w.n_layers):
-        k = w.ksize(i)
-        K = rng.standard_normal((C, C, k, k), dtype=np.float32)
-        K *= np.float32(np.sqrt(2.0 / (k * k * C)))              # N(0, 2/(k^2 C))
+        kh, kw = w.kshape(i)
+        K = rng.standard_normal((w.chan(i + 1), w.chan(i), kh, kw), dtype=np.float32)
+        K *= np.float32(np.sqrt(2.0 / (kh * kw * w.chan(i))))              # N(0, 2/(k_h k_w C_in))
         Ws.append(rnd(K))
     bs: List[Optional[np.ndarray]] = [None] * w.n_layers
     if w.kind != "mixed":
@@ -172,7 +186,7 @@ def step_flops(w: Workload) -> int:
     C, H, Wd = w.dims
     macs = 0
     for i in range(w.n_layers):
-        per = w.B * H * Wd * C * C * w.ksize(i) ** 2
+        per = w.B * H * Wd * w.chan(i) * w.chan(i + 1) * w.kshape(i)[0] * w.kshape(i)[1]
         macs += (3 if i >= 1 else 2) * per
     if w.kind == "mixed":
         d = w.fc_dims

@@ -165,14 +165,17 @@ def fc_layers(dims: Sequence[int], bias: bool = True, relu: bool = True) -> List
                   d_out=int(dims[i])) for i in range(1, len(dims))]
 
 
-def conv_layers(n: int, C_: int, H: int, W: int, relu: bool = True, k=3, split: int = SPLIT_DOMAIN) -> List[Layer]:
-    """n convolution layers C -> C on H x W images, domain-split (row strips) or, with split=SPLIT_BATCH,
-    batch-parallel on 1 x P (Section 3's improved case); `k` is the kernel size (3 or 1), one value for all
-    layers or one per layer."""
-    ks = [k] * n if isinstance(k, int) else list(k)
+def conv_layers(n: int, C_: int, H: int, W: int, relu: bool = True, k=3, split: int = SPLIT_DOMAIN, channels=()) -> List[Layer]:
+    """n convolution layers on H x W images, domain-split (row strips) or, with split=SPLIT_BATCH,
+    batch-parallel on 1 x P (Section 3's improved case); `k` is the kernel size, k or (k_h, k_w), one value for all
+    layers or one per layer; `channels` = (C_0, .., C_n) when the layers change the channel count (else C -> C)."""
+    ks = [k] * n if isinstance(k, (int, tuple)) else list(k)
     assert len(ks) == n
-    return [Layer(kind=CONV3X3, split=split, relu=int(relu), bias=0, d_in=C_ * H * W, d_out=C_ * H * W,
-                  C_in=C_, C_out=C_, H=H, W=W, kh=ks[i], kw=ks[i]) for i in range(n)]
+    ks = [(q, q) if isinstance(q, int) else (int(q[0]), int(q[1])) for q in ks]
+    ch = list(channels) if channels else [C_] * (n + 1)
+    assert len(ch) == n + 1
+    return [Layer(kind=CONV3X3, split=split, relu=int(relu), bias=0, d_in=ch[i] * H * W, d_out=ch[i + 1] * H * W,
+                  C_in=ch[i], C_out=ch[i + 1], H=H, W=W, kh=ks[i][0], kw=ks[i][1]) for i in range(n)]
 
 
 def _layer_array(layers: Sequence[Layer]):

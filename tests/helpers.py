@@ -202,7 +202,7 @@ def oracle_kernel(K):
     """The oracle's 3 x 3 layer for a device kernel: a 1 x 1 kernel [O, C, 1, 1] is the 3 x 3 kernel whose
     centre tap holds it and whose other taps are zero (the same correlation)."""
     K = np.asarray(K, np.float64)
-    if K.shape[2] == 3:
+    if K.shape[2:] != (1, 1):
         return K
     K3 = np.zeros(K.shape[:2] + (3, 3), np.float64)
     K3[:, :, 1, 1] = K[:, :, 0, 0]
@@ -228,14 +228,14 @@ def oracle_conv_step(w, inp, strips=None, grid=None, eta=None):
     return O.train_step_blocked(layers, X, None, "half_ssq", eta, P_r, P_c, store=bf16_store)
 
 
-def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1, eta=None):
+def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1, eta=None, max_partials=0):
     import torch
     from paper_1712_04432_b200 import mbd
     C_, H, Wd = w.dims
     L = w.n_layers
     eta = w.eta if eta is None else eta
-    net = mbd.Net(mbd.conv_layers(L, C_, H, Wd, k=[w.ksize(i) for i in range(L)]), w.B, P_r, P_c, mbd.BF16,
-                  mbd.LOSS_HALF_SSQ, 0)
+    net = mbd.Net(mbd.conv_layers(L, C_, H, Wd, k=[w.kshape(i) for i in range(L)], channels=w.channels), w.B, P_r, P_c, mbd.BF16,
+                  mbd.LOSS_HALF_SSQ, max_partials)
     for i in range(L):
         net.set_weights(i, to_dev(inp.Ws[i], True))
     X = to_dev(inp.X, True)

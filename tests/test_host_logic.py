@@ -35,12 +35,16 @@ def test_invalid_and_unsupported():
     assert create(fc, 8, max_partials=-1) == mbd.E_INVALID
     assert create(mbd.fc_layers((64, 32)) + mbd.fc_layers((48, 16)), 8) == mbd.E_INVALID   # dims do not chain
     assert create(mbd.fc_layers((60, 30)), 8) == mbd.E_UNSUPPORTED                         # bf16 needs multiples of 8
-    conv5 = mbd.conv_layers(1, 64, 8, 16)
-    conv5[0].kh = conv5[0].kw = 5
-    assert create(conv5, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
-    conv13 = mbd.conv_layers(1, 64, 8, 16)
-    conv13[0].kh = 1                                                                       # 1 x 3: neither 3 x 3 nor 1 x 1
-    assert create(conv13, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
+    conv9 = mbd.conv_layers(1, 64, 8, 16)
+    conv9[0].kh = conv9[0].kw = 9                                                          # kernels up to 7 x 7
+    assert create(conv9, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
+    conv43 = mbd.conv_layers(1, 64, 8, 16)
+    conv43[0].kh = 4                                                                       # even sizes have no centre tap
+    assert create(conv43, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
+    assert create(mbd.conv_layers(1, 12, 8, 16), 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED      # channels: multiples of 8
+    assert create(mbd.conv_layers(2, 16, 8, 16, channels=(16, 32, 8))[:1] + mbd.conv_layers(1, 16, 8, 16), 4,
+                  loss=mbd.LOSS_HALF_SSQ) == mbd.E_INVALID                                 # channel counts do not chain
+    assert create(mbd.conv_layers(2, 16, 8, 16, k=[(5, 5), (1, 7)], channels=(16, 32, 8)), 4, loss=mbd.LOSS_HALF_SSQ) in (mbd.OK, mbd.E_CUDA)
     assert create(mbd.conv_layers(2, 64, 8, 16, k=[3, 1]), 4, loss=mbd.LOSS_HALF_SSQ) in (mbd.OK, mbd.E_CUDA)   # valid; E_CUDA only without a device
     assert create(mbd.conv_layers(1, 64, 8, 16), 4, loss=mbd.LOSS_SOFTMAX_CE) == mbd.E_UNSUPPORTED
     assert create(fc, 8, loss=mbd.LOSS_NONE) == mbd.E_UNSUPPORTED                          # "no loss" is for convolution stacks

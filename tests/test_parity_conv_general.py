@@ -1,0 +1,103 @@
+"""Convolution layers the 64-channel 3 x 3 / 1 x 1 kernels do not cover -- other odd kernel sizes (5 x 5, 1 x 7,
+7 x 1, mixed in one network), channel counts that change from layer to layer and are not multiples of 64 -- on row
+strips with floor(k_h/2) halo rows (Section 2.2) and P_c batch blocks: forward outputs, J, the back-propagated
+gradients, the kernel gradients and the applied update against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+from paper_1712_04432_b200 import inputs as I
+from tests.helpers import compare_conv_step, gpu_conv_step, oracle_conv_step, oracle_with_eta, rel_fro, update_sized_eta
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+CASES = {
+    # name: (channels C_0..C_L, kernel shapes, H, W, B)
+    "five_by_five_then_three": ((16, 32, 24), ((5, 5), (3, 3)), 12, 20, 4),
+    "wide_and_tall_kernels": ((8, 8, 8), ((1, 7), (7, 1)), 12, 18, 3),
+    "channel_blocks_of_64": ((64, 128, 64), ((3, 3), (1, 1)), 16, 24, 4),
+    "three_layers_7x7_first": ((8, 40, 72, 16), ((7, 7), (3, 5), (5, 3)), 18, 14, 2),
+}
+
+
+def stored_hidden(o):
+    return [np.ascontiguousarray(x, np.float32) for x in o["Xs"][1:]]
+
+
+@pytest.fixture(scope="module", params=sorted(CASES))
+def case(request):
+    ch, ks, H, W, B = CASES[request.param]
+    w = I.conv_workload(ch[0], H, W, B, n_layers=len(ks), name=request.param, ksizes=ks, channels=ch)
+    inp = I.make_inputs(w, seed=61)
+    o = oracle_conv_step(w, inp)
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    return w, inp, oracle_with_eta(o, inp.Ws, [None] * w.n_layers, w.B, eta), eta
+
+
+@pytest.mark.parametrize("P_r,P_c,mp", [(1, 1, 0), (2, 1, 0), (3, 2, 4), (1, 2, 1), (6, 1, 2)])
+@pytest.mark.parametrize("fused", [False, True])
+def test_general_layers_on_strips_and_batch_blocks(case, P_r, P_c, mp, fused):
+    w, inp, o, eta = case
+    H = w.dims[1]
+    if H % P_r:
+        pytest.skip("strips of equal height on this path")
+    if P_c > w.B:
+        pytest.skip("more batch blocks than samples")
+    if P_r > 1 and H // P_r < max(w.kshape(i)[0] // 2 for i in range(w.n_layers)):
+        pytest.skip("a strip shorter than its halo: refused by mbd_net_create (see the last test)")
+    g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o), P_c=P_c, eta=eta, max_partials=mp)
+    compare_conv_step(g, o, TOL, fused, init=inp, require_sized=True)
+
+
+def test_strip_formulation_of_the_oracle_agrees():
+    ch, ks, H, W, B = CASES["five_by_five_then_three"]
+    w = I.conv_workload(ch[0], H, W, B, n_layers=len(ks), name="strips", ksizes=ks, channels=ch)
+    inp = I.make_inputs(w, seed=62)
+    ob = oracle_conv_step(w, inp, grid=(3, 2))             # strips with two halo rows, partials per process
+    g = gpu_conv_step(w, inp, 3, P_c=2, force_acts=stored_hidden(ob))
+    compare_conv_step(g, ob, TOL)
+
+
+def test_listed_64_channel_layers_through_the_general_path(monkeypatch):
+    # the layers that have kernels of their own, forced onto the contraction kernel: same oracle, same tolerance,
+    # and the two device paths agree with each other far below it
+    w = I.conv_workload(64, 16, 40, 3, name="conv_both_paths")
+    inp = I.make_inputs(w, seed=63)
+    o = oracle_conv_step(w, inp)
+    own = gpu_conv_step(w, inp, 2, force_acts=stored_hidden(o))
+    monkeypatch.setenv("MBD_CONV_GENERAL", "1")
+    gen = gpu_conv_step(w, inp, 2, force_acts=stored_hidden(o))
+    compare_conv_step(gen, o, TOL)
+    for i in range(w.n_layers):
+        assert rel_fro(gen["act"][i], own["act"][i]) < 5e-3 and rel_fro(gen["dW"][i], own["dW"][i]) < 1e-3, i
+    assert abs(gen["J"] - own["J"]) < 1e-3 * abs(own["J"])
+
+
+def test_free_running_step_and_reproducibility():
+    ch, ks, H, W, B = CASES["channel_blocks_of_64"]
+    w = I.conv_workload(ch[0], H, W, B, n_layers=len(ks), name="free", ksizes=ks, channels=ch)
+    inp = I.make_inputs(w, seed=64)
+    o = oracle_conv_step(w, inp)
+    a = gpu_conv_step(w, inp, 2, fused=True, P_c=2)
+    compare_conv_step(a, o, TOL, fused=True, tol_below_relu=2e-2)
+    b = gpu_conv_step(w, inp, 2, fused=True, P_c=2)
+    for i in range(w.n_layers):
+        assert np.array_equal(a["new_W"][i], b["new_W"][i]) and np.array_equal(a["dY"][i], b["dY"][i])
+
+
+def test_unsupported_shapes_are_refused():
+    from paper_1712_04432_b200 import mbd
+    for kw in (dict(k=(4, 3)), dict(k=9), dict(channels=(12, 8, 8)), dict(channels=(8, 4, 8))):
+        layers = mbd.conv_layers(2, 8, 12, 12, **{"k": 3, **kw}) if "channels" not in kw else \
+            mbd.conv_layers(2, kw["channels"][0], 12, 12, channels=kw["channels"])
+        with pytest.raises(mbd.MbdError) as e:
+            mbd.Net(layers, 2, 1, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+        assert e.value.status == mbd.E_UNSUPPORTED, kw
+    # a 7-row kernel needs three halo rows from the adjacent strip: strips of two rows cannot supply them
+    with pytest.raises(mbd.MbdError) as e:
+        mbd.Net(mbd.conv_layers(1, 8, 12, 12, k=7), 2, 6, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+    assert e.value.status == mbd.E_GRID
+    # strips of unequal height exist only for the 64-channel layers
+    with pytest.raises(mbd.MbdError) as e:
+        mbd.Net(mbd.conv_layers(1, 8, 13, 12, k=5), 2, 2, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+    assert e.value.status == mbd.E_UNSUPPORTED
