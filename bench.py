@@ -128,8 +128,12 @@ def workload_config(w, grid, max_partials):
         desc = (f"{w.name}: {w.n_layers}x conv3x3 {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, then FC "
                 f"{'-'.join(str(d) for d in w.fc_dims)}, B={w.B}, ReLU, softmax-CE, {w.dtype}")
     else:
-        ks = "x".join(str(w.ksize(0)) * 2)
-        desc = f"{w.name}: {w.n_layers}x conv{ks} {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, B={w.B}, half-SSQ, {w.dtype}"
+        if w.channels or any(w.kshape(i) != w.kshape(0) for i in range(w.n_layers)):
+            lay = ", ".join(f"{w.kshape(i)[0]}x{w.kshape(i)[1]} {w.chan(i)}->{w.chan(i + 1)}" for i in range(w.n_layers))
+            desc = f"{w.name}: conv layers {lay} on {w.dims[1]}x{w.dims[2]}, B={w.B}, half-SSQ, {w.dtype}"
+        else:
+            ks = "x".join(str(w.ksize(0)) * 2)
+            desc = f"{w.name}: {w.n_layers}x conv{ks} {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, B={w.B}, half-SSQ, {w.dtype}"
     return dict(workload=desc, grid=f"{grid[0]}x{grid[1]}", max_partials=max_partials, batch=w.B,
                 l2="weights + activations per step exceed the 126 MB L2 (no flush needed)"
                 if I.step_flops(w) > 1e12 else "L2 flushed by a 256 MB write between steps")
@@ -164,7 +168,7 @@ def oracle_sample(w, inp):
     Bs, Hs = 1, min(H, 56)
     def as3x3(k):          # the oracle's layer is 3 x 3: a 1 x 1 kernel is its centre tap
         k = k.astype(np.float64)
-        if k.shape[-1] == 3:
+        if k.shape[2:] != (1, 1):
             return k
         k3 = np.zeros(k.shape[:2] + (3, 3))
         k3[:, :, 1, 1] = k[:, :, 0, 0]
@@ -289,8 +293,8 @@ def run_ours(args):
         labels_host = torch.from_numpy(inp.labels).pin_memory()
     else:
         C_, H, Wd = w.dims
-        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.ksize(i) for i in range(w.n_layers)]), w.B, grid[0], grid[1],
-                      mbd.BF16, mbd.LOSS_HALF_SSQ, args.max_partials)
+        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.kshape(i) for i in range(w.n_layers)], channels=w.channels),
+                      w.B, grid[0], grid[1], mbd.BF16, mbd.LOSS_HALF_SSQ, args.max_partials)
         for i, Ki in enumerate(inp.Ws):
             net.set_weights(i, dev(Ki))
         labels = labels_host = None

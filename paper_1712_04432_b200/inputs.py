@@ -91,6 +91,10 @@ WORKLOADS = {
     "cfg5": Workload("cfg5", "fc", (8192,) * 9, 8192, "bf16", "normal", "softmax_ce",
                      grids=[(1, 1), (16, 16), (64, 4), (4, 64)]),
 }
+# Not a listed configuration: convolution layers the 64-channel kernels do not cover (5 x 5 and 3 x 3 kernels,
+# 64 -> 128 -> 128 channels, 112 x 112 images), for measuring the general convolution path.
+WORKLOADS["conv5x5"] = Workload("conv5x5", "conv", (64, 112, 112), 32, "bf16", "normal", "half_ssq", eta=1e-7, n_layers=2,
+                                grids=[(1, 1), (2, 1), (4, 1), (8, 1)], ksizes=((5, 5), (3, 3)), channels=(64, 128, 128))
 
 
 def mixed_workload(C, H, W, n_conv, fc_dims, B, name="custom_mixed", grids=(), ksizes=()) -> "Workload":

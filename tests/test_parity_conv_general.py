@@ -6,7 +6,8 @@ import numpy as np
 import pytest
 
 from paper_1712_04432_b200 import inputs as I
-from tests.helpers import compare_conv_step, gpu_conv_step, oracle_conv_step, oracle_with_eta, rel_fro, update_sized_eta
+from tests.helpers import (compare_conv_step, compare_mixed_step, gpu_conv_step, gpu_mixed_step, oracle_conv_step, oracle_mixed_acts,
+                           oracle_mixed_step, oracle_with_eta, rel_fro, update_sized_eta)
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-2
@@ -83,6 +84,19 @@ def test_free_running_step_and_reproducibility():
     b = gpu_conv_step(w, inp, 2, fused=True, P_c=2)
     for i in range(w.n_layers):
         assert np.array_equal(a["new_W"][i], b["new_W"][i]) and np.array_equal(a["dY"][i], b["dY"][i])
+
+
+@pytest.mark.parametrize("grid,mp,fused", [((1, 1), 1, False), ((2, 3), 4, True), ((4, 2), 2, False)])
+def test_integrated_stack_on_general_convolutions(grid, mp, fused):
+    # Section 2.4 on layers of the general path: a 5 x 5 and a 3 x 3 convolution with 16 channels on 8 x 20 images, then
+    # model-parallel fully connected layers 2560 -> 64 -> 16 on the same grid
+    w = I.mixed_workload(16, 8, 20, 2, (64, 16), 6, name="mixed_general", ksizes=(5, 3))
+    inp = I.make_inputs(w, seed=65)
+    o = oracle_mixed_step(w, inp)
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    o = oracle_with_eta(o, inp.Ws, inp.bs, w.B, eta)
+    g = gpu_mixed_step(w, inp, grid, mp, fused=fused, force_acts=oracle_mixed_acts(o, w), eta=eta)
+    compare_mixed_step(g, o, w, TOL, fused=fused, init=inp, require_sized=True)
 
 
 def test_unsupported_shapes_are_refused():
