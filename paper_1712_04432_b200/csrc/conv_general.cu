@@ -38,74 +38,101 @@ struct Geo {
 };
 
 // ------------------------------------------------------------------------------ layout kernels
-// NCHW -> pixel-major (own pixels only; padding and halos are the business of pad_fix_kernel).
-// One thread per (pixel, 8 channels): eight reads that are coalesced across the warp (consecutive w), one 16-byte store.
+// NCHW <-> pixel-major (own pixels only; padding and halos are the business of pad_fix_kernel).  A block moves a
+// tile of 32 consecutive pixels of one image row x 64 channels through shared memory, so that both sides are
+// accessed in runs: 64 bytes per channel on the NCHW side, 128 bytes per pixel on the pixel-major side.
+// grid = (B * H, ceil(W / 32), ceil(C / 64)), 256 threads.
 __global__ void __launch_bounds__(256)
 nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C) {
-  const int c8 = C / 8;
-  const long long total = static_cast<long long>(g.B) * g.H * g.W * c8;
-  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
-    const int w = static_cast<int>(i % g.W);
-    long long q = i / g.W;
-    const int h = static_cast<int>(q % g.H); q /= g.H;
-    const int cg = static_cast<int>(q % c8);
-    const int b = static_cast<int>(q / c8);
-    const int s = h / g.Hs, r = h - s * g.Hs + g.ph;
-    uint16_t v[8];
+  __shared__ uint16_t tile[64][34];
+  const int w0 = blockIdx.y * 32, b = blockIdx.x / g.H, h = blockIdx.x - b * g.H, c0 = blockIdx.z * 64;
+  const int t = threadIdx.x;
+  {
+    const int c = t >> 2, wq = (t & 3) * 8;           // channel c0 + c, pixels w0 + wq .. + 7
+    if (c0 + c < C) {
+      const bf16* q = src + ((static_cast<long long>(b) * C + c0 + c) * g.H + h) * g.W + w0 + wq;
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
-      v[j] = __bfloat16_as_ushort(src[((static_cast<long long>(b) * C + cg * 8 + j) * g.H + h) * g.W + w]);
-    uint4 o;
-    o.x = v[0] | (static_cast<uint32_t>(v[1]) << 16); o.y = v[2] | (static_cast<uint32_t>(v[3]) << 16);
-    o.z = v[4] | (static_cast<uint32_t>(v[5]) << 16); o.w = v[6] | (static_cast<uint32_t>(v[7]) << 16);
-    const long long p = ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w + g.pw;
-    *reinterpret_cast<uint4*>(dst + p * C + cg * 8) = o;
+      for (int j = 0; j < 8; ++j) tile[c][wq + j] = w0 + wq + j < g.W ? __bfloat16_as_ushort(q[j]) : 0;
+    }
   }
+  __syncthreads();
+  const int px = t >> 3, cg = t & 7;                  // pixel w0 + px, channels c0 + 8 cg .. + 7
+  if (w0 + px >= g.W || c0 + cg * 8 >= C) return;
+  uint16_t v[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) v[j] = tile[cg * 8 + j][px];
+  uint4 o;
+  o.x = v[0] | (static_cast<uint32_t>(v[1]) << 16); o.y = v[2] | (static_cast<uint32_t>(v[3]) << 16);
+  o.z = v[4] | (static_cast<uint32_t>(v[5]) << 16); o.w = v[6] | (static_cast<uint32_t>(v[7]) << 16);
+  const int s = h / g.Hs, r = h - s * g.Hs + g.ph;
+  const long long p = ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w0 + px + g.pw;
+  *reinterpret_cast<uint4*>(dst + p * C + c0 + cg * 8) = o;
 }
 
-template <typename T>   // T = bf16 (activations, gradients)
 __global__ void __launch_bounds__(256)
-pix_to_nchw_kernel(const T* __restrict__ src, T* __restrict__ dst, Geo g, int C) {
-  const long long total = static_cast<long long>(g.B) * C * g.H * g.W;
-  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
-    const int w = static_cast<int>(i % g.W);
-    long long q = i / g.W;
-    const int h = static_cast<int>(q % g.H); q /= g.H;
-    const int c = static_cast<int>(q % C);
-    const int b = static_cast<int>(q / C);
-    const int s = h / g.Hs, r = h - s * g.Hs + g.ph;
-    const long long p = ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w + g.pw;
-    dst[i] = src[p * C + c];
+pix_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C) {
+  __shared__ uint16_t tile[64][34];
+  const int w0 = blockIdx.y * 32, b = blockIdx.x / g.H, h = blockIdx.x - b * g.H, c0 = blockIdx.z * 64;
+  const int t = threadIdx.x;
+  {
+    const int px = t >> 3, cg = t & 7;
+    if (w0 + px < g.W && c0 + cg * 8 < C) {
+      const int s = h / g.Hs, r = h - s * g.Hs + g.ph;
+      const long long p = ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w0 + px + g.pw;
+      const uint4 q = *reinterpret_cast<const uint4*>(src + p * C + c0 + cg * 8);
+      const uint32_t wv[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        tile[cg * 8 + 2 * j][px] = static_cast<uint16_t>(wv[j] & 0xFFFFu);
+        tile[cg * 8 + 2 * j + 1][px] = static_cast<uint16_t>(wv[j] >> 16);
+      }
+    }
   }
+  __syncthreads();
+  const int c = t >> 2, wq = (t & 3) * 8;
+  if (c0 + c >= C) return;
+  bf16* q = dst + ((static_cast<long long>(b) * C + c0 + c) * g.H + h) * g.W + w0 + wq;
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    if (w0 + wq + j < g.W) q[j] = __ushort_as_bfloat16(tile[c][wq + j]);
 }
 
 // Everything that is not a strip's own pixel: the padding columns and the image's outer rows become zero; a halo
 // row becomes the copy of the neighbouring strip's boundary row (fill_halos) -- the halo exchange of Section 2.2:
 // floor(k_h/2) rows per neighbour and direction -- or zero (a gradient about to enter the weight-gradient sum, whose
-// pixels must each be counted once).  One thread per 16 bytes of the tensor; own pixels are left alone.
+// pixels must each be counted once).  One thread per 16 bytes of padding: per strip 2 ph whole rows, then the 2 pw
+// side columns of its Hs own rows.
 __global__ void __launch_bounds__(256)
 pad_fix_kernel(bf16* __restrict__ T, Geo g, int C, int fill_halos) {
   const int c8 = C / 8;
-  const long long total = g.Ptot * c8;
+  const int n_rows = 2 * g.ph * g.Wp * c8;             // chunks in the halo rows of a strip
+  const int n_side = g.Hs * 2 * g.pw * c8;             // chunks in the side columns of its own rows
+  const int per_strip = n_rows + n_side;
+  const long long total = g.Z * per_strip;
   for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
-    const int cg = static_cast<int>(i % c8);
-    const long long p = i / c8;
-    const int x = static_cast<int>(p % g.Wp);
-    const long long zr = p / g.Wp;
-    const int r = static_cast<int>(zr % g.R);
-    const long long z = zr / g.R;
-    const bool own_col = x >= g.pw && x < g.pw + g.W;
-    const bool own_row = r >= g.ph && r < g.ph + g.Hs;
-    if (own_col && own_row) continue;
+    const long long z = i / per_strip;
+    int k = static_cast<int>(i - z * per_strip);
+    int r, x, cg;
+    if (k < n_rows) {
+      cg = k % c8; k /= c8;
+      x = k % g.Wp; k /= g.Wp;                         // k: 0 .. 2 ph - 1
+      r = k < g.ph ? k : k + g.Hs;
+    } else {
+      k -= n_rows;
+      cg = k % c8; k /= c8;
+      const int side = k % (2 * g.pw); k /= 2 * g.pw;  // k: own row 0 .. Hs - 1
+      x = side < g.pw ? side : side + g.W;
+      r = k + g.ph;
+    }
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (fill_halos && own_col && !own_row) {
+    if (fill_halos && x >= g.pw && x < g.pw + g.W && (r < g.ph || r >= g.ph + g.Hs)) {
       const int s = static_cast<int>(z % g.P_r);
       if (r < g.ph && s > 0)                        // rows above the strip: the last rows of the strip above
         v = *reinterpret_cast<const uint4*>(T + ((((z - 1) * g.R) + r + g.Hs) * g.Wp + x) * C + cg * 8);
       else if (r >= g.ph + g.Hs && s < g.P_r - 1)   // rows below it: the first rows of the strip below
         v = *reinterpret_cast<const uint4*>(T + ((((z + 1) * g.R) + r - g.Hs) * g.Wp + x) * C + cg * 8);
     }
-    *reinterpret_cast<uint4*>(T + p * C + cg * 8) = v;
+    *reinterpret_cast<uint4*>(T + ((z * g.R + r) * g.Wp + x) * C + cg * 8) = v;
   }
 }
 
@@ -227,7 +254,8 @@ mbd_status run(GenConv* c, TcGemm& t, int cls, double flops, const Epi& epi) {
 
 void pad_fix(GenConv* c, bf16* T, int C, bool fill_halos) {
   c->prof->begin(MBD_K_HALO, static_cast<double>(c->g.Ptot - static_cast<long long>(c->g.Z) * c->g.Hs * c->g.W) * C * 2.0, c->stream);
-  pad_fix_kernel<<<grid_1d(c->g.Ptot * (C / 8), c->num_sms), 256, 0, c->stream>>>(T, c->g, C, fill_halos ? 1 : 0);
+  const long long chunks = c->g.Z * (2ll * c->g.ph * c->g.Wp + 2ll * c->g.Hs * c->g.pw) * (C / 8);
+  if (chunks > 0) pad_fix_kernel<<<grid_1d(chunks, c->num_sms), 256, 0, c->stream>>>(T, c->g, C, fill_halos ? 1 : 0);
   c->prof->end();
 }
 
@@ -367,16 +395,16 @@ mbd_status gconv_get_weights(GenConv* c, int i, void* K_dev) {
 
 namespace {
 void stage(GenConv* c, const bf16* nchw, bf16* dst, int C, bool fill_halos) {
-  const long long n = static_cast<long long>(c->g.B) * c->g.H * c->g.W * (C / 8);
+  const dim3 grid(static_cast<unsigned>(c->g.B) * c->g.H, (c->g.W + 31) / 32, (C + 63) / 64);
   c->prof->begin(MBD_K_HALO, 2.0 * c->g.B * C * c->g.H * c->g.W * 2.0, c->stream);
-  nchw_to_pix_kernel<<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(nchw, dst, c->g, C);
+  nchw_to_pix_kernel<<<grid, 256, 0, c->stream>>>(nchw, dst, c->g, C);
   c->prof->end();
   pad_fix(c, dst, C, fill_halos);
 }
 void unstage(GenConv* c, const bf16* src, bf16* nchw, int C) {
-  const long long n = static_cast<long long>(c->g.B) * C * c->g.H * c->g.W;
-  c->prof->begin(MBD_K_HALO, 2.0 * n * 2.0, c->stream);
-  pix_to_nchw_kernel<bf16><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(src, nchw, c->g, C);
+  const dim3 grid(static_cast<unsigned>(c->g.B) * c->g.H, (c->g.W + 31) / 32, (C + 63) / 64);
+  c->prof->begin(MBD_K_HALO, 2.0 * c->g.B * C * c->g.H * c->g.W * 2.0, c->stream);
+  pix_to_nchw_kernel<<<grid, 256, 0, c->stream>>>(src, nchw, c->g, C);
   c->prof->end();
 }
 }  // namespace
