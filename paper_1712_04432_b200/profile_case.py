@@ -17,8 +17,10 @@ fc:     `launches` training steps of a small fully connected net (softmax, bias-
         the products are launched as a workload on that logical grid launches them (two layers of
         8192 x 8192 at batch 8192 on 16x16 with 2 partials: the benchmark's three products, one of each
         per step plus a second forward and backward-weight product).
-conv:   `launches` training steps of the two-layer 3x3 convolution stack on `batch` images of
-64 x image x image (default 224), cut into `strips` row strips.
+conv:   `launches` training steps of a two-layer convolution stack on `batch` images of
+C_0 x image x image (default 64 x 224 x 224, 3 x 3 kernels), cut into `strips` row strips; --ksizes / --channels
+select other odd kernel sizes and channel counts (the general convolution path), e.g.
+    python -m paper_1712_04432_b200.profile_case conv --batch 16 --strips 2 --image 112 --ksizes 5,3 --channels 64,128,128
 """
 import argparse
 
