@@ -128,8 +128,9 @@ def workload_config(w, grid, max_partials):
         desc = (f"{w.name}: {w.n_layers}x conv3x3 {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, then FC "
                 f"{'-'.join(str(d) for d in w.fc_dims)}, B={w.B}, ReLU, softmax-CE, {w.dtype}")
     else:
-        if w.channels or any(w.kshape(i) != w.kshape(0) for i in range(w.n_layers)):
-            lay = ", ".join(f"{w.kshape(i)[0]}x{w.kshape(i)[1]} {w.chan(i)}->{w.chan(i + 1)}" for i in range(w.n_layers))
+        if w.channels or w.strides or any(w.kshape(i) != w.kshape(0) for i in range(w.n_layers)):
+            lay = ", ".join(f"{w.kshape(i)[0]}x{w.kshape(i)[1]}{'/' + str(w.stride(i)) if w.stride(i) > 1 else ''} {w.chan(i)}->{w.chan(i + 1)}"
+                            for i in range(w.n_layers))
             desc = f"{w.name}: conv layers {lay} on {w.dims[1]}x{w.dims[2]}, B={w.B}, half-SSQ, {w.dtype}"
         else:
             ks = "x".join(str(w.ksize(0)) * 2)
@@ -293,7 +294,8 @@ def run_ours(args):
         labels_host = torch.from_numpy(inp.labels).pin_memory()
     else:
         C_, H, Wd = w.dims
-        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.kshape(i) for i in range(w.n_layers)], channels=w.channels),
+        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.kshape(i) for i in range(w.n_layers)], channels=w.channels,
+                                      strides=w.strides),
                       w.B, grid[0], grid[1], mbd.BF16, mbd.LOSS_HALF_SSQ, args.max_partials)
         for i, Ki in enumerate(inp.Ws):
             net.set_weights(i, dev(Ki))

@@ -78,15 +78,17 @@ enum { MBD_LOSS_SOFTMAX_CE = 0, MBD_LOSS_HALF_SSQ = 1,
                                  mbd_set_tensor(MBD_T_DY, L-1) between the forward and the backward pass
                                  (the stack is the lower part of a larger network). */
 
-/* One layer.  FC: d_in, d_out.  Convolution (kh x kw, both odd, stride 1, zero pad floor(k/2), NCHW; see
- * mbd_net_create for the shapes that exist): C_in, C_out, H, W, kh, kw; d_in = C_in*H*W, d_out = C_out*H*W;
- * |W_i| = kh kw C_in C_out (Eq. 2).
+/* One layer.  FC: d_in, d_out.  Convolution (kh x kw, both odd, zero pad floor(k/2), NCHW; see mbd_net_create
+ * for the shapes that exist): C_in, C_out, kh, kw, the INPUT image size H x W and the stride (0 or 1: every
+ * position; s: the positions (s h', s w') of the stride-1 result, an H/s x W/s output -- H and W must be multiples of
+ * s); d_in = C_in*H*W, d_out = C_out*(H/s)*(W/s); |W_i| = kh kw C_in C_out (Eq. 2).
  * relu: apply f = ReLU after this layer (ignored for the last layer).
  * bias: FC only. */
 typedef struct {
   int32_t kind, split, relu, bias;
   int64_t d_in, d_out;
   int32_t C_in, C_out, H, W, kh, kw;
+  int32_t stride, reserved;
 } mbd_layer;
 
 /* Words (matrix elements) one process moves for one layer under the chosen
@@ -148,14 +150,15 @@ enum {
  * a strip would be shorter than its halo, or (batch-split convolutions) P_r P_c > B.
  * Batch-split convolutions (MBD_SPLIT_BATCH) are cut into P_r P_c batch blocks and no strips; between them
  * and the fully connected layers on P_r x P_c lies the re-distribution of Eq. 6 (mbd_redistribute_time).
- * Convolutions (kind MBD_CONV3X3 whatever the kernel size; Section 2.2): stride 1, zero padding floor(k/2), k_h and
- * k_w odd and at most 7, C_in and C_out multiples of 8, C_in of a layer = C_out of the layer below, one image size
- * for all of them; weights [C_out][C_in][k_h][k_w] ([C_out][C_in] for 1x1).  A strip needs floor(k_h/2) halo rows
- * from each neighbour, which must be the adjacent strip's own rows: MBD_E_GRID when H / P_r < floor(k_h/2).  The
- * layers with 64 channels and 3x3 or 1x1 kernels run on kernels of their own; every other shape runs as products
- * of row-shifted views on the contraction kernel of the fully connected layers, and there strips of unequal
+ * Convolutions (kind MBD_CONV3X3 whatever the kernel size; Section 2.2): zero padding floor(k/2), k_h and
+ * k_w odd and at most 7, stride 1 to 4 (the same in both directions), C_in and C_out multiples of 8, C_in of a layer =
+ * C_out of the layer below, H x W of a layer = the output size of the layer below (H/s x W/s of its input);
+ * weights [C_out][C_in][k_h][k_w] ([C_out][C_in] for 1x1).  A strip needs floor(k_h/2) halo rows
+ * from each neighbour, which must be the adjacent strip's own rows: MBD_E_GRID when a strip is shorter than that.  The
+ * stride-1 layers with 64 channels and 3x3 or 1x1 kernels run on kernels of their own; every other shape runs as
+ * products of row-shifted views on the contraction kernel of the fully connected layers, and there strips of unequal
  * height, fp32 master weights, momentum and the interior / boundary calls are MBD_E_UNSUPPORTED.
- * MBD_E_UNSUPPORTED for other convolutions (even or larger kernels, other channel counts, a stride),
+ * MBD_E_UNSUPPORTED for other convolutions (even or larger kernels, other channel counts, larger strides),
  * a convolution above a fully connected layer, half-SSQ with
  * fully connected layers or softmax-CE without them, or bf16 FC dims that are not
  * multiples of 8. */

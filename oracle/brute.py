@@ -96,6 +96,27 @@ def conv3x3_dK(dY, X, ksize=(3, 3)):
     return dK
 
 
+def conv_strided(K, X, s):
+    """Y[b][o][h'][w'] = sum_{c,u,v} K[o][c][u][v] X[b][c][s h'+u-p_h][s w'+v-p_w], p = floor(k/2)."""
+    KH, KW = len(K[0][0]), len(K[0][0][0])
+    B, C, H, W = len(X), len(X[0]), len(X[0][0]), len(X[0][0][0])
+    O = len(K)
+    Y = [[[[0.0] * (W // s) for _ in range(H // s)] for _ in range(O)] for _ in range(B)]
+    for b in range(B):
+        for o in range(O):
+            for h in range(H // s):
+                for w in range(W // s):
+                    acc = 0.0
+                    for c in range(C):
+                        for u in range(KH):
+                            for v in range(KW):
+                                hh, ww = s * h + u - KH // 2, s * w + v - KW // 2
+                                if 0 <= hh < H and 0 <= ww < W:
+                                    acc += K[o][c][u][v] * X[b][c][hh][ww]
+                    Y[b][o][h][w] = acc
+    return Y
+
+
 def softmax_ce_column(y, label):
     """Loss and gradient for one sample, without the max-subtraction trick
     (safe for the small logits the tests use)."""

@@ -35,9 +35,15 @@ def d_in(layer: Dict) -> int:
     return layer["d_in"]
 
 
+def out_hw(layer: Dict):
+    """Output image size of a convolution: a stride-s layer keeps every s-th position of its H x W input."""
+    s = max(1, layer.get("stride", 1))
+    return layer["H"] // s, layer["W"] // s
+
+
 def d_out(layer: Dict) -> int:
     if layer["kind"] == "conv":
-        return layer["H"] * layer["W"] * layer["C_out"]
+        return out_hw(layer)[0] * out_hw(layer)[1] * layer["C_out"]
     return layer["d_out"]
 
 
@@ -67,7 +73,7 @@ def eq7_domain_words(layers: Sequence[Dict], B: int, P: int) -> int:
     for l in layers:
         if P > 1:
             tot += B * l["W"] * l["C_in"] * (l["kh"] // 2)
-            tot += B * l["W"] * l["C_out"] * (l["kh"] // 2)
+            tot += B * out_hw(l)[1] * l["C_out"] * (l["kh"] // 2)          # Y_W Y_C floor(k_h/2) (Eq. 7)
         tot += _int(Fraction(2 * (P - 1) * n_weights(l), P))
     return tot
 
@@ -96,7 +102,7 @@ def layer_words(layers: Sequence[Dict], B: int, P_r: int, P_c: int) -> List[Dict
         else:
             if P_r > 1:
                 row["halo_fwd"] = _int(Fraction(B * l["W"] * l["C_in"] * (l["kh"] // 2), P_c))
-                row["halo_bwd"] = _int(Fraction(B * l["W"] * l["C_out"] * (l["kh"] // 2), P_c))
+                row["halo_bwd"] = _int(Fraction(B * out_hw(l)[1] * l["C_out"] * (l["kh"] // 2), P_c))
             row["allreduce_dw"] = _int(Fraction(2 * (P - 1) * n_weights(l), P))
         rows.append(row)
     return rows

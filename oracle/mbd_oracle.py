@@ -57,6 +57,7 @@ class Conv3x3:
     K: np.ndarray
     relu: bool = True
     split: str = "domain"
+    stride: int = 1      # s > 1: the layer keeps the positions (s h', s w') of the stride-1 result (un-blocked step only)
 
 
 def balanced_ranges(n: int, P: int):
@@ -173,6 +174,31 @@ def conv3x3_dK(dY, X, ksize=(3, 3)):
     return dK
 
 
+def conv_strided(K, X, s):
+    """A stride-s convolution is the stride-1 correlation kept at every s-th position in both directions:
+    Y[b,o,h',w'] = conv3x3(K, X)[b,o,s h',s w'] (H and W multiples of s)."""
+    assert X.shape[2] % s == 0 and X.shape[3] % s == 0
+    return conv3x3(K, X)[:, :, ::s, ::s]
+
+
+def _zero_stuffed(dY, s):
+    """The gradient of a stride-s layer's output, put back at the positions (s h', s w') of the stride-1 result,
+    zero elsewhere: what the kept positions' adjoint is."""
+    dY = np.asarray(dY, F64)
+    B, O, Ho, Wo = dY.shape
+    full = np.zeros((B, O, Ho * s, Wo * s), F64)
+    full[:, :, ::s, ::s] = dY
+    return full
+
+
+def conv_strided_dX(K, dY, s):
+    return conv3x3_dX(K, _zero_stuffed(dY, s))
+
+
+def conv_strided_dK(dY, X, ksize, s):
+    return conv3x3_dK(_zero_stuffed(dY, s), X, ksize)
+
+
 def softmax_ce(Y_L, labels):
     """J = sum_b [logsumexp_k Y[k,b] - Y[y_b,b]];  dY[:,b] = softmax(Y[:,b]) - e_{y_b}.
 
@@ -235,6 +261,8 @@ def forward(layers: Sequence, X1, store=None):
     for i, lay in enumerate(layers):
         if isinstance(lay, FC):
             Y = affine(lay.W, Xs[i], lay.b)
+        elif lay.stride > 1:
+            Y = conv_strided(lay.K, Xs[i], lay.stride)
         else:
             Y = conv3x3(lay.K, Xs[i])
         Ys.append(Y)
@@ -271,10 +299,17 @@ def train_step(layers: Sequence, X1, labels, loss: str, eta: float, store=None):
         if isinstance(lay, FC):
             dWs[i] = fc_dW(dYs[i], Xs[i])
             dbs[i] = dYs[i].sum(axis=1) if lay.b is not None else None
+        elif lay.stride > 1:
+            dWs[i] = conv_strided_dK(dYs[i], Xs[i], lay.K.shape[2:], lay.stride)
         else:
             dWs[i] = conv3x3_dK(dYs[i], Xs[i], lay.K.shape[2:])
         if i > 0:
-            dXs[i] = fc_dX(lay.W, dYs[i]) if isinstance(lay, FC) else conv3x3_dX(lay.K, dYs[i])
+            if isinstance(lay, FC):
+                dXs[i] = fc_dX(lay.W, dYs[i])
+            elif lay.stride > 1:
+                dXs[i] = conv_strided_dX(lay.K, dYs[i], lay.stride)
+            else:
+                dXs[i] = conv3x3_dX(lay.K, dYs[i])
             dXs[i] = _below(dXs[i], Ys[i - 1])
             prev = layers[i - 1]
             dYs[i - 1] = dXs[i] * (Ys[i - 1] > 0.0) if prev.relu else dXs[i]

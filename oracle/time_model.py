@@ -38,7 +38,7 @@ from __future__ import annotations
 from fractions import Fraction
 from typing import Dict, List, Optional, Sequence, Tuple
 
-from .comm_words import d_in, d_out, n_weights
+from .comm_words import d_in, d_out, n_weights, out_hw
 
 TERMS = ("allgather_y", "allreduce_dx", "allreduce_dw", "halo_fwd", "halo_bwd")
 
@@ -93,7 +93,7 @@ def layer_words_exact(layers: Sequence[Dict], B: int, P_r: int, P_c: int) -> Lis
         else:
             if P_r > 1:
                 row["halo_fwd"] = Fraction(B, P_c) * l["W"] * l["C_in"] * (l["kh"] // 2)
-                row["halo_bwd"] = Fraction(B, P_c) * l["W"] * l["C_out"] * (l["kh"] // 2)
+                row["halo_bwd"] = Fraction(B, P_c) * out_hw(l)[1] * l["C_out"] * (l["kh"] // 2)
             row["allreduce_dw"] = 2 * Fraction(P - 1, P) * n_weights(l)
         rows.append(row)
     return rows
@@ -133,7 +133,7 @@ def eq7_domain_time(layers: Sequence[Dict], B: int, P: int, alpha: float, beta: 
     for l in layers:
         if P > 1 and l["kh"] // 2 > 0:
             t += alpha + beta * B * l["W"] * l["C_in"] * (l["kh"] // 2)
-            t += alpha + beta * B * l["W"] * l["C_out"] * (l["kh"] // 2)
+            t += alpha + beta * B * out_hw(l)[1] * l["C_out"] * (l["kh"] // 2)
         t += 2.0 * (alpha * lg + beta * float(Fraction((P - 1) * n_weights(l), P)))
     return t
 

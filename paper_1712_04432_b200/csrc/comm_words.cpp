@@ -32,8 +32,10 @@ extern "C" mbd_status mbd_comm_words(const mbd_layer* layers, int L, int64_t B, 
     if (l.kind == MBD_CONV3X3) {
       if (l.C_in < 1 || l.C_out < 1 || l.H < 1 || l.W < 1 || l.kh < 1 || l.kw < 1) return MBD_E_INVALID;
       nW = static_cast<i128>(l.kh) * l.kw * l.C_in * l.C_out;      // Eq. 2
+      const int st = l.stride > 1 ? l.stride : 1;
+      if (l.H % st || l.W % st) return MBD_E_INVALID;
       din = static_cast<i128>(l.H) * l.W * l.C_in;
-      dout = static_cast<i128>(l.H) * l.W * l.C_out;
+      dout = static_cast<i128>(l.H / st) * (l.W / st) * l.C_out;      // a stride-s layer keeps every s-th position
     } else if (l.kind == MBD_FC) {
       if (l.d_in < 1 || l.d_out < 1) return MBD_E_INVALID;
       nW = static_cast<i128>(l.d_in) * l.d_out;
@@ -51,7 +53,7 @@ extern "C" mbd_status mbd_comm_words(const mbd_layer* layers, int L, int64_t B, 
       if (l.kind != MBD_CONV3X3) return MBD_E_INVALID;   // no halo notion for an FC layer
       if (P_r > 1) {
         ok = ok && ceil_div_to_i64(static_cast<i128>(B) * l.W * l.C_in * (l.kh / 2), P_c, &w.halo_fwd);
-        ok = ok && ceil_div_to_i64(static_cast<i128>(B) * l.W * l.C_out * (l.kh / 2), P_c, &w.halo_bwd);
+        ok = ok && ceil_div_to_i64(static_cast<i128>(B) * (l.W / (l.stride > 1 ? l.stride : 1)) * l.C_out * (l.kh / 2), P_c, &w.halo_bwd);   // Y_W
       }
       ok = ok && ceil_div_to_i64(static_cast<i128>(2) * (P - 1) * nW, P, &w.allreduce_dw);
     } else if (l.split == MBD_SPLIT_BATCH) {

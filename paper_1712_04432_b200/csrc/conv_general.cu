@@ -190,23 +190,51 @@ __global__ void pack_dw_kernel(const float* __restrict__ K, float* __restrict__ 
   }
 }
 
+// A strided layer (stride s) reads its input through s^2 phase planes: plane (a, b) holds the pixels (s h' + a, s w' + b)
+// of every strip in the geometry of the layer's OUTPUT (`go`), so that tap (u, v), with u - k_h/2 = s du + a and
+// v - k_w/2 = s dv + b, reads plane (a, b) at the output pixel shifted by (du, dv): the strided layer becomes a
+// stride-1 product over shifted views again, with no position computed that is not kept.
+// decimate: own pixels of T (geometry gi) -> planes P[s^2][go.Ptot][C]; undecimate: the way back (a gradient).
+__global__ void __launch_bounds__(256)
+decimate_kernel(const bf16* __restrict__ T, bf16* __restrict__ P, Geo gi, Geo go, int C, int s, int to_planes) {
+  const int c8 = C / 8;
+  const long long total = gi.Z * gi.Hs * gi.W * c8;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
+    const int cg = static_cast<int>(i % c8);
+    long long q = i / c8;
+    const int w = static_cast<int>(q % gi.W); q /= gi.W;
+    const int h = static_cast<int>(q % gi.Hs);
+    const long long z = q / gi.Hs;
+    const int a = h % s, b = w % s;
+    const long long pin = (z * gi.R + h + gi.ph) * gi.Wp + w + gi.pw;
+    const long long pout = (a * s + b) * go.Ptot + (z * go.R + h / s + go.ph) * go.Wp + w / s + go.pw;
+    if (to_planes) *reinterpret_cast<uint4*>(P + pout * C + cg * 8) = *reinterpret_cast<const uint4*>(T + pin * C + cg * 8);
+    else *reinterpret_cast<uint4*>(const_cast<bf16*>(T) + pin * C + cg * 8) = *reinterpret_cast<const uint4*>(P + pout * C + cg * 8);
+  }
+}
+
 int grid_1d(long long n, int num_sms) {
   const long long b = (n + 255) / 256;
   const long long cap = static_cast<long long>(num_sms) * 16;
   return static_cast<int>(std::max(1ll, std::min(b, cap)));
 }
 int round64(int c) { return (c + 63) / 64 * 64; }
+int floor_div(int a, int b) { return a >= 0 ? a / b : -((-a + b - 1) / b); }
 
 }  // namespace
 
 struct GenConv {
   int L = 0;
-  Geo g{};
-  int P = 1, S = 1;                       // processes of the grid; fp32 partial sums per weight gradient asked for
-  std::vector<int> Cin, Cout, kh, kw, relu, taps, Cp;
+  int64_t B = 0;
+  int P_r = 1, P = 1, S = 1;              // strips; processes of the grid; fp32 partial sums per weight gradient asked for
+  std::vector<Geo> geo;                   // geometry of tensor i (act[i]; dY[i] has that of act[i + 1])
+  std::vector<int> Cin, Cout, kh, kw, relu, taps, Cp, stride;
   std::vector<bf16*> act, dY, Wm;
+  std::vector<bf16*> xph, dxph;           // strided layers: phase planes of the input / of the gradient below
   std::vector<float*> dWm;
-  std::vector<TcGemm> fwd, bwd_data, bwd_weight;
+  std::vector<TcGemm> fwd, bwd_weight;
+  std::vector<std::vector<TcGemm>> bwd_data;   // one product (stride 1) or one per phase plane
+  std::vector<std::vector<int>> bwd_taps;      // taps of each of those products (an empty plane gets zeros)
   float* partials = nullptr;
   float* loss_part = nullptr;
   int loss_grid = 0;
@@ -252,17 +280,34 @@ mbd_status run(GenConv* c, TcGemm& t, int cls, double flops, const Epi& epi) {
   return MBD_OK;
 }
 
-void pad_fix(GenConv* c, bf16* T, int C, bool fill_halos) {
-  c->prof->begin(MBD_K_HALO, static_cast<double>(c->g.Ptot - static_cast<long long>(c->g.Z) * c->g.Hs * c->g.W) * C * 2.0, c->stream);
-  const long long chunks = c->g.Z * (2ll * c->g.ph * c->g.Wp + 2ll * c->g.Hs * c->g.pw) * (C / 8);
-  if (chunks > 0) pad_fix_kernel<<<grid_1d(chunks, c->num_sms), 256, 0, c->stream>>>(T, c->g, C, fill_halos ? 1 : 0);
+// `planes` > 1: the tensor is that many phase planes of geometry g, one after another (the strips of plane q are
+// strips q Z .. of the stack; Z is a multiple of P_r, so a strip's neighbours are in its own plane)
+void pad_fix(GenConv* c, bf16* T, Geo g, int C, bool fill_halos, int planes = 1) {
+  g.Z *= planes;
+  g.Ptot *= planes;
+  const long long chunks = g.Z * (2ll * g.ph * g.Wp + 2ll * g.Hs * g.pw) * (C / 8);
+  c->prof->begin(MBD_K_HALO, static_cast<double>(chunks) * 16.0, c->stream);
+  if (chunks > 0) pad_fix_kernel<<<grid_1d(chunks, c->num_sms), 256, 0, c->stream>>>(T, g, C, fill_halos ? 1 : 0);
   c->prof->end();
 }
 
-void set_shift(TcGemm& t, int mode, int taps, int blocks, int Cp, int kh, int kw, int Wp) {
-  t.cv.mode = mode; t.cv.taps = taps; t.cv.blocks = blocks; t.cv.Cp = Cp;
+void decimate(GenConv* c, const bf16* T, bf16* planes, const Geo& gi, const Geo& go, int C, int s, bool to_planes) {
+  const long long n = gi.Z * gi.Hs * gi.W * (C / 8);
+  c->prof->begin(MBD_K_HALO, static_cast<double>(n) * 32.0, c->stream);
+  decimate_kernel<<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(T, planes, gi, go, C, s, to_planes ? 1 : 0);
+  c->prof->end();
+}
+
+// Offsets of a layer's taps in pixel rows of the tensor its products read: stride 1: the input itself in geometry g;
+// stride s: the phase planes in the OUTPUT geometry g (plane start + shift inside the plane).
+void tap_offsets(int kh, int kw, int s, const Geo& g, int* off, int* plane) {
   for (int u = 0; u < kh; ++u)
-    for (int v = 0; v < kw; ++v) t.cv.off[u * kw + v] = (u - kh / 2) * Wp + (v - kw / 2);
+    for (int v = 0; v < kw; ++v) {
+      const int du = floor_div(u - kh / 2, s), dv = floor_div(v - kw / 2, s);
+      const int a = (u - kh / 2) - du * s, b = (v - kw / 2) - dv * s;
+      plane[u * kw + v] = a * s + b;
+      off[u * kw + v] = du * g.Wp + dv;
+    }
 }
 
 }  // namespace
@@ -272,7 +317,7 @@ bool gconv_needed(const mbd_layer* layers, int L) {
   for (int i = 0; i < L; ++i) {
     const mbd_layer& l = layers[i];
     const bool k3 = l.kh == 3 && l.kw == 3, k1 = l.kh == 1 && l.kw == 1;
-    if (!(k3 || k1) || l.C_in != 64 || l.C_out != 64) return true;
+    if (!(k3 || k1) || l.C_in != 64 || l.C_out != 64 || l.stride > 1) return true;
   }
   return false;
 }
@@ -283,6 +328,8 @@ void gconv_destroy(GenConv* c) {
   for (size_t i = 0; i < c->dY.size(); ++i)
     if (c->dY[i] && (c->act.size() <= static_cast<size_t>(c->L) || c->dY[i] != c->act[c->L])) cudaFree(c->dY[i]);
   for (bf16* p : c->Wm) cudaFree(p);
+  for (bf16* p : c->xph) cudaFree(p);
+  for (bf16* p : c->dxph) cudaFree(p);
   for (float* p : c->dWm) cudaFree(p);
   cudaFree(c->partials); cudaFree(c->loss_part);
   delete c;
@@ -291,25 +338,33 @@ void gconv_destroy(GenConv* c) {
 mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, int max_partials, int num_sms, int* status,
                         cudaStream_t stream, Profiler* prof, bool fc_above, GenConv** out) {
   if (tc_gemm_init() != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
-  const int H = layers[0].H, W = layers[0].W;
-  int ph = 0, pw = 0;
+  // one padding for every tensor: what the widest reach of any layer needs at the resolution it works in
+  int ph = 0, pw = 0, H = layers[0].H, W = layers[0].W;
   for (int i = 0; i < L; ++i) {
     const mbd_layer& l = layers[i];
-    if (l.kh < 1 || l.kw < 1 || l.kh > 7 || l.kw > 7 || l.kh % 2 == 0 || l.kw % 2 == 0) return MBD_E_UNSUPPORTED;
+    const int s = l.stride > 1 ? l.stride : 1;
+    if (l.kh < 1 || l.kw < 1 || l.kh > 7 || l.kw > 7 || l.kh % 2 == 0 || l.kw % 2 == 0 || s > 4) return MBD_E_UNSUPPORTED;
     if (l.C_in < 8 || l.C_out < 8 || l.C_in % 8 || l.C_out % 8) return MBD_E_UNSUPPORTED;       // 16-byte rows for TMA
     if (i > 0 && l.C_in != layers[i - 1].C_out) return MBD_E_INVALID;
-    ph = std::max(ph, l.kh / 2); pw = std::max(pw, l.kw / 2);
+    if (l.H != H || l.W != W || H % s || W % s) return MBD_E_INVALID;                            // sizes chain through the strides
+    if (H % P_r != 0 || (H / s) % P_r != 0) return MBD_E_UNSUPPORTED;                            // strips of equal height on this path
+    ph = std::max(ph, (l.kh / 2 + s - 1) / s); pw = std::max(pw, (l.kw / 2 + s - 1) / s);
+    H /= s; W /= s;
   }
-  if (H % P_r != 0) return MBD_E_UNSUPPORTED;            // strips of equal height on this path
-  const int Hs = H / P_r;
-  if (P_r > 1 && Hs < ph) return MBD_E_GRID;             // a halo row must come from the adjacent strip
   GenConv* c = new (std::nothrow) GenConv();
   if (!c) return MBD_E_ALLOC;
-  c->L = L; c->status = status; c->stream = stream; c->prof = prof; c->num_sms = num_sms; c->fc_above = fc_above;
-  Geo& g = c->g;
-  g.B = static_cast<int>(B); g.H = H; g.W = W; g.P_r = P_r; g.Hs = Hs; g.ph = ph; g.pw = pw;
-  g.R = Hs + 2 * ph; g.Wp = W + 2 * pw; g.Z = B * P_r; g.Ptot = g.Z * g.R * g.Wp;
-  if (B > INT32_MAX / std::max(1, P_r) || g.Ptot > INT32_MAX - 512) { delete c; return MBD_E_UNSUPPORTED; }   // TMA coordinates are 32-bit
+  c->L = L; c->B = B; c->P_r = P_r; c->status = status; c->stream = stream; c->prof = prof; c->num_sms = num_sms; c->fc_above = fc_above;
+  c->geo.resize(L + 1);
+  H = layers[0].H; W = layers[0].W;
+  for (int t = 0; t <= L; ++t) {
+    Geo& g = c->geo[t];
+    g.B = static_cast<int>(B); g.H = H; g.W = W; g.P_r = P_r; g.Hs = H / P_r; g.ph = ph; g.pw = pw;
+    g.R = g.Hs + 2 * ph; g.Wp = W + 2 * pw; g.Z = B * P_r; g.Ptot = g.Z * g.R * g.Wp;
+    if (P_r > 1 && g.Hs < ph) { delete c; return MBD_E_GRID; }             // a halo row must come from the adjacent strip
+    const int s = t < L && layers[t].stride > 1 ? layers[t].stride : 1;
+    if (B > INT32_MAX / std::max(1, P_r) || g.Ptot * s * s > INT32_MAX - 512) { delete c; return MBD_E_UNSUPPORTED; }   // TMA coordinates are 32-bit
+    if (t < L) { H /= s; W /= s; }
+  }
   c->P = P_r * P_c;
   c->S = max_partials < 1 ? 1 : std::min(c->P, max_partials);
   auto alloc = [&](void** p, size_t bytes) -> bool {
@@ -318,59 +373,86 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
   };
   bool ok = true;
   c->act.assign(L + 1, nullptr); c->dY.assign(L, nullptr); c->Wm.assign(L, nullptr); c->dWm.assign(L, nullptr);
-  c->fwd.resize(L); c->bwd_data.resize(L); c->bwd_weight.resize(L);
+  c->xph.assign(L, nullptr); c->dxph.assign(L, nullptr);
+  c->fwd.resize(L); c->bwd_data.resize(L); c->bwd_taps.resize(L); c->bwd_weight.resize(L);
   for (int i = 0; i < L; ++i) {
     const mbd_layer& l = layers[i];
     c->Cin.push_back(l.C_in); c->Cout.push_back(l.C_out); c->kh.push_back(l.kh); c->kw.push_back(l.kw);
+    c->stride.push_back(l.stride > 1 ? l.stride : 1);
     // the output of the last layer of a convolution-only network goes into the half-SSQ loss as it is
     c->relu.push_back((i == L - 1 && !fc_above) ? 0 : l.relu);
     c->taps.push_back(l.kh * l.kw); c->Cp.push_back(round64(l.C_in));
   }
-  // (a slack of one tile of rows behind every tensor is not needed: rows outside a tensor map read as zero)
   for (int i = 0; i <= L && ok; ++i) {
     const int C = i == 0 ? c->Cin[0] : c->Cout[i - 1];
-    ok = alloc(reinterpret_cast<void**>(&c->act[i]), static_cast<size_t>(g.Ptot) * C * 2);
+    ok = alloc(reinterpret_cast<void**>(&c->act[i]), static_cast<size_t>(c->geo[i].Ptot) * C * 2);
   }
   for (int i = 0; i < L && ok; ++i) {
-    if (i < L - 1 || fc_above) ok = alloc(reinterpret_cast<void**>(&c->dY[i]), static_cast<size_t>(g.Ptot) * c->Cout[i] * 2);
+    const Geo& go = c->geo[i + 1];
+    if (i < L - 1 || fc_above) ok = alloc(reinterpret_cast<void**>(&c->dY[i]), static_cast<size_t>(go.Ptot) * c->Cout[i] * 2);
     else c->dY[i] = c->act[L];                       // half-SSQ loss: dY_L = Y_L
     const size_t nw = static_cast<size_t>(c->Cout[i]) * c->taps[i] * c->Cp[i];
     ok = ok && alloc(reinterpret_cast<void**>(&c->Wm[i]), nw * 2) && alloc(reinterpret_cast<void**>(&c->dWm[i]), nw * 4);
+    if (c->stride[i] > 1) {
+      const size_t pl = static_cast<size_t>(c->stride[i]) * c->stride[i] * go.Ptot * c->Cin[i] * 2;
+      ok = ok && alloc(reinterpret_cast<void**>(&c->xph[i]), pl);
+      if (i > 0) ok = ok && alloc(reinterpret_cast<void**>(&c->dxph[i]), pl);
+    }
   }
   c->loss_grid = num_sms * 4;
   ok = ok && alloc(reinterpret_cast<void**>(&c->loss_part), sizeof(float) * c->loss_grid);
   if (!ok) { gconv_destroy(c); return MBD_E_ALLOC; }
   size_t part_elems = 0;
   for (int i = 0; i < L; ++i) {
-    const int Cin = c->Cin[i], Cout = c->Cout[i], taps = c->taps[i], Cp = c->Cp[i], Cop = round64(Cout);
+    const int Cin = c->Cin[i], Cout = c->Cout[i], taps = c->taps[i], Cp = c->Cp[i], Cop = round64(Cout), s = c->stride[i];
     const int ldw = taps * Cp;
+    const Geo& go = c->geo[i + 1];                   // the products run over the pixels of the layer's output geometry
+    const int M = static_cast<int>(go.Ptot);
+    bf16* xin = s > 1 ? c->xph[i] : c->act[i];       // what the forward and weight-gradient products read
+    int off[49], plane[49];
+    tap_offsets(c->kh[i], c->kw[i], s, go, off, plane);
     // forward
     TcGemm& f = c->fwd[i];
     f = TcGemm{};
-    f.variant = 0; f.M = static_cast<int>(g.Ptot); f.N = Cout; f.K = taps * Cp; f.k_splits = 1; f.status = status;
-    set_shift(f, 1, taps, Cp / 64, Cp, c->kh[i], c->kw[i], g.Wp);
-    f.cv_a_inner = Cin;
+    f.variant = 0; f.M = M; f.N = Cout; f.K = taps * Cp; f.k_splits = 1; f.status = status;
+    f.cv.mode = 1; f.cv.taps = taps; f.cv.blocks = Cp / 64; f.cv.Cp = Cp;
+    for (int t = 0; t < taps; ++t) { f.cv.off[t] = plane[t] * M + off[t]; f.cv.tap[t] = t; }
+    f.cv_a_inner = Cin; f.cv_a_rows = static_cast<int64_t>(s) * s * M;
     const Epi ef = make_epi_act(c->act[i + 1], Cout, 1, c->relu[i]);
-    if (tc_gemm_prepare(f, c->act[i], Cin, c->Wm[i], ldw, num_sms, &ef) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
-    // backward-data
+    if (tc_gemm_prepare(f, xin, Cin, c->Wm[i], ldw, num_sms, &ef) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
+    // backward-data: one product (stride 1), or one per phase plane with the taps that read that plane
     if (i > 0) {
-      TcGemm& d = c->bwd_data[i];
-      d = TcGemm{};
-      d.variant = 1; d.M = static_cast<int>(g.Ptot); d.N = Cin; d.K = taps * Cop; d.k_splits = 1; d.status = status;
-      set_shift(d, 2, taps, Cop / 64, Cp, c->kh[i], c->kw[i], g.Wp);
-      d.cv_a_inner = Cout; d.cv_b_inner = ldw; d.cv_b_rows = Cout;
-      const Epi ed = make_epi_mask(c->dY[i - 1], Cin, c->relu[i - 1] ? c->act[i] : nullptr, Cin);
-      if (tc_gemm_prepare(d, c->dY[i], Cout, c->Wm[i], ldw, num_sms, &ed) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
+      c->bwd_data[i].resize(s * s);
+      c->bwd_taps[i].assign(s * s, 0);
+      for (int q = 0; q < s * s; ++q) {
+        TcGemm& d = c->bwd_data[i][q];
+        d = TcGemm{};
+        d.variant = 1; d.M = M; d.N = Cin; d.k_splits = 1; d.status = status;
+        d.cv.mode = 2; d.cv.blocks = Cop / 64; d.cv.Cp = Cp;
+        int n = 0;
+        for (int t = 0; t < taps; ++t)
+          if (plane[t] == q) { d.cv.off[n] = off[t]; d.cv.tap[n] = t; ++n; }
+        d.cv.taps = n;
+        c->bwd_taps[i][q] = n;
+        if (n == 0) continue;                          // no tap reads this plane: its gradient is zero
+        d.K = n * Cop;
+        d.cv_a_inner = Cout; d.cv_b_inner = ldw; d.cv_b_rows = Cout;
+        bf16* outp = s > 1 ? c->dxph[i] + static_cast<size_t>(q) * M * Cin : c->dY[i - 1];
+        const bf16* maskp = !c->relu[i - 1] ? nullptr : (s > 1 ? c->xph[i] + static_cast<size_t>(q) * M * Cin : c->act[i]);
+        const Epi ed = make_epi_mask(outp, Cin, maskp, Cin);
+        if (tc_gemm_prepare(d, c->dY[i], Cout, c->Wm[i], ldw, num_sms, &ed) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
+      }
     }
     // backward-weight: few output tiles, a very long K (all pixels): the planner cuts K to fill the SMs
     TcGemm& w = c->bwd_weight[i];
     w = TcGemm{};
-    w.variant = 2; w.M = Cout; w.N = ldw; w.K = static_cast<int>(g.Ptot); w.k_splits = c->S; w.status = status;
+    w.variant = 2; w.M = Cout; w.N = ldw; w.K = M; w.k_splits = c->S; w.status = status;
     w.allow_extra_split = 1;
-    set_shift(w, 3, taps, 0, Cp, c->kh[i], c->kw[i], g.Wp);
-    w.cv_b_inner = Cin; w.cv_b_rows = g.Ptot;
+    w.cv.mode = 3; w.cv.taps = taps; w.cv.blocks = 0; w.cv.Cp = Cp;
+    for (int t = 0; t < taps; ++t) { w.cv.off[t] = plane[t] * M + off[t]; w.cv.tap[t] = t; }
+    w.cv_b_inner = Cin; w.cv_b_rows = static_cast<int64_t>(s) * s * M;
     const Epi ew = make_epi_sgd(c->Wm[i], ldw, 0.f);
-    if (tc_gemm_prepare(w, c->dY[i], Cout, c->act[i], Cin, num_sms, &ew) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
+    if (tc_gemm_prepare(w, c->dY[i], Cout, xin, Cin, num_sms, &ew) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
     if (w.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(w.k_splits) * Cout * ldw);
   }
   if (part_elems && !alloc(reinterpret_cast<void**>(&c->partials), part_elems * 4)) { gconv_destroy(c); return MBD_E_ALLOC; }
@@ -379,7 +461,7 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
   return MBD_OK;
 }
 
-size_t gconv_input_bytes(const GenConv* c) { return static_cast<size_t>(c->g.B) * c->Cin[0] * c->g.H * c->g.W * 2; }
+size_t gconv_input_bytes(const GenConv* c) { return static_cast<size_t>(c->B) * c->Cin[0] * c->geo[0].H * c->geo[0].W * 2; }
 int gconv_last_relu(const GenConv* c) { return c->relu[c->L - 1]; }
 
 mbd_status gconv_set_weights(GenConv* c, int i, const void* K_dev) {
@@ -394,38 +476,45 @@ mbd_status gconv_get_weights(GenConv* c, int i, void* K_dev) {
 }
 
 namespace {
-void stage(GenConv* c, const bf16* nchw, bf16* dst, int C, bool fill_halos) {
-  const dim3 grid(static_cast<unsigned>(c->g.B) * c->g.H, (c->g.W + 31) / 32, (C + 63) / 64);
-  c->prof->begin(MBD_K_HALO, 2.0 * c->g.B * C * c->g.H * c->g.W * 2.0, c->stream);
-  nchw_to_pix_kernel<<<grid, 256, 0, c->stream>>>(nchw, dst, c->g, C);
+void stage(GenConv* c, const bf16* nchw, bf16* dst, const Geo& g, int C, bool fill_halos) {
+  const dim3 grid(static_cast<unsigned>(g.B) * g.H, (g.W + 31) / 32, (C + 63) / 64);
+  c->prof->begin(MBD_K_HALO, 2.0 * g.B * C * g.H * g.W * 2.0, c->stream);
+  nchw_to_pix_kernel<<<grid, 256, 0, c->stream>>>(nchw, dst, g, C);
   c->prof->end();
-  pad_fix(c, dst, C, fill_halos);
+  pad_fix(c, dst, g, C, fill_halos);
 }
-void unstage(GenConv* c, const bf16* src, bf16* nchw, int C) {
-  const dim3 grid(static_cast<unsigned>(c->g.B) * c->g.H, (c->g.W + 31) / 32, (C + 63) / 64);
-  c->prof->begin(MBD_K_HALO, 2.0 * c->g.B * C * c->g.H * c->g.W * 2.0, c->stream);
-  pix_to_nchw_kernel<<<grid, 256, 0, c->stream>>>(src, nchw, c->g, C);
+void unstage(GenConv* c, const bf16* src, bf16* nchw, const Geo& g, int C) {
+  const dim3 grid(static_cast<unsigned>(g.B) * g.H, (g.W + 31) / 32, (C + 63) / 64);
+  c->prof->begin(MBD_K_HALO, 2.0 * g.B * C * g.H * g.W * 2.0, c->stream);
+  pix_to_nchw_kernel<<<grid, 256, 0, c->stream>>>(src, nchw, g, C);
   c->prof->end();
 }
 }  // namespace
 
 mbd_status gconv_stage_input(GenConv* c, const void* X_nchw) {
-  stage(c, static_cast<const bf16*>(X_nchw), c->act[0], c->Cin[0], true);     // the forward halo exchange of the input rides along
+  stage(c, static_cast<const bf16*>(X_nchw), c->act[0], c->geo[0], c->Cin[0], true);     // the forward halo exchange of the input rides along
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
 mbd_status gconv_forward_layer(GenConv* c, int i, float* loss_sum_dev) {
   if (i < 0 || i >= c->L) return MBD_E_INVALID;
   const bool last = i == c->L - 1;
-  const double flops = 2.0 * c->g.B * c->g.H * c->g.W * c->taps[i] * c->Cin[i] * c->Cout[i];     // the method's flops
+  const Geo& go = c->geo[i + 1];
+  const int s = c->stride[i];
+  const double flops = 2.0 * c->B * go.H * go.W * c->taps[i] * c->Cin[i] * c->Cout[i];     // the method's flops
+  if (s > 1) {
+    // the input's own pixels sorted into the s^2 phase planes; their halo rows exchanged plane by plane
+    decimate(c, c->act[i], c->xph[i], c->geo[i], go, c->Cin[i], s, true);
+    pad_fix(c, c->xph[i], go, c->Cin[i], true, s * s);
+  }
   const Epi e = make_epi_act(c->act[i + 1], c->Cout[i], 1, c->relu[i]);
-  mbd_status s = run(c, c->fwd[i], MBD_K_CONV_FWD, flops, e);
-  if (s != MBD_OK) return s;
+  mbd_status st = run(c, c->fwd[i], MBD_K_CONV_FWD, flops, e);
+  if (st != MBD_OK) return st;
   // the output's halo exchange for the next layer (first halo term of Eq. 7); the last output is the top gradient of
   // the half-SSQ loss and enters the weight-gradient sum: zeros outside the strips' own pixels
-  pad_fix(c, c->act[i + 1], c->Cout[i], !last);
+  pad_fix(c, c->act[i + 1], go, c->Cout[i], !last);
   if (last && loss_sum_dev && !c->fc_above) {
-    const long long n8 = c->g.Ptot * c->Cout[i] / 8;
+    const long long n8 = go.Ptot * c->Cout[i] / 8;
     c->prof->begin(MBD_K_OTHER, static_cast<double>(n8) * 16.0, c->stream);
     ssq_partial_kernel<<<c->loss_grid, 256, 0, c->stream>>>(c->act[i + 1], n8, c->loss_part);
     if (sum_f32_launch(c->loss_part, c->loss_grid, 0.5f, loss_sum_dev, c->stream) != cudaSuccess) return MBD_E_CUDA;
@@ -443,24 +532,35 @@ mbd_status gconv_forward(GenConv* c, const void* X_nchw, float* loss_sum_dev) {
 mbd_status gconv_backward_layer(GenConv* c, int i, float fused_eta) {
   if (i < 0 || i >= c->L) return MBD_E_INVALID;
   const bool fused = fused_eta > 0.f;
-  const float scale = -fused_eta / static_cast<float>(c->g.B);
-  const double flops = 2.0 * c->g.B * c->g.H * c->g.W * c->taps[i] * c->Cin[i] * c->Cout[i];
+  const float scale = -fused_eta / static_cast<float>(c->B);
+  const Geo& go = c->geo[i + 1];
+  const int s = c->stride[i], Cin = c->Cin[i];
+  const double flops = 2.0 * c->B * go.H * go.W * c->taps[i] * Cin * c->Cout[i];
   const int ldw = c->taps[i] * c->Cp[i];
   if (i > 0) {
     // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0] -- with the
     // weights as they are BEFORE this step's update, so this product comes first
-    if (c->g.P_r > 1) pad_fix(c, c->dY[i], c->Cout[i], true);
-    const Epi ed = make_epi_mask(c->dY[i - 1], c->Cin[i], c->relu[i - 1] ? c->act[i] : nullptr, c->Cin[i]);
-    mbd_status s = run(c, c->bwd_data[i], MBD_K_CONV_BWD_DATA, flops, ed);
-    if (s != MBD_OK) return s;
-    pad_fix(c, c->dY[i - 1], c->Cin[i], false);
-    if (c->g.P_r > 1) pad_fix(c, c->dY[i], c->Cout[i], false);      // the halo copies must not enter the sum below
+    if (c->P_r > 1) pad_fix(c, c->dY[i], go, c->Cout[i], true);
+    for (int q = 0; q < s * s; ++q) {
+      bf16* outp = s > 1 ? c->dxph[i] + static_cast<size_t>(q) * go.Ptot * Cin : c->dY[i - 1];
+      if (c->bwd_taps[i][q] == 0) {                // (a 1 x 1 kernel with stride 2: three of four planes)
+        if (cudaMemsetAsync(outp, 0, static_cast<size_t>(go.Ptot) * Cin * 2, c->stream) != cudaSuccess) return MBD_E_CUDA;
+        continue;
+      }
+      const bf16* maskp = !c->relu[i - 1] ? nullptr : (s > 1 ? c->xph[i] + static_cast<size_t>(q) * go.Ptot * Cin : c->act[i]);
+      const Epi ed = make_epi_mask(outp, Cin, maskp, Cin);
+      const mbd_status st = run(c, c->bwd_data[i][q], MBD_K_CONV_BWD_DATA, flops * c->bwd_taps[i][q] / c->taps[i], ed);
+      if (st != MBD_OK) return st;
+    }
+    if (s > 1) decimate(c, c->dY[i - 1], c->dxph[i], c->geo[i], go, Cin, s, false);      // the planes' own pixels back in place
+    pad_fix(c, c->dY[i - 1], c->geo[i], Cin, false);
+    if (c->P_r > 1) pad_fix(c, c->dY[i], go, c->Cout[i], false);      // the halo copies must not enter the sum below
   }
   // dY_i is zero outside the strips' own pixels here: every pixel enters the weight gradient once (the sum over the
   // strips and batch blocks is the all-reduce over all P processes, last term of Eq. 9)
   const Epi ew = fused ? make_epi_sgd(c->Wm[i], ldw, scale) : make_epi_act(c->dWm[i], ldw, 0, 0);
-  const mbd_status s = run(c, c->bwd_weight[i], MBD_K_CONV_BWD_WEIGHT, flops, ew);
-  if (s != MBD_OK) return s;
+  const mbd_status st = run(c, c->bwd_weight[i], MBD_K_CONV_BWD_WEIGHT, flops, ew);
+  if (st != MBD_OK) return st;
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
@@ -471,7 +571,7 @@ mbd_status gconv_backward(GenConv* c, float fused_eta) {
 }
 
 mbd_status gconv_sgd_step(GenConv* c, float eta) {
-  const float scale = -eta / static_cast<float>(c->g.B);
+  const float scale = -eta / static_cast<float>(c->B);
   for (int i = 0; i < c->L; ++i) {
     const long long n = static_cast<long long>(c->Cout[i]) * c->taps[i] * c->Cp[i];
     c->prof->begin(MBD_K_SGD, static_cast<double>(n) * 8.0, c->stream);
@@ -482,13 +582,13 @@ mbd_status gconv_sgd_step(GenConv* c, float eta) {
 }
 
 mbd_status gconv_output_to_nchw(GenConv* c, void* dst) {
-  unstage(c, c->act[c->L], static_cast<bf16*>(dst), c->Cout[c->L - 1]);
+  unstage(c, c->act[c->L], static_cast<bf16*>(dst), c->geo[c->L], c->Cout[c->L - 1]);
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
 mbd_status gconv_top_grad_from_nchw(GenConv* c, const void* src) {
   if (!c->fc_above) return MBD_E_STATE;
-  stage(c, static_cast<const bf16*>(src), c->dY[c->L - 1], c->Cout[c->L - 1], false);
+  stage(c, static_cast<const bf16*>(src), c->dY[c->L - 1], c->geo[c->L], c->Cout[c->L - 1], false);
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
@@ -503,16 +603,25 @@ mbd_status gconv_get_tensor(GenConv* c, int which, int layer, void* dst, size_t 
   }
   if (which != MBD_T_ACT && which != MBD_T_DY) return MBD_E_INVALID;
   const int C = c->Cout[layer];
-  if (bytes != static_cast<size_t>(c->g.B) * C * c->g.H * c->g.W * 2) return MBD_E_INVALID;
-  unstage(c, which == MBD_T_ACT ? c->act[layer + 1] : c->dY[layer], static_cast<bf16*>(dst), C);
+  const Geo& g = c->geo[layer + 1];
+  if (bytes != static_cast<size_t>(c->B) * C * g.H * g.W * 2) return MBD_E_INVALID;
+  unstage(c, which == MBD_T_ACT ? c->act[layer + 1] : c->dY[layer], static_cast<bf16*>(dst), g, C);
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
 mbd_status gconv_set_tensor(GenConv* c, int which, int layer, const void* src, size_t bytes) {
   if (layer < 0 || layer >= c->L || which != MBD_T_ACT) return MBD_E_INVALID;
   const int C = c->Cout[layer];
-  if (bytes != static_cast<size_t>(c->g.B) * C * c->g.H * c->g.W * 2) return MBD_E_INVALID;
-  stage(c, static_cast<const bf16*>(src), c->act[layer + 1], C, layer + 1 < c->L);
+  const Geo& g = c->geo[layer + 1];
+  if (bytes != static_cast<size_t>(c->B) * C * g.H * g.W * 2) return MBD_E_INVALID;
+  stage(c, static_cast<const bf16*>(src), c->act[layer + 1], g, C, layer + 1 < c->L);
+  // a strided layer above reads its phase planes, made from this tensor in its forward pass: refresh them, so that
+  // the ReLU decisions of the backward pass are taken on what was just stored
+  if (layer + 1 < c->L && c->stride[layer + 1] > 1) {
+    const int s = c->stride[layer + 1];
+    decimate(c, c->act[layer + 1], c->xph[layer + 1], g, c->geo[layer + 2], C, s, true);
+    pad_fix(c, c->xph[layer + 1], c->geo[layer + 2], C, true, s * s);
+  }
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 

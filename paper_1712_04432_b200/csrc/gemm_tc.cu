@@ -334,7 +334,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               load(sb, &tmB, kb * BK, col0);
             } else {
 #pragma unroll
-              for (int c = 0; c < BNL / 64; ++c) load(sb + c * (64 * BK * 2), &tmB, t * p.cv.Cp + col0 + c * 64, cb * 64);
+              for (int c = 0; c < BNL / 64; ++c) load(sb + c * (64 * BK * 2), &tmB, p.cv.tap[t] * p.cv.Cp + col0 + c * 64, cb * 64);
             }
           } else {
             // convolution, backward-weight: K = pixels; an output column chunk = (tap, 64 input channels)
@@ -1084,7 +1084,7 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
   }
   const bool a_mn = g.variant == 2, b_mn = g.variant >= 1;
   if (g.cv.mode != 0 && g.cv.mode != g.variant + 1) return cudaErrorInvalidValue;
-  if (!a_mn) e = make_map(&g.tmA, A, g.cv.mode ? g.cv_a_inner : g.K, g.M, lda, BK, BM * g.MH);   // A[M,K]: inner = K; box = the rows one CTA loads
+  if (!a_mn) e = make_map(&g.tmA, A, g.cv.mode ? g.cv_a_inner : g.K, g.cv.mode && g.cv_a_rows ? g.cv_a_rows : g.M, lda, BK, BM * g.MH);   // A[M,K]: inner = K; box = the rows one CTA loads
   else e = make_map(&g.tmA, A, g.M, g.K, lda, 64, BK);             // A[K,M]: inner = M, one 64-wide chunk per box
   if (e != cudaSuccess) return e;
   if (!b_mn) e = make_map(&g.tmB, B, g.K, g.N, ldb, BK, g.pair ? g.BN / 2 : g.BN);    // B[N,K]

@@ -95,9 +95,13 @@ struct Epi {
 // output channel); A tile at row m0 - off[t]; the B tile is rows 64 ob.. of the weight matrix [C_out][taps Cp] at
 // column t Cp + n0.  mode 3 (backward-weight, variant 2): K = pixels; the B chunk of output columns n0.. = (tap t,
 // channels n0 - t Cp ..) starts at pixel row k0 + off[t].  Rows outside the tensor read as zero (TMA fill).
+// A strided layer reads phase-decimated copies of its input stored one after another (plane (a, b) holds the pixels
+// (s h' + a, s w' + b)): its offsets then include the plane's start, and backward-data runs once per plane with the
+// taps that read it -- `tap[j]` is the position in the weight matrix of the j-th tap of such a subset.
 struct ConvShift {
   int mode, taps, blocks, Cp;      // blocks: 64-wide k-blocks per tap (modes 1, 2)
   int off[49];
+  int tap[49];                     // mode 2: weight-matrix tap of the j-th tap of this product (identity for stride 1)
 };
 
 struct TcGemm {
@@ -131,6 +135,7 @@ struct TcGemm {
   // Convolution as a contraction over shifted views (set before tc_gemm_prepare; cv.mode = 0: a plain product)
   ConvShift cv = {};
   int64_t cv_a_inner = 0;      // modes 1, 2: channels per pixel of the A tensor (its rows are pixels)
+  int64_t cv_a_rows = 0;       // modes 1, 2: rows of the A tensor as stored, if more than M (phase planes); 0 = M
   int64_t cv_b_inner = 0, cv_b_rows = 0;   // modes 2, 3: extent of the B tensor as stored (inner, rows)
 };
 

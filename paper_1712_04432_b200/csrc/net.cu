@@ -300,7 +300,11 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
       if (l.d_in < 1 || l.d_out < 1) return MBD_E_INVALID;
       if (l.split != MBD_SPLIT_MODEL) return MBD_E_INVALID;
       if (i > Lc && l.d_in != layers[i - 1].d_out) return MBD_E_INVALID;
-      if (i == Lc && mixed && l.d_in != static_cast<int64_t>(layers[Lc - 1].C_out) * layers[0].H * layers[0].W) return MBD_E_INVALID;
+      if (i == Lc && mixed) {
+        const mbd_layer& lc = layers[Lc - 1];
+        const int st = lc.stride > 1 ? lc.stride : 1;
+        if (l.d_in != static_cast<int64_t>(lc.C_out) * (lc.H / st) * (lc.W / st)) return MBD_E_INVALID;
+      }
       if (P_r > l.d_out) return MBD_E_GRID;
       if (dtype == MBD_BF16 && (l.d_in % 8 || l.d_out % 8)) return MBD_E_UNSUPPORTED;
       if (l.d_in > INT32_MAX || l.d_out > INT32_MAX || B > INT32_MAX) return MBD_E_UNSUPPORTED;
@@ -316,7 +320,13 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
       } else if (l.H < 1 || l.W < 1 || P_r > l.H || (P_r > 1 && l.H / P_r < l.kh / 2)) {
         return MBD_E_GRID;   // a strip needs >= 1 row, and its halo rows come from the adjacent strip only
       }
-      if (i > 0 && (l.H != layers[0].H || l.W != layers[0].W)) return MBD_E_INVALID;
+      const int st = l.stride > 1 ? l.stride : 1;
+      if (st > 4 || l.H % st || l.W % st) return l.stride > 4 ? MBD_E_UNSUPPORTED : MBD_E_INVALID;
+      if (i > 0) {                                                       // the image sizes chain through the strides
+        const int ps = layers[i - 1].stride > 1 ? layers[i - 1].stride : 1;
+        if (l.H != layers[i - 1].H / ps || l.W != layers[i - 1].W / ps) return MBD_E_INVALID;
+      }
+      if (l.split == MBD_SPLIT_DOMAIN && P_r > l.H / st) return MBD_E_GRID;
     } else {
       return MBD_E_INVALID;
     }

@@ -27,7 +27,8 @@ bool layer_dims(const mbd_layer& l, Dims* d) {
     if (l.C_in < 1 || l.C_out < 1 || l.H < 1 || l.W < 1 || l.kh < 1 || l.kw < 1) return false;
     d->nW = static_cast<double>(l.kh) * l.kw * l.C_in * l.C_out;      // Eq. 2
     d->din = static_cast<double>(l.H) * l.W * l.C_in;
-    d->dout = static_cast<double>(l.H) * l.W * l.C_out;
+    const int st = l.stride > 1 ? l.stride : 1;                      // a stride-s layer keeps every s-th position
+    d->dout = static_cast<double>(l.H / st) * (l.W / st) * l.C_out;
     d->conv = true;
     return true;
   }
@@ -61,7 +62,7 @@ mbd_status layer_row(const mbd_layer& l, int split, bool first, double B, int P_
     if (P_r > 1 && l.kh / 2 > 0) {         // a 1 x 1 convolution exchanges nothing (remark after Eq. 7)
       const double rows = static_cast<double>(l.kh / 2);
       t->halo_fwd = m.alpha + m.beta * (B / pc) * l.W * l.C_in * rows;
-      t->halo_bwd = m.alpha + m.beta * (B / pc) * l.W * l.C_out * rows;
+      t->halo_bwd = m.alpha + m.beta * (B / pc) * (l.W / (l.stride > 1 ? l.stride : 1)) * l.C_out * rows;     // Y_W
     }
     t->allreduce_dw = 2.0 * (m.alpha * ceil_log2(static_cast<long long>(P_r) * P_c) + m.beta * ((P - 1.0) / P) * d.nW);
     return MBD_OK;
@@ -77,7 +78,8 @@ bool feasible(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, bool 
     const mbd_layer& l = layers[i];
     if (fc_only && l.kind != MBD_FC) continue;
     if (l.split == MBD_SPLIT_MODEL) {
-      const double dout = l.kind == MBD_FC ? static_cast<double>(l.d_out) : static_cast<double>(l.H) * l.W * l.C_out;
+      const int st = l.stride > 1 ? l.stride : 1;
+      const double dout = l.kind == MBD_FC ? static_cast<double>(l.d_out) : static_cast<double>(l.H / st) * (l.W / st) * l.C_out;
       if (static_cast<double>(P_r) > dout) return false;
     } else if (l.split == MBD_SPLIT_BATCH) {
       if (static_cast<int64_t>(P_r) * P_c > B) return false;

@@ -57,6 +57,7 @@ class Workload:
     fc_dims: Tuple[int, ...] = ()  # mixed: C*H*W -> ... -> classes above the n_layers convolutions
     ksizes: Tuple = ()             # conv, mixed: kernel size per convolution, k or (k_h, k_w); empty = all 3 x 3
     channels: Tuple[int, ...] = () # conv: C_0 .. C_L (layer i maps C_{i-1} -> C_i); empty = dims[0] everywhere
+    strides: Tuple[int, ...] = ()  # conv: stride per layer; empty = 1 everywhere
 
     def ksize(self, i: int) -> int:
         k = self.ksizes[i] if self.ksizes else 3
@@ -66,6 +67,16 @@ class Workload:
     def kshape(self, i: int) -> Tuple[int, int]:
         k = self.ksizes[i] if self.ksizes else 3
         return (k, k) if isinstance(k, int) else (int(k[0]), int(k[1]))
+
+    def stride(self, i: int) -> int:
+        return self.strides[i] if self.strides else 1
+
+    def out_hw(self, i: int) -> Tuple[int, int]:
+        """Output image size of convolution layer i (dims[1:] is the network input's)."""
+        H, W = self.dims[1], self.dims[2]
+        for j in range(i + 1):
+            H, W = H // self.stride(j), W // self.stride(j)
+        return H, W
 
     def chan(self, i: int) -> int:
         """Channels of tensor i (0 = the input)."""
@@ -95,14 +106,21 @@ WORKLOADS = {
 # 64 -> 128 -> 128 channels, 112 x 112 images), for measuring the general convolution path.
 WORKLOADS["conv5x5"] = Workload("conv5x5", "conv", (64, 112, 112), 32, "bf16", "normal", "half_ssq", eta=1e-7, n_layers=2,
                                 grids=[(1, 1), (2, 1), (4, 1), (8, 1)], ksizes=((5, 5), (3, 3)), channels=(64, 128, 128))
+# The same two layers on 224 x 224 inputs, the first with stride 2 (its output is the 112 x 112 image of conv5x5).
+WORKLOADS["conv5x5s2"] = Workload("conv5x5s2", "conv", (64, 224, 224), 32, "bf16", "normal", "half_ssq", eta=1e-7, n_layers=2,
+                                  grids=[(1, 1), (2, 1), (4, 1), (8, 1)], ksizes=((5, 5), (3, 3)), channels=(64, 128, 128),
+                                  strides=(2, 1))
 
 
-def mixed_workload(C, H, W, n_conv, fc_dims, B, name="custom_mixed", grids=(), ksizes=()) -> "Workload":
-    """n_conv 3x3 convolutions C -> C on H x W images, then a fully connected stack
-    C*H*W -> fc_dims[0] -> ... -> fc_dims[-1] with softmax cross-entropy."""
-    d = (int(C) * int(H) * int(W),) + tuple(int(x) for x in fc_dims)
-    return Workload(name, "mixed", (int(C), int(H), int(W)), int(B), "bf16", "normal", "softmax_ce",
-                    n_layers=int(n_conv), grids=list(grids), fc_dims=d, ksizes=tuple(ksizes))
+def mixed_workload(C, H, W, n_conv, fc_dims, B, name="custom_mixed", grids=(), ksizes=(), channels=(), strides=()) -> "Workload":
+    """n_conv convolutions (3x3, C -> C unless ksizes / channels / strides say otherwise) on H x W images, then a fully
+    connected stack C_L*H_L*W_L -> fc_dims[0] -> ... -> fc_dims[-1] with softmax cross-entropy."""
+    w = Workload(name, "mixed", (int(C), int(H), int(W)), int(B), "bf16", "normal", "softmax_ce",
+                 n_layers=int(n_conv), grids=list(grids), ksizes=tuple(ksizes), channels=tuple(int(c) for c in channels),
+                 strides=tuple(int(s) for s in strides))
+    Ho, Wo = w.out_hw(int(n_conv) - 1)
+    w.fc_dims = (w.chan(int(n_conv)) * Ho * Wo,) + tuple(int(x) for x in fc_dims)
+    return w
 
 
 # Beyond the five configurations: the integrated network of Section 2.4 in miniature (convolutions on
@@ -120,12 +138,13 @@ def fc_workload(dims, B, dtype="bf16", x_dist="normal", name="custom") -> Worklo
     return Workload(name, "fc", tuple(int(d) for d in dims), int(B), dtype, x_dist, "softmax_ce")
 
 
-def conv_workload(C, H, W, B, n_layers=2, dtype="bf16", name="custom_conv", ksizes=(), channels=()) -> Workload:
+def conv_workload(C, H, W, B, n_layers=2, dtype="bf16", name="custom_conv", ksizes=(), channels=(), strides=()) -> Workload:
     """`channels` = (C_0, .., C_L) for layers that change the channel count (then C = C_0)."""
     if channels:
         assert len(channels) == n_layers + 1 and channels[0] == C
     return Workload(name, "conv", (int(C), int(H), int(W)), int(B), dtype, "normal",
-                    "half_ssq", n_layers=n_layers, ksizes=tuple(ksizes), channels=tuple(int(c) for c in channels))
+                    "half_ssq", n_layers=n_layers, ksizes=tuple(ksizes), channels=tuple(int(c) for c in channels),
+                    strides=tuple(int(s) for s in strides))
 
 
 @dataclass
@@ -190,7 +209,7 @@ def step_flops(w: Workload) -> int:
     C, H, Wd = w.dims
     macs = 0
     for i in range(w.n_layers):
-        per = w.B * H * Wd * w.chan(i) * w.chan(i + 1) * w.kshape(i)[0] * w.kshape(i)[1]
+        per = w.B * w.out_hw(i)[0] * w.out_hw(i)[1] * w.chan(i) * w.chan(i + 1) * w.kshape(i)[0] * w.kshape(i)[1]
         macs += (3 if i >= 1 else 2) * per
     if w.kind == "mixed":
         d = w.fc_dims

@@ -44,7 +44,7 @@ class Layer(C.Structure):
     _fields_ = [("kind", C.c_int32), ("split", C.c_int32), ("relu", C.c_int32), ("bias", C.c_int32),
                 ("d_in", C.c_int64), ("d_out", C.c_int64),
                 ("C_in", C.c_int32), ("C_out", C.c_int32), ("H", C.c_int32), ("W", C.c_int32),
-                ("kh", C.c_int32), ("kw", C.c_int32)]
+                ("kh", C.c_int32), ("kw", C.c_int32), ("stride", C.c_int32), ("reserved", C.c_int32)]
 
 
 TAIL_STORE, TAIL_MASK, TAIL_SGD = range(3)
@@ -165,17 +165,26 @@ def fc_layers(dims: Sequence[int], bias: bool = True, relu: bool = True) -> List
                   d_out=int(dims[i])) for i in range(1, len(dims))]
 
 
-def conv_layers(n: int, C_: int, H: int, W: int, relu: bool = True, k=3, split: int = SPLIT_DOMAIN, channels=()) -> List[Layer]:
-    """n convolution layers on H x W images, domain-split (row strips) or, with split=SPLIT_BATCH,
+def conv_layers(n: int, C_: int, H: int, W: int, relu: bool = True, k=3, split: int = SPLIT_DOMAIN, channels=(),
+                strides=()) -> List[Layer]:
+    """n convolution layers on H x W input images, domain-split (row strips) or, with split=SPLIT_BATCH,
     batch-parallel on 1 x P (Section 3's improved case); `k` is the kernel size, k or (k_h, k_w), one value for all
-    layers or one per layer; `channels` = (C_0, .., C_n) when the layers change the channel count (else C -> C)."""
+    layers or one per layer; `channels` = (C_0, .., C_n) when the layers change the channel count (else C -> C);
+    `strides` = one stride per layer (default 1): layer i then maps H_i x W_i images to H_i/s x W_i/s ones."""
     ks = [k] * n if isinstance(k, (int, tuple)) else list(k)
     assert len(ks) == n
     ks = [(q, q) if isinstance(q, int) else (int(q[0]), int(q[1])) for q in ks]
     ch = list(channels) if channels else [C_] * (n + 1)
-    assert len(ch) == n + 1
-    return [Layer(kind=CONV3X3, split=split, relu=int(relu), bias=0, d_in=ch[i] * H * W, d_out=ch[i + 1] * H * W,
-                  C_in=ch[i], C_out=ch[i + 1], H=H, W=W, kh=ks[i][0], kw=ks[i][1]) for i in range(n)]
+    st = list(strides) if strides else [1] * n
+    assert len(ch) == n + 1 and len(st) == n
+    out = []
+    for i in range(n):
+        assert H % st[i] == 0 and W % st[i] == 0
+        Ho, Wo = H // st[i], W // st[i]
+        out.append(Layer(kind=CONV3X3, split=split, relu=int(relu), bias=0, d_in=ch[i] * H * W, d_out=ch[i + 1] * Ho * Wo,
+                         C_in=ch[i], C_out=ch[i + 1], H=H, W=W, kh=ks[i][0], kw=ks[i][1], stride=st[i]))
+        H, W = Ho, Wo
+    return out
 
 
 def _layer_array(layers: Sequence[Layer]):
@@ -377,10 +386,10 @@ class Net:
         last = layer == self.L - 1
         conv = l.kind == CONV3X3
         if which == T_ACT:
-            shape, dt = ((self.B, l.C_out, l.H, l.W) if conv else (self.B, l.d_out)), \
+            shape, dt = ((self.B, l.C_out, l.H // max(1, l.stride), l.W // max(1, l.stride)) if conv else (self.B, l.d_out)), \
                 (t.float32 if (last and not conv) else self.act_dtype)
         elif which == T_DY:
-            shape, dt = ((self.B, l.C_out, l.H, l.W) if conv else (self.B, l.d_out)), self.act_dtype
+            shape, dt = ((self.B, l.C_out, l.H // max(1, l.stride), l.W // max(1, l.stride)) if conv else (self.B, l.d_out)), self.act_dtype
         elif which in (T_DW, T_MASTER, T_VELOCITY):
             shape, dt = self._wshape(layer), t.float32
         elif which in (T_DB, T_VELOCITY_BIAS):

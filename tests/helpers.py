@@ -219,7 +219,7 @@ def oracle_conv_step(w, inp, strips=None, grid=None, eta=None):
     rounded to bf16 like the device's.  `strips` = P_r (or `grid` = (P_r, P_c)) runs the
     strip / halo formulation."""
     from oracle import mbd_oracle as O
-    layers = [O.Conv3x3(oracle_kernel(k), relu=True) for k in inp.Ws]
+    layers = [O.Conv3x3(oracle_kernel(k), relu=True, stride=w.stride(i)) for i, k in enumerate(inp.Ws)]
     X = inp.X.astype(np.float64)
     eta = w.eta if eta is None else eta
     if strips is None and grid is None:
@@ -234,7 +234,7 @@ def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1, eta=None, 
     C_, H, Wd = w.dims
     L = w.n_layers
     eta = w.eta if eta is None else eta
-    net = mbd.Net(mbd.conv_layers(L, C_, H, Wd, k=[w.kshape(i) for i in range(L)], channels=w.channels), w.B, P_r, P_c, mbd.BF16,
+    net = mbd.Net(mbd.conv_layers(L, C_, H, Wd, k=[w.kshape(i) for i in range(L)], channels=w.channels, strides=w.strides), w.B, P_r, P_c, mbd.BF16,
                   mbd.LOSS_HALF_SSQ, max_partials)
     for i in range(L):
         net.set_weights(i, to_dev(inp.Ws[i], True))
@@ -299,7 +299,7 @@ def oracle_mixed_step(w, inp, blocked_grid=None, eta=None, conv_split="domain"):
     flattened activation; stored activations rounded to bf16 like the device's."""
     from oracle import mbd_oracle as O
     Lc = w.n_layers
-    layers = [O.Conv3x3(oracle_kernel(inp.Ws[i]), relu=True, split=conv_split) for i in range(Lc)]
+    layers = [O.Conv3x3(oracle_kernel(inp.Ws[i]), relu=True, split=conv_split, stride=w.stride(i)) for i in range(Lc)]
     for i in range(Lc, w.L):
         layers.append(O.FC(inp.Ws[i].astype(np.float64), inp.bs[i].astype(np.float64), relu=True))
     X = inp.X.astype(np.float64)
@@ -313,7 +313,8 @@ def mixed_layers(w, conv_split=None):
     from paper_1712_04432_b200 import mbd
     C_, H, Wd = w.dims
     split = mbd.SPLIT_DOMAIN if conv_split in (None, "domain") else mbd.SPLIT_BATCH
-    return mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.ksize(i) for i in range(w.n_layers)], split=split) + mbd.fc_layers(w.fc_dims, bias=True)
+    return mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.kshape(i) for i in range(w.n_layers)], split=split, channels=w.channels,
+                           strides=w.strides) + mbd.fc_layers(w.fc_dims, bias=True)
 
 
 def oracle_mixed_acts(o, w):
@@ -324,7 +325,7 @@ def oracle_mixed_acts(o, w):
     for i in range(w.L - 1):
         x = o["Xs"][i + 1]
         if i < w.n_layers:
-            x = x if x.ndim == 4 else np.ascontiguousarray(x.T).reshape(w.B, C_, H, Wd)
+            x = x if x.ndim == 4 else np.ascontiguousarray(x.T).reshape(w.B, w.chan(i + 1), *w.out_hw(i))
         else:
             x = x.T
         out.append(np.ascontiguousarray(x, np.float32))
@@ -391,7 +392,7 @@ def compare_mixed_step(g, o, w, tol, fused=False, tol_below_relu=None, init=None
     def dev_layout(a, i):
         """oracle tensor of layer i's output side -> the device's layout"""
         if i < Lc:
-            return a if a.ndim == 4 else np.ascontiguousarray(a.T).reshape(w.B, C_, H, Wd)
+            return a if a.ndim == 4 else np.ascontiguousarray(a.T).reshape(w.B, w.chan(w.n_layers), *w.out_hw(w.n_layers - 1))
         return a.T
 
     assert abs(g["J"] - o["J"]) <= max(tol, 1e-4) * abs(o["J"]), (g["J"], o["J"])

@@ -36,7 +36,7 @@ def _as_layers(rows):
         else:
             out.append(mbd.Layer(kind=mbd.CONV3X3, split={"domain": mbd.SPLIT_DOMAIN, "batch": mbd.SPLIT_BATCH}.get(l["split"], mbd.SPLIT_MODEL),
                                  relu=1, bias=0, d_in=l["C_in"] * l["H"] * l["W"], d_out=l["C_out"] * l["H"] * l["W"],
-                                 C_in=l["C_in"], C_out=l["C_out"], H=l["H"], W=l["W"], kh=l["kh"], kw=l["kw"]))
+                                 C_in=l["C_in"], C_out=l["C_out"], H=l["H"], W=l["W"], kh=l["kh"], kw=l["kw"], stride=l.get("stride", 0)))
     return out
 
 
@@ -74,6 +74,27 @@ def test_comm_words_of_batch_parallel_convolutions(P_r, P_c):
     with pytest.raises(mbd.MbdError) as e:
         mbd.comm_words(_as_layers(net), 12, 4, 4)            # 16 processes, 12 samples
     assert e.value.status == mbd.E_GRID
+
+
+@pytest.mark.parametrize("P_r,P_c", [(1, 1), (2, 3), (4, 1), (1, 6)])
+def test_comm_words_of_strided_and_wide_kernels(P_r, P_c):
+    # a 7 x 7 stride-2 layer: halo rows floor(7/2) = 3; the forward halo is X_W X_C wide (input), the backward one
+    # Y_W Y_C (the output is half as wide); a model-split strided layer gathers an output of a quarter of the positions
+    dom = [dict(kind="conv", split="domain", C_in=8, C_out=64, H=48, W=32, kh=7, kw=7, stride=2),
+           dict(kind="conv", split="domain", C_in=64, C_out=64, H=24, W=16, kh=5, kw=3)]
+    got = mbd.comm_words(_as_layers(dom), 12, P_r, P_c)
+    assert got == CW.layer_words(dom, 12, P_r, P_c)
+    if P_r > 1:
+        assert got[0]["halo_fwd"] == -(-12 * 32 * 8 * 3 // P_c) and got[0]["halo_bwd"] == -(-12 * 16 * 64 * 3 // P_c)
+        assert got[1]["halo_fwd"] == got[1]["halo_bwd"] == -(-12 * 16 * 64 * 2 // P_c)
+    mod = [dict(kind="conv", split="model", C_in=8, C_out=24, H=12, W=12, kh=3, kw=3, stride=2)] * 1
+    got = mbd.comm_words(_as_layers(mod), 12, P_r, P_c)
+    assert got == CW.layer_words(mod, 12, P_r, P_c)
+    assert got[0]["allgather_y"] == -(-12 * (P_r - 1) * 24 * 6 * 6 // (P_r * P_c))
+    bad = _as_layers([dict(kind="conv", split="domain", C_in=8, C_out=8, H=9, W=12, kh=3, kw=3, stride=2)])
+    with pytest.raises(mbd.MbdError) as e:
+        mbd.comm_words(bad, 12, 1, 1)                # 9 rows do not divide by the stride
+    assert e.value.status == mbd.E_INVALID
 
 
 def test_comm_words_rejects_bad_arguments():

@@ -45,6 +45,18 @@ def test_invalid_and_unsupported():
     assert create(mbd.conv_layers(2, 16, 8, 16, channels=(16, 32, 8))[:1] + mbd.conv_layers(1, 16, 8, 16), 4,
                   loss=mbd.LOSS_HALF_SSQ) == mbd.E_INVALID                                 # channel counts do not chain
     assert create(mbd.conv_layers(2, 16, 8, 16, k=[(5, 5), (1, 7)], channels=(16, 32, 8)), 4, loss=mbd.LOSS_HALF_SSQ) in (mbd.OK, mbd.E_CUDA)
+    # strides: the image sizes must chain (H_{i+1} = H_i / s_i), divide by the stride, and the stride is at most 4
+    assert create(mbd.conv_layers(2, 16, 16, 16, strides=(2, 1)), 4, loss=mbd.LOSS_HALF_SSQ) in (mbd.OK, mbd.E_CUDA)
+    unchained = mbd.conv_layers(2, 16, 16, 16, strides=(2, 1))
+    unchained[1].H = 16
+    assert create(unchained, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_INVALID
+    odd = mbd.conv_layers(1, 16, 16, 16)
+    odd[0].stride = 3                                                                      # 16 rows, stride 3
+    assert create(odd, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_INVALID
+    far = mbd.conv_layers(1, 16, 40, 40)
+    far[0].stride = 5
+    assert create(far, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
+    assert create(mbd.conv_layers(1, 16, 16, 16, strides=(2,)), 4, 16, 1, loss=mbd.LOSS_HALF_SSQ) == mbd.E_GRID    # 8 output rows, 16 strips
     assert create(mbd.conv_layers(2, 64, 8, 16, k=[3, 1]), 4, loss=mbd.LOSS_HALF_SSQ) in (mbd.OK, mbd.E_CUDA)   # valid; E_CUDA only without a device
     assert create(mbd.conv_layers(1, 64, 8, 16), 4, loss=mbd.LOSS_SOFTMAX_CE) == mbd.E_UNSUPPORTED
     assert create(fc, 8, loss=mbd.LOSS_NONE) == mbd.E_UNSUPPORTED                          # "no loss" is for convolution stacks

@@ -363,6 +363,51 @@ def test_wide_kernel_tap_direction_and_finite_differences():
         assert abs((J(K, Xp) - J(K, Xm)) / (2 * eps) - dX[idx]) < 1e-6 * max(1.0, abs(dX[idx]))
 
 
+@pytest.mark.parametrize("ksize,s", [((3, 3), 2), ((5, 5), 2), ((7, 7), 2), ((3, 3), 3), ((1, 1), 2), ((5, 3), 4)])
+def test_strided_convolution(ksize, s):
+    # scalar loops over the strided index, the adjoint identities of the three strided functions, central differences
+    # of J = sum(Y^2)/2, and stride 1 as the un-strided functions
+    kh, kw = ksize
+    r = rng(66)
+    H, W = 12, 24
+    K, X = r.standard_normal((3, 2, kh, kw)) / 3, r.standard_normal((2, 2, H, W))
+    Y = O.conv_strided(K, X, s)
+    assert Y.shape == (2, 3, H // s, W // s)
+    assert relerr(Y, np.array(brute.conv_strided(K.tolist(), X.tolist(), s))) < 1e-14
+    dY = r.standard_normal(Y.shape)
+    lhs = float(np.sum(dY * Y))
+    assert abs(lhs - float(np.sum(O.conv_strided_dX(K, dY, s) * X))) < 1e-11 * abs(lhs)
+    assert abs(lhs - float(np.sum(O.conv_strided_dK(dY, X, ksize, s) * K))) < 1e-11 * abs(lhs)
+    assert np.array_equal(O.conv_strided(K, X, 1), O.conv3x3(K, X))
+    J = lambda K_, X_: 0.5 * float(np.sum(O.conv_strided(K_, X_, s) ** 2))
+    dK, dX = O.conv_strided_dK(Y, X, ksize, s), O.conv_strided_dX(K, Y, s)
+    eps = 1e-6
+    for idx in [(0, 0, 0, 0), (2, 1, kh - 1, kw // 2)]:
+        Kp, Km = K.copy(), K.copy(); Kp[idx] += eps; Km[idx] -= eps
+        assert abs((J(Kp, X) - J(Km, X)) / (2 * eps) - dK[idx]) < 1e-6 * max(1.0, abs(dK[idx]))
+    for idx in [(0, 0, 0, 0), (1, 1, 5, 7), (0, 1, H - 1, W - 1)]:
+        Xp, Xm = X.copy(), X.copy(); Xp[idx] += eps; Xm[idx] -= eps
+        assert abs((J(K, Xp) - J(K, Xm)) / (2 * eps) - dX[idx]) < 1e-6 * max(1.0, abs(dX[idx]))
+
+
+def test_strided_layer_inside_a_training_step():
+    # a stride-2 layer between two stride-1 layers: the step's gradients against central differences of its loss
+    r = rng(67)
+    layers = [O.Conv3x3(r.standard_normal((3, 2, 3, 3)) / 3), O.Conv3x3(r.standard_normal((4, 3, 5, 5)) / 5, stride=2),
+              O.Conv3x3(r.standard_normal((2, 4, 3, 3)) / 4)]
+    X = r.standard_normal((2, 2, 8, 12))
+    res = O.train_step(layers, X, None, "half_ssq", 0.0)
+    assert res["Ys"][1].shape == (2, 4, 4, 6) and res["Ys"][2].shape == (2, 2, 4, 6)
+    eps = 1e-6
+    for li, idx in [(0, (1, 0, 2, 1)), (1, (3, 2, 0, 4)), (2, (0, 3, 1, 1))]:
+        def J(delta):
+            ls = [O.Conv3x3(l.K.copy(), l.relu, l.split, l.stride) for l in layers]
+            ls[li].K[idx] += delta
+            return O.total_loss(ls, X, None, "half_ssq")
+        fd = (J(eps) - J(-eps)) / (2 * eps)
+        assert abs(fd - res["dWs"][li][idx]) < 1e-5 * max(1.0, abs(fd)), (li, fd, res["dWs"][li][idx])
+
+
 def test_conv_centre_tap_is_per_pixel_fc():
     # a kernel with only its centre tap is the 1x1 convolution: Y[:, :, h, w] = M X[:, :, h, w]
     K, X, _ = conv_case(seed=51)

@@ -86,12 +86,60 @@ def test_free_running_step_and_reproducibility():
         assert np.array_equal(a["new_W"][i], b["new_W"][i]) and np.array_equal(a["dY"][i], b["dY"][i])
 
 
+STRIDED = {
+    # name: (channels, kernel shapes, strides, H, W, B)
+    "stride2_3x3_between_unit_layers": ((16, 24, 32, 16), ((3, 3), (3, 3), (3, 3)), (1, 2, 1), 16, 24, 3),
+    "stride2_5x5_first": ((8, 32, 16), ((5, 5), (3, 3)), (2, 1), 24, 16, 4),
+    "stride2_7x7_then_stride2_1x1": ((8, 64, 72), ((7, 7), (1, 1)), (2, 2), 24, 32, 2),
+    "stride3_3x3_and_stride4_5x3": ((16, 16, 8), ((3, 3), (5, 3)), (3, 4), 48, 24, 2),
+}
+
+
+@pytest.fixture(scope="module", params=sorted(STRIDED))
+def strided(request):
+    ch, ks, st, H, W, B = STRIDED[request.param]
+    w = I.conv_workload(ch[0], H, W, B, n_layers=len(ks), name=request.param, ksizes=ks, channels=ch, strides=st)
+    inp = I.make_inputs(w, seed=71)
+    o = oracle_conv_step(w, inp)
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    return w, inp, oracle_with_eta(o, inp.Ws, [None] * w.n_layers, w.B, eta), eta
+
+
+@pytest.mark.parametrize("P_r,P_c,mp", [(1, 1, 0), (2, 1, 0), (2, 2, 4), (4, 1, 2)])
+@pytest.mark.parametrize("fused", [False, True])
+def test_strided_layers(strided, P_r, P_c, mp, fused):
+    # A stride-s layer keeps every s-th position of the stride-1 result (Section 2.2 speaks of the halo only; the halo a
+    # strip needs is still floor(k_h/2) input rows).  The device never computes a position it does not keep: it reads
+    # its input through s^2 phase planes, each a stride-1 shifted-view product again.
+    w, inp, o, eta = strided
+    H_last = w.out_hw(w.n_layers - 1)[0]
+    if H_last % P_r or (P_r > 1 and H_last // P_r < 2):
+        pytest.skip("strips of equal height, no shorter than the halo, at every resolution")
+    g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o), P_c=P_c, eta=eta, max_partials=mp)
+    assert g["act"][-1].shape[2:] == w.out_hw(w.n_layers - 1)
+    compare_conv_step(g, o, TOL, fused, init=inp, require_sized=True)
+
+
 @pytest.mark.parametrize("grid,mp,fused", [((1, 1), 1, False), ((2, 3), 4, True), ((4, 2), 2, False)])
 def test_integrated_stack_on_general_convolutions(grid, mp, fused):
     # Section 2.4 on layers of the general path: a 5 x 5 and a 3 x 3 convolution with 16 channels on 8 x 20 images, then
     # model-parallel fully connected layers 2560 -> 64 -> 16 on the same grid
     w = I.mixed_workload(16, 8, 20, 2, (64, 16), 6, name="mixed_general", ksizes=(5, 3))
     inp = I.make_inputs(w, seed=65)
+    o = oracle_mixed_step(w, inp)
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    o = oracle_with_eta(o, inp.Ws, inp.bs, w.B, eta)
+    g = gpu_mixed_step(w, inp, grid, mp, fused=fused, force_acts=oracle_mixed_acts(o, w), eta=eta)
+    compare_mixed_step(g, o, w, TOL, fused=fused, init=inp, require_sized=True)
+
+
+@pytest.mark.parametrize("grid,mp,fused", [((1, 1), 1, True), ((2, 2), 2, False)])
+def test_integrated_stack_with_a_strided_layer(grid, mp, fused):
+    # 3 x 3 stride 2 (16 -> 32 channels, 16 x 24 -> 8 x 12), 3 x 3 stride 1, then FC 3072 -> 48 -> 16: the first fully
+    # connected layer reads C_L * H_L * W_L values per sample
+    w = I.mixed_workload(16, 16, 24, 2, (48, 16), 4, name="mixed_strided", ksizes=(3, 3), channels=(16, 32, 32), strides=(2, 1))
+    assert w.fc_dims[0] == 32 * 8 * 12
+    inp = I.make_inputs(w, seed=72)
     o = oracle_mixed_step(w, inp)
     eta = update_sized_eta(o, inp.Ws, w.B)
     o = oracle_with_eta(o, inp.Ws, inp.bs, w.B, eta)
