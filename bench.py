@@ -175,7 +175,7 @@ def oracle_sample(w, inp):
         k3[:, :, 1, 1] = k[:, :, 0, 0]
         return k3
 
-    layers = [O.Conv3x3(as3x3(k)) for k in inp.Ws]
+    layers = [O.Conv3x3(as3x3(k), stride=w.stride(i)) for i, k in enumerate(inp.Ws)]
     X = inp.X[:Bs, :, :Hs, :].astype(np.float64)
     t0 = time.perf_counter()
     O.train_step(layers, X, None, "half_ssq", w.eta)
