@@ -336,7 +336,9 @@ __device__ __forceinline__ FwdRun fwd_run(const FwdParams& p, long long pos, lon
 __device__ __forceinline__ int acc_block(int g) { return 7 - (g & 7); }
 
 // PACKED: several strips per tile (narrow images); the wide instantiation keeps its single box per row.
-template <bool PACKED>
+// UNEVEN: strips of unequal height (H mod P_r != 0): only this instantiation carries the dead-row handling -- as a
+// run-time case in the common one it cost 1 - 7 % of the epilogue-bound launches.
+template <bool PACKED, bool UNEVEN>
 __global__ void __launch_bounds__(FWD_THREADS, 1)
 conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
                 const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmMask, const FwdParams p) {
@@ -536,7 +538,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           if (q.x0 >= p.nseg * FWD_PIX) { q.x0 = 0; q.z += pack; }
         }
       };
-      const bool uneven = strips_uneven(p.H, p.P_r, p.Hs);
+      constexpr bool uneven = UNEVEN;
       const int sub = FWD_PIX / pack;                   // tile positions per strip
       const int sub_bytes = sub * 128;
       auto load_mask = [&](int k, const Pos& q) {
@@ -630,7 +632,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             const int zj = z + j;
             if (zj >= p.Z) break;
             const int hs_j = uneven ? strip_height(zj % p.P_r, p.H, p.P_r, p.Hs) : p.Hs;
-            if (row > hs_j) continue;                  // dead row of a short strip
+            if (uneven && row > hs_j) continue;        // dead row of a short strip
             const uint32_t src = stg_out + buf * FWD_TILE_BYTES + j * sub_bytes;
             asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
                          ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(row), "r"(zj), "r"(src)
@@ -639,7 +641,7 @@ conv_fwd_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             // halo row of the strip above / below it in the same image.
             if (row == 1 && p.P_r > 1 && zj % p.P_r > 0)
               asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
-                           ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(strip_height(zj % p.P_r - 1, p.H, p.P_r, p.Hs) + 1), "r"(zj - 1), "r"(src)
+                           ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(0), "r"(x0), "r"(uneven ? strip_height(zj % p.P_r - 1, p.H, p.P_r, p.Hs) + 1 : p.Hs + 1), "r"(zj - 1), "r"(src)
                            : "memory");
             if (row == hs_j && p.P_r > 1 && zj % p.P_r < p.P_r - 1)
               asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
@@ -924,8 +926,10 @@ cudaError_t conv_init() {
   cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
   if (e != cudaSuccess) return e;
   if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
-  if ((e = cudaFuncSetAttribute(conv_fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(conv_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(conv_fwd_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(conv_fwd_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(conv_fwd_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(conv_fwd_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM)) != cudaSuccess) return e;
   g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   return cudaSuccess;
@@ -1002,10 +1006,13 @@ void launch_fwd(ConvNet* c, int cls, int layer, const CUtensorMap& in, const CUt
   if (mode == MODE_STORE_SSQ && !loss_add) cudaMemsetAsync(c->loss_part, 0, sizeof(float) * c->grid * 8, c->stream);
   const double flops = 2.0 * c->B * c->H * c->W * (c->k1[layer] ? 1.0 : 9.0) * C * C * nrows / c->Hs;   // the method's flops, not the kernel's
   c->prof->begin(cls, flops);
+  const bool uneven = c->H % c->P_r != 0;
   if (c->pack > 1)
-    launch_pdl(conv_fwd_kernel<true>, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, out_tile, mask_tile ? *mask_tile : out_tile, p);
+    launch_pdl(uneven ? conv_fwd_kernel<true, true> : conv_fwd_kernel<true, false>, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, out_tile,
+               mask_tile ? *mask_tile : out_tile, p);
   else
-    launch_pdl(conv_fwd_kernel<false>, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, out_tile, mask_tile ? *mask_tile : out_tile, p);
+    launch_pdl(uneven ? conv_fwd_kernel<false, true> : conv_fwd_kernel<false, false>, dim3(grid), dim3(FWD_THREADS), FWD_SMEM, c->stream, 1, in, w, out_tile,
+               mask_tile ? *mask_tile : out_tile, p);
   c->prof->end();
 }
 
