@@ -157,7 +157,7 @@ enum {
  * from each neighbour, which must be the adjacent strip's own rows: MBD_E_GRID when a strip is shorter than that.  The
  * stride-1 layers with 64 channels and 3x3 or 1x1 kernels run on kernels of their own; every other shape runs as
  * products of row-shifted views on the contraction kernel of the fully connected layers, and there strips of unequal
- * height, fp32 master weights, momentum and the interior / boundary calls are MBD_E_UNSUPPORTED.
+ * height, the interior / boundary calls and mbd_conv_outer_rows are MBD_E_UNSUPPORTED.
  * MBD_E_UNSUPPORTED for other convolutions (even or larger kernels, other channel counts, larger strides),
  * a convolution above a fully connected layer, half-SSQ with
  * fully connected layers or softmax-CE without them, or bf16 FC dims that are not

@@ -1126,7 +1126,7 @@ mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev) {
 }
 
 mbd_status conv_enable_master(ConvNet* c) {
-  if (c->gen) return MBD_E_UNSUPPORTED;
+  if (c->gen) return gconv_enable_master(c->gen);
   if (!c->K32.empty()) return MBD_OK;
   std::vector<float*> m(c->L, nullptr);
   for (int i = 0; i < c->L; ++i) {
@@ -1142,7 +1142,7 @@ mbd_status conv_enable_master(ConvNet* c) {
 }
 
 mbd_status conv_enable_momentum(ConvNet* c, float mu) {
-  if (c->gen) return MBD_E_UNSUPPORTED;
+  if (c->gen) return gconv_enable_momentum(c->gen, mu);
   if (c->Vk.empty()) {
     std::vector<float*> v(c->L, nullptr);
     for (int i = 0; i < c->L; ++i) {

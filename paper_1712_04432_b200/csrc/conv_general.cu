@@ -232,6 +232,8 @@ struct GenConv {
   std::vector<bf16*> act, dY, Wm;
   std::vector<bf16*> xph, dxph;           // strided layers: phase planes of the input / of the gradient below
   std::vector<float*> dWm;
+  std::vector<float*> Wm32, Vm;           // fp32 master weights / momentum velocities in the layout of Wm (empty unless enabled)
+  float mu = 0.f;
   std::vector<TcGemm> fwd, bwd_weight;
   std::vector<std::vector<TcGemm>> bwd_data;   // one product (stride 1) or one per phase plane
   std::vector<std::vector<int>> bwd_taps;      // taps of each of those products (an empty plane gets zeros)
@@ -331,6 +333,8 @@ void gconv_destroy(GenConv* c) {
   for (bf16* p : c->xph) cudaFree(p);
   for (bf16* p : c->dxph) cudaFree(p);
   for (float* p : c->dWm) cudaFree(p);
+  for (float* p : c->Wm32) cudaFree(p);
+  for (float* p : c->Vm) cudaFree(p);
   cudaFree(c->partials); cudaFree(c->loss_part);
   delete c;
 }
@@ -467,8 +471,59 @@ int gconv_last_relu(const GenConv* c) { return c->relu[c->L - 1]; }
 mbd_status gconv_set_weights(GenConv* c, int i, const void* K_dev) {
   const long long n = static_cast<long long>(c->Cout[i]) * c->taps[i] * c->Cp[i];
   pack_w_kernel<<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(static_cast<const bf16*>(K_dev), c->Wm[i], c->Cout[i], c->Cin[i], c->taps[i], c->Cp[i]);
+  if (!c->Wm32.empty() && widen_bf16_launch(c->Wm[i], c->Wm32[i], n, c->num_sms, c->stream) != cudaSuccess) return MBD_E_CUDA;
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
+
+// fp32 master weights / momentum: the update leaves the weight-gradient product (which then only materialises dWm)
+// and becomes one streaming kernel per layer over the internal weight layout -- as for the fully connected layers.
+mbd_status gconv_enable_master(GenConv* c) {
+  if (!c->Wm32.empty()) return MBD_OK;
+  std::vector<float*> m(c->L, nullptr);
+  for (int i = 0; i < c->L; ++i) {
+    const long long n = static_cast<long long>(c->Cout[i]) * c->taps[i] * c->Cp[i];
+    if (cudaMalloc(reinterpret_cast<void**>(&m[i]), n * 4) != cudaSuccess || widen_bf16_launch(c->Wm[i], m[i], n, c->num_sms, c->stream) != cudaSuccess) {
+      (void)cudaGetLastError();
+      for (float* q : m) cudaFree(q);
+      return MBD_E_ALLOC;
+    }
+  }
+  c->Wm32 = m;
+  return MBD_OK;
+}
+
+mbd_status gconv_enable_momentum(GenConv* c, float mu) {
+  if (c->Vm.empty()) {
+    std::vector<float*> v(c->L, nullptr);
+    for (int i = 0; i < c->L; ++i)
+      if (cudaMalloc(reinterpret_cast<void**>(&v[i]), static_cast<size_t>(c->Cout[i]) * c->taps[i] * c->Cp[i] * 4) != cudaSuccess) {
+        (void)cudaGetLastError();
+        for (float* q : v) cudaFree(q);
+        return MBD_E_ALLOC;
+      }
+    c->Vm = v;
+  }
+  for (int i = 0; i < c->L; ++i)
+    if (cudaMemsetAsync(c->Vm[i], 0, static_cast<size_t>(c->Cout[i]) * c->taps[i] * c->Cp[i] * 4, c->stream) != cudaSuccess) return MBD_E_CUDA;
+  c->mu = mu;
+  return MBD_OK;
+}
+
+namespace {
+// Eq. 1 (or its momentum form) from the materialised gradient of layer i
+mbd_status update_from_gradient(GenConv* c, int i, float eta) {
+  const long long n = static_cast<long long>(c->Cout[i]) * c->taps[i] * c->Cp[i];
+  const float scale = -eta / static_cast<float>(c->B);
+  float* w32 = c->Wm32.empty() ? nullptr : c->Wm32[i];
+  c->prof->begin(MBD_K_SGD, static_cast<double>(n) * (8.0 + (w32 ? 8.0 : 0.0) + (c->Vm.empty() ? 0.0 : 8.0)), c->stream);
+  cudaError_t e;
+  if (!c->Vm.empty()) e = sgd_momentum_update_launch(c->Wm[i], 1, w32, c->Vm[i], c->dWm[i], n, c->mu, 1.f / static_cast<float>(c->B), eta, c->num_sms, c->stream);
+  else if (w32) e = sgd_master_update_launch(w32, c->Wm[i], c->dWm[i], n, scale, c->num_sms, c->stream);
+  else e = sgd_update_launch(c->Wm[i], 1, c->dWm[i], n, scale, c->num_sms, c->stream);
+  c->prof->end();
+  return e == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+}  // namespace
 mbd_status gconv_get_weights(GenConv* c, int i, void* K_dev) {
   const long long n = static_cast<long long>(c->Cout[i]) * c->Cin[i] * c->taps[i];
   unpack_w_kernel<bf16><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(c->Wm[i], static_cast<bf16*>(K_dev), c->Cout[i], c->Cin[i], c->taps[i], c->Cp[i]);
@@ -531,7 +586,8 @@ mbd_status gconv_forward(GenConv* c, const void* X_nchw, float* loss_sum_dev) {
 
 mbd_status gconv_backward_layer(GenConv* c, int i, float fused_eta) {
   if (i < 0 || i >= c->L) return MBD_E_INVALID;
-  const bool fused = fused_eta > 0.f;
+  const bool own_update = !c->Wm32.empty() || !c->Vm.empty();      // masters / momentum: gradient first, then the update kernel
+  const bool fused = fused_eta > 0.f && !own_update;
   const float scale = -fused_eta / static_cast<float>(c->B);
   const Geo& go = c->geo[i + 1];
   const int s = c->stride[i], Cin = c->Cin[i];
@@ -561,6 +617,7 @@ mbd_status gconv_backward_layer(GenConv* c, int i, float fused_eta) {
   const Epi ew = fused ? make_epi_sgd(c->Wm[i], ldw, scale) : make_epi_act(c->dWm[i], ldw, 0, 0);
   const mbd_status st = run(c, c->bwd_weight[i], MBD_K_CONV_BWD_WEIGHT, flops, ew);
   if (st != MBD_OK) return st;
+  if (own_update && fused_eta > 0.f && update_from_gradient(c, i, fused_eta) != MBD_OK) return MBD_E_CUDA;
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
@@ -571,13 +628,8 @@ mbd_status gconv_backward(GenConv* c, float fused_eta) {
 }
 
 mbd_status gconv_sgd_step(GenConv* c, float eta) {
-  const float scale = -eta / static_cast<float>(c->B);
-  for (int i = 0; i < c->L; ++i) {
-    const long long n = static_cast<long long>(c->Cout[i]) * c->taps[i] * c->Cp[i];
-    c->prof->begin(MBD_K_SGD, static_cast<double>(n) * 8.0, c->stream);
-    if (sgd_update_launch(c->Wm[i], 1, c->dWm[i], n, scale, c->num_sms, c->stream) != cudaSuccess) return MBD_E_CUDA;
-    c->prof->end();
-  }
+  for (int i = 0; i < c->L; ++i)
+    if (update_from_gradient(c, i, eta) != MBD_OK) return MBD_E_CUDA;
   return MBD_OK;
 }
 
@@ -594,10 +646,12 @@ mbd_status gconv_top_grad_from_nchw(GenConv* c, const void* src) {
 
 mbd_status gconv_get_tensor(GenConv* c, int which, int layer, void* dst, size_t bytes) {
   if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
-  if (which == MBD_T_DW) {
+  if (which == MBD_T_DW || which == MBD_T_MASTER || which == MBD_T_VELOCITY) {
     const long long n = static_cast<long long>(c->Cout[layer]) * c->Cin[layer] * c->taps[layer];
     if (bytes != static_cast<size_t>(n) * 4) return MBD_E_INVALID;
-    unpack_w_kernel<float><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(c->dWm[layer], static_cast<float*>(dst), c->Cout[layer], c->Cin[layer],
+    if ((which == MBD_T_MASTER && c->Wm32.empty()) || (which == MBD_T_VELOCITY && c->Vm.empty())) return MBD_E_STATE;
+    const float* src32 = which == MBD_T_DW ? c->dWm[layer] : which == MBD_T_MASTER ? c->Wm32[layer] : c->Vm[layer];
+    unpack_w_kernel<float><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(src32, static_cast<float*>(dst), c->Cout[layer], c->Cin[layer],
                                                                           c->taps[layer], c->Cp[layer]);
     return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
   }

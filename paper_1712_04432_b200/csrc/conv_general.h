@@ -22,6 +22,8 @@ mbd_status gconv_forward(GenConv* c, const void* X_nchw, float* loss_sum_dev);
 mbd_status gconv_backward_layer(GenConv* c, int layer, float fused_eta);
 mbd_status gconv_backward(GenConv* c, float fused_eta);
 mbd_status gconv_sgd_step(GenConv* c, float eta);
+mbd_status gconv_enable_master(GenConv* c);                 // fp32 master weights from now on
+mbd_status gconv_enable_momentum(GenConv* c, float mu);     // heavy-ball momentum from now on, velocities zero
 mbd_status gconv_get_tensor(GenConv* c, int which, int layer, void* dst, size_t bytes);
 mbd_status gconv_set_tensor(GenConv* c, int which, int layer, const void* src, size_t bytes);
 mbd_status gconv_set_dw(GenConv* c, int layer, const void* src, size_t bytes);

@@ -147,6 +147,53 @@ def test_integrated_stack_with_a_strided_layer(grid, mp, fused):
     compare_mixed_step(g, o, w, TOL, fused=fused, init=inp, require_sized=True)
 
 
+@pytest.mark.parametrize("master,mu", [(True, None), (False, 0.9), (True, 0.9)])
+def test_master_weights_and_momentum_on_general_layers(master, mu):
+    # the update as a kernel of its own over the internal weight layout: from the gradient the device itself
+    # materialised, three steps, mbd_backward(eta) and mbd_backward(0) + mbd_sgd_step(eta) bit for bit
+    import torch
+    from oracle import mbd_oracle as O
+    from paper_1712_04432_b200 import mbd
+    from tests.helpers import to_dev, to_np
+    ch, ks, st, H, W, B = (16, 24, 32), ((5, 5), (3, 3)), (1, 2), 16, 24, 3
+    w = I.conv_workload(ch[0], H, W, B, n_layers=2, name="gen_update", ksizes=ks, channels=ch, strides=st)
+    inp = I.make_inputs(w, seed=73)
+    X = to_dev(inp.X, True)
+    eta = 1e-3
+
+    def make():
+        net = mbd.Net(mbd.conv_layers(2, ch[0], H, W, k=list(ks), channels=ch, strides=st), B, 2, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 2)
+        if master:
+            net.enable_master_weights()
+        for i in range(2):
+            net.set_weights(i, to_dev(inp.Ws[i], True))
+        if mu is not None:
+            net.enable_momentum(mu)
+        return net
+    a, b = make(), make()
+    for step in range(3):
+        W_old = [to_np(a.get_tensor(mbd.T_MASTER, i)) if master else to_np(a.get_weights(i)) for i in range(2)]
+        V_old = [to_np(a.get_tensor(mbd.T_VELOCITY, i)) if mu is not None else np.zeros_like(W_old[i]) for i in range(2)]
+        a.forward(X); a.backward(0.0)
+        dW = [to_np(a.get_tensor(mbd.T_DW, i)) for i in range(2)]
+        a.sgd_step(eta)
+        b.forward(X); b.backward(eta)
+        a.poll(); b.poll()
+        for i in range(2):
+            W_want, V_want = O.sgd_momentum(W_old[i], V_old[i], dW[i], eta, B, mu if mu is not None else 0.0)
+            if mu is not None:
+                assert rel_fro(to_np(a.get_tensor(mbd.T_VELOCITY, i)), V_want) < 1e-6, (step, i)
+            if master:
+                assert rel_fro(to_np(a.get_tensor(mbd.T_MASTER, i)), W_want) < 1e-6, (step, i)
+                assert torch.equal(a.get_tensor(mbd.T_MASTER, i).to(torch.bfloat16), a.get_weights(i))
+                assert torch.equal(a.get_tensor(mbd.T_MASTER, i), b.get_tensor(mbd.T_MASTER, i)), (step, i)
+            else:
+                assert rel_fro(to_np(a.get_weights(i)), W_want) < 3e-3, (step, i)
+            assert torch.equal(a.get_weights(i), b.get_weights(i)), (step, i)
+            assert np.linalg.norm(dW[i]) > 0
+    a.close(); b.close()
+
+
 def test_unsupported_shapes_are_refused():
     from paper_1712_04432_b200 import mbd
     for kw in (dict(k=(4, 3)), dict(k=9), dict(channels=(12, 8, 8)), dict(channels=(8, 4, 8))):
