@@ -151,7 +151,7 @@ enum {
  * Batch-split convolutions (MBD_SPLIT_BATCH) are cut into P_r P_c batch blocks and no strips; between them
  * and the fully connected layers on P_r x P_c lies the re-distribution of Eq. 6 (mbd_redistribute_time).
  * Convolutions (kind MBD_CONV3X3 whatever the kernel size; Section 2.2): zero padding floor(k/2), k_h and
- * k_w odd and at most 7, stride 1 to 4 (the same in both directions), C_in and C_out multiples of 8, C_in of a layer =
+ * k_w odd and at most 11, stride 1 to 4 (the same in both directions), C_in and C_out multiples of 8, C_in of a layer =
  * C_out of the layer below, H x W of a layer = the output size of the layer below (H/s x W/s of its input);
  * weights [C_out][C_in][k_h][k_w] ([C_out][C_in] for 1x1).  A strip needs floor(k_h/2) halo rows
  * from each neighbour, which must be the adjacent strip's own rows: MBD_E_GRID when a strip is shorter than that.  The

@@ -1,4 +1,4 @@
-// General domain-parallel convolution layers (Section 2.2 / 2.4): any odd k_h x k_w up to 7 x 7, stride 1, zero
+// General domain-parallel convolution layers (Section 2.2 / 2.4): any odd k_h x k_w up to 11 x 11, stride 1 to 4, zero
 // padding floor(k/2), C_in and C_out multiples of 8, row strips with floor(k_h/2) halo rows.  The layers with 64
 // channels and 3 x 3 / 1 x 1 kernels have kernels of their own (conv.cu); everything else runs here, on the
 // tensor-core contraction kernel of the fully connected layers (gemm_tc.cu) fed with shifted views.
@@ -347,7 +347,7 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
   for (int i = 0; i < L; ++i) {
     const mbd_layer& l = layers[i];
     const int s = l.stride > 1 ? l.stride : 1;
-    if (l.kh < 1 || l.kw < 1 || l.kh > 7 || l.kw > 7 || l.kh % 2 == 0 || l.kw % 2 == 0 || s > 4) return MBD_E_UNSUPPORTED;
+    if (l.kh < 1 || l.kw < 1 || l.kh > 11 || l.kw > 11 || l.kh % 2 == 0 || l.kw % 2 == 0 || s > 4) return MBD_E_UNSUPPORTED;
     if (l.C_in < 8 || l.C_out < 8 || l.C_in % 8 || l.C_out % 8) return MBD_E_UNSUPPORTED;       // 16-byte rows for TMA
     if (i > 0 && l.C_in != layers[i - 1].C_out) return MBD_E_INVALID;
     if (l.H != H || l.W != W || H % s || W % s) return MBD_E_INVALID;                            // sizes chain through the strides
@@ -413,7 +413,7 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
     const Geo& go = c->geo[i + 1];                   // the products run over the pixels of the layer's output geometry
     const int M = static_cast<int>(go.Ptot);
     bf16* xin = s > 1 ? c->xph[i] : c->act[i];       // what the forward and weight-gradient products read
-    int off[49], plane[49];
+    int off[MAX_TAPS], plane[MAX_TAPS];
     tap_offsets(c->kh[i], c->kw[i], s, go, off, plane);
     // forward
     TcGemm& f = c->fwd[i];

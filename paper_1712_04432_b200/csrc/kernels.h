@@ -98,10 +98,11 @@ struct Epi {
 // A strided layer reads phase-decimated copies of its input stored one after another (plane (a, b) holds the pixels
 // (s h' + a, s w' + b)): its offsets then include the plane's start, and backward-data runs once per plane with the
 // taps that read it -- `tap[j]` is the position in the weight matrix of the j-th tap of such a subset.
+constexpr int MAX_TAPS = 121;      // kernels up to 11 x 11
 struct ConvShift {
   int mode, taps, blocks, Cp;      // blocks: 64-wide k-blocks per tap (modes 1, 2)
-  int off[49];
-  int tap[49];                     // mode 2: weight-matrix tap of the j-th tap of this product (identity for stride 1)
+  int off[MAX_TAPS];
+  int tap[MAX_TAPS];               // mode 2: weight-matrix tap of the j-th tap of this product (identity for stride 1)
 };
 
 struct TcGemm {

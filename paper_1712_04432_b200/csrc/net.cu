@@ -309,8 +309,8 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
       if (dtype == MBD_BF16 && (l.d_in % 8 || l.d_out % 8)) return MBD_E_UNSUPPORTED;
       if (l.d_in > INT32_MAX || l.d_out > INT32_MAX || B > INT32_MAX) return MBD_E_UNSUPPORTED;
     } else if (l.kind == MBD_CONV3X3) {
-      // stride 1, "same" padding; odd kernel sizes up to 7, channel counts that are multiples of 8
-      if (l.kh < 1 || l.kw < 1 || l.kh > 7 || l.kw > 7 || l.kh % 2 == 0 || l.kw % 2 == 0 || dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
+      // "same" padding; odd kernel sizes up to 11, channel counts that are multiples of 8
+      if (l.kh < 1 || l.kw < 1 || l.kh > 11 || l.kw > 11 || l.kh % 2 == 0 || l.kw % 2 == 0 || dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
       if (l.C_in < 8 || l.C_out < 8 || l.C_in % 8 || l.C_out % 8) return MBD_E_UNSUPPORTED;
       if (i > 0 && l.C_in != layers[i - 1].C_out) return MBD_E_INVALID;
       if (l.split != MBD_SPLIT_DOMAIN && l.split != MBD_SPLIT_BATCH) return MBD_E_UNSUPPORTED;

@@ -36,7 +36,7 @@ def test_invalid_and_unsupported():
     assert create(mbd.fc_layers((64, 32)) + mbd.fc_layers((48, 16)), 8) == mbd.E_INVALID   # dims do not chain
     assert create(mbd.fc_layers((60, 30)), 8) == mbd.E_UNSUPPORTED                         # bf16 needs multiples of 8
     conv9 = mbd.conv_layers(1, 64, 8, 16)
-    conv9[0].kh = conv9[0].kw = 9                                                          # kernels up to 7 x 7
+    conv9[0].kh = conv9[0].kw = 13                                                         # kernels up to 11 x 11
     assert create(conv9, 4, loss=mbd.LOSS_HALF_SSQ) == mbd.E_UNSUPPORTED
     conv43 = mbd.conv_layers(1, 64, 8, 16)
     conv43[0].kh = 4                                                                       # even sizes have no centre tap

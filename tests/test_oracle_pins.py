@@ -363,7 +363,7 @@ def test_wide_kernel_tap_direction_and_finite_differences():
         assert abs((J(K, Xp) - J(K, Xm)) / (2 * eps) - dX[idx]) < 1e-6 * max(1.0, abs(dX[idx]))
 
 
-@pytest.mark.parametrize("ksize,s", [((3, 3), 2), ((5, 5), 2), ((7, 7), 2), ((3, 3), 3), ((1, 1), 2), ((5, 3), 4)])
+@pytest.mark.parametrize("ksize,s", [((3, 3), 2), ((5, 5), 2), ((7, 7), 2), ((3, 3), 3), ((1, 1), 2), ((5, 3), 4), ((11, 11), 4)])
 def test_strided_convolution(ksize, s):
     # scalar loops over the strided index, the adjoint identities of the three strided functions, central differences
     # of J = sum(Y^2)/2, and stride 1 as the un-strided functions

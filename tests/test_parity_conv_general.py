@@ -1,5 +1,5 @@
 """Convolution layers the 64-channel 3 x 3 / 1 x 1 kernels do not cover -- other odd kernel sizes (5 x 5, 1 x 7,
-7 x 1, mixed in one network), channel counts that change from layer to layer and are not multiples of 64 -- on row
+7 x 1, 9 x 9, 11 x 11, mixed in one network), strides 2 to 4, channel counts that change from layer to layer and are not multiples of 64 -- on row
 strips with floor(k_h/2) halo rows (Section 2.2) and P_c batch blocks: forward outputs, J, the back-propagated
 gradients, the kernel gradients and the applied update against the fp64 oracle, through the C ABI."""
 import numpy as np
@@ -92,6 +92,9 @@ STRIDED = {
     "stride2_5x5_first": ((8, 32, 16), ((5, 5), (3, 3)), (2, 1), 24, 16, 4),
     "stride2_7x7_then_stride2_1x1": ((8, 64, 72), ((7, 7), (1, 1)), (2, 2), 24, 32, 2),
     "stride3_3x3_and_stride4_5x3": ((16, 16, 8), ((3, 3), (5, 3)), (3, 4), 48, 24, 2),
+    # the kernel sizes and strides of the network of Section 3 (its first layers: 11 x 11 stride 4, then 5 x 5, then 3 x 3)
+    "stride4_11x11_then_5x5_then_3x3": ((8, 96, 64, 48), ((11, 11), (5, 5), (3, 3)), (4, 1, 1), 32, 48, 2),
+    "unit_9x9_and_1x11": ((8, 16, 8), ((9, 9), (1, 11)), (1, 1), 12, 24, 2),
 }
 
 
@@ -113,7 +116,8 @@ def test_strided_layers(strided, P_r, P_c, mp, fused):
     # its input through s^2 phase planes, each a stride-1 shifted-view product again.
     w, inp, o, eta = strided
     H_last = w.out_hw(w.n_layers - 1)[0]
-    if H_last % P_r or (P_r > 1 and H_last // P_r < 2):
+    halo = max(-(-(w.kshape(i)[0] // 2) // w.stride(i)) for i in range(w.n_layers))      # rows a strip needs from a neighbour
+    if H_last % P_r or (P_r > 1 and H_last // P_r < halo):
         pytest.skip("strips of equal height, no shorter than the halo, at every resolution")
     g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o), P_c=P_c, eta=eta, max_partials=mp)
     assert g["act"][-1].shape[2:] == w.out_hw(w.n_layers - 1)
@@ -196,7 +200,7 @@ def test_master_weights_and_momentum_on_general_layers(master, mu):
 
 def test_unsupported_shapes_are_refused():
     from paper_1712_04432_b200 import mbd
-    for kw in (dict(k=(4, 3)), dict(k=9), dict(channels=(12, 8, 8)), dict(channels=(8, 4, 8))):
+    for kw in (dict(k=(4, 3)), dict(k=13), dict(channels=(12, 8, 8)), dict(channels=(8, 4, 8))):
         layers = mbd.conv_layers(2, 8, 12, 12, **{"k": 3, **kw}) if "channels" not in kw else \
             mbd.conv_layers(2, kw["channels"][0], 12, 12, channels=kw["channels"])
         with pytest.raises(mbd.MbdError) as e:
