@@ -125,8 +125,14 @@ def workload_config(w, grid, max_partials):
     if w.kind == "fc":
         desc = f"{w.name}: FC stack {'-'.join(str(d) for d in w.dims)}, B={w.B}, ReLU, softmax-CE, {w.dtype}"
     elif w.kind == "mixed":
-        desc = (f"{w.name}: {w.n_layers}x conv3x3 {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, then FC "
-                f"{'-'.join(str(d) for d in w.fc_dims)}, B={w.B}, ReLU, softmax-CE, {w.dtype}")
+        if w.channels or w.strides or w.ksizes:
+            lay = ", ".join(f"{w.kshape(i)[0]}x{w.kshape(i)[1]}{'/' + str(w.stride(i)) if w.stride(i) > 1 else ''} {w.chan(i)}->{w.chan(i + 1)}"
+                            for i in range(w.n_layers))
+            desc = (f"{w.name}: conv layers {lay} on {w.dims[1]}x{w.dims[2]}, then FC "
+                    f"{'-'.join(str(d) for d in w.fc_dims)}, B={w.B}, ReLU, softmax-CE, {w.dtype}")
+        else:
+            desc = (f"{w.name}: {w.n_layers}x conv3x3 {w.dims[0]}ch on {w.dims[1]}x{w.dims[2]}, then FC "
+                    f"{'-'.join(str(d) for d in w.fc_dims)}, B={w.B}, ReLU, softmax-CE, {w.dtype}")
     else:
         if w.channels or w.strides or any(w.kshape(i) != w.kshape(0) for i in range(w.n_layers)):
             lay = ", ".join(f"{w.kshape(i)[0]}x{w.kshape(i)[1]}{'/' + str(w.stride(i)) if w.stride(i) > 1 else ''} {w.chan(i)}->{w.chan(i + 1)}"
@@ -158,7 +164,7 @@ def oracle_sample(w, inp):
         return flops_per_sample * Bs, dt, f"whole {len(layers)}-layer network, first {Bs} of {w.B} samples, fp64 numpy"
     if w.kind == "mixed":
         Bs = min(w.B, 4)
-        layers = [O.Conv3x3(inp.Ws[i].astype(np.float64)) for i in range(w.n_layers)]
+        layers = [O.Conv3x3(inp.Ws[i].astype(np.float64), stride=w.stride(i)) for i in range(w.n_layers)]
         layers += [O.FC(inp.Ws[i].astype(np.float64), inp.bs[i].astype(np.float64)) for i in range(w.n_layers, w.L)]
         X = inp.X[:Bs].astype(np.float64)
         t0 = time.perf_counter()
@@ -286,7 +292,8 @@ def run_ours(args):
         labels_host = torch.from_numpy(inp.labels).pin_memory()
     elif w.kind == "mixed":
         C_, H, Wd = w.dims
-        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd) + mbd.fc_layers(w.fc_dims, bias=True), w.B, grid[0], grid[1],
+        net = mbd.Net(mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.kshape(i) for i in range(w.n_layers)], channels=w.channels,
+                                      strides=w.strides) + mbd.fc_layers(w.fc_dims, bias=True), w.B, grid[0], grid[1],
                       mbd.BF16, mbd.LOSS_SOFTMAX_CE, args.max_partials)
         for i, Wi in enumerate(inp.Ws):
             net.set_weights(i, dev(Wi), None if inp.bs[i] is None else torch.from_numpy(inp.bs[i]).cuda())
@@ -439,7 +446,8 @@ def run_ours(args):
         if w.kind == "conv":
             kname = "conv_fwd_kernel (forward, backward-data) + conv_wgrad_kernel"
         elif w.kind == "mixed":
-            kname = "conv_fwd_kernel + conv_wgrad_kernel (convolutions), gemm_tc_kernel (fully connected layers)"
+            kname = ("gemm_tc_kernel (convolutions as shifted-view products, fully connected layers)" if (w.channels or w.strides) else
+                     "conv_fwd_kernel + conv_wgrad_kernel (convolutions), gemm_tc_kernel (fully connected layers)")
         elif bf:
             kname = "gemm_tc_kernel (all three operand layouts)"
         else:

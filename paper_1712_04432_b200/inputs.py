@@ -129,6 +129,16 @@ WORKLOADS["mixed"] = mixed_workload(64, 56, 56, 2, (1024, 1024, 1000), 256, name
                                     grids=[(1, 1), (4, 4), (8, 1), (2, 8)])
 
 
+# Not a listed configuration: the layer shapes of the network of the paper's Section 3 (five convolutions: 11 x 11 stride 4,
+# 5 x 5, three 3 x 3; then a three-layer classifier), with what this library has in place of what it lacks: the three
+# input channels padded to 8, no channel groups, no normalisation, and the two later pooling stages as strides of the
+# second and fifth convolution (192 x 192 inputs: 48 x 48 after the first layer, 24 x 24, 12 x 12 at the classifier).
+WORKLOADS["alexlike"] = mixed_workload(8, 192, 192, 5, (4096, 4096, 1000), 128, name="alexlike",
+                                       grids=[(1, 1), (2, 8), (4, 4), (1, 16)],
+                                       ksizes=((11, 11), (5, 5), (3, 3), (3, 3), (3, 3)), channels=(8, 96, 256, 384, 384, 256),
+                                       strides=(4, 2, 1, 1, 2))
+
+
 # The layers the paper singles out as needing no halo exchange (remark after Eq. 7): cfg4's stack with 1 x 1 kernels.
 WORKLOADS["conv1x1"] = Workload("conv1x1", "conv", (64, 224, 224), 32, "bf16", "normal", "half_ssq", eta=1e-7,
                                 n_layers=2, grids=[(1, 1), (2, 1), (4, 1), (8, 1)], ksizes=(1, 1))

@@ -198,6 +198,21 @@ def test_master_weights_and_momentum_on_general_layers(master, mu):
     a.close(); b.close()
 
 
+@pytest.mark.parametrize("grid,mp,fused", [((1, 1), 1, True), ((3, 2), 2, False), ((2, 2), 4, True)])
+def test_layer_shapes_of_the_networks_of_section_3(grid, mp, fused):
+    # the `alexlike` workload of the benchmark in miniature: 11 x 11 stride 4 (8 -> 96 channels), 5 x 5 stride 2 (96 -> 256),
+    # 3 x 3 (256 -> 384 -> 384), 3 x 3 stride 2 (384 -> 256), then model-parallel fully connected layers, on 96 x 96 inputs
+    w = I.mixed_workload(8, 96, 96, 5, (64, 32, 16), 4, name="alexlike_small", ksizes=((11, 11), (5, 5), (3, 3), (3, 3), (3, 3)),
+                         channels=(8, 96, 256, 384, 384, 256), strides=(4, 2, 1, 1, 2))
+    assert w.fc_dims[0] == 256 * 6 * 6 and [w.out_hw(i) for i in range(5)] == [(24, 24), (12, 12), (12, 12), (12, 12), (6, 6)]
+    inp = I.make_inputs(w, seed=74)
+    o = oracle_mixed_step(w, inp)
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    o = oracle_with_eta(o, inp.Ws, inp.bs, w.B, eta)
+    g = gpu_mixed_step(w, inp, grid, mp, fused=fused, force_acts=oracle_mixed_acts(o, w), eta=eta)
+    compare_mixed_step(g, o, w, TOL, fused=fused, init=inp, require_sized=True)
+
+
 def test_unsupported_shapes_are_refused():
     from paper_1712_04432_b200 import mbd
     for kw in (dict(k=(4, 3)), dict(k=13), dict(channels=(12, 8, 8)), dict(channels=(8, 4, 8))):
