@@ -320,8 +320,9 @@ def run_ours(args):
 
     # Small workloads are dominated by launch cost: their timed steps replay the CUDA graph the
     # library captures (mbd_train_step); the per-kernel events then come from a second, directly
-    # launched pass.  The large workload launches directly with the events inside the timed region.
-    use_graph = flops < 1e12
+    # launched pass.  The large fully connected workload launches directly with the events inside the timed region
+    # (23 long kernels per step); a convolution stack has dozens of short launches whatever its size.
+    use_graph = flops < 1e12 or w.kind != "fc"
 
     def step():
         if flush is not None:
