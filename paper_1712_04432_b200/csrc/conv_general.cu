@@ -51,8 +51,18 @@ nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, 
     const int c = t >> 2, wq = (t & 3) * 8;           // channel c0 + c, pixels w0 + wq .. + 7
     if (c0 + c < C) {
       const bf16* q = src + ((static_cast<long long>(b) * C + c0 + c) * g.H + h) * g.W + w0 + wq;
+      if ((g.W & 7) == 0 && w0 + wq + 8 <= g.W && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {      // 16 aligned bytes
+        const uint4 v = __ldcs(reinterpret_cast<const uint4*>(q));
+        const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-      for (int j = 0; j < 8; ++j) tile[c][wq + j] = w0 + wq + j < g.W ? __bfloat16_as_ushort(q[j]) : 0;
+        for (int j = 0; j < 4; ++j) {
+          tile[c][wq + 2 * j] = static_cast<uint16_t>(wv[j] & 0xFFFFu);
+          tile[c][wq + 2 * j + 1] = static_cast<uint16_t>(wv[j] >> 16);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) tile[c][wq + j] = w0 + wq + j < g.W ? __bfloat16_as_ushort(q[j]) : 0;
+      }
     }
   }
   __syncthreads();
@@ -92,9 +102,16 @@ pix_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, 
   const int c = t >> 2, wq = (t & 3) * 8;
   if (c0 + c >= C) return;
   bf16* q = dst + ((static_cast<long long>(b) * C + c0 + c) * g.H + h) * g.W + w0 + wq;
+  if ((g.W & 7) == 0 && w0 + wq + 8 <= g.W && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+    uint4 v;
+    v.x = tile[c][wq + 0] | (static_cast<uint32_t>(tile[c][wq + 1]) << 16); v.y = tile[c][wq + 2] | (static_cast<uint32_t>(tile[c][wq + 3]) << 16);
+    v.z = tile[c][wq + 4] | (static_cast<uint32_t>(tile[c][wq + 5]) << 16); v.w = tile[c][wq + 6] | (static_cast<uint32_t>(tile[c][wq + 7]) << 16);
+    *reinterpret_cast<uint4*>(q) = v;
+  } else {
 #pragma unroll
-  for (int j = 0; j < 8; ++j)
-    if (w0 + wq + j < g.W) q[j] = __ushort_as_bfloat16(tile[c][wq + j]);
+    for (int j = 0; j < 8; ++j)
+      if (w0 + wq + j < g.W) q[j] = __ushort_as_bfloat16(tile[c][wq + j]);
+  }
 }
 
 // Everything that is not a strip's own pixel: the padding columns and the image's outer rows become zero; a halo
