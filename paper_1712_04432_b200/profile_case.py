@@ -38,6 +38,7 @@ def main():
     ap.add_argument("--image", type=int, default=224)
     ap.add_argument("--ksizes", default="3,3", help="conv: kernel size of each of the two layers (odd, up to 7)")
     ap.add_argument("--channels", default="64,64,64", help="conv: channels C_0,C_1,C_2 of the two layers (multiples of 8)")
+    ap.add_argument("--strides", default="1,1", help="conv: stride of each of the two layers (1 to 4)")
     ap.add_argument("--size", type=int, default=8192)
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--splits", type=int, default=2)
@@ -97,7 +98,8 @@ def conv_case(a):
     g = torch.Generator(device="cuda").manual_seed(0)
     ks = [int(k) for k in a.ksizes.split(",")]
     ch = [int(c) for c in a.channels.split(",")]
-    net = mbd.Net(mbd.conv_layers(2, ch[0], a.image, a.image, k=ks, channels=ch), a.batch, a.strips, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+    st = [int(x) for x in a.strides.split(",")]
+    net = mbd.Net(mbd.conv_layers(2, ch[0], a.image, a.image, k=ks, channels=ch, strides=st), a.batch, a.strips, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
     for i in range(2):
         K = (torch.randn((ch[i + 1], ch[i], ks[i], ks[i]), generator=g, device="cuda") * (2.0 / (ch[i] * ks[i] ** 2)) ** 0.5).to(torch.bfloat16)
         net.set_weights(i, K)
@@ -112,7 +114,7 @@ def conv_case(a):
     ev1.record()
     torch.cuda.synchronize()
     net.poll()
-    print(f"conv batch={a.batch} image={a.image} strips={a.strips} kernels={ks} channels={ch}: {ev0.elapsed_time(ev1) / a.launches:.3f} ms per step, J = {J.item():.4e}")
+    print(f"conv batch={a.batch} image={a.image} strips={a.strips} kernels={ks} channels={ch} strides={st}: {ev0.elapsed_time(ev1) / a.launches:.3f} ms per step, J = {J.item():.4e}")
 
 
 if __name__ == "__main__":
