@@ -335,9 +335,12 @@ MBD_API int64_t mbd_launch_count(const mbd_net* net);
  * k_pieces > 1 means a reduce_partials launch follows; tma_epilogue = 1: the tail operation the plan was made for (bias +
  * ReLU, ReLU mask, fused update) moves its global data by TMA; tma_epilogue = 2: the k_pieces fp32 partial sums are
  * stored by TMA (short pieces on 128-row tiles); ctas: CTAs launched.
- * MBD_E_UNSUPPORTED for fp32 networks and convolution layers, MBD_E_INVALID for a product the layer
- * does not have (backward-data of the network's first layer). */
-typedef struct { int32_t tile_m, tile_n, cta_pair, k_pieces, tma_epilogue, ctas, running_sum, reserved; } mbd_plan;
+ * k_blocks: 64-deep blocks of the product's K range (for a general convolution layer (taps x channel blocks), or its
+ * tap runs when a first layer with few input channels folds several taps into one block).
+ * MBD_E_UNSUPPORTED for fp32 networks and for the convolution layers that run on kernels of their own (64 channels,
+ * 3x3 / 1x1, stride 1), MBD_E_INVALID for a product the layer does not have (backward-data of the network's first
+ * layer). */
+typedef struct { int32_t tile_m, tile_n, cta_pair, k_pieces, tma_epilogue, ctas, running_sum, k_blocks; } mbd_plan;
 MBD_API mbd_status mbd_get_plan(const mbd_net* net, int layer, int product, mbd_plan* out_host);
 
 /* Stand-alone dense contraction on the tensor cores, used by the unit tests:

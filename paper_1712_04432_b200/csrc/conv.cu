@@ -1309,6 +1309,10 @@ mbd_status conv_outer_rows(ConvNet* c, int which, int layer, int side, void* row
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
+mbd_status conv_get_product(const ConvNet* c, int layer, int product, const TcGemm** out) {
+  return c->gen ? gconv_get_product(c->gen, layer, product, out) : MBD_E_UNSUPPORTED;
+}
+
 mbd_status conv_set_dw(ConvNet* c, int layer, const void* src, size_t bytes) {
   if (c->gen) return gconv_set_dw(c->gen, layer, src, bytes);
   if (layer < 0 || layer >= c->L) return MBD_E_INVALID;

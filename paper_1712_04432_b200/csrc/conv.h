@@ -33,4 +33,7 @@ mbd_status conv_forward_layer(ConvNet* c, int layer, float* loss_sum_dev, int ro
 mbd_status conv_backward_layer(ConvNet* c, int layer, float fused_eta, int rows);
 mbd_status conv_outer_rows(ConvNet* c, int which, int layer, int side, void* rows, size_t bytes, int set);
 mbd_status conv_set_dw(ConvNet* c, int layer, const void* src, size_t bytes);
+// the contraction a general convolution layer launches for `product` (0 forward, 1 backward-data, 2 backward-weight);
+// MBD_E_UNSUPPORTED for the layers that run on the convolution kernels of their own
+mbd_status conv_get_product(const ConvNet* c, int layer, int product, const TcGemm** out);
 }  // namespace mbd

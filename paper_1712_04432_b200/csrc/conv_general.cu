@@ -177,33 +177,29 @@ ssq_partial_kernel(const bf16* __restrict__ T, long long n8, float* __restrict__
   if (threadIdx.x == 0) part[blockIdx.x] = sh[0];
 }
 
-// Public kernel K[o][c][u][v]  <->  internal Wm[o][t = u kw + v][c padded to Cp].
-__global__ void pack_w_kernel(const bf16* __restrict__ K, bf16* __restrict__ Wm, int Cout, int Cin, int taps, int Cp) {
-  const long long n = static_cast<long long>(Cout) * taps * Cp;
+// Public kernel K[o][c][u][v]  <->  internal Wm[o][j], j < ldw.  `colmap[j]` = t * Cin + c (t = u kw + v) for the kernel
+// element that column j holds, or -1 for a padding column (a zero weight that stays zero).  Unfolded layers:
+// j = t * Cp + c with the channels padded to Cp; a folded first layer: j = run * 64 + g * Cin + c (see fold_runs).
+template <typename T>
+__global__ void pack_w_kernel(const T* __restrict__ K, T* __restrict__ Wm, const int* __restrict__ colmap, int Cout, int Cin, int taps, int ldw) {
+  const long long n = static_cast<long long>(Cout) * ldw;
   for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
-    const int c = static_cast<int>(i % Cp);
-    const int t = static_cast<int>((i / Cp) % taps);
-    const int o = static_cast<int>(i / (static_cast<long long>(Cp) * taps));
-    Wm[i] = c < Cin ? K[(static_cast<long long>(o) * Cin + c) * taps + t] : __float2bfloat16(0.f);
+    const int j = static_cast<int>(i % ldw);
+    const int o = static_cast<int>(i / ldw);
+    const int m = colmap[j];
+    T v = T(0.f);
+    if (m >= 0) v = K[(static_cast<long long>(o) * Cin + m % Cin) * taps + m / Cin];
+    Wm[i] = v;
   }
 }
 template <typename T>
-__global__ void unpack_w_kernel(const T* __restrict__ Wm, T* __restrict__ K, int Cout, int Cin, int taps, int Cp) {
-  const long long n = static_cast<long long>(Cout) * Cin * taps;
+__global__ void unpack_w_kernel(const T* __restrict__ Wm, T* __restrict__ K, const int* __restrict__ colmap, int Cout, int Cin, int taps, int ldw) {
+  const long long n = static_cast<long long>(Cout) * ldw;
   for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
-    const int t = static_cast<int>(i % taps);
-    const int c = static_cast<int>((i / taps) % Cin);
-    const int o = static_cast<int>(i / (static_cast<long long>(taps) * Cin));
-    K[i] = Wm[(static_cast<long long>(o) * taps + t) * Cp + c];
-  }
-}
-__global__ void pack_dw_kernel(const float* __restrict__ K, float* __restrict__ Wm, int Cout, int Cin, int taps, int Cp) {
-  const long long n = static_cast<long long>(Cout) * taps * Cp;
-  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
-    const int c = static_cast<int>(i % Cp);
-    const int t = static_cast<int>((i / Cp) % taps);
-    const int o = static_cast<int>(i / (static_cast<long long>(Cp) * taps));
-    Wm[i] = c < Cin ? K[(static_cast<long long>(o) * Cin + c) * taps + t] : 0.f;
+    const int j = static_cast<int>(i % ldw);
+    const int o = static_cast<int>(i / ldw);
+    const int m = colmap[j];
+    if (m >= 0) K[(static_cast<long long>(o) * Cin + m % Cin) * taps + m / Cin] = Wm[i];
   }
 }
 
@@ -246,6 +242,9 @@ struct GenConv {
   int P_r = 1, P = 1, S = 1;              // strips; processes of the grid; fp32 partial sums per weight gradient asked for
   std::vector<Geo> geo;                   // geometry of tensor i (act[i]; dY[i] has that of act[i + 1])
   std::vector<int> Cin, Cout, kh, kw, relu, taps, Cp, stride;
+  std::vector<int> ldw;                   // columns of the internal weight matrix of layer i
+  std::vector<int*> colmap;               // device: column -> kernel element (see pack_w_kernel)
+  std::vector<int> folded;                // layer 0 with few input channels: several taps per 64-wide k-block (fold_runs)
   std::vector<bf16*> act, dY, Wm;
   std::vector<bf16*> xph, dxph;           // strided layers: phase planes of the input / of the gradient below
   std::vector<float*> dWm;
@@ -329,6 +328,35 @@ void tap_offsets(int kh, int kw, int s, const Geo& g, int* off, int* plane) {
     }
 }
 
+// A first layer with few input channels (8, 16 or 32) would fill an eighth to a half of a 64-wide k-block per tap.  Its
+// input is pixel-major, so the channels of G = 64 / C_in CONSECUTIVE pixels are 64 contiguous elements: through a
+// tensor map whose rows overlap (row pitch = one pixel = C_in elements, row length 64) one TMA box holds the operands
+// of G horizontally adjacent taps at once.  A run = up to G taps of one kernel row that read the same phase plane at
+// consecutive pixels; the k-blocks of the folded layer are its runs (columns of absent taps carry zero weights).
+struct Run { int plane, off, n, tap[8]; };
+std::vector<Run> fold_runs(int kh, int kw, int s, int Cin, const Geo& g) {
+  int off[MAX_TAPS], plane[MAX_TAPS];
+  tap_offsets(kh, kw, s, g, off, plane);
+  const int G = 64 / Cin;
+  std::vector<Run> runs;
+  std::vector<char> used(kh * kw, 0);
+  for (int t = 0; t < kh * kw; ++t) {
+    if (used[t]) continue;
+    Run r{};
+    r.plane = plane[t]; r.off = off[t]; r.n = 0;
+    for (int g2 = 0; g2 < G; ++g2) r.tap[g2] = -1;
+    // taps of the same kernel row (same u) in the same plane, at this tap's pixel + 0 .. G-1
+    for (int t2 = t; t2 < kh * kw && t2 / kw == t / kw; ++t2)
+      if (!used[t2] && plane[t2] == r.plane && off[t2] - r.off >= 0 && off[t2] - r.off < G) {
+        r.tap[off[t2] - r.off] = t2;
+        used[t2] = 1;
+        ++r.n;
+      }
+    runs.push_back(r);
+  }
+  return runs;
+}
+
 }  // namespace
 
 bool gconv_needed(const mbd_layer* layers, int L) {
@@ -347,6 +375,7 @@ void gconv_destroy(GenConv* c) {
   for (size_t i = 0; i < c->dY.size(); ++i)
     if (c->dY[i] && (c->act.size() <= static_cast<size_t>(c->L) || c->dY[i] != c->act[c->L])) cudaFree(c->dY[i]);
   for (bf16* p : c->Wm) cudaFree(p);
+  for (int* p : c->colmap) cudaFree(p);
   for (bf16* p : c->xph) cudaFree(p);
   for (bf16* p : c->dxph) cudaFree(p);
   for (float* p : c->dWm) cudaFree(p);
@@ -404,19 +433,48 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
     c->relu.push_back((i == L - 1 && !fc_above) ? 0 : l.relu);
     c->taps.push_back(l.kh * l.kw); c->Cp.push_back(round64(l.C_in));
   }
+  // (256 bytes of slack behind the tensors a folded layer reads: its last rows reach up to 64 - C_in elements further)
   for (int i = 0; i <= L && ok; ++i) {
     const int C = i == 0 ? c->Cin[0] : c->Cout[i - 1];
-    ok = alloc(reinterpret_cast<void**>(&c->act[i]), static_cast<size_t>(c->geo[i].Ptot) * C * 2);
+    ok = alloc(reinterpret_cast<void**>(&c->act[i]), static_cast<size_t>(c->geo[i].Ptot) * C * 2 + 256);
+  }
+  // internal weight layouts
+  c->ldw.assign(L, 0); c->colmap.assign(L, nullptr); c->folded.assign(L, 0);
+  std::vector<std::vector<Run>> runs(L);
+  for (int i = 0; i < L && ok; ++i) {
+    const int Cin = c->Cin[i], taps = c->taps[i], Cp = c->Cp[i];
+    std::vector<int> map;
+    const bool fold = i == 0 && (Cin == 8 || Cin == 16 || Cin == 32) && taps > 1 && !getenv("MBD_CONV_NO_FOLD");      // tuning knob
+    if (fold) {
+      runs[i] = fold_runs(c->kh[i], c->kw[i], c->stride[i], Cin, c->geo[i + 1]);
+      if (static_cast<int>(runs[i].size()) <= MAX_TAPS && static_cast<int>(runs[i].size()) * 64 < taps * Cp) {
+        c->folded[i] = 1;
+        map.assign(runs[i].size() * 64, -1);
+        for (size_t r = 0; r < runs[i].size(); ++r)
+          for (int g2 = 0; g2 < 64 / Cin; ++g2)
+            if (runs[i][r].tap[g2] >= 0)
+              for (int ch = 0; ch < Cin; ++ch) map[r * 64 + g2 * Cin + ch] = runs[i][r].tap[g2] * Cin + ch;
+      }
+    }
+    if (!c->folded[i]) {
+      map.assign(static_cast<size_t>(taps) * Cp, -1);
+      for (int t = 0; t < taps; ++t)
+        for (int ch = 0; ch < Cin; ++ch) map[static_cast<size_t>(t) * Cp + ch] = t * Cin + ch;
+    }
+    c->ldw[i] = static_cast<int>(map.size());
+    ok = alloc(reinterpret_cast<void**>(&c->colmap[i]), map.size() * sizeof(int)) &&
+         cudaMemcpyAsync(c->colmap[i], map.data(), map.size() * sizeof(int), cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+         cudaStreamSynchronize(stream) == cudaSuccess;          // `map` is a local
   }
   for (int i = 0; i < L && ok; ++i) {
     const Geo& go = c->geo[i + 1];
     if (i < L - 1 || fc_above) ok = alloc(reinterpret_cast<void**>(&c->dY[i]), static_cast<size_t>(go.Ptot) * c->Cout[i] * 2);
     else c->dY[i] = c->act[L];                       // half-SSQ loss: dY_L = Y_L
-    const size_t nw = static_cast<size_t>(c->Cout[i]) * c->taps[i] * c->Cp[i];
+    const size_t nw = static_cast<size_t>(c->Cout[i]) * c->ldw[i];
     ok = ok && alloc(reinterpret_cast<void**>(&c->Wm[i]), nw * 2) && alloc(reinterpret_cast<void**>(&c->dWm[i]), nw * 4);
     if (c->stride[i] > 1) {
       const size_t pl = static_cast<size_t>(c->stride[i]) * c->stride[i] * go.Ptot * c->Cin[i] * 2;
-      ok = ok && alloc(reinterpret_cast<void**>(&c->xph[i]), pl);
+      ok = ok && alloc(reinterpret_cast<void**>(&c->xph[i]), pl + 256);
       if (i > 0) ok = ok && alloc(reinterpret_cast<void**>(&c->dxph[i]), pl);
     }
   }
@@ -426,7 +484,7 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
   size_t part_elems = 0;
   for (int i = 0; i < L; ++i) {
     const int Cin = c->Cin[i], Cout = c->Cout[i], taps = c->taps[i], Cp = c->Cp[i], Cop = round64(Cout), s = c->stride[i];
-    const int ldw = taps * Cp;
+    const int ldw = c->ldw[i];
     const Geo& go = c->geo[i + 1];                   // the products run over the pixels of the layer's output geometry
     const int M = static_cast<int>(go.Ptot);
     bf16* xin = s > 1 ? c->xph[i] : c->act[i];       // what the forward and weight-gradient products read
@@ -435,10 +493,18 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
     // forward
     TcGemm& f = c->fwd[i];
     f = TcGemm{};
-    f.variant = 0; f.M = M; f.N = Cout; f.K = taps * Cp; f.k_splits = 1; f.status = status;
-    f.cv.mode = 1; f.cv.taps = taps; f.cv.blocks = Cp / 64; f.cv.Cp = Cp;
-    for (int t = 0; t < taps; ++t) { f.cv.off[t] = plane[t] * M + off[t]; f.cv.tap[t] = t; }
-    f.cv_a_inner = Cin; f.cv_a_rows = static_cast<int64_t>(s) * s * M;
+    f.variant = 0; f.M = M; f.N = Cout; f.K = ldw; f.k_splits = 1; f.status = status;
+    f.cv.mode = 1;
+    if (c->folded[i]) {            // k-block = run; the A rows are the overlapping 64-element windows of the pixel-major input
+      f.cv.taps = static_cast<int>(runs[i].size()); f.cv.blocks = 1; f.cv.Cp = 64;
+      for (int r = 0; r < f.cv.taps; ++r) { f.cv.off[r] = runs[i][r].plane * M + runs[i][r].off; f.cv.tap[r] = r; }
+      f.cv_a_inner = 64;
+    } else {
+      f.cv.taps = taps; f.cv.blocks = Cp / 64; f.cv.Cp = Cp;
+      for (int t = 0; t < taps; ++t) { f.cv.off[t] = plane[t] * M + off[t]; f.cv.tap[t] = t; }
+      f.cv_a_inner = Cin;
+    }
+    f.cv_a_rows = static_cast<int64_t>(s) * s * M;
     const Epi ef = make_epi_act(c->act[i + 1], Cout, 1, c->relu[i]);
     if (tc_gemm_prepare(f, xin, Cin, c->Wm[i], ldw, num_sms, &ef) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
     // backward-data: one product (stride 1), or one per phase plane with the taps that read that plane
@@ -469,9 +535,17 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
     w = TcGemm{};
     w.variant = 2; w.M = Cout; w.N = ldw; w.K = M; w.k_splits = c->S; w.status = status;
     w.allow_extra_split = 1;
-    w.cv.mode = 3; w.cv.taps = taps; w.cv.blocks = 0; w.cv.Cp = Cp;
-    for (int t = 0; t < taps; ++t) { w.cv.off[t] = plane[t] * M + off[t]; w.cv.tap[t] = t; }
-    w.cv_b_inner = Cin; w.cv_b_rows = static_cast<int64_t>(s) * s * M;
+    w.cv.mode = 3; w.cv.blocks = 0;
+    if (c->folded[i]) {
+      w.cv.taps = static_cast<int>(runs[i].size()); w.cv.Cp = 64;
+      for (int r = 0; r < w.cv.taps; ++r) { w.cv.off[r] = runs[i][r].plane * M + runs[i][r].off; w.cv.tap[r] = r; }
+      w.cv_b_inner = 64;
+    } else {
+      w.cv.taps = taps; w.cv.Cp = Cp;
+      for (int t = 0; t < taps; ++t) { w.cv.off[t] = plane[t] * M + off[t]; w.cv.tap[t] = t; }
+      w.cv_b_inner = Cin;
+    }
+    w.cv_b_rows = static_cast<int64_t>(s) * s * M;
     const Epi ew = make_epi_sgd(c->Wm[i], ldw, 0.f);
     if (tc_gemm_prepare(w, c->dY[i], Cout, xin, Cin, num_sms, &ew) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
     if (w.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(w.k_splits) * Cout * ldw);
@@ -486,8 +560,8 @@ size_t gconv_input_bytes(const GenConv* c) { return static_cast<size_t>(c->B) * 
 int gconv_last_relu(const GenConv* c) { return c->relu[c->L - 1]; }
 
 mbd_status gconv_set_weights(GenConv* c, int i, const void* K_dev) {
-  const long long n = static_cast<long long>(c->Cout[i]) * c->taps[i] * c->Cp[i];
-  pack_w_kernel<<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(static_cast<const bf16*>(K_dev), c->Wm[i], c->Cout[i], c->Cin[i], c->taps[i], c->Cp[i]);
+  const long long n = static_cast<long long>(c->Cout[i]) * c->ldw[i];
+  pack_w_kernel<bf16><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(static_cast<const bf16*>(K_dev), c->Wm[i], c->colmap[i], c->Cout[i], c->Cin[i], c->taps[i], c->ldw[i]);
   if (!c->Wm32.empty() && widen_bf16_launch(c->Wm[i], c->Wm32[i], n, c->num_sms, c->stream) != cudaSuccess) return MBD_E_CUDA;
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
@@ -498,7 +572,7 @@ mbd_status gconv_enable_master(GenConv* c) {
   if (!c->Wm32.empty()) return MBD_OK;
   std::vector<float*> m(c->L, nullptr);
   for (int i = 0; i < c->L; ++i) {
-    const long long n = static_cast<long long>(c->Cout[i]) * c->taps[i] * c->Cp[i];
+    const long long n = static_cast<long long>(c->Cout[i]) * c->ldw[i];
     if (cudaMalloc(reinterpret_cast<void**>(&m[i]), n * 4) != cudaSuccess || widen_bf16_launch(c->Wm[i], m[i], n, c->num_sms, c->stream) != cudaSuccess) {
       (void)cudaGetLastError();
       for (float* q : m) cudaFree(q);
@@ -513,7 +587,7 @@ mbd_status gconv_enable_momentum(GenConv* c, float mu) {
   if (c->Vm.empty()) {
     std::vector<float*> v(c->L, nullptr);
     for (int i = 0; i < c->L; ++i)
-      if (cudaMalloc(reinterpret_cast<void**>(&v[i]), static_cast<size_t>(c->Cout[i]) * c->taps[i] * c->Cp[i] * 4) != cudaSuccess) {
+      if (cudaMalloc(reinterpret_cast<void**>(&v[i]), static_cast<size_t>(c->Cout[i]) * c->ldw[i] * 4) != cudaSuccess) {
         (void)cudaGetLastError();
         for (float* q : v) cudaFree(q);
         return MBD_E_ALLOC;
@@ -521,7 +595,7 @@ mbd_status gconv_enable_momentum(GenConv* c, float mu) {
     c->Vm = v;
   }
   for (int i = 0; i < c->L; ++i)
-    if (cudaMemsetAsync(c->Vm[i], 0, static_cast<size_t>(c->Cout[i]) * c->taps[i] * c->Cp[i] * 4, c->stream) != cudaSuccess) return MBD_E_CUDA;
+    if (cudaMemsetAsync(c->Vm[i], 0, static_cast<size_t>(c->Cout[i]) * c->ldw[i] * 4, c->stream) != cudaSuccess) return MBD_E_CUDA;
   c->mu = mu;
   return MBD_OK;
 }
@@ -529,7 +603,7 @@ mbd_status gconv_enable_momentum(GenConv* c, float mu) {
 namespace {
 // Eq. 1 (or its momentum form) from the materialised gradient of layer i
 mbd_status update_from_gradient(GenConv* c, int i, float eta) {
-  const long long n = static_cast<long long>(c->Cout[i]) * c->taps[i] * c->Cp[i];
+  const long long n = static_cast<long long>(c->Cout[i]) * c->ldw[i];
   const float scale = -eta / static_cast<float>(c->B);
   float* w32 = c->Wm32.empty() ? nullptr : c->Wm32[i];
   c->prof->begin(MBD_K_SGD, static_cast<double>(n) * (8.0 + (w32 ? 8.0 : 0.0) + (c->Vm.empty() ? 0.0 : 8.0)), c->stream);
@@ -542,8 +616,8 @@ mbd_status update_from_gradient(GenConv* c, int i, float eta) {
 }
 }  // namespace
 mbd_status gconv_get_weights(GenConv* c, int i, void* K_dev) {
-  const long long n = static_cast<long long>(c->Cout[i]) * c->Cin[i] * c->taps[i];
-  unpack_w_kernel<bf16><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(c->Wm[i], static_cast<bf16*>(K_dev), c->Cout[i], c->Cin[i], c->taps[i], c->Cp[i]);
+  const long long n = static_cast<long long>(c->Cout[i]) * c->ldw[i];
+  unpack_w_kernel<bf16><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(c->Wm[i], static_cast<bf16*>(K_dev), c->colmap[i], c->Cout[i], c->Cin[i], c->taps[i], c->ldw[i]);
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
@@ -609,7 +683,7 @@ mbd_status gconv_backward_layer(GenConv* c, int i, float fused_eta) {
   const Geo& go = c->geo[i + 1];
   const int s = c->stride[i], Cin = c->Cin[i];
   const double flops = 2.0 * c->B * go.H * go.W * c->taps[i] * Cin * c->Cout[i];
-  const int ldw = c->taps[i] * c->Cp[i];
+  const int ldw = c->ldw[i];
   if (i > 0) {
     // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0] -- with the
     // weights as they are BEFORE this step's update, so this product comes first
@@ -668,8 +742,8 @@ mbd_status gconv_get_tensor(GenConv* c, int which, int layer, void* dst, size_t 
     if (bytes != static_cast<size_t>(n) * 4) return MBD_E_INVALID;
     if ((which == MBD_T_MASTER && c->Wm32.empty()) || (which == MBD_T_VELOCITY && c->Vm.empty())) return MBD_E_STATE;
     const float* src32 = which == MBD_T_DW ? c->dWm[layer] : which == MBD_T_MASTER ? c->Wm32[layer] : c->Vm[layer];
-    unpack_w_kernel<float><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(src32, static_cast<float*>(dst), c->Cout[layer], c->Cin[layer],
-                                                                          c->taps[layer], c->Cp[layer]);
+    unpack_w_kernel<float><<<grid_1d(static_cast<long long>(c->Cout[layer]) * c->ldw[layer], c->num_sms), 256, 0, c->stream>>>(
+        src32, static_cast<float*>(dst), c->colmap[layer], c->Cout[layer], c->Cin[layer], c->taps[layer], c->ldw[layer]);
     return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
   }
   if (which != MBD_T_ACT && which != MBD_T_DY) return MBD_E_INVALID;
@@ -696,12 +770,24 @@ mbd_status gconv_set_tensor(GenConv* c, int which, int layer, const void* src, s
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
+mbd_status gconv_get_product(const GenConv* c, int layer, int product, const TcGemm** out) {
+  if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
+  if (product == 1 && layer == 0) return MBD_E_INVALID;                 // nothing is propagated below the first layer
+  if (product == 1) {                                                   // (a strided layer: the first plane that has taps)
+    for (size_t q = 0; q < c->bwd_data[layer].size(); ++q)
+      if (c->bwd_taps[layer][q] > 0) { *out = &c->bwd_data[layer][q]; return MBD_OK; }
+    return MBD_E_INVALID;
+  }
+  *out = product == 0 ? &c->fwd[layer] : &c->bwd_weight[layer];
+  return MBD_OK;
+}
+
 mbd_status gconv_set_dw(GenConv* c, int layer, const void* src, size_t bytes) {
   if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
-  const long long n = static_cast<long long>(c->Cout[layer]) * c->taps[layer] * c->Cp[layer];
+  const long long n = static_cast<long long>(c->Cout[layer]) * c->ldw[layer];
   if (bytes != static_cast<size_t>(c->Cout[layer]) * c->Cin[layer] * c->taps[layer] * 4) return MBD_E_INVALID;
-  pack_dw_kernel<<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(static_cast<const float*>(src), c->dWm[layer], c->Cout[layer], c->Cin[layer],
-                                                                c->taps[layer], c->Cp[layer]);
+  pack_w_kernel<float><<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(static_cast<const float*>(src), c->dWm[layer], c->colmap[layer], c->Cout[layer],
+                                                                      c->Cin[layer], c->taps[layer], c->ldw[layer]);
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 

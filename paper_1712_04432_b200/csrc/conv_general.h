@@ -27,6 +27,7 @@ mbd_status gconv_enable_momentum(GenConv* c, float mu);     // heavy-ball moment
 mbd_status gconv_get_tensor(GenConv* c, int which, int layer, void* dst, size_t bytes);
 mbd_status gconv_set_tensor(GenConv* c, int which, int layer, const void* src, size_t bytes);
 mbd_status gconv_set_dw(GenConv* c, int layer, const void* src, size_t bytes);
+mbd_status gconv_get_product(const GenConv* c, int layer, int product, const TcGemm** out);
 mbd_status gconv_output_to_nchw(GenConv* c, void* dst);
 mbd_status gconv_top_grad_from_nchw(GenConv* c, const void* src);
 size_t gconv_input_bytes(const GenConv* c);

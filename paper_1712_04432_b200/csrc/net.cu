@@ -973,11 +973,18 @@ extern "C" int64_t mbd_launch_count(const mbd_net* n) { return n ? n->prof.total
 extern "C" mbd_status mbd_get_plan(const mbd_net* n, int layer, int product, mbd_plan* out) {
   if (!n || !out || product < 0 || product > 2) return MBD_E_INVALID;
   if (layer < 0 || layer >= n->Lc + n->L) return MBD_E_INVALID;
-  if (n->dtype != MBD_BF16 || layer < n->Lc) return MBD_E_UNSUPPORTED;
-  const int i = layer - n->Lc;
-  if (product == 1 && i == 0 && !n->mixed) return MBD_E_INVALID;
-  const Layer& l = n->layers[i];
-  const TcGemm& g = product == 0 ? l.fwd : product == 1 ? l.bwd_data : l.bwd_weight;
+  if (n->dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
+  const TcGemm* gp = nullptr;
+  if (layer < n->Lc) {
+    const mbd_status s = conv_get_product(n->conv, layer, product, &gp);     // general convolution layers only
+    if (s != MBD_OK) return s;
+  } else {
+    const int i = layer - n->Lc;
+    if (product == 1 && i == 0 && !n->mixed) return MBD_E_INVALID;
+    const Layer& l = n->layers[i];
+    gp = product == 0 ? &l.fwd : product == 1 ? &l.bwd_data : &l.bwd_weight;
+  }
+  const TcGemm& g = *gp;
   out->tile_m = 128 * g.MH * (g.pair ? 2 : 1);
   out->tile_n = g.BN;
   out->cta_pair = g.pair;
@@ -985,7 +992,7 @@ extern "C" mbd_status mbd_get_plan(const mbd_net* n, int layer, int product, mbd
   out->tma_epilogue = g.te_planes ? 2 : g.te;
   out->ctas = g.grid;
   out->running_sum = g.join > 1 ? 2 : g.fix;
-  out->reserved = 0;
+  out->k_blocks = (g.K + 63) / 64;
   return MBD_OK;
 }
 

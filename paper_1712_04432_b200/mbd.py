@@ -60,7 +60,7 @@ class Tail(C.Structure):
 class Plan(C.Structure):
     """mbd_plan: how one product of a layer is launched (see include/mbd.h)."""
     _fields_ = [("tile_m", C.c_int32), ("tile_n", C.c_int32), ("cta_pair", C.c_int32), ("k_pieces", C.c_int32),
-                ("tma_epilogue", C.c_int32), ("ctas", C.c_int32), ("running_sum", C.c_int32), ("reserved", C.c_int32)]
+                ("tma_epilogue", C.c_int32), ("ctas", C.c_int32), ("running_sum", C.c_int32), ("k_blocks", C.c_int32)]
 
 
 class Words(C.Structure):

@@ -213,6 +213,41 @@ def test_layer_shapes_of_the_networks_of_section_3(grid, mp, fused):
     compare_mixed_step(g, o, w, TOL, fused=fused, init=inp, require_sized=True)
 
 
+@pytest.mark.parametrize("name,Cin,k,s,blocks_folded,blocks_plain", [
+    ("3x3", 8, (3, 3), 1, 3, 9),              # a row of three taps of 8 channels fits one 64-wide block
+    ("7x7", 16, (7, 7), 1, 14, 49),           # four taps of 16 channels per block: two blocks per kernel row
+    ("11x11 stride 4", 8, (11, 11), 4, 44, 121),    # 16 phase planes, up to three taps of a row per plane
+    ("5x5 stride 2", 32, (5, 5), 2, 15, 25)])
+def test_first_layer_with_few_channels_folds_its_taps(monkeypatch, name, Cin, k, s, blocks_folded, blocks_plain):
+    # The input is pixel-major, so the channels of consecutive pixels are contiguous: through a tensor map whose rows
+    # overlap, one 64-element operand row holds 64 / C_in horizontally adjacent taps.  Fewer, fuller k-blocks, the
+    # same sums: both forms against the oracle, and against each other far below the tolerance.
+    from paper_1712_04432_b200 import mbd
+    H, W, B = 8 * s * 2, 12 * s, 3
+    w = I.conv_workload(Cin, H, W, B, n_layers=2, name="fold", ksizes=(k, (3, 3)), channels=(Cin, 40, 24), strides=(s, 1))
+    inp = I.make_inputs(w, seed=75)
+    o = oracle_conv_step(w, inp)
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    o = oracle_with_eta(o, inp.Ws, inp.bs, w.B, eta)
+    res = {}
+    for fold in (True, False):
+        if not fold:
+            monkeypatch.setenv("MBD_CONV_NO_FOLD", "1")
+        net = mbd.Net(mbd.conv_layers(2, Cin, H, W, k=[k, (3, 3)], channels=(Cin, 40, 24), strides=(s, 1)), B, 2, 1, mbd.BF16,
+                      mbd.LOSS_HALF_SSQ, 2)
+        want = blocks_folded if fold else blocks_plain
+        assert net.plan(0, 0)["k_blocks"] == want, (name, net.plan(0, 0))
+        assert net.plan(0, 2)["ctas"] > 0 and net.plan(1, 0)["k_blocks"] == 9           # 40 channels: one block per tap
+        net.close()
+        for fused in (False, True):
+            g = gpu_conv_step(w, inp, 2, fused=fused, force_acts=stored_hidden(o), eta=eta, max_partials=2)
+            compare_conv_step(g, o, TOL, fused, init=inp, require_sized=True)
+            res[(fold, fused)] = g
+    a, b = res[(True, False)], res[(False, False)]
+    for i in range(2):
+        assert rel_fro(a["act"][i], b["act"][i]) < 5e-3 and rel_fro(a["dW"][i], b["dW"][i]) < 1e-3, (name, i)
+
+
 def test_unsupported_shapes_are_refused():
     from paper_1712_04432_b200 import mbd
     for kw in (dict(k=(4, 3)), dict(k=13), dict(channels=(12, 8, 8)), dict(channels=(8, 4, 8))):
