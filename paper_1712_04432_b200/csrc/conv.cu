@@ -251,15 +251,16 @@ wgrad_finish_kernel(const float* __restrict__ part, int G, float* __restrict__ d
   const int i = blockIdx.x * 64 + j;
   const int g0 = (q * G) / 4, g1 = ((q + 1) * G) / 4;
   float s = 0.f;
-  int g = g0;
-  for (; g + 8 <= g1; g += 8) {
-    float v[8];
+  // twelve loads in flight per thread, the ragged tail as guarded loads of the same batch (a tail of dependent single
+  // loads had cost as many round trips as the batches before it); the additions keep their ascending order
+  for (int g = g0; g < g1; g += 12) {
+    float v[12];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) v[e] = __ldcs(part + static_cast<int64_t>(g + e) * 9 * C * C + i);
+    for (int e = 0; e < 12; ++e) v[e] = g + e < g1 ? __ldcs(part + static_cast<int64_t>(g + e) * 9 * C * C + i) : 0.f;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) s += v[e];
+    for (int e = 0; e < 12; ++e)
+      if (g + e < g1) s += v[e];
   }
-  for (; g < g1; ++g) s += part[static_cast<int64_t>(g) * 9 * C * C + i];
   sub[q][j] = s;
   __syncthreads();
   if (q != 0) return;
