@@ -248,6 +248,23 @@ def test_first_layer_with_few_channels_folds_its_taps(monkeypatch, name, Cin, k,
         assert rel_fro(a["act"][i], b["act"][i]) < 5e-3 and rel_fro(a["dW"][i], b["dW"][i]) < 1e-3, (name, i)
 
 
+@pytest.mark.parametrize("ch,ks,st,H,W,B,P_r,P_c", [
+    ((8, 8), ((7, 7),), (1,), 4, 4, 1, 1, 1),                # an image smaller than its kernel, one sample
+    ((24, 16, 8), ((3, 5), (1, 1)), (1, 1), 5, 37, 5, 1, 5),  # odd width, one sample per batch block
+    ((8, 72), ((9, 1),), (1,), 16, 3, 2, 2, 1),              # three pixels per row, a tall kernel, two strips of 8 rows
+    ((16, 8), ((3, 3),), (4,), 8, 8, 3, 2, 1),               # stride 4 down to 2 x 2 outputs, strips of one row
+    ((32, 40), ((5, 5),), (2,), 4, 6, 2, 1, 2)])             # stride 2 on a 4 x 6 image
+def test_small_and_ragged_shapes(ch, ks, st, H, W, B, P_r, P_c):
+    w = I.conv_workload(ch[0], H, W, B, n_layers=len(ks), name="edge", ksizes=ks, channels=ch, strides=st)
+    inp = I.make_inputs(w, seed=76)
+    o = oracle_conv_step(w, inp)
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    o = oracle_with_eta(o, inp.Ws, inp.bs, w.B, eta)
+    for fused in (False, True):
+        g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o), P_c=P_c, eta=eta, max_partials=2)
+        compare_conv_step(g, o, TOL, fused, init=inp, require_sized=True)
+
+
 def test_unsupported_shapes_are_refused():
     from paper_1712_04432_b200 import mbd
     for kw in (dict(k=(4, 3)), dict(k=13), dict(channels=(12, 8, 8)), dict(channels=(8, 4, 8))):
