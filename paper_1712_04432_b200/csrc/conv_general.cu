@@ -209,7 +209,7 @@ __global__ void unpack_w_kernel(const T* __restrict__ Wm, T* __restrict__ K, con
 // stride-1 product over shifted views again, with no position computed that is not kept.
 // decimate: own pixels of T (geometry gi) -> planes P[s^2][go.Ptot][C]; undecimate: the way back (a gradient).
 __global__ void __launch_bounds__(256)
-decimate_kernel(const bf16* __restrict__ T, bf16* __restrict__ P, Geo gi, Geo go, int C, int s, int to_planes) {
+decimate_kernel(bf16* __restrict__ T, bf16* __restrict__ P, Geo gi, Geo go, int C, int s, int to_planes) {
   const int c8 = C / 8;
   const long long total = gi.Z * gi.Hs * gi.W * c8;
   for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
@@ -222,7 +222,7 @@ decimate_kernel(const bf16* __restrict__ T, bf16* __restrict__ P, Geo gi, Geo go
     const long long pin = (z * gi.R + h + gi.ph) * gi.Wp + w + gi.pw;
     const long long pout = (a * s + b) * go.Ptot + (z * go.R + h / s + go.ph) * go.Wp + w / s + go.pw;
     if (to_planes) *reinterpret_cast<uint4*>(P + pout * C + cg * 8) = *reinterpret_cast<const uint4*>(T + pin * C + cg * 8);
-    else *reinterpret_cast<uint4*>(const_cast<bf16*>(T) + pin * C + cg * 8) = *reinterpret_cast<const uint4*>(P + pout * C + cg * 8);
+    else *reinterpret_cast<uint4*>(T + pin * C + cg * 8) = *reinterpret_cast<const uint4*>(P + pout * C + cg * 8);
   }
 }
 
@@ -309,7 +309,7 @@ void pad_fix(GenConv* c, bf16* T, Geo g, int C, bool fill_halos, int planes = 1)
   c->prof->end();
 }
 
-void decimate(GenConv* c, const bf16* T, bf16* planes, const Geo& gi, const Geo& go, int C, int s, bool to_planes) {
+void decimate(GenConv* c, bf16* T, bf16* planes, const Geo& gi, const Geo& go, int C, int s, bool to_planes) {
   const long long n = gi.Z * gi.Hs * gi.W * (C / 8);
   c->prof->begin(MBD_K_HALO, static_cast<double>(n) * 32.0, c->stream);
   decimate_kernel<<<grid_1d(n, c->num_sms), 256, 0, c->stream>>>(T, planes, gi, go, C, s, to_planes ? 1 : 0);
