@@ -61,11 +61,13 @@ constexpr int FWD_SMEM = FWD_W_BYTES + FWD1_STAGES * FWD1_ROW_BYTES + 4 * FWD_TI
 static_assert(FWD_SMEM <= 227 * 1024, "forward kernel's shared memory");
 constexpr int FWD_THREADS = 320;      // producer warp, MMA warp, 8 epilogue warps
 constexpr int WG_PIX = 128;           // pixels (reduction length) per backward-weight block
-constexpr int WG_XSTAGES = 4;          // X rows: one box of 130 pixels each (17 KB), each row used once
-constexpr int WG_YSTAGES = 6;          // dY rows: 16 KB each, plus 2 mirror slots
+constexpr int WG_XSTAGES = 4;          // X rows: one box of 130 pixels each (17 KB), each row used once; 3 x 3 layers take them in pairs
+constexpr int WG_YSTAGES = 6;          // dY rows: 16 KB each, plus mirror slots
+constexpr int WG_YMIRROR = 3;          // a window of up to four dY rows is contiguous: the first three slots are mirrored behind the last
 constexpr int WG_CHUNK = WG_PIX * 128;
 constexpr int WG_XROW_BYTES = 17 * 1024;   // 130 x 128 B, padded to the swizzle span; the views may read one row past the box
-constexpr int WG_SMEM = WG_XSTAGES * WG_XROW_BYTES + (WG_YSTAGES + 2) * WG_CHUNK + 1024;
+constexpr int WG_SMEM = WG_XSTAGES * WG_XROW_BYTES + (WG_YSTAGES + WG_YMIRROR) * WG_CHUNK + 1024;
+static_assert(WG_SMEM <= 227 * 1024, "backward-weight kernel's shared memory");
 constexpr int NUM_THREADS = 192;
 
 enum { MODE_RELU_STORE = 0, MODE_STORE_SSQ = 1, MODE_MASK = 2 };
@@ -702,10 +704,14 @@ __device__ __forceinline__ WgRun wg_run(const WgParams& p, long long pos, long l
 }
 
 // One X row (one box of 130 pixels, read through three shifted views) meets the up to three dY rows it contributes to in ONE
-// instruction group: B = [dY_{r-2} | dY_{r-1} | dY_r] (N = 64 per row, rows adjacent in the dY
-// ring), A = (shift 0 | shift 1) and (shift 2 | don't care), so tap (u, v) accumulates in
-// TMEM lanes (v, c) and columns (2 - u, o).  The dY ring mirrors its first two slots behind
-// its last one so that a window of three rows is always contiguous in shared memory.
+// instruction: B = [dY_{r-2} | dY_{r-1} | dY_r] (N = 64 per row, rows adjacent in the dY ring), A = (shift 0 | shift 1),
+// so tap (u, v <= 1) accumulates in TMEM lanes (v, c) and columns (2 - u, o).  The third shift has only 64 lanes of its
+// own: the X rows are taken in PAIRS (r, r + 1; two adjacent ring stages) and one instruction A = (shift 2 of row r |
+// shift 2 of row r + 1) meets the four dY rows r-2 .. r+1 (N = 256): lanes 0-63 accumulate tap (u, 2) in column block
+// 2 - u, lanes 64-127 in block 3 - u (block 3 of the first half and block 0 of the second are products no tap
+// needs), and the epilogue adds the two halves.  Five instructions of 128 x (192, 192, 256) per pair of rows instead
+// of four of 128 x 192 with half the lanes of every second one wasted.  An odd last row pairs with a row of zeros.
+// The dY ring mirrors its first three slots behind its last one so that a window is always contiguous in shared memory.
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const WgParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -760,34 +766,59 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         const int x0 = run.seg * WG_PIX;
         // 3 x 3: n dY rows meet n + 2 X rows (from the row above the first one on); 1 x 1: their own n X rows
         const int n_x = p.k1 ? run.n : run.n + 2, xrow0 = p.k1 ? run.h0 + 1 : run.h0;
-        for (int r = 0; r < n_x && ok; ++r) {
-          if (r < run.n) {
-            ok = mbar_wait(smem_u32(&yempty[ys]), yph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
-            if (!ok) break;
-            const uint32_t fy = smem_u32(&yfull[ys]);
-            const bool mirrored = ys < 2 && !p.k1;       // (a 1 x 1 layer reads one dY row at a time: no window)
-            mbar_expect_tx(fy, mirrored ? 2 * WG_CHUNK : WG_CHUNK);
-            for (int j = 0; j < p.pack; ++j) {     // one box per strip of the group (pixels beyond W and strips beyond Z read as zeros)
-              // the dead row of a short strip holds the neighbour's row (it is that strip's halo row): read the all-zero row instead
-              const int yrow = run.h0 + r + 1 == p.Hs && strips_uneven(p.H, p.P_r, p.Hs) && p.Hs > strip_height((z + j) % p.P_r, p.H, p.P_r, p.Hs)
-                                   ? p.Hs + 1 : run.h0 + r + 1;
-              tma_load_4d(yring + ys * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, yrow, z + j, fy);
-              if (mirrored) tma_load_4d(yring + (WG_YSTAGES + ys) * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, yrow, z + j, fy);
-            }
-            if (++ys == WG_YSTAGES) { ys = 0; yph ^= 1u; }
+        auto load_y = [&](int r) {            // dY row r of the run into the next ring slot (and its mirror)
+          ok = mbar_wait(smem_u32(&yempty[ys]), yph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
+          if (!ok) return;
+          const uint32_t fy = smem_u32(&yfull[ys]);
+          const bool mirrored = ys < WG_YMIRROR && !p.k1;       // (a 1 x 1 layer reads one dY row at a time: no window)
+          mbar_expect_tx(fy, mirrored ? 2 * WG_CHUNK : WG_CHUNK);
+          for (int j = 0; j < p.pack; ++j) {     // one box per strip of the group (pixels beyond W and strips beyond Z read as zeros)
+            // the dead row of a short strip holds the neighbour's row (it is that strip's halo row): read the all-zero row instead
+            const int yrow = run.h0 + r + 1 == p.Hs && strips_uneven(p.H, p.P_r, p.Hs) && p.Hs > strip_height((z + j) % p.P_r, p.H, p.P_r, p.Hs)
+                                 ? p.Hs + 1 : run.h0 + r + 1;
+            tma_load_4d(yring + ys * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, yrow, z + j, fy);
+            if (mirrored) tma_load_4d(yring + (WG_YSTAGES + ys) * WG_CHUNK + j * sub_bytes, &tmY, 0, x0, yrow, z + j, fy);
           }
-          ok = mbar_wait(smem_u32(&xempty[xs]), xph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
-          if (!ok) break;
-          const uint32_t fb = smem_u32(&xfull[xs]);
+          if (++ys == WG_YSTAGES) { ys = 0; yph ^= 1u; }
+        };
+        // one X row into ring stage `stage`, counted on barrier `fb`; row < 0: a row of zeros (a coordinate outside
+        // the tensor: TMA fills the box and counts its bytes all the same)
+        auto load_x = [&](int stage, int row, uint32_t fb) {
+          const int yc = row < 0 ? -8 : row;
           if (p.pack == 1) {
-            mbar_expect_tx(fb, (WG_PIX + 2) * 128);
-            tma_load_4d(xring + xs * WG_XROW_BYTES, &tmX, 0, x0 - 1, xrow0 + r, z, fb);
+            tma_load_4d(xring + stage * WG_XROW_BYTES, &tmX, 0, x0 - 1, yc, z, fb);
           } else {
-            mbar_expect_tx(fb, WG_PIX * 128);
             for (int j = 0; j < p.pack; ++j)
-              tma_load_4d(xring + xs * WG_XROW_BYTES + j * sub_bytes, &tmX, 0, -1, xrow0 + r, z + j, fb);
+              tma_load_4d(xring + stage * WG_XROW_BYTES + j * sub_bytes, &tmX, 0, -1, yc, z + j, fb);
           }
-          if (++xs == WG_XSTAGES) { xs = 0; xph ^= 1u; }
+        };
+        const int x_bytes = p.pack == 1 ? (WG_PIX + 2) * 128 : WG_PIX * 128;
+        if (p.k1) {
+          for (int r = 0; r < n_x && ok; ++r) {
+            load_y(r);
+            if (!ok) break;
+            ok = mbar_wait(smem_u32(&xempty[xs]), xph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
+            if (!ok) break;
+            const uint32_t fb = smem_u32(&xfull[xs]);
+            mbar_expect_tx(fb, x_bytes);
+            load_x(xs, xrow0 + r, fb);
+            if (++xs == WG_XSTAGES) { xs = 0; xph ^= 1u; }
+          }
+        } else {
+          // X rows in pairs: stages (xs, xs + 1) with xs even, both counted on the barrier of stage xs
+          for (int r = 0; r < n_x && ok; r += 2) {
+            if (r < run.n) load_y(r);
+            if (ok && r + 1 < run.n) load_y(r + 1);
+            if (!ok) break;
+            ok = mbar_wait(smem_u32(&xempty[xs]), xph ^ 1u, abortp, p.status, DEV_TIMEOUT_PRODUCER);
+            if (!ok) break;
+            const uint32_t fb = smem_u32(&xfull[xs]);
+            mbar_expect_tx(fb, 2 * x_bytes);
+            load_x(xs, xrow0 + r, fb);
+            load_x(xs + 1, r + 1 < n_x ? xrow0 + r + 1 : -1, fb);
+            xs += 2;
+            if (xs == WG_XSTAGES) { xs = 0; xph ^= 1u; }
+          }
         }
       }
     }
@@ -825,9 +856,10 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           y_slot0 = (y_slot0 + run.n) % WG_YSTAGES;
           continue;
         }
-        for (int r = 0; r < run.n + 2 && ok; ++r) {
-          const int i_hi = min(r, run.n - 1), i_lo = max(0, r - 2);
-          while (yhave <= i_hi && ok) {
+        for (int r = 0; r < run.n + 2 && ok; r += 2) {
+          const bool two = r + 1 < run.n + 2;                  // (an odd last row is paired with a row of zeros)
+          const int i_top = min(two ? r + 1 : r, run.n - 1);   // last dY row any instruction of this pair reads
+          while (yhave <= i_top && ok) {
             ok = mbar_wait(smem_u32(&yfull[yw]), ywph, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
             if (++yw == WG_YSTAGES) { yw = 0; ywph ^= 1u; }
             ++yhave;
@@ -836,23 +868,37 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           ok = mbar_wait(smem_u32(&xfull[xw]), xwph, abortp, p.status, DEV_TIMEOUT_MMA_FULL);
           if (!ok) break;
           tc_fence_after();
-          const int n = i_hi - i_lo + 1;                       // dY rows in the window
-          const int b0 = 2 - (r - i_lo);                       // column block of the first of them
-          const uint32_t idesc = make_idesc(128, 64 * n, 1, 1);
-          const int ys0 = (y_slot0 + i_lo) % WG_YSTAGES;       // window may run into the mirror slots
-          const uint64_t bdesc = make_desc(yring + ys0 * WG_CHUNK, WG_CHUNK, 1024);
           // The operand shifted by v pixels is the view of the box that starts v pixel rows (128 bytes) in; the
-          // two 64-channel chunks of an M = 128 operand are two such views, one row apart (leading offset 128).
+          // two 64-channel chunks of an M = 128 operand are two such views: one pixel row apart (shifts 0 | 1 of one
+          // X row, leading offset 128) or one ring stage apart (shift 2 of two X rows, leading offset = the stage size).
           const uint32_t xa = xring + xw * WG_XROW_BYTES;
-          const uint64_t a01 = make_desc(xa, 128, 1024);                      // lanes: (shift 0 | shift 1) x c
-          const uint64_t a2x = make_desc(xa + 2 * 128, 128, 1024);            // lanes: (shift 2 | don't care) x c
-          for (int k = 0; k < ksteps; ++k) {
-            tc_mma_bf16(tmem_base + b0 * 64, a01 + k * 128, bdesc + k * 128, idesc, 1u);
-            tc_mma_bf16(tmem_base + 256 + b0 * 64, a2x + k * 128, bdesc + k * 128, idesc, 1u);
+          for (int h = 0; h < (two ? 2 : 1); ++h) {            // shifts 0 | 1 of X row r + h against its window of dY rows
+            const int rr = r + h;
+            const int i_hi = min(rr, run.n - 1), i_lo = max(0, rr - 2);
+            const int n = i_hi - i_lo + 1;                     // dY rows in the window
+            const int b0 = 2 - (rr - i_lo);                    // column block of the first of them
+            const uint32_t idesc = make_idesc(128, 64 * n, 1, 1);
+            const int ys0 = (y_slot0 + i_lo) % WG_YSTAGES;     // window may run into the mirror slots
+            const uint64_t bdesc = make_desc(yring + ys0 * WG_CHUNK, WG_CHUNK, 1024);
+            const uint64_t a01 = make_desc(xa + h * WG_XROW_BYTES, 128, 1024);          // lanes: (shift 0 | shift 1) x c
+            for (int k = 0; k < ksteps; ++k) tc_mma_bf16(tmem_base + b0 * 64, a01 + k * 128, bdesc + k * 128, idesc, 1u);
+          }
+          {   // shift 2 of both rows against dY rows r-2 .. r+1: lanes 0-63 block 2 - u, lanes 64-127 block 3 - u
+            const int i_lo = max(0, r - 2);
+            const int n = i_top - i_lo + 1;
+            const int b0 = 2 - (r - i_lo);
+            const uint32_t idesc = make_idesc(128, 64 * n, 1, 1);
+            const int ys0 = (y_slot0 + i_lo) % WG_YSTAGES;
+            const uint64_t bdesc = make_desc(yring + ys0 * WG_CHUNK, WG_CHUNK, 1024);
+            const uint64_t a22 = make_desc(xa + 2 * 128, WG_XROW_BYTES, 1024);        // lanes: (row r | row r + 1) shift 2 x c
+            for (int k = 0; k < ksteps; ++k) tc_mma_bf16(tmem_base + 256 + b0 * 64, a22 + k * 128, bdesc + k * 128, idesc, 1u);
           }
           tc_commit(smem_u32(&xempty[xw]));
-          if (++xw == WG_XSTAGES) { xw = 0; xwph ^= 1u; }
-          if (r >= 2) tc_commit(smem_u32(&yempty[(y_slot0 + r - 2) % WG_YSTAGES]));   // dY row r-2 has no later reader
+          xw += 2;
+          if (xw == WG_XSTAGES) { xw = 0; xwph ^= 1u; }
+          // dY rows r - 2 and r - 1 have no later reader
+          if (r >= 2) tc_commit(smem_u32(&yempty[(y_slot0 + r - 2) % WG_YSTAGES]));
+          if (r >= 1 && r - 1 < run.n) tc_commit(smem_u32(&yempty[(y_slot0 + r - 1) % WG_YSTAGES]));
         }
         y_slot0 = (y_slot0 + run.n) % WG_YSTAGES;
       }
@@ -861,9 +907,9 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   } else {
     const int q = warp & 3;
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
-    {   // zero both accumulators (columns 0..191 and 256..447) before the first MMA
-      for (int cb = 0; cb < 12; ++cb) {
-        const uint32_t col = (cb < 6 ? 0 : 256) + (cb % 6) * 32;
+    {   // zero both accumulators (columns 0..191 and 256..511) before the first MMA
+      for (int cb = 0; cb < 14; ++cb) {
+        const uint32_t col = cb < 6 ? cb * 32 : 256 + (cb - 6) * 32;
         asm volatile(
             "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
             "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
@@ -882,26 +928,61 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       const int row = q * 32 + lane;                 // TMEM lane: (shift-in-pair, c)
       const int c = row & 63;
       float* dst_base = p.part + static_cast<int64_t>(blockIdx.x) * 9 * C * C;
-      for (int a = 0; a < 6; ++a) {
-        const int pair = a / 3, blk = a % 3;
-        const int u = 2 - blk;
-        const int v = pair == 0 ? (row >> 6) : 2;
-        const bool keep = pair == 0 || row < 64;
+      // shifts 0 and 1: lanes (v, c), column blocks 2 - u
+      for (int blk = 0; blk < 3; ++blk) {
+        const int u = 2 - blk, v = row >> 6;
         float* dst = dst_base + ((u * 3 + v) * C + c) * C;
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
           uint32_t r[32];
-          tc_ld32(lane_base + pair * 256 + blk * 64 + half * 32, r);
+          tc_ld32(lane_base + blk * 64 + half * 32, r);
           tc_wait_ld();
-          if (keep) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<float4*>(dst + half * 32 + j * 4) =
+                make_float4(__uint_as_float(r[j * 4]), __uint_as_float(r[j * 4 + 1]), __uint_as_float(r[j * 4 + 2]),
+                            __uint_as_float(r[j * 4 + 3]));
+        }
+      }
+      // shift 2: lanes 64-127 (the second X row of every pair) hand their blocks 3 - u over through shared memory (the
+      // rings are idle now: every MMA has completed), lanes 0-63 add them to their blocks 2 - u and store tap (u, 2)
+      float* comb = reinterpret_cast<float*>(smem_raw + (xring - smem_u32(smem_raw)));      // [64 c][3 u][64 o] floats, 48 KB
+      if (row >= 64 && !p.k1) {                  // (a 1 x 1 layer forms no shift-2 tap: that accumulator is zero)
+        for (int u = 0; u < 3; ++u) {
+#pragma unroll 1
+          for (int half = 0; half < 2; ++half) {
+            uint32_t r[32];
+            tc_ld32(lane_base + 256 + (3 - u) * 64 + half * 32, r);
+            tc_wait_ld();
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-              *reinterpret_cast<float4*>(dst + half * 32 + j * 4) =
+              *reinterpret_cast<float4*>(comb + (c * 3 + u) * C + half * 32 + j * 4) =
                   make_float4(__uint_as_float(r[j * 4]), __uint_as_float(r[j * 4 + 1]), __uint_as_float(r[j * 4 + 2]),
                               __uint_as_float(r[j * 4 + 3]));
           }
         }
       }
+      asm volatile("bar.sync 2, 128;" ::: "memory");           // the four epilogue warps
+      if (row < 64) {
+        for (int u = 0; u < 3; ++u) {
+          float* dst = dst_base + ((u * 3 + 2) * C + c) * C;
+#pragma unroll 1
+          for (int half = 0; half < 2; ++half) {
+            uint32_t r[32];
+            tc_ld32(lane_base + 256 + (2 - u) * 64 + half * 32, r);
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float4 o = p.k1 ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(comb + (c * 3 + u) * C + half * 32 + j * 4);
+              *reinterpret_cast<float4*>(dst + half * 32 + j * 4) =
+                  make_float4(__uint_as_float(r[j * 4]) + o.x, __uint_as_float(r[j * 4 + 1]) + o.y, __uint_as_float(r[j * 4 + 2]) + o.z,
+                              __uint_as_float(r[j * 4 + 3]) + o.w);
+            }
+          }
+        }
+      }
+    } else {
+      asm volatile("bar.sync 2, 128;" ::: "memory");           // (keeps the barrier's count when the wait gave up)
     }
   }
 
