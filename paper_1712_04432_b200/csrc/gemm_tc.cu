@@ -16,7 +16,7 @@
 // Tile shapes: 128 x 128, 128 x 256, 256 x 256 per CTA, or 256 x 256 per CTA pair
 // (cta_group::2); tc_gemm_prepare picks one per contraction with a small cost model.  With a
 // bf16 result on 128-row tiles the epilogue moves all its global data by TMA through per-warp
-// staging boxes.  Tuning knobs (environment): MBD_TC_MH, MBD_TC_BN, MBD_TC_PAIR, MBD_TC_GROUP_M, MBD_TC_DEBUG,
+// staging boxes.  Tuning knobs (environment): MBD_TC_MH, MBD_TC_BN, MBD_TC_PAIR, MBD_TC_GROUP_M, MBD_TC_DEBUG, MBD_TC_X_POW2,
 // MBD_TC_NO_TE.
 // Every mbarrier wait is bounded; on time-out the kernel records a code and leaves.
 #include <stdio.h>
@@ -1015,12 +1015,13 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
     double best = 1e30;
     int best_bn = 128, best_mh = 1, best_x = 1, best_pair = 0, best_join = 0;
     const int x_max = g.allow_extra_split ? 32 : 1;
+    const bool x_any = getenv("MBD_TC_X_POW2") == nullptr;      // tuning knob: extra cuts in powers of two only
     for (int cand = 0; cand < 4; ++cand) {           // 0: 128-row tiles, 1: 256-row tiles, 2: CTA pairs, 3: pairs of 256-row CTAs
       const int mh = (cand == 1 || cand == 3) ? 2 : 1;
       const bool pair = cand >= 2;
       for (int bn = pair ? 256 : 128; bn <= 256; bn += 128) {
         for (int jn = 0; jn <= (join_ok && g.k_splits * mh * bn <= 512 ? 1 : 0); ++jn) {
-        for (int x = 1; x <= (jn ? 1 : x_max); x *= 2) {
+        for (int x = 1; x <= (jn ? 1 : x_max); x = x_any ? x + 1 : x * 2) {
           const long long S = jn ? 1 : 1ll * g.k_splits * x;
           if (S > kb_total || (x > 1 && kb_total / S < 8)) continue;
           const double kb = static_cast<double>(kb_total) / S;
