@@ -39,58 +39,82 @@ struct Geo {
 
 // ------------------------------------------------------------------------------ layout kernels
 // NCHW <-> pixel-major (own pixels only; padding and halos are the business of pad_fix_kernel).  A block moves a
-// tile of 32 consecutive pixels of one image row x 64 channels through shared memory, so that both sides are
-// accessed in runs: 64 bytes per channel on the NCHW side, 128 bytes per pixel on the pixel-major side.
-// grid = (B * H, ceil(W / 32), ceil(C / 64)), 256 threads.
+// tile of 64 rows x 32 pixels through shared memory, a row being one channel of a run of 32 consecutive pixels of
+// one image (pixels counted through the image, h * W + w: a channel plane is contiguous in NCHW), so that both sides
+// are accessed in runs: 64 bytes per channel on the NCHW side, 16 bytes x the layer's channels per pixel on the
+// pixel-major side.  With 64 channels or more the rows are 64 channels of one run; with fewer (cpb = C < 64 channels
+// per block) they are the channels of G = 64 / cpb runs, so that a block still moves about 4 KB (an 8-channel input
+// tensor: 256 pixels per block instead of 32).  grid = (ceil(H W / (32 G)), B, ceil(C / cpb)), 256 threads.
+struct StageTile {
+  int cpb, G;                        // channels per block (a multiple of 8, at most 64), pixel runs per block
+};
+__host__ __device__ inline StageTile stage_tile(int C) {
+  StageTile t;
+  t.cpb = C < 64 ? C : 64;
+  t.G = 64 / t.cpb;
+  return t;
+}
+__device__ __forceinline__ long long pix_index(const Geo& g, int b, int q) {     // pixel q = h * W + w of image b in the padded layout
+  const int h = q / g.W, w = q - h * g.W;
+  const int s = h / g.Hs, r = h - s * g.Hs + g.ph;
+  return ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w + g.pw;
+}
+
 __global__ void __launch_bounds__(256)
 nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C) {
   __shared__ uint16_t tile[64][34];
-  const int w0 = blockIdx.y * 32, b = blockIdx.x / g.H, h = blockIdx.x - b * g.H, c0 = blockIdx.z * 64;
+  const StageTile st = stage_tile(C);
+  const int HW = g.H * g.W;
+  const int b = blockIdx.y, q0 = blockIdx.x * 32 * st.G, c0 = blockIdx.z * st.cpb;
   const int t = threadIdx.x;
   {
-    const int c = t >> 2, wq = (t & 3) * 8;           // channel c0 + c, pixels w0 + wq .. + 7
-    if (c0 + c < C) {
-      const bf16* q = src + ((static_cast<long long>(b) * C + c0 + c) * g.H + h) * g.W + w0 + wq;
-      if ((g.W & 7) == 0 && w0 + wq + 8 <= g.W && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {      // 16 aligned bytes
-        const uint4 v = __ldcs(reinterpret_cast<const uint4*>(q));
+    const int row = t >> 2, wq = (t & 3) * 8;         // row = (run, channel); pixels q .. q + 7 of that run
+    const int pg = row / st.cpb, c = row - pg * st.cpb;
+    const int q = q0 + pg * 32 + wq;
+    if (pg < st.G && c0 + c < C && q < HW) {
+      const bf16* p = src + (static_cast<long long>(b) * C + c0 + c) * HW + q;
+      if ((HW & 7) == 0 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {      // 16 aligned bytes, all inside the plane
+        const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p));
         const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          tile[c][wq + 2 * j] = static_cast<uint16_t>(wv[j] & 0xFFFFu);
-          tile[c][wq + 2 * j + 1] = static_cast<uint16_t>(wv[j] >> 16);
+          tile[row][wq + 2 * j] = static_cast<uint16_t>(wv[j] & 0xFFFFu);
+          tile[row][wq + 2 * j + 1] = static_cast<uint16_t>(wv[j] >> 16);
         }
       } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) tile[c][wq + j] = w0 + wq + j < g.W ? __bfloat16_as_ushort(q[j]) : 0;
+        for (int j = 0; j < 8; ++j) tile[row][wq + j] = q + j < HW ? __bfloat16_as_ushort(p[j]) : 0;
       }
     }
   }
   __syncthreads();
-  const int px = t >> 3, cg = t & 7;                  // pixel w0 + px, channels c0 + 8 cg .. + 7
-  if (w0 + px >= g.W || c0 + cg * 8 >= C) return;
+  const int px = t >> 3, cg = t & 7;                  // rows 8 cg .. 8 cg + 7: eight channels of one run; pixel px of it
+  const int pg = cg * 8 / st.cpb, c = cg * 8 - pg * st.cpb;
+  const int q = q0 + pg * 32 + px;
+  if (pg >= st.G || q >= HW || c0 + c >= C) return;
   uint16_t v[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) v[j] = tile[cg * 8 + j][px];
   uint4 o;
   o.x = v[0] | (static_cast<uint32_t>(v[1]) << 16); o.y = v[2] | (static_cast<uint32_t>(v[3]) << 16);
   o.z = v[4] | (static_cast<uint32_t>(v[5]) << 16); o.w = v[6] | (static_cast<uint32_t>(v[7]) << 16);
-  const int s = h / g.Hs, r = h - s * g.Hs + g.ph;
-  const long long p = ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w0 + px + g.pw;
-  *reinterpret_cast<uint4*>(dst + p * C + c0 + cg * 8) = o;
+  *reinterpret_cast<uint4*>(dst + pix_index(g, b, q) * C + c0 + c) = o;
 }
 
 __global__ void __launch_bounds__(256)
 pix_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C) {
   __shared__ uint16_t tile[64][34];
-  const int w0 = blockIdx.y * 32, b = blockIdx.x / g.H, h = blockIdx.x - b * g.H, c0 = blockIdx.z * 64;
+  const StageTile st = stage_tile(C);
+  const int HW = g.H * g.W;
+  const int b = blockIdx.y, q0 = blockIdx.x * 32 * st.G, c0 = blockIdx.z * st.cpb;
   const int t = threadIdx.x;
   {
     const int px = t >> 3, cg = t & 7;
-    if (w0 + px < g.W && c0 + cg * 8 < C) {
-      const int s = h / g.Hs, r = h - s * g.Hs + g.ph;
-      const long long p = ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w0 + px + g.pw;
-      const uint4 q = *reinterpret_cast<const uint4*>(src + p * C + c0 + cg * 8);
-      const uint32_t wv[4] = {q.x, q.y, q.z, q.w};
+    const int pg = cg * 8 / st.cpb, c = cg * 8 - pg * st.cpb;
+    const int q = q0 + pg * 32 + px;
+    if (pg < st.G && q < HW && c0 + c < C) {
+      const uint4 v = *reinterpret_cast<const uint4*>(src + pix_index(g, b, q) * C + c0 + c);
+      const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         tile[cg * 8 + 2 * j][px] = static_cast<uint16_t>(wv[j] & 0xFFFFu);
@@ -99,18 +123,20 @@ pix_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, 
     }
   }
   __syncthreads();
-  const int c = t >> 2, wq = (t & 3) * 8;
-  if (c0 + c >= C) return;
-  bf16* q = dst + ((static_cast<long long>(b) * C + c0 + c) * g.H + h) * g.W + w0 + wq;
-  if ((g.W & 7) == 0 && w0 + wq + 8 <= g.W && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+  const int row = t >> 2, wq = (t & 3) * 8;
+  const int pg = row / st.cpb, c = row - pg * st.cpb;
+  const int q = q0 + pg * 32 + wq;
+  if (pg >= st.G || c0 + c >= C || q >= HW) return;
+  bf16* p = dst + (static_cast<long long>(b) * C + c0 + c) * HW + q;
+  if ((HW & 7) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
     uint4 v;
-    v.x = tile[c][wq + 0] | (static_cast<uint32_t>(tile[c][wq + 1]) << 16); v.y = tile[c][wq + 2] | (static_cast<uint32_t>(tile[c][wq + 3]) << 16);
-    v.z = tile[c][wq + 4] | (static_cast<uint32_t>(tile[c][wq + 5]) << 16); v.w = tile[c][wq + 6] | (static_cast<uint32_t>(tile[c][wq + 7]) << 16);
-    *reinterpret_cast<uint4*>(q) = v;
+    v.x = tile[row][wq + 0] | (static_cast<uint32_t>(tile[row][wq + 1]) << 16); v.y = tile[row][wq + 2] | (static_cast<uint32_t>(tile[row][wq + 3]) << 16);
+    v.z = tile[row][wq + 4] | (static_cast<uint32_t>(tile[row][wq + 5]) << 16); v.w = tile[row][wq + 6] | (static_cast<uint32_t>(tile[row][wq + 7]) << 16);
+    *reinterpret_cast<uint4*>(p) = v;
   } else {
 #pragma unroll
     for (int j = 0; j < 8; ++j)
-      if (w0 + wq + j < g.W) q[j] = __ushort_as_bfloat16(tile[c][wq + j]);
+      if (q + j < HW) p[j] = __ushort_as_bfloat16(tile[row][wq + j]);
   }
 }
 
@@ -623,14 +649,16 @@ mbd_status gconv_get_weights(GenConv* c, int i, void* K_dev) {
 
 namespace {
 void stage(GenConv* c, const bf16* nchw, bf16* dst, const Geo& g, int C, bool fill_halos) {
-  const dim3 grid(static_cast<unsigned>(g.B) * g.H, (g.W + 31) / 32, (C + 63) / 64);
+  const StageTile t = stage_tile(C);
+  const dim3 grid((g.H * g.W + 32 * t.G - 1) / (32 * t.G), static_cast<unsigned>(g.B), (C + t.cpb - 1) / t.cpb);
   c->prof->begin(MBD_K_HALO, 2.0 * g.B * C * g.H * g.W * 2.0, c->stream);
   nchw_to_pix_kernel<<<grid, 256, 0, c->stream>>>(nchw, dst, g, C);
   c->prof->end();
   pad_fix(c, dst, g, C, fill_halos);
 }
 void unstage(GenConv* c, const bf16* src, bf16* nchw, const Geo& g, int C) {
-  const dim3 grid(static_cast<unsigned>(g.B) * g.H, (g.W + 31) / 32, (C + 63) / 64);
+  const StageTile t = stage_tile(C);
+  const dim3 grid((g.H * g.W + 32 * t.G - 1) / (32 * t.G), static_cast<unsigned>(g.B), (C + t.cpb - 1) / t.cpb);
   c->prof->begin(MBD_K_HALO, 2.0 * g.B * C * g.H * g.W * 2.0, c->stream);
   pix_to_nchw_kernel<<<grid, 256, 0, c->stream>>>(src, nchw, g, C);
   c->prof->end();
