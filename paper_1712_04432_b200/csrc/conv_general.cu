@@ -60,16 +60,17 @@ __device__ __forceinline__ long long pix_index(const Geo& g, int b, int q) {    
   return ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w + g.pw;
 }
 
+// WIDE: 64 channels per block, one run (no division by the channel count)
+template <bool WIDE>
 __global__ void __launch_bounds__(256)
-nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C) {
+nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C, StageTile st) {
   __shared__ uint16_t tile[64][34];
-  const StageTile st = stage_tile(C);
   const int HW = g.H * g.W;
   const int b = blockIdx.y, q0 = blockIdx.x * 32 * st.G, c0 = blockIdx.z * st.cpb;
   const int t = threadIdx.x;
   {
     const int row = t >> 2, wq = (t & 3) * 8;         // row = (run, channel); pixels q .. q + 7 of that run
-    const int pg = row / st.cpb, c = row - pg * st.cpb;
+    const int pg = WIDE ? 0 : row / st.cpb, c = row - pg * st.cpb;
     const int q = q0 + pg * 32 + wq;
     if (pg < st.G && c0 + c < C && q < HW) {
       const bf16* p = src + (static_cast<long long>(b) * C + c0 + c) * HW + q;
@@ -89,7 +90,7 @@ nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, 
   }
   __syncthreads();
   const int px = t >> 3, cg = t & 7;                  // rows 8 cg .. 8 cg + 7: eight channels of one run; pixel px of it
-  const int pg = cg * 8 / st.cpb, c = cg * 8 - pg * st.cpb;
+  const int pg = WIDE ? 0 : cg * 8 / st.cpb, c = cg * 8 - pg * st.cpb;
   const int q = q0 + pg * 32 + px;
   if (pg >= st.G || q >= HW || c0 + c >= C) return;
   uint16_t v[8];
@@ -101,16 +102,16 @@ nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, 
   *reinterpret_cast<uint4*>(dst + pix_index(g, b, q) * C + c0 + c) = o;
 }
 
+template <bool WIDE>
 __global__ void __launch_bounds__(256)
-pix_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C) {
+pix_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C, StageTile st) {
   __shared__ uint16_t tile[64][34];
-  const StageTile st = stage_tile(C);
   const int HW = g.H * g.W;
   const int b = blockIdx.y, q0 = blockIdx.x * 32 * st.G, c0 = blockIdx.z * st.cpb;
   const int t = threadIdx.x;
   {
     const int px = t >> 3, cg = t & 7;
-    const int pg = cg * 8 / st.cpb, c = cg * 8 - pg * st.cpb;
+    const int pg = WIDE ? 0 : cg * 8 / st.cpb, c = cg * 8 - pg * st.cpb;
     const int q = q0 + pg * 32 + px;
     if (pg < st.G && q < HW && c0 + c < C) {
       const uint4 v = *reinterpret_cast<const uint4*>(src + pix_index(g, b, q) * C + c0 + c);
@@ -124,7 +125,7 @@ pix_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, 
   }
   __syncthreads();
   const int row = t >> 2, wq = (t & 3) * 8;
-  const int pg = row / st.cpb, c = row - pg * st.cpb;
+  const int pg = WIDE ? 0 : row / st.cpb, c = row - pg * st.cpb;
   const int q = q0 + pg * 32 + wq;
   if (pg >= st.G || c0 + c >= C || q >= HW) return;
   bf16* p = dst + (static_cast<long long>(b) * C + c0 + c) * HW + q;
@@ -652,7 +653,8 @@ void stage(GenConv* c, const bf16* nchw, bf16* dst, const Geo& g, int C, bool fi
   const StageTile t = stage_tile(C);
   const dim3 grid((g.H * g.W + 32 * t.G - 1) / (32 * t.G), static_cast<unsigned>(g.B), (C + t.cpb - 1) / t.cpb);
   c->prof->begin(MBD_K_HALO, 2.0 * g.B * C * g.H * g.W * 2.0, c->stream);
-  nchw_to_pix_kernel<<<grid, 256, 0, c->stream>>>(nchw, dst, g, C);
+  if (t.cpb == 64) nchw_to_pix_kernel<true><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t);
+  else nchw_to_pix_kernel<false><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t);
   c->prof->end();
   pad_fix(c, dst, g, C, fill_halos);
 }
@@ -660,7 +662,8 @@ void unstage(GenConv* c, const bf16* src, bf16* nchw, const Geo& g, int C) {
   const StageTile t = stage_tile(C);
   const dim3 grid((g.H * g.W + 32 * t.G - 1) / (32 * t.G), static_cast<unsigned>(g.B), (C + t.cpb - 1) / t.cpb);
   c->prof->begin(MBD_K_HALO, 2.0 * g.B * C * g.H * g.W * 2.0, c->stream);
-  pix_to_nchw_kernel<<<grid, 256, 0, c->stream>>>(src, nchw, g, C);
+  if (t.cpb == 64) pix_to_nchw_kernel<true><<<grid, 256, 0, c->stream>>>(src, nchw, g, C, t);
+  else pix_to_nchw_kernel<false><<<grid, 256, 0, c->stream>>>(src, nchw, g, C, t);
   c->prof->end();
 }
 }  // namespace
