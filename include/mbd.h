@@ -343,6 +343,20 @@ MBD_API int64_t mbd_launch_count(const mbd_net* net);
 typedef struct { int32_t tile_m, tile_n, cta_pair, k_pieces, tma_epilogue, ctas, running_sum, k_blocks; } mbd_plan;
 MBD_API mbd_status mbd_get_plan(const mbd_net* net, int layer, int product, mbd_plan* out_host);
 
+/* The same plan for a stand-alone bf16 product of Section 1 (variant as in mbd_gemm_bf16: 0 = forward Y = W X,
+ * 1 = backward-data, 2 = backward-weight; output M x N, reduction length K), computed on the host without touching a
+ * device: the planner is a cost model over tile shapes and cuts of K for `num_sms` SMs (>= 2), so its choices can be
+ * inspected and tested where there is no GPU.  k_pieces >= 1: the pieces of K the caller's grid asks for (Appendix A.2:
+ * the partial sums over a process group).  flags: MBD_PLAN_EXTRA_CUTS: the planner may cut K further to fill the SMs
+ * (what a network allows for its forward and backward-data products and for the weight gradients of general
+ * convolutions); MBD_PLAN_INTERMEDIATE: the pieces need not be kept as planes of their own (max_partials < P), so
+ * they may be joined in tensor memory or added as a running sum; MBD_PLAN_BF16_RESULT: the result is bf16 behind a
+ * tail operation, so the TMA epilogue is possible.  k_blocks = ceil(K / 64).  The environment's tuning knobs apply
+ * as they do to a network.  MBD_E_INVALID for bad arguments, MBD_E_UNSUPPORTED for an extent beyond 2^31 - 1. */
+enum { MBD_PLAN_EXTRA_CUTS = 1, MBD_PLAN_INTERMEDIATE = 2, MBD_PLAN_BF16_RESULT = 4 };
+MBD_API mbd_status mbd_plan_product(int variant, int64_t M, int64_t N, int64_t K, int k_pieces, int flags, int num_sms,
+                                    mbd_plan* out_host);
+
 /* Stand-alone dense contraction on the tensor cores, used by the unit tests:
  *   variant 0 (forward)          D[M,N] = A[M,K]   * B[N,K]^T   A, B row-major, K contiguous
  *   variant 1 (backward-data)    D[M,N] = A[M,K]   * B[K,N]     B row-major, N contiguous

@@ -991,10 +991,10 @@ cudaError_t selftest_timeout_launch(int* status, int limit_ms, cudaStream_t stre
   return cudaGetLastError();
 }
 
-cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B, int64_t ldb, int num_sms,
-                            const Epi* te_epi) {
-  cudaError_t e = tc_gemm_init();
-  if (e != cudaSuccess) return e;
+// Everything about a contraction's launch that is decided on the host and needs no device: tile shape, CTA pairs,
+// the pieces of K (the caller's, the planner's own cuts, pieces joined in tensor memory, the running sum), planes
+// stored by TMA, the TMA epilogue (`want_te`: the result is bf16 and goes through an epilogue operation), the grid.
+void tc_gemm_plan(TcGemm& g, int num_sms, bool want_te) {
   const int kb_total = (g.K + BK - 1) / BK;
   if (g.k_splits > kb_total) g.k_splits = kb_total;
   // Tile shape and (for the network's own contractions) an extra cut of K, chosen by a small cost
@@ -1083,15 +1083,6 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
     const long long pairs = total < num_sms / 2 ? total : num_sms / 2;
     g.grid = static_cast<int>(2 * pairs);
   }
-  const bool a_mn = g.variant == 2, b_mn = g.variant >= 1;
-  if (g.cv.mode != 0 && g.cv.mode != g.variant + 1) return cudaErrorInvalidValue;
-  if (!a_mn) e = make_map(&g.tmA, A, g.cv.mode ? g.cv_a_inner : g.K, g.cv.mode && g.cv_a_rows ? g.cv_a_rows : g.M, lda, BK, BM * g.MH);   // A[M,K]: inner = K; box = the rows one CTA loads
-  else e = make_map(&g.tmA, A, g.M, g.K, lda, 64, BK);             // A[K,M]: inner = M, one 64-wide chunk per box
-  if (e != cudaSuccess) return e;
-  if (!b_mn) e = make_map(&g.tmB, B, g.K, g.N, ldb, BK, g.pair ? g.BN / 2 : g.BN);    // B[N,K]
-  else if (g.cv.mode) e = make_map(&g.tmB, B, g.cv_b_inner, g.cv_b_rows, ldb, 64, BK);     // the tensor as stored; the kernel shifts
-  else e = make_map(&g.tmB, B, g.N, g.K, ldb, 64, BK);             // B[K,N]
-  if (e != cudaSuccess) return e;
   // Running sum instead of S planes and a reduction launch: when the pieces of a tile are far apart in the
   // work order (at least as many tiles as CTA slots: the pieces of one tile never run at the same time) ...
   {
@@ -1114,18 +1105,33 @@ cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B
     const int kb_piece = kb_total / (g.k_splits > 0 ? g.k_splits : 1);
     g.te_planes = g.k_splits > 1 && !g.fix && g.MH == 1 && (g.N & 3) == 0 && kb_piece < 32 && !getenv("MBD_TC_NO_TE");
   }
-  // TMA epilogue: bf16 output of an unsplit contraction on 128-row tiles
-  g.te = 0;
+  // TMA epilogue: bf16 output of an unsplit contraction on 128-row tiles (the maps are made by tc_gemm_prepare)
+  g.te = want_te && g.MH == 1 && g.k_splits == 1 && !getenv("MBD_TC_NO_TE") ? 1 : 0;
+}
+
+cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B, int64_t ldb, int num_sms,
+                            const Epi* te_epi) {
+  cudaError_t e = tc_gemm_init();
+  if (e != cudaSuccess) return e;
+  if (g.cv.mode != 0 && g.cv.mode != g.variant + 1) return cudaErrorInvalidValue;
+  tc_gemm_plan(g, num_sms, te_epi && te_epi->out_bf16 && te_epi->out);
+  const bool a_mn = g.variant == 2, b_mn = g.variant >= 1;
+  if (!a_mn) e = make_map(&g.tmA, A, g.cv.mode ? g.cv_a_inner : g.K, g.cv.mode && g.cv_a_rows ? g.cv_a_rows : g.M, lda, BK, BM * g.MH);   // A[M,K]: inner = K; box = the rows one CTA loads
+  else e = make_map(&g.tmA, A, g.M, g.K, lda, 64, BK);             // A[K,M]: inner = M, one 64-wide chunk per box
+  if (e != cudaSuccess) return e;
+  if (!b_mn) e = make_map(&g.tmB, B, g.K, g.N, ldb, BK, g.pair ? g.BN / 2 : g.BN);    // B[N,K]
+  else if (g.cv.mode) e = make_map(&g.tmB, B, g.cv_b_inner, g.cv_b_rows, ldb, 64, BK);     // the tensor as stored; the kernel shifts
+  else e = make_map(&g.tmB, B, g.N, g.K, ldb, 64, BK);             // B[K,N]
+  if (e != cudaSuccess) return e;
   g.tmOut = g.tmA;
   g.tmAux = g.tmA;
-  if (te_epi && te_epi->out_bf16 && te_epi->out && g.MH == 1 && g.k_splits == 1 && !getenv("MBD_TC_NO_TE")) {
+  if (g.te) {
     e = make_map(&g.tmOut, te_epi->out, g.N, g.M, te_epi->ldo, 64, 32);
     if (e != cudaSuccess) return e;
     if (te_epi->op == EPI_MASK && te_epi->mask) {
       e = make_map(&g.tmAux, te_epi->mask, g.N, g.M, te_epi->ldmask, 64, 32);
       if (e != cudaSuccess) return e;
     }
-    g.te = 1;
     g.te_epi = *te_epi;
   }
   return e;

@@ -140,7 +140,10 @@ struct TcGemm {
   int64_t cv_b_inner = 0, cv_b_rows = 0;   // modes 2, 3: extent of the B tensor as stored (inner, rows)
 };
 
-// Fills tmA/tmB/BN/grid.  Returns cudaSuccess or an error.
+// The host-side part of tc_gemm_prepare: from M, N, K, variant, k_splits, allow_extra_split, allow_fix it fills BN, MH, pair,
+// k_splits, join, fix, flag_words, te_planes, te (`want_te`: a bf16 result behind an epilogue operation), grid.  Touches no device.
+void tc_gemm_plan(TcGemm& g, int num_sms, bool want_te);
+// Plans (tc_gemm_plan), then fills the tensor maps.  Returns cudaSuccess or an error.
 // `te_epi` (may be null): the epilogue this contraction will run with, if its output is bf16;
 // lets the plan move the epilogue's global traffic with TMA.
 cudaError_t tc_gemm_prepare(TcGemm& g, const void* A, int64_t lda, const void* B, int64_t ldb,

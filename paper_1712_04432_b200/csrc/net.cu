@@ -970,6 +970,19 @@ extern "C" mbd_status mbd_poll_status(mbd_net* n) {
 
 extern "C" int64_t mbd_launch_count(const mbd_net* n) { return n ? n->prof.total_launches : -1; }
 
+namespace {
+void fill_plan(const TcGemm& g, mbd_plan* out) {
+  out->tile_m = 128 * g.MH * (g.pair ? 2 : 1);
+  out->tile_n = g.BN;
+  out->cta_pair = g.pair;
+  out->k_pieces = g.join > 1 ? g.join : g.k_splits;
+  out->tma_epilogue = g.te_planes ? 2 : g.te;
+  out->ctas = g.grid;
+  out->running_sum = g.join > 1 ? 2 : g.fix;
+  out->k_blocks = (g.K + 63) / 64;
+}
+}  // namespace
+
 extern "C" mbd_status mbd_get_plan(const mbd_net* n, int layer, int product, mbd_plan* out) {
   if (!n || !out || product < 0 || product > 2) return MBD_E_INVALID;
   if (layer < 0 || layer >= n->Lc + n->L) return MBD_E_INVALID;
@@ -984,15 +997,23 @@ extern "C" mbd_status mbd_get_plan(const mbd_net* n, int layer, int product, mbd
     const Layer& l = n->layers[i];
     gp = product == 0 ? &l.fwd : product == 1 ? &l.bwd_data : &l.bwd_weight;
   }
-  const TcGemm& g = *gp;
-  out->tile_m = 128 * g.MH * (g.pair ? 2 : 1);
-  out->tile_n = g.BN;
-  out->cta_pair = g.pair;
-  out->k_pieces = g.join > 1 ? g.join : g.k_splits;
-  out->tma_epilogue = g.te_planes ? 2 : g.te;
-  out->ctas = g.grid;
-  out->running_sum = g.join > 1 ? 2 : g.fix;
-  out->k_blocks = (g.K + 63) / 64;
+  fill_plan(*gp, out);
+  return MBD_OK;
+}
+
+extern "C" mbd_status mbd_plan_product(int variant, int64_t M, int64_t N, int64_t K, int k_pieces, int flags, int num_sms,
+                                       mbd_plan* out) {
+  if (!out || variant < 0 || variant > 2 || M < 1 || N < 1 || K < 1 || k_pieces < 1 || num_sms < 2) return MBD_E_INVALID;
+  if (flags & ~(MBD_PLAN_EXTRA_CUTS | MBD_PLAN_INTERMEDIATE | MBD_PLAN_BF16_RESULT)) return MBD_E_INVALID;
+  if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return MBD_E_UNSUPPORTED;
+  TcGemm g{};
+  g.variant = variant;
+  g.M = static_cast<int>(M); g.N = static_cast<int>(N); g.K = static_cast<int>(K);
+  g.k_splits = k_pieces;
+  g.allow_extra_split = (flags & MBD_PLAN_EXTRA_CUTS) != 0;
+  g.allow_fix = (flags & MBD_PLAN_INTERMEDIATE) != 0;
+  tc_gemm_plan(g, num_sms, (flags & MBD_PLAN_BF16_RESULT) != 0);
+  fill_plan(g, out);
   return MBD_OK;
 }
 

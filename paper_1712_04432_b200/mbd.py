@@ -31,7 +31,7 @@ EXPORTS = ["mbd_net_create", "mbd_net_destroy", "mbd_set_weights", "mbd_get_weig
            "mbd_comm_time", "mbd_redistribute_time", "mbd_total_time", "mbd_grid_table", "mbd_choose_grid",
            "mbd_enable_master_weights", "mbd_enable_momentum", "mbd_block_gemm_bf16", "mbd_block_reduce", "mbd_softmax_xent",
            "mbd_conv_stage_input", "mbd_conv_forward_layer", "mbd_conv_backward_layer", "mbd_conv_outer_rows",
-           "mbd_get_plan", "mbd_conv_forward_layer_rows", "mbd_conv_backward_layer_rows"]
+           "mbd_get_plan", "mbd_plan_product", "mbd_conv_forward_layer_rows", "mbd_conv_backward_layer_rows"]
 
 
 class MbdError(RuntimeError):
@@ -141,6 +141,7 @@ def lib():
         L.mbd_launch_count.argtypes = [vp]
         L.mbd_launch_count.restype = i64
         L.mbd_get_plan.argtypes = [vp, i32, i32, C.POINTER(Plan)]
+        L.mbd_plan_product.argtypes = [i32, i64, i64, i64, i32, i32, i32, C.POINTER(Plan)]
         L.mbd_gemm_bf16.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp, vp]
         L.mbd_gemm_bf16_noalloc.argtypes = [i32, i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
         L.mbd_selftest_timeout.argtypes = [i32, vp]
@@ -433,6 +434,17 @@ class Net:
         p = Plan()
         _check(lib().mbd_get_plan(self._h, layer, product, C.byref(p)), "mbd_get_plan")
         return {k: int(getattr(p, k)) for k, _ in Plan._fields_}
+
+
+PLAN_EXTRA_CUTS, PLAN_INTERMEDIATE, PLAN_BF16_RESULT = 1, 2, 4
+
+
+def plan_product(variant: int, M: int, N: int, K: int, k_pieces: int = 1, flags: int = 0, num_sms: int = 148) -> Dict[str, int]:
+    """mbd_plan_product: the launch plan of a stand-alone bf16 product, computed on the host (no device needed)."""
+    p = Plan()
+    _check(lib().mbd_plan_product(int(variant), C.c_int64(M), C.c_int64(N), C.c_int64(K), int(k_pieces), int(flags),
+                                  int(num_sms), C.byref(p)), "mbd_plan_product")
+    return {k: int(getattr(p, k)) for k, _ in Plan._fields_}
 
 
 def gemm_bf16(variant: int, A, B, k_splits: int = 1, return_partials: bool = False):
