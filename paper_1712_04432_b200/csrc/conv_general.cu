@@ -60,10 +60,22 @@ __device__ __forceinline__ long long pix_index(const Geo& g, int b, int q) {    
   return ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w + g.pw;
 }
 
+// The same pixel in the s^2 phase planes a strided layer reads its input through (see decimate_kernel): plane
+// (h mod s, w mod s) of the strip, at (h / s, w / s) in the geometry `go` of the layer's output.
+__device__ __forceinline__ long long plane_index(const Geo& g, const Geo& go, int s, int b, int q) {
+  const int h = q / g.W, w = q - h * g.W;
+  const int st = h / g.Hs, hl = h - st * g.Hs;
+  const int hq = hl / s, wq = w / s;
+  const long long z = static_cast<long long>(b) * g.P_r + st;
+  return ((hl - hq * s) * s + (w - wq * s)) * go.Ptot + (z * go.R + hq + go.ph) * go.Wp + wq + go.pw;
+}
+
 // WIDE: 64 channels per block, one run (no division by the channel count)
-template <bool WIDE>
+// PLANES: the destination is the phase planes of a stride-s layer (geometry go), not the tensor in geometry g: the input
+// of a strided first layer goes from NCHW straight into the form its products read
+template <bool WIDE, bool PLANES>
 __global__ void __launch_bounds__(256)
-nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C, StageTile st) {
+nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C, StageTile st, Geo go, int s) {
   __shared__ uint16_t tile[64][34];
   const int HW = g.H * g.W;
   const int b = blockIdx.y, q0 = blockIdx.x * 32 * st.G, c0 = blockIdx.z * st.cpb;
@@ -99,7 +111,7 @@ nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, 
   uint4 o;
   o.x = v[0] | (static_cast<uint32_t>(v[1]) << 16); o.y = v[2] | (static_cast<uint32_t>(v[3]) << 16);
   o.z = v[4] | (static_cast<uint32_t>(v[5]) << 16); o.w = v[6] | (static_cast<uint32_t>(v[7]) << 16);
-  *reinterpret_cast<uint4*>(dst + pix_index(g, b, q) * C + c0 + c) = o;
+  *reinterpret_cast<uint4*>(dst + (PLANES ? plane_index(g, go, s, b, q) : pix_index(g, b, q)) * C + c0 + c) = o;
 }
 
 template <bool WIDE>
@@ -463,6 +475,7 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
   // (256 bytes of slack behind the tensors a folded layer reads: its last rows reach up to 64 - C_in elements further)
   for (int i = 0; i <= L && ok; ++i) {
     const int C = i == 0 ? c->Cin[0] : c->Cout[i - 1];
+    if (i == 0 && c->stride[0] > 1) continue;          // the input of a strided first layer lives in its phase planes only
     ok = alloc(reinterpret_cast<void**>(&c->act[i]), static_cast<size_t>(c->geo[i].Ptot) * C * 2 + 256);
   }
   // internal weight layouts
@@ -649,14 +662,22 @@ mbd_status gconv_get_weights(GenConv* c, int i, void* K_dev) {
 }
 
 namespace {
-void stage(GenConv* c, const bf16* nchw, bf16* dst, const Geo& g, int C, bool fill_halos) {
+// go / s: the tensor is the input of a stride-s layer whose output has geometry *go: it is stored as that layer's
+// phase planes (dst = the planes), and the planes' padding and halo rows are fixed instead of the tensor's
+void stage(GenConv* c, const bf16* nchw, bf16* dst, const Geo& g, int C, bool fill_halos, const Geo* go = nullptr, int s = 1) {
   const StageTile t = stage_tile(C);
   const dim3 grid((g.H * g.W + 32 * t.G - 1) / (32 * t.G), static_cast<unsigned>(g.B), (C + t.cpb - 1) / t.cpb);
   c->prof->begin(MBD_K_HALO, 2.0 * g.B * C * g.H * g.W * 2.0, c->stream);
-  if (t.cpb == 64) nchw_to_pix_kernel<true><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t);
-  else nchw_to_pix_kernel<false><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t);
+  if (go) {
+    if (t.cpb == 64) nchw_to_pix_kernel<true, true><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t, *go, s);
+    else nchw_to_pix_kernel<false, true><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t, *go, s);
+  } else {
+    if (t.cpb == 64) nchw_to_pix_kernel<true, false><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t, g, 1);
+    else nchw_to_pix_kernel<false, false><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t, g, 1);
+  }
   c->prof->end();
-  pad_fix(c, dst, g, C, fill_halos);
+  if (go) pad_fix(c, dst, *go, C, fill_halos, s * s);
+  else pad_fix(c, dst, g, C, fill_halos);
 }
 void unstage(GenConv* c, const bf16* src, bf16* nchw, const Geo& g, int C) {
   const StageTile t = stage_tile(C);
@@ -669,7 +690,10 @@ void unstage(GenConv* c, const bf16* src, bf16* nchw, const Geo& g, int C) {
 }  // namespace
 
 mbd_status gconv_stage_input(GenConv* c, const void* X_nchw) {
-  stage(c, static_cast<const bf16*>(X_nchw), c->act[0], c->geo[0], c->Cin[0], true);     // the forward halo exchange of the input rides along
+  if (c->stride[0] > 1)      // a strided first layer: straight into its phase planes (the input has no other reader)
+    stage(c, static_cast<const bf16*>(X_nchw), c->xph[0], c->geo[0], c->Cin[0], true, &c->geo[1], c->stride[0]);
+  else
+    stage(c, static_cast<const bf16*>(X_nchw), c->act[0], c->geo[0], c->Cin[0], true);     // the forward halo exchange of the input rides along
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
@@ -679,7 +703,7 @@ mbd_status gconv_forward_layer(GenConv* c, int i, float* loss_sum_dev) {
   const Geo& go = c->geo[i + 1];
   const int s = c->stride[i];
   const double flops = 2.0 * c->B * go.H * go.W * c->taps[i] * c->Cin[i] * c->Cout[i];     // the method's flops
-  if (s > 1) {
+  if (s > 1 && i > 0) {       // (the network's input was staged as planes)
     // the input's own pixels sorted into the s^2 phase planes; their halo rows exchanged plane by plane
     decimate(c, c->act[i], c->xph[i], c->geo[i], go, c->Cin[i], s, true);
     pad_fix(c, c->xph[i], go, c->Cin[i], true, s * s);
