@@ -39,12 +39,13 @@ struct Geo {
 
 // ------------------------------------------------------------------------------ layout kernels
 // NCHW <-> pixel-major (own pixels only; padding and halos are the business of pad_fix_kernel).  A block moves a
-// tile of 64 rows x 32 pixels through shared memory, a row being one channel of a run of 32 consecutive pixels of
-// one image (pixels counted through the image, h * W + w: a channel plane is contiguous in NCHW), so that both sides
-// are accessed in runs: 64 bytes per channel on the NCHW side, 16 bytes x the layer's channels per pixel on the
-// pixel-major side.  With 64 channels or more the rows are 64 channels of one run; with fewer (cpb = C < 64 channels
-// per block) they are the channels of G = 64 / cpb runs, so that a block still moves about 4 KB (an 8-channel input
-// tensor: 256 pixels per block instead of 32).  grid = (ceil(H W / (32 G)), B, ceil(C / cpb)), 256 threads.
+// tile of 32 rows x 32 pixels of 32-bit words through shared memory, a row being one PAIR of channels of a run of 32
+// consecutive pixels of one image (pixels counted through the image, h * W + w: a channel plane is contiguous in
+// NCHW), so that both sides are accessed 16 bytes at a time -- 8 pixels of a channel on the NCHW side, 8 channels of a
+// pixel on the pixel-major side -- and shared memory holds whole words at an odd pitch (no bank conflicts in either
+// phase).  With 64 channels or more the rows are the 32 pairs of 64 channels of one run; with fewer (cpb = C < 64
+// channels per block) they are the pairs of G = 64 / cpb runs, so that a block still moves about 4 KB (an 8-channel
+// input tensor: 256 pixels per block instead of 32).  grid = (ceil(H W / (32 G)), B, ceil(C / cpb)), 128 threads.
 struct StageTile {
   int cpb, G;                        // channels per block (a multiple of 8, at most 64), pixel runs per block
 };
@@ -74,82 +75,100 @@ __device__ __forceinline__ long long plane_index(const Geo& g, const Geo& go, in
 // PLANES: the destination is the phase planes of a stride-s layer (geometry go), not the tensor in geometry g: the input
 // of a strided first layer goes from NCHW straight into the form its products read
 template <bool WIDE, bool PLANES>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 nchw_to_pix_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C, StageTile st, Geo go, int s) {
-  __shared__ uint16_t tile[64][34];
+  __shared__ uint32_t tile[32][33];                   // [pixel of its run][pair row]
   const int HW = g.H * g.W;
   const int b = blockIdx.y, q0 = blockIdx.x * 32 * st.G, c0 = blockIdx.z * st.cpb;
+  const int hp = st.cpb >> 1;                         // pair rows per run
   const int t = threadIdx.x;
   {
-    const int row = t >> 2, wq = (t & 3) * 8;         // row = (run, channel); pixels q .. q + 7 of that run
-    const int pg = WIDE ? 0 : row / st.cpb, c = row - pg * st.cpb;
-    const int q = q0 + pg * 32 + wq;
-    if (pg < st.G && c0 + c < C && q < HW) {
-      const bf16* p = src + (static_cast<long long>(b) * C + c0 + c) * HW + q;
+    const int pr = t >> 2, wq = (t & 3) * 8;          // pair row = (run, channel pair); pixels q .. q + 7 of that run
+    const int pg = WIDE ? 0 : pr / hp, cp = pr - pg * hp;
+    const int q = q0 + pg * 32 + wq, ch = c0 + 2 * cp;
+    if (pg < st.G && ch < C && q < HW) {
+      const bf16* p0 = src + (static_cast<long long>(b) * C + ch) * HW + q;
+      const bf16* p1 = p0 + HW;
+      uint16_t lo[8], hi[8];
       if ((HW & 7) == 0 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {      // 16 aligned bytes, all inside the plane
-        const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p));
-        const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+        const uint4 a = __ldcs(reinterpret_cast<const uint4*>(p0)), c = __ldcs(reinterpret_cast<const uint4*>(p1));
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          tile[row][wq + 2 * j] = static_cast<uint16_t>(wv[j] & 0xFFFFu);
-          tile[row][wq + 2 * j + 1] = static_cast<uint16_t>(wv[j] >> 16);
+        for (int i = 0; i < 4; ++i) {
+          lo[2 * i] = aw[i] & 0xFFFFu; lo[2 * i + 1] = aw[i] >> 16;
+          hi[2 * i] = cw[i] & 0xFFFFu; hi[2 * i + 1] = cw[i] >> 16;
         }
       } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) tile[row][wq + j] = q + j < HW ? __bfloat16_as_ushort(p[j]) : 0;
+        for (int i = 0; i < 8; ++i) {
+          const bool in = q + i < HW;
+          lo[i] = in ? __bfloat16_as_ushort(p0[i]) : 0;
+          hi[i] = in ? __bfloat16_as_ushort(p1[i]) : 0;
+        }
       }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) tile[wq + i][pr] = static_cast<uint32_t>(lo[i]) | (static_cast<uint32_t>(hi[i]) << 16);
     }
   }
   __syncthreads();
-  const int px = t >> 3, cg = t & 7;                  // rows 8 cg .. 8 cg + 7: eight channels of one run; pixel px of it
-  const int pg = WIDE ? 0 : cg * 8 / st.cpb, c = cg * 8 - pg * st.cpb;
-  const int q = q0 + pg * 32 + px;
-  if (pg >= st.G || q >= HW || c0 + c >= C) return;
-  uint16_t v[8];
+  const int px = t >> 2;                              // pixel px of its run; two groups of four pair rows = 8 channels each
 #pragma unroll
-  for (int j = 0; j < 8; ++j) v[j] = tile[cg * 8 + j][px];
-  uint4 o;
-  o.x = v[0] | (static_cast<uint32_t>(v[1]) << 16); o.y = v[2] | (static_cast<uint32_t>(v[3]) << 16);
-  o.z = v[4] | (static_cast<uint32_t>(v[5]) << 16); o.w = v[6] | (static_cast<uint32_t>(v[7]) << 16);
-  *reinterpret_cast<uint4*>(dst + (PLANES ? plane_index(g, go, s, b, q) : pix_index(g, b, q)) * C + c0 + c) = o;
+  for (int k = 0; k < 2; ++k) {
+    const int pr0 = ((t & 3) + 4 * k) * 4;          // (the four threads of a pixel cover 64 contiguous bytes per access)
+    const int pg = WIDE ? 0 : pr0 / hp, cp0 = pr0 - pg * hp;       // (hp is a multiple of 4: the four rows lie in one run)
+    const int q = q0 + pg * 32 + px, ch = c0 + 2 * cp0;
+    if (pg >= st.G || q >= HW || ch >= C) continue;
+    uint4 o;
+    o.x = tile[px][pr0]; o.y = tile[px][pr0 + 1]; o.z = tile[px][pr0 + 2]; o.w = tile[px][pr0 + 3];
+    *reinterpret_cast<uint4*>(dst + (PLANES ? plane_index(g, go, s, b, q) : pix_index(g, b, q)) * C + ch) = o;
+  }
 }
 
 template <bool WIDE>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 pix_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, int C, StageTile st) {
-  __shared__ uint16_t tile[64][34];
+  __shared__ uint32_t tile[32][33];
   const int HW = g.H * g.W;
   const int b = blockIdx.y, q0 = blockIdx.x * 32 * st.G, c0 = blockIdx.z * st.cpb;
+  const int hp = st.cpb >> 1;
   const int t = threadIdx.x;
   {
-    const int px = t >> 3, cg = t & 7;
-    const int pg = WIDE ? 0 : cg * 8 / st.cpb, c = cg * 8 - pg * st.cpb;
-    const int q = q0 + pg * 32 + px;
-    if (pg < st.G && q < HW && c0 + c < C) {
-      const uint4 v = *reinterpret_cast<const uint4*>(src + pix_index(g, b, q) * C + c0 + c);
-      const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+    const int px = t >> 2;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        tile[cg * 8 + 2 * j][px] = static_cast<uint16_t>(wv[j] & 0xFFFFu);
-        tile[cg * 8 + 2 * j + 1][px] = static_cast<uint16_t>(wv[j] >> 16);
-      }
+    for (int k = 0; k < 2; ++k) {
+      const int pr0 = ((t & 3) + 4 * k) * 4;          // (the four threads of a pixel cover 64 contiguous bytes per access)
+      const int pg = WIDE ? 0 : pr0 / hp, cp0 = pr0 - pg * hp;
+      const int q = q0 + pg * 32 + px, ch = c0 + 2 * cp0;
+      if (pg >= st.G || q >= HW || ch >= C) continue;
+      const uint4 v = *reinterpret_cast<const uint4*>(src + pix_index(g, b, q) * C + ch);
+      tile[px][pr0] = v.x; tile[px][pr0 + 1] = v.y; tile[px][pr0 + 2] = v.z; tile[px][pr0 + 3] = v.w;
     }
   }
   __syncthreads();
-  const int row = t >> 2, wq = (t & 3) * 8;
-  const int pg = WIDE ? 0 : row / st.cpb, c = row - pg * st.cpb;
-  const int q = q0 + pg * 32 + wq;
-  if (pg >= st.G || c0 + c >= C || q >= HW) return;
-  bf16* p = dst + (static_cast<long long>(b) * C + c0 + c) * HW + q;
+  const int pr = t >> 2, wq = (t & 3) * 8;
+  const int pg = WIDE ? 0 : pr / hp, cp = pr - pg * hp;
+  const int q = q0 + pg * 32 + wq, ch = c0 + 2 * cp;
+  if (pg >= st.G || ch >= C || q >= HW) return;
+  uint32_t w[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) w[i] = tile[wq + i][pr];
+  bf16* p0 = dst + (static_cast<long long>(b) * C + ch) * HW + q;
+  bf16* p1 = p0 + HW;
   if ((HW & 7) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
-    uint4 v;
-    v.x = tile[row][wq + 0] | (static_cast<uint32_t>(tile[row][wq + 1]) << 16); v.y = tile[row][wq + 2] | (static_cast<uint32_t>(tile[row][wq + 3]) << 16);
-    v.z = tile[row][wq + 4] | (static_cast<uint32_t>(tile[row][wq + 5]) << 16); v.w = tile[row][wq + 6] | (static_cast<uint32_t>(tile[row][wq + 7]) << 16);
-    *reinterpret_cast<uint4*>(p) = v;
+    uint4 a, c;
+    a.x = (w[0] & 0xFFFFu) | (w[1] << 16); a.y = (w[2] & 0xFFFFu) | (w[3] << 16);
+    a.z = (w[4] & 0xFFFFu) | (w[5] << 16); a.w = (w[6] & 0xFFFFu) | (w[7] << 16);
+    c.x = (w[0] >> 16) | (w[1] & 0xFFFF0000u); c.y = (w[2] >> 16) | (w[3] & 0xFFFF0000u);
+    c.z = (w[4] >> 16) | (w[5] & 0xFFFF0000u); c.w = (w[6] >> 16) | (w[7] & 0xFFFF0000u);
+    *reinterpret_cast<uint4*>(p0) = a;
+    *reinterpret_cast<uint4*>(p1) = c;
   } else {
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
-      if (q + j < HW) p[j] = __ushort_as_bfloat16(tile[row][wq + j]);
+    for (int i = 0; i < 8; ++i)
+      if (q + i < HW) {
+        p0[i] = __ushort_as_bfloat16(static_cast<uint16_t>(w[i] & 0xFFFFu));
+        p1[i] = __ushort_as_bfloat16(static_cast<uint16_t>(w[i] >> 16));
+      }
   }
 }
 
@@ -669,11 +688,11 @@ void stage(GenConv* c, const bf16* nchw, bf16* dst, const Geo& g, int C, bool fi
   const dim3 grid((g.H * g.W + 32 * t.G - 1) / (32 * t.G), static_cast<unsigned>(g.B), (C + t.cpb - 1) / t.cpb);
   c->prof->begin(MBD_K_HALO, 2.0 * g.B * C * g.H * g.W * 2.0, c->stream);
   if (go) {
-    if (t.cpb == 64) nchw_to_pix_kernel<true, true><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t, *go, s);
-    else nchw_to_pix_kernel<false, true><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t, *go, s);
+    if (t.cpb == 64) nchw_to_pix_kernel<true, true><<<grid, 128, 0, c->stream>>>(nchw, dst, g, C, t, *go, s);
+    else nchw_to_pix_kernel<false, true><<<grid, 128, 0, c->stream>>>(nchw, dst, g, C, t, *go, s);
   } else {
-    if (t.cpb == 64) nchw_to_pix_kernel<true, false><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t, g, 1);
-    else nchw_to_pix_kernel<false, false><<<grid, 256, 0, c->stream>>>(nchw, dst, g, C, t, g, 1);
+    if (t.cpb == 64) nchw_to_pix_kernel<true, false><<<grid, 128, 0, c->stream>>>(nchw, dst, g, C, t, g, 1);
+    else nchw_to_pix_kernel<false, false><<<grid, 128, 0, c->stream>>>(nchw, dst, g, C, t, g, 1);
   }
   c->prof->end();
   if (go) pad_fix(c, dst, *go, C, fill_halos, s * s);
@@ -683,8 +702,8 @@ void unstage(GenConv* c, const bf16* src, bf16* nchw, const Geo& g, int C) {
   const StageTile t = stage_tile(C);
   const dim3 grid((g.H * g.W + 32 * t.G - 1) / (32 * t.G), static_cast<unsigned>(g.B), (C + t.cpb - 1) / t.cpb);
   c->prof->begin(MBD_K_HALO, 2.0 * g.B * C * g.H * g.W * 2.0, c->stream);
-  if (t.cpb == 64) pix_to_nchw_kernel<true><<<grid, 256, 0, c->stream>>>(src, nchw, g, C, t);
-  else pix_to_nchw_kernel<false><<<grid, 256, 0, c->stream>>>(src, nchw, g, C, t);
+  if (t.cpb == 64) pix_to_nchw_kernel<true><<<grid, 128, 0, c->stream>>>(src, nchw, g, C, t);
+  else pix_to_nchw_kernel<false><<<grid, 128, 0, c->stream>>>(src, nchw, g, C, t);
   c->prof->end();
 }
 }  // namespace
