@@ -92,6 +92,7 @@ struct Params {
   int* status;
   int te;                 // epilogue moves its global data with TMA through shared memory
   int te_prefetch;        // TMA epilogue requests its boxes one tile ahead
+  int te_ring;            // every CTA has one work unit: the epilogue's staging boxes lie in the operand ring, which is idle by then
   int fix;                // running sum: piece s adds its accumulator to the sum pieces 0..s-1 left in `partials`
                           // (1: the pieces of a raster group follow one another; 2: all tiles piece by piece)
   int* flags;             // fix: one word per (tile, CTA of the pair, 128-row half, epilogue warp); zero between launches
@@ -246,7 +247,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int acc_stride = join * ACC_COLS;
   const int acc_bufs = JOIN && join > 1 ? (2 * acc_stride <= 512 ? 2 : 1) : ACC_BUFS;
   const int tmem_cols = JOIN && join > 1 ? 512 : TMEM_COLS;
-  const int stages = te ? (p.te == 2 ? STAGES_TEP : STAGES_TE) : STAGES;
+  // One work unit per CTA (p.te_ring): nothing is loaded after the unit's last k-block, so the staging boxes of the
+  // TMA epilogue take the ring's first bytes once the accumulator is complete and the ring keeps all its stages.
+  const bool te_ring = te && p.te_ring != 0;
+  const int stages = te && !te_ring ? (p.te == 2 ? STAGES_TEP : STAGES_TE) : STAGES;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;        // 0 = the CTA that issues the MMAs
@@ -422,7 +426,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // piece the epilogue is most of a tile's time, and row-per-lane stores of 16 bytes keep the LSU busy
       // for 32 cycles each; the bulk store takes the LSU out of the path.
       const int e = warp - 2;
-      const uint32_t stg = ring + STAGES_TEP * STAGE_BYTES + e * (2 * 4096);
+      const uint32_t stg = ring + (te_ring ? 0 : STAGES_TEP * STAGE_BYTES) + e * (2 * 4096);
       uint8_t* stg_gen = smem_raw + (stg - smem_u32(smem_raw));
       int it = 0, nb = 0;
       bool ok = true;
@@ -478,7 +482,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // tile's epilogue and the next tile's main loop instead of standing between two tiles (with K = B
       // of a few hundred, a tile's main loop is only a few microseconds long).
       const int e = warp - 2;
-      const uint32_t stg = ring + STAGES_TE * STAGE_BYTES + e * (TE_BOXES * 4096);
+      const uint32_t stg = ring + (te_ring ? 0 : STAGES_TE * STAGE_BYTES) + e * (TE_BOXES * 4096);
       uint8_t* stg_gen = smem_raw + (stg - smem_u32(smem_raw));
       uint32_t lphase = 0;
       const bool need_load = p.epi.op == EPI_SGD || (p.epi.op == EPI_MASK && p.epi.mask != nullptr);
@@ -1101,9 +1105,14 @@ void tc_gemm_plan(TcGemm& g, int num_sms, bool want_te) {
   // its predecessor's row-per-lane stores are (measured: batch-512 backward-weight products in 16 pieces of 8
   // k-blocks 0.49 -> 0.31 ms); long pieces hide those stores and keep the two extra ring stages instead
   // (8192-deep pieces of 64 k-blocks on CTA pairs: 2.5 % slower with the bulk stores).  The map is made at launch.
+  // A launch with one work unit per CTA has no next tile to hide stores under, and its ring is idle once the unit's
+  // accumulator is complete: the staging boxes then lie in the ring itself (te_ring), all stages are kept, and pieces
+  // of any length leave by TMA store (measured: the forward products of the batch-256 network, cut in 4 by the planner).
   {
     const int kb_piece = kb_total / (g.k_splits > 0 ? g.k_splits : 1);
-    g.te_planes = g.k_splits > 1 && !g.fix && g.MH == 1 && (g.N & 3) == 0 && kb_piece < 32 && !getenv("MBD_TC_NO_TE");
+    const int slots = g.pair ? num_sms / 2 : num_sms;
+    g.te_ring = total <= slots && !getenv("MBD_TC_NO_TE_RING");                     // tuning knob
+    g.te_planes = g.k_splits > 1 && !g.fix && g.MH == 1 && (g.N & 3) == 0 && (kb_piece < 32 || g.te_ring) && !getenv("MBD_TC_NO_TE");
   }
   // TMA epilogue: bf16 output of an unsplit contraction on 128-row tiles (the maps are made by tc_gemm_prepare)
   g.te = want_te && g.MH == 1 && g.k_splits == 1 && !getenv("MBD_TC_NO_TE") ? 1 : 0;
@@ -1150,6 +1159,7 @@ cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
   p.fix = g.fix && g.pair && g.flags != nullptr;
   if (p.fix && getenv("MBD_FIX_PLAIN_ORDER")) p.fix = 2;                 // tuning knob
   p.te_prefetch = getenv("MBD_TE_NO_PREFETCH") ? 0 : 1;                  // tuning knob
+  p.te_ring = 0;
   p.flags = g.flags;
   p.join = g.join > 1 ? g.join : 1;
   p.cv = g.cv;
@@ -1165,12 +1175,15 @@ cudaError_t tc_gemm_launch(const TcGemm& g, cudaStream_t stream) {
       g.planes_base = g.partials;
     }
     p.te = 2;
+    p.te_ring = g.te_ring;
     TcGemm h = g;
     h.tmOut = g.tmPlanes;
     if (g.variant == 0) return launch_t<0, 0>(h, p, stream);
     if (g.variant == 1) return launch_t<0, 1>(h, p, stream);
     return launch_t<1, 1>(h, p, stream);
   }
+  // (a tail operation that reads -- old weights, a mask source -- requests its boxes while the ring is still in use)
+  p.te_ring = p.te == 1 && g.te_ring && (g.epi.op == EPI_ACT || (g.epi.op == EPI_MASK && g.epi.mask == nullptr));
   if (g.variant == 0) return launch_t<0, 0>(g, p, stream);
   if (g.variant == 1) return launch_t<0, 1>(g, p, stream);
   return launch_t<1, 1>(g, p, stream);

@@ -110,6 +110,7 @@ struct TcGemm {
   CUtensorMap tmOut, tmAux;   // output / mask-source maps of the TMA epilogue (valid when te)
   int te;                     // plan allows the TMA epilogue for te_epi
   int te_planes;              // out: the S > 1 fp32 planes leave through TMA stores (short pieces on 128-row tiles)
+  int te_ring;                // out: one work unit per CTA: the TMA epilogue's staging boxes lie in the idle operand ring
   Epi te_epi;
   int variant;
   int BN;               // CTA tile width: 256 or 128

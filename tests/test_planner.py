@@ -87,8 +87,10 @@ def test_plan_invariants_over_random_products():
             assert p["k_pieces"] in (2, 4) and p["k_pieces"] * (rows_per_cta // 128) * p["tile_n"] <= 512, what
         if p["tma_epilogue"] == 1:                  # bf16 result through TMA boxes: 128 rows per CTA, nothing left for a reduction
             assert flags & BF and rows_per_cta == 128 and (p["k_pieces"] == 1 or p["running_sum"] == 2), what
-        if p["tma_epilogue"] == 2:                  # planes stored by TMA: short pieces that are kept
-            assert p["k_pieces"] > 1 and p["running_sum"] == 0 and rows_per_cta == 128 and kb // p["k_pieces"] < 32, what
+        if p["tma_epilogue"] == 2:                  # planes stored by TMA: kept pieces that are short, or one work unit per CTA
+            slots = sms // 2 if p["cta_pair"] else sms
+            assert p["k_pieces"] > 1 and p["running_sum"] == 0 and rows_per_cta == 128, what
+            assert kb // p["k_pieces"] < 32 or units(p, M, N) <= slots, what
 
 
 def test_plan_query_rejects_bad_arguments():
