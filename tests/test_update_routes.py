@@ -114,6 +114,32 @@ def test_planes_stored_by_tma_equal_planes_stored_from_registers(monkeypatch, ne
     compare_fc_step(a, o, TOL, False, init=inp, require_sized=True)
 
 
+def test_planes_stored_from_the_idle_ring_equal_planes_stored_from_registers(monkeypatch):
+    # A product whose work units all run at once (one per CTA) has an idle operand ring once its accumulator is
+    # complete: the staging boxes of the TMA stores lie there, so pieces of any length leave by TMA.  The batch-256
+    # network's first forward product (256 x 4096 x 9216, cut in 4 by the planner: 36 k-blocks per piece, 128 CTAs) is
+    # such a launch; the same planes stored by the epilogue's own stores must give every bit of the step.
+    from paper_1712_04432_b200 import mbd
+    w = I.WORKLOADS["cfg2"]
+    inp = I.make_inputs(w, seed=5)
+
+    def fwd_plan():
+        net = mbd.Net(mbd.fc_layers(w.dims, bias=True), w.B, 1, 1, mbd.BF16, mbd.LOSS_SOFTMAX_CE, 2)
+        q = net.plan(0, 0)
+        net.close()
+        return q
+    q = fwd_plan()
+    assert q["k_pieces"] == 4 and q["k_blocks"] // q["k_pieces"] >= 32 and q["tma_epilogue"] == 2, q
+    a = gpu_fc_step(w, inp, (1, 1), max_partials=2, fused=True)
+    monkeypatch.setenv("MBD_TC_NO_TE_RING", "1")
+    assert fwd_plan()["tma_epilogue"] == 0
+    b = gpu_fc_step(w, inp, (1, 1), max_partials=2, fused=True)
+    for i in range(len(inp.Ws)):
+        assert np.array_equal(a["act"][i], b["act"][i]) and np.array_equal(a["dY"][i], b["dY"][i]), i
+        assert np.array_equal(a["new_W"][i], b["new_W"][i]) and np.array_equal(a["new_b"][i], b["new_b"][i]), i
+    assert a["J"] == b["J"]
+
+
 @pytest.mark.parametrize("grid,mp", [((1, 4), 2), ((4, 8), 4), ((8, 1), 2), ((4, 4), 2)])
 @pytest.mark.parametrize("fused", [True, False])
 def test_pieces_joined_in_tensor_memory_equal_planes_and_reduction(monkeypatch, net_case, grid, mp, fused):
