@@ -16,7 +16,7 @@
 // Tile shapes: 128 x 128, 128 x 256, 256 x 256 per CTA, or 256 x 256 per CTA pair
 // (cta_group::2); tc_gemm_prepare picks one per contraction with a small cost model.  With a
 // bf16 result on 128-row tiles the epilogue moves all its global data by TMA through per-warp
-// staging boxes.  Tuning knobs (environment): MBD_TC_MH, MBD_TC_BN, MBD_TC_PAIR, MBD_TC_GROUP_M, MBD_TC_DEBUG, MBD_TC_X_POW2,
+// staging boxes.  Tuning knobs (environment): MBD_TC_MH, MBD_TC_BN, MBD_TC_PAIR, MBD_TC_GROUP_M, MBD_TC_DEBUG, MBD_TC_X_POW2, MBD_TC_NO_TE_RING,
 // MBD_TC_NO_TE.
 // Every mbarrier wait is bounded; on time-out the kernel records a code and leaves.
 #include <stdio.h>
