@@ -103,3 +103,25 @@ def test_plan_query_rejects_bad_arguments():
     with pytest.raises(mbd.MbdError) as e:
         mbd.plan_product(0, 1 << 31, 128, 128, 1, 0, SMS)
     assert e.value.status == mbd.E_UNSUPPORTED
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name", ["cfg2", "cfg3"])
+def test_host_plan_is_the_plan_a_network_runs(name):
+    # what mbd_plan_product computes without a device is what mbd_net_create plans for the products of a network on
+    # the 1 x 1 grid: forward and backward-data may be cut further by the planner, every piece is intermediate, hidden
+    # results are bf16
+    import torch
+    from paper_1712_04432_b200 import inputs
+    w = inputs.WORKLOADS[name]
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    net = mbd.Net(mbd.fc_layers(w.dims, bias=True), w.B, 1, 1, mbd.BF16, mbd.LOSS_SOFTMAX_CE, 2)
+    L = len(w.dims) - 1
+    for i in range(L):
+        d_in, d_out = w.dims[i], w.dims[i + 1]
+        if i < L - 1:                                             # (the last layer's logits are fp32: no TMA epilogue)
+            assert net.plan(i, 0) == mbd.plan_product(0, w.B, d_out, d_in, 1, X | I | BF, sms), (i, "forward")
+        if i > 0:
+            assert net.plan(i, 1) == mbd.plan_product(1, w.B, d_in, d_out, 1, X | I | BF, sms), (i, "backward-data")
+        assert net.plan(i, 2) == mbd.plan_product(2, d_out, d_in, w.B, 1, I | BF, sms), (i, "backward-weight")
+    net.close()
