@@ -53,7 +53,9 @@ class Conv3x3:
     K is [C_out, C_in, k_h, k_w].
     split (used by the blocked step only): "domain" = row strips over the P_r groups (Section 2.2 / 2.4);
     "batch" = the layer forced onto a 1 x P grid, P = P_r P_c (Section 3's improved case: pure batch
-    parallelism in the convolutional layers, P_r x P_c grids in the fully connected ones)."""
+    parallelism in the convolutional layers, P_r x P_c grids in the fully connected ones);
+    "model" = the layer in L_M (Section 2.3 / 2.4, Eq. 8 with |W| = k_h k_w C_in C_out): the P_r groups split the
+    output channels (the rows of the layer's weight matrix), the P_c groups the batch, no strips."""
     K: np.ndarray
     relu: bool = True
     split: str = "domain"
@@ -483,6 +485,27 @@ def conv3x3_dK_grid(dY, X, P_r, P_c, ksize=(3, 3)):
     return dK, parts
 
 
+def conv3x3_model_blocked(K, X, P_r):
+    """Forward of a model-parallel convolution: process group r computes the output channels of its block of
+    filters, [o0, o1) = balanced range r of C_out, from the whole input; the blocks are concatenated (the
+    all-gather of Appendix A.1).  No sum is formed, so the result is conv3x3(K, X) itself."""
+    K = np.asarray(K, F64)
+    return np.concatenate([conv3x3(K[o0:o1], X) for (o0, o1) in balanced_ranges(K.shape[0], P_r)], axis=1)
+
+
+def conv3x3_dX_model_blocked(K, dY, P_r):
+    """Backward-data of a model-parallel convolution (Appendix A.2: dX = sum over the P_r groups of W_r^T dY_r):
+    group r back-propagates the gradient of its own output channels through its own filters; the P_r partial
+    results are added in ascending r (the all-reduce of Eq. 8's second term).  Returns (sum, partials)."""
+    K = np.asarray(K, F64)
+    dY = np.asarray(dY, F64)
+    parts = [conv3x3_dX(K[o0:o1], dY[:, o0:o1]) for (o0, o1) in balanced_ranges(K.shape[0], P_r)]
+    total = np.zeros_like(parts[0])
+    for p in parts:
+        total = total + p
+    return total, parts
+
+
 def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
                        P_r: int, P_c: int, store=None):
     """The step of `train_step`, every contraction formed block by block over
@@ -491,13 +514,16 @@ def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
     batch over P_c; convolution layers split the image into P_r row strips and
     the batch over P_c (Eq. 9: their weight gradient is summed over all
     P = P_r P_c processes); convolution layers with split == "batch" are cut into
-    P_r P_c batch blocks and no strips (Section 3's improved case)."""
+    P_r P_c batch blocks and no strips (Section 3's improved case); convolution layers with split == "model"
+    split their output channels over P_r and the batch over P_c, like an FC layer."""
     L = len(layers)
     Xs = [np.asarray(X1, F64)]
     Ys = []
     for i, lay in enumerate(layers):
         if isinstance(lay, FC):
             Y = fc_forward_blocked(lay.W, Xs[i], lay.b, P_r, P_c)
+        elif lay.split == "model":
+            Y = conv3x3_model_blocked(lay.K, Xs[i], P_r)
         else:
             Y = conv3x3_strips(lay.K, Xs[i], 1 if lay.split == "batch" else P_r)
         Ys.append(Y)
@@ -519,6 +545,8 @@ def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
                 for (c0, c1) in balanced_ranges(B, P_c):
                     db = db + dYs[i][:, c0:c1].sum(axis=1)
                 dbs[i] = db
+        elif lay.split == "model":
+            dWs[i], _ = conv3x3_dK_grid(dYs[i], Xs[i], 1, P_c, lay.K.shape[2:])            # rows of dK are independent: one partial per batch block
         elif lay.split == "batch":
             dWs[i], _ = conv3x3_dK_grid(dYs[i], Xs[i], 1, P_r * P_c, lay.K.shape[2:])      # one partial per process of the 1 x P grid
         else:
@@ -526,6 +554,8 @@ def train_step_blocked(layers: Sequence, X1, labels, loss: str, eta: float,
         if i > 0:
             if isinstance(lay, FC):
                 dXs[i], _ = fc_dX_blocked(lay.W, dYs[i], P_r, P_c)
+            elif lay.split == "model":
+                dXs[i], _ = conv3x3_dX_model_blocked(lay.K, dYs[i], P_r)
             else:
                 dXs[i] = conv3x3_dX_strips(lay.K, dYs[i], 1 if lay.split == "batch" else P_r)
             dXs[i] = _below(dXs[i], Ys[i - 1])

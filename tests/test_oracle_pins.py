@@ -626,6 +626,33 @@ def test_batch_split_convolutions_in_the_blocked_step(grid):
         assert np.array_equal(c["dWs"][i], d["dWs"][i]) and np.array_equal(c["Ys"][i], d["Ys"][i])
 
 
+@pytest.mark.parametrize("grid", [(2, 3), (4, 1), (3, 2), (1, 6)])
+def test_model_split_convolutions_in_the_blocked_step(grid):
+    """Convolutions in L_M (Section 2.3 / 2.4): output channels over the P_r groups, batch over P_c.  Re-blocking changes no
+    sum (the step equals the un-blocked one); a group's partial of dX is the back-propagation of ITS output channels alone
+    (brute force with the other filters zeroed), and the forward blocks are the un-blocked output's channels."""
+    import dataclasses
+    layers, X, labels = mixed_case(78, B=6, H=8)
+    model = [dataclasses.replace(l, split="model") if isinstance(l, O.Conv3x3) else l for l in layers]
+    a = O.train_step(layers, X, labels, "softmax_ce", 0.01)
+    b = O.train_step_blocked(model, X, labels, "softmax_ce", 0.01, *grid)
+    assert abs(a["J"] - b["J"]) < 1e-12 * abs(a["J"])
+    for i in range(4):
+        assert relerr(b["Ys"][i], a["Ys"][i]) < 1e-12 and relerr(b["dWs"][i], a["dWs"][i]) < 1e-12
+        assert relerr(b["new_W"][i], a["new_W"][i]) < 1e-12
+    for i in range(1, 4):
+        assert relerr(b["dXs"][i], a["dXs"][i]) < 1e-12
+    K, Xc, dY = conv_case(seed=79)
+    P_r = grid[0]
+    assert relerr(O.conv3x3_model_blocked(K, Xc, P_r), O.conv3x3(K, Xc)) < 1e-13        # (no sum is formed: library blocking only)
+    total, parts = O.conv3x3_dX_model_blocked(K, dY, P_r)
+    assert len(parts) == P_r and relerr(total, O.conv3x3_dX(K, dY)) < 1e-13
+    r = P_r - 1
+    o0, o1 = O.balanced_ranges(K.shape[0], P_r)[r]
+    Kz = np.zeros_like(K); Kz[o0:o1] = K[o0:o1]
+    assert relerr(parts[r], brute.conv3x3_dX(Kz, dY)) < 1e-12 if o1 > o0 else np.all(parts[r] == 0)
+
+
 def test_conv_weight_gradient_partials_over_the_whole_grid():
     """P_r x P_c partials, one per process, whose sum is the un-blocked gradient (last term of Eq. 9)."""
     r = rng(75)
