@@ -150,6 +150,12 @@ enum {
  * a strip would be shorter than its halo, or (batch-split convolutions) P_r P_c > B.
  * Batch-split convolutions (MBD_SPLIT_BATCH) are cut into P_r P_c batch blocks and no strips; between them
  * and the fully connected layers on P_r x P_c lies the re-distribution of Eq. 6 (mbd_redistribute_time).
+ * Model-split convolutions (MBD_SPLIT_MODEL: convolutions in L_M, Eq. 8 with |W| = k_h k_w C_in C_out) are cut like
+ * a fully connected layer: the P_r groups split the output channels, the P_c groups the batch, no strips; dX is the
+ * sum over the groups' partial results (min(P_r, max_partials) partial sums, added in ascending group order), dK a
+ * sum over the batch blocks.  Stride 1, and C_out a multiple of 64 P_r (a group's channels are whole 64-channel
+ * blocks of the backward-data product's K range): MBD_E_UNSUPPORTED otherwise.  All convolutions of a network are
+ * split alike.
  * Convolutions (kind MBD_CONV3X3 whatever the kernel size; Section 2.2): zero padding floor(k/2), k_h and
  * k_w odd and at most 11, stride 1 to 4 (the same in both directions), C_in and C_out multiples of 8, C_in of a layer =
  * C_out of the layer below, H x W of a layer = the output size of the layer below (H/s x W/s of its input);

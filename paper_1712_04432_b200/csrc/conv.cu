@@ -1108,11 +1108,11 @@ void launch_stage_in(ConvNet* c, const bf16* nchw, bf16* strips) {
 }  // namespace
 
 mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, int max_partials, int num_sms, int* status,
-                       cudaStream_t stream, Profiler* prof, bool fc_above, ConvNet** out) {
+                       cudaStream_t stream, Profiler* prof, bool fc_above, int model_P_r, ConvNet** out) {
   if (gconv_needed(layers, L)) {
     ConvNet* c = new (std::nothrow) ConvNet();
     if (!c) return MBD_E_ALLOC;
-    const mbd_status s = gconv_create(layers, L, B, P_r, P_c, max_partials, num_sms, status, stream, prof, fc_above, &c->gen);
+    const mbd_status s = gconv_create(layers, L, B, P_r, P_c, max_partials, num_sms, status, stream, prof, fc_above, model_P_r, &c->gen);
     if (s != MBD_OK) { delete c; return s; }
     c->L = L; c->B = B;
     *out = c;

@@ -298,6 +298,7 @@ struct GenConv {
   int L = 0;
   int64_t B = 0;
   int P_r = 1, P = 1, S = 1;              // strips; processes of the grid; fp32 partial sums per weight gradient asked for
+  int model_P_r = 1, S_dx = 1;            // model-parallel layers: groups that split the output channels; partial sums per dX asked for
   std::vector<Geo> geo;                   // geometry of tensor i (act[i]; dY[i] has that of act[i + 1])
   std::vector<int> Cin, Cout, kh, kw, relu, taps, Cp, stride;
   std::vector<int> ldw;                   // columns of the internal weight matrix of layer i
@@ -423,6 +424,7 @@ bool gconv_needed(const mbd_layer* layers, int L) {
     const mbd_layer& l = layers[i];
     const bool k3 = l.kh == 3 && l.kw == 3, k1 = l.kh == 1 && l.kw == 1;
     if (!(k3 || k1) || l.C_in != 64 || l.C_out != 64 || l.stride > 1) return true;
+    if (l.split == MBD_SPLIT_MODEL) return true;      // output channels over the P_r groups: products with a cut of K over channel blocks
   }
   return false;
 }
@@ -444,7 +446,7 @@ void gconv_destroy(GenConv* c) {
 }
 
 mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, int max_partials, int num_sms, int* status,
-                        cudaStream_t stream, Profiler* prof, bool fc_above, GenConv** out) {
+                        cudaStream_t stream, Profiler* prof, bool fc_above, int model_P_r, GenConv** out) {
   if (tc_gemm_init() != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
   // one padding for every tensor: what the widest reach of any layer needs at the resolution it works in
   int ph = 0, pw = 0, H = layers[0].H, W = layers[0].W;
@@ -475,6 +477,11 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
   }
   c->P = P_r * P_c;
   c->S = max_partials < 1 ? 1 : std::min(c->P, max_partials);
+  // Model-parallel layers (Eq. 8): no strips (P_r = 1 here), the weight gradient's rows are independent, so its partial
+  // sums are over the P_c batch blocks (c->S above), and dX = sum over the model_P_r groups of W_r^T dY_r is a cut of
+  // backward-data's K range over blocks of output channels
+  c->model_P_r = model_P_r < 1 ? 1 : model_P_r;
+  c->S_dx = max_partials < 1 ? 1 : std::min(c->model_P_r, max_partials);
   auto alloc = [&](void** p, size_t bytes) -> bool {
     if (cudaMalloc(p, bytes) != cudaSuccess) { (void)cudaGetLastError(); *p = nullptr; return false; }
     return cudaMemsetAsync(*p, 0, bytes, stream) == cudaSuccess;
@@ -573,8 +580,10 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
       for (int q = 0; q < s * s; ++q) {
         TcGemm& d = c->bwd_data[i][q];
         d = TcGemm{};
-        d.variant = 1; d.M = M; d.N = Cin; d.k_splits = 1; d.status = status;
+        d.variant = 1; d.M = M; d.N = Cin; d.k_splits = c->S_dx; d.status = status;
+        d.allow_fix = c->S_dx < c->model_P_r;          // fewer partial sums than groups: intermediate ones, they may stay in tensor memory
         d.cv.mode = 2; d.cv.blocks = Cop / 64; d.cv.Cp = Cp;
+        d.cv.chan_major = c->model_P_r > 1;            // pieces of K = blocks of output channels, every tap of each
         int n = 0;
         for (int t = 0; t < taps; ++t)
           if (plane[t] == q) { d.cv.off[n] = off[t]; d.cv.tap[n] = t; ++n; }
@@ -587,6 +596,7 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
         const bf16* maskp = !c->relu[i - 1] ? nullptr : (s > 1 ? c->xph[i] + static_cast<size_t>(q) * M * Cin : c->act[i]);
         const Epi ed = make_epi_mask(outp, Cin, maskp, Cin);
         if (tc_gemm_prepare(d, c->dY[i], Cout, c->Wm[i], ldw, num_sms, &ed) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
+        if (d.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(d.k_splits) * M * Cin);
       }
     }
     // backward-weight: few output tiles, a very long K (all pixels): the planner cuts K to fill the SMs

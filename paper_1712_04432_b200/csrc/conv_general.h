@@ -12,7 +12,7 @@ namespace mbd {
 struct GenConv;
 bool gconv_needed(const mbd_layer* layers, int L);
 mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, int max_partials, int num_sms, int* status,
-                        cudaStream_t stream, Profiler* prof, bool fc_above, GenConv** out);
+                        cudaStream_t stream, Profiler* prof, bool fc_above, int model_P_r, GenConv** out);
 void gconv_destroy(GenConv* c);
 mbd_status gconv_set_weights(GenConv* c, int layer, const void* K_dev);     // K[C_out][C_in][k_h][k_w] bf16
 mbd_status gconv_get_weights(GenConv* c, int layer, void* K_dev);

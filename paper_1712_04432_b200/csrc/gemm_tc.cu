@@ -332,7 +332,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           } else if (A_MN == 0) {
             // convolution, forward (B K-major) or backward-data (B MN-major): k-block = (tap, 64-channel block)
-            const int t = kb / p.cv.blocks, cb = kb - t * p.cv.blocks;
+            int t, cb;
+            if (p.cv.chan_major) { cb = kb / p.cv.taps; t = kb - cb * p.cv.taps; }
+            else { t = kb / p.cv.blocks; cb = kb - t * p.cv.blocks; }
             load(sa, &tmA, cb * 64, B_MN == 0 ? row0 + p.cv.off[t] : row0 - p.cv.off[t]);
             if (B_MN == 0) {
               load(sb, &tmB, kb * BK, col0);

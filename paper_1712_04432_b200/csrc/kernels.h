@@ -103,6 +103,8 @@ struct ConvShift {
   int mode, taps, blocks, Cp;      // blocks: 64-wide k-blocks per tap (modes 1, 2)
   int off[MAX_TAPS];
   int tap[MAX_TAPS];               // mode 2: weight-matrix tap of the j-th tap of this product (identity for stride 1)
+  int chan_major;                  // mode 2: k-block = (64-channel block, tap) instead of (tap, block): a cut of K into pieces
+                                   // is then a cut of the output channels into blocks (model-parallel convolutions)
 };
 
 struct TcGemm {

@@ -313,10 +313,16 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
       if (l.kh < 1 || l.kw < 1 || l.kh > 11 || l.kw > 11 || l.kh % 2 == 0 || l.kw % 2 == 0 || dtype != MBD_BF16) return MBD_E_UNSUPPORTED;
       if (l.C_in < 8 || l.C_out < 8 || l.C_in % 8 || l.C_out % 8) return MBD_E_UNSUPPORTED;
       if (i > 0 && l.C_in != layers[i - 1].C_out) return MBD_E_INVALID;
-      if (l.split != MBD_SPLIT_DOMAIN && l.split != MBD_SPLIT_BATCH) return MBD_E_UNSUPPORTED;
+      if (l.split != MBD_SPLIT_DOMAIN && l.split != MBD_SPLIT_BATCH && l.split != MBD_SPLIT_MODEL) return MBD_E_INVALID;
       if (l.split != layers[0].split) return MBD_E_UNSUPPORTED;          // all convolutions split alike
       if (l.split == MBD_SPLIT_BATCH) {                                  // 1 x P: one sample per process at least
         if (l.H < 1 || l.W < 1 || static_cast<int64_t>(P_r) * P_c > B) return MBD_E_GRID;
+      } else if (l.split == MBD_SPLIT_MODEL) {
+        // L_M (Eq. 8): the P_r groups split the output channels.  A group's block must be whole 64-channel k-blocks of
+        // the backward-data product, whose K range is cut over these blocks; stride 1 only
+        if (l.H < 1 || l.W < 1) return MBD_E_GRID;
+        if (P_r > l.C_out) return MBD_E_GRID;
+        if (l.stride > 1 || (P_r > 1 && l.C_out % (64 * P_r) != 0)) return MBD_E_UNSUPPORTED;
       } else if (l.H < 1 || l.W < 1 || P_r > l.H || (P_r > 1 && l.H / P_r < l.kh / 2)) {
         return MBD_E_GRID;   // a strip needs >= 1 row, and its halo rows come from the adjacent strip only
       }
@@ -369,8 +375,10 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   if (Lc > 0) {
     // batch-split convolutions (Section 3's improved case) run on 1 x P: no strips, whatever P_r is
     const bool batch_split = layers[0].split == MBD_SPLIT_BATCH;
-    st = conv_create(layers, Lc, B, batch_split ? 1 : P_r, batch_split ? P_r * P_c : P_c, n->max_partials, n->num_sms, n->status, n->stream, &n->prof,
-                     mixed || loss == MBD_LOSS_NONE, &n->conv);
+    // model-split convolutions (L_M): no strips either; the P_r groups split the output channels, the P_c groups the batch
+    const bool model_split = layers[0].split == MBD_SPLIT_MODEL;
+    st = conv_create(layers, Lc, B, batch_split || model_split ? 1 : P_r, batch_split ? P_r * P_c : P_c, n->max_partials, n->num_sms, n->status, n->stream, &n->prof,
+                     mixed || loss == MBD_LOSS_NONE, model_split ? P_r : 1, &n->conv);
     if (st != MBD_OK) { free_net(n); return st; }
     if (is_conv) {
       *out = n;

@@ -169,7 +169,8 @@ def fc_layers(dims: Sequence[int], bias: bool = True, relu: bool = True) -> List
 def conv_layers(n: int, C_: int, H: int, W: int, relu: bool = True, k=3, split: int = SPLIT_DOMAIN, channels=(),
                 strides=()) -> List[Layer]:
     """n convolution layers on H x W input images, domain-split (row strips) or, with split=SPLIT_BATCH,
-    batch-parallel on 1 x P (Section 3's improved case); `k` is the kernel size, k or (k_h, k_w), one value for all
+    batch-parallel on 1 x P (Section 3's improved case) or, with split=SPLIT_MODEL, model-parallel like a fully
+    connected layer (output channels over P_r, batch over P_c: Eq. 8); `k` is the kernel size, k or (k_h, k_w), one value for all
     layers or one per layer; `channels` = (C_0, .., C_n) when the layers change the channel count (else C -> C);
     `strides` = one stride per layer (default 1): layer i then maps H_i x W_i images to H_i/s x W_i/s ones."""
     ks = [k] * n if isinstance(k, (int, tuple)) else list(k)

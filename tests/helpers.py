@@ -214,12 +214,12 @@ def like_device(ref, got):
     ref = np.asarray(ref)
     return ref[:, :, 1:2, 1:2] if (ref.ndim == 4 and got.shape[-1] == 1 and ref.shape[-1] == 3) else ref
 
-def oracle_conv_step(w, inp, strips=None, grid=None, eta=None):
+def oracle_conv_step(w, inp, strips=None, grid=None, eta=None, split="domain"):
     """fp64 oracle step for a domain-parallel conv workload (NCHW); stored activations are
     rounded to bf16 like the device's.  `strips` = P_r (or `grid` = (P_r, P_c)) runs the
     strip / halo formulation."""
     from oracle import mbd_oracle as O
-    layers = [O.Conv3x3(oracle_kernel(k), relu=True, stride=w.stride(i)) for i, k in enumerate(inp.Ws)]
+    layers = [O.Conv3x3(oracle_kernel(k), relu=True, stride=w.stride(i), split=split) for i, k in enumerate(inp.Ws)]
     X = inp.X.astype(np.float64)
     eta = w.eta if eta is None else eta
     if strips is None and grid is None:
@@ -228,13 +228,14 @@ def oracle_conv_step(w, inp, strips=None, grid=None, eta=None):
     return O.train_step_blocked(layers, X, None, "half_ssq", eta, P_r, P_c, store=bf16_store)
 
 
-def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1, eta=None, max_partials=0):
+def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1, eta=None, max_partials=0, split=None, plans=None):
     import torch
     from paper_1712_04432_b200 import mbd
     C_, H, Wd = w.dims
     L = w.n_layers
     eta = w.eta if eta is None else eta
-    net = mbd.Net(mbd.conv_layers(L, C_, H, Wd, k=[w.kshape(i) for i in range(L)], channels=w.channels, strides=w.strides), w.B, P_r, P_c, mbd.BF16,
+    kw = {} if split is None else dict(split=split)
+    net = mbd.Net(mbd.conv_layers(L, C_, H, Wd, k=[w.kshape(i) for i in range(L)], channels=w.channels, strides=w.strides, **kw), w.B, P_r, P_c, mbd.BF16,
                   mbd.LOSS_HALF_SSQ, max_partials)
     for i in range(L):
         net.set_weights(i, to_dev(inp.Ws[i], True))
@@ -257,6 +258,9 @@ def gpu_conv_step(w, inp, P_r=1, fused=False, force_acts=None, P_c=1, eta=None, 
     out["dY"] = [to_np(net.get_tensor(mbd.T_DY, i)) for i in range(L)]
     out["new_W"] = [to_np(net.get_weights(i)) for i in range(L)]
     out["launches"] = net.launch_count
+    if plans is not None:                      # (layer, product) -> mbd_get_plan, for the caller's assertions
+        for key in list(plans):
+            plans[key] = net.plan(*key)
     net.close()
     return out
 
@@ -312,7 +316,7 @@ def oracle_mixed_step(w, inp, blocked_grid=None, eta=None, conv_split="domain"):
 def mixed_layers(w, conv_split=None):
     from paper_1712_04432_b200 import mbd
     C_, H, Wd = w.dims
-    split = mbd.SPLIT_DOMAIN if conv_split in (None, "domain") else mbd.SPLIT_BATCH
+    split = {None: mbd.SPLIT_DOMAIN, "domain": mbd.SPLIT_DOMAIN, "batch": mbd.SPLIT_BATCH, "model": mbd.SPLIT_MODEL}[conv_split]
     return mbd.conv_layers(w.n_layers, C_, H, Wd, k=[w.kshape(i) for i in range(w.n_layers)], split=split, channels=w.channels,
                            strides=w.strides) + mbd.fc_layers(w.fc_dims, bias=True)
 

@@ -281,3 +281,64 @@ def test_unsupported_shapes_are_refused():
     with pytest.raises(mbd.MbdError) as e:
         mbd.Net(mbd.conv_layers(1, 8, 13, 12, k=5), 2, 2, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
     assert e.value.status == mbd.E_UNSUPPORTED
+
+
+MODEL_CASES = {
+    # convolutions in L_M: channels C_0..C_L (every C_out a multiple of 64 P_r), kernel shapes, H, W, B
+    "five_by_five_then_three_on_wide_layers": ((16, 128, 256), ((5, 5), (3, 3)), 12, 16, 4),
+    "three_by_three_then_one_by_one": ((64, 256, 256), ((3, 3), (1, 1)), 10, 12, 6),
+}
+
+
+@pytest.mark.parametrize("name", sorted(MODEL_CASES))
+@pytest.mark.parametrize("grid,mp", [((2, 1), 2), ((2, 2), 2), ((1, 2), 2), ((2, 2), 1), ((4, 2), 2), ((4, 1), 4)])
+@pytest.mark.parametrize("fused", [False, True])
+def test_model_parallel_convolutions(name, grid, mp, fused):
+    # Eq. 8 for convolution layers: the P_r groups split the output channels, the P_c groups the batch; dX is the sum
+    # over the groups' partial results (a cut of the backward-data product's K range over blocks of output channels),
+    # dK a sum over the batch blocks.  Against the oracle's blocked step of the same grid.
+    from paper_1712_04432_b200 import mbd
+    ch, ks, H, W, B = MODEL_CASES[name]
+    P_r, P_c = grid
+    w = I.conv_workload(ch[0], H, W, B, n_layers=len(ks), name=name, ksizes=ks, channels=ch)
+    inp = I.make_inputs(w, seed=81)
+    if any(c % (64 * P_r) for c in ch[1:]):
+        with pytest.raises(mbd.MbdError) as e:
+            gpu_conv_step(w, inp, P_r, P_c=P_c, max_partials=mp, split=mbd.SPLIT_MODEL)
+        assert e.value.status == mbd.E_UNSUPPORTED          # a group's channels must be whole 64-channel blocks
+        return
+    o = oracle_conv_step(w, inp, grid=grid, split="model")
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    o = oracle_conv_step(w, inp, grid=grid, split="model", eta=eta)
+    plans = {(1, 1): None, (1, 2): None}
+    g = gpu_conv_step(w, inp, P_r, fused=fused, force_acts=stored_hidden(o), P_c=P_c, eta=eta, max_partials=mp, split=mbd.SPLIT_MODEL,
+                      plans=plans)
+    compare_conv_step(g, o, TOL, fused, init=inp, require_sized=True)
+    assert plans[(1, 1)]["k_pieces"] == min(P_r, mp), plans              # dX: one partial sum per group (or per max_partials)
+    assert plans[(1, 2)]["k_pieces"] % min(P_c, mp) == 0, plans          # dK: batch blocks first, then the planner's own cuts
+
+
+def test_model_parallel_convolutions_equal_the_unsplit_layers_up_to_the_order_of_sums():
+    from paper_1712_04432_b200 import mbd
+    ch, ks, H, W, B = MODEL_CASES["five_by_five_then_three_on_wide_layers"]
+    w = I.conv_workload(ch[0], H, W, B, n_layers=len(ks), name="model_vs_unsplit", ksizes=ks, channels=ch)
+    inp = I.make_inputs(w, seed=82)
+    a = gpu_conv_step(w, inp, 1, P_c=1)
+    b = gpu_conv_step(w, inp, 2, P_c=2, max_partials=2, split=mbd.SPLIT_MODEL)
+    for i in range(w.n_layers):
+        assert np.array_equal(a["act"][i], b["act"][i]), i                 # forward: no sum is cut
+        # (dY below the top is stored in bf16 after sums taken in another order: a few roundings differ)
+        assert rel_fro(b["dW"][i], a["dW"][i]) < 1e-3 and rel_fro(b["dY"][i], a["dY"][i]) < 1e-2, i
+
+
+@pytest.mark.parametrize("grid,mp,fused", [((2, 2), 2, True), ((2, 3), 1, False), ((1, 1), 1, True)])
+def test_integrated_stack_with_model_parallel_convolutions(grid, mp, fused):
+    # every layer in L_M: convolutions and fully connected layers alike split their outputs over P_r and the batch over
+    # P_c (Eq. 8 for the whole network); 5 x 5 and 3 x 3 on 16 -> 128 -> 128 channels, then FC 12288 -> 64 -> 16
+    w = I.mixed_workload(16, 8, 12, 2, (64, 16), 6, name="mixed_model_split", ksizes=((5, 5), (3, 3)), channels=(16, 128, 128))
+    inp = I.make_inputs(w, seed=83)
+    o = oracle_mixed_step(w, inp, blocked_grid=grid, conv_split="model")
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    o = oracle_mixed_step(w, inp, blocked_grid=grid, conv_split="model", eta=eta)
+    g = gpu_mixed_step(w, inp, grid, mp, fused=fused, force_acts=oracle_mixed_acts(o, w), eta=eta, conv_split="model")
+    compare_mixed_step(g, o, w, TOL, fused=fused, init=inp, require_sized=True)
