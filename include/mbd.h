@@ -154,8 +154,11 @@ enum {
  * a fully connected layer: the P_r groups split the output channels, the P_c groups the batch, no strips; dX is the
  * sum over the groups' partial results (min(P_r, max_partials) partial sums, added in ascending group order), dK a
  * sum over the batch blocks.  Stride 1, and C_out a multiple of 64 P_r (a group's channels are whole 64-channel
- * blocks of the backward-data product's K range): MBD_E_UNSUPPORTED otherwise.  All convolutions of a network are
- * split alike.
+ * blocks of the backward-data product's K range): MBD_E_UNSUPPORTED otherwise.
+ * The convolutions of one network may be split in different ways, each layer in L_M or L_D on its own (Section 2.4):
+ * between two runs of layers with different kinds the activation and, backward, its gradient change their
+ * distribution (the re-distribution of Eq. 6; here a pass through the NCHW form).  Such a network runs on the
+ * contraction kernel whatever its shapes; strips of unequal height and the row-range calls are then unsupported.
  * Convolutions (kind MBD_CONV3X3 whatever the kernel size; Section 2.2): zero padding floor(k/2), k_h and
  * k_w odd and at most 11, stride 1 to 4 (the same in both directions), C_in and C_out multiples of 8, C_in of a layer =
  * C_out of the layer below, H x W of a layer = the output size of the layer below (H/s x W/s of its input);

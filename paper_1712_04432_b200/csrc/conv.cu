@@ -1055,6 +1055,11 @@ struct ConvNet {
   std::vector<bf16*> K, Wf, Wb;
   std::vector<float*> dK;
   GenConv* gen = nullptr;            // layers these kernels do not cover: every call is forwarded (conv_general.cu)
+  // Convolutions split in different ways within one stack (each layer in L_M or L_D on its own, Section 2.4): one general
+  // stack per run of layers with the same split, chained through NCHW buffers -- the re-distribution between two
+  // distributions of an activation (Eq. 6) -- forward (activations) and backward (gradients)
+  struct Seg { GenConv* g; int first, n; bf16* out_nchw; };
+  std::vector<Seg> segs;
   std::vector<float*> K32;           // fp32 master weights (empty unless enabled)
   std::vector<float*> Vk;            // momentum: velocities of the kernels (empty unless enabled), canonical [o][c][3][3]
   float mu = 0.f;
@@ -1107,12 +1112,61 @@ void launch_stage_in(ConvNet* c, const bf16* nchw, bf16* strips) {
 
 }  // namespace
 
-mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, int max_partials, int num_sms, int* status,
-                       cudaStream_t stream, Profiler* prof, bool fc_above, int model_P_r, ConvNet** out) {
+namespace {
+// how a split kind uses the P_r x P_c grid: strips, batch blocks, groups over the output channels
+void kind_grid(int split, int P_r, int P_c, int* strips, int* blocks, int* model_groups) {
+  if (split == MBD_SPLIT_BATCH) { *strips = 1; *blocks = P_r * P_c; *model_groups = 1; }        // Section 3's improved case: 1 x P
+  else if (split == MBD_SPLIT_MODEL) { *strips = 1; *blocks = P_c; *model_groups = P_r; }       // L_M: Eq. 8
+  else { *strips = P_r; *blocks = P_c; *model_groups = 1; }                                     // L_D: Eq. 7
+}
+// the general stack that holds `layer` (rewritten to its index there); null for the 64-channel kernels
+GenConv* gen_of(const ConvNet* c, int* layer, int* seg = nullptr) {
+  if (c->gen) return c->gen;
+  for (size_t k = 0; k < c->segs.size(); ++k)
+    if (*layer >= c->segs[k].first && *layer < c->segs[k].first + c->segs[k].n) {
+      *layer -= c->segs[k].first;
+      if (seg) *seg = static_cast<int>(k);
+      return c->segs[k].g;
+    }
+  return c->segs.empty() ? nullptr : c->segs.back().g;         // (out of range: the callee reports it)
+}
+}  // namespace
+
+mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r_grid, int P_c_grid, int max_partials, int num_sms, int* status,
+                       cudaStream_t stream, Profiler* prof, bool fc_above, ConvNet** out) {
+  bool uniform = true;
+  for (int i = 1; i < L; ++i) uniform = uniform && layers[i].split == layers[0].split;
+  if (!uniform) {
+    ConvNet* c = new (std::nothrow) ConvNet();
+    if (!c) return MBD_E_ALLOC;
+    c->L = L; c->B = B; c->stream = stream;
+    for (int a = 0; a < L;) {
+      int b = a + 1;
+      while (b < L && layers[b].split == layers[a].split) ++b;
+      int strips, blocks, groups;
+      kind_grid(layers[a].split, P_r_grid, P_c_grid, &strips, &blocks, &groups);
+      ConvNet::Seg sg{nullptr, a, b - a, nullptr};
+      const mbd_status s = gconv_create(layers + a, b - a, B, strips, blocks, max_partials, num_sms, status, stream, prof, b < L ? true : fc_above,
+                                        groups, a > 0, a > 0 ? layers[a - 1].relu : 0, &sg.g);
+      if (s != MBD_OK) { conv_destroy(c); return s; }
+      c->segs.push_back(sg);
+      a = b;
+    }
+    for (size_t k = 0; k + 1 < c->segs.size(); ++k)
+      if (cudaMalloc(reinterpret_cast<void**>(&c->segs[k].out_nchw), gconv_input_bytes(c->segs[k + 1].g)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        conv_destroy(c);
+        return MBD_E_ALLOC;
+      }
+    *out = c;
+    return MBD_OK;
+  }
+  int P_r, P_c, model_P_r;
+  kind_grid(layers[0].split, P_r_grid, P_c_grid, &P_r, &P_c, &model_P_r);
   if (gconv_needed(layers, L)) {
     ConvNet* c = new (std::nothrow) ConvNet();
     if (!c) return MBD_E_ALLOC;
-    const mbd_status s = gconv_create(layers, L, B, P_r, P_c, max_partials, num_sms, status, stream, prof, fc_above, model_P_r, &c->gen);
+    const mbd_status s = gconv_create(layers, L, B, P_r, P_c, max_partials, num_sms, status, stream, prof, fc_above, model_P_r, false, 0, &c->gen);
     if (s != MBD_OK) { delete c; return s; }
     c->L = L; c->B = B;
     *out = c;
@@ -1174,6 +1228,12 @@ mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P
 
 void conv_destroy(ConvNet* c) {
   if (c && c->gen) { gconv_destroy(c->gen); delete c; return; }
+  if (c && !c->segs.empty()) {
+    for (ConvNet::Seg& sg : c->segs) { gconv_destroy(sg.g); cudaFree(sg.out_nchw); }
+    (void)cudaGetLastError();
+    delete c;
+    return;
+  }
   if (!c) return;
   for (size_t i = 0; i < c->act.size(); ++i) cudaFree(c->act[i]);
   for (int i = 0; i < c->L; ++i)
@@ -1196,7 +1256,7 @@ mbd_status launch_pack(ConvNet* c, int layer) {
 }  // namespace
 
 mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev) {
-  if (c->gen) return gconv_set_weights(c->gen, layer, K_dev);
+  if (GenConv* g = gen_of(c, &layer)) return gconv_set_weights(g, layer, K_dev);
   if (c->k1[layer]) {
     embed_1x1_kernel<<<(9 * C * C + 255) / 256, 256, 0, c->stream>>>(static_cast<const bf16*>(K_dev), c->K[layer]);
     if (cudaGetLastError() != cudaSuccess) return MBD_E_CUDA;
@@ -1209,6 +1269,10 @@ mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev) {
 
 mbd_status conv_enable_master(ConvNet* c) {
   if (c->gen) return gconv_enable_master(c->gen);
+  if (!c->segs.empty()) {
+    for (ConvNet::Seg& sg : c->segs) { const mbd_status st = gconv_enable_master(sg.g); if (st != MBD_OK) return st; }
+    return MBD_OK;
+  }
   if (!c->K32.empty()) return MBD_OK;
   std::vector<float*> m(c->L, nullptr);
   for (int i = 0; i < c->L; ++i) {
@@ -1225,6 +1289,10 @@ mbd_status conv_enable_master(ConvNet* c) {
 
 mbd_status conv_enable_momentum(ConvNet* c, float mu) {
   if (c->gen) return gconv_enable_momentum(c->gen, mu);
+  if (!c->segs.empty()) {
+    for (ConvNet::Seg& sg : c->segs) { const mbd_status st = gconv_enable_momentum(sg.g, mu); if (st != MBD_OK) return st; }
+    return MBD_OK;
+  }
   if (c->Vk.empty()) {
     std::vector<float*> v(c->L, nullptr);
     for (int i = 0; i < c->L; ++i) {
@@ -1255,7 +1323,7 @@ mbd_status momentum_update(ConvNet* c, int i, float eta) {
 }  // namespace
 
 mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev) {
-  if (c->gen) return gconv_get_weights(c->gen, layer, K_dev);
+  if (GenConv* g = gen_of(c, &layer)) return gconv_get_weights(g, layer, K_dev);
   if (c->k1[layer]) {
     extract_1x1_kernel<bf16><<<(C * C + 255) / 256, 256, 0, c->stream>>>(c->K[layer], static_cast<bf16*>(K_dev));
     return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
@@ -1264,12 +1332,16 @@ mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev) {
   return MBD_OK;
 }
 
-size_t conv_input_bytes(const ConvNet* c) { return c->gen ? gconv_input_bytes(c->gen) : static_cast<size_t>(c->B) * C * c->H * c->W * 2; }
+size_t conv_input_bytes(const ConvNet* c) {
+  if (!c->segs.empty()) return gconv_input_bytes(c->segs[0].g);
+  return c->gen ? gconv_input_bytes(c->gen) : static_cast<size_t>(c->B) * C * c->H * c->W * 2;
+}
 
 // The step, piece by piece (a multi-process driver exchanges the image's outer halo rows between the pieces;
 // conv_forward / conv_backward below are these pieces in a row).
 mbd_status conv_stage_input(ConvNet* c, const void* X_nchw) {
   if (c->gen) return gconv_stage_input(c->gen, X_nchw);
+  if (!c->segs.empty()) return gconv_stage_input(c->segs[0].g, X_nchw);
   // the input goes into strips (with the halo rows between its own strips); the operand layouts of the weights
   // are kept current by whatever changes the weights (conv_set_weights, the fused update, conv_sgd_step)
   launch_stage_in(c, static_cast<const bf16*>(X_nchw), c->act[0]);
@@ -1300,6 +1372,18 @@ void for_rows(const ConvNet* c, int layer, int rows, F launch) {
 
 mbd_status conv_forward_layer(ConvNet* c, int i, float* loss_sum_dev, int rows) {
   if (c->gen) return rows == MBD_ROWS_ALL ? gconv_forward_layer(c->gen, i, loss_sum_dev) : MBD_E_UNSUPPORTED;
+  if (!c->segs.empty()) {
+    if (rows != MBD_ROWS_ALL) return MBD_E_UNSUPPORTED;
+    if (i < 0 || i >= c->L) return MBD_E_INVALID;
+    int k = 0, j = i;
+    GenConv* g = gen_of(c, &j, &k);
+    if (j == 0 && k > 0) {       // the output of the run below, re-distributed: out of its layout into NCHW, from there into this run's
+      mbd_status st = gconv_output_to_nchw(c->segs[k - 1].g, c->segs[k - 1].out_nchw);
+      if (st == MBD_OK) st = gconv_stage_input(g, c->segs[k - 1].out_nchw);
+      if (st != MBD_OK) return st;
+    }
+    return gconv_forward_layer(g, j, loss_sum_dev);
+  }
   if (i < 0 || i >= c->L) return MBD_E_INVALID;
   if (rows != MBD_ROWS_ALL && (c->P_r != 1 || (rows != MBD_ROWS_INTERIOR && rows != MBD_ROWS_BOUNDARY))) return MBD_E_UNSUPPORTED;
   const bool last = i == c->L - 1;
@@ -1322,7 +1406,7 @@ mbd_status conv_forward_layer(ConvNet* c, int i, float* loss_sum_dev, int rows) 
 }
 
 mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
-  if (c->gen) return gconv_forward(c->gen, X_nchw, loss_sum_dev);
+  if (c->gen) return gconv_forward(c->gen, X_nchw, loss_sum_dev);      // (a stack of several runs goes layer by layer, below)
   mbd_status s = conv_stage_input(c, X_nchw);
   for (int i = 0; i < c->L && s == MBD_OK; ++i) s = conv_forward_layer(c, i, loss_sum_dev, MBD_ROWS_ALL);
   return s;
@@ -1330,6 +1414,18 @@ mbd_status conv_forward(ConvNet* c, const void* X_nchw, float* loss_sum_dev) {
 
 mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta, int rows) {
   if (c->gen) return rows == MBD_ROWS_ALL ? gconv_backward_layer(c->gen, i, fused_eta) : MBD_E_UNSUPPORTED;
+  if (!c->segs.empty()) {
+    if (rows != MBD_ROWS_ALL) return MBD_E_UNSUPPORTED;
+    if (i < 0 || i >= c->L) return MBD_E_INVALID;
+    int k = 0, j = i;
+    GenConv* g = gen_of(c, &j, &k);
+    mbd_status st = gconv_backward_layer(g, j, fused_eta);
+    if (st == MBD_OK && j == 0 && k > 0) {       // the gradient w.r.t. this run's input goes back to the run below the same way
+      st = gconv_input_grad_to_nchw(g, c->segs[k - 1].out_nchw);
+      if (st == MBD_OK) st = gconv_top_grad_from_nchw(c->segs[k - 1].g, c->segs[k - 1].out_nchw);
+    }
+    return st;
+  }
   if (i < 0 || i >= c->L) return MBD_E_INVALID;
   if (rows != MBD_ROWS_ALL && (c->P_r != 1 || (rows != MBD_ROWS_INTERIOR && rows != MBD_ROWS_BOUNDARY))) return MBD_E_UNSUPPORTED;
   const bool momentum = !c->Vk.empty();
@@ -1367,7 +1463,7 @@ mbd_status conv_backward_layer(ConvNet* c, int i, float fused_eta, int rows) {
 }
 
 mbd_status conv_backward(ConvNet* c, float fused_eta) {
-  if (c->gen) return gconv_backward(c->gen, fused_eta);
+  if (c->gen) return gconv_backward(c->gen, fused_eta);      // (a stack of several runs goes layer by layer, below)
   mbd_status s = MBD_OK;
   for (int i = c->L - 1; i >= 0 && s == MBD_OK; --i) s = conv_backward_layer(c, i, fused_eta, MBD_ROWS_ALL);
   return s;
@@ -1377,7 +1473,7 @@ mbd_status conv_backward(ConvNet* c, float fused_eta) {
 // read out, or its upper / lower halo row (zero unless a neighbour supplies it) is written.  `side` 0 = top,
 // 1 = bottom; the row buffer is [B][W][C] bf16.  which / layer as in conv_get_tensor; layer -1 = the staged input.
 mbd_status conv_outer_rows(ConvNet* c, int which, int layer, int side, void* rows, size_t bytes, int set) {
-  if (c->gen) return MBD_E_UNSUPPORTED;
+  if (c->gen || !c->segs.empty()) return MBD_E_UNSUPPORTED;
   if (layer < -1 || layer >= c->L || (side != 0 && side != 1)) return MBD_E_INVALID;
   if (bytes != static_cast<size_t>(c->B) * c->W * C * 2) return MBD_E_INVALID;
   bf16* buf = which == MBD_T_ACT ? c->act[layer + 1] : (which == MBD_T_DY && layer >= 0) ? c->dY[layer] : nullptr;
@@ -1392,11 +1488,12 @@ mbd_status conv_outer_rows(ConvNet* c, int which, int layer, int side, void* row
 }
 
 mbd_status conv_get_product(const ConvNet* c, int layer, int product, const TcGemm** out) {
-  return c->gen ? gconv_get_product(c->gen, layer, product, out) : MBD_E_UNSUPPORTED;
+  if (const GenConv* g = gen_of(c, &layer)) return gconv_get_product(g, layer, product, out);
+  return MBD_E_UNSUPPORTED;
 }
 
 mbd_status conv_set_dw(ConvNet* c, int layer, const void* src, size_t bytes) {
-  if (c->gen) return gconv_set_dw(c->gen, layer, src, bytes);
+  if (GenConv* g = gen_of(c, &layer)) return gconv_set_dw(g, layer, src, bytes);
   if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
   if (c->k1[layer]) {
     if (bytes != C * C * 4) return MBD_E_INVALID;
@@ -1409,6 +1506,10 @@ mbd_status conv_set_dw(ConvNet* c, int layer, const void* src, size_t bytes) {
 
 mbd_status conv_sgd_step(ConvNet* c, float eta) {
   if (c->gen) return gconv_sgd_step(c->gen, eta);
+  if (!c->segs.empty()) {
+    for (ConvNet::Seg& sg : c->segs) { const mbd_status st = gconv_sgd_step(sg.g, eta); if (st != MBD_OK) return st; }
+    return MBD_OK;
+  }
   const float scale = -eta / static_cast<float>(c->B);
   for (int i = 0; i < c->L; ++i) {
     if (!c->Vk.empty()) {
@@ -1430,6 +1531,7 @@ mbd_status conv_sgd_step(ConvNet* c, float eta) {
 // and that layer's input gradient goes back into strips, its boundary rows also into the neighbours' halos.
 mbd_status conv_output_to_nchw(ConvNet* c, void* dst) {
   if (c->gen) return gconv_output_to_nchw(c->gen, dst);
+  if (!c->segs.empty()) return gconv_output_to_nchw(c->segs.back().g, dst);
   dim3 g((c->H * c->W + 31) / 32, static_cast<unsigned>(c->B));
   c->prof->begin(MBD_K_HALO, 2.0 * c->B * C * c->H * c->W * 2.0);
   strips_to_nchw_kernel<<<g, 128, 0, c->stream>>>(c->act[c->L], static_cast<bf16*>(dst), c->H, c->W, c->P_r, c->Hs);
@@ -1439,15 +1541,19 @@ mbd_status conv_output_to_nchw(ConvNet* c, void* dst) {
 
 mbd_status conv_top_grad_from_nchw(ConvNet* c, const void* src) {
   if (c->gen) return gconv_top_grad_from_nchw(c->gen, src);
+  if (!c->segs.empty()) return gconv_top_grad_from_nchw(c->segs.back().g, src);
   if (!c->fc_above) return MBD_E_STATE;
   launch_stage_in(c, static_cast<const bf16*>(src), c->dY[c->L - 1]);
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 
-int conv_last_relu(const ConvNet* c) { return c->gen ? gconv_last_relu(c->gen) : c->relu[c->L - 1]; }
+int conv_last_relu(const ConvNet* c) {
+  if (!c->segs.empty()) return gconv_last_relu(c->segs.back().g);
+  return c->gen ? gconv_last_relu(c->gen) : c->relu[c->L - 1];
+}
 
 mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t bytes) {
-  if (c->gen) return gconv_get_tensor(c->gen, which, layer, dst, bytes);
+  if (GenConv* g = gen_of(c, &layer)) return gconv_get_tensor(g, which, layer, dst, bytes);
   const size_t nchw_bytes = conv_input_bytes(c);
   if (which == MBD_T_DW || which == MBD_T_MASTER || which == MBD_T_VELOCITY) {
     if (layer < 0 || layer >= c->L) return MBD_E_INVALID;
@@ -1477,7 +1583,16 @@ mbd_status conv_get_tensor(ConvNet* c, int which, int layer, void* dst, size_t b
 }
 
 mbd_status conv_set_tensor(ConvNet* c, int which, int layer, const void* src, size_t bytes) {
-  if (c->gen) return gconv_set_tensor(c->gen, which, layer, src, bytes);
+  {
+    int k = -1, local = layer;
+    if (GenConv* g = gen_of(c, &local, &k)) {
+      const mbd_status st = gconv_set_tensor(g, which, local, src, bytes);
+      // the last activation of a run of layers is also the staged input of the next run: it follows what was set
+      if (st == MBD_OK && which == MBD_T_ACT && k >= 0 && k + 1 < static_cast<int>(c->segs.size()) && local == c->segs[k].n - 1)
+        return gconv_stage_input(c->segs[k + 1].g, src);
+      return st;
+    }
+  }
   if (layer < 0 || layer >= c->L || bytes != conv_input_bytes(c)) return MBD_E_INVALID;
   bf16* dst = which == MBD_T_ACT ? c->act[layer + 1] : which == MBD_T_DY ? c->dY[layer] : nullptr;
   if (!dst) return MBD_E_INVALID;

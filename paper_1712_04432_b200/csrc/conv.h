@@ -10,7 +10,7 @@
 namespace mbd {
 struct ConvNet;
 mbd_status conv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, int max_partials, int num_sms, int* status,
-                       cudaStream_t stream, Profiler* prof, bool fc_above, int model_P_r, ConvNet** out);
+                       cudaStream_t stream, Profiler* prof, bool fc_above, ConvNet** out);
 void conv_destroy(ConvNet* c);
 mbd_status conv_set_weights(ConvNet* c, int layer, const void* K_dev);
 mbd_status conv_get_weights(ConvNet* c, int layer, void* K_dev);

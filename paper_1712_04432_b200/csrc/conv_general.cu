@@ -299,6 +299,9 @@ struct GenConv {
   int64_t B = 0;
   int P_r = 1, P = 1, S = 1;              // strips; processes of the grid; fp32 partial sums per weight gradient asked for
   int model_P_r = 1, S_dx = 1;            // model-parallel layers: groups that split the output channels; partial sums per dX asked for
+  bool need_dx0 = false;                  // this stack continues another one: the gradient w.r.t. its input is formed too (dX0)
+  int in_relu = 0;                        // ... and its input is the ReLU output of the layer below (mask of that gradient)
+  bf16* dX0 = nullptr;
   std::vector<Geo> geo;                   // geometry of tensor i (act[i]; dY[i] has that of act[i + 1])
   std::vector<int> Cin, Cout, kh, kw, relu, taps, Cp, stride;
   std::vector<int> ldw;                   // columns of the internal weight matrix of layer i
@@ -441,12 +444,12 @@ void gconv_destroy(GenConv* c) {
   for (float* p : c->dWm) cudaFree(p);
   for (float* p : c->Wm32) cudaFree(p);
   for (float* p : c->Vm) cudaFree(p);
-  cudaFree(c->partials); cudaFree(c->loss_part);
+  cudaFree(c->partials); cudaFree(c->loss_part); cudaFree(c->dX0);
   delete c;
 }
 
 mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, int max_partials, int num_sms, int* status,
-                        cudaStream_t stream, Profiler* prof, bool fc_above, int model_P_r, GenConv** out) {
+                        cudaStream_t stream, Profiler* prof, bool fc_above, int model_P_r, bool need_dx0, int in_relu, GenConv** out) {
   if (tc_gemm_init() != cudaSuccess) { (void)cudaGetLastError(); return MBD_E_CUDA; }
   // one padding for every tensor: what the widest reach of any layer needs at the resolution it works in
   int ph = 0, pw = 0, H = layers[0].H, W = layers[0].W;
@@ -480,6 +483,7 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
   // Model-parallel layers (Eq. 8): no strips (P_r = 1 here), the weight gradient's rows are independent, so its partial
   // sums are over the P_c batch blocks (c->S above), and dX = sum over the model_P_r groups of W_r^T dY_r is a cut of
   // backward-data's K range over blocks of output channels
+  c->need_dx0 = need_dx0; c->in_relu = in_relu;
   c->model_P_r = model_P_r < 1 ? 1 : model_P_r;
   c->S_dx = max_partials < 1 ? 1 : std::min(c->model_P_r, max_partials);
   auto alloc = [&](void** p, size_t bytes) -> bool {
@@ -501,16 +505,17 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
   // (256 bytes of slack behind the tensors a folded layer reads: its last rows reach up to 64 - C_in elements further)
   for (int i = 0; i <= L && ok; ++i) {
     const int C = i == 0 ? c->Cin[0] : c->Cout[i - 1];
-    if (i == 0 && c->stride[0] > 1) continue;          // the input of a strided first layer lives in its phase planes only
+    if (i == 0 && c->stride[0] > 1 && !need_dx0) continue;          // the input of a strided first layer lives in its phase planes only
     ok = alloc(reinterpret_cast<void**>(&c->act[i]), static_cast<size_t>(c->geo[i].Ptot) * C * 2 + 256);
   }
+  if (need_dx0) ok = ok && alloc(reinterpret_cast<void**>(&c->dX0), static_cast<size_t>(c->geo[0].Ptot) * c->Cin[0] * 2);
   // internal weight layouts
   c->ldw.assign(L, 0); c->colmap.assign(L, nullptr); c->folded.assign(L, 0);
   std::vector<std::vector<Run>> runs(L);
   for (int i = 0; i < L && ok; ++i) {
     const int Cin = c->Cin[i], taps = c->taps[i], Cp = c->Cp[i];
     std::vector<int> map;
-    const bool fold = i == 0 && (Cin == 8 || Cin == 16 || Cin == 32) && taps > 1 && !getenv("MBD_CONV_NO_FOLD");      // tuning knob
+    const bool fold = i == 0 && !need_dx0 && (Cin == 8 || Cin == 16 || Cin == 32) && taps > 1 && !getenv("MBD_CONV_NO_FOLD");      // tuning knob (a folded layer has no backward-data product)
     if (fold) {
       runs[i] = fold_runs(c->kh[i], c->kw[i], c->stride[i], Cin, c->geo[i + 1]);
       if (static_cast<int>(runs[i].size()) <= MAX_TAPS && static_cast<int>(runs[i].size()) * 64 < taps * Cp) {
@@ -541,7 +546,7 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
     if (c->stride[i] > 1) {
       const size_t pl = static_cast<size_t>(c->stride[i]) * c->stride[i] * go.Ptot * c->Cin[i] * 2;
       ok = ok && alloc(reinterpret_cast<void**>(&c->xph[i]), pl + 256);
-      if (i > 0) ok = ok && alloc(reinterpret_cast<void**>(&c->dxph[i]), pl);
+      if (i > 0 || need_dx0) ok = ok && alloc(reinterpret_cast<void**>(&c->dxph[i]), pl);
     }
   }
   c->loss_grid = num_sms * 4;
@@ -574,7 +579,7 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
     const Epi ef = make_epi_act(c->act[i + 1], Cout, 1, c->relu[i]);
     if (tc_gemm_prepare(f, xin, Cin, c->Wm[i], ldw, num_sms, &ef) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
     // backward-data: one product (stride 1), or one per phase plane with the taps that read that plane
-    if (i > 0) {
+    if (i > 0 || need_dx0) {
       c->bwd_data[i].resize(s * s);
       c->bwd_taps[i].assign(s * s, 0);
       for (int q = 0; q < s * s; ++q) {
@@ -592,8 +597,8 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
         if (n == 0) continue;                          // no tap reads this plane: its gradient is zero
         d.K = n * Cop;
         d.cv_a_inner = Cout; d.cv_b_inner = ldw; d.cv_b_rows = Cout;
-        bf16* outp = s > 1 ? c->dxph[i] + static_cast<size_t>(q) * M * Cin : c->dY[i - 1];
-        const bf16* maskp = !c->relu[i - 1] ? nullptr : (s > 1 ? c->xph[i] + static_cast<size_t>(q) * M * Cin : c->act[i]);
+        bf16* outp = s > 1 ? c->dxph[i] + static_cast<size_t>(q) * M * Cin : (i > 0 ? c->dY[i - 1] : c->dX0);
+        const bf16* maskp = !(i > 0 ? c->relu[i - 1] : c->in_relu) ? nullptr : (s > 1 ? c->xph[i] + static_cast<size_t>(q) * M * Cin : c->act[i]);
         const Epi ed = make_epi_mask(outp, Cin, maskp, Cin);
         if (tc_gemm_prepare(d, c->dY[i], Cout, c->Wm[i], ldw, num_sms, &ed) != cudaSuccess) { gconv_destroy(c); return MBD_E_CUDA; }
         if (d.k_splits > 1) part_elems = std::max(part_elems, static_cast<size_t>(d.k_splits) * M * Cin);
@@ -719,7 +724,7 @@ void unstage(GenConv* c, const bf16* src, bf16* nchw, const Geo& g, int C) {
 }  // namespace
 
 mbd_status gconv_stage_input(GenConv* c, const void* X_nchw) {
-  if (c->stride[0] > 1)      // a strided first layer: straight into its phase planes (the input has no other reader)
+  if (c->stride[0] > 1 && !c->need_dx0)      // a strided first layer: straight into its phase planes (the input has no other reader)
     stage(c, static_cast<const bf16*>(X_nchw), c->xph[0], c->geo[0], c->Cin[0], true, &c->geo[1], c->stride[0]);
   else
     stage(c, static_cast<const bf16*>(X_nchw), c->act[0], c->geo[0], c->Cin[0], true);     // the forward halo exchange of the input rides along
@@ -732,7 +737,7 @@ mbd_status gconv_forward_layer(GenConv* c, int i, float* loss_sum_dev) {
   const Geo& go = c->geo[i + 1];
   const int s = c->stride[i];
   const double flops = 2.0 * c->B * go.H * go.W * c->taps[i] * c->Cin[i] * c->Cout[i];     // the method's flops
-  if (s > 1 && i > 0) {       // (the network's input was staged as planes)
+  if (s > 1 && (i > 0 || c->need_dx0)) {       // (otherwise the network's input was staged as planes)
     // the input's own pixels sorted into the s^2 phase planes; their halo rows exchanged plane by plane
     decimate(c, c->act[i], c->xph[i], c->geo[i], go, c->Cin[i], s, true);
     pad_fix(c, c->xph[i], go, c->Cin[i], true, s * s);
@@ -768,23 +773,25 @@ mbd_status gconv_backward_layer(GenConv* c, int i, float fused_eta) {
   const int s = c->stride[i], Cin = c->Cin[i];
   const double flops = 2.0 * c->B * go.H * go.W * c->taps[i] * Cin * c->Cout[i];
   const int ldw = c->ldw[i];
-  if (i > 0) {
+  if (i > 0 || c->need_dx0) {
+    bf16* below = i > 0 ? c->dY[i - 1] : c->dX0;
+    const int relu_below = i > 0 ? c->relu[i - 1] : c->in_relu;
     // backward halo exchange (second halo term of Eq. 7), then dY_{i-1} = convT(K_i, dY_i) * [X_i > 0] -- with the
     // weights as they are BEFORE this step's update, so this product comes first
     if (c->P_r > 1) pad_fix(c, c->dY[i], go, c->Cout[i], true);
     for (int q = 0; q < s * s; ++q) {
-      bf16* outp = s > 1 ? c->dxph[i] + static_cast<size_t>(q) * go.Ptot * Cin : c->dY[i - 1];
+      bf16* outp = s > 1 ? c->dxph[i] + static_cast<size_t>(q) * go.Ptot * Cin : below;
       if (c->bwd_taps[i][q] == 0) {                // (a 1 x 1 kernel with stride 2: three of four planes)
         if (cudaMemsetAsync(outp, 0, static_cast<size_t>(go.Ptot) * Cin * 2, c->stream) != cudaSuccess) return MBD_E_CUDA;
         continue;
       }
-      const bf16* maskp = !c->relu[i - 1] ? nullptr : (s > 1 ? c->xph[i] + static_cast<size_t>(q) * go.Ptot * Cin : c->act[i]);
+      const bf16* maskp = !relu_below ? nullptr : (s > 1 ? c->xph[i] + static_cast<size_t>(q) * go.Ptot * Cin : c->act[i]);
       const Epi ed = make_epi_mask(outp, Cin, maskp, Cin);
       const mbd_status st = run(c, c->bwd_data[i][q], MBD_K_CONV_BWD_DATA, flops * c->bwd_taps[i][q] / c->taps[i], ed);
       if (st != MBD_OK) return st;
     }
-    if (s > 1) decimate(c, c->dY[i - 1], c->dxph[i], c->geo[i], go, Cin, s, false);      // the planes' own pixels back in place
-    pad_fix(c, c->dY[i - 1], c->geo[i], Cin, false);
+    if (s > 1) decimate(c, below, c->dxph[i], c->geo[i], go, Cin, s, false);      // the planes' own pixels back in place
+    pad_fix(c, below, c->geo[i], Cin, false);
     if (c->P_r > 1) pad_fix(c, c->dY[i], go, c->Cout[i], false);      // the halo copies must not enter the sum below
   }
   // dY_i is zero outside the strips' own pixels here: every pixel enters the weight gradient once (the sum over the
@@ -816,6 +823,13 @@ mbd_status gconv_output_to_nchw(GenConv* c, void* dst) {
 mbd_status gconv_top_grad_from_nchw(GenConv* c, const void* src) {
   if (!c->fc_above) return MBD_E_STATE;
   stage(c, static_cast<const bf16*>(src), c->dY[c->L - 1], c->geo[c->L], c->Cout[c->L - 1], false);
+  return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
+}
+
+// The gradient w.r.t. this stack's input (a stack that continues another one: need_dx0), back in NCHW
+mbd_status gconv_input_grad_to_nchw(GenConv* c, void* dst) {
+  if (!c->need_dx0) return MBD_E_STATE;
+  unstage(c, c->dX0, static_cast<bf16*>(dst), c->geo[0], c->Cin[0]);
   return cudaGetLastError() == cudaSuccess ? MBD_OK : MBD_E_CUDA;
 }
 

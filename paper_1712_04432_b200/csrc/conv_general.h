@@ -12,7 +12,7 @@ namespace mbd {
 struct GenConv;
 bool gconv_needed(const mbd_layer* layers, int L);
 mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int P_c, int max_partials, int num_sms, int* status,
-                        cudaStream_t stream, Profiler* prof, bool fc_above, int model_P_r, GenConv** out);
+                        cudaStream_t stream, Profiler* prof, bool fc_above, int model_P_r, bool need_dx0, int in_relu, GenConv** out);
 void gconv_destroy(GenConv* c);
 mbd_status gconv_set_weights(GenConv* c, int layer, const void* K_dev);     // K[C_out][C_in][k_h][k_w] bf16
 mbd_status gconv_get_weights(GenConv* c, int layer, void* K_dev);
@@ -29,6 +29,7 @@ mbd_status gconv_set_tensor(GenConv* c, int which, int layer, const void* src, s
 mbd_status gconv_set_dw(GenConv* c, int layer, const void* src, size_t bytes);
 mbd_status gconv_get_product(const GenConv* c, int layer, int product, const TcGemm** out);
 mbd_status gconv_output_to_nchw(GenConv* c, void* dst);
+mbd_status gconv_input_grad_to_nchw(GenConv* c, void* dst_nchw);
 mbd_status gconv_top_grad_from_nchw(GenConv* c, const void* src);
 size_t gconv_input_bytes(const GenConv* c);
 int gconv_last_relu(const GenConv* c);

@@ -314,7 +314,6 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
       if (l.C_in < 8 || l.C_out < 8 || l.C_in % 8 || l.C_out % 8) return MBD_E_UNSUPPORTED;
       if (i > 0 && l.C_in != layers[i - 1].C_out) return MBD_E_INVALID;
       if (l.split != MBD_SPLIT_DOMAIN && l.split != MBD_SPLIT_BATCH && l.split != MBD_SPLIT_MODEL) return MBD_E_INVALID;
-      if (l.split != layers[0].split) return MBD_E_UNSUPPORTED;          // all convolutions split alike
       if (l.split == MBD_SPLIT_BATCH) {                                  // 1 x P: one sample per process at least
         if (l.H < 1 || l.W < 1 || static_cast<int64_t>(P_r) * P_c > B) return MBD_E_GRID;
       } else if (l.split == MBD_SPLIT_MODEL) {
@@ -373,12 +372,9 @@ extern "C" mbd_status mbd_net_create(const mbd_layer* layers, int L, int64_t B, 
   if (cudaMemsetAsync(n->status, 0, sizeof(int), n->stream) != cudaSuccess) { free_net(n); return MBD_E_CUDA; }
 
   if (Lc > 0) {
-    // batch-split convolutions (Section 3's improved case) run on 1 x P: no strips, whatever P_r is
-    const bool batch_split = layers[0].split == MBD_SPLIT_BATCH;
-    // model-split convolutions (L_M): no strips either; the P_r groups split the output channels, the P_c groups the batch
-    const bool model_split = layers[0].split == MBD_SPLIT_MODEL;
-    st = conv_create(layers, Lc, B, batch_split || model_split ? 1 : P_r, batch_split ? P_r * P_c : P_c, n->max_partials, n->num_sms, n->status, n->stream, &n->prof,
-                     mixed || loss == MBD_LOSS_NONE, model_split ? P_r : 1, &n->conv);
+    // how each convolution uses the grid follows from its split kind (strips, batch blocks on 1 x P, groups over the
+    // output channels): conv_create works that out, layer by layer
+    st = conv_create(layers, Lc, B, P_r, P_c, n->max_partials, n->num_sms, n->status, n->stream, &n->prof, mixed || loss == MBD_LOSS_NONE, &n->conv);
     if (st != MBD_OK) { free_net(n); return st; }
     if (is_conv) {
       *out = n;

@@ -178,12 +178,13 @@ def conv_layers(n: int, C_: int, H: int, W: int, relu: bool = True, k=3, split: 
     ks = [(q, q) if isinstance(q, int) else (int(q[0]), int(q[1])) for q in ks]
     ch = list(channels) if channels else [C_] * (n + 1)
     st = list(strides) if strides else [1] * n
-    assert len(ch) == n + 1 and len(st) == n
+    sp = [split] * n if isinstance(split, int) else [int(q) for q in split]      # one split kind for all layers, or one per layer
+    assert len(ch) == n + 1 and len(st) == n and len(sp) == n
     out = []
     for i in range(n):
         assert H % st[i] == 0 and W % st[i] == 0
         Ho, Wo = H // st[i], W // st[i]
-        out.append(Layer(kind=CONV3X3, split=split, relu=int(relu), bias=0, d_in=ch[i] * H * W, d_out=ch[i + 1] * Ho * Wo,
+        out.append(Layer(kind=CONV3X3, split=sp[i], relu=int(relu), bias=0, d_in=ch[i] * H * W, d_out=ch[i + 1] * Ho * Wo,
                          C_in=ch[i], C_out=ch[i + 1], H=H, W=W, kh=ks[i][0], kw=ks[i][1], stride=st[i]))
         H, W = Ho, Wo
     return out

@@ -219,7 +219,8 @@ def oracle_conv_step(w, inp, strips=None, grid=None, eta=None, split="domain"):
     rounded to bf16 like the device's.  `strips` = P_r (or `grid` = (P_r, P_c)) runs the
     strip / halo formulation."""
     from oracle import mbd_oracle as O
-    layers = [O.Conv3x3(oracle_kernel(k), relu=True, stride=w.stride(i), split=split) for i, k in enumerate(inp.Ws)]
+    splits = [split] * len(inp.Ws) if isinstance(split, str) else list(split)
+    layers = [O.Conv3x3(oracle_kernel(k), relu=True, stride=w.stride(i), split=splits[i]) for i, k in enumerate(inp.Ws)]
     X = inp.X.astype(np.float64)
     eta = w.eta if eta is None else eta
     if strips is None and grid is None:

@@ -342,3 +342,63 @@ def test_integrated_stack_with_model_parallel_convolutions(grid, mp, fused):
     o = oracle_mixed_step(w, inp, blocked_grid=grid, conv_split="model", eta=eta)
     g = gpu_mixed_step(w, inp, grid, mp, fused=fused, force_acts=oracle_mixed_acts(o, w), eta=eta, conv_split="model")
     compare_mixed_step(g, o, w, TOL, fused=fused, init=inp, require_sized=True)
+
+
+SPLIT_OF = {"domain": 1, "batch": 2, "model": 0}          # mbd.SPLIT_DOMAIN, SPLIT_BATCH, SPLIT_MODEL
+
+
+@pytest.mark.parametrize("kinds", [("domain", "domain", "model"), ("domain", "model", "model"), ("model", "domain", "batch"),
+                                   ("batch", "model", "domain")])
+@pytest.mark.parametrize("grid,mp", [((2, 2), 2), ((2, 1), 1), ((1, 3), 3)])
+@pytest.mark.parametrize("fused", [False, True])
+def test_each_convolution_in_the_set_of_its_own(kinds, grid, mp, fused):
+    # Section 2.4: every layer is in L_M or L_D on its own.  Three convolutions (5 x 5, 3 x 3, 3 x 3 on 16 -> 128 -> 128 -> 128
+    # channels) whose split kinds differ: runs of equal kind are stacks of their own, and between two runs the activation
+    # (forward) and its gradient (backward) change their distribution.  Against the oracle's blocked step with the same
+    # kinds on the same grid.
+    assert SPLIT_OF == {"domain": 1, "batch": 2, "model": 0}
+    ch, ks, H, W, B = (16, 128, 128, 128), ((5, 5), (3, 3), (3, 3)), 12, 16, 6
+    w = I.conv_workload(ch[0], H, W, B, n_layers=3, name="mixed_kinds", ksizes=ks, channels=ch)
+    inp = I.make_inputs(w, seed=84)
+    o = oracle_conv_step(w, inp, grid=grid, split=kinds)
+    eta = update_sized_eta(o, inp.Ws, w.B)
+    o = oracle_conv_step(w, inp, grid=grid, split=kinds, eta=eta)
+    g = gpu_conv_step(w, inp, grid[0], fused=fused, force_acts=stored_hidden(o), P_c=grid[1], eta=eta, max_partials=mp,
+                      split=[SPLIT_OF[k] for k in kinds])
+    compare_conv_step(g, o, TOL, fused, init=inp, require_sized=True)
+
+
+def test_integrated_stack_with_convolutions_of_different_kinds():
+    # domain-split 5 x 5, model-split 3 x 3, then model-split fully connected layers on one 2 x 2 grid
+    from paper_1712_04432_b200 import mbd
+    import torch
+    from tests.helpers import to_dev, to_np
+    from oracle import mbd_oracle as O
+    from tests.helpers import bf16_store, oracle_kernel
+    w = I.mixed_workload(16, 8, 12, 2, (64, 16), 6, name="mixed_kinds_fc", ksizes=((5, 5), (3, 3)), channels=(16, 128, 128))
+    inp = I.make_inputs(w, seed=85)
+    kinds = ("domain", "model")
+    layers = [O.Conv3x3(oracle_kernel(inp.Ws[i]), relu=True, split=kinds[i]) for i in range(2)]
+    layers += [O.FC(inp.Ws[i].astype(np.float64), inp.bs[i].astype(np.float64), relu=True) for i in range(2, w.L)]
+    o = O.train_step_blocked(layers, inp.X.astype(np.float64), inp.labels, "softmax_ce", w.eta, 2, 2, store=bf16_store)
+    spec = mbd.conv_layers(2, 16, 8, 12, k=[(5, 5), (3, 3)], channels=(16, 128, 128), split=[mbd.SPLIT_DOMAIN, mbd.SPLIT_MODEL]) + \
+        mbd.fc_layers(w.fc_dims, bias=True)
+    net = mbd.Net(spec, w.B, 2, 2, mbd.BF16, mbd.LOSS_SOFTMAX_CE, 2)
+    for i in range(w.L):
+        if i < 2:
+            net.set_weights(i, to_dev(inp.Ws[i], True))
+        else:
+            net.set_weights(i, to_dev(inp.Ws[i], True), torch.from_numpy(inp.bs[i]).cuda())
+    J = torch.zeros(1, dtype=torch.float32, device="cuda")
+    net.forward(to_dev(inp.X, True), torch.from_numpy(inp.labels).cuda(), J)
+    acts = oracle_mixed_acts(o, w)
+    for i in range(w.L - 1):
+        assert rel_fro(to_np(net.get_tensor(mbd.T_ACT, i)), acts[i]) < TOL, i
+        net.set_tensor(mbd.T_ACT, i, to_dev(acts[i], True))
+    assert abs(float(J.item()) - o["J"]) < 1e-2 * abs(o["J"])
+    net.backward(0.0)
+    net.poll()
+    for i in range(w.L):
+        got = to_np(net.get_tensor(mbd.T_DW, i))
+        assert rel_fro(got, o["dWs"][i].reshape(got.shape)) < TOL, f"dW[{i}]"
+    net.close()
