@@ -402,3 +402,45 @@ def test_integrated_stack_with_convolutions_of_different_kinds():
         got = to_np(net.get_tensor(mbd.T_DW, i))
         assert rel_fro(got, o["dWs"][i].reshape(got.shape)) < TOL, f"dW[{i}]"
     net.close()
+
+
+@pytest.mark.parametrize("master,mu", [(True, None), (False, 0.9)])
+def test_masters_and_momentum_on_a_stack_of_different_kinds(master, mu):
+    # the update kernels run per run of layers: mbd_backward(eta) and mbd_backward(0) + mbd_sgd_step(eta) bit for bit,
+    # and the step itself against Eq. 1 / the heavy-ball form on the gradient the device materialised
+    import torch
+    from oracle import mbd_oracle as O
+    from paper_1712_04432_b200 import mbd
+    from tests.helpers import to_dev, to_np
+    ch, ks, H, W, B = (16, 128, 128), ((5, 5), (3, 3)), 8, 12, 4
+    w = I.conv_workload(ch[0], H, W, B, n_layers=2, name="kinds_update", ksizes=ks, channels=ch)
+    inp = I.make_inputs(w, seed=86)
+    X = to_dev(inp.X, True)
+    eta = 1e-3
+
+    def make():
+        net = mbd.Net(mbd.conv_layers(2, ch[0], H, W, k=list(ks), channels=ch, split=[mbd.SPLIT_DOMAIN, mbd.SPLIT_MODEL]), B, 2, 2, mbd.BF16,
+                      mbd.LOSS_HALF_SSQ, 2)
+        if master:
+            net.enable_master_weights()
+        for i in range(2):
+            net.set_weights(i, to_dev(inp.Ws[i], True))
+        if mu is not None:
+            net.enable_momentum(mu)
+        return net
+    a, b = make(), make()
+    for step in range(2):
+        W_old = [to_np(a.get_tensor(mbd.T_MASTER, i)) if master else to_np(a.get_weights(i)) for i in range(2)]
+        V_old = [to_np(a.get_tensor(mbd.T_VELOCITY, i)) if mu is not None else np.zeros_like(W_old[i]) for i in range(2)]
+        a.forward(X); a.backward(0.0)
+        dW = [to_np(a.get_tensor(mbd.T_DW, i)) for i in range(2)]
+        a.sgd_step(eta)
+        b.forward(X); b.backward(eta)
+        a.poll(); b.poll()
+        for i in range(2):
+            W_want, _ = O.sgd_momentum(W_old[i], V_old[i], dW[i], eta, B, mu if mu is not None else 0.0)
+            got = to_np(a.get_tensor(mbd.T_MASTER, i)) if master else to_np(a.get_weights(i))
+            assert rel_fro(got, W_want) < (1e-6 if master else 3e-3), (step, i)
+            assert torch.equal(a.get_weights(i), b.get_weights(i)), (step, i)
+            assert np.linalg.norm(dW[i]) > 0
+    a.close(); b.close()
