@@ -158,15 +158,16 @@ enum {
  * The convolutions of one network may be split in different ways, each layer in L_M or L_D on its own (Section 2.4):
  * between two runs of layers with different kinds the activation and, backward, its gradient change their
  * distribution (the re-distribution of Eq. 6; here a pass through the NCHW form).  Such a network runs on the
- * contraction kernel whatever its shapes; strips of unequal height and the row-range calls are then unsupported.
+ * contraction kernel whatever its shapes; the row-range calls are then unsupported.
  * Convolutions (kind MBD_CONV3X3 whatever the kernel size; Section 2.2): zero padding floor(k/2), k_h and
  * k_w odd and at most 11, stride 1 to 4 (the same in both directions), C_in and C_out multiples of 8, C_in of a layer =
  * C_out of the layer below, H x W of a layer = the output size of the layer below (H/s x W/s of its input);
  * weights [C_out][C_in][k_h][k_w] ([C_out][C_in] for 1x1).  A strip needs floor(k_h/2) halo rows
  * from each neighbour, which must be the adjacent strip's own rows: MBD_E_GRID when a strip is shorter than that.  The
  * stride-1 layers with 64 channels and 3x3 or 1x1 kernels run on kernels of their own; every other shape runs as
- * products of row-shifted views on the contraction kernel of the fully connected layers, and there strips of unequal
- * height, the interior / boundary calls and mbd_conv_outer_rows are MBD_E_UNSUPPORTED.
+ * products of row-shifted views on the contraction kernel of the fully connected layers; there the interior /
+ * boundary calls and mbd_conv_outer_rows are MBD_E_UNSUPPORTED, and so are strips of unequal height under a strided
+ * layer (H and H / s of a strided layer must be multiples of P_r).
  * MBD_E_UNSUPPORTED for other convolutions (even or larger kernels, other channel counts, larger strides),
  * a convolution above a fully connected layer, half-SSQ with
  * fully connected layers or softmax-CE without them, or bf16 FC dims that are not

@@ -55,9 +55,19 @@ __host__ __device__ inline StageTile stage_tile(int C) {
   t.G = 64 / t.cpb;
   return t;
 }
+// Strips of an image: the balanced ranges [floor(s H / P_r), floor((s + 1) H / P_r)) -- heights differ by at most one row;
+// every strip has Hs = ceil(H / P_r) row slots, and a shorter strip's last slot is a dead row (zero, like the padding).
+__host__ __device__ __forceinline__ bool geo_ragged(const Geo& g) { return g.Hs * g.P_r != g.H; }
+__host__ __device__ __forceinline__ int geo_first(const Geo& g, int s) {
+  return !geo_ragged(g) ? s * g.Hs : static_cast<int>((static_cast<long long>(s) * g.H) / g.P_r);
+}
+__host__ __device__ __forceinline__ int geo_height(const Geo& g, int s) { return !geo_ragged(g) ? g.Hs : geo_first(g, s + 1) - geo_first(g, s); }
+__host__ __device__ __forceinline__ int geo_strip_of(const Geo& g, int h) {
+  return !geo_ragged(g) ? h / g.Hs : static_cast<int>(((static_cast<long long>(h) + 1) * g.P_r - 1) / g.H);
+}
 __device__ __forceinline__ long long pix_index(const Geo& g, int b, int q) {     // pixel q = h * W + w of image b in the padded layout
   const int h = q / g.W, w = q - h * g.W;
-  const int s = h / g.Hs, r = h - s * g.Hs + g.ph;
+  const int s = geo_strip_of(g, h), r = h - geo_first(g, s) + g.ph;
   return ((static_cast<long long>(b) * g.P_r + s) * g.R + r) * g.Wp + w + g.pw;
 }
 
@@ -175,37 +185,42 @@ pix_to_nchw_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst, Geo g, 
 // Everything that is not a strip's own pixel: the padding columns and the image's outer rows become zero; a halo
 // row becomes the copy of the neighbouring strip's boundary row (fill_halos) -- the halo exchange of Section 2.2:
 // floor(k_h/2) rows per neighbour and direction -- or zero (a gradient about to enter the weight-gradient sum, whose
-// pixels must each be counted once).  One thread per 16 bytes of padding: per strip 2 ph whole rows, then the 2 pw
-// side columns of its Hs own rows.
+// pixels must each be counted once); the dead row of a strip that is one row shorter than the slots becomes zero.
+// One thread per 16 bytes of padding: per strip the 2 ph halo rows (and one more row slot when heights differ), then
+// the 2 pw side columns of its own rows.
 __global__ void __launch_bounds__(256)
 pad_fix_kernel(bf16* __restrict__ T, Geo g, int C, int fill_halos) {
   const int c8 = C / 8;
-  const int n_rows = 2 * g.ph * g.Wp * c8;             // chunks in the halo rows of a strip
+  const int extra = geo_ragged(g) ? 1 : 0;
+  const int n_rows = (2 * g.ph + extra) * g.Wp * c8;   // chunks in the rows of a strip that are not its own
   const int n_side = g.Hs * 2 * g.pw * c8;             // chunks in the side columns of its own rows
   const int per_strip = n_rows + n_side;
   const long long total = g.Z * per_strip;
   for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
     const long long z = i / per_strip;
     int k = static_cast<int>(i - z * per_strip);
+    const int s = static_cast<int>(z % g.P_r);
+    const int hs = geo_height(g, s);                   // this strip's own rows: ph .. ph + hs - 1
     int r, x, cg;
     if (k < n_rows) {
       cg = k % c8; k /= c8;
-      x = k % g.Wp; k /= g.Wp;                         // k: 0 .. 2 ph - 1
-      r = k < g.ph ? k : k + g.Hs;
+      x = k % g.Wp; k /= g.Wp;                         // k: 0 .. 2 ph - 1 (+ 1)
+      r = k < g.ph ? k : k + hs;
+      if (r >= g.R) continue;                          // (a strip of full height has no dead row)
     } else {
       k -= n_rows;
       cg = k % c8; k /= c8;
-      const int side = k % (2 * g.pw); k /= 2 * g.pw;  // k: own row 0 .. Hs - 1
+      const int side = k % (2 * g.pw); k /= 2 * g.pw;  // k: row slot 0 .. Hs - 1
+      if (k >= hs) continue;                           // (the dead row was zeroed as a whole)
       x = side < g.pw ? side : side + g.W;
       r = k + g.ph;
     }
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (fill_halos && x >= g.pw && x < g.pw + g.W && (r < g.ph || r >= g.ph + g.Hs)) {
-      const int s = static_cast<int>(z % g.P_r);
-      if (r < g.ph && s > 0)                        // rows above the strip: the last rows of the strip above
-        v = *reinterpret_cast<const uint4*>(T + ((((z - 1) * g.R) + r + g.Hs) * g.Wp + x) * C + cg * 8);
-      else if (r >= g.ph + g.Hs && s < g.P_r - 1)   // rows below it: the first rows of the strip below
-        v = *reinterpret_cast<const uint4*>(T + ((((z + 1) * g.R) + r - g.Hs) * g.Wp + x) * C + cg * 8);
+    if (fill_halos && x >= g.pw && x < g.pw + g.W) {
+      if (r < g.ph && s > 0)                                        // rows above the strip: the last rows of the strip above
+        v = *reinterpret_cast<const uint4*>(T + ((((z - 1) * g.R) + r + geo_height(g, s - 1)) * g.Wp + x) * C + cg * 8);
+      else if (r >= g.ph + hs && r < 2 * g.ph + hs && s < g.P_r - 1)   // rows below it: the first rows of the strip below
+        v = *reinterpret_cast<const uint4*>(T + ((((z + 1) * g.R) + r - hs) * g.Wp + x) * C + cg * 8);
     }
     *reinterpret_cast<uint4*>(T + ((z * g.R + r) * g.Wp + x) * C + cg * 8) = v;
   }
@@ -365,7 +380,7 @@ mbd_status run(GenConv* c, TcGemm& t, int cls, double flops, const Epi& epi) {
 void pad_fix(GenConv* c, bf16* T, Geo g, int C, bool fill_halos, int planes = 1) {
   g.Z *= planes;
   g.Ptot *= planes;
-  const long long chunks = g.Z * (2ll * g.ph * g.Wp + 2ll * g.Hs * g.pw) * (C / 8);
+  const long long chunks = g.Z * ((2ll * g.ph + (geo_ragged(g) ? 1 : 0)) * g.Wp + 2ll * g.Hs * g.pw) * (C / 8);
   c->prof->begin(MBD_K_HALO, static_cast<double>(chunks) * 16.0, c->stream);
   if (chunks > 0) pad_fix_kernel<<<grid_1d(chunks, c->num_sms), 256, 0, c->stream>>>(T, g, C, fill_halos ? 1 : 0);
   c->prof->end();
@@ -460,7 +475,7 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
     if (l.C_in < 8 || l.C_out < 8 || l.C_in % 8 || l.C_out % 8) return MBD_E_UNSUPPORTED;       // 16-byte rows for TMA
     if (i > 0 && l.C_in != layers[i - 1].C_out) return MBD_E_INVALID;
     if (l.H != H || l.W != W || H % s || W % s) return MBD_E_INVALID;                            // sizes chain through the strides
-    if (H % P_r != 0 || (H / s) % P_r != 0) return MBD_E_UNSUPPORTED;                            // strips of equal height on this path
+    if ((H % P_r != 0 || (H / s) % P_r != 0) && s > 1) return MBD_E_UNSUPPORTED;                 // a strided layer's phase planes need strips of equal height
     ph = std::max(ph, (l.kh / 2 + s - 1) / s); pw = std::max(pw, (l.kw / 2 + s - 1) / s);
     H /= s; W /= s;
   }
@@ -471,9 +486,9 @@ mbd_status gconv_create(const mbd_layer* layers, int L, int64_t B, int P_r, int 
   H = layers[0].H; W = layers[0].W;
   for (int t = 0; t <= L; ++t) {
     Geo& g = c->geo[t];
-    g.B = static_cast<int>(B); g.H = H; g.W = W; g.P_r = P_r; g.Hs = H / P_r; g.ph = ph; g.pw = pw;
+    g.B = static_cast<int>(B); g.H = H; g.W = W; g.P_r = P_r; g.Hs = (H + P_r - 1) / P_r; g.ph = ph; g.pw = pw;      // row slots: the tallest strip
     g.R = g.Hs + 2 * ph; g.Wp = W + 2 * pw; g.Z = B * P_r; g.Ptot = g.Z * g.R * g.Wp;
-    if (P_r > 1 && g.Hs < ph) { delete c; return MBD_E_GRID; }             // a halo row must come from the adjacent strip
+    if (P_r > 1 && H / P_r < ph) { delete c; return MBD_E_GRID; }          // a halo row must come from the adjacent strip (the shortest one too)
     const int s = t < L && layers[t].stride > 1 ? layers[t].stride : 1;
     if (B > INT32_MAX / std::max(1, P_r) || g.Ptot * s * s > INT32_MAX - 512) { delete c; return MBD_E_UNSUPPORTED; }   // TMA coordinates are 32-bit
     if (t < L) { H /= s; W /= s; }

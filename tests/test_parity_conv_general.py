@@ -40,8 +40,6 @@ def case(request):
 def test_general_layers_on_strips_and_batch_blocks(case, P_r, P_c, mp, fused):
     w, inp, o, eta = case
     H = w.dims[1]
-    if H % P_r:
-        pytest.skip("strips of equal height on this path")
     if P_c > w.B:
         pytest.skip("more batch blocks than samples")
     if P_r > 1 and H // P_r < max(w.kshape(i)[0] // 2 for i in range(w.n_layers)):
@@ -57,6 +55,23 @@ def test_strip_formulation_of_the_oracle_agrees():
     ob = oracle_conv_step(w, inp, grid=(3, 2))             # strips with two halo rows, partials per process
     g = gpu_conv_step(w, inp, 3, P_c=2, force_acts=stored_hidden(ob))
     compare_conv_step(g, ob, TOL)
+
+
+@pytest.mark.parametrize("name,grid", [("channel_blocks_of_64", (3, 2)), ("five_by_five_then_three", (5, 1)), ("three_layers_7x7_first", (4, 2))])
+def test_strips_of_unequal_height_on_the_general_path(name, grid):
+    # H mod P_r != 0: the balanced ranges of rows (16 rows on 3 strips: 5, 5, 6; 12 on 5: 2, 2, 2, 3, 3; 18 on 4: 4, 5, 4, 5);
+    # every strip has ceil(H / P_r) row slots, the last slot of a shorter strip is a dead row that stays zero, and a
+    # strip's lower halo rows follow its last OWN row.  Against the oracle's strip formulation on the same ranges.
+    ch, ks, H, W, B = CASES[name]
+    assert H % grid[0] != 0
+    w = I.conv_workload(ch[0], H, W, B, n_layers=len(ks), name="ragged_" + name, ksizes=ks, channels=ch)
+    inp = I.make_inputs(w, seed=64)
+    ob = oracle_conv_step(w, inp, grid=grid)
+    eta = update_sized_eta(ob, inp.Ws, w.B)
+    ob = oracle_conv_step(w, inp, grid=grid, eta=eta)
+    for fused in (False, True):
+        g = gpu_conv_step(w, inp, grid[0], fused=fused, P_c=grid[1], force_acts=stored_hidden(ob), eta=eta, max_partials=2)
+        compare_conv_step(g, ob, TOL, fused, init=inp, require_sized=True)
 
 
 def test_listed_64_channel_layers_through_the_general_path(monkeypatch):
@@ -277,9 +292,9 @@ def test_unsupported_shapes_are_refused():
     with pytest.raises(mbd.MbdError) as e:
         mbd.Net(mbd.conv_layers(1, 8, 12, 12, k=7), 2, 6, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
     assert e.value.status == mbd.E_GRID
-    # strips of unequal height exist only for the 64-channel layers
+    # strips of unequal height: not under a strided layer (its phase planes are cut per strip)
     with pytest.raises(mbd.MbdError) as e:
-        mbd.Net(mbd.conv_layers(1, 8, 13, 12, k=5), 2, 2, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
+        mbd.Net(mbd.conv_layers(1, 8, 20, 12, k=5, strides=(2,)), 2, 3, 1, mbd.BF16, mbd.LOSS_HALF_SSQ, 0)
     assert e.value.status == mbd.E_UNSUPPORTED
 
 
