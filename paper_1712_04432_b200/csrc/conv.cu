@@ -80,7 +80,6 @@ enum { MODE_RELU_STORE = 0, MODE_STORE_SSQ = 1, MODE_MASK = 2 };
 // backward-weight product) the all-zero row Hs + 1 is read in its place.
 __host__ __device__ __forceinline__ int strip_first(int s, int H, int P) { return static_cast<int>((static_cast<long long>(s) * H) / P); }
 __host__ __device__ __forceinline__ int strip_height(int s, int H, int P) { return strip_first(s + 1, H, P) - strip_first(s, H, P); }
-__host__ __device__ __forceinline__ int strip_of_row(int h, int H, int P) { return static_cast<int>(((static_cast<long long>(h) + 1) * P - 1) / H); }
 // The same inside the kernels, where they sit on the epilogue's critical path: strips of equal height (H = Hs P, the
 // common case) need no division by P at all, the others one in 32 bits (H P < 2^31 is checked when the network is made).
 __device__ __forceinline__ bool strips_uneven(int H, int P, int Hs) { return Hs * P != H; }

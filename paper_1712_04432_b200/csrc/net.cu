@@ -578,7 +578,6 @@ extern "C" mbd_status mbd_forward(mbd_net* n, const void* X_dev, const int32_t* 
   const int bf = n->dtype == MBD_BF16;
   for (int i = 0; i < n->L; ++i) {
     Layer& l = n->layers[i];
-    const bool last = i == n->L - 1;
     const Epi e = fwd_epi(n, i);
     s = run_gemm(n, l.fwd, 0, n->B, l.d_out, l.d_in, layer_input(n, i), l.d_in, l.W, l.d_in, 1, e);
     if (s != MBD_OK) return s;
