@@ -459,3 +459,31 @@ def test_masters_and_momentum_on_a_stack_of_different_kinds(master, mu):
             assert torch.equal(a.get_weights(i), b.get_weights(i)), (step, i)
             assert np.linalg.norm(dW[i]) > 0
     a.close(); b.close()
+
+
+def test_graph_replay_of_a_stack_of_different_kinds_equals_direct_launches():
+    # mbd_train_step captures the step once and replays it: runs of layers, re-distributions and all
+    import torch
+    from paper_1712_04432_b200 import mbd
+    from tests.helpers import to_dev
+    ch, ks, H, W, B = (16, 128, 128, 128), ((5, 5), (3, 3), (1, 1)), 8, 12, 4
+    w = I.conv_workload(ch[0], H, W, B, n_layers=3, name="kinds_graph", ksizes=ks, channels=ch)
+    inp = I.make_inputs(w, seed=87)
+    X = to_dev(inp.X, True)
+
+    def make():
+        net = mbd.Net(mbd.conv_layers(3, ch[0], H, W, k=list(ks), channels=ch, split=[mbd.SPLIT_DOMAIN, mbd.SPLIT_MODEL, mbd.SPLIT_BATCH]), B, 2, 2,
+                      mbd.BF16, mbd.LOSS_HALF_SSQ, 2)
+        for i in range(3):
+            net.set_weights(i, to_dev(inp.Ws[i], True))
+        return net
+    a, b = make(), make()
+    Ja, Jb = torch.zeros(1, device="cuda"), torch.zeros(1, device="cuda")
+    for step in range(3):
+        a.train_step(X, None, 1e-4, Ja)
+        b.forward(X, None, Jb); b.backward(1e-4)
+        a.poll(); b.poll()
+        assert float(Ja.item()) == float(Jb.item()) and float(Ja.item()) > 0, step
+        for i in range(3):
+            assert torch.equal(a.get_weights(i), b.get_weights(i)), (step, i)
+    a.close(); b.close()
